@@ -1,0 +1,407 @@
+"""CPU oracle for one ReDrafter speculative decode step.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain reference that the CUDA
+library is compared against.  It shares no code with the CUDA path and must never
+be imported by the product package; only tests, the smoke check and the benchmark's
+CPU-baseline leg use it.
+
+Everything is numpy, float64 by default, one sequence at a time (a batch is a
+Python loop over independent sequences, Appendix A.1: the batch is only a leading
+dimension).  The steps follow the paper's order (Section 3.4):
+
+    draft (Sections 3.1, 3.2)  ->  dedup_prefix / pack_beam (Section 3.3, Appendix A.1)
+    ->  LLM verification forward (Section 3.4)  ->  greedy acceptance (Section 3.4)
+
+The paper is silent on several points (activation, head depth, the LLM's
+architecture, KV cache handling, tie breaking).  The readings used here:
+
+  * f = SiLU; the head is `n_head_layers` residual layers x <- x + SiLU(A x + c) of
+    width 2d followed by a bias-free projection to the vocabulary and a softmax.
+  * s_1 := e_1 is the embedding of the token the LLM just produced (Section 3.1);
+    the first drafter call applies the head to [s_1, h] directly, later calls
+    first update s_t = f(U s_{t-1} + W e_t + b) with e_t the embedding of the token
+    drafted by the previous call.
+  * Beam length L = number of drafter calls = drafted tokens per candidate
+    (Appendix A.2.1); the guaranteed root token is extra.
+  * The LLM is Llama-style: pre-norm RMSNorm, rotary embedding with the half-split
+    pairing (i, i + hd/2), multi-head attention with scale hd^-1/2, SwiGLU, no biases.
+  * Candidates are ordered by (score descending, flat index ascending); argmax ties
+    go to the lowest index; equal accepted lengths go to the lowest beam index.
+  * The dedup listing in Appendix A.1 is read through its comment and its printed
+    example: compare candidate i with candidate j position by position, a prefix of
+    length j+1 is shared when all of its j+1 positions match, and the FIRST such
+    candidate is reported.
+
+Parity pins (tests/test_oracle_*.py): the printed dedup example, brute-force
+prefix sets, packed-tree == per-beam causal verification, speculative == plain
+greedy decoding, beam width 1 == greedy drafting, exhaustive beam search on a tiny
+vocabulary, closed forms for the RNN cell and the head, library cross-checks.
+Parity unpinned: nothing in the paper prints a weights-to-beams example, so the
+drafter's exact beams are pinned by properties only.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+F = np.float64
+
+
+# ----------------------------------------------------------------------------
+# elementary functions
+# ----------------------------------------------------------------------------
+def silu(x):
+    return x / (1.0 + np.exp(-x))
+
+
+def log_softmax(z):
+    """Natural-log softmax of a vector (Section 3.1: standard softmax layer)."""
+    m = np.max(z)
+    return z - (m + np.log(np.sum(np.exp(z - m))))
+
+
+def rmsnorm(x, gain, eps):
+    """x: [rows, d].  y = x / sqrt(mean(x^2) + eps) * gain."""
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x / np.sqrt(ms + eps) * gain
+
+
+def rope(x, pos, theta):
+    """Rotary embedding, half-split pairing.  x: [rows, heads, hd]; pos: [rows]."""
+    hd = x.shape[-1]
+    half = hd // 2
+    inv_freq = theta ** (-(np.arange(half, dtype=F) * 2.0) / hd)
+    ang = np.asarray(pos, dtype=F)[:, None] * inv_freq[None, :]          # [rows, half]
+    c = np.cos(ang)[:, None, :]
+    s = np.sin(ang)[:, None, :]
+    x1 = x[..., :half]
+    x2 = x[..., half:]
+    return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
+
+
+def argmax_first(v):
+    """Index of the maximum; the lowest index on ties."""
+    return int(np.argmax(v))
+
+
+def top_k_ordered(values, k):
+    """Indices of the k largest values ordered by (value desc, index asc)."""
+    order = np.lexsort((np.arange(values.shape[0]), -values))
+    return order[:k]
+
+
+# ----------------------------------------------------------------------------
+# target LLM (verification forward, Section 3.4)
+# ----------------------------------------------------------------------------
+class KVCache:
+    """Per-sequence cache: k, v of shape [n_layers, max_ctx, n_heads, hd]."""
+
+    def __init__(self, n_layers, max_ctx, n_heads, hd, dtype=F):
+        self.k = np.zeros((n_layers, max_ctx, n_heads, hd), dtype=dtype)
+        self.v = np.zeros((n_layers, max_ctx, n_heads, hd), dtype=dtype)
+
+
+def llm_forward(W, cfg, tokens, pos, mask, kv, ctx, dtype=F, want_logits=True):
+    """Forward over `tokens` (rows) with explicit positions and mask.
+
+    Row n attends cache slots [0, ctx) and the rows m with mask[n, m] True (self
+    included); its key/value are written provisionally to slot ctx + n.
+    Returns (hidden [rows, d] after the final norm, logits [rows, V] or None).
+    """
+    H = cfg["n_heads"]
+    d = cfg["d_model"]
+    hd = d // H
+    eps = cfg["rms_eps"]
+    theta = cfg["rope_theta"]
+    tokens = np.asarray(tokens)
+    n = tokens.shape[0]
+    assert ctx + n <= kv.k.shape[1], "KV cache capacity exceeded"
+    mask = np.asarray(mask, dtype=bool)
+    x = W["tok_emb"][tokens].astype(dtype)
+    scale = 1.0 / np.sqrt(hd)
+    for l in range(cfg["n_layers"]):
+        a = rmsnorm(x, W["attn_norm"][l].astype(dtype), eps)
+        qkv = a @ W["wqkv"][l].astype(dtype).T                          # [n, 3d]
+        q = rope(qkv[:, :d].reshape(n, H, hd), pos, theta)
+        k = rope(qkv[:, d:2 * d].reshape(n, H, hd), pos, theta)
+        v = qkv[:, 2 * d:].reshape(n, H, hd)
+        kv.k[l, ctx:ctx + n] = k
+        kv.v[l, ctx:ctx + n] = v
+        attn = np.zeros((n, H, hd), dtype=dtype)
+        for r in range(n):
+            slots = np.concatenate([np.arange(ctx), ctx + np.nonzero(mask[r])[0]])
+            kk = kv.k[l, slots].astype(dtype)                           # [keys, H, hd]
+            vv = kv.v[l, slots].astype(dtype)
+            sc = np.einsum("hd,khd->hk", q[r], kk) * scale              # [H, keys]
+            sc = sc - sc.max(axis=1, keepdims=True)
+            p = np.exp(sc)
+            p = p / p.sum(axis=1, keepdims=True)
+            attn[r] = np.einsum("hk,khd->hd", p, vv)
+        x = x + attn.reshape(n, d) @ W["wo"][l].astype(dtype).T
+        f = rmsnorm(x, W["ffn_norm"][l].astype(dtype), eps)
+        gu = f @ W["w_gate_up"][l].astype(dtype).T                      # [n, 2F]: gate rows then up rows
+        Fd = cfg["d_ffn"]
+        act = silu(gu[:, :Fd]) * gu[:, Fd:]
+        x = x + act @ W["w_down"][l].astype(dtype).T
+    hidden = rmsnorm(x, W["final_norm"].astype(dtype), eps)
+    logits = hidden @ W["lm_head"].astype(dtype).T if want_logits else None
+    return hidden, logits
+
+
+def prefill(W, cfg, prompt, kv, dtype=F):
+    """Causal forward over the prompt.  Returns (ctx, root token g, h)."""
+    P = len(prompt)
+    mask = np.tril(np.ones((P, P), dtype=bool))
+    hidden, _ = llm_forward(W, cfg, prompt, np.arange(P), mask, kv, 0, dtype, want_logits=False)
+    logits_last = hidden[P - 1] @ W["lm_head"].astype(dtype).T
+    return P, argmax_first(logits_last), hidden[P - 1].copy()
+
+
+def ar_step(W, cfg, kv, ctx, g, dtype=F):
+    """One plain autoregressive step: feed g at position ctx, return next token, h, logits."""
+    hidden, logits = llm_forward(W, cfg, [g], [ctx], np.ones((1, 1), bool), kv, ctx, dtype)
+    return argmax_first(logits[0]), hidden[0].copy(), logits[0]
+
+
+# ----------------------------------------------------------------------------
+# drafter (Sections 3.1 and 3.2)
+# ----------------------------------------------------------------------------
+def rnn_cell(D, s_prev, e, dtype=F):
+    """s_t = f(U s_{t-1} + W e_t + b) (Section 3.1)."""
+    return silu(D["rnn_u"].astype(dtype) @ s_prev + D["rnn_w"].astype(dtype) @ e + D["rnn_b"].astype(dtype))
+
+
+def draft_head(D, g_t, dtype=F):
+    """MLP layers with skip connections, then the vocabulary projection (Section 3.1).  Returns logits."""
+    x = g_t
+    for A, c in zip(D["head_w"], D["head_b"]):
+        x = x + silu(A.astype(dtype) @ x + c.astype(dtype))
+    return D["draft_out"].astype(dtype) @ x
+
+
+def beam_search(D, E, g, h, beam_width, beam_length, dtype=F, return_logp=False):
+    """Beam search over the drafter (Section 3.2).
+
+    Returns beams [BW, L] (int64), scores [BW]: candidates sorted by cumulative
+    log-probability, descending.  With return_logp also the per-call candidate
+    arrays (for gap-gated comparisons).
+    """
+    V = D["draft_out"].shape[0]
+    assert beam_width <= V
+    E = E.astype(dtype) if E.dtype != dtype else E
+    h = np.asarray(h, dtype=dtype)
+    s1 = E[g]
+    logp = log_softmax(draft_head(D, np.concatenate([s1, h]), dtype))
+    top = top_k_ordered(logp, beam_width)
+    hist = [[int(v)] for v in top]
+    scores = logp[top].copy()
+    states = [s1.copy() for _ in range(beam_width)]
+    cand_log = [logp.copy()]
+    for _t in range(2, beam_length + 1):
+        cand = np.empty(beam_width * V, dtype=dtype)
+        new_states = []
+        for b in range(beam_width):
+            s = rnn_cell(D, states[b], E[hist[b][-1]], dtype)
+            new_states.append(s)
+            lp = log_softmax(draft_head(D, np.concatenate([s, h]), dtype))
+            cand[b * V:(b + 1) * V] = scores[b] + lp
+        top = top_k_ordered(cand, beam_width)
+        cand_log.append(cand)
+        hist = [hist[int(c) // V] + [int(c) % V] for c in top]
+        states = [new_states[int(c) // V] for c in top]
+        scores = cand[top].copy()
+    beams = np.array(hist, dtype=np.int64).reshape(beam_width, beam_length)
+    if return_logp:
+        return beams, scores, cand_log
+    return beams, scores
+
+
+def sequence_logprob(D, E, g, h, seq, dtype=F):
+    """log p_draft(seq | g, h): the drafter run along one fixed sequence."""
+    E = E.astype(dtype)
+    s = E[g]
+    total = 0.0
+    for t, tok in enumerate(seq):
+        if t > 0:
+            s = rnn_cell(D, s, E[seq[t - 1]], dtype)
+        lp = log_softmax(draft_head(D, np.concatenate([s, np.asarray(h, dtype=dtype)]), dtype))
+        total += lp[tok]
+    return total
+
+
+# ----------------------------------------------------------------------------
+# dynamic tree attention (Section 3.3, Appendix A.1)
+# ----------------------------------------------------------------------------
+def dedup_prefix(beam):
+    """prefix_tree[i][j] = smallest k with beam[k][:j+1] == beam[i][:j+1]."""
+    # The definition written out (Appendix A.1, first paragraph): for every candidate
+    # i and prefix length j+1, scan the candidates in index order and report the
+    # first one whose leading j+1 tokens are the same.
+    beam = np.asarray(beam)
+    bw, bl = beam.shape
+    prefix_tree = np.zeros((bw, bl), dtype=np.int64)
+    for i in range(bw):
+        for j in range(bl):
+            for k in range(bw):
+                if all(beam[k][c] == beam[i][c] for c in range(j + 1)):
+                    prefix_tree[i, j] = k
+                    break
+    return prefix_tree
+
+
+def pack_beam(beam_aug, ctx):
+    """Compress the augmented beam [root | drafts] ([BW, L+1]) into the packed beam.
+
+    Token (i, j) is kept iff prefix_tree[i][j] == i (Appendix A.1: tokens with
+    prefix_tree[i][j] < i can be condensed); kept tokens are numbered in row-major
+    order.  Returns a dict with
+      tokens[N], n, unpack[BW, L+1], pos[N] = ctx + depth, depth[N], parent[N]
+      (-1 for the root), mask[N, N] (row n sees its ancestors and itself).
+    """
+    beam_aug = np.asarray(beam_aug)
+    bw, cols = beam_aug.shape
+    assert np.all(beam_aug[:, 0] == beam_aug[0, 0]), "column 0 is the shared root"
+    pt = dedup_prefix(beam_aug)
+    keep = pt == np.arange(bw)[:, None]
+    index = np.cumsum(keep.reshape(-1)).reshape(bw, cols) - 1            # inclusive scan - 1 on kept
+    n = int(keep.sum())
+    tokens = np.zeros(n, dtype=np.int64)
+    depth = np.zeros(n, dtype=np.int64)
+    unpack = np.zeros((bw, cols), dtype=np.int64)
+    for i in range(bw):
+        for j in range(cols):
+            unpack[i, j] = index[pt[i, j], j]
+            if keep[i, j]:
+                tokens[index[i, j]] = beam_aug[i, j]
+                depth[index[i, j]] = j
+    parent = np.full(n, -1, dtype=np.int64)
+    mask = np.zeros((n, n), dtype=bool)
+    for i in range(bw):
+        for j in range(cols):
+            r = unpack[i, j]
+            if j > 0:
+                parent[r] = unpack[i, j - 1]
+            mask[r, unpack[i, :j + 1]] = True
+    return dict(tokens=tokens, n=n, unpack=unpack, pos=ctx + depth, depth=depth,
+                parent=parent, mask=mask, prefix_tree=pt)
+
+
+def flat_beam(beam_aug, ctx):
+    """The no-tree-attention arm (Figure 3(a)): every candidate keeps all its tokens
+    except the shared root, which is sent once.  Same output dict as pack_beam."""
+    beam_aug = np.asarray(beam_aug)
+    bw, cols = beam_aug.shape
+    n = 1 + bw * (cols - 1)
+    tokens = np.zeros(n, dtype=np.int64)
+    depth = np.zeros(n, dtype=np.int64)
+    unpack = np.zeros((bw, cols), dtype=np.int64)
+    tokens[0] = beam_aug[0, 0]
+    for i in range(bw):
+        for j in range(1, cols):
+            r = 1 + i * (cols - 1) + (j - 1)
+            unpack[i, j] = r
+            tokens[r] = beam_aug[i, j]
+            depth[r] = j
+    parent = np.full(n, -1, dtype=np.int64)
+    mask = np.zeros((n, n), dtype=bool)
+    for i in range(bw):
+        for j in range(cols):
+            r = unpack[i, j]
+            if j > 0:
+                parent[r] = unpack[i, j - 1]
+            mask[r, unpack[i, :j + 1]] = True
+    return dict(tokens=tokens, n=n, unpack=unpack, pos=ctx + depth, depth=depth,
+                parent=parent, mask=mask)
+
+
+# ----------------------------------------------------------------------------
+# greedy acceptance + KV compaction (Section 3.4)
+# ----------------------------------------------------------------------------
+def accept_greedy(beams, unpack, llm_argmax):
+    """Longest prefix of a candidate whose tokens equal the LLM's greedy tokens.
+
+    beams [BW, L]; unpack [BW, L+1] (column 0 = root); llm_argmax[N] = the LLM's
+    greedy next token after each packed node.  Returns (a, best, emitted) where
+    emitted = accepted draft tokens followed by the bonus token.
+    """
+    beams = np.asarray(beams)
+    bw, L = beams.shape
+    best, a = 0, -1
+    for i in range(bw):
+        ai = 0
+        while ai < L and beams[i, ai] == llm_argmax[unpack[i, ai]]:
+            ai += 1
+        if ai > a:
+            a, best = ai, i
+    bonus = int(llm_argmax[unpack[best, a]])
+    emitted = [int(t) for t in beams[best, :a]] + [bonus]
+    return a, best, emitted
+
+
+def compact_kv(kv, ctx, unpack, best, a):
+    """Move the accepted path's provisional K/V rows to slots ctx+1 .. ctx+a."""
+    for j in range(1, a + 1):
+        src = ctx + int(unpack[best, j])
+        dst = ctx + j
+        if src != dst:
+            kv.k[:, dst] = kv.k[:, src]
+            kv.v[:, dst] = kv.v[:, src]
+    return ctx + 1 + a
+
+
+# ----------------------------------------------------------------------------
+# the whole step (Section 3.4) for one sequence
+# ----------------------------------------------------------------------------
+def spec_step(W, D, cfg, kv, ctx, g, h, beam_width, beam_length, planted=None,
+              tree=True, dtype=F, run_drafter=True):
+    """One speculative decode step.  Returns a dict with every intermediate.
+
+    planted: optional [BW, L] beams used in place of the drafter's (the drafter
+    still runs when run_drafter is True, as in the timed planted-beam mode).
+    """
+    out = {}
+    if run_drafter or planted is None:
+        beams, scores = beam_search(D, W["tok_emb"], g, h, beam_width, beam_length, dtype)
+        out["drafted_beams"], out["scores"] = beams, scores
+    if planted is not None:
+        beams = np.asarray(planted, dtype=np.int64)
+    beam_aug = np.concatenate([np.full((beams.shape[0], 1), g, dtype=np.int64), beams], axis=1)
+    packed = pack_beam(beam_aug, ctx) if tree else flat_beam(beam_aug, ctx)
+    hidden, logits = llm_forward(W, cfg, packed["tokens"], packed["pos"], packed["mask"], kv, ctx, dtype)
+    am = np.argmax(logits, axis=1)
+    a, best, emitted = accept_greedy(beams, packed["unpack"], am)
+    node = int(packed["unpack"][best, a])
+    new_ctx = compact_kv(kv, ctx, packed["unpack"], best, a)
+    out.update(beams=beams, packed=packed, hidden=hidden, logits=logits, argmax=am,
+               n_accept=a, best=best, emitted=emitted, ctx=new_ctx, g=emitted[-1],
+               h=hidden[node].copy())
+    return out
+
+
+def generate_ar(W, cfg, prompt, n_tokens, max_ctx, dtype=F):
+    """Plain greedy decoding: the definition the speculative path must reproduce."""
+    kv = KVCache(cfg["n_layers"], max_ctx, cfg["n_heads"], cfg["d_model"] // cfg["n_heads"], dtype)
+    ctx, g, h = prefill(W, cfg, prompt, kv, dtype)
+    out = [g]
+    while len(out) < n_tokens:
+        nxt, h, _ = ar_step(W, cfg, kv, ctx, g, dtype)
+        ctx += 1
+        g = nxt
+        out.append(g)
+    return out, kv, ctx
+
+
+def generate_spec(W, D, cfg, prompt, n_steps, beam_width, beam_length, max_ctx,
+                  planted_fn=None, tree=True, dtype=F):
+    """Speculative decoding for n_steps.  planted_fn(step, ctx, g) -> beams or None."""
+    kv = KVCache(cfg["n_layers"], max_ctx, cfg["n_heads"], cfg["d_model"] // cfg["n_heads"], dtype)
+    ctx, g, h = prefill(W, cfg, prompt, kv, dtype)
+    out = [g]
+    accepted = []
+    for step in range(n_steps):
+        planted = planted_fn(step, len(out), g) if planted_fn is not None else None
+        r = spec_step(W, D, cfg, kv, ctx, g, h, beam_width, beam_length, planted, tree, dtype,
+                      run_drafter=planted is None)
+        ctx, g, h = r["ctx"], r["g"], r["h"]
+        out.extend(r["emitted"])
+        accepted.append(r["n_accept"])
+    return out, accepted, kv, ctx
