@@ -49,6 +49,18 @@ F = np.float64
 # ----------------------------------------------------------------------------
 # elementary functions
 # ----------------------------------------------------------------------------
+def _c(a, dtype):
+    """The array in the working precision (no copy when it already is)."""
+    return np.asarray(a, dtype=dtype)
+
+
+def convert_weights(W, D, dtype):
+    """Copies of the weight dicts in the working precision, so later calls do not convert again."""
+    def conv(v):
+        return [_c(t, dtype) for t in v] if isinstance(v, list) else _c(v, dtype)
+    return {k: conv(v) for k, v in W.items()}, {k: conv(v) for k, v in D.items()}
+
+
 def silu(x):
     return x / (1.0 + np.exp(-x))
 
@@ -116,11 +128,11 @@ def llm_forward(W, cfg, tokens, pos, mask, kv, ctx, dtype=F, want_logits=True):
     n = tokens.shape[0]
     assert ctx + n <= kv.k.shape[1], "KV cache capacity exceeded"
     mask = np.asarray(mask, dtype=bool)
-    x = W["tok_emb"][tokens].astype(dtype)
+    x = np.asarray(W["tok_emb"][tokens], dtype=dtype)
     scale = 1.0 / np.sqrt(hd)
     for l in range(cfg["n_layers"]):
-        a = rmsnorm(x, W["attn_norm"][l].astype(dtype), eps)
-        qkv = a @ W["wqkv"][l].astype(dtype).T                          # [n, 3d]
+        a = rmsnorm(x, _c(W["attn_norm"][l], dtype), eps)
+        qkv = a @ _c(W["wqkv"][l], dtype).T                          # [n, 3d]
         q = rope(qkv[:, :d].reshape(n, H, hd), pos, theta)
         k = rope(qkv[:, d:2 * d].reshape(n, H, hd), pos, theta)
         v = qkv[:, 2 * d:].reshape(n, H, hd)
@@ -136,14 +148,14 @@ def llm_forward(W, cfg, tokens, pos, mask, kv, ctx, dtype=F, want_logits=True):
             p = np.exp(sc)
             p = p / p.sum(axis=1, keepdims=True)
             attn[r] = np.einsum("hk,khd->hd", p, vv)
-        x = x + attn.reshape(n, d) @ W["wo"][l].astype(dtype).T
-        f = rmsnorm(x, W["ffn_norm"][l].astype(dtype), eps)
-        gu = f @ W["w_gate_up"][l].astype(dtype).T                      # [n, 2F]: gate rows then up rows
+        x = x + attn.reshape(n, d) @ _c(W["wo"][l], dtype).T
+        f = rmsnorm(x, _c(W["ffn_norm"][l], dtype), eps)
+        gu = f @ _c(W["w_gate_up"][l], dtype).T                      # [n, 2F]: gate rows then up rows
         Fd = cfg["d_ffn"]
         act = silu(gu[:, :Fd]) * gu[:, Fd:]
-        x = x + act @ W["w_down"][l].astype(dtype).T
-    hidden = rmsnorm(x, W["final_norm"].astype(dtype), eps)
-    logits = hidden @ W["lm_head"].astype(dtype).T if want_logits else None
+        x = x + act @ _c(W["w_down"][l], dtype).T
+    hidden = rmsnorm(x, _c(W["final_norm"], dtype), eps)
+    logits = hidden @ _c(W["lm_head"], dtype).T if want_logits else None
     return hidden, logits
 
 
@@ -152,7 +164,7 @@ def prefill(W, cfg, prompt, kv, dtype=F):
     P = len(prompt)
     mask = np.tril(np.ones((P, P), dtype=bool))
     hidden, _ = llm_forward(W, cfg, prompt, np.arange(P), mask, kv, 0, dtype, want_logits=False)
-    logits_last = hidden[P - 1] @ W["lm_head"].astype(dtype).T
+    logits_last = hidden[P - 1] @ _c(W["lm_head"], dtype).T
     return P, argmax_first(logits_last), hidden[P - 1].copy()
 
 
@@ -167,15 +179,15 @@ def ar_step(W, cfg, kv, ctx, g, dtype=F):
 # ----------------------------------------------------------------------------
 def rnn_cell(D, s_prev, e, dtype=F):
     """s_t = f(U s_{t-1} + W e_t + b) (Section 3.1)."""
-    return silu(D["rnn_u"].astype(dtype) @ s_prev + D["rnn_w"].astype(dtype) @ e + D["rnn_b"].astype(dtype))
+    return silu(_c(D["rnn_u"], dtype) @ s_prev + _c(D["rnn_w"], dtype) @ e + _c(D["rnn_b"], dtype))
 
 
 def draft_head(D, g_t, dtype=F):
     """MLP layers with skip connections, then the vocabulary projection (Section 3.1).  Returns logits."""
     x = g_t
     for A, c in zip(D["head_w"], D["head_b"]):
-        x = x + silu(A.astype(dtype) @ x + c.astype(dtype))
-    return D["draft_out"].astype(dtype) @ x
+        x = x + silu(_c(A, dtype) @ x + _c(c, dtype))
+    return _c(D["draft_out"], dtype) @ x
 
 
 def beam_search(D, E, g, h, beam_width, beam_length, dtype=F, return_logp=False):
@@ -187,7 +199,7 @@ def beam_search(D, E, g, h, beam_width, beam_length, dtype=F, return_logp=False)
     """
     V = D["draft_out"].shape[0]
     assert beam_width <= V
-    E = E.astype(dtype) if E.dtype != dtype else E
+    E = _c(E, dtype)
     h = np.asarray(h, dtype=dtype)
     s1 = E[g]
     logp = log_softmax(draft_head(D, np.concatenate([s1, h]), dtype))
@@ -217,7 +229,7 @@ def beam_search(D, E, g, h, beam_width, beam_length, dtype=F, return_logp=False)
 
 def sequence_logprob(D, E, g, h, seq, dtype=F):
     """log p_draft(seq | g, h): the drafter run along one fixed sequence."""
-    E = E.astype(dtype)
+    E = _c(E, dtype)
     s = E[g]
     total = 0.0
     for t, tok in enumerate(seq):

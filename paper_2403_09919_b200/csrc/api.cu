@@ -1,0 +1,537 @@
+// C-ABI entry points (include/redrafter.h): handle, workspace carve-up, and the host-side
+// sequencing of the kernels of one speculative decode step (Section 3.4).  No kernel here.
+#include <stdarg.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "rd_internal.cuh"
+
+using namespace rd;
+
+namespace {
+
+struct Bump {  // carve-up of the caller's workspace; with base == nullptr it only measures
+  char* base;
+  size_t off;
+  template <typename T> T* take(size_t count) {
+    off = (off + 255) & ~size_t(255);
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += count * sizeof(T);
+    return p;
+  }
+};
+
+struct Workspace {
+  // decode state
+  int32_t *ctx, *root, *status;
+  float* h;
+  // row tables of the current forward
+  int32_t *row_tok, *row_seq, *row_pos, *row_slot, *row_ncache, *row_local, *row_out_index, *m_total, *last_row;
+  // activations of the forward (compact rows)
+  float *x, *qkv, *gu, *hidden_f, *logits;
+  void *a_t, *attn_t, *act_t, *hidden_t, *h_t;
+  int32_t* argmax_c;
+  // step-internal packed beam, beams, verify outputs, accept scratch
+  rd_packed pk;
+  int32_t *beams, *argmax_p, *n_accept, *best, *ctx_prev, *acc_tokens;
+  float *scores, *hidden_p;
+  // drafter
+  void *xc_t, *x0_t, *x1_t, *x2_t, *sprev_t, *e_t;
+  float *xc_f, *x0_f, *x1_f, *x2_f, *tmp_f, *dlogits, *lse, *cand_val, *score_a, *score_b;
+  int32_t *cand_idx, *hist_a, *hist_b, *one_b, *one_r;
+};
+
+size_t esize(int dtype) { return dtype == RD_DTYPE_FP32 ? 4 : 2; }
+
+}  // namespace
+
+struct rd_handle {
+  rd_config cfg;
+  Dims dm;
+  int m_cap;  // rows one forward pass can hold
+  Workspace ws;
+  char* kv;
+  size_t kv_plane;  // elements per (layer, K|V) plane
+  std::vector<const void*> attn_norm, wqkv, wo, ffn_norm, w_gate_up, w_down, head_w, head_b;
+  rd_weights w;
+  bool prefilled;
+  int batch;      // active sequences
+  int ctx_bound;  // host-side upper bound of every sequence's context length
+  int64_t launches;
+  char err[512];
+};
+
+namespace {
+
+int fail(rd_handle* h, int code, const char* fmt, ...) {
+  if (h) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(h->err, sizeof(h->err), fmt, ap);
+    va_end(ap);
+  }
+  return code;
+}
+
+bool make_dims(const rd_config* c, Dims* dm) {
+  if (!c || c->struct_bytes != (int32_t)sizeof(rd_config)) return false;
+  if (c->n_layers <= 0 || c->d_model <= 0 || c->n_heads <= 0 || c->d_ffn <= 0 || c->vocab <= 0) return false;
+  if (c->d_model % c->n_heads) return false;
+  if (c->max_batch <= 0 || c->max_ctx <= 0 || c->beam_width <= 0 || c->beam_length <= 0) return false;
+  if (c->dtype != RD_DTYPE_FP32 && c->dtype != RD_DTYPE_BF16) return false;
+  if (c->n_head_layers < 0 || c->d_rnn != c->d_model) return false;
+  dm->n_layers = c->n_layers; dm->d = c->d_model; dm->H = c->n_heads; dm->hd = c->d_model / c->n_heads;
+  dm->F = c->d_ffn; dm->V = c->vocab; dm->dr = c->d_rnn; dm->dh = c->d_rnn + c->d_model;
+  dm->n_head_layers = c->n_head_layers; dm->B = c->max_batch; dm->max_ctx = c->max_ctx;
+  dm->BW = c->beam_width; dm->L = c->beam_length; dm->NMAX = 1 + c->beam_width * c->beam_length;
+  dm->MW = (dm->NMAX + 31) / 32; dm->eps = c->rms_eps; dm->theta = c->rope_theta; dm->dtype = c->dtype;
+  return true;
+}
+
+int shape_ok(const Dims& dm) {
+  const int vec = dm.dtype == RD_DTYPE_FP32 ? 4 : 8;
+  if (dm.hd != 64 && dm.hd != 128) return 0;
+  if (dm.d % vec || dm.F % vec || dm.dh % vec) return 0;
+  if (dm.BW > dm.V || dm.BW > 128) return 0;
+  if (dm.BW * (dm.L + 1) > 1024 || dm.NMAX > 1024) return 0;
+  return 1;
+}
+
+int m_cap_of(const Dims& dm) {
+  const int v = dm.B * dm.NMAX;
+  return v > 256 ? v : 256;
+}
+
+void carve(Bump& bp, const Dims& dm, int m_cap, Workspace* w) {
+  const size_t es = esize(dm.dtype);
+  const int B = dm.B, R = dm.B * dm.BW, C = dm.L + 1;
+  w->ctx = bp.take<int32_t>(B); w->root = bp.take<int32_t>(B); w->status = bp.take<int32_t>(4);
+  w->h = bp.take<float>((size_t)B * dm.d);
+  w->row_tok = bp.take<int32_t>(m_cap); w->row_seq = bp.take<int32_t>(m_cap); w->row_pos = bp.take<int32_t>(m_cap);
+  w->row_slot = bp.take<int32_t>(m_cap); w->row_ncache = bp.take<int32_t>(m_cap); w->row_local = bp.take<int32_t>(m_cap);
+  w->row_out_index = bp.take<int32_t>(m_cap); w->m_total = bp.take<int32_t>(4); w->last_row = bp.take<int32_t>(B);
+  w->x = bp.take<float>((size_t)m_cap * dm.d);
+  w->qkv = bp.take<float>((size_t)m_cap * 3 * dm.d);
+  w->gu = bp.take<float>((size_t)m_cap * 2 * dm.F);
+  w->hidden_f = bp.take<float>((size_t)m_cap * dm.d);
+  w->logits = bp.take<float>((size_t)m_cap * dm.V);
+  w->a_t = bp.take<char>((size_t)m_cap * dm.d * es);
+  w->attn_t = bp.take<char>((size_t)m_cap * dm.d * es);
+  w->act_t = bp.take<char>((size_t)m_cap * dm.F * es);
+  w->hidden_t = bp.take<char>((size_t)m_cap * dm.d * es);
+  w->h_t = bp.take<char>((size_t)B * dm.d * es);
+  w->argmax_c = bp.take<int32_t>(m_cap);
+  w->pk.tokens = bp.take<int32_t>((size_t)B * dm.NMAX); w->pk.n = bp.take<int32_t>(B);
+  w->pk.unpack = bp.take<int32_t>((size_t)R * C); w->pk.pos = bp.take<int32_t>((size_t)B * dm.NMAX);
+  w->pk.mask = bp.take<uint32_t>((size_t)B * dm.NMAX * dm.MW); w->pk.parent = bp.take<int32_t>((size_t)B * dm.NMAX);
+  w->beams = bp.take<int32_t>((size_t)R * dm.L); w->argmax_p = bp.take<int32_t>((size_t)B * dm.NMAX);
+  w->n_accept = bp.take<int32_t>(B); w->best = bp.take<int32_t>(B); w->ctx_prev = bp.take<int32_t>(B);
+  w->acc_tokens = bp.take<int32_t>((size_t)B * C);
+  w->scores = bp.take<float>(R); w->hidden_p = bp.take<float>((size_t)B * dm.NMAX * dm.d);
+  w->xc_t = bp.take<char>((size_t)B * dm.dh * es); w->x0_t = bp.take<char>((size_t)R * dm.dh * es);
+  w->x1_t = bp.take<char>((size_t)R * dm.dh * es); w->x2_t = bp.take<char>((size_t)R * dm.dh * es);
+  w->sprev_t = bp.take<char>((size_t)R * dm.dr * es); w->e_t = bp.take<char>((size_t)R * dm.d * es);
+  w->xc_f = bp.take<float>((size_t)B * dm.dh); w->x0_f = bp.take<float>((size_t)R * dm.dh);
+  w->x1_f = bp.take<float>((size_t)R * dm.dh); w->x2_f = bp.take<float>((size_t)R * dm.dh);
+  w->tmp_f = bp.take<float>((size_t)R * dm.dr); w->dlogits = bp.take<float>((size_t)R * dm.V);
+  w->lse = bp.take<float>(R); w->cand_val = bp.take<float>((size_t)R * dm.BW);
+  w->score_a = bp.take<float>(R); w->score_b = bp.take<float>(R);
+  w->cand_idx = bp.take<int32_t>((size_t)R * dm.BW); w->hist_a = bp.take<int32_t>((size_t)R * dm.L);
+  w->hist_b = bp.take<int32_t>((size_t)R * dm.L); w->one_b = bp.take<int32_t>(4); w->one_r = bp.take<int32_t>(4);
+  bp.take<char>(256);
+}
+
+#define CK(h, expr)                                                                              \
+  do {                                                                                           \
+    cudaError_t e__ = (expr);                                                                    \
+    if (e__ != cudaSuccess) return fail(h, RD_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e__)); \
+    (h)->launches++;                                                                             \
+  } while (0)
+#define CKRT(h, expr)                                                                            \
+  do {                                                                                           \
+    cudaError_t e__ = (expr);                                                                    \
+    if (e__ != cudaSuccess) return fail(h, RD_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e__)); \
+  } while (0)
+
+Epilogue ep_store(float* out, int ld) {
+  Epilogue e{};
+  e.out_f32 = out; e.ld_out_f32 = ld;
+  return e;
+}
+
+// One projection; picks the kernel.
+int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, const int32_t* m_total, int m_max,
+         const Epilogue& ep, cudaStream_t st) {
+  CK(h, launch_gemm_simt(h->dm.dtype, A, lda, W, N, K, m_total, m_max, ep, st));
+  return RD_OK;
+}
+
+char* kv_plane_ptr(rd_handle* h, int layer, int which) {
+  return h->kv + ((size_t)(layer * 2 + which)) * h->kv_plane * esize(h->dm.dtype);
+}
+
+// Embedding -> n_layers x {attention block, FFN block} -> final norm.  Rows and masks come from the
+// row tables in the workspace; results: ws.hidden_f / ws.hidden_t (compact rows).
+int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, cudaStream_t st) {
+  Workspace& w = h->ws;
+  const Dims& dm = h->dm;
+  RowTables rt{w.row_tok, w.row_seq, w.row_pos, w.row_slot, w.row_ncache, w.row_local, mask, w.m_total};
+  CK(h, launch_embed(dm.dtype, h->w.tok_emb, w.row_tok, w.x, dm.d, dm.V, w.m_total, m_max, w.status, st));
+  for (int l = 0; l < dm.n_layers; ++l) {
+    CK(h, launch_rmsnorm(dm.dtype, w.x, h->attn_norm[l], w.a_t, nullptr, dm.d, dm.eps, w.m_total, m_max, st));
+    int rc = gemm(h, w.a_t, dm.d, h->wqkv[l], 3 * dm.d, dm.d, w.m_total, m_max, ep_store(w.qkv, 3 * dm.d), st);
+    if (rc) return rc;
+    CK(h, launch_rope_kv(dm.dtype, w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), rt, dm, m_max, w.status, st));
+    CK(h, launch_attention(dm.dtype, w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.attn_t, rt, dm, m_max, st));
+    Epilogue eo{};
+    eo.resid = w.x; eo.ld_resid = dm.d; eo.out_f32 = w.x; eo.ld_out_f32 = dm.d;
+    rc = gemm(h, w.attn_t, dm.d, h->wo[l], dm.d, dm.d, w.m_total, m_max, eo, st);
+    if (rc) return rc;
+    CK(h, launch_rmsnorm(dm.dtype, w.x, h->ffn_norm[l], w.a_t, nullptr, dm.d, dm.eps, w.m_total, m_max, st));
+    rc = gemm(h, w.a_t, dm.d, h->w_gate_up[l], 2 * dm.F, dm.d, w.m_total, m_max, ep_store(w.gu, 2 * dm.F), st);
+    if (rc) return rc;
+    CK(h, launch_swiglu(dm.dtype, w.gu, w.act_t, dm.F, w.m_total, m_max, st));
+    rc = gemm(h, w.act_t, dm.F, h->w_down[l], dm.d, dm.F, w.m_total, m_max, eo, st);
+    if (rc) return rc;
+  }
+  CK(h, launch_rmsnorm(dm.dtype, w.x, h->w.final_norm, w.hidden_t, w.hidden_f, dm.d, dm.eps, w.m_total, m_max, st));
+  return RD_OK;
+}
+
+int check_stepable(rd_handle* h) {
+  if (!h) return RD_ERR_INVALID_ARG;
+  if (!h->prefilled) return fail(h, RD_ERR_STATE, "no state: call redrafter_prefill or redrafter_set_state first");
+  if (h->ctx_bound + h->dm.NMAX > h->dm.max_ctx)
+    return fail(h, RD_ERR_CAPACITY, "context bound %d + %d packed rows exceeds max_ctx %d", h->ctx_bound, h->dm.NMAX,
+                h->dm.max_ctx);
+  return RD_OK;
+}
+
+int do_draft(rd_handle* h, cudaStream_t st, int32_t* beams, float* scores) {
+  Workspace& w = h->ws;
+  const Dims& dm = h->dm;
+  const int B = h->batch, R = B * dm.BW;
+  CK(h, launch_draft_init(dm.dtype, h->w.tok_emb, w.root, w.h, w.xc_t, w.xc_f, w.sprev_t, dm, B, w.status, st));
+  if (dm.L > 1) CK(h, launch_fill_h(dm.dtype, w.h, w.x0_t, w.x0_f, dm, B, st));
+  float *sc_in = w.score_a, *sc_out = w.score_b;
+  int32_t *hi_in = w.hist_a, *hi_out = w.hist_b;
+  for (int call = 1; call <= dm.L; ++call) {
+    const int rows = call == 1 ? B : R;
+    const int32_t* mt = call == 1 ? w.one_b : w.one_r;
+    const void* xin_t = call == 1 ? w.xc_t : w.x0_t;
+    const float* xin_f = call == 1 ? w.xc_f : w.x0_f;
+    if (call > 1) {
+      // s_t = SiLU(U s_{t-1} + W e_t + b), written into the first d_rnn columns of x0 = [s_t, h]
+      int rc = gemm(h, w.sprev_t, dm.dr, h->w.rnn_u, dm.dr, dm.dr, mt, rows, ep_store(w.tmp_f, dm.dr), st);
+      if (rc) return rc;
+      Epilogue e{};
+      e.addend = w.tmp_f; e.ld_addend = dm.dr; e.bias = h->w.rnn_b; e.silu = 1;
+      e.out_f32 = w.x0_f; e.ld_out_f32 = dm.dh; e.out_t = w.x0_t; e.ld_out_t = dm.dh;
+      rc = gemm(h, w.e_t, dm.d, h->w.rnn_w, dm.dr, dm.d, mt, rows, e, st);
+      if (rc) return rc;
+    }
+    for (int l = 0; l < dm.n_head_layers; ++l) {
+      Epilogue e{};
+      e.bias = h->head_b[l]; e.silu = 1; e.resid = xin_f; e.ld_resid = dm.dh;
+      float* of = (l & 1) ? w.x2_f : w.x1_f;
+      void* ot = (l & 1) ? w.x2_t : w.x1_t;
+      e.out_f32 = of; e.ld_out_f32 = dm.dh; e.out_t = ot; e.ld_out_t = dm.dh;
+      int rc = gemm(h, xin_t, dm.dh, h->head_w[l], dm.dh, dm.dh, mt, rows, e, st);
+      if (rc) return rc;
+      xin_t = ot; xin_f = of;
+    }
+    int rc = gemm(h, xin_t, dm.dh, h->w.draft_out, dm.V, dm.dh, mt, rows, ep_store(w.dlogits, dm.V), st);
+    if (rc) return rc;
+    CK(h, launch_row_topk(w.dlogits, dm.V, dm.BW, w.lse, w.cand_val, w.cand_idx, rows, st));
+    CK(h, launch_beam_merge(dm.dtype, call, w.lse, w.cand_val, w.cand_idx, sc_in, sc_out, hi_in, hi_out, h->w.tok_emb,
+                            w.x0_f, dm.dh, w.sprev_t, w.e_t, dm, B, beams, scores, st));
+    float* tf = sc_in; sc_in = sc_out; sc_out = tf;
+    int32_t* ti = hi_in; hi_in = hi_out; hi_out = ti;
+  }
+  return RD_OK;
+}
+
+int do_verify(rd_handle* h, const rd_packed& pk, cudaStream_t st, int32_t* argmax, float* hidden, float* logits) {
+  Workspace& w = h->ws;
+  const Dims& dm = h->dm;
+  const int B = h->batch, m_max = B * dm.NMAX;
+  CK(h, launch_build_rows_tree(pk, w.ctx, w.row_tok, w.row_seq, w.row_pos, w.row_slot, w.row_ncache, w.row_local,
+                               w.row_out_index, w.m_total, dm, B, w.status, st));
+  int rc = forward_layers(h, pk.mask, m_max, st);
+  if (rc) return rc;
+  rc = gemm(h, w.hidden_t, dm.d, h->w.lm_head, dm.V, dm.d, w.m_total, m_max, ep_store(w.logits, dm.V), st);
+  if (rc) return rc;
+  CK(h, launch_fill_i32(argmax, -1, B * dm.NMAX, st));
+  CK(h, launch_argmax_rows(w.logits, dm.V, argmax, w.row_out_index, w.m_total, m_max, st));
+  if (hidden) CK(h, launch_scatter_rows(w.hidden_f, dm.d, hidden, w.row_out_index, w.m_total, m_max, st));
+  if (logits) CK(h, launch_scatter_rows(w.logits, dm.V, logits, w.row_out_index, w.m_total, m_max, st));
+  return RD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t redrafter_workspace_bytes(const rd_config* cfg) {
+  Dims dm;
+  if (!make_dims(cfg, &dm) || !shape_ok(dm)) return 0;
+  Bump bp{nullptr, 0};
+  Workspace w;
+  carve(bp, dm, m_cap_of(dm), &w);
+  return bp.off;
+}
+
+size_t redrafter_kv_bytes(const rd_config* cfg) {
+  Dims dm;
+  if (!make_dims(cfg, &dm)) return 0;
+  return (size_t)dm.n_layers * 2 * dm.B * dm.H * (size_t)dm.max_ctx * dm.hd * esize(dm.dtype);
+}
+
+int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, size_t kv_bytes, void* workspace,
+                   size_t ws_bytes, rd_handle** out) {
+  if (!cfg || !wt || !kv_cache || !workspace || !out) return RD_ERR_INVALID_ARG;
+  *out = nullptr;
+  Dims dm;
+  if (!make_dims(cfg, &dm)) return RD_ERR_INVALID_ARG;
+  if (!shape_ok(dm)) return RD_ERR_SHAPE;
+  if (((uintptr_t)kv_cache | (uintptr_t)workspace) & 255) return RD_ERR_INVALID_ARG;
+  if (kv_bytes < redrafter_kv_bytes(cfg) || ws_bytes < redrafter_workspace_bytes(cfg)) return RD_ERR_CAPACITY;
+  if (!wt->tok_emb || !wt->final_norm || !wt->lm_head || !wt->attn_norm || !wt->wqkv || !wt->wo || !wt->ffn_norm ||
+      !wt->w_gate_up || !wt->w_down || !wt->rnn_u || !wt->rnn_w || !wt->rnn_b || !wt->draft_out ||
+      (dm.n_head_layers && (!wt->head_w || !wt->head_b)))
+    return RD_ERR_INVALID_ARG;
+  rd_handle* h = new (std::nothrow) rd_handle();
+  if (!h) return RD_ERR_INVALID_ARG;
+  h->cfg = *cfg; h->dm = dm; h->m_cap = m_cap_of(dm);
+  h->kv = (char*)kv_cache;
+  h->kv_plane = (size_t)dm.B * dm.H * (size_t)dm.max_ctx * dm.hd;
+  h->w = *wt;
+  for (int l = 0; l < dm.n_layers; ++l) {
+    h->attn_norm.push_back(wt->attn_norm[l]); h->wqkv.push_back(wt->wqkv[l]); h->wo.push_back(wt->wo[l]);
+    h->ffn_norm.push_back(wt->ffn_norm[l]); h->w_gate_up.push_back(wt->w_gate_up[l]); h->w_down.push_back(wt->w_down[l]);
+    if (!wt->attn_norm[l] || !wt->wqkv[l] || !wt->wo[l] || !wt->ffn_norm[l] || !wt->w_gate_up[l] || !wt->w_down[l]) {
+      delete h;
+      return RD_ERR_INVALID_ARG;
+    }
+  }
+  for (int l = 0; l < dm.n_head_layers; ++l) {
+    h->head_w.push_back(wt->head_w[l]); h->head_b.push_back(wt->head_b[l]);
+    if (!wt->head_w[l] || !wt->head_b[l]) { delete h; return RD_ERR_INVALID_ARG; }
+  }
+  Bump bp{(char*)workspace, 0};
+  carve(bp, dm, h->m_cap, &h->ws);
+  h->prefilled = false; h->batch = dm.B; h->ctx_bound = 0; h->launches = 0; h->err[0] = 0;
+  // clear the state and the constants the kernels read from device memory
+  cudaError_t e = cudaMemsetAsync(workspace, 0, (size_t)((char*)h->ws.x - (char*)workspace), 0);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(0);
+  if (e != cudaSuccess) { delete h; return RD_ERR_CUDA; }
+  *out = h;
+  return RD_OK;
+}
+
+int redrafter_destroy(rd_handle* h) {
+  if (!h) return RD_ERR_INVALID_ARG;
+  delete h;
+  return RD_OK;
+}
+
+const char* redrafter_last_error(const rd_handle* h) { return h ? h->err : "null handle"; }
+
+int64_t redrafter_launch_count(const rd_handle* h) { return h ? h->launches : 0; }
+
+static int set_row_counts(rd_handle* h, cudaStream_t st) {
+  CK(h, launch_fill_i32(h->ws.one_b, h->batch, 1, st));
+  CK(h, launch_fill_i32(h->ws.one_r, h->batch * h->dm.BW, 1, st));
+  return RD_OK;
+}
+
+int redrafter_prefill(rd_handle* h, const int32_t* tokens, const int32_t* prompt_len, int32_t max_prompt, int32_t batch,
+                      void* stream) {
+  if (!h || !tokens || !prompt_len) return RD_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const Dims& dm = h->dm;
+  Workspace& w = h->ws;
+  if (batch <= 0 || batch > dm.B) return fail(h, RD_ERR_INVALID_ARG, "batch %d outside [1, %d]", batch, dm.B);
+  int longest = 0;
+  for (int b = 0; b < batch; ++b) {
+    if (prompt_len[b] <= 0 || prompt_len[b] > max_prompt) return fail(h, RD_ERR_INVALID_ARG, "prompt_len[%d] = %d", b, prompt_len[b]);
+    if (prompt_len[b] + dm.NMAX > dm.max_ctx) return fail(h, RD_ERR_CAPACITY, "prompt %d of length %d leaves no room for a step", b, prompt_len[b]);
+    longest = prompt_len[b] > longest ? prompt_len[b] : longest;
+  }
+  h->batch = batch;
+  int rc = set_row_counts(h, st);
+  if (rc) return rc;
+  // passes of up to m_cap rows; a sequence's rows may span passes (its earlier rows are in the cache by then)
+  const int cap = h->m_cap;
+  std::vector<int32_t> tok(cap), seq(cap), pos(cap), ncache(cap), local(cap), last(batch);
+  int b = 0, done = 0;  // next sequence, tokens of it already processed
+  while (b < batch) {
+    int m = 0;
+    for (int i = 0; i < batch; ++i) last[i] = -1;
+    while (b < batch && m < cap) {
+      const int take = (prompt_len[b] - done) < (cap - m) ? (prompt_len[b] - done) : (cap - m);
+      for (int i = 0; i < take; ++i) {
+        tok[m] = tokens[(size_t)b * max_prompt + done + i];
+        seq[m] = b; pos[m] = done + i; ncache[m] = done + i + 1; local[m] = 0;
+        ++m;
+      }
+      done += take;
+      if (done == prompt_len[b]) { last[b] = m - 1; ++b; done = 0; }
+    }
+    const size_t nb = (size_t)m * sizeof(int32_t);
+    CKRT(h, cudaMemcpyAsync(w.row_tok, tok.data(), nb, cudaMemcpyHostToDevice, st));
+    CKRT(h, cudaMemcpyAsync(w.row_seq, seq.data(), nb, cudaMemcpyHostToDevice, st));
+    CKRT(h, cudaMemcpyAsync(w.row_pos, pos.data(), nb, cudaMemcpyHostToDevice, st));
+    CKRT(h, cudaMemcpyAsync(w.row_slot, pos.data(), nb, cudaMemcpyHostToDevice, st));
+    CKRT(h, cudaMemcpyAsync(w.row_ncache, ncache.data(), nb, cudaMemcpyHostToDevice, st));
+    CKRT(h, cudaMemcpyAsync(w.row_local, local.data(), nb, cudaMemcpyHostToDevice, st));
+    CKRT(h, cudaMemcpyAsync(w.last_row, last.data(), batch * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    CKRT(h, cudaMemcpyAsync(w.m_total, &m, sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    CKRT(h, cudaStreamSynchronize(st));  // the host staging vectors are reused by the next pass
+    rc = forward_layers(h, nullptr, m, st);
+    if (rc) return rc;
+    CK(h, launch_prefill_finish(w.hidden_f, w.last_row, w.h, dm.d, batch, st));
+  }
+  // root token: the greedy token after the prompt = argmax(lm_head h)
+  CK(h, launch_cast_rows(dm.dtype, w.h, w.h_t, batch * dm.d, st));
+  rc = gemm(h, w.h_t, dm.d, h->w.lm_head, dm.V, dm.d, w.one_b, batch, ep_store(w.logits, dm.V), st);
+  if (rc) return rc;
+  CK(h, launch_argmax_rows(w.logits, dm.V, w.root, nullptr, w.one_b, batch, st));
+  CKRT(h, cudaMemcpyAsync(w.ctx, prompt_len, batch * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+  h->prefilled = true;
+  h->ctx_bound = longest;
+  return RD_OK;
+}
+
+int redrafter_draft(rd_handle* h, void* stream, int32_t* beams, float* scores) {
+  int rc = check_stepable(h);
+  if (rc) return rc;
+  if (!beams) return fail(h, RD_ERR_INVALID_ARG, "beams is null");
+  return do_draft(h, (cudaStream_t)stream, beams, scores);
+}
+
+static bool packed_ok(const rd_packed* p) {
+  return p && p->tokens && p->n && p->unpack && p->pos && p->mask && p->parent;
+}
+
+int redrafter_pack(rd_handle* h, const int32_t* beams, void* stream, const rd_packed* out) {
+  int rc = check_stepable(h);
+  if (rc) return rc;
+  if (!beams || !packed_ok(out)) return fail(h, RD_ERR_INVALID_ARG, "null beams or packed member");
+  cudaStream_t st = (cudaStream_t)stream;
+  CK(h, launch_pack(beams, h->ws.root, h->ws.ctx, *out, h->dm, h->batch, (h->cfg.flags & RD_FLAG_NO_TREE) ? 1 : 0, st));
+  return RD_OK;
+}
+
+int redrafter_verify(rd_handle* h, const rd_packed* packed, void* stream, int32_t* argmax, float* hidden, float* logits) {
+  int rc = check_stepable(h);
+  if (rc) return rc;
+  if (!packed_ok(packed) || !argmax) return fail(h, RD_ERR_INVALID_ARG, "null packed member or argmax");
+  return do_verify(h, *packed, (cudaStream_t)stream, argmax, hidden, logits);
+}
+
+int redrafter_accept(rd_handle* h, const int32_t* beams, const rd_packed* packed, const int32_t* argmax,
+                     const float* hidden, void* stream, const rd_accept_out* out) {
+  int rc = check_stepable(h);
+  if (rc) return rc;
+  if (!beams || !packed_ok(packed) || !argmax || !hidden) return fail(h, RD_ERR_INVALID_ARG, "null argument");
+  Workspace& w = h->ws;
+  rd_accept_out o{};
+  if (out) o = *out;
+  CK(h, launch_accept(h->dm.dtype, beams, *packed, argmax, hidden, h->kv, w.ctx, w.root, w.h, o, w.n_accept, w.best,
+                      w.ctx_prev, h->dm, h->batch, w.status, (cudaStream_t)stream));
+  h->launches++;  // accept + compaction
+  h->ctx_bound += 1 + h->dm.L;
+  return RD_OK;
+}
+
+int redrafter_step(rd_handle* h, const int32_t* planted_beams, void* stream, const rd_accept_out* out) {
+  int rc = check_stepable(h);
+  if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  Workspace& w = h->ws;
+  rc = do_draft(h, st, w.beams, w.scores);
+  if (rc) return rc;
+  const int32_t* beams = planted_beams ? planted_beams : w.beams;
+  CK(h, launch_pack(beams, w.root, w.ctx, w.pk, h->dm, h->batch, (h->cfg.flags & RD_FLAG_NO_TREE) ? 1 : 0, st));
+  rc = do_verify(h, w.pk, st, w.argmax_p, w.hidden_p, nullptr);
+  if (rc) return rc;
+  rd_accept_out o{};
+  if (out) o = *out;
+  CK(h, launch_accept(h->dm.dtype, beams, w.pk, w.argmax_p, w.hidden_p, h->kv, w.ctx, w.root, w.h, o, w.n_accept,
+                      w.best, w.ctx_prev, h->dm, h->batch, w.status, st));
+  h->launches++;
+  h->ctx_bound += 1 + h->dm.L;
+  return RD_OK;
+}
+
+int redrafter_ar_step(rd_handle* h, void* stream, int32_t* token) {
+  if (!h) return RD_ERR_INVALID_ARG;
+  if (!h->prefilled) return fail(h, RD_ERR_STATE, "no state: call redrafter_prefill or redrafter_set_state first");
+  if (h->ctx_bound + 1 > h->dm.max_ctx) return fail(h, RD_ERR_CAPACITY, "KV cache full");
+  cudaStream_t st = (cudaStream_t)stream;
+  Workspace& w = h->ws;
+  const Dims& dm = h->dm;
+  const int B = h->batch;
+  CK(h, launch_build_rows_ar(w.root, w.ctx, w.row_tok, w.row_seq, w.row_pos, w.row_slot, w.row_ncache, w.row_local,
+                             w.row_out_index, w.m_total, dm, B, w.status, st));
+  int rc = forward_layers(h, nullptr, B, st);
+  if (rc) return rc;
+  rc = gemm(h, w.hidden_t, dm.d, h->w.lm_head, dm.V, dm.d, w.m_total, B, ep_store(w.logits, dm.V), st);
+  if (rc) return rc;
+  CK(h, launch_argmax_rows(w.logits, dm.V, w.argmax_c, nullptr, w.m_total, B, st));
+  CK(h, launch_ar_finish(w.argmax_c, w.hidden_f, w.ctx, w.root, w.h, token, dm, B, st));
+  h->ctx_bound += 1;
+  return RD_OK;
+}
+
+int redrafter_get_state(rd_handle* h, void* stream, int32_t* ctx, int32_t* root, float* hvec) {
+  if (!h) return RD_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t B = h->batch;
+  if (ctx) CKRT(h, cudaMemcpyAsync(ctx, h->ws.ctx, B * sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
+  if (root) CKRT(h, cudaMemcpyAsync(root, h->ws.root, B * sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
+  if (hvec) CKRT(h, cudaMemcpyAsync(hvec, h->ws.h, B * h->dm.d * sizeof(float), cudaMemcpyDeviceToDevice, st));
+  return RD_OK;
+}
+
+int redrafter_set_state(rd_handle* h, void* stream, const int32_t* ctx, const int32_t* root, const float* hvec,
+                        int32_t batch) {
+  if (!h) return RD_ERR_INVALID_ARG;
+  if (batch <= 0 || batch > h->dm.B) return fail(h, RD_ERR_INVALID_ARG, "batch %d outside [1, %d]", batch, h->dm.B);
+  cudaStream_t st = (cudaStream_t)stream;
+  h->batch = batch;
+  int rc = set_row_counts(h, st);
+  if (rc) return rc;
+  const size_t B = batch;
+  if (ctx) CKRT(h, cudaMemcpyAsync(h->ws.ctx, ctx, B * sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
+  if (root) CKRT(h, cudaMemcpyAsync(h->ws.root, root, B * sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
+  if (hvec) CKRT(h, cudaMemcpyAsync(h->ws.h, hvec, B * h->dm.d * sizeof(float), cudaMemcpyDeviceToDevice, st));
+  h->prefilled = true;
+  return RD_OK;
+}
+
+int redrafter_set_ctx_bound(rd_handle* h, int32_t max_ctx_now) {
+  if (!h || max_ctx_now < 0) return RD_ERR_INVALID_ARG;
+  h->ctx_bound = max_ctx_now;
+  return RD_OK;
+}
+
+int redrafter_poll(rd_handle* h, void* stream) {
+  if (!h) return RD_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  int32_t v = 0;
+  CKRT(h, cudaMemcpyAsync(&v, h->ws.status, sizeof(v), cudaMemcpyDeviceToHost, st));
+  CKRT(h, cudaStreamSynchronize(st));
+  if (v == 0) return RD_OK;
+  CKRT(h, cudaMemsetAsync(h->ws.status, 0, sizeof(int32_t), st));
+  if (v & DEV_ERR_TIMEOUT) return fail(h, RD_ERR_TIMEOUT, "device status 0x%x: a bounded wait gave up", v);
+  if (v & DEV_ERR_CAPACITY) return fail(h, RD_ERR_CAPACITY, "device status 0x%x: a KV slot beyond max_ctx was skipped", v);
+  return fail(h, RD_ERR_INVALID_ARG, "device status 0x%x: token id or index out of range", v);
+}
+
+}  // extern "C"

@@ -1,0 +1,225 @@
+// Beam search over the RNN drafter (Sections 3.1, 3.2): the small kernels around the
+// projections.  A drafter call t works on R = B*BW rows (call 1: B rows):
+//   rnn:   s_t = SiLU(U s_{t-1} + W e_t + b)            two projections with a fused epilogue
+//   head:  x <- x + SiLU(A_l x + c_l), x_0 = [s_t, h]   one projection per layer, fused epilogue
+//   out:   logits = O x                                  one projection
+//   row_topk:   per row, log-sum-exp and the BW best logits (value desc, index asc)
+//   beam_merge: per sequence, score_r + logit - lse_r over the BW*BW survivors, best BW in
+//               (score desc, flat index r*V + v asc) order; reorders histories and states and
+//               gathers the next call's inputs (e_{t+1} = E[token], s_t of the parent).
+#include "rd_internal.cuh"
+
+namespace rd {
+
+#define RD_DISPATCH(dtype, ...)                                \
+  if ((dtype) == RD_DTYPE_FP32) { using T = float; __VA_ARGS__; } \
+  else { using T = __nv_bfloat16; __VA_ARGS__; }
+
+// ---------------------------------------------------------------- call-1 input and s_1
+// x[b] = [E[g_b], h_b] for the first call; sprev[r] = E[g_b] = s_1 for every beam row of b.
+template <typename T>
+__global__ void draft_init_kernel(const T* __restrict__ emb, const int32_t* __restrict__ root, const float* __restrict__ h,
+                                  T* __restrict__ x_t, float* __restrict__ x_f, T* __restrict__ sprev_t, Dims dm,
+                                  int* status) {
+  const int b = blockIdx.x;
+  int g = root[b];
+  if (g < 0 || g >= dm.V) {
+    if (threadIdx.x == 0) atomicOr(status, DEV_ERR_TOKEN_RANGE);
+    g = min(max(g, 0), dm.V - 1);
+  }
+  const int d = dm.d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    const T e = emb[(size_t)g * d + i];
+    x_t[(size_t)b * dm.dh + i] = e;
+    x_f[(size_t)b * dm.dh + i] = to_f<T>(e);
+    const float hv = h[(size_t)b * d + i];
+    x_t[(size_t)b * dm.dh + dm.dr + i] = from_f<T>(hv);
+    x_f[(size_t)b * dm.dh + dm.dr + i] = hv;
+    for (int k = 0; k < dm.BW; ++k) sprev_t[((size_t)b * dm.BW + k) * dm.dr + i] = e;
+  }
+}
+
+cudaError_t launch_draft_init(int dtype, const void* emb, const int32_t* root, const float* h, void* x_t, float* x_f,
+                              void* sprev_t, const Dims& dm, int B, int* status, cudaStream_t st) {
+  RD_DISPATCH(dtype, draft_init_kernel<T><<<B, 256, 0, st>>>((const T*)emb, root, h, (T*)x_t, x_f, (T*)sprev_t, dm, status));
+  return cudaGetLastError();
+}
+
+// h part of g_t = [s_t, h] for every beam row (constant over the calls of one step).
+template <typename T>
+__global__ void fill_h_kernel(const float* __restrict__ h, T* __restrict__ x_t, float* __restrict__ x_f, Dims dm) {
+  const int r = blockIdx.x, b = r / dm.BW;
+  for (int i = threadIdx.x; i < dm.d; i += blockDim.x) {
+    const float hv = h[(size_t)b * dm.d + i];
+    x_t[(size_t)r * dm.dh + dm.dr + i] = from_f<T>(hv);
+    x_f[(size_t)r * dm.dh + dm.dr + i] = hv;
+  }
+}
+
+cudaError_t launch_fill_h(int dtype, const float* h, void* x_t, float* x_f, const Dims& dm, int B, cudaStream_t st) {
+  RD_DISPATCH(dtype, fill_h_kernel<T><<<B * dm.BW, 256, 0, st>>>(h, (T*)x_t, x_f, dm));
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- per-row log-sum-exp + top-BW
+// Ordering (value desc, index asc).  Selection is stateless: pass p picks the best element that
+// comes strictly after the element picked by pass p-1, so nothing is marked or modified.
+struct Cand {
+  float v;
+  int i;
+};
+__device__ __forceinline__ bool cand_before(float va, int ia, float vb, int ib) {  // a ranks before b
+  return va > vb || (va == vb && ia < ib);
+}
+__device__ __forceinline__ Cand cand_best(Cand a, Cand b) { return cand_before(a.v, a.i, b.v, b.i) ? a : b; }
+__device__ __forceinline__ Cand block_best(Cand c, Cand* sh) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    Cand t;
+    t.v = __shfl_xor_sync(0xffffffffu, c.v, o);
+    t.i = __shfl_xor_sync(0xffffffffu, c.i, o);
+    c = cand_best(c, t);
+  }
+  __syncthreads();
+  if (lane == 0) sh[w] = c;
+  __syncthreads();
+  Cand r = lane < nw ? sh[lane] : Cand{-INFINITY, 0x7fffffff};
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    Cand t;
+    t.v = __shfl_xor_sync(0xffffffffu, r.v, o);
+    t.i = __shfl_xor_sync(0xffffffffu, r.i, o);
+    r = cand_best(r, t);
+  }
+  return r;  // identical in every thread
+}
+
+__global__ void __launch_bounds__(1024) row_topk_kernel(const float* __restrict__ logits, int V, int BW,
+                                                         float* __restrict__ lse, float* __restrict__ val,
+                                                         int32_t* __restrict__ idx) {
+  __shared__ Cand sh[32];
+  __shared__ float shf[32];
+  const int r = blockIdx.x;
+  const float* z = logits + (size_t)r * V;
+  // max, then sum of exp
+  Cand c{-INFINITY, 0x7fffffff};
+  for (int i = threadIdx.x; i < V; i += blockDim.x) c = cand_best(c, Cand{z[i], i});
+  Cand top = block_best(c, sh);
+  float s = 0.f;
+  for (int i = threadIdx.x; i < V; i += blockDim.x) s += expf(z[i] - top.v);
+  {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    __syncthreads();
+    if (lane == 0) shf[w] = s;
+    __syncthreads();
+    s = lane < nw ? shf[lane] : 0.f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  }
+  if (threadIdx.x == 0) {
+    lse[r] = top.v + logf(s);
+    val[(size_t)r * BW] = top.v;
+    idx[(size_t)r * BW] = top.i;
+  }
+  Cand prev = top;
+  for (int p = 1; p < BW; ++p) {
+    Cand best{-INFINITY, 0x7fffffff};
+    for (int i = threadIdx.x; i < V; i += blockDim.x) {
+      const float v = z[i];
+      if (cand_before(prev.v, prev.i, v, i)) best = cand_best(best, Cand{v, i});
+    }
+    best = block_best(best, sh);
+    if (threadIdx.x == 0) {
+      val[(size_t)r * BW + p] = best.v;
+      idx[(size_t)r * BW + p] = best.i == 0x7fffffff ? 0 : best.i;
+    }
+    prev = best;
+  }
+}
+
+cudaError_t launch_row_topk(const float* logits, int V, int BW, float* lse, float* val, int32_t* idx, int rows,
+                            cudaStream_t st) {
+  row_topk_kernel<<<rows, 1024, 0, st>>>(logits, V, BW, lse, val, idx);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- cross-row merge + reorder + gather
+// One CTA per sequence.  call == 1: the single row's top-BW become the beams.  call >= 2: best BW of
+// the BW*BW survivors.  Writes score_out[k], hist_out[k][0..call-1], and the next call's inputs
+// sprev_t[k] = s_t of the parent (read from s_new_f with row stride ld_s; skipped for call 1, where
+// every beam keeps s_1) and e_t[k] = E[token_k].  On the last call also the public outputs.
+template <typename T>
+__global__ void __launch_bounds__(256) beam_merge_kernel(int call, const float* __restrict__ lse,
+                                                          const float* __restrict__ val, const int32_t* __restrict__ idx,
+                                                          const float* __restrict__ score_in, float* __restrict__ score_out,
+                                                          const int32_t* __restrict__ hist_in, int32_t* __restrict__ hist_out,
+                                                          const T* __restrict__ emb, const float* __restrict__ s_new_f,
+                                                          int ld_s, T* __restrict__ sprev_t, T* __restrict__ e_t, Dims dm,
+                                                          int32_t* __restrict__ beams_out, float* __restrict__ scores_out) {
+  __shared__ Cand sh[32];
+  __shared__ int sel_parent[64], sel_tok[64];
+  __shared__ float sel_score[64];
+  const int b = blockIdx.x, BW = dm.BW, L = dm.L, V = dm.V;
+  const int rows = call == 1 ? 1 : BW;
+  const int row0 = call == 1 ? b : b * BW;
+  const int n_cand = rows * BW;
+  // candidate c = (row r = c / BW, rank j = c % BW): score and flat index
+  Cand prev{INFINITY, -1};
+  for (int p = 0; p < BW; ++p) {
+    Cand best{-INFINITY, 0x7fffffff};
+    for (int c = threadIdx.x; c < n_cand; c += blockDim.x) {
+      const int r = c / BW;
+      const size_t o = (size_t)(row0 + r) * BW + (c - r * BW);
+      const float base = call == 1 ? 0.f : score_in[row0 + r];
+      const float sc = base + (val[o] - lse[row0 + r]);
+      const int flat = r * V + idx[o];
+      if (cand_before(prev.v, prev.i, sc, flat)) best = cand_best(best, Cand{sc, flat});
+    }
+    best = block_best(best, sh);
+    if (threadIdx.x == 0) {
+      sel_parent[p] = best.i / V;
+      sel_tok[p] = best.i - (best.i / V) * V;
+      sel_score[p] = best.v;
+    }
+    prev = best;
+  }
+  __syncthreads();
+  for (int k = threadIdx.x; k < BW; k += blockDim.x) {
+    const int orow = b * BW + k;
+    score_out[orow] = sel_score[k];
+    const int prow = b * BW + sel_parent[k];
+    for (int t = 0; t < call - 1; ++t) hist_out[(size_t)orow * L + t] = hist_in[(size_t)prow * L + t];
+    hist_out[(size_t)orow * L + call - 1] = sel_tok[k];
+    if (call == L) {
+      for (int t = 0; t < L - 1; ++t) beams_out[(size_t)orow * L + t] = hist_in[(size_t)prow * L + t];
+      beams_out[(size_t)orow * L + L - 1] = sel_tok[k];
+      if (scores_out) scores_out[orow] = sel_score[k];
+    }
+  }
+  if (call < L) {
+    for (int k = 0; k < BW; ++k) {
+      const int orow = b * BW + k;
+      const T* e = emb + (size_t)sel_tok[k] * dm.d;
+      for (int i = threadIdx.x; i < dm.d; i += blockDim.x) e_t[(size_t)orow * dm.d + i] = e[i];
+      if (call > 1) {
+        const float* s = s_new_f + (size_t)(b * BW + sel_parent[k]) * ld_s;
+        for (int i = threadIdx.x; i < dm.dr; i += blockDim.x) sprev_t[(size_t)orow * dm.dr + i] = from_f<T>(s[i]);
+      }
+    }
+  }
+}
+
+cudaError_t launch_beam_merge(int dtype, int call, const float* lse, const float* val, const int32_t* idx,
+                              const float* score_in, float* score_out, const int32_t* hist_in, int32_t* hist_out,
+                              const void* emb, const float* s_new_f, int ld_s, void* sprev_t, void* e_t,
+                              const Dims& dm, int B, int32_t* beams_out, float* scores_out, cudaStream_t st) {
+  RD_DISPATCH(dtype, beam_merge_kernel<T><<<B, 256, 0, st>>>(call, lse, val, idx, score_in, score_out, hist_in, hist_out,
+                                                           (const T*)emb, s_new_f, ld_s, (T*)sprev_t, (T*)e_t, dm,
+                                                           beams_out, scores_out));
+  return cudaGetLastError();
+}
+
+}  // namespace rd

@@ -1,0 +1,114 @@
+// Internal declarations shared by the translation units of libredrafter.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "redrafter.h"
+
+namespace rd {
+
+// ---- device status word bits (OR-ed by kernels, read by redrafter_poll) ----
+enum : int {
+  DEV_ERR_TOKEN_RANGE = 1 << 0,  // a token id outside [0, vocab) was clamped
+  DEV_ERR_INDEX_RANGE = 1 << 1,  // a packed/unpack/slot index outside its range was skipped
+  DEV_ERR_TIMEOUT = 1 << 2,      // a bounded wait (mbarrier) gave up
+  DEV_ERR_CAPACITY = 1 << 3      // a KV slot beyond max_ctx was skipped
+};
+
+// ---- element type helpers ----
+template <typename T> __device__ __forceinline__ float to_f(T v);
+template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float silu_f(float v) { return v / (1.0f + __expf(-v)); }
+
+// Row tables of one forward pass over M rows (device memory).  A row is one token of one
+// sequence; it attends cache slots [0, n_cache) of its sequence plus, when mask != nullptr,
+// the rows (seq_rowbase[seq] + j) whose bit j is set in its mask row (tree attention).
+struct RowTables {
+  const int32_t* tok;         // [M] token id
+  const int32_t* seq;         // [M] sequence index b
+  const int32_t* pos;         // [M] position id (rotary embedding)
+  const int32_t* slot;        // [M] cache slot the row's K/V are written to
+  const int32_t* n_cache;     // [M] number of leading cache slots the row attends
+  const int32_t* local;       // [M] index of the row inside its sequence's group of rows (its mask row)
+  const uint32_t* mask;       // [B][NMAX][MW] tree mask or nullptr (causal: n_cache covers everything)
+  const int32_t* m_total;     // [1] number of valid rows (device)
+};
+
+// Epilogue of every projection: v = acc (+ addend) (+ bias[n]) -> act -> (+ resid) -> out.
+struct Epilogue {
+  const float* addend;   // [M][ld_addend] or nullptr
+  const void* bias;      // [N] in weight dtype or nullptr
+  const float* resid;    // [M][ld_resid] or nullptr (may alias out_f32)
+  float* out_f32;        // [M][ld_out_f32] or nullptr
+  void* out_t;           // [M][ld_out_t] in activation dtype, or nullptr
+  int ld_addend, ld_resid, ld_out_f32, ld_out_t;
+  int silu;              // apply SiLU after bias
+};
+
+struct Dims {
+  int n_layers, d, H, hd, F, V, dr, dh, n_head_layers;
+  int B, max_ctx, BW, L, NMAX, MW;
+  float eps, theta;
+  int dtype;
+};
+
+// ---- launchers (definitions in the .cu files; all enqueue on `st`, return cudaGetLastError) ----
+// Y[m][n] = sum_k A[m][k] W[n][k], M rows given by *m_total (<= m_max), on CUDA cores.
+cudaError_t launch_gemm_simt(int dtype, const void* A, int lda, const void* W, int N, int K, const int32_t* m_total,
+                             int m_max, const Epilogue& ep, cudaStream_t st);
+
+cudaError_t launch_embed(int dtype, const void* emb, const int32_t* tok, float* x, int d, int V, const int32_t* m_total,
+                         int m_max, int* status, cudaStream_t st);
+cudaError_t launch_rmsnorm(int dtype, const float* x, const void* gain, void* out_t, float* out_f32, int d, float eps,
+                           const int32_t* m_total, int m_max, cudaStream_t st);
+cudaError_t launch_rope_kv(int dtype, float* qkv, void* kcache, void* vcache, const RowTables& rt, const Dims& dm,
+                           int m_max, int* status, cudaStream_t st);
+cudaError_t launch_attention(int dtype, const float* qkv, const void* kcache, const void* vcache, void* out_t,
+                             const RowTables& rt, const Dims& dm, int m_max, cudaStream_t st);
+cudaError_t launch_swiglu(int dtype, const float* gu, void* out_t, int F, const int32_t* m_total, int m_max,
+                          cudaStream_t st);
+cudaError_t launch_argmax_rows(const float* logits, int V, int32_t* out, const int32_t* out_index,
+                               const int32_t* m_total, int m_max, cudaStream_t st);
+
+// drafter
+cudaError_t launch_draft_init(int dtype, const void* emb, const int32_t* root, const float* h, void* x_t, float* x_f,
+                              void* sprev_t, const Dims& dm, int B, int* status, cudaStream_t st);
+cudaError_t launch_row_topk(const float* logits, int V, int BW, float* lse, float* val, int32_t* idx, int rows,
+                            cudaStream_t st);
+cudaError_t launch_beam_merge(int dtype, int call, const float* lse, const float* val, const int32_t* idx,
+                              const float* score_in, float* score_out, const int32_t* hist_in, int32_t* hist_out,
+                              const void* emb, const float* s_new_f, int ld_s, void* sprev_t, void* e_t,
+                              const Dims& dm, int B, int32_t* beams_out, float* scores_out, cudaStream_t st);
+cudaError_t launch_fill_h(int dtype, const float* h, void* x_t, float* x_f, const Dims& dm, int B, cudaStream_t st);
+
+// pack / accept
+cudaError_t launch_pack(const int32_t* beams, const int32_t* root, const int32_t* ctx, const rd_packed& out,
+                        const Dims& dm, int B, int no_tree, cudaStream_t st);
+cudaError_t launch_build_rows_tree(const rd_packed& pk, const int32_t* ctx, int32_t* row_tok, int32_t* row_seq,
+                                   int32_t* row_pos, int32_t* row_slot, int32_t* row_ncache, int32_t* row_local,
+                                   int32_t* row_out_index, int32_t* m_total, const Dims& dm, int B, int* status,
+                                   cudaStream_t st);
+cudaError_t launch_build_rows_ar(const int32_t* root, const int32_t* ctx, int32_t* row_tok, int32_t* row_seq,
+                                 int32_t* row_pos, int32_t* row_slot, int32_t* row_ncache, int32_t* row_local,
+                                 int32_t* row_out_index, int32_t* m_total, const Dims& dm, int B, int* status,
+                                 cudaStream_t st);
+cudaError_t launch_scatter_rows(const float* src, int width, float* dst, const int32_t* row_out_index,
+                                const int32_t* m_total, int m_max, cudaStream_t st);
+cudaError_t launch_cast_rows(int dtype, const float* src, void* dst, int n, cudaStream_t st);
+cudaError_t launch_fill_i32(int32_t* p, int32_t v, int n, cudaStream_t st);
+cudaError_t launch_accept(int dtype, const int32_t* beams, const rd_packed& pk, const int32_t* argmax,
+                          const float* hidden, void* kcache, int32_t* ctx, int32_t* root, float* h,
+                          const rd_accept_out& out, int32_t* n_accept_ws, int32_t* best_ws, int32_t* ctx_prev,
+                          const Dims& dm, int B, int* status, cudaStream_t st);
+cudaError_t launch_ar_finish(const int32_t* argmax_c, const float* hidden_c, int32_t* ctx, int32_t* root, float* h,
+                             int32_t* token_out, const Dims& dm, int B, cudaStream_t st);
+cudaError_t launch_prefill_finish(const float* hidden_c, const int32_t* last_row, float* h, int d, int B,
+                                  cudaStream_t st);
+
+}  // namespace rd
