@@ -1,0 +1,406 @@
+"""Benchmark of one ReDrafter speculative decode step on B200 (see the design doc for the contract).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 7b] [--impl ours|reference]
+
+A step is one pass of the whole hot path (draft -> pack -> verify -> accept) for one batch; the
+default workload is the Vicuna-7B-shaped bs1 configuration.  Prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from paper_2403_09919_b200 import synth  # noqa: E402
+
+METRIC = "decode tokens/s (7B-shape, bs1)"
+UNIT = "tokens/s"
+
+
+# --------------------------------------------------------------------------- helpers
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled every 200 ms while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def step_bytes(cfg, ctx, n_rows=None):
+    """Algorithmic bytes one step must read: LLM weights once, drafter weights once per call
+    (head on each of the L calls, RNN on L-1), KV cache of the context once."""
+    es = 4 if cfg["dtype"] == "fp32" else 2
+    d, Fd, V, L = cfg["d_model"], cfg["d_ffn"], cfg["vocab"], cfg["beam_length"]
+    dh = cfg["d_rnn"] + d
+    per_layer = 4 * d * d + 3 * d * Fd
+    llm = cfg["n_layers"] * per_layer + V * d
+    head = cfg["n_head_layers"] * dh * dh + V * dh
+    rnn = cfg["d_rnn"] * (cfg["d_rnn"] + d)
+    kv = cfg["n_layers"] * 2 * d * ctx
+    return dict(llm=llm * es, drafter=(L * head + (L - 1) * rnn) * es, kv=kv * es,
+                total=(llm + L * head + (L - 1) * rnn + kv) * es, ar=(llm + kv) * es)
+
+
+# --------------------------------------------------------------------------- CPU oracle legs
+class OracleSample:
+    """The oracle on a depth-reduced copy of the workload: full per-layer shapes, `sample_layers`
+    layers, fp32 numpy arithmetic.  One step is timed in parts and scaled to the full depth:
+    t_step = t_draft + t_pack + (n_layers / sample_layers) * t_layers + t_lm_head + t_accept."""
+
+    def __init__(self, cfg, sample_layers=2):
+        self.cfg = cfg
+        self.sample_layers = min(sample_layers, cfg["n_layers"])
+        self.c = synth.with_layers(cfg, self.sample_layers)
+        w = synth.make_weights(self.c, "cpu")
+        self.W, self.D = synth.weights_to_numpy(w, self.c)
+
+    def step(self, seed=0):
+        from oracle import redrafter_oracle as ora
+        cfg, c, W, D = self.cfg, self.c, self.W, self.D
+        dt = np.float32
+        BW, L = cfg["beam_width"], cfg["beam_length"]
+        rng = np.random.default_rng(seed)
+        hd = c["d_model"] // c["n_heads"]
+        ctx = cfg["prompt_len"] if isinstance(cfg["prompt_len"], int) else cfg["prompt_len"][1]
+        kv = ora.KVCache(c["n_layers"], ctx + 1 + BW * L, c["n_heads"], hd, dt)
+        kv.k[:, :ctx] = rng.normal(size=kv.k[:, :ctx].shape).astype(dt)      # a filled cache of the right size
+        kv.v[:, :ctx] = rng.normal(size=kv.v[:, :ctx].shape).astype(dt)
+        g = int(rng.integers(0, c["vocab"]))
+        h = rng.normal(size=c["d_model"]).astype(dt)
+        t0 = time.perf_counter()
+        beams, _ = ora.beam_search(D, W["tok_emb"], g, h, BW, L, dt)
+        t1 = time.perf_counter()
+        aug = np.concatenate([np.full((BW, 1), g), beams], axis=1)
+        p = ora.pack_beam(aug, ctx)
+        t2 = time.perf_counter()
+        hidden, _ = ora.llm_forward(W, c, p["tokens"], p["pos"], p["mask"], kv, ctx, dt, want_logits=False)
+        t3 = time.perf_counter()
+        logits = hidden @ W["lm_head"].T
+        am = logits.argmax(1)
+        t4 = time.perf_counter()
+        a, best, emitted = ora.accept_greedy(beams, p["unpack"], am)
+        ora.compact_kv(kv, ctx, p["unpack"], best, a)
+        t5 = time.perf_counter()
+        scale = cfg["n_layers"] / self.sample_layers
+        full = (t1 - t0) + (t2 - t1) + scale * (t3 - t2) + (t4 - t3) + (t5 - t4)
+        return dict(step_s=full, tokens=len(emitted), cpu_s=t5 - t0, rows=int(p["n"]))
+
+    def run(self, steps, warmup=0):
+        for s in range(warmup):
+            self.step(1000 + s)
+        tot_s, tot_tok, cpu_s, rows = 0.0, 0, 0.0, 0
+        for s in range(steps):
+            r = self.step(s)
+            tot_s += r["step_s"]; tot_tok += r["tokens"]; cpu_s += r["cpu_s"]; rows += r["rows"]
+        sample = (f"{steps} oracle steps on a {self.sample_layers}-layer copy of the workload at full per-layer shapes "
+                  f"(fp32 numpy, filled cache of {self.cfg['prompt_len']} tokens, drafter's own beams, mean {rows / steps:.0f} "
+                  f"packed rows); the layer time is scaled by n_layers/{self.sample_layers}; {cpu_s:.1f} s of CPU work")
+        return dict(value=tot_tok / tot_s, ms_per_step=1e3 * tot_s / steps, sample=sample)
+
+
+def cpu_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, cfg):
+    """--impl reference: the oracle, as it stands, on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = max(1, min(args.steps, args.reference_max_steps))
+    r = OracleSample(cfg, args.oracle_layers).run(steps, warmup=min(args.warmup, 1))
+    value, sample = r["value"], r["sample"]
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+            "warmup": min(args.warmup, 1), "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": workload_config(args, cfg),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_cores(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def workload_config(args, cfg):
+    return {"workload": f"{args.workload}: {cfg['n_layers']} layers d={cfg['d_model']} heads={cfg['n_heads']} ffn={cfg['d_ffn']} "
+                        f"vocab={cfg['vocab']} {cfg['dtype']}, batch {cfg['max_batch']}, prompt {cfg['prompt_len']} uniform-random "
+                        f"tokens, beam width {cfg['beam_width']}, beam length {cfg['beam_length']}, greedy acceptance, random-init weights",
+            "beams": "drafter's own (random-init drafter and LLM are uncorrelated: about 1 token per step by construction)",
+            "l2": "inputs larger than L2: every step streams all weights (>= 13 GB at 7B) so nothing is reused from the 126 MB L2",
+            "parallelism": "replicas only (no collective)"}
+
+
+# --------------------------------------------------------------------------- GPU legs
+def timed_loop(eng, n, fn):
+    """n calls of fn between two events on the current stream; returns ms."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(n):
+        fn(i)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="7b", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--layers", type=int, default=0, help="depth-reduced run (0 = the workload's depth)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--oracle-layers", type=int, default=2)
+    ap.add_argument("--reference-max-steps", type=int, default=8)
+    ap.add_argument("--cpu-steps", type=int, default=6)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the planted-beam and autoregressive comparison legs")
+    args = ap.parse_args()
+    cfg = dict(synth.CONFIGS[args.workload])
+    if args.layers:
+        cfg = synth.with_layers(cfg, args.layers)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    device = f"cuda:{local_rank}"
+    torch.cuda.set_device(device)
+    from paper_2403_09919_b200 import binding
+
+    B, BW, L = cfg["max_batch"], cfg["beam_width"], cfg["beam_length"]
+    need = args.warmup + args.steps
+    cfg["max_ctx"] = max(cfg["max_ctx"], (cfg["prompt_len"] if isinstance(cfg["prompt_len"], int) else cfg["prompt_len"][1])
+                         + need * (L + 1) + 2 + BW * L)
+    w = synth.make_weights(cfg, device)
+    eng = binding.ReDrafter(cfg, w, device=device)
+    prompts = synth.make_prompts(cfg, B, seed=cfg.get("seed", 0) + 100 * rank)
+    out = binding.AcceptOut(B, L, device)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+
+    # ---- main leg: K steps, inputs resident in HBM, no host sync inside
+    eng.prefill(prompts)
+    for _ in range(args.warmup):
+        eng.step(None, out)
+    eng.poll()
+    n_acc = torch.zeros(args.steps, B, dtype=torch.int32, device=device)
+    launches0 = eng.launch_count()
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+
+    def one(i):
+        eng.step(None, out)
+        n_acc[i].copy_(out.n_accept)
+    ms = timed_loop(eng, args.steps, one)
+    clocks = sampler.stop()
+    launches = eng.launch_count() - launches0
+    barrier()
+    eng.poll()
+    tokens = int(n_acc.sum().item()) + args.steps * B
+    ctx_end, _, _ = eng.get_state()
+    ctx_mid = float(ctx_end.float().mean().item()) - 0.5 * tokens / B
+    if dist is not None:
+        t = torch.tensor([ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+        tk = torch.tensor([tokens], device=device, dtype=torch.int64)
+        dist.all_reduce(tk)
+        tokens = int(tk.item())
+    value = tokens / (ms * 1e-3)
+    ms_per_step = ms / args.steps
+
+    # ---- e2e leg: the same steps driven the way a serving loop does, results read to the host each step
+    pin_a = torch.zeros(B, dtype=torch.int32).pin_memory()
+    pin_t = torch.zeros(B, L + 1, dtype=torch.int32).pin_memory()
+    e2e_tokens = [0]
+
+    def one_e2e(i):
+        eng.step(None, out)
+        pin_a.copy_(out.n_accept, non_blocking=True)
+        pin_t.copy_(out.tokens, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        e2e_tokens[0] += int(pin_a.sum()) + B
+    eng.prefill(prompts)
+    for _ in range(args.warmup):
+        eng.step(None, out)
+    barrier()
+    ms_e2e = timed_loop(eng, args.steps, one_e2e)
+    if dist is not None:
+        t = torch.tensor([ms_e2e], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+        tk = torch.tensor([e2e_tokens[0]], device=device, dtype=torch.int64)
+        dist.all_reduce(tk)
+        e2e_tokens[0] = int(tk.item())
+    e2e = {"value": e2e_tokens[0] / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 0,
+           "d2h_bytes_per_step": int(B * (L + 2) * 4), "ms_per_step": ms_e2e / args.steps,
+           "note": "redrafter_step through the C ABI; the accepted tokens are copied to pinned host memory and the stream "
+                   "is synchronised every step; a step has no host-side input (state, KV cache and weights are device "
+                   "resident by design; the prompt's H2D copy happens in redrafter_prefill, outside the decode loop)"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if cfg["dtype"] == "bf16" else "f32", "data": "synthetic", "config": workload_config(args, cfg),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+            "tokens_per_step": tokens / (args.steps * B * world)}
+
+    if rank == 0:
+        # ---- roofline of the dominant kernel (the weight-streaming projection), timed per launch with CUDA events
+        peak, peak_src = measured_peaks()
+        prof_steps = min(8, args.steps)
+        eng.prefill(prompts)
+        for _ in range(args.warmup):
+            eng.step(None, out)
+        eng.profile(True)
+        for _ in range(prof_steps):
+            eng.step(None, out)
+            gm = eng.profile_read(0)
+            at = eng.profile_read(1)
+        eng.profile(False)
+        g_ms, g_bytes, g_n = gm
+        achieved = g_bytes / (g_ms * 1e-3) / 1e9 if g_ms > 0 else 0.0
+        sb = step_bytes(cfg, ctx_mid)
+        line["roofline"] = {"bound": "hbm", "kernel": "projection (weight-streaming GEMM)", "achieved": achieved, "peak": peak,
+                            "unit": "GB/s", "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
+                            "launches_per_step": g_n / prof_steps, "ms_per_step_in_kernel": g_ms / prof_steps,
+                            "attention_ms_per_step": at[0] / prof_steps}
+        line["step_roofline"] = {"algorithmic_bytes_per_step": sb["total"], "achieved_gbs": sb["total"] / (ms_per_step * 1e-3) / 1e9,
+                                 "frac_of_measured_peak": sb["total"] / (ms_per_step * 1e-3) / 1e9 / peak,
+                                 "frac_of_nominal_8tbs": sb["total"] / (ms_per_step * 1e-3) / 8e12,
+                                 "mean_ctx": ctx_mid, "bytes": sb}
+        if not args.no_extras:
+            # ---- autoregressive comparator built from the same kernels, and the planted-beam mode
+            n_ar = need * (L + 1) + 1
+            eng.prefill(prompts)
+            tok = torch.zeros(B, dtype=torch.int32, device=device)
+            _, root, _ = eng.get_state()
+            cont = torch.zeros(n_ar + 1, B, dtype=torch.int32, device=device)
+            cont[0].copy_(root)
+            for _ in range(args.warmup):
+                eng.ar_step(tok)
+            eng.prefill(prompts)
+
+            def one_ar(i):
+                eng.ar_step(tok)
+                cont[i + 1].copy_(tok)
+            ms_ar = timed_loop(eng, n_ar, one_ar)
+            eng.poll()
+            line["autoregressive"] = {"tokens_per_s": n_ar * B / (ms_ar * 1e-3), "ms_per_step": ms_ar / n_ar,
+                                      "frac_of_measured_peak": sb["ar"] / (ms_ar / n_ar * 1e-3) / 1e9 / peak}
+            cont_h = cont.cpu().numpy()                                   # [n_ar+1, B]; row 0 = root after prefill
+            rng = np.random.default_rng(2000 + cfg.get("seed", 0))
+            planted = np.zeros((need, B, BW, L), dtype=np.int32)
+            posn = np.ones(B, dtype=np.int64)
+            exp_acc = np.zeros((need, B), dtype=np.int64)
+            for s in range(need):
+                for b in range(B):
+                    c = cont_h[posn[b]:posn[b] + L, b]
+                    planted[s, b] = synth.plant_beams(c, BW, L, cfg["vocab"], rng, p=cfg.get("plant_p", 0.3),
+                                                      rho=cfg.get("plant_rho", 0.0))
+                    exp_acc[s, b] = synth.first_mismatch(planted[s, b], c).max()
+                    posn[b] += exp_acc[s, b] + 1
+            planted_d = torch.from_numpy(planted).to(device)
+            eng.prefill(prompts)
+            for s in range(args.warmup):
+                eng.step(planted_d[s], out)
+            acc_p = torch.zeros(args.steps, B, dtype=torch.int32, device=device)
+
+            def one_p(i):
+                eng.step(planted_d[args.warmup + i], out)
+                acc_p[i].copy_(out.n_accept)
+            ms_p = timed_loop(eng, args.steps, one_p)
+            eng.poll()
+            tok_p = int(acc_p.sum().item()) + args.steps * B
+            line["planted"] = {"tokens_per_s": tok_p / (ms_p * 1e-3), "ms_per_step": ms_p / args.steps,
+                               "tokens_per_step": tok_p / (args.steps * B),
+                               "matches_closed_form": bool((acc_p.cpu().numpy() == exp_acc[args.warmup:]).all()),
+                               "speedup_vs_autoregressive": (tok_p / ms_p) / (n_ar * B / ms_ar),
+                               "note": "beams = the LLM's own greedy continuation with each token replaced at p=0.3"}
+            line["speedup_vs_autoregressive"] = value / world / (n_ar * B / (ms_ar * 1e-3))
+        if not args.no_cpu_baseline and world == 1:
+            r = OracleSample(cfg, args.oracle_layers).run(args.cpu_steps, warmup=1)
+            line["cpu_baseline"] = {"value": r["value"], "unit": UNIT, "cores": cpu_cores(), "kind": "oracle",
+                                    "ms_per_step": r["ms_per_step"], "sample": r["sample"]}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -24,7 +24,8 @@ STATUS = {0: "RD_OK", 1: "RD_ERR_INVALID_ARG", 2: "RD_ERR_SHAPE", 3: "RD_ERR_CAP
 EXPORTS = ["redrafter_workspace_bytes", "redrafter_kv_bytes", "redrafter_init", "redrafter_destroy",
            "redrafter_last_error", "redrafter_prefill", "redrafter_draft", "redrafter_pack", "redrafter_verify",
            "redrafter_accept", "redrafter_step", "redrafter_ar_step", "redrafter_get_state", "redrafter_set_state",
-           "redrafter_set_ctx_bound", "redrafter_poll", "redrafter_launch_count"]
+           "redrafter_set_ctx_bound", "redrafter_poll", "redrafter_launch_count", "redrafter_profile",
+           "redrafter_profile_read"]
 
 
 class RdConfig(C.Structure):
@@ -81,6 +82,9 @@ def lib():
         L.redrafter_poll.argtypes = [vp, vp]
         L.redrafter_launch_count.restype = C.c_int64
         L.redrafter_launch_count.argtypes = [vp]
+        L.redrafter_profile.argtypes = [vp, C.c_int]
+        L.redrafter_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                             C.POINTER(C.c_int64)]
         _lib = L
     return _lib
 
@@ -269,6 +273,15 @@ class ReDrafter:
 
     def poll(self):
         self._ck(self.L.redrafter_poll(self.h, _stream()))
+
+    def profile(self, enable):
+        self._ck(self.L.redrafter_profile(self.h, 1 if enable else 0))
+
+    def profile_read(self, cls):
+        """(ms, bytes, launches) summed since profile(True) for class 0 (projections) or 1 (attention)."""
+        ms, by, n = C.c_double(), C.c_double(), C.c_int64()
+        self._ck(self.L.redrafter_profile_read(self.h, cls, C.byref(ms), C.byref(by), C.byref(n)))
+        return ms.value, by.value, n.value
 
     def launch_count(self):
         return int(self.L.redrafter_launch_count(self.h))

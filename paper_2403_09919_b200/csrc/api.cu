@@ -62,6 +62,12 @@ struct rd_handle {
   int batch;      // active sequences
   int ctx_bound;  // host-side upper bound of every sequence's context length
   int64_t launches;
+  // optional per-launch timing of the projections (class 0) and the attention kernel (class 1)
+  bool profiling;
+  std::vector<cudaEvent_t> ev[2];   // start/stop pairs
+  size_t ev_used[2];
+  double prof_ms[2], prof_bytes[2];
+  int64_t prof_n[2];
   char err[512];
 };
 
@@ -157,6 +163,28 @@ void carve(Bump& bp, const Dims& dm, int m_cap, Workspace* w) {
     if (e__ != cudaSuccess) return fail(h, RD_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e__)); \
   } while (0)
 
+// Event pair around one launch when profiling is on (cudaEventCreate happens on first use only).
+struct ProfScope {
+  rd_handle* h; int cls; cudaStream_t st; bool on;
+  ProfScope(rd_handle* h_, int cls_, double bytes, cudaStream_t st_) : h(h_), cls(cls_), st(st_), on(h_->profiling) {
+    if (!on) return;
+    auto& v = h->ev[cls];
+    if (h->ev_used[cls] + 2 > v.size()) {
+      cudaEvent_t a, b;
+      if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { on = false; return; }
+      v.push_back(a); v.push_back(b);
+    }
+    cudaEventRecord(v[h->ev_used[cls]], st);
+    h->prof_bytes[cls] += bytes;
+    h->prof_n[cls]++;
+  }
+  ~ProfScope() {
+    if (!on) return;
+    cudaEventRecord(h->ev[cls][h->ev_used[cls] + 1], st);
+    h->ev_used[cls] += 2;
+  }
+};
+
 Epilogue ep_store(float* out, int ld) {
   Epilogue e{};
   e.out_f32 = out; e.ld_out_f32 = ld;
@@ -166,6 +194,7 @@ Epilogue ep_store(float* out, int ld) {
 // One projection; picks the kernel.
 int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, const int32_t* m_total, int m_max,
          const Epilogue& ep, cudaStream_t st) {
+  ProfScope ps(h, 0, (double)N * K * esize(h->dm.dtype), st);
   CK(h, launch_gemm_simt(h->dm.dtype, A, lda, W, N, K, m_total, m_max, ep, st));
   return RD_OK;
 }
@@ -186,7 +215,10 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, cudaStream_t s
     int rc = gemm(h, w.a_t, dm.d, h->wqkv[l], 3 * dm.d, dm.d, w.m_total, m_max, ep_store(w.qkv, 3 * dm.d), st);
     if (rc) return rc;
     CK(h, launch_rope_kv(dm.dtype, w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), rt, dm, m_max, w.status, st));
-    CK(h, launch_attention(dm.dtype, w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.attn_t, rt, dm, m_max, st));
+    {
+      ProfScope ps(h, 1, 0.0, st);
+      CK(h, launch_attention(dm.dtype, w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.attn_t, rt, dm, m_max, st));
+    }
     Epilogue eo{};
     eo.resid = w.x; eo.ld_resid = dm.d; eo.out_f32 = w.x; eo.ld_out_f32 = dm.d;
     rc = gemm(h, w.attn_t, dm.d, h->wo[l], dm.d, dm.d, w.m_total, m_max, eo, st);
@@ -325,6 +357,8 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
   Bump bp{(char*)workspace, 0};
   carve(bp, dm, h->m_cap, &h->ws);
   h->prefilled = false; h->batch = dm.B; h->ctx_bound = 0; h->launches = 0; h->err[0] = 0;
+  h->profiling = false;
+  for (int c = 0; c < 2; ++c) { h->ev_used[c] = 0; h->prof_ms[c] = 0; h->prof_bytes[c] = 0; h->prof_n[c] = 0; }
   // clear the state and the constants the kernels read from device memory
   cudaError_t e = cudaMemsetAsync(workspace, 0, (size_t)((char*)h->ws.x - (char*)workspace), 0);
   if (e == cudaSuccess) e = cudaStreamSynchronize(0);
@@ -335,6 +369,8 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
 
 int redrafter_destroy(rd_handle* h) {
   if (!h) return RD_ERR_INVALID_ARG;
+  for (int c = 0; c < 2; ++c)
+    for (cudaEvent_t e : h->ev[c]) cudaEventDestroy(e);
   delete h;
   return RD_OK;
 }
@@ -518,6 +554,31 @@ int redrafter_set_state(rd_handle* h, void* stream, const int32_t* ctx, const in
 int redrafter_set_ctx_bound(rd_handle* h, int32_t max_ctx_now) {
   if (!h || max_ctx_now < 0) return RD_ERR_INVALID_ARG;
   h->ctx_bound = max_ctx_now;
+  return RD_OK;
+}
+
+int redrafter_profile(rd_handle* h, int enable) {
+  if (!h) return RD_ERR_INVALID_ARG;
+  h->profiling = enable != 0;
+  if (enable)
+    for (int c = 0; c < 2; ++c) { h->ev_used[c] = 0; h->prof_ms[c] = 0; h->prof_bytes[c] = 0; h->prof_n[c] = 0; }
+  return RD_OK;
+}
+
+int redrafter_profile_read(rd_handle* h, int32_t cls, double* ms, double* bytes, int64_t* launches) {
+  if (!h || cls < 0 || cls > 1) return RD_ERR_INVALID_ARG;
+  double total = h->prof_ms[cls];
+  for (size_t i = 0; i + 1 < h->ev_used[cls]; i += 2) {
+    CKRT(h, cudaEventSynchronize(h->ev[cls][i + 1]));
+    float t = 0.f;
+    CKRT(h, cudaEventElapsedTime(&t, h->ev[cls][i], h->ev[cls][i + 1]));
+    total += t;
+  }
+  h->prof_ms[cls] = total;
+  h->ev_used[cls] = 0;
+  if (ms) *ms = total;
+  if (bytes) *bytes = h->prof_bytes[cls];
+  if (launches) *launches = h->prof_n[cls];
   return RD_OK;
 }
 
