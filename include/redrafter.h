@@ -124,7 +124,8 @@ RD_API int redrafter_init(const rd_config* cfg, const rd_weights* weights, void*
 /* Free the host-side handle.  Does not touch device memory. */
 RD_API int redrafter_destroy(rd_handle* h);
 
-/* Message of the last failing call on this handle (host string, valid until the next call). */
+/* Message of the last failing call on this handle (host string, valid until the next call).
+ * With h == NULL: why the last redrafter_init failed. */
 RD_API const char* redrafter_last_error(const rd_handle* h);
 
 /* Causal forward over the prompts (the state before the first step, Figure 2): fills the KV

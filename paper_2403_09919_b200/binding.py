@@ -190,7 +190,7 @@ class ReDrafter:
         rc = self.L.redrafter_init(C.byref(self.c_cfg), C.byref(w), self.kv.data_ptr(), kv_bytes,
                                    self.workspace.data_ptr(), ws_bytes, C.byref(hp))
         if rc:
-            raise RdError(rc, "redrafter_init failed")
+            raise RdError(rc, "redrafter_init failed: " + self.L.redrafter_last_error(None).decode())
         self.h = hp
         self.B = cfg["max_batch"]
         self.BW, self.Lb, self.d, self.V = cfg["beam_width"], cfg["beam_length"], cfg["d_model"], cfg["vocab"]

@@ -6,6 +6,7 @@
 #include <string.h>
 
 #include <new>
+#include <unordered_map>
 #include <vector>
 
 #include "rd_internal.cuh"
@@ -43,9 +44,16 @@ struct Workspace {
   void *xc_t, *x0_t, *x1_t, *x2_t, *sprev_t, *e_t;
   float *xc_f, *x0_f, *x1_f, *x2_f, *tmp_f, *dlogits, *lse, *cand_val, *score_a, *score_b;
   int32_t *cand_idx, *hist_a, *hist_b, *one_b, *one_r;
+  // tensor-core projection scratch
+  int32_t* tc_counters;
+  float* tc_partial;
 };
 
 size_t esize(int dtype) { return dtype == RD_DTYPE_FP32 ? 4 : 2; }
+
+struct alignas(64) TensorMapBox {  // opaque storage of one CUtensorMap (128 bytes)
+  unsigned char bytes[128];
+};
 
 }  // namespace
 
@@ -62,6 +70,10 @@ struct rd_handle {
   int batch;      // active sequences
   int ctx_bound;  // host-side upper bound of every sequence's context length
   int64_t launches;
+  // tensor-core path (bf16): TMA descriptors by base pointer, launch geometry
+  bool use_tc;
+  int tc_grid, tc_smem;
+  std::unordered_map<const void*, TensorMapBox> maps;
   // optional per-launch timing of the projections (class 0) and the attention kernel (class 1)
   bool profiling;
   std::vector<cudaEvent_t> ev[2];   // start/stop pairs
@@ -72,6 +84,17 @@ struct rd_handle {
 };
 
 namespace {
+
+char g_init_err[512] = "";  // why the last redrafter_init failed (there is no handle to hold it)
+
+int init_fail(rd_handle* h, int code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_init_err, sizeof(g_init_err), fmt, ap);
+  va_end(ap);
+  delete h;
+  return code;
+}
 
 int fail(rd_handle* h, int code, const char* fmt, ...) {
   if (h) {
@@ -107,6 +130,8 @@ int shape_ok(const Dims& dm) {
   return 1;
 }
 
+constexpr int TC_MAX_GRID = 160;  // upper bound of the SM count the scratch is sized for
+
 int m_cap_of(const Dims& dm) {
   const int v = dm.B * dm.NMAX;
   return v > 256 ? v : 256;
@@ -120,6 +145,14 @@ void carve(Bump& bp, const Dims& dm, int m_cap, Workspace* w) {
   w->row_tok = bp.take<int32_t>(m_cap); w->row_seq = bp.take<int32_t>(m_cap); w->row_pos = bp.take<int32_t>(m_cap);
   w->row_slot = bp.take<int32_t>(m_cap); w->row_ncache = bp.take<int32_t>(m_cap); w->row_local = bp.take<int32_t>(m_cap);
   w->row_out_index = bp.take<int32_t>(m_cap); w->m_total = bp.take<int32_t>(4); w->last_row = bp.take<int32_t>(B);
+  w->one_b = bp.take<int32_t>(4); w->one_r = bp.take<int32_t>(4);
+  {
+    int max_n = 3 * dm.d;
+    if (2 * dm.F > max_n) max_n = 2 * dm.F;
+    if (dm.V > max_n) max_n = dm.V;
+    if (dm.dh > max_n) max_n = dm.dh;
+    w->tc_counters = bp.take<int32_t>(tc_counter_ints(max_n, m_cap));
+  }
   w->x = bp.take<float>((size_t)m_cap * dm.d);
   w->qkv = bp.take<float>((size_t)m_cap * 3 * dm.d);
   w->gu = bp.take<float>((size_t)m_cap * 2 * dm.F);
@@ -147,7 +180,8 @@ void carve(Bump& bp, const Dims& dm, int m_cap, Workspace* w) {
   w->lse = bp.take<float>(R); w->cand_val = bp.take<float>((size_t)R * dm.BW);
   w->score_a = bp.take<float>(R); w->score_b = bp.take<float>(R);
   w->cand_idx = bp.take<int32_t>((size_t)R * dm.BW); w->hist_a = bp.take<int32_t>((size_t)R * dm.L);
-  w->hist_b = bp.take<int32_t>((size_t)R * dm.L); w->one_b = bp.take<int32_t>(4); w->one_r = bp.take<int32_t>(4);
+  w->hist_b = bp.take<int32_t>((size_t)R * dm.L);
+  w->tc_partial = bp.take<float>(dm.dtype == RD_DTYPE_BF16 ? tc_partial_floats(TC_MAX_GRID, tc_pick_mt(m_cap)) : 0);
   bp.take<char>(256);
 }
 
@@ -195,6 +229,14 @@ Epilogue ep_store(float* out, int ld) {
 int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, const int32_t* m_total, int m_max,
          const Epilogue& ep, cudaStream_t st) {
   ProfScope ps(h, 0, (double)N * K * esize(h->dm.dtype), st);
+  if (h->use_tc) {
+    auto ia = h->maps.find(A), iw = h->maps.find(W);
+    if (ia == h->maps.end() || iw == h->maps.end() || lda != K)
+      return fail(h, RD_ERR_STATE, "projection operand without a TMA descriptor");
+    CK(h, launch_gemm_tc(&iw->second, &ia->second, N, K, m_total, m_max, ep, h->ws.tc_partial, h->ws.tc_counters,
+                         h->ws.status, h->tc_grid, h->tc_smem, st));
+    return RD_OK;
+  }
   CK(h, launch_gemm_simt(h->dm.dtype, A, lda, W, N, K, m_total, m_max, ep, st));
   return RD_OK;
 }
@@ -356,6 +398,44 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
   }
   Bump bp{(char*)workspace, 0};
   carve(bp, dm, h->m_cap, &h->ws);
+  h->use_tc = dm.dtype == RD_DTYPE_BF16 && !(cfg->flags & RD_FLAG_FORCE_SIMT);
+  if (h->use_tc) {
+    int dev = 0, sms = 0;
+    cudaError_t ce = cudaGetDevice(&dev);
+    if (ce == cudaSuccess) ce = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (ce == cudaSuccess) ce = tc_prepare(&h->tc_smem);
+    if (ce != cudaSuccess || sms <= 0)
+      return init_fail(h, RD_ERR_CUDA, "tensor-core path set-up: %s", cudaGetErrorString(ce));
+    h->tc_grid = sms < TC_MAX_GRID ? sms : TC_MAX_GRID;
+    if (dm.d % 8 || dm.F % 8 || dm.dh % 8) return init_fail(h, RD_ERR_SHAPE, "bf16 needs d_model, d_ffn multiples of 8");
+    bool ok = true;
+    int failed_rc = 0;
+    const void* failed_ptr = nullptr;
+    auto add_w = [&](const void* p, int N, int K) {
+      if (!ok) return;
+      failed_rc = tc_make_map(&h->maps[p], p, (uint64_t)N, (uint64_t)K, (uint32_t)tc_weight_box_rows());
+      if (failed_rc) { ok = false; failed_ptr = p; }
+    };
+    auto add_a = [&](const void* p, int rows, int K) {
+      if (!ok) return;
+      failed_rc = tc_make_map(&h->maps[p], p, (uint64_t)rows, (uint64_t)K, (uint32_t)tc_act_box_rows());
+      if (failed_rc) { ok = false; failed_ptr = p; }
+    };
+    for (int l = 0; l < dm.n_layers; ++l) {
+      add_w(h->wqkv[l], 3 * dm.d, dm.d); add_w(h->wo[l], dm.d, dm.d);
+      add_w(h->w_gate_up[l], 2 * dm.F, dm.d); add_w(h->w_down[l], dm.d, dm.F);
+    }
+    add_w(wt->lm_head, dm.V, dm.d); add_w(wt->rnn_u, dm.dr, dm.dr); add_w(wt->rnn_w, dm.dr, dm.d);
+    for (int l = 0; l < dm.n_head_layers; ++l) add_w(h->head_w[l], dm.dh, dm.dh);
+    add_w(wt->draft_out, dm.V, dm.dh);
+    const Workspace& w = h->ws;
+    const int R = dm.B * dm.BW;
+    add_a(w.a_t, h->m_cap, dm.d); add_a(w.attn_t, h->m_cap, dm.d); add_a(w.act_t, h->m_cap, dm.F);
+    add_a(w.hidden_t, h->m_cap, dm.d); add_a(w.h_t, dm.B, dm.d);
+    add_a(w.xc_t, dm.B, dm.dh); add_a(w.x0_t, R, dm.dh); add_a(w.x1_t, R, dm.dh); add_a(w.x2_t, R, dm.dh);
+    add_a(w.sprev_t, R, dm.dr); add_a(w.e_t, R, dm.d);
+    if (!ok) return init_fail(h, RD_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d for operand %p", failed_rc, failed_ptr);
+  }
   h->prefilled = false; h->batch = dm.B; h->ctx_bound = 0; h->launches = 0; h->err[0] = 0;
   h->profiling = false;
   for (int c = 0; c < 2; ++c) { h->ev_used[c] = 0; h->prof_ms[c] = 0; h->prof_bytes[c] = 0; h->prof_n[c] = 0; }
@@ -375,7 +455,7 @@ int redrafter_destroy(rd_handle* h) {
   return RD_OK;
 }
 
-const char* redrafter_last_error(const rd_handle* h) { return h ? h->err : "null handle"; }
+const char* redrafter_last_error(const rd_handle* h) { return h ? h->err : g_init_err; }
 
 int64_t redrafter_launch_count(const rd_handle* h) { return h ? h->launches : 0; }
 

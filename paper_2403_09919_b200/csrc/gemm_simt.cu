@@ -6,6 +6,7 @@
 // stream: one warp owns one weight row, reads it once with 128-bit loads and keeps MT running
 // sums, so the weight is read exactly once per MT rows.
 #include "rd_internal.cuh"
+#include "epilogue.cuh"
 
 namespace rd {
 
@@ -38,16 +39,6 @@ template <> struct Vec<__nv_bfloat16> {
     unpack(__ldcs(reinterpret_cast<const uint4*>(p)), v);
   }
 };
-
-template <typename T>
-__device__ __forceinline__ void apply_epilogue(const Epilogue& ep, int m, int n, float v) {
-  if (ep.addend) v += ep.addend[(size_t)m * ep.ld_addend + n];
-  if (ep.bias) v += to_f<T>(reinterpret_cast<const T*>(ep.bias)[n]);
-  if (ep.silu) v = silu_f(v);
-  if (ep.resid) v += ep.resid[(size_t)m * ep.ld_resid + n];
-  if (ep.out_f32) ep.out_f32[(size_t)m * ep.ld_out_f32 + n] = v;
-  if (ep.out_t) reinterpret_cast<T*>(ep.out_t)[(size_t)m * ep.ld_out_t + n] = from_f<T>(v);
-}
 
 // grid (ceil(N / 8), ceil(m_max / MT)), block 256 = 8 warps, one weight row per warp.
 template <typename T, int MT>

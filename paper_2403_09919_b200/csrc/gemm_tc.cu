@@ -1,0 +1,427 @@
+// Weight-streaming projection on the 5th-generation tensor cores (tcgen05 + TMEM + TMA), bf16.
+//
+//   Y[m][n] = sum_k A[m][k] W[n][k]        A: [M][K] activations, W: [N][K] weights, both K-major
+//
+// At decode time M (packed tokens x batch) is small and the projection is bound by the weight
+// stream, so the operands are swapped: the WEIGHT tile is the 128-row MMA "A" operand and the
+// activations are the MMA "B" operand, N_mma = MT rows (a multiple of 16, at most 256).  The
+// accumulator D[n][m] lives in TMEM: lane = weight row, column = activation row.
+//
+// Schedule: persistent, one CTA per SM, stream-K.  The work is the list of (tile, k-block) units,
+// tile = (128 weight rows) x (MT activation rows), k-block = 64 columns; CTA c owns the contiguous
+// unit range [c*U/G, (c+1)*U/G), so every SM streams the same number of weight bytes whatever the
+// shape.  A CTA whose range cuts a tile writes its fp32 partial to scratch; the last contributor
+// of that tile (found with an atomic counter, never by waiting) adds the partials in CTA order --
+// a fixed order, so results are deterministic -- and applies the epilogue.
+//
+// Roles: warp 0 = TMA producer (weights 128x64 per stage, activations MT x 64 as 16-row boxes),
+// warp 1 = MMA issuer and TMEM owner, warps 2..5 = epilogue (tcgen05.ld, one TMEM lane quarter
+// each).  Two TMEM accumulators alternate so the epilogue of one segment overlaps the MMAs of the
+// next; the smem ring (full/empty mbarriers) never drains between tiles.
+//
+// Every mbarrier wait is bounded (one second); on expiry the CTA raises DEV_ERR_TIMEOUT in the
+// status word, lets its copies land, frees its TMEM and exits; later launches see the flag and
+// return at once.
+#include <cuda.h>
+
+#include "epilogue.cuh"
+#include "rd_internal.cuh"
+
+namespace rd {
+
+namespace {
+
+constexpr int TILE_N = 128;       // weight rows per tile (MMA M)
+constexpr int TILE_K = 64;        // bf16 per k-block = one 128-byte swizzle row
+constexpr int W_STAGE_BYTES = TILE_N * TILE_K * 2;
+constexpr int A_BOX_ROWS = 16;
+constexpr int A_BOX_BYTES = A_BOX_ROWS * TILE_K * 2;
+constexpr int NUM_THREADS = 192;
+constexpr unsigned long long WAIT_LIMIT_NS = 1000000000ull;
+
+struct TcParams {
+  int N, K, nkb, n_tiles, mt, m_tiles_max, stages, tmem_cols;
+  const int32_t* m_total;
+  float* partial;     // [2 * gridDim.x][mt * 128]
+  int32_t* counters;  // [n_tiles * m_tiles_max], zero between launches
+  int32_t* status;
+  Epilogue ep;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ unsigned long long globaltimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded wait.  Returns false when the CTA is aborting (this or another role gave up).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try(bar, parity)) return true;
+    if ((it & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (globaltimer() - t0 > WAIT_LIMIT_NS) {
+        *abort_flag = 1;
+        atomicOr(status, DEV_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+      "l"(map), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows of 128 bytes, 8-row groups
+// 1024 bytes apart (stride byte offset), descriptor version 1 (sm_100), leading offset unused (1).
+__device__ __forceinline__ uint64_t umma_desc(uint32_t addr) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// Unit range of CTA c: [c*U/G, (c+1)*U/G).
+__device__ __forceinline__ long long range_begin(long long c, long long U, long long G) { return c * U / G; }
+// The CTA whose range holds unit u (the largest c with range_begin(c) <= u).
+__device__ __forceinline__ int cta_of_unit(long long u, long long U, long long G) {
+  long long c = ((u + 1) * G - 1) / U;
+  return (int)(c > G - 1 ? G - 1 : c);
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
+                                                                 const __grid_constant__ CUtensorMap map_a,
+                                                                 const TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  // leave at once when an earlier launch already timed out; one thread reads the flag so that the
+  // whole CTA takes the same branch
+  __shared__ int skip_launch;
+  if (threadIdx.x == 0) skip_launch = (*(volatile int32_t*)p.status & DEV_ERR_TIMEOUT) ? 1 : 0;
+  __syncthreads();
+  if (skip_launch) return;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int M = *p.m_total;
+  const int m_tiles = (M + p.mt - 1) / p.mt;
+  const long long G = gridDim.x;
+  const long long U = (long long)p.n_tiles * m_tiles * p.nkb;
+  const long long u0 = range_begin(blockIdx.x, U, G), u1 = range_begin(blockIdx.x + 1, U, G);
+
+  // ---- shared memory carve-up (stage buffers 1024-byte aligned for the 128-byte swizzle)
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  const uint32_t a_stage_bytes = (uint32_t)p.mt * TILE_K * 2;
+  const uint32_t stage_bytes = W_STAGE_BYTES + a_stage_bytes;
+  const uint32_t bar_base = base + p.stages * stage_bytes;  // 8-byte aligned
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (p.stages + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * p.stages + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * p.stages + 2 + a); };
+  uint8_t* misc = smem_raw + (bar_base - raw) + 8u * (2 * p.stages + 4);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
+  volatile int* last_flag = reinterpret_cast<volatile int*>(misc + 8);
+  volatile int* epi_ok = reinterpret_cast<volatile int*>(misc + 12);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
+    *abort_flag = 0;
+    *last_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
+                 "r"((uint32_t)p.tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ===================== TMA producer =====================
+    if (lane == 0 && u0 < u1) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (long long u = u0; u < u1 && ok;) {
+        const int t = (int)(u / p.nkb), kb0 = (int)(u - (long long)t * p.nkb);
+        const int kb1 = (int)min((long long)p.nkb, kb0 + (u1 - u));
+        const int n_tile = t / m_tiles, m_tile = t - n_tile * m_tiles;
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
+          const int s = it % p.stages;
+          const uint32_t ph = (it / p.stages) & 1u;
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+          const uint32_t dst = base + s * stage_bytes;
+          mbar_expect_tx(full_bar(s), stage_bytes);
+          tma_load_2d(dst, &map_w, full_bar(s), kb * TILE_K, n_tile * TILE_N);
+          for (int j = 0; j < p.mt / A_BOX_ROWS; ++j)
+            tma_load_2d(dst + W_STAGE_BYTES + j * A_BOX_BYTES, &map_a, full_bar(s), kb * TILE_K,
+                        m_tile * p.mt + j * A_BOX_ROWS);
+        }
+        u += kb1 - kb0;
+      }
+      if (!ok) {  // give the copies already issued time to land before the CTA's shared memory is released
+        const unsigned long long t0 = globaltimer();
+        while (globaltimer() - t0 < 2000000ull) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer =====================
+    if (lane == 0 && u0 < u1) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.mt >> 3) << 17) | ((uint32_t)(TILE_N >> 4) << 24);
+      uint32_t it = 0, seg = 0;
+      bool ok = true;
+      for (long long u = u0; u < u1 && ok; ++seg) {
+        const int t = (int)(u / p.nkb), kb0 = (int)(u - (long long)t * p.nkb);
+        const int kb1 = (int)min((long long)p.nkb, kb0 + (u1 - u));
+        const uint32_t a = seg & 1u, aph = (seg >> 1) & 1u;
+        if (!mbar_wait(tempty_bar(a), aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + a * (uint32_t)p.mt;
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
+          const int s = it % p.stages;
+          const uint32_t ph = (it / p.stages) & 1u;
+          if (!mbar_wait(full_bar(s), ph, abort_flag, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t wdesc = umma_desc(base + s * stage_bytes);
+          const uint64_t adesc = umma_desc(base + s * stage_bytes + W_STAGE_BYTES);
+#pragma unroll
+          for (int k = 0; k < TILE_K / 16; ++k)
+            umma_bf16(d_tmem, wdesc + 2 * k, adesc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+          umma_commit(empty_bar(s));  // the stage is free once these MMAs have read it
+        }
+        if (ok) umma_commit(tfull_bar(a));
+        u += kb1 - kb0;
+      }
+    }
+  } else {
+    // ===================== epilogue (warps 2..5) =====================
+    const int q = warp & 3;                 // TMEM lane quarter this warp may read
+    const int row = q * 32 + lane;          // weight row inside the tile
+    const int et = threadIdx.x - 64;        // 0..127
+    uint32_t seg = 0;
+    bool ok = true;
+    for (long long u = u0; u < u1 && ok; ++seg) {
+      const int t = (int)(u / p.nkb), kb0 = (int)(u - (long long)t * p.nkb);
+      const int kb1 = (int)min((long long)p.nkb, kb0 + (u1 - u));
+      const int n_tile = t / m_tiles, m_tile = t - n_tile * m_tiles;
+      const uint32_t a = seg & 1u, aph = (seg >> 1) & 1u;
+      const bool complete = (kb0 == 0 && kb1 == p.nkb);
+      const int n = n_tile * TILE_N + row;
+      const int m_base = m_tile * p.mt;
+      // one thread does the bounded wait and tells the others, so that all 128 take the same branch
+      if (et == 0) *epi_ok = mbar_wait(tfull_bar(a), aph, abort_flag, p.status) ? 1 : 0;
+      epi_bar_sync();
+      if (!*epi_ok) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * (uint32_t)p.mt;
+      // slot 0 = this CTA's first segment, slot 1 = its last (a range has at most two cut tiles)
+      float* my_partial = p.partial + ((size_t)blockIdx.x * 2 + (u == u0 ? 0 : 1)) * ((size_t)p.mt * TILE_N);
+      for (int c0 = 0; c0 < p.mt; c0 += 16) {
+        uint32_t r[16];
+        tmem_ld16(taddr + c0, r);
+        if (complete) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int m = m_base + c0 + j;
+            if (m < M && n < p.N) apply_epilogue<__nv_bfloat16>(p.ep, m, n, __uint_as_float(r[j]));
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) my_partial[(size_t)(c0 + j) * TILE_N + row] = __uint_as_float(r[j]);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(tempty_bar(a));  // the accumulator may be overwritten
+      if (!complete) {
+        // publish the partial, then find out whether this CTA is the tile's last contributor
+        __threadfence();
+        epi_bar_sync();
+        const long long tu0 = (long long)t * p.nkb, tu1 = tu0 + p.nkb;
+        const int c_first = cta_of_unit(tu0, U, G), c_last = cta_of_unit(tu1 - 1, U, G);
+        if (et == 0) {
+          int contributors = 0;
+          for (int c = c_first; c <= c_last; ++c) contributors += range_begin(c, U, G) < range_begin(c + 1, U, G) ? 1 : 0;
+          const int old = atomicAdd(p.counters + t, 1);
+          *last_flag = (old == contributors - 1) ? 1 : 0;
+          if (old == contributors - 1) p.counters[t] = 0;  // ready for the next launch
+        }
+        epi_bar_sync();
+        if (*last_flag) {
+          __threadfence();
+          for (int c0 = 0; c0 < p.mt; c0 += 16) {
+            float acc[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) acc[j] = 0.f;
+            for (int c = c_first; c <= c_last; ++c) {
+              const long long cb = range_begin(c, U, G), ce = range_begin(c + 1, U, G);
+              if (cb >= ce) continue;
+              const int slot = (cb / p.nkb == t) ? 0 : 1;
+              const float* pp = p.partial + ((size_t)c * 2 + slot) * ((size_t)p.mt * TILE_N) + (size_t)c0 * TILE_N + row;
+#pragma unroll
+              for (int j = 0; j < 16; ++j) acc[j] += __ldcg(pp + (size_t)j * TILE_N);
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int m = m_base + c0 + j;
+              if (m < M && n < p.N) apply_epilogue<__nv_bfloat16>(p.ep, m, n, acc[j]);
+            }
+          }
+        }
+        epi_bar_sync();  // last_flag is rewritten by the next cut segment
+      }
+      u += kb1 - kb0;
+    }
+  }
+
+  // ---- teardown: everyone meets, then the allocating warp frees the TMEM columns
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
+  }
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+// Tensor map of a row-major bf16 matrix [rows][cols] with a (box_rows x 64) box and 128-byte swizzle.
+int tc_make_map(void* out_map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return -1;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * 2};
+  const cuuint32_t box[2] = {TILE_K, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn((CUtensorMap*)out_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box,
+                        estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return (int)r;
+}
+
+int tc_weight_box_rows() { return TILE_N; }
+int tc_act_box_rows() { return A_BOX_ROWS; }
+
+// Activation rows per tile for a launch whose row count is at most m_max.
+int tc_pick_mt(int m_max) {
+  const int m_tiles = (m_max + 255) / 256;
+  const int per = (m_max + m_tiles - 1) / m_tiles;
+  int mt = (per + 15) / 16 * 16;
+  return mt < 16 ? 16 : mt;
+}
+
+size_t tc_partial_floats(int grid, int mt) { return (size_t)2 * grid * mt * TILE_N; }
+size_t tc_counter_ints(int N, int m_max) { return (size_t)((N + TILE_N - 1) / TILE_N) * ((m_max + 15) / 16); }
+
+cudaError_t tc_prepare(int* smem_limit_out) {
+  int dev = 0, lim = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  e = cudaDeviceGetAttribute(&lim, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  if (e != cudaSuccess) return e;
+  cudaFuncAttributes fa;
+  e = cudaFuncGetAttributes(&fa, gemm_tc_kernel);
+  if (e != cudaSuccess) return e;
+  lim -= (int)fa.sharedSizeBytes;  // the opt-in limit covers static + dynamic shared memory
+  e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
+  if (smem_limit_out) *smem_limit_out = lim;
+  return e;
+}
+
+cudaError_t launch_gemm_tc(const void* map_w, const void* map_a, int N, int K, const int32_t* m_total, int m_max,
+                           const Epilogue& ep, float* partial, int32_t* counters, int32_t* status, int grid,
+                           int smem_limit, cudaStream_t st) {
+  if (m_max <= 0) return cudaSuccess;
+  TcParams p;
+  p.N = N; p.K = K; p.nkb = (K + TILE_K - 1) / TILE_K; p.n_tiles = (N + TILE_N - 1) / TILE_N;
+  p.mt = tc_pick_mt(m_max);
+  p.m_tiles_max = (m_max + p.mt - 1) / p.mt;
+  const int stage_bytes = W_STAGE_BYTES + p.mt * TILE_K * 2;
+  const int overhead = 1024 + 8 * (2 * 16 + 4) + 64;
+  int stages = (smem_limit - overhead) / stage_bytes;
+  if (stages > 16) stages = 16;
+  if (stages < 2) return cudaErrorInvalidConfiguration;
+  p.stages = stages;
+  int cols = 32;
+  while (cols < 2 * p.mt) cols <<= 1;
+  p.tmem_cols = cols;
+  p.m_total = m_total; p.partial = partial; p.counters = counters; p.status = status; p.ep = ep;
+  const size_t smem = (size_t)stages * stage_bytes + overhead;
+  gemm_tc_kernel<<<grid, NUM_THREADS, smem, st>>>(*(const CUtensorMap*)map_w, *(const CUtensorMap*)map_a, p);
+  return cudaGetLastError();
+}
+
+}  // namespace rd

@@ -63,6 +63,18 @@ struct Dims {
 cudaError_t launch_gemm_simt(int dtype, const void* A, int lda, const void* W, int N, int K, const int32_t* m_total,
                              int m_max, const Epilogue& ep, cudaStream_t st);
 
+// Tensor-core (tcgen05) projection, bf16 only.  Operands are passed as TMA descriptors.
+int tc_make_map(void* out_map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows);
+int tc_weight_box_rows();
+int tc_act_box_rows();
+int tc_pick_mt(int m_max);
+size_t tc_partial_floats(int grid, int mt);
+size_t tc_counter_ints(int N, int m_max);
+cudaError_t tc_prepare(int* smem_limit_out);
+cudaError_t launch_gemm_tc(const void* map_w, const void* map_a, int N, int K, const int32_t* m_total, int m_max,
+                           const Epilogue& ep, float* partial, int32_t* counters, int32_t* status, int grid,
+                           int smem_limit, cudaStream_t st);
+
 cudaError_t launch_embed(int dtype, const void* emb, const int32_t* tok, float* x, int d, int V, const int32_t* m_total,
                          int m_max, int* status, cudaStream_t st);
 cudaError_t launch_rmsnorm(int dtype, const float* x, const void* gain, void* out_t, float* out_f32, int d, float eps,
