@@ -27,3 +27,36 @@ def read_golden(name):
     path = os.path.join(ROOT, "tests", "golden", name)
     with open(path) as f:
         return [ln.strip() for ln in f if ln.strip() and not ln.startswith("#")]
+
+
+# ---------------------------------------------------------------------------- GPU rigs
+def dev(a, dtype=None):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a)).to("cuda:0", torch.int32 if dtype is None else dtype)
+
+
+def top2_gap(logits):
+    s = np.sort(logits, axis=-1)
+    return s[..., -1] - s[..., -2]
+
+
+class Rig:
+    """A model on the GPU (through the C ABI) plus the same stored weight values for the oracle."""
+
+    def __init__(self, name="tiny", flags=0, cfg=None, oracle_dtype=np.float64, **over):
+        from oracle import redrafter_oracle as ora
+        from paper_2403_09919_b200 import binding
+        self.binding = binding
+        self.ora = ora
+        self.cfg = dict(synth.CONFIGS[name] if cfg is None else cfg, **over)
+        self.w = synth.make_weights(self.cfg, "cuda:0")
+        self.W, self.D = synth.weights_to_numpy(self.w, self.cfg)
+        self.odt = oracle_dtype
+        if oracle_dtype != np.float32:
+            self.W, self.D = ora.convert_weights(self.W, self.D, oracle_dtype)
+        self.eng = binding.ReDrafter(self.cfg, self.w, flags=flags)
+        self.hd = self.cfg["d_model"] // self.cfg["n_heads"]
+
+    def new_kv(self):
+        c = self.cfg
+        return self.ora.KVCache(c["n_layers"], c["max_ctx"], c["n_heads"], self.hd, self.odt)

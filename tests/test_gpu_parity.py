@@ -16,36 +16,12 @@ GAP = 0.05
 TOL_FP32 = 2e-3
 
 
-def dev(a, dtype=torch.int32):
-    return torch.from_numpy(np.ascontiguousarray(a)).to("cuda:0", dtype)
-
-
-class Rig:
-    """A tiny model on the GPU plus the same weights for the oracle."""
-
-    def __init__(self, name="tiny", flags=0, **over):
-        from paper_2403_09919_b200 import binding
-        self.binding = binding
-        self.cfg = dict(synth.CONFIGS[name], **over)
-        self.w = synth.make_weights(self.cfg, "cuda:0")
-        self.W, self.D = synth.weights_to_numpy(self.w, self.cfg)
-        self.eng = binding.ReDrafter(self.cfg, self.w, flags=flags)
-        c = self.cfg
-        self.hd = c["d_model"] // c["n_heads"]
-
-    def new_kv(self):
-        c = self.cfg
-        return ora.KVCache(c["n_layers"], c["max_ctx"], c["n_heads"], self.hd)
+from helpers import Rig, dev, top2_gap  # noqa: E402
 
 
 @pytest.fixture(scope="module")
 def rig():
     return Rig()
-
-
-def top2_gap(logits):
-    s = np.sort(logits, axis=-1)
-    return s[..., -1] - s[..., -2]
 
 
 # ------------------------------------------------------------------ pack
