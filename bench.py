@@ -331,6 +331,7 @@ def main():
             eng.step(None, out)
             gm = eng.profile_read(0)
             at = eng.profile_read(1)
+            others = [eng.profile_read(c) for c in range(2, 8)]
         eng.profile(False)
         g_ms, g_bytes, g_n = gm
         achieved = g_bytes / (g_ms * 1e-3) / 1e9 if g_ms > 0 else 0.0
@@ -338,7 +339,11 @@ def main():
         line["roofline"] = {"bound": "hbm", "kernel": "projection (weight-streaming GEMM)", "achieved": achieved, "peak": peak,
                             "unit": "GB/s", "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
                             "launches_per_step": g_n / prof_steps, "ms_per_step_in_kernel": g_ms / prof_steps,
-                            "attention_ms_per_step": at[0] / prof_steps}
+                            "attention_ms_per_step": at[0] / prof_steps,
+                            "other_ms_per_step": {n: round(o[0] / prof_steps, 4) for n, o in
+                                                  zip(("rmsnorm", "rope", "swiglu", "draft_select", "pack_accept", "misc"), others)},
+                            "other_launches_per_step": {n: o[2] / prof_steps for n, o in
+                                                        zip(("rmsnorm", "rope", "swiglu", "draft_select", "pack_accept", "misc"), others)}}
         line["step_roofline"] = {"algorithmic_bytes_per_step": sb["total"], "achieved_gbs": sb["total"] / (ms_per_step * 1e-3) / 1e9,
                                  "frac_of_measured_peak": sb["total"] / (ms_per_step * 1e-3) / 1e9 / peak,
                                  "frac_of_nominal_8tbs": sb["total"] / (ms_per_step * 1e-3) / 8e12,
@@ -363,34 +368,53 @@ def main():
             line["autoregressive"] = {"tokens_per_s": n_ar * B / (ms_ar * 1e-3), "ms_per_step": ms_ar / n_ar,
                                       "frac_of_measured_peak": sb["ar"] / (ms_ar / n_ar * 1e-3) / 1e9 / peak}
             cont_h = cont.cpu().numpy()                                   # [n_ar+1, B]; row 0 = root after prefill
+            # Planted-beam mode, teacher-forced on the autoregressive stream: beams for every stream position are
+            # planted up front; each step the host reads the accepted length (as a serving loop does), advances
+            # the position and hands the step the stream's own token as root.  Accepted tokens are stream tokens by
+            # construction; only a bonus token can differ (a near-tie between the two kernels' summation orders),
+            # which the root hand-off overrides -- counted as "bonus_flips".
             rng = np.random.default_rng(2000 + cfg.get("seed", 0))
-            planted = np.zeros((need, B, BW, L), dtype=np.int32)
-            posn = np.ones(B, dtype=np.int64)
-            exp_acc = np.zeros((need, B), dtype=np.int64)
-            for s in range(need):
+            n_pos = n_ar - L
+            table = np.zeros((n_pos, B, BW, L), dtype=np.int32)
+            for p_ in range(1, n_pos):
                 for b in range(B):
-                    c = cont_h[posn[b]:posn[b] + L, b]
-                    planted[s, b] = synth.plant_beams(c, BW, L, cfg["vocab"], rng, p=cfg.get("plant_p", 0.3),
-                                                      rho=cfg.get("plant_rho", 0.0))
-                    exp_acc[s, b] = synth.first_mismatch(planted[s, b], c).max()
-                    posn[b] += exp_acc[s, b] + 1
-            planted_d = torch.from_numpy(planted).to(device)
+                    table[p_, b] = synth.plant_beams(cont_h[p_:p_ + L, b], BW, L, cfg["vocab"], rng, p=cfg.get("plant_p", 0.3),
+                                                     rho=cfg.get("plant_rho", 0.0))
+            table_d = torch.from_numpy(table).to(device)
             eng.prefill(prompts)
-            for s in range(args.warmup):
-                eng.step(planted_d[s], out)
-            acc_p = torch.zeros(args.steps, B, dtype=torch.int32, device=device)
+            posn = np.ones(B, dtype=np.int64)
+            beams_d = torch.zeros(B, BW, L, dtype=torch.int32, device=device)
+            pin_a2 = torch.zeros(B, dtype=torch.int32).pin_memory()
+            pin_t2 = torch.zeros(B, L + 1, dtype=torch.int32).pin_memory()
+            stats = dict(tokens=0, flips=0, closed=0, steps=0)
 
-            def one_p(i):
-                eng.step(planted_d[args.warmup + i], out)
-                acc_p[i].copy_(out.n_accept)
+            def one_p(i, count=True):
+                for b in range(B):
+                    beams_d[b].copy_(table_d[posn[b], b])
+                eng.step(beams_d, out)
+                pin_a2.copy_(out.n_accept, non_blocking=True)
+                pin_t2.copy_(out.tokens, non_blocking=True)
+                torch.cuda.current_stream().synchronize()
+                for b in range(B):
+                    a_ = int(pin_a2[b])
+                    if count:
+                        stats["tokens"] += a_ + 1
+                        stats["steps"] += 1
+                        stats["closed"] += int(a_ == synth.first_mismatch(table[posn[b], b], cont_h[posn[b]:posn[b] + L, b]).max())
+                        stats["flips"] += int(int(pin_t2[b, a_]) != int(cont_h[posn[b] + a_, b]))
+                    posn[b] += a_ + 1
+                eng.set_state(None, cont[posn[0] - 1] if B == 1 else torch.stack([cont[posn[b] - 1, b] for b in range(B)]), None)
+            for s_ in range(args.warmup):
+                one_p(s_, count=False)
             ms_p = timed_loop(eng, args.steps, one_p)
             eng.poll()
-            tok_p = int(acc_p.sum().item()) + args.steps * B
+            tok_p = stats["tokens"]
             line["planted"] = {"tokens_per_s": tok_p / (ms_p * 1e-3), "ms_per_step": ms_p / args.steps,
-                               "tokens_per_step": tok_p / (args.steps * B),
-                               "matches_closed_form": bool((acc_p.cpu().numpy() == exp_acc[args.warmup:]).all()),
+                               "tokens_per_step": tok_p / max(1, stats["steps"]),
+                               "steps_matching_closed_form": stats["closed"], "bonus_flips": stats["flips"],
                                "speedup_vs_autoregressive": (tok_p / ms_p) / (n_ar * B / ms_ar),
-                               "note": "beams = the LLM's own greedy continuation with each token replaced at p=0.3"}
+                               "note": "beams = the autoregressive stream's continuation with each token replaced at p=0.3; "
+                                       "teacher-forced root, accepted length read by the host every step (one sync per step)"}
             line["speedup_vs_autoregressive"] = value / world / (n_ar * B / (ms_ar * 1e-3))
         if not args.no_cpu_baseline and world == 1:
             r = OracleSample(cfg, args.oracle_layers).run(args.cpu_steps, warmup=1)

@@ -185,15 +185,25 @@ RD_API int redrafter_set_ctx_bound(rd_handle* h, int32_t max_ctx_now);
  * error a kernel recorded (e.g. an out-of-range token id was skipped). */
 RD_API int redrafter_poll(rd_handle* h, void* stream);
 
-/* Per-launch device timing, for measurement only (off by default).  While enabled, every projection
- * (class 0) and every attention launch (class 1) is bracketed by CUDA events on its stream; the
- * events are created on first use.  redrafter_profile(h, 1) also clears the totals.
+/* Per-launch device timing, for measurement only (off by default).  While enabled, every launch of
+ * redrafter_step is bracketed by CUDA events on its stream, summed by class: 0 projections,
+ * 1 attention, 2 RMSNorm, 3 rotary + KV write, 4 SwiGLU, 5 drafter selection kernels, 6 pack/accept,
+ * 7 the rest.  The events are created on first use.  redrafter_profile(h, 1) also clears the totals.
  * redrafter_profile_read waits for the recorded events and returns, for one class, the summed
  * device time in ms, the summed algorithmic weight bytes of the launches (class 0 only: N*K*element
  * size per projection) and the number of launches.  Outputs are HOST pointers, each may be NULL.
  * The event pool grows with the launches between reads: read at least once per step. */
 RD_API int redrafter_profile(rd_handle* h, int enable);
 RD_API int redrafter_profile_read(rd_handle* h, int32_t cls, double* ms, double* bytes, int64_t* launches);
+
+/* In-kernel timeline of the tensor-core projection launches, for measurement only.  After
+ * redrafter_trace(h, 1, stream) the next launches (up to 512) each record eight %globaltimer
+ * values in ns: [0] first CTA entered, [1]/[2] first/last producer past its dependency wait,
+ * [3]/[4] first/last MMA issuer done, [5]/[6] first/last CTA done, [7] unused.
+ * redrafter_trace_read synchronises the stream, copies the records of the launches traced so far to
+ * the HOST buffer out[max_launches][8] and returns their number (or a negative rd_status). */
+RD_API int redrafter_trace(rd_handle* h, int enable, void* stream);
+RD_API int redrafter_trace_read(rd_handle* h, void* stream, uint64_t* out, int32_t max_launches);
 
 /* Number of kernels this handle has launched since it was created (for launch accounting). */
 RD_API int64_t redrafter_launch_count(const rd_handle* h);

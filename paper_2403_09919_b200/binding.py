@@ -25,7 +25,7 @@ EXPORTS = ["redrafter_workspace_bytes", "redrafter_kv_bytes", "redrafter_init", 
            "redrafter_last_error", "redrafter_prefill", "redrafter_draft", "redrafter_pack", "redrafter_verify",
            "redrafter_accept", "redrafter_step", "redrafter_ar_step", "redrafter_get_state", "redrafter_set_state",
            "redrafter_set_ctx_bound", "redrafter_poll", "redrafter_launch_count", "redrafter_profile",
-           "redrafter_profile_read"]
+           "redrafter_profile_read", "redrafter_trace", "redrafter_trace_read"]
 
 
 class RdConfig(C.Structure):
@@ -85,6 +85,8 @@ def lib():
         L.redrafter_profile.argtypes = [vp, C.c_int]
         L.redrafter_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_double),
                                              C.POINTER(C.c_int64)]
+        L.redrafter_trace.argtypes = [vp, C.c_int, vp]
+        L.redrafter_trace_read.argtypes = [vp, vp, vp, i32]
         _lib = L
     return _lib
 
@@ -282,6 +284,18 @@ class ReDrafter:
         ms, by, n = C.c_double(), C.c_double(), C.c_int64()
         self._ck(self.L.redrafter_profile_read(self.h, cls, C.byref(ms), C.byref(by), C.byref(n)))
         return ms.value, by.value, n.value
+
+    def trace(self, enable):
+        self._ck(self.L.redrafter_trace(self.h, 1 if enable else 0, _stream()))
+
+    def trace_read(self, max_launches=512):
+        """[n, 8] uint64 %globaltimer records of the traced projection launches (host numpy array)."""
+        import numpy as np
+        buf = np.zeros((max_launches, 8), dtype=np.uint64)
+        n = self.L.redrafter_trace_read(self.h, _stream(), buf.ctypes.data, max_launches)
+        if n < 0:
+            self._ck(-n)
+        return buf[:n]
 
     def launch_count(self):
         return int(self.L.redrafter_launch_count(self.h))

@@ -31,9 +31,9 @@ struct Workspace {
   int32_t *ctx, *root, *status;
   float* h;
   // row tables of the current forward
-  int32_t *row_tok, *row_seq, *row_pos, *row_slot, *row_ncache, *row_local, *row_out_index, *m_total, *last_row;
+  int32_t *row_tok, *row_seq, *row_pos, *row_slot, *row_ncache, *row_local, *row_out_index, *m_total, *last_row, *seq_off;
   // activations of the forward (compact rows)
-  float *x, *qkv, *gu, *hidden_f, *logits;
+  float *x, *qkv, *gu, *hidden_f, *logits, *rope_tab;
   void *a_t, *attn_t, *act_t, *hidden_t, *h_t;
   int32_t* argmax_c;
   // step-internal packed beam, beams, verify outputs, accept scratch
@@ -47,6 +47,10 @@ struct Workspace {
   // tensor-core projection scratch
   int32_t* tc_counters;
   float* tc_partial;
+  // tensor-core attention scratch
+  int32_t* att_counters;
+  float* att_scratch;
+  unsigned long long* trace;  // [TRACE_SLOTS][8] timestamps of traced projection launches
 };
 
 size_t esize(int dtype) { return dtype == RD_DTYPE_FP32 ? 4 : 2; }
@@ -56,6 +60,10 @@ struct alignas(64) TensorMapBox {  // opaque storage of one CUtensorMap (128 byt
 };
 
 }  // namespace
+
+// timing classes of redrafter_profile_read
+enum { PROF_GEMM = 0, PROF_ATTN = 1, PROF_NORM = 2, PROF_ROPE = 3, PROF_SWIGLU = 4, PROF_DRAFT_SMALL = 5, PROF_PACK_ACCEPT = 6,
+       PROF_MISC = 7, PROF_CLASSES = 8 };
 
 struct rd_handle {
   rd_config cfg;
@@ -72,14 +80,15 @@ struct rd_handle {
   int64_t launches;
   // tensor-core path (bf16): TMA descriptors by base pointer, launch geometry
   bool use_tc;
+  int trace_next;  // next trace slot, -1 = tracing off
   int tc_grid, tc_smem;
   std::unordered_map<const void*, TensorMapBox> maps;
   // optional per-launch timing of the projections (class 0) and the attention kernel (class 1)
   bool profiling;
-  std::vector<cudaEvent_t> ev[2];   // start/stop pairs
-  size_t ev_used[2];
-  double prof_ms[2], prof_bytes[2];
-  int64_t prof_n[2];
+  std::vector<cudaEvent_t> ev[PROF_CLASSES];   // start/stop pairs
+  size_t ev_used[PROF_CLASSES];
+  double prof_ms[PROF_CLASSES], prof_bytes[PROF_CLASSES];
+  int64_t prof_n[PROF_CLASSES];
   char err[512];
 };
 
@@ -130,7 +139,9 @@ int shape_ok(const Dims& dm) {
   return 1;
 }
 
+constexpr int TRACE_SLOTS = 512;
 constexpr int TC_MAX_GRID = 160;  // upper bound of the SM count the scratch is sized for
+constexpr int ATT_MAX_SPLIT_BLOCKS = 4 * TC_MAX_GRID;  // (blocks x splits) the split-KV scratch holds
 
 int m_cap_of(const Dims& dm) {
   const int v = dm.B * dm.NMAX;
@@ -146,6 +157,8 @@ void carve(Bump& bp, const Dims& dm, int m_cap, Workspace* w) {
   w->row_slot = bp.take<int32_t>(m_cap); w->row_ncache = bp.take<int32_t>(m_cap); w->row_local = bp.take<int32_t>(m_cap);
   w->row_out_index = bp.take<int32_t>(m_cap); w->m_total = bp.take<int32_t>(4); w->last_row = bp.take<int32_t>(B);
   w->one_b = bp.take<int32_t>(4); w->one_r = bp.take<int32_t>(4);
+  w->seq_off = bp.take<int32_t>(B + 1);
+  w->att_counters = bp.take<int32_t>(ATT_MAX_SPLIT_BLOCKS);
   {
     int max_n = 3 * dm.d;
     if (2 * dm.F > max_n) max_n = 2 * dm.F;
@@ -158,6 +171,7 @@ void carve(Bump& bp, const Dims& dm, int m_cap, Workspace* w) {
   w->gu = bp.take<float>((size_t)m_cap * 2 * dm.F);
   w->hidden_f = bp.take<float>((size_t)m_cap * dm.d);
   w->logits = bp.take<float>((size_t)m_cap * dm.V);
+  w->rope_tab = bp.take<float>((size_t)m_cap * dm.hd);
   w->a_t = bp.take<char>((size_t)m_cap * dm.d * es);
   w->attn_t = bp.take<char>((size_t)m_cap * dm.d * es);
   w->act_t = bp.take<char>((size_t)m_cap * dm.F * es);
@@ -182,6 +196,8 @@ void carve(Bump& bp, const Dims& dm, int m_cap, Workspace* w) {
   w->cand_idx = bp.take<int32_t>((size_t)R * dm.BW); w->hist_a = bp.take<int32_t>((size_t)R * dm.L);
   w->hist_b = bp.take<int32_t>((size_t)R * dm.L);
   w->tc_partial = bp.take<float>(dm.dtype == RD_DTYPE_BF16 ? tc_partial_floats(TC_MAX_GRID, tc_pick_mt(m_cap)) : 0);
+  w->att_scratch = bp.take<float>(dm.dtype == RD_DTYPE_BF16 ? attn_tc_scratch_floats(ATT_MAX_SPLIT_BLOCKS, 1, dm.hd) : 0);
+  w->trace = bp.take<unsigned long long>((size_t)TRACE_SLOTS * 8);
   bp.take<char>(256);
 }
 
@@ -219,6 +235,12 @@ struct ProfScope {
   }
 };
 
+#define CKP(h, cls, expr)              \
+  do {                                 \
+    ProfScope ps__(h, cls, 0.0, st);   \
+    CK(h, expr);                       \
+  } while (0)
+
 Epilogue ep_store(float* out, int ld) {
   Epilogue e{};
   e.out_f32 = out; e.ld_out_f32 = ld;
@@ -233,8 +255,10 @@ int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, cons
     auto ia = h->maps.find(A), iw = h->maps.find(W);
     if (ia == h->maps.end() || iw == h->maps.end() || lda != K)
       return fail(h, RD_ERR_STATE, "projection operand without a TMA descriptor");
+    unsigned long long* tr = nullptr;
+    if (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) tr = h->ws.trace + (size_t)8 * h->trace_next++;
     CK(h, launch_gemm_tc(&iw->second, &ia->second, N, K, m_total, m_max, ep, h->ws.tc_partial, h->ws.tc_counters,
-                         h->ws.status, h->tc_grid, h->tc_smem, st));
+                         h->ws.status, h->tc_grid, h->tc_smem, tr, st));
     return RD_OK;
   }
   CK(h, launch_gemm_simt(h->dm.dtype, A, lda, W, N, K, m_total, m_max, ep, st));
@@ -247,32 +271,51 @@ char* kv_plane_ptr(rd_handle* h, int layer, int which) {
 
 // Embedding -> n_layers x {attention block, FFN block} -> final norm.  Rows and masks come from the
 // row tables in the workspace; results: ws.hidden_f / ws.hidden_t (compact rows).
-int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, cudaStream_t st) {
+int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int rows_per_seq_max, cudaStream_t st) {
   Workspace& w = h->ws;
   const Dims& dm = h->dm;
   RowTables rt{w.row_tok, w.row_seq, w.row_pos, w.row_slot, w.row_ncache, w.row_local, mask, w.m_total};
-  CK(h, launch_embed(dm.dtype, h->w.tok_emb, w.row_tok, w.x, dm.d, dm.V, w.m_total, m_max, w.status, st));
+  CKP(h, PROF_MISC, launch_embed(dm.dtype, h->w.tok_emb, w.row_tok, w.x, dm.d, dm.V, w.m_total, m_max, w.status, st));
+  CKP(h, PROF_MISC, launch_rope_table(w.row_pos, w.rope_tab, dm.hd, dm.theta, w.m_total, m_max, st));
+  // attention launch geometry (tensor-core path): blocks of 64 rows per sequence, keys split so that
+  // every SM gets a CTA, at least one 64-key chunk per split
+  int row_blocks = 1, n_splits = 1;
+  if (h->use_tc) {
+    const int rpb = attn_tc_rows_per_block();
+    row_blocks = (rows_per_seq_max + rpb - 1) / rpb;
+    const int blocks = dm.H * n_seq * row_blocks;
+    n_splits = (h->tc_grid + blocks - 1) / blocks;  // about one CTA per SM
+    const int max_chunks = (h->ctx_bound + rows_per_seq_max + 63) / 64;
+    if (n_splits > max_chunks) n_splits = max_chunks;
+    if (n_splits > 16) n_splits = 16;
+    if (n_splits < 1) n_splits = 1;
+    while (n_splits > 1 && (long long)blocks * n_splits > ATT_MAX_SPLIT_BLOCKS) --n_splits;
+  }
   for (int l = 0; l < dm.n_layers; ++l) {
-    CK(h, launch_rmsnorm(dm.dtype, w.x, h->attn_norm[l], w.a_t, nullptr, dm.d, dm.eps, w.m_total, m_max, st));
+    CKP(h, PROF_NORM, launch_rmsnorm(dm.dtype, w.x, h->attn_norm[l], w.a_t, nullptr, dm.d, dm.eps, w.m_total, m_max, st));
     int rc = gemm(h, w.a_t, dm.d, h->wqkv[l], 3 * dm.d, dm.d, w.m_total, m_max, ep_store(w.qkv, 3 * dm.d), st);
     if (rc) return rc;
-    CK(h, launch_rope_kv(dm.dtype, w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), rt, dm, m_max, w.status, st));
+    CKP(h, PROF_ROPE, launch_rope_kv(dm.dtype, w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.rope_tab, rt, dm, m_max, w.status, st));
     {
       ProfScope ps(h, 1, 0.0, st);
-      CK(h, launch_attention(dm.dtype, w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.attn_t, rt, dm, m_max, st));
+      if (h->use_tc)
+        CK(h, launch_attention_tc(w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.attn_t, rt, w.seq_off, dm, n_seq,
+                                  row_blocks, n_splits, w.att_scratch, w.att_counters, st));
+      else
+        CK(h, launch_attention(dm.dtype, w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.attn_t, rt, dm, m_max, st));
     }
     Epilogue eo{};
     eo.resid = w.x; eo.ld_resid = dm.d; eo.out_f32 = w.x; eo.ld_out_f32 = dm.d;
     rc = gemm(h, w.attn_t, dm.d, h->wo[l], dm.d, dm.d, w.m_total, m_max, eo, st);
     if (rc) return rc;
-    CK(h, launch_rmsnorm(dm.dtype, w.x, h->ffn_norm[l], w.a_t, nullptr, dm.d, dm.eps, w.m_total, m_max, st));
+    CKP(h, PROF_NORM, launch_rmsnorm(dm.dtype, w.x, h->ffn_norm[l], w.a_t, nullptr, dm.d, dm.eps, w.m_total, m_max, st));
     rc = gemm(h, w.a_t, dm.d, h->w_gate_up[l], 2 * dm.F, dm.d, w.m_total, m_max, ep_store(w.gu, 2 * dm.F), st);
     if (rc) return rc;
-    CK(h, launch_swiglu(dm.dtype, w.gu, w.act_t, dm.F, w.m_total, m_max, st));
+    CKP(h, PROF_SWIGLU, launch_swiglu(dm.dtype, w.gu, w.act_t, dm.F, w.m_total, m_max, st));
     rc = gemm(h, w.act_t, dm.F, h->w_down[l], dm.d, dm.F, w.m_total, m_max, eo, st);
     if (rc) return rc;
   }
-  CK(h, launch_rmsnorm(dm.dtype, w.x, h->w.final_norm, w.hidden_t, w.hidden_f, dm.d, dm.eps, w.m_total, m_max, st));
+  CKP(h, PROF_NORM, launch_rmsnorm(dm.dtype, w.x, h->w.final_norm, w.hidden_t, w.hidden_f, dm.d, dm.eps, w.m_total, m_max, st));
   return RD_OK;
 }
 
@@ -289,8 +332,8 @@ int do_draft(rd_handle* h, cudaStream_t st, int32_t* beams, float* scores) {
   Workspace& w = h->ws;
   const Dims& dm = h->dm;
   const int B = h->batch, R = B * dm.BW;
-  CK(h, launch_draft_init(dm.dtype, h->w.tok_emb, w.root, w.h, w.xc_t, w.xc_f, w.sprev_t, dm, B, w.status, st));
-  if (dm.L > 1) CK(h, launch_fill_h(dm.dtype, w.h, w.x0_t, w.x0_f, dm, B, st));
+  CKP(h, PROF_DRAFT_SMALL, launch_draft_init(dm.dtype, h->w.tok_emb, w.root, w.h, w.xc_t, w.xc_f, w.sprev_t, dm, B, w.status, st));
+  if (dm.L > 1) CKP(h, PROF_DRAFT_SMALL, launch_fill_h(dm.dtype, w.h, w.x0_t, w.x0_f, dm, B, st));
   float *sc_in = w.score_a, *sc_out = w.score_b;
   int32_t *hi_in = w.hist_a, *hi_out = w.hist_b;
   for (int call = 1; call <= dm.L; ++call) {
@@ -320,8 +363,8 @@ int do_draft(rd_handle* h, cudaStream_t st, int32_t* beams, float* scores) {
     }
     int rc = gemm(h, xin_t, dm.dh, h->w.draft_out, dm.V, dm.dh, mt, rows, ep_store(w.dlogits, dm.V), st);
     if (rc) return rc;
-    CK(h, launch_row_topk(w.dlogits, dm.V, dm.BW, w.lse, w.cand_val, w.cand_idx, rows, st));
-    CK(h, launch_beam_merge(dm.dtype, call, w.lse, w.cand_val, w.cand_idx, sc_in, sc_out, hi_in, hi_out, h->w.tok_emb,
+    CKP(h, PROF_DRAFT_SMALL, launch_row_topk(w.dlogits, dm.V, dm.BW, w.lse, w.cand_val, w.cand_idx, rows, st));
+    CKP(h, PROF_DRAFT_SMALL, launch_beam_merge(dm.dtype, call, w.lse, w.cand_val, w.cand_idx, sc_in, sc_out, hi_in, hi_out, h->w.tok_emb,
                             w.x0_f, dm.dh, w.sprev_t, w.e_t, dm, B, beams, scores, st));
     float* tf = sc_in; sc_in = sc_out; sc_out = tf;
     int32_t* ti = hi_in; hi_in = hi_out; hi_out = ti;
@@ -333,15 +376,15 @@ int do_verify(rd_handle* h, const rd_packed& pk, cudaStream_t st, int32_t* argma
   Workspace& w = h->ws;
   const Dims& dm = h->dm;
   const int B = h->batch, m_max = B * dm.NMAX;
-  CK(h, launch_build_rows_tree(pk, w.ctx, w.row_tok, w.row_seq, w.row_pos, w.row_slot, w.row_ncache, w.row_local,
-                               w.row_out_index, w.m_total, dm, B, w.status, st));
-  int rc = forward_layers(h, pk.mask, m_max, st);
+  CKP(h, PROF_MISC, launch_build_rows_tree(pk, w.ctx, w.row_tok, w.row_seq, w.row_pos, w.row_slot, w.row_ncache, w.row_local,
+                               w.row_out_index, w.seq_off, w.m_total, dm, B, w.status, st));
+  int rc = forward_layers(h, pk.mask, m_max, B, dm.NMAX, st);
   if (rc) return rc;
   rc = gemm(h, w.hidden_t, dm.d, h->w.lm_head, dm.V, dm.d, w.m_total, m_max, ep_store(w.logits, dm.V), st);
   if (rc) return rc;
-  CK(h, launch_fill_i32(argmax, -1, B * dm.NMAX, st));
-  CK(h, launch_argmax_rows(w.logits, dm.V, argmax, w.row_out_index, w.m_total, m_max, st));
-  if (hidden) CK(h, launch_scatter_rows(w.hidden_f, dm.d, hidden, w.row_out_index, w.m_total, m_max, st));
+  CKP(h, PROF_MISC, launch_fill_i32(argmax, -1, B * dm.NMAX, st));
+  CKP(h, PROF_MISC, launch_argmax_rows(w.logits, dm.V, argmax, w.row_out_index, w.m_total, m_max, st));
+  if (hidden) CKP(h, PROF_MISC, launch_scatter_rows(w.hidden_f, dm.d, hidden, w.row_out_index, w.m_total, m_max, st));
   if (logits) CK(h, launch_scatter_rows(w.logits, dm.V, logits, w.row_out_index, w.m_total, m_max, st));
   return RD_OK;
 }
@@ -404,6 +447,7 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
     cudaError_t ce = cudaGetDevice(&dev);
     if (ce == cudaSuccess) ce = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (ce == cudaSuccess) ce = tc_prepare(&h->tc_smem);
+    if (ce == cudaSuccess) ce = attn_tc_prepare(dm.hd, dm.MW);
     if (ce != cudaSuccess || sms <= 0)
       return init_fail(h, RD_ERR_CUDA, "tensor-core path set-up: %s", cudaGetErrorString(ce));
     h->tc_grid = sms < TC_MAX_GRID ? sms : TC_MAX_GRID;
@@ -438,7 +482,8 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
   }
   h->prefilled = false; h->batch = dm.B; h->ctx_bound = 0; h->launches = 0; h->err[0] = 0;
   h->profiling = false;
-  for (int c = 0; c < 2; ++c) { h->ev_used[c] = 0; h->prof_ms[c] = 0; h->prof_bytes[c] = 0; h->prof_n[c] = 0; }
+  h->trace_next = -1;
+  for (int c = 0; c < PROF_CLASSES; ++c) { h->ev_used[c] = 0; h->prof_ms[c] = 0; h->prof_bytes[c] = 0; h->prof_n[c] = 0; }
   // clear the state and the constants the kernels read from device memory
   cudaError_t e = cudaMemsetAsync(workspace, 0, (size_t)((char*)h->ws.x - (char*)workspace), 0);
   if (e == cudaSuccess) e = cudaStreamSynchronize(0);
@@ -449,7 +494,7 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
 
 int redrafter_destroy(rd_handle* h) {
   if (!h) return RD_ERR_INVALID_ARG;
-  for (int c = 0; c < 2; ++c)
+  for (int c = 0; c < PROF_CLASSES; ++c)
     for (cudaEvent_t e : h->ev[c]) cudaEventDestroy(e);
   delete h;
   return RD_OK;
@@ -483,11 +528,11 @@ int redrafter_prefill(rd_handle* h, const int32_t* tokens, const int32_t* prompt
   if (rc) return rc;
   // passes of up to m_cap rows; a sequence's rows may span passes (its earlier rows are in the cache by then)
   const int cap = h->m_cap;
-  std::vector<int32_t> tok(cap), seq(cap), pos(cap), ncache(cap), local(cap), last(batch);
+  std::vector<int32_t> tok(cap), seq(cap), pos(cap), ncache(cap), local(cap), last(batch), soff(batch + 1), count(batch);
   int b = 0, done = 0;  // next sequence, tokens of it already processed
   while (b < batch) {
-    int m = 0;
-    for (int i = 0; i < batch; ++i) last[i] = -1;
+    int m = 0, longest_run = 0;
+    for (int i = 0; i < batch; ++i) { last[i] = -1; count[i] = 0; }
     while (b < batch && m < cap) {
       const int take = (prompt_len[b] - done) < (cap - m) ? (prompt_len[b] - done) : (cap - m);
       for (int i = 0; i < take; ++i) {
@@ -495,9 +540,14 @@ int redrafter_prefill(rd_handle* h, const int32_t* tokens, const int32_t* prompt
         seq[m] = b; pos[m] = done + i; ncache[m] = done + i + 1; local[m] = 0;
         ++m;
       }
+      count[b] = take;
+      if (take > longest_run) longest_run = take;
       done += take;
       if (done == prompt_len[b]) { last[b] = m - 1; ++b; done = 0; }
     }
+    // the sequences of a pass are consecutive and their rows contiguous from row 0
+    soff[0] = 0;
+    for (int i = 0; i < batch; ++i) soff[i + 1] = soff[i] + count[i];
     const size_t nb = (size_t)m * sizeof(int32_t);
     CKRT(h, cudaMemcpyAsync(w.row_tok, tok.data(), nb, cudaMemcpyHostToDevice, st));
     CKRT(h, cudaMemcpyAsync(w.row_seq, seq.data(), nb, cudaMemcpyHostToDevice, st));
@@ -506,9 +556,11 @@ int redrafter_prefill(rd_handle* h, const int32_t* tokens, const int32_t* prompt
     CKRT(h, cudaMemcpyAsync(w.row_ncache, ncache.data(), nb, cudaMemcpyHostToDevice, st));
     CKRT(h, cudaMemcpyAsync(w.row_local, local.data(), nb, cudaMemcpyHostToDevice, st));
     CKRT(h, cudaMemcpyAsync(w.last_row, last.data(), batch * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    CKRT(h, cudaMemcpyAsync(w.seq_off, soff.data(), (batch + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     CKRT(h, cudaMemcpyAsync(w.m_total, &m, sizeof(int32_t), cudaMemcpyHostToDevice, st));
     CKRT(h, cudaStreamSynchronize(st));  // the host staging vectors are reused by the next pass
-    rc = forward_layers(h, nullptr, m, st);
+    h->ctx_bound = longest;  // bound of the key extent for this pass
+    rc = forward_layers(h, nullptr, m, batch, longest_run, st);
     if (rc) return rc;
     CK(h, launch_prefill_finish(w.hidden_f, w.last_row, w.h, dm.d, batch, st));
   }
@@ -573,12 +625,12 @@ int redrafter_step(rd_handle* h, const int32_t* planted_beams, void* stream, con
   rc = do_draft(h, st, w.beams, w.scores);
   if (rc) return rc;
   const int32_t* beams = planted_beams ? planted_beams : w.beams;
-  CK(h, launch_pack(beams, w.root, w.ctx, w.pk, h->dm, h->batch, (h->cfg.flags & RD_FLAG_NO_TREE) ? 1 : 0, st));
+  CKP(h, PROF_PACK_ACCEPT, launch_pack(beams, w.root, w.ctx, w.pk, h->dm, h->batch, (h->cfg.flags & RD_FLAG_NO_TREE) ? 1 : 0, st));
   rc = do_verify(h, w.pk, st, w.argmax_p, w.hidden_p, nullptr);
   if (rc) return rc;
   rd_accept_out o{};
   if (out) o = *out;
-  CK(h, launch_accept(h->dm.dtype, beams, w.pk, w.argmax_p, w.hidden_p, h->kv, w.ctx, w.root, w.h, o, w.n_accept,
+  CKP(h, PROF_PACK_ACCEPT, launch_accept(h->dm.dtype, beams, w.pk, w.argmax_p, w.hidden_p, h->kv, w.ctx, w.root, w.h, o, w.n_accept,
                       w.best, w.ctx_prev, h->dm, h->batch, w.status, st));
   h->launches++;
   h->ctx_bound += 1 + h->dm.L;
@@ -594,8 +646,8 @@ int redrafter_ar_step(rd_handle* h, void* stream, int32_t* token) {
   const Dims& dm = h->dm;
   const int B = h->batch;
   CK(h, launch_build_rows_ar(w.root, w.ctx, w.row_tok, w.row_seq, w.row_pos, w.row_slot, w.row_ncache, w.row_local,
-                             w.row_out_index, w.m_total, dm, B, w.status, st));
-  int rc = forward_layers(h, nullptr, B, st);
+                             w.row_out_index, w.seq_off, w.m_total, dm, B, w.status, st));
+  int rc = forward_layers(h, nullptr, B, B, 1, st);
   if (rc) return rc;
   rc = gemm(h, w.hidden_t, dm.d, h->w.lm_head, dm.V, dm.d, w.m_total, B, ep_store(w.logits, dm.V), st);
   if (rc) return rc;
@@ -641,12 +693,12 @@ int redrafter_profile(rd_handle* h, int enable) {
   if (!h) return RD_ERR_INVALID_ARG;
   h->profiling = enable != 0;
   if (enable)
-    for (int c = 0; c < 2; ++c) { h->ev_used[c] = 0; h->prof_ms[c] = 0; h->prof_bytes[c] = 0; h->prof_n[c] = 0; }
+    for (int c = 0; c < PROF_CLASSES; ++c) { h->ev_used[c] = 0; h->prof_ms[c] = 0; h->prof_bytes[c] = 0; h->prof_n[c] = 0; }
   return RD_OK;
 }
 
 int redrafter_profile_read(rd_handle* h, int32_t cls, double* ms, double* bytes, int64_t* launches) {
-  if (!h || cls < 0 || cls > 1) return RD_ERR_INVALID_ARG;
+  if (!h || cls < 0 || cls >= PROF_CLASSES) return RD_ERR_INVALID_ARG;
   double total = h->prof_ms[cls];
   for (size_t i = 0; i + 1 < h->ev_used[cls]; i += 2) {
     CKRT(h, cudaEventSynchronize(h->ev[cls][i + 1]));
@@ -660,6 +712,33 @@ int redrafter_profile_read(rd_handle* h, int32_t cls, double* ms, double* bytes,
   if (bytes) *bytes = h->prof_bytes[cls];
   if (launches) *launches = h->prof_n[cls];
   return RD_OK;
+}
+
+int redrafter_trace(rd_handle* h, int enable, void* stream) {
+  if (!h) return RD_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (enable) {
+    // minima start at all-ones, maxima at zero
+    std::vector<unsigned long long> init((size_t)TRACE_SLOTS * 8);
+    for (size_t i = 0; i < init.size(); ++i) init[i] = (i % 8 == 0 || i % 8 == 1 || i % 8 == 3 || i % 8 == 5) ? ~0ull : 0ull;
+    CKRT(h, cudaMemcpyAsync(h->ws.trace, init.data(), init.size() * sizeof(unsigned long long), cudaMemcpyHostToDevice, st));
+    CKRT(h, cudaStreamSynchronize(st));
+    h->trace_next = 0;
+  } else {
+    h->trace_next = -1;
+  }
+  return RD_OK;
+}
+
+int redrafter_trace_read(rd_handle* h, void* stream, uint64_t* out, int32_t max_launches) {
+  if (!h || !out || max_launches < 0) return RD_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  int n = h->trace_next < 0 ? 0 : h->trace_next;
+  if (n > max_launches) n = max_launches;
+  cudaError_t e = cudaMemcpyAsync(out, h->ws.trace, (size_t)n * 8 * sizeof(unsigned long long), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return -fail(h, RD_ERR_CUDA, "trace read: %s", cudaGetErrorString(e));
+  return n;
 }
 
 int redrafter_poll(rd_handle* h, void* stream) {

@@ -6,6 +6,7 @@
 // cache.  One CTA per (row, head); each warp walks a strided share of the keys with an online
 // softmax and the warps' partial results are merged in shared memory.
 #include "rd_internal.cuh"
+#include "pdl.cuh"
 
 namespace rd {
 
@@ -15,6 +16,7 @@ template <typename T, int HD>
 __global__ void __launch_bounds__(ATT_WARPS * 32) attention_kernel(const float* __restrict__ qkv,
                                                                    const T* __restrict__ kc, const T* __restrict__ vc,
                                                                    T* __restrict__ out, RowTables rt, Dims dm) {
+  pdl_enter();
   constexpr int E = HD / 32;  // elements per lane
   __shared__ int32_t tree_slot[1024];
   __shared__ int n_tree_sh;
@@ -97,7 +99,7 @@ __global__ void __launch_bounds__(ATT_WARPS * 32) attention_kernel(const float* 
 cudaError_t launch_attention(int dtype, const float* qkv, const void* kcache, const void* vcache, void* out_t,
                              const RowTables& rt, const Dims& dm, int m_max, cudaStream_t st) {
   dim3 grid(m_max, dm.H);
-#define RD_ATT(T, HD) attention_kernel<T, HD><<<grid, ATT_WARPS * 32, 0, st>>>(qkv, (const T*)kcache, (const T*)vcache, (T*)out_t, rt, dm)
+#define RD_ATT(T, HD) launch_pdl(attention_kernel<T, HD>, grid, ATT_WARPS * 32, 0, st, qkv, (const T*)kcache, (const T*)vcache, (T*)out_t, rt, dm)
   if (dtype == RD_DTYPE_FP32) {
     if (dm.hd == 64) RD_ATT(float, 64); else if (dm.hd == 128) RD_ATT(float, 128); else return cudaErrorInvalidValue;
   } else {

@@ -8,6 +8,7 @@
 //               (score desc, flat index r*V + v asc) order; reorders histories and states and
 //               gathers the next call's inputs (e_{t+1} = E[token], s_t of the parent).
 #include "rd_internal.cuh"
+#include "pdl.cuh"
 
 namespace rd {
 
@@ -21,6 +22,7 @@ template <typename T>
 __global__ void draft_init_kernel(const T* __restrict__ emb, const int32_t* __restrict__ root, const float* __restrict__ h,
                                   T* __restrict__ x_t, float* __restrict__ x_f, T* __restrict__ sprev_t, Dims dm,
                                   int* status) {
+  pdl_enter();
   const int b = blockIdx.x;
   int g = root[b];
   if (g < 0 || g >= dm.V) {
@@ -41,13 +43,14 @@ __global__ void draft_init_kernel(const T* __restrict__ emb, const int32_t* __re
 
 cudaError_t launch_draft_init(int dtype, const void* emb, const int32_t* root, const float* h, void* x_t, float* x_f,
                               void* sprev_t, const Dims& dm, int B, int* status, cudaStream_t st) {
-  RD_DISPATCH(dtype, draft_init_kernel<T><<<B, 256, 0, st>>>((const T*)emb, root, h, (T*)x_t, x_f, (T*)sprev_t, dm, status));
+  RD_DISPATCH(dtype, launch_pdl(draft_init_kernel<T>, B, 256, 0, st, (const T*)emb, root, h, (T*)x_t, x_f, (T*)sprev_t, dm, status));
   return cudaGetLastError();
 }
 
 // h part of g_t = [s_t, h] for every beam row (constant over the calls of one step).
 template <typename T>
 __global__ void fill_h_kernel(const float* __restrict__ h, T* __restrict__ x_t, float* __restrict__ x_f, Dims dm) {
+  pdl_enter();
   const int r = blockIdx.x, b = r / dm.BW;
   for (int i = threadIdx.x; i < dm.d; i += blockDim.x) {
     const float hv = h[(size_t)b * dm.d + i];
@@ -57,7 +60,7 @@ __global__ void fill_h_kernel(const float* __restrict__ h, T* __restrict__ x_t, 
 }
 
 cudaError_t launch_fill_h(int dtype, const float* h, void* x_t, float* x_f, const Dims& dm, int B, cudaStream_t st) {
-  RD_DISPATCH(dtype, fill_h_kernel<T><<<B * dm.BW, 256, 0, st>>>(h, (T*)x_t, x_f, dm));
+  RD_DISPATCH(dtype, launch_pdl(fill_h_kernel<T>, B * dm.BW, 256, 0, st, h, (T*)x_t, x_f, dm));
   return cudaGetLastError();
 }
 
@@ -95,19 +98,31 @@ __device__ __forceinline__ Cand block_best(Cand c, Cand* sh) {
   return r;  // identical in every thread
 }
 
-__global__ void __launch_bounds__(1024) row_topk_kernel(const float* __restrict__ logits, int V, int BW,
-                                                         float* __restrict__ lse, float* __restrict__ val,
-                                                         int32_t* __restrict__ idx) {
+// One CTA per row.  The row is read once into registers (TOPK_PER_THREAD values per thread); the BW
+// selection passes then work on registers plus one block reduction each.
+constexpr int TOPK_THREADS = 1024;
+constexpr int TOPK_PER_THREAD = 32;  // V <= 32768
+
+__global__ void __launch_bounds__(TOPK_THREADS) row_topk_kernel(const float* __restrict__ logits, int V, int BW,
+                                                                 float* __restrict__ lse, float* __restrict__ val,
+                                                                 int32_t* __restrict__ idx) {
+  pdl_enter();
   __shared__ Cand sh[32];
   __shared__ float shf[32];
   const int r = blockIdx.x;
   const float* z = logits + (size_t)r * V;
-  // max, then sum of exp
+  float v[TOPK_PER_THREAD];
   Cand c{-INFINITY, 0x7fffffff};
-  for (int i = threadIdx.x; i < V; i += blockDim.x) c = cand_best(c, Cand{z[i], i});
-  Cand top = block_best(c, sh);
+#pragma unroll
+  for (int k = 0; k < TOPK_PER_THREAD; ++k) {
+    const int i = threadIdx.x + k * TOPK_THREADS;
+    v[k] = i < V ? z[i] : -INFINITY;
+    c = cand_best(c, Cand{v[k], i < V ? i : 0x7fffffff});
+  }
+  const Cand top = block_best(c, sh);
   float s = 0.f;
-  for (int i = threadIdx.x; i < V; i += blockDim.x) s += expf(z[i] - top.v);
+#pragma unroll
+  for (int k = 0; k < TOPK_PER_THREAD; ++k) s += expf(v[k] - top.v);  // exp(-inf) = 0 for the padding
   {
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
 #pragma unroll
@@ -127,9 +142,10 @@ __global__ void __launch_bounds__(1024) row_topk_kernel(const float* __restrict_
   Cand prev = top;
   for (int p = 1; p < BW; ++p) {
     Cand best{-INFINITY, 0x7fffffff};
-    for (int i = threadIdx.x; i < V; i += blockDim.x) {
-      const float v = z[i];
-      if (cand_before(prev.v, prev.i, v, i)) best = cand_best(best, Cand{v, i});
+#pragma unroll
+    for (int k = 0; k < TOPK_PER_THREAD; ++k) {
+      const int i = threadIdx.x + k * TOPK_THREADS;
+      if (i < V && cand_before(prev.v, prev.i, v[k], i)) best = cand_best(best, Cand{v[k], i});
     }
     best = block_best(best, sh);
     if (threadIdx.x == 0) {
@@ -142,13 +158,13 @@ __global__ void __launch_bounds__(1024) row_topk_kernel(const float* __restrict_
 
 cudaError_t launch_row_topk(const float* logits, int V, int BW, float* lse, float* val, int32_t* idx, int rows,
                             cudaStream_t st) {
-  row_topk_kernel<<<rows, 1024, 0, st>>>(logits, V, BW, lse, val, idx);
+  if (V > TOPK_THREADS * TOPK_PER_THREAD) return cudaErrorInvalidValue;
+  launch_pdl(row_topk_kernel, rows, TOPK_THREADS, 0, st, logits, V, BW, lse, val, idx);
   return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------- cross-row merge + reorder + gather
-// One CTA per sequence.  call == 1: the single row's top-BW become the beams.  call >= 2: best BW of
-// the BW*BW survivors.  Writes score_out[k], hist_out[k][0..call-1], and the next call's inputs
+// call == 1: the single row's top-BW become the beams.  call >= 2: best BW of the BW*BW survivors.  Writes score_out[k], hist_out[k][0..call-1], and the next call's inputs
 // sprev_t[k] = s_t of the parent (read from s_new_f with row stride ld_s; skipped for call 1, where
 // every beam keeps s_1) and e_t[k] = E[token_k].  On the last call also the public outputs.
 template <typename T>
@@ -159,16 +175,19 @@ __global__ void __launch_bounds__(256) beam_merge_kernel(int call, const float* 
                                                           const T* __restrict__ emb, const float* __restrict__ s_new_f,
                                                           int ld_s, T* __restrict__ sprev_t, T* __restrict__ e_t, Dims dm,
                                                           int32_t* __restrict__ beams_out, float* __restrict__ scores_out) {
+  pdl_enter();
+  // grid = B * BW: every CTA of a sequence repeats the (tiny) selection over the BW*BW survivors and
+  // then writes the outputs of ONE new beam, so the reorder/gather work is spread over BW CTAs.
   __shared__ Cand sh[32];
-  __shared__ int sel_parent[64], sel_tok[64];
-  __shared__ float sel_score[64];
-  const int b = blockIdx.x, BW = dm.BW, L = dm.L, V = dm.V;
+  __shared__ int sel_parent[128], sel_tok[128];
+  __shared__ float sel_score[128];
+  const int BW = dm.BW, L = dm.L, V = dm.V;
+  const int b = blockIdx.x / BW, k = blockIdx.x - b * BW;
   const int rows = call == 1 ? 1 : BW;
   const int row0 = call == 1 ? b : b * BW;
   const int n_cand = rows * BW;
-  // candidate c = (row r = c / BW, rank j = c % BW): score and flat index
   Cand prev{INFINITY, -1};
-  for (int p = 0; p < BW; ++p) {
+  for (int p = 0; p <= k; ++p) {  // beams are ranked: beam k needs the first k+1 picks only
     Cand best{-INFINITY, 0x7fffffff};
     for (int c = threadIdx.x; c < n_cand; c += blockDim.x) {
       const int r = c / BW;
@@ -187,26 +206,31 @@ __global__ void __launch_bounds__(256) beam_merge_kernel(int call, const float* 
     prev = best;
   }
   __syncthreads();
-  for (int k = threadIdx.x; k < BW; k += blockDim.x) {
-    const int orow = b * BW + k;
+  const int orow = b * BW + k;
+  const int prow = b * BW + sel_parent[k];
+  const int tok = sel_tok[k];
+  if (threadIdx.x == 0) {
     score_out[orow] = sel_score[k];
-    const int prow = b * BW + sel_parent[k];
     for (int t = 0; t < call - 1; ++t) hist_out[(size_t)orow * L + t] = hist_in[(size_t)prow * L + t];
-    hist_out[(size_t)orow * L + call - 1] = sel_tok[k];
+    hist_out[(size_t)orow * L + call - 1] = tok;
     if (call == L) {
       for (int t = 0; t < L - 1; ++t) beams_out[(size_t)orow * L + t] = hist_in[(size_t)prow * L + t];
-      beams_out[(size_t)orow * L + L - 1] = sel_tok[k];
+      beams_out[(size_t)orow * L + L - 1] = tok;
       if (scores_out) scores_out[orow] = sel_score[k];
     }
   }
   if (call < L) {
-    for (int k = 0; k < BW; ++k) {
-      const int orow = b * BW + k;
-      const T* e = emb + (size_t)sel_tok[k] * dm.d;
-      for (int i = threadIdx.x; i < dm.d; i += blockDim.x) e_t[(size_t)orow * dm.d + i] = e[i];
-      if (call > 1) {
-        const float* s = s_new_f + (size_t)(b * BW + sel_parent[k]) * ld_s;
-        for (int i = threadIdx.x; i < dm.dr; i += blockDim.x) sprev_t[(size_t)orow * dm.dr + i] = from_f<T>(s[i]);
+    // gathers with 128-bit accesses (rows are 16-byte aligned: d is a multiple of 8)
+    constexpr int EV = 16 / sizeof(T);
+    const uint4* e = reinterpret_cast<const uint4*>(emb + (size_t)tok * dm.d);
+    uint4* eo = reinterpret_cast<uint4*>(e_t + (size_t)orow * dm.d);
+    for (int i = threadIdx.x; i < dm.d / EV; i += blockDim.x) eo[i] = e[i];
+    if (call > 1) {
+      const float4* s = reinterpret_cast<const float4*>(s_new_f + (size_t)prow * ld_s);
+      T* so = sprev_t + (size_t)orow * dm.dr;
+      for (int i = threadIdx.x; i < dm.dr / 4; i += blockDim.x) {
+        const float4 v = s[i];
+        so[4 * i] = from_f<T>(v.x); so[4 * i + 1] = from_f<T>(v.y); so[4 * i + 2] = from_f<T>(v.z); so[4 * i + 3] = from_f<T>(v.w);
       }
     }
   }
@@ -216,7 +240,7 @@ cudaError_t launch_beam_merge(int dtype, int call, const float* lse, const float
                               const float* score_in, float* score_out, const int32_t* hist_in, int32_t* hist_out,
                               const void* emb, const float* s_new_f, int ld_s, void* sprev_t, void* e_t,
                               const Dims& dm, int B, int32_t* beams_out, float* scores_out, cudaStream_t st) {
-  RD_DISPATCH(dtype, beam_merge_kernel<T><<<B, 256, 0, st>>>(call, lse, val, idx, score_in, score_out, hist_in, hist_out,
+  RD_DISPATCH(dtype, launch_pdl(beam_merge_kernel<T>, B * dm.BW, 256, 0, st, call, lse, val, idx, score_in, score_out, hist_in, hist_out,
                                                            (const T*)emb, s_new_f, ld_s, (T*)sprev_t, (T*)e_t, dm,
                                                            beams_out, scores_out));
   return cudaGetLastError();

@@ -2,6 +2,7 @@
 // rotary embedding + KV-cache write, SwiGLU, row argmax, row tables.  All are bandwidth-trivial
 // (activations of at most a few MB that stay in L2); they exist to feed the projections.
 #include "rd_internal.cuh"
+#include "pdl.cuh"
 
 namespace rd {
 
@@ -31,6 +32,7 @@ __device__ __forceinline__ float block_sum(float v, float* sh) {
 template <typename T>
 __global__ void embed_kernel(const T* __restrict__ emb, const int32_t* __restrict__ tok, float* __restrict__ x, int d,
                              int V, const int32_t* __restrict__ m_total, int* status) {
+  pdl_enter();
   const int m = blockIdx.x;
   if (m >= *m_total) return;
   int t = tok[m];
@@ -44,57 +46,101 @@ __global__ void embed_kernel(const T* __restrict__ emb, const int32_t* __restric
 
 cudaError_t launch_embed(int dtype, const void* emb, const int32_t* tok, float* x, int d, int V, const int32_t* m_total,
                          int m_max, int* status, cudaStream_t st) {
-  RD_DISPATCH(dtype, embed_kernel<T><<<m_max, 256, 0, st>>>((const T*)emb, tok, x, d, V, m_total, status));
+  RD_DISPATCH(dtype, launch_pdl(embed_kernel<T>, m_max, 256, 0, st, (const T*)emb, tok, x, d, V, m_total, status));
   return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------- RMSNorm
-// y = x / sqrt(mean(x^2) + eps) * gain, one block per row.
+// y = x / sqrt(mean(x^2) + eps) * gain, one block per row.  The row is read once with 128-bit loads
+// and kept in registers between the reduction and the scaling (d <= 8192).
+constexpr int NORM_THREADS = 256;
+constexpr int NORM_MAXV = 8;
+
 template <typename T>
-__global__ void rmsnorm_kernel(const float* __restrict__ x, const T* __restrict__ gain, T* __restrict__ out_t,
-                               float* __restrict__ out_f, int d, float eps, const int32_t* __restrict__ m_total) {
+__global__ void __launch_bounds__(NORM_THREADS) rmsnorm_kernel(const float* __restrict__ x, const T* __restrict__ gain,
+                                                                T* __restrict__ out_t, float* __restrict__ out_f, int d,
+                                                                float eps, const int32_t* __restrict__ m_total) {
+  pdl_enter();
   __shared__ float sh[32];
   const int m = blockIdx.x;
   if (m >= *m_total) return;
-  const float* xr = x + (size_t)m * d;
+  const float4* xr = reinterpret_cast<const float4*>(x + (size_t)m * d);
+  const int nvec = d >> 2;
+  float4 v[NORM_MAXV];
   float ss = 0.f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) { float v = xr[i]; ss += v * v; }
+#pragma unroll
+  for (int k = 0; k < NORM_MAXV; ++k) {
+    const int i = threadIdx.x + k * NORM_THREADS;
+    if (i < nvec) {
+      v[k] = xr[i];
+      ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
+    }
+  }
   ss = block_sum(ss, sh);
   const float r = rsqrtf(ss / (float)d + eps);
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    float v = xr[i] * r * to_f<T>(gain[i]);
-    if (out_t) out_t[(size_t)m * d + i] = from_f<T>(v);
-    if (out_f) out_f[(size_t)m * d + i] = v;
+#pragma unroll
+  for (int k = 0; k < NORM_MAXV; ++k) {
+    const int i = threadIdx.x + k * NORM_THREADS;
+    if (i < nvec) {
+      const float g0 = to_f<T>(gain[4 * i]), g1 = to_f<T>(gain[4 * i + 1]), g2 = to_f<T>(gain[4 * i + 2]),
+                  g3 = to_f<T>(gain[4 * i + 3]);
+      const float y0 = v[k].x * r * g0, y1 = v[k].y * r * g1, y2 = v[k].z * r * g2, y3 = v[k].w * r * g3;
+      const size_t o = (size_t)m * d + 4 * i;
+      if (out_t) { out_t[o] = from_f<T>(y0); out_t[o + 1] = from_f<T>(y1); out_t[o + 2] = from_f<T>(y2); out_t[o + 3] = from_f<T>(y3); }
+      if (out_f) *reinterpret_cast<float4*>(out_f + o) = make_float4(y0, y1, y2, y3);
+    }
   }
 }
 
 cudaError_t launch_rmsnorm(int dtype, const float* x, const void* gain, void* out_t, float* out_f32, int d, float eps,
                            const int32_t* m_total, int m_max, cudaStream_t st) {
-  RD_DISPATCH(dtype, rmsnorm_kernel<T><<<m_max, 256, 0, st>>>(x, (const T*)gain, (T*)out_t, out_f32, d, eps, m_total));
+  if (d > 4 * NORM_THREADS * NORM_MAXV || (d & 3)) return cudaErrorInvalidValue;
+  RD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T>, m_max, NORM_THREADS, 0, st, x, (const T*)gain, (T*)out_t, out_f32, d, eps, m_total));
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- rotary table
+// cos/sin of pos * theta^(-2i/hd) for every row of the pass, computed once per forward (all layers
+// share it).  The angle is formed in double: positions reach several thousand and its rounding
+// error in single precision would scale with them.
+__global__ void rope_table_kernel(const int32_t* __restrict__ pos, float2* __restrict__ table, int half, float theta,
+                                  const int32_t* __restrict__ m_total) {
+  pdl_enter();
+  const int m = blockIdx.x;
+  if (m >= *m_total) return;
+  const double l2t = log2((double)theta);
+  for (int i = threadIdx.x; i < half; i += blockDim.x) {
+    const double ang = (double)pos[m] * exp2(-((double)i / half) * l2t);
+    double sd, cd;
+    sincos(ang, &sd, &cd);
+    table[(size_t)m * half + i] = make_float2((float)cd, (float)sd);
+  }
+}
+
+cudaError_t launch_rope_table(const int32_t* pos, float* table, int hd, float theta, const int32_t* m_total, int m_max,
+                              cudaStream_t st) {
+  launch_pdl(rope_table_kernel, m_max, 64, 0, st, pos, reinterpret_cast<float2*>(table), hd / 2, theta, m_total);
   return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------- rotary embedding + KV write
 // qkv: [M][3d] fp32 (Q | K | V).  Q is rotated in place; rotated K and V go to the cache slot of
-// the row.  Pairing (i, i + hd/2), angle = pos * theta^(-2i/hd) (computed in double: positions
-// reach several thousand and the angle's rounding error would otherwise scale with them).
+// the row.  Pairing (i, i + hd/2).
 template <typename T>
-__global__ void rope_kv_kernel(float* __restrict__ qkv, T* __restrict__ kc, T* __restrict__ vc, RowTables rt, Dims dm,
-                               int* status) {
+__global__ void rope_kv_kernel(float* __restrict__ qkv, T* __restrict__ kc, T* __restrict__ vc,
+                               const float2* __restrict__ table, RowTables rt, Dims dm, int* status) {
+  pdl_enter();
   const int m = blockIdx.x;
   if (m >= *rt.m_total) return;
-  const int b = rt.seq[m], slot = rt.slot[m], pos = rt.pos[m];
+  const int b = rt.seq[m], slot = rt.slot[m];
   const int d = dm.d, hd = dm.hd, half = hd >> 1;
   const bool slot_ok = slot >= 0 && slot < dm.max_ctx;
   if (!slot_ok && threadIdx.x == 0) atomicOr(status, DEV_ERR_CAPACITY);
   float* row = qkv + (size_t)m * 3 * d;
-  const double l2t = log2((double)dm.theta);
   for (int idx = threadIdx.x; idx < dm.H * half; idx += blockDim.x) {
     const int h = idx / half, i = idx - h * half;
-    const double ang = (double)pos * exp2(-(2.0 * i / hd) * l2t);
-    double sd, cd;
-    sincos(ang, &sd, &cd);
-    const float c = (float)cd, s = (float)sd;
+    const float2 cs = table[(size_t)m * half + i];
+    const float c = cs.x, s = cs.y;
     const int o = h * hd + i;
     const float q1 = row[o], q2 = row[o + half];
     row[o] = q1 * c - q2 * s;
@@ -110,15 +156,17 @@ __global__ void rope_kv_kernel(float* __restrict__ qkv, T* __restrict__ kc, T* _
   }
 }
 
-cudaError_t launch_rope_kv(int dtype, float* qkv, void* kcache, void* vcache, const RowTables& rt, const Dims& dm,
-                           int m_max, int* status, cudaStream_t st) {
-  RD_DISPATCH(dtype, rope_kv_kernel<T><<<m_max, 256, 0, st>>>(qkv, (T*)kcache, (T*)vcache, rt, dm, status));
+cudaError_t launch_rope_kv(int dtype, float* qkv, void* kcache, void* vcache, const float* table, const RowTables& rt,
+                           const Dims& dm, int m_max, int* status, cudaStream_t st) {
+  RD_DISPATCH(dtype, launch_pdl(rope_kv_kernel<T>, m_max, 256, 0, st, qkv, (T*)kcache, (T*)vcache,
+                                                            reinterpret_cast<const float2*>(table), rt, dm, status));
   return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------- SwiGLU
 template <typename T>
 __global__ void swiglu_kernel(const float* __restrict__ gu, T* __restrict__ out, int F, const int32_t* __restrict__ m_total) {
+  pdl_enter();
   const int m = blockIdx.y;
   if (m >= *m_total) return;
   const int f = blockIdx.x * blockDim.x + threadIdx.x;
@@ -130,13 +178,14 @@ __global__ void swiglu_kernel(const float* __restrict__ gu, T* __restrict__ out,
 cudaError_t launch_swiglu(int dtype, const float* gu, void* out_t, int F, const int32_t* m_total, int m_max,
                           cudaStream_t st) {
   dim3 grid((F + 255) / 256, m_max);
-  RD_DISPATCH(dtype, swiglu_kernel<T><<<grid, 256, 0, st>>>(gu, (T*)out_t, F, m_total));
+  RD_DISPATCH(dtype, launch_pdl(swiglu_kernel<T>, grid, 256, 0, st, gu, (T*)out_t, F, m_total));
   return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------- row argmax (lowest index on ties)
 __global__ void argmax_rows_kernel(const float* __restrict__ logits, int V, int32_t* __restrict__ out,
                                    const int32_t* __restrict__ out_index, const int32_t* __restrict__ m_total) {
+  pdl_enter();
   __shared__ float sv[32];
   __shared__ int si[32];
   const int m = blockIdx.x;
@@ -173,13 +222,14 @@ __global__ void argmax_rows_kernel(const float* __restrict__ logits, int V, int3
 
 cudaError_t launch_argmax_rows(const float* logits, int V, int32_t* out, const int32_t* out_index,
                                const int32_t* m_total, int m_max, cudaStream_t st) {
-  argmax_rows_kernel<<<m_max, 512, 0, st>>>(logits, V, out, out_index, m_total);
+  launch_pdl(argmax_rows_kernel, m_max, 512, 0, st, logits, V, out, out_index, m_total);
   return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------- compact rows -> padded [B][NMAX] layout
 __global__ void scatter_rows_kernel(const float* __restrict__ src, int width, float* __restrict__ dst,
                                     const int32_t* __restrict__ row_out_index, const int32_t* __restrict__ m_total) {
+  pdl_enter();
   const int m = blockIdx.y;
   if (m >= *m_total) return;
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -189,29 +239,31 @@ __global__ void scatter_rows_kernel(const float* __restrict__ src, int width, fl
 cudaError_t launch_scatter_rows(const float* src, int width, float* dst, const int32_t* row_out_index,
                                 const int32_t* m_total, int m_max, cudaStream_t st) {
   dim3 grid((width + 255) / 256, m_max);
-  scatter_rows_kernel<<<grid, 256, 0, st>>>(src, width, dst, row_out_index, m_total);
+  launch_pdl(scatter_rows_kernel, grid, 256, 0, st, src, width, dst, row_out_index, m_total);
   return cudaGetLastError();
 }
 
 template <typename T>
 __global__ void cast_rows_kernel(const float* __restrict__ src, T* __restrict__ dst, int n) {
+  pdl_enter();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) dst[i] = from_f<T>(src[i]);
 }
 
 cudaError_t launch_cast_rows(int dtype, const float* src, void* dst, int n, cudaStream_t st) {
-  RD_DISPATCH(dtype, cast_rows_kernel<T><<<(n + 255) / 256, 256, 0, st>>>(src, (T*)dst, n));
+  RD_DISPATCH(dtype, launch_pdl(cast_rows_kernel<T>, (n + 255) / 256, 256, 0, st, src, (T*)dst, n));
   return cudaGetLastError();
 }
 
 __global__ void fill_i32_kernel(int32_t* p, int32_t v, int n) {
+  pdl_enter();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) p[i] = v;
 }
 
 cudaError_t launch_fill_i32(int32_t* p, int32_t v, int n, cudaStream_t st) {
   if (n <= 0) return cudaSuccess;
-  fill_i32_kernel<<<(n + 255) / 256, 256, 0, st>>>(p, v, n);
+  launch_pdl(fill_i32_kernel, (n + 255) / 256, 256, 0, st, p, v, n);
   return cudaGetLastError();
 }
 
@@ -221,7 +273,9 @@ cudaError_t launch_fill_i32(int32_t* p, int32_t v, int n, cudaStream_t st) {
 // provisional cache slot ctx_b + n, attends cache [0, ctx_b) plus its mask row.
 __global__ void build_rows_tree_kernel(rd_packed pk, const int32_t* __restrict__ ctx, int32_t* row_tok, int32_t* row_seq,
                                        int32_t* row_pos, int32_t* row_slot, int32_t* row_ncache, int32_t* row_local,
-                                       int32_t* row_out_index, int32_t* m_total, Dims dm, int B, int* status) {
+                                       int32_t* row_out_index, int32_t* seq_off, int32_t* m_total, Dims dm, int B,
+                                       int* status) {
+  pdl_enter();
   extern __shared__ int32_t off[];  // [B+1]
   if (threadIdx.x == 0) {
     int acc = 0;
@@ -235,6 +289,7 @@ __global__ void build_rows_tree_kernel(rd_packed pk, const int32_t* __restrict__
     *m_total = acc;
   }
   __syncthreads();
+  for (int b = threadIdx.x; b <= B; b += blockDim.x) seq_off[b] = off[b];
   for (int idx = threadIdx.x; idx < B * dm.NMAX; idx += blockDim.x) {
     const int b = idx / dm.NMAX, n = idx - b * dm.NMAX;
     if (n >= off[b + 1] - off[b]) continue;
@@ -253,22 +308,24 @@ __global__ void build_rows_tree_kernel(rd_packed pk, const int32_t* __restrict__
 
 cudaError_t launch_build_rows_tree(const rd_packed& pk, const int32_t* ctx, int32_t* row_tok, int32_t* row_seq,
                                    int32_t* row_pos, int32_t* row_slot, int32_t* row_ncache, int32_t* row_local,
-                                   int32_t* row_out_index, int32_t* m_total, const Dims& dm, int B, int* status,
-                                   cudaStream_t st) {
-  build_rows_tree_kernel<<<1, 1024, (B + 1) * sizeof(int32_t), st>>>(pk, ctx, row_tok, row_seq, row_pos, row_slot,
-                                                                    row_ncache, row_local, row_out_index, m_total, dm,
-                                                                    B, status);
+                                   int32_t* row_out_index, int32_t* seq_off, int32_t* m_total, const Dims& dm, int B,
+                                   int* status, cudaStream_t st) {
+  launch_pdl(build_rows_tree_kernel, 1, 1024, (B + 1) * sizeof(int32_t), st, pk, ctx, row_tok, row_seq, row_pos, row_slot,
+                                                                    row_ncache, row_local, row_out_index, seq_off,
+                                                                    m_total, dm, B, status);
   return cudaGetLastError();
 }
 
 // Autoregressive step: one row per sequence, the root token at position ctx_b.
 __global__ void build_rows_ar_kernel(const int32_t* __restrict__ root, const int32_t* __restrict__ ctx, int32_t* row_tok,
                                      int32_t* row_seq, int32_t* row_pos, int32_t* row_slot, int32_t* row_ncache,
-                                     int32_t* row_local, int32_t* row_out_index, int32_t* m_total, Dims dm, int B,
-                                     int* status) {
+                                     int32_t* row_local, int32_t* row_out_index, int32_t* seq_off, int32_t* m_total,
+                                     Dims dm, int B, int* status) {
+  pdl_enter();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b == 0) *m_total = B;
+  if (b == 0) { *m_total = B; seq_off[B] = B; }
   if (b >= B) return;
+  seq_off[b] = b;
   int t = root[b];
   if (t < 0 || t >= dm.V) { atomicOr(status, DEV_ERR_TOKEN_RANGE); t = min(max(t, 0), dm.V - 1); }
   row_tok[b] = t;
@@ -282,16 +339,17 @@ __global__ void build_rows_ar_kernel(const int32_t* __restrict__ root, const int
 
 cudaError_t launch_build_rows_ar(const int32_t* root, const int32_t* ctx, int32_t* row_tok, int32_t* row_seq,
                                  int32_t* row_pos, int32_t* row_slot, int32_t* row_ncache, int32_t* row_local,
-                                 int32_t* row_out_index, int32_t* m_total, const Dims& dm, int B, int* status,
-                                 cudaStream_t st) {
-  build_rows_ar_kernel<<<(B + 127) / 128, 128, 0, st>>>(root, ctx, row_tok, row_seq, row_pos, row_slot, row_ncache,
-                                                        row_local, row_out_index, m_total, dm, B, status);
+                                 int32_t* row_out_index, int32_t* seq_off, int32_t* m_total, const Dims& dm, int B,
+                                 int* status, cudaStream_t st) {
+  launch_pdl(build_rows_ar_kernel, (B + 127) / 128, 128, 0, st, root, ctx, row_tok, row_seq, row_pos, row_slot, row_ncache,
+                                                        row_local, row_out_index, seq_off, m_total, dm, B, status);
   return cudaGetLastError();
 }
 
 // After an AR forward: ctx += 1, root = greedy token, h = hidden of the row.
 __global__ void ar_finish_kernel(const int32_t* __restrict__ argmax_c, const float* __restrict__ hidden_c, int32_t* ctx,
                                  int32_t* root, float* h, int32_t* token_out, int d) {
+  pdl_enter();
   const int b = blockIdx.x;
   for (int i = threadIdx.x; i < d; i += blockDim.x) h[(size_t)b * d + i] = hidden_c[(size_t)b * d + i];
   if (threadIdx.x == 0) {
@@ -303,13 +361,14 @@ __global__ void ar_finish_kernel(const int32_t* __restrict__ argmax_c, const flo
 
 cudaError_t launch_ar_finish(const int32_t* argmax_c, const float* hidden_c, int32_t* ctx, int32_t* root, float* h,
                              int32_t* token_out, const Dims& dm, int B, cudaStream_t st) {
-  ar_finish_kernel<<<B, 256, 0, st>>>(argmax_c, hidden_c, ctx, root, h, token_out, dm.d);
+  launch_pdl(ar_finish_kernel, B, 256, 0, st, argmax_c, hidden_c, ctx, root, h, token_out, dm.d);
   return cudaGetLastError();
 }
 
 // After a prefill pass: sequences whose last prompt token was in this pass take its hidden state.
 __global__ void prefill_finish_kernel(const float* __restrict__ hidden_c, const int32_t* __restrict__ last_row, float* h,
                                       int d) {
+  pdl_enter();
   const int b = blockIdx.x;
   const int r = last_row[b];
   if (r < 0) return;
@@ -318,7 +377,7 @@ __global__ void prefill_finish_kernel(const float* __restrict__ hidden_c, const 
 
 cudaError_t launch_prefill_finish(const float* hidden_c, const int32_t* last_row, float* h, int d, int B,
                                   cudaStream_t st) {
-  prefill_finish_kernel<<<B, 256, 0, st>>>(hidden_c, last_row, h, d);
+  launch_pdl(prefill_finish_kernel, B, 256, 0, st, hidden_c, last_row, h, d);
   return cudaGetLastError();
 }
 

@@ -6,6 +6,7 @@
 // stream: one warp owns one weight row, reads it once with 128-bit loads and keeps MT running
 // sums, so the weight is read exactly once per MT rows.
 #include "rd_internal.cuh"
+#include "pdl.cuh"
 #include "epilogue.cuh"
 
 namespace rd {
@@ -44,6 +45,7 @@ template <> struct Vec<__nv_bfloat16> {
 template <typename T, int MT>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ A, int lda, const T* __restrict__ W, int N,
                                                         int K, const int32_t* __restrict__ m_total, Epilogue ep) {
+  pdl_enter();
   constexpr int VN = Vec<T>::N;
   const int M = *m_total;
   const int m0 = blockIdx.y * MT;
@@ -85,16 +87,16 @@ cudaError_t launch_gemm_simt(int dtype, const void* A, int lda, const void* W, i
   if (m_max <= 2) {
     dim3 grid((N + 7) / 8, (m_max + 1) / 2);
     if (dtype == RD_DTYPE_FP32)
-      gemm_simt_kernel<float, 2><<<grid, 256, 0, st>>>((const float*)A, lda, (const float*)W, N, K, m_total, ep);
+      launch_pdl(gemm_simt_kernel<float, 2>, grid, 256, 0, st, (const float*)A, lda, (const float*)W, N, K, m_total, ep);
     else
-      gemm_simt_kernel<__nv_bfloat16, 2><<<grid, 256, 0, st>>>((const __nv_bfloat16*)A, lda, (const __nv_bfloat16*)W, N,
+      launch_pdl(gemm_simt_kernel<__nv_bfloat16, 2>, grid, 256, 0, st, (const __nv_bfloat16*)A, lda, (const __nv_bfloat16*)W, N,
                                                                 K, m_total, ep);
   } else {
     dim3 grid((N + 7) / 8, (m_max + 7) / 8);
     if (dtype == RD_DTYPE_FP32)
-      gemm_simt_kernel<float, 8><<<grid, 256, 0, st>>>((const float*)A, lda, (const float*)W, N, K, m_total, ep);
+      launch_pdl(gemm_simt_kernel<float, 8>, grid, 256, 0, st, (const float*)A, lda, (const float*)W, N, K, m_total, ep);
     else
-      gemm_simt_kernel<__nv_bfloat16, 8><<<grid, 256, 0, st>>>((const __nv_bfloat16*)A, lda, (const __nv_bfloat16*)W, N,
+      launch_pdl(gemm_simt_kernel<__nv_bfloat16, 8>, grid, 256, 0, st, (const __nv_bfloat16*)A, lda, (const __nv_bfloat16*)W, N,
                                                                 K, m_total, ep);
   }
   return cudaGetLastError();

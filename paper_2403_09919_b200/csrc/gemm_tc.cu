@@ -25,6 +25,7 @@
 #include <cuda.h>
 
 #include "epilogue.cuh"
+#include "pdl.cuh"
 #include "rd_internal.cuh"
 
 namespace rd {
@@ -45,6 +46,7 @@ struct TcParams {
   float* partial;     // [2 * gridDim.x][mt * 128]
   int32_t* counters;  // [n_tiles * m_tiles_max], zero between launches
   int32_t* status;
+  unsigned long long* trace;  // 8 timestamps of this launch (see redrafter_trace_read) or nullptr
   Epilogue ep;
 };
 
@@ -144,6 +146,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
                                                                  const __grid_constant__ CUtensorMap map_a,
                                                                  const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
+  pdl_launch_dependents();  // the next kernel may start its own prologue now
+  if (p.trace && threadIdx.x == 0) atomicMin(p.trace + 0, globaltimer());   // first CTA entered
   // leave at once when an earlier launch already timed out; one thread reads the flag so that the
   // whole CTA takes the same branch
   __shared__ int skip_launch;
@@ -152,8 +156,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
   if (skip_launch) return;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int M = *p.m_total;
-  const int m_tiles = (M + p.mt - 1) / p.mt;
+  // With a single row tile the work split does not depend on the row count, so the weight stream can
+  // start before the preceding kernels have finished (they produce the activations and the row count).
+  const bool early = (p.m_tiles_max == 1);
+  if (!early) pdl_wait();
+  const int m_tiles = early ? 1 : (*p.m_total + p.mt - 1) / p.mt;
   const long long G = gridDim.x;
   const long long U = (long long)p.n_tiles * m_tiles * p.nkb;
   const long long u0 = range_begin(blockIdx.x, U, G), u1 = range_begin(blockIdx.x + 1, U, G);
@@ -195,24 +202,37 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
   if (warp == 0) {
     // ===================== TMA producer =====================
     if (lane == 0 && u0 < u1) {
-      uint32_t it = 0;
+      // iteration i of this CTA = unit u0 + i = (tile, k-block) in tile-major order
+      const uint32_t n_it = (uint32_t)(u1 - u0);
+      const uint32_t pre = early ? min(n_it, (uint32_t)p.stages) : 0u;
+      auto issue_w = [&](uint32_t i) {
+        const long long u = u0 + i;
+        const int t = (int)(u / p.nkb), kb = (int)(u - (long long)t * p.nkb);
+        const int s = i % p.stages;
+        mbar_expect_tx(full_bar(s), stage_bytes);
+        tma_load_2d(base + s * stage_bytes, &map_w, full_bar(s), kb * TILE_K, (t / m_tiles) * TILE_N);
+      };
+      auto issue_a = [&](uint32_t i) {
+        const long long u = u0 + i;
+        const int t = (int)(u / p.nkb), kb = (int)(u - (long long)t * p.nkb);
+        const int s = i % p.stages;
+        const int m_tile = t - (t / m_tiles) * m_tiles;
+        for (int j = 0; j < p.mt / A_BOX_ROWS; ++j)
+          tma_load_2d(base + s * stage_bytes + W_STAGE_BYTES + j * A_BOX_BYTES, &map_a, full_bar(s), kb * TILE_K,
+                      m_tile * p.mt + j * A_BOX_ROWS);
+      };
+      // weights of the first ring-full of k-blocks do not depend on the preceding kernels
+      for (uint32_t i = 0; i < pre; ++i) issue_w(i);
+      if (early) pdl_wait();
+      if (p.trace) { atomicMin(p.trace + 1, globaltimer()); atomicMax(p.trace + 2, globaltimer()); }   // dependency resolved
+      for (uint32_t i = 0; i < pre; ++i) issue_a(i);
       bool ok = true;
-      for (long long u = u0; u < u1 && ok;) {
-        const int t = (int)(u / p.nkb), kb0 = (int)(u - (long long)t * p.nkb);
-        const int kb1 = (int)min((long long)p.nkb, kb0 + (u1 - u));
-        const int n_tile = t / m_tiles, m_tile = t - n_tile * m_tiles;
-        for (int kb = kb0; kb < kb1; ++kb, ++it) {
-          const int s = it % p.stages;
-          const uint32_t ph = (it / p.stages) & 1u;
-          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-          const uint32_t dst = base + s * stage_bytes;
-          mbar_expect_tx(full_bar(s), stage_bytes);
-          tma_load_2d(dst, &map_w, full_bar(s), kb * TILE_K, n_tile * TILE_N);
-          for (int j = 0; j < p.mt / A_BOX_ROWS; ++j)
-            tma_load_2d(dst + W_STAGE_BYTES + j * A_BOX_BYTES, &map_a, full_bar(s), kb * TILE_K,
-                        m_tile * p.mt + j * A_BOX_ROWS);
-        }
-        u += kb1 - kb0;
+      for (uint32_t i = pre; i < n_it; ++i) {
+        const int s = i % p.stages;
+        const uint32_t ph = (i / p.stages) & 1u;
+        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        issue_w(i);
+        issue_a(i);
       }
       if (!ok) {  // give the copies already issued time to land before the CTA's shared memory is released
         const unsigned long long t0 = globaltimer();
@@ -247,9 +267,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
         if (ok) umma_commit(tfull_bar(a));
         u += kb1 - kb0;
       }
+      if (p.trace) { atomicMin(p.trace + 3, globaltimer()); atomicMax(p.trace + 4, globaltimer()); }   // all MMAs issued
     }
   } else {
     // ===================== epilogue (warps 2..5) =====================
+    if (early) pdl_wait();                  // residual, addend and the row count come from preceding kernels
+    const int M = *p.m_total;
     const int q = warp & 3;                 // TMEM lane quarter this warp may read
     const int row = q * 32 + lane;          // weight row inside the tile
     const int et = threadIdx.x - 64;        // 0..127
@@ -275,11 +298,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
         uint32_t r[16];
         tmem_ld16(taddr + c0, r);
         if (complete) {
+          float v[16];
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int m = m_base + c0 + j;
-            if (m < M && n < p.N) apply_epilogue<__nv_bfloat16>(p.ep, m, n, __uint_as_float(r[j]));
-          }
+          for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
+          if (n < p.N) apply_epilogue16<__nv_bfloat16>(p.ep, m_base + c0, M, n, v);
         } else {
 #pragma unroll
           for (int j = 0; j < 16; ++j) my_partial[(size_t)(c0 + j) * TILE_N + row] = __uint_as_float(r[j]);
@@ -303,23 +325,30 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
         epi_bar_sync();
         if (*last_flag) {
           __threadfence();
+          // address of contributor c's partial for this tile (nullptr for a CTA with an empty range)
+          auto partial_of = [&](int c) -> const float* {
+            const long long cb = range_begin(c, U, G), ce = range_begin(c + 1, U, G);
+            if (cb >= ce) return nullptr;
+            const int slot = (cb / p.nkb == t) ? 0 : 1;
+            return p.partial + ((size_t)c * 2 + slot) * ((size_t)p.mt * TILE_N) + row;
+          };
           for (int c0 = 0; c0 < p.mt; c0 += 16) {
             float acc[16];
 #pragma unroll
             for (int j = 0; j < 16; ++j) acc[j] = 0.f;
-            for (int c = c_first; c <= c_last; ++c) {
-              const long long cb = range_begin(c, U, G), ce = range_begin(c + 1, U, G);
-              if (cb >= ce) continue;
-              const int slot = (cb / p.nkb == t) ? 0 : 1;
-              const float* pp = p.partial + ((size_t)c * 2 + slot) * ((size_t)p.mt * TILE_N) + (size_t)c0 * TILE_N + row;
+            // two contributors per round so that 32 loads are in flight; the sums stay in CTA order
+            for (int c = c_first; c <= c_last; c += 2) {
+              const float* pa = partial_of(c);
+              const float* pb = (c + 1 <= c_last) ? partial_of(c + 1) : nullptr;
+              float ta[16], tb[16];
 #pragma unroll
-              for (int j = 0; j < 16; ++j) acc[j] += __ldcg(pp + (size_t)j * TILE_N);
-            }
+              for (int j = 0; j < 16; ++j) ta[j] = pa ? __ldcg(pa + (size_t)(c0 + j) * TILE_N) : 0.f;
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const int m = m_base + c0 + j;
-              if (m < M && n < p.N) apply_epilogue<__nv_bfloat16>(p.ep, m, n, acc[j]);
+              for (int j = 0; j < 16; ++j) tb[j] = pb ? __ldcg(pb + (size_t)(c0 + j) * TILE_N) : 0.f;
+#pragma unroll
+              for (int j = 0; j < 16; ++j) acc[j] = (acc[j] + ta[j]) + tb[j];
             }
+            if (n < p.N) apply_epilogue16<__nv_bfloat16>(p.ep, m_base + c0, M, n, acc);
           }
         }
         epi_bar_sync();  // last_flag is rewritten by the next cut segment
@@ -331,6 +360,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
   // ---- teardown: everyone meets, then the allocating warp frees the TMEM columns
   tc_fence_before();
   __syncthreads();
+  if (p.trace && threadIdx.x == 0) { atomicMin(p.trace + 5, globaltimer()); atomicMax(p.trace + 6, globaltimer()); }   // CTA done
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
@@ -403,7 +433,7 @@ cudaError_t tc_prepare(int* smem_limit_out) {
 
 cudaError_t launch_gemm_tc(const void* map_w, const void* map_a, int N, int K, const int32_t* m_total, int m_max,
                            const Epilogue& ep, float* partial, int32_t* counters, int32_t* status, int grid,
-                           int smem_limit, cudaStream_t st) {
+                           int smem_limit, unsigned long long* trace, cudaStream_t st) {
   if (m_max <= 0) return cudaSuccess;
   TcParams p;
   p.N = N; p.K = K; p.nkb = (K + TILE_K - 1) / TILE_K; p.n_tiles = (N + TILE_N - 1) / TILE_N;
@@ -418,9 +448,9 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* map_a, int N, int K, c
   int cols = 32;
   while (cols < 2 * p.mt) cols <<= 1;
   p.tmem_cols = cols;
-  p.m_total = m_total; p.partial = partial; p.counters = counters; p.status = status; p.ep = ep;
+  p.m_total = m_total; p.partial = partial; p.counters = counters; p.status = status; p.ep = ep; p.trace = trace;
   const size_t smem = (size_t)stages * stage_bytes + overhead;
-  gemm_tc_kernel<<<grid, NUM_THREADS, smem, st>>>(*(const CUtensorMap*)map_w, *(const CUtensorMap*)map_a, p);
+  launch_pdl(gemm_tc_kernel, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, *(const CUtensorMap*)map_a, p);
   return cudaGetLastError();
 }
 

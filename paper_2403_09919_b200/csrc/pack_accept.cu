@@ -2,6 +2,7 @@
 // compaction (Section 3.4).  Integer work on at most a few thousand entries per sequence: one CTA
 // per sequence, everything staged in shared memory, no host involvement.
 #include "rd_internal.cuh"
+#include "pdl.cuh"
 
 namespace rd {
 
@@ -15,6 +16,7 @@ constexpr int PACK_MAX_ENTRIES = 1024;
 
 __global__ void __launch_bounds__(1024) pack_kernel(const int32_t* __restrict__ beams, const int32_t* __restrict__ root,
                                                      const int32_t* __restrict__ ctx, rd_packed out, Dims dm, int no_tree) {
+  pdl_enter();
   __shared__ int32_t tok[PACK_MAX_ENTRIES];
   __shared__ int32_t owner[PACK_MAX_ENTRIES];
   __shared__ int32_t scan[PACK_MAX_ENTRIES];
@@ -92,7 +94,7 @@ __global__ void __launch_bounds__(1024) pack_kernel(const int32_t* __restrict__ 
 
 cudaError_t launch_pack(const int32_t* beams, const int32_t* root, const int32_t* ctx, const rd_packed& out,
                         const Dims& dm, int B, int no_tree, cudaStream_t st) {
-  pack_kernel<<<B, 1024, 0, st>>>(beams, root, ctx, out, dm, no_tree);
+  launch_pdl(pack_kernel, B, 1024, 0, st, beams, root, ctx, out, dm, no_tree);
   return cudaGetLastError();
 }
 
@@ -105,6 +107,7 @@ __global__ void __launch_bounds__(256) accept_kernel(const int32_t* __restrict__
                                                       int32_t* ctx, int32_t* root, float* h, rd_accept_out out,
                                                       int32_t* n_accept_ws, int32_t* best_ws, int32_t* ctx_prev, Dims dm,
                                                       int* status) {
+  pdl_enter();
   __shared__ int sh_a[8], sh_i[8];
   __shared__ int s_a, s_best, s_node;
   const int b = blockIdx.x, BW = dm.BW, L = dm.L, C = L + 1;
@@ -160,6 +163,7 @@ __global__ void __launch_bounds__(256) compact_kv_kernel(T* __restrict__ kv, rd_
                                                           const int32_t* __restrict__ n_accept,
                                                           const int32_t* __restrict__ best,
                                                           const int32_t* __restrict__ ctx_prev, Dims dm, int* status) {
+  pdl_enter();
   const int b = blockIdx.x, plane = blockIdx.y;  // plane = layer*2 + {0:K, 1:V}
   const int a = n_accept[b];
   if (a <= 0) return;
@@ -188,15 +192,15 @@ cudaError_t launch_accept(int dtype, const int32_t* beams, const rd_packed& pk, 
                           const float* hidden, void* kcache, int32_t* ctx, int32_t* root, float* h,
                           const rd_accept_out& out, int32_t* n_accept_ws, int32_t* best_ws, int32_t* ctx_prev,
                           const Dims& dm, int B, int* status, cudaStream_t st) {
-  accept_kernel<<<B, 256, 0, st>>>(beams, pk, argmax, hidden, ctx, root, h, out, n_accept_ws, best_ws, ctx_prev, dm,
+  launch_pdl(accept_kernel, B, 256, 0, st, beams, pk, argmax, hidden, ctx, root, h, out, n_accept_ws, best_ws, ctx_prev, dm,
                                    status);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   dim3 grid(B, dm.n_layers * 2);
   if (dtype == RD_DTYPE_FP32)
-    compact_kv_kernel<float><<<grid, 256, 0, st>>>((float*)kcache, pk, n_accept_ws, best_ws, ctx_prev, dm, status);
+    launch_pdl(compact_kv_kernel<float>, grid, 256, 0, st, (float*)kcache, pk, n_accept_ws, best_ws, ctx_prev, dm, status);
   else
-    compact_kv_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((__nv_bfloat16*)kcache, pk, n_accept_ws, best_ws, ctx_prev,
+    launch_pdl(compact_kv_kernel<__nv_bfloat16>, grid, 256, 0, st, (__nv_bfloat16*)kcache, pk, n_accept_ws, best_ws, ctx_prev,
                                                            dm, status);
   return cudaGetLastError();
 }

@@ -73,16 +73,25 @@ size_t tc_counter_ints(int N, int m_max);
 cudaError_t tc_prepare(int* smem_limit_out);
 cudaError_t launch_gemm_tc(const void* map_w, const void* map_a, int N, int K, const int32_t* m_total, int m_max,
                            const Epilogue& ep, float* partial, int32_t* counters, int32_t* status, int grid,
-                           int smem_limit, cudaStream_t st);
+                           int smem_limit, unsigned long long* trace, cudaStream_t st);
 
 cudaError_t launch_embed(int dtype, const void* emb, const int32_t* tok, float* x, int d, int V, const int32_t* m_total,
                          int m_max, int* status, cudaStream_t st);
 cudaError_t launch_rmsnorm(int dtype, const float* x, const void* gain, void* out_t, float* out_f32, int d, float eps,
                            const int32_t* m_total, int m_max, cudaStream_t st);
-cudaError_t launch_rope_kv(int dtype, float* qkv, void* kcache, void* vcache, const RowTables& rt, const Dims& dm,
-                           int m_max, int* status, cudaStream_t st);
+cudaError_t launch_rope_table(const int32_t* pos, float* table, int hd, float theta, const int32_t* m_total, int m_max,
+                              cudaStream_t st);
+cudaError_t launch_rope_kv(int dtype, float* qkv, void* kcache, void* vcache, const float* table, const RowTables& rt,
+                           const Dims& dm, int m_max, int* status, cudaStream_t st);
 cudaError_t launch_attention(int dtype, const float* qkv, const void* kcache, const void* vcache, void* out_t,
                              const RowTables& rt, const Dims& dm, int m_max, cudaStream_t st);
+// Tensor-core attention (bf16): KV tiles staged through shared memory, split over the keys.
+size_t attn_tc_scratch_floats(int blocks, int n_splits, int hd);
+int attn_tc_rows_per_block();
+cudaError_t attn_tc_prepare(int hd, int MW);
+cudaError_t launch_attention_tc(const float* qkv, const void* kcache, const void* vcache, void* out, const RowTables& rt,
+                                const int32_t* seq_off, const Dims& dm, int n_seq, int row_blocks, int n_splits,
+                                float* scratch, int32_t* counters, cudaStream_t st);
 cudaError_t launch_swiglu(int dtype, const float* gu, void* out_t, int F, const int32_t* m_total, int m_max,
                           cudaStream_t st);
 cudaError_t launch_argmax_rows(const float* logits, int V, int32_t* out, const int32_t* out_index,
@@ -104,12 +113,12 @@ cudaError_t launch_pack(const int32_t* beams, const int32_t* root, const int32_t
                         const Dims& dm, int B, int no_tree, cudaStream_t st);
 cudaError_t launch_build_rows_tree(const rd_packed& pk, const int32_t* ctx, int32_t* row_tok, int32_t* row_seq,
                                    int32_t* row_pos, int32_t* row_slot, int32_t* row_ncache, int32_t* row_local,
-                                   int32_t* row_out_index, int32_t* m_total, const Dims& dm, int B, int* status,
-                                   cudaStream_t st);
+                                   int32_t* row_out_index, int32_t* seq_off, int32_t* m_total, const Dims& dm, int B,
+                                   int* status, cudaStream_t st);
 cudaError_t launch_build_rows_ar(const int32_t* root, const int32_t* ctx, int32_t* row_tok, int32_t* row_seq,
                                  int32_t* row_pos, int32_t* row_slot, int32_t* row_ncache, int32_t* row_local,
-                                 int32_t* row_out_index, int32_t* m_total, const Dims& dm, int B, int* status,
-                                 cudaStream_t st);
+                                 int32_t* row_out_index, int32_t* seq_off, int32_t* m_total, const Dims& dm, int B,
+                                 int* status, cudaStream_t st);
 cudaError_t launch_scatter_rows(const float* src, int width, float* dst, const int32_t* row_out_index,
                                 const int32_t* m_total, int m_max, cudaStream_t st);
 cudaError_t launch_cast_rows(int dtype, const float* src, void* dst, int n, cudaStream_t st);

@@ -206,29 +206,51 @@ def test_batched_ragged_many_rows():
         assert (argmax[b, :n].cpu().numpy()[sure] == rl.argmax(1)[sure]).all()
 
 
-def test_free_running_speculative_equals_autoregressive_on_gpu():
-    """Lossless property on the bf16 kernels themselves: planted-beam speculative decoding emits the
-    stream of the same kernels' autoregressive decoding, and accepted lengths equal the closed form."""
+def test_free_running_lossless_up_to_the_first_near_tie():
+    """Lossless property, free running on the bf16 kernels: both the GPU's autoregressive stream and
+    its planted-beam speculative stream reproduce the oracle's greedy stream for as long as the
+    oracle's top-2 logit gap exceeds 0.05 at every token (the two GPU paths sum in different orders,
+    so beyond a near-tie they may legitimately part), and accepted lengths follow the closed form."""
     rig = Rig(cfg=RAGGED)
     cfg = rig.cfg
     BW, L = cfg["beam_width"], cfg["beam_length"]
-    prompt = np.random.default_rng(4).integers(0, 1000, size=64)
-    steps = 20
+    n_tok = 48
+    best = None
+    for seed in range(4, 40):                      # the first prompt whose greedy stream stays decided for a while
+        prompt = np.random.default_rng(seed).integers(0, 1000, size=64)
+        kv = rig.new_kv()
+        ctx, g, h = ora.prefill(rig.W, cfg, prompt, kv)
+        ref, decisive = [g], None
+        for i in range(n_tok + L):
+            g, h, logits = ora.ar_step(rig.W, cfg, kv, ctx, g)
+            ctx += 1
+            if decisive is None and top2_gap(logits) <= 0.05:
+                decisive = len(ref)                # ref[:decisive] are decided, the next token is a near-tie
+            ref.append(g)
+        decisive = len(ref) - L if decisive is None else min(decisive, len(ref) - L)
+        if decisive >= 18:
+            best = (prompt, ref, decisive)
+            break
+    assert best is not None
+    prompt, ref, decisive = best
     rig.eng.prefill([prompt])
     tok = torch.zeros(1, dtype=torch.int32, device="cuda:0")
     ar = [int(rig.eng.get_state()[1][0])]
-    for _ in range(steps * (L + 1) + 1):
+    for _ in range(decisive - 1):
         rig.eng.ar_step(tok)
         ar.append(int(tok[0]))
+    assert ar == ref[:decisive]
     rig.eng.prefill([prompt])
     rng = np.random.default_rng(5)
     out = rig.binding.AcceptOut(1, L, "cuda:0")
-    spec = [ar[0]]
-    for _ in range(steps):
-        planted = synth.plant_beams(ar[len(spec):len(spec) + L], BW, L, cfg["vocab"], rng, p=0.3, rho=0.3)
+    spec = [int(rig.eng.get_state()[1][0])]
+    steps = 0
+    while len(spec) + L + 1 <= decisive:
+        planted = synth.plant_beams(ref[len(spec):len(spec) + L], BW, L, cfg["vocab"], rng, p=0.3, rho=0.3)
         rig.eng.step(dev(planted[None]), out)
         a = int(out.n_accept[0])
-        assert a == synth.first_mismatch(planted, ar[len(spec):len(spec) + L]).max()
+        assert a == synth.first_mismatch(planted, ref[len(spec):len(spec) + L]).max()
         spec.extend(out.tokens[0, :a + 1].tolist())
+        steps += 1
     rig.eng.poll()
-    assert spec == ar[:len(spec)]
+    assert steps >= 2 and spec == ref[:len(spec)]
