@@ -5,8 +5,10 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <map>
 #include <new>
 #include <unordered_map>
+#include <utility>
 #include <vector>
 
 #include "rd_internal.cuh"
@@ -33,7 +35,7 @@ struct Workspace {
   // row tables of the current forward
   int32_t *row_tok, *row_seq, *row_pos, *row_slot, *row_ncache, *row_local, *row_out_index, *m_total, *last_row, *seq_off;
   // activations of the forward (compact rows)
-  float *x, *qkv, *gu, *hidden_f, *logits, *rope_tab;
+  float *x, *qkv, *proj_d, *gu, *hidden_f, *logits, *rope_tab;
   void *a_t, *attn_t, *act_t, *hidden_t, *h_t;
   int32_t* argmax_c;
   // step-internal packed beam, beams, verify outputs, accept scratch
@@ -41,11 +43,10 @@ struct Workspace {
   int32_t *beams, *argmax_p, *n_accept, *best, *ctx_prev, *acc_tokens;
   float *scores, *hidden_p;
   // drafter
-  void *xc_t, *x0_t, *x1_t, *x2_t, *sprev_t, *e_t;
-  float *xc_f, *x0_f, *x1_f, *x2_f, *tmp_f, *dlogits, *lse, *cand_val, *score_a, *score_b;
+  void *xc_t, *x0_t, *x1_t, *x2_t, *se_t, *uw;   // se_t: [R][d_rnn + d] = [s ; e]; uw: [d_rnn][d_rnn + d] = [U W]
+  float *xc_f, *x0_f, *x1_f, *x2_f, *sraw, *hraw, *dlogits, *lse, *cand_val, *score_a, *score_b;
   int32_t *cand_idx, *hist_a, *hist_b, *one_b, *one_r;
   // tensor-core projection scratch
-  int32_t* tc_counters;
   float* tc_partial;
   // tensor-core attention scratch
   int32_t* att_counters;
@@ -55,8 +56,9 @@ struct Workspace {
 
 size_t esize(int dtype) { return dtype == RD_DTYPE_FP32 ? 4 : 2; }
 
-struct alignas(64) TensorMapBox {  // opaque storage of one CUtensorMap (128 bytes)
+struct alignas(64) TensorMapBox {  // opaque storage of one CUtensorMap (128 bytes) + the matrix it describes
   unsigned char bytes[128];
+  int rows, cols;
 };
 
 }  // namespace
@@ -82,7 +84,9 @@ struct rd_handle {
   bool use_tc;
   int trace_next;  // next trace slot, -1 = tracing off
   int tc_grid, tc_smem;
-  std::unordered_map<const void*, TensorMapBox> maps;
+  std::unordered_map<const void*, TensorMapBox> maps;               // weights
+  std::unordered_map<const void*, std::pair<int, int>> act_shape;   // activation buffers: rows, cols
+  std::map<std::pair<const void*, int>, TensorMapBox> act_maps;     // by (buffer, rows per box), made on first use
   // optional per-launch timing of the projections (class 0) and the attention kernel (class 1)
   bool profiling;
   std::vector<cudaEvent_t> ev[PROF_CLASSES];   // start/stop pairs
@@ -133,7 +137,7 @@ bool make_dims(const rd_config* c, Dims* dm) {
 int shape_ok(const Dims& dm) {
   const int vec = dm.dtype == RD_DTYPE_FP32 ? 4 : 8;
   if (dm.hd != 64 && dm.hd != 128) return 0;
-  if (dm.d % vec || dm.F % vec || dm.dh % vec) return 0;
+  if (dm.d % vec || dm.F % vec || dm.dh % vec || dm.V % 4) return 0;
   if (dm.BW > dm.V || dm.BW > 128) return 0;
   if (dm.BW * (dm.L + 1) > 1024 || dm.NMAX > 1024) return 0;
   return 1;
@@ -159,15 +163,9 @@ void carve(Bump& bp, const Dims& dm, int m_cap, Workspace* w) {
   w->one_b = bp.take<int32_t>(4); w->one_r = bp.take<int32_t>(4);
   w->seq_off = bp.take<int32_t>(B + 1);
   w->att_counters = bp.take<int32_t>(ATT_MAX_SPLIT_BLOCKS);
-  {
-    int max_n = 3 * dm.d;
-    if (2 * dm.F > max_n) max_n = 2 * dm.F;
-    if (dm.V > max_n) max_n = dm.V;
-    if (dm.dh > max_n) max_n = dm.dh;
-    w->tc_counters = bp.take<int32_t>(tc_counter_ints(max_n, m_cap));
-  }
   w->x = bp.take<float>((size_t)m_cap * dm.d);
   w->qkv = bp.take<float>((size_t)m_cap * 3 * dm.d);
+  w->proj_d = bp.take<float>((size_t)m_cap * dm.d);
   w->gu = bp.take<float>((size_t)m_cap * 2 * dm.F);
   w->hidden_f = bp.take<float>((size_t)m_cap * dm.d);
   w->logits = bp.take<float>((size_t)m_cap * dm.V);
@@ -187,10 +185,11 @@ void carve(Bump& bp, const Dims& dm, int m_cap, Workspace* w) {
   w->scores = bp.take<float>(R); w->hidden_p = bp.take<float>((size_t)B * dm.NMAX * dm.d);
   w->xc_t = bp.take<char>((size_t)B * dm.dh * es); w->x0_t = bp.take<char>((size_t)R * dm.dh * es);
   w->x1_t = bp.take<char>((size_t)R * dm.dh * es); w->x2_t = bp.take<char>((size_t)R * dm.dh * es);
-  w->sprev_t = bp.take<char>((size_t)R * dm.dr * es); w->e_t = bp.take<char>((size_t)R * dm.d * es);
+  w->se_t = bp.take<char>((size_t)R * (dm.dr + dm.d) * es); w->uw = bp.take<char>((size_t)dm.dr * (dm.dr + dm.d) * es);
   w->xc_f = bp.take<float>((size_t)B * dm.dh); w->x0_f = bp.take<float>((size_t)R * dm.dh);
   w->x1_f = bp.take<float>((size_t)R * dm.dh); w->x2_f = bp.take<float>((size_t)R * dm.dh);
-  w->tmp_f = bp.take<float>((size_t)R * dm.dr); w->dlogits = bp.take<float>((size_t)R * dm.V);
+  w->sraw = bp.take<float>((size_t)R * dm.dr); w->hraw = bp.take<float>((size_t)R * dm.dh);
+  w->dlogits = bp.take<float>((size_t)R * dm.V);
   w->lse = bp.take<float>(R); w->cand_val = bp.take<float>((size_t)R * dm.BW);
   w->score_a = bp.take<float>(R); w->score_b = bp.take<float>(R);
   w->cand_idx = bp.take<int32_t>((size_t)R * dm.BW); w->hist_a = bp.take<int32_t>((size_t)R * dm.L);
@@ -241,27 +240,39 @@ struct ProfScope {
     CK(h, expr);                       \
   } while (0)
 
-Epilogue ep_store(float* out, int ld) {
-  Epilogue e{};
-  e.out_f32 = out; e.ld_out_f32 = ld;
-  return e;
-}
-
-// One projection; picks the kernel.
-int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, const int32_t* m_total, int m_max,
-         const Epilogue& ep, cudaStream_t st) {
+// One projection Y = A W^T into the fp32 buffer `raw` (row stride ld_raw); fills `out` for the consumer.
+// `next_w`: the weight matrix of the projection that follows in the step (its first tiles are prefetched
+// into L2), or nullptr.
+int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, const int32_t* m_total, int m_max, float* raw,
+         int ld_raw, GemmOut* out, const void* next_w, cudaStream_t st) {
   ProfScope ps(h, 0, (double)N * K * esize(h->dm.dtype), st);
   if (h->use_tc) {
-    auto ia = h->maps.find(A), iw = h->maps.find(W);
-    if (ia == h->maps.end() || iw == h->maps.end() || lda != K)
+    auto iw = h->maps.find(W);
+    auto is = h->act_shape.find(A);
+    if (iw == h->maps.end() || is == h->act_shape.end() || lda != K || is->second.second != K)
       return fail(h, RD_ERR_STATE, "projection operand without a TMA descriptor");
+    const int mt = tc_pick_mt(m_max > 0 ? m_max : 1);
+    auto key = std::make_pair(A, mt);
+    auto ia = h->act_maps.find(key);
+    if (ia == h->act_maps.end()) {
+      TensorMapBox box;
+      box.rows = is->second.first; box.cols = K;
+      const int rc = tc_make_map(&box, A, (uint64_t)box.rows, (uint64_t)K, (uint32_t)mt);
+      if (rc) return fail(h, RD_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d for an activation buffer", rc);
+      ia = h->act_maps.emplace(key, box).first;
+    }
     unsigned long long* tr = nullptr;
     if (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) tr = h->ws.trace + (size_t)8 * h->trace_next++;
-    CK(h, launch_gemm_tc(&iw->second, &ia->second, N, K, m_total, m_max, ep, h->ws.tc_partial, h->ws.tc_counters,
-                         h->ws.status, h->tc_grid, h->tc_smem, tr, st));
+    const TensorMapBox* nx = nullptr;
+    if (next_w) {
+      auto in = h->maps.find(next_w);
+      if (in != h->maps.end()) nx = &in->second;
+    }
+    CK(h, launch_gemm_tc(&iw->second, &ia->second, N, K, m_total, m_max, raw, ld_raw, h->ws.tc_partial, h->ws.status,
+                         h->tc_grid, h->tc_smem, tr, nx, nx ? nx->rows : 0, nx ? nx->cols : 0, out, st));
     return RD_OK;
   }
-  CK(h, launch_gemm_simt(h->dm.dtype, A, lda, W, N, K, m_total, m_max, ep, st));
+  CK(h, launch_gemm_simt(h->dm.dtype, A, lda, W, N, K, m_total, m_max, raw, ld_raw, out, st));
   return RD_OK;
 }
 
@@ -271,7 +282,8 @@ char* kv_plane_ptr(rd_handle* h, int layer, int which) {
 
 // Embedding -> n_layers x {attention block, FFN block} -> final norm.  Rows and masks come from the
 // row tables in the workspace; results: ws.hidden_f / ws.hidden_t (compact rows).
-int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int rows_per_seq_max, cudaStream_t st) {
+int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int rows_per_seq_max, const void* after_w,
+                   cudaStream_t st) {
   Workspace& w = h->ws;
   const Dims& dm = h->dm;
   RowTables rt{w.row_tok, w.row_seq, w.row_pos, w.row_slot, w.row_ncache, w.row_local, mask, w.m_total};
@@ -291,11 +303,15 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
     if (n_splits < 1) n_splits = 1;
     while (n_splits > 1 && (long long)blocks * n_splits > ATT_MAX_SPLIT_BLOCKS) --n_splits;
   }
+  GemmOut g_qkv, g_o, g_gu, g_dn;
   for (int l = 0; l < dm.n_layers; ++l) {
-    CKP(h, PROF_NORM, launch_rmsnorm(dm.dtype, w.x, h->attn_norm[l], w.a_t, nullptr, dm.d, dm.eps, w.m_total, m_max, st));
-    int rc = gemm(h, w.a_t, dm.d, h->wqkv[l], 3 * dm.d, dm.d, w.m_total, m_max, ep_store(w.qkv, 3 * dm.d), st);
+    // attention block: (x += down of the previous layer) -> norm -> QKV -> rotary + KV write -> attention -> O
+    CKP(h, PROF_NORM, launch_rmsnorm(dm.dtype, w.x, l ? &g_dn : nullptr, h->attn_norm[l], w.a_t, nullptr, dm.d, dm.eps,
+                                     w.m_total, m_max, st));
+    int rc = gemm(h, w.a_t, dm.d, h->wqkv[l], 3 * dm.d, dm.d, w.m_total, m_max, w.qkv, 3 * dm.d, &g_qkv, h->wo[l], st);
     if (rc) return rc;
-    CKP(h, PROF_ROPE, launch_rope_kv(dm.dtype, w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.rope_tab, rt, dm, m_max, w.status, st));
+    CKP(h, PROF_ROPE, launch_rope_kv(dm.dtype, w.qkv, g_qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.rope_tab, rt, dm,
+                                     m_max, w.status, st));
     {
       ProfScope ps(h, 1, 0.0, st);
       if (h->use_tc)
@@ -304,18 +320,19 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
       else
         CK(h, launch_attention(dm.dtype, w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.attn_t, rt, dm, m_max, st));
     }
-    Epilogue eo{};
-    eo.resid = w.x; eo.ld_resid = dm.d; eo.out_f32 = w.x; eo.ld_out_f32 = dm.d;
-    rc = gemm(h, w.attn_t, dm.d, h->wo[l], dm.d, dm.d, w.m_total, m_max, eo, st);
+    rc = gemm(h, w.attn_t, dm.d, h->wo[l], dm.d, dm.d, w.m_total, m_max, w.proj_d, dm.d, &g_o, h->w_gate_up[l], st);
     if (rc) return rc;
-    CKP(h, PROF_NORM, launch_rmsnorm(dm.dtype, w.x, h->ffn_norm[l], w.a_t, nullptr, dm.d, dm.eps, w.m_total, m_max, st));
-    rc = gemm(h, w.a_t, dm.d, h->w_gate_up[l], 2 * dm.F, dm.d, w.m_total, m_max, ep_store(w.gu, 2 * dm.F), st);
+    // FFN block: (x += O) -> norm -> gate|up -> SwiGLU -> down
+    CKP(h, PROF_NORM, launch_rmsnorm(dm.dtype, w.x, &g_o, h->ffn_norm[l], w.a_t, nullptr, dm.d, dm.eps, w.m_total, m_max, st));
+    rc = gemm(h, w.a_t, dm.d, h->w_gate_up[l], 2 * dm.F, dm.d, w.m_total, m_max, w.gu, 2 * dm.F, &g_gu, h->w_down[l], st);
     if (rc) return rc;
-    CKP(h, PROF_SWIGLU, launch_swiglu(dm.dtype, w.gu, w.act_t, dm.F, w.m_total, m_max, st));
-    rc = gemm(h, w.act_t, dm.F, h->w_down[l], dm.d, dm.F, w.m_total, m_max, eo, st);
+    CKP(h, PROF_SWIGLU, launch_swiglu(dm.dtype, g_gu, w.act_t, dm.F, w.m_total, m_max, st));
+    rc = gemm(h, w.act_t, dm.F, h->w_down[l], dm.d, dm.F, w.m_total, m_max, w.proj_d, dm.d, &g_dn,
+              l + 1 < dm.n_layers ? h->wqkv[l + 1] : after_w, st);
     if (rc) return rc;
   }
-  CKP(h, PROF_NORM, launch_rmsnorm(dm.dtype, w.x, h->w.final_norm, w.hidden_t, w.hidden_f, dm.d, dm.eps, w.m_total, m_max, st));
+  CKP(h, PROF_NORM, launch_rmsnorm(dm.dtype, w.x, &g_dn, h->w.final_norm, w.hidden_t, w.hidden_f, dm.d, dm.eps, w.m_total,
+                                   m_max, st));
   return RD_OK;
 }
 
@@ -332,40 +349,38 @@ int do_draft(rd_handle* h, cudaStream_t st, int32_t* beams, float* scores) {
   Workspace& w = h->ws;
   const Dims& dm = h->dm;
   const int B = h->batch, R = B * dm.BW;
-  CKP(h, PROF_DRAFT_SMALL, launch_draft_init(dm.dtype, h->w.tok_emb, w.root, w.h, w.xc_t, w.xc_f, w.sprev_t, dm, B, w.status, st));
+  CKP(h, PROF_DRAFT_SMALL, launch_draft_init(dm.dtype, h->w.tok_emb, w.root, w.h, w.xc_t, w.xc_f, w.se_t, dm, B, w.status, st));
   if (dm.L > 1) CKP(h, PROF_DRAFT_SMALL, launch_fill_h(dm.dtype, w.h, w.x0_t, w.x0_f, dm, B, st));
   float *sc_in = w.score_a, *sc_out = w.score_b;
   int32_t *hi_in = w.hist_a, *hi_out = w.hist_b;
+  GemmOut g;
   for (int call = 1; call <= dm.L; ++call) {
     const int rows = call == 1 ? B : R;
     const int32_t* mt = call == 1 ? w.one_b : w.one_r;
     const void* xin_t = call == 1 ? w.xc_t : w.x0_t;
     const float* xin_f = call == 1 ? w.xc_f : w.x0_f;
     if (call > 1) {
-      // s_t = SiLU(U s_{t-1} + W e_t + b), written into the first d_rnn columns of x0 = [s_t, h]
-      int rc = gemm(h, w.sprev_t, dm.dr, h->w.rnn_u, dm.dr, dm.dr, mt, rows, ep_store(w.tmp_f, dm.dr), st);
+      // s_t = SiLU([U W][s_{t-1}; e_t] + b), written into the first d_rnn columns of x0 = [s_t, h]
+      int rc = gemm(h, w.se_t, dm.dr + dm.d, w.uw, dm.dr, dm.dr + dm.d, mt, rows, w.sraw, dm.dr, &g,
+                    dm.n_head_layers ? h->head_w[0] : h->w.draft_out, st);
       if (rc) return rc;
-      Epilogue e{};
-      e.addend = w.tmp_f; e.ld_addend = dm.dr; e.bias = h->w.rnn_b; e.silu = 1;
-      e.out_f32 = w.x0_f; e.ld_out_f32 = dm.dh; e.out_t = w.x0_t; e.ld_out_t = dm.dh;
-      rc = gemm(h, w.e_t, dm.d, h->w.rnn_w, dm.dr, dm.d, mt, rows, e, st);
-      if (rc) return rc;
+      CKP(h, PROF_DRAFT_SMALL, launch_act(dm.dtype, g, h->w.rnn_b, nullptr, 0, w.x0_f, w.x0_t, dm.dh, dm.dr, mt, rows, st));
     }
     for (int l = 0; l < dm.n_head_layers; ++l) {
-      Epilogue e{};
-      e.bias = h->head_b[l]; e.silu = 1; e.resid = xin_f; e.ld_resid = dm.dh;
       float* of = (l & 1) ? w.x2_f : w.x1_f;
       void* ot = (l & 1) ? w.x2_t : w.x1_t;
-      e.out_f32 = of; e.ld_out_f32 = dm.dh; e.out_t = ot; e.ld_out_t = dm.dh;
-      int rc = gemm(h, xin_t, dm.dh, h->head_w[l], dm.dh, dm.dh, mt, rows, e, st);
+      int rc = gemm(h, xin_t, dm.dh, h->head_w[l], dm.dh, dm.dh, mt, rows, w.hraw, dm.dh, &g,
+                    l + 1 < dm.n_head_layers ? h->head_w[l + 1] : h->w.draft_out, st);
       if (rc) return rc;
+      CKP(h, PROF_DRAFT_SMALL, launch_act(dm.dtype, g, h->head_b[l], xin_f, dm.dh, of, ot, dm.dh, dm.dh, mt, rows, st));
       xin_t = ot; xin_f = of;
     }
-    int rc = gemm(h, xin_t, dm.dh, h->w.draft_out, dm.V, dm.dh, mt, rows, ep_store(w.dlogits, dm.V), st);
+    int rc = gemm(h, xin_t, dm.dh, h->w.draft_out, dm.V, dm.dh, mt, rows, w.dlogits, dm.V, &g,
+                  call < dm.L ? (const void*)w.uw : h->wqkv[0], st);
     if (rc) return rc;
-    CKP(h, PROF_DRAFT_SMALL, launch_row_topk(w.dlogits, dm.V, dm.BW, w.lse, w.cand_val, w.cand_idx, rows, st));
-    CKP(h, PROF_DRAFT_SMALL, launch_beam_merge(dm.dtype, call, w.lse, w.cand_val, w.cand_idx, sc_in, sc_out, hi_in, hi_out, h->w.tok_emb,
-                            w.x0_f, dm.dh, w.sprev_t, w.e_t, dm, B, beams, scores, st));
+    CKP(h, PROF_DRAFT_SMALL, launch_row_topk(g, dm.V, dm.BW, w.lse, w.cand_val, w.cand_idx, rows, mt, st));
+    CKP(h, PROF_DRAFT_SMALL, launch_beam_merge(dm.dtype, call, w.lse, w.cand_val, w.cand_idx, sc_in, sc_out, hi_in, hi_out,
+                                               h->w.tok_emb, w.x0_f, dm.dh, w.se_t, dm, B, beams, scores, st));
     float* tf = sc_in; sc_in = sc_out; sc_out = tf;
     int32_t* ti = hi_in; hi_in = hi_out; hi_out = ti;
   }
@@ -378,12 +393,14 @@ int do_verify(rd_handle* h, const rd_packed& pk, cudaStream_t st, int32_t* argma
   const int B = h->batch, m_max = B * dm.NMAX;
   CKP(h, PROF_MISC, launch_build_rows_tree(pk, w.ctx, w.row_tok, w.row_seq, w.row_pos, w.row_slot, w.row_ncache, w.row_local,
                                w.row_out_index, w.seq_off, w.m_total, dm, B, w.status, st));
-  int rc = forward_layers(h, pk.mask, m_max, B, dm.NMAX, st);
+  int rc = forward_layers(h, pk.mask, m_max, B, dm.NMAX, h->w.lm_head, st);
   if (rc) return rc;
-  rc = gemm(h, w.hidden_t, dm.d, h->w.lm_head, dm.V, dm.d, w.m_total, m_max, ep_store(w.logits, dm.V), st);
+  GemmOut g;
+  rc = gemm(h, w.hidden_t, dm.d, h->w.lm_head, dm.V, dm.d, w.m_total, m_max, w.logits, dm.V, &g,
+            dm.n_head_layers ? h->head_w[0] : h->w.draft_out, st);  // the next step starts with the drafter
   if (rc) return rc;
   CKP(h, PROF_MISC, launch_fill_i32(argmax, -1, B * dm.NMAX, st));
-  CKP(h, PROF_MISC, launch_argmax_rows(w.logits, dm.V, argmax, w.row_out_index, w.m_total, m_max, st));
+  CKP(h, PROF_MISC, launch_argmax_rows(w.logits, g, dm.V, argmax, w.row_out_index, w.m_total, m_max, st));
   if (hidden) CKP(h, PROF_MISC, launch_scatter_rows(w.hidden_f, dm.d, hidden, w.row_out_index, w.m_total, m_max, st));
   if (logits) CK(h, launch_scatter_rows(w.logits, dm.V, logits, w.row_out_index, w.m_total, m_max, st));
   return RD_OK;
@@ -457,19 +474,17 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
     const void* failed_ptr = nullptr;
     auto add_w = [&](const void* p, int N, int K) {
       if (!ok) return;
-      failed_rc = tc_make_map(&h->maps[p], p, (uint64_t)N, (uint64_t)K, (uint32_t)tc_weight_box_rows());
+      TensorMapBox& box = h->maps[p];
+      box.rows = N; box.cols = K;
+      failed_rc = tc_make_map(&box, p, (uint64_t)N, (uint64_t)K, (uint32_t)tc_weight_box_rows());
       if (failed_rc) { ok = false; failed_ptr = p; }
     };
-    auto add_a = [&](const void* p, int rows, int K) {
-      if (!ok) return;
-      failed_rc = tc_make_map(&h->maps[p], p, (uint64_t)rows, (uint64_t)K, (uint32_t)tc_act_box_rows());
-      if (failed_rc) { ok = false; failed_ptr = p; }
-    };
+    auto add_a = [&](const void* p, int rows, int K) { h->act_shape[p] = std::make_pair(rows, K); };
     for (int l = 0; l < dm.n_layers; ++l) {
       add_w(h->wqkv[l], 3 * dm.d, dm.d); add_w(h->wo[l], dm.d, dm.d);
       add_w(h->w_gate_up[l], 2 * dm.F, dm.d); add_w(h->w_down[l], dm.d, dm.F);
     }
-    add_w(wt->lm_head, dm.V, dm.d); add_w(wt->rnn_u, dm.dr, dm.dr); add_w(wt->rnn_w, dm.dr, dm.d);
+    add_w(wt->lm_head, dm.V, dm.d); add_w(h->ws.uw, dm.dr, dm.dr + dm.d);
     for (int l = 0; l < dm.n_head_layers; ++l) add_w(h->head_w[l], dm.dh, dm.dh);
     add_w(wt->draft_out, dm.V, dm.dh);
     const Workspace& w = h->ws;
@@ -477,7 +492,7 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
     add_a(w.a_t, h->m_cap, dm.d); add_a(w.attn_t, h->m_cap, dm.d); add_a(w.act_t, h->m_cap, dm.F);
     add_a(w.hidden_t, h->m_cap, dm.d); add_a(w.h_t, dm.B, dm.d);
     add_a(w.xc_t, dm.B, dm.dh); add_a(w.x0_t, R, dm.dh); add_a(w.x1_t, R, dm.dh); add_a(w.x2_t, R, dm.dh);
-    add_a(w.sprev_t, R, dm.dr); add_a(w.e_t, R, dm.d);
+    add_a(w.se_t, R, dm.dr + dm.d);
     if (!ok) return init_fail(h, RD_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d for operand %p", failed_rc, failed_ptr);
   }
   h->prefilled = false; h->batch = dm.B; h->ctx_bound = 0; h->launches = 0; h->err[0] = 0;
@@ -486,6 +501,14 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
   for (int c = 0; c < PROF_CLASSES; ++c) { h->ev_used[c] = 0; h->prof_ms[c] = 0; h->prof_bytes[c] = 0; h->prof_n[c] = 0; }
   // clear the state and the constants the kernels read from device memory
   cudaError_t e = cudaMemsetAsync(workspace, 0, (size_t)((char*)h->ws.x - (char*)workspace), 0);
+  // [U W]: the RNN's two matrices side by side, so that s_t needs one projection over [s ; e]
+  const size_t es_ = esize(dm.dtype);
+  if (e == cudaSuccess)
+    e = cudaMemcpy2DAsync(h->ws.uw, (size_t)(dm.dr + dm.d) * es_, wt->rnn_u, (size_t)dm.dr * es_, (size_t)dm.dr * es_, dm.dr,
+                          cudaMemcpyDeviceToDevice, 0);
+  if (e == cudaSuccess)
+    e = cudaMemcpy2DAsync((char*)h->ws.uw + (size_t)dm.dr * es_, (size_t)(dm.dr + dm.d) * es_, wt->rnn_w, (size_t)dm.d * es_,
+                          (size_t)dm.d * es_, dm.dr, cudaMemcpyDeviceToDevice, 0);
   if (e == cudaSuccess) e = cudaStreamSynchronize(0);
   if (e != cudaSuccess) { delete h; return RD_ERR_CUDA; }
   *out = h;
@@ -560,15 +583,16 @@ int redrafter_prefill(rd_handle* h, const int32_t* tokens, const int32_t* prompt
     CKRT(h, cudaMemcpyAsync(w.m_total, &m, sizeof(int32_t), cudaMemcpyHostToDevice, st));
     CKRT(h, cudaStreamSynchronize(st));  // the host staging vectors are reused by the next pass
     h->ctx_bound = longest;  // bound of the key extent for this pass
-    rc = forward_layers(h, nullptr, m, batch, longest_run, st);
+    rc = forward_layers(h, nullptr, m, batch, longest_run, nullptr, st);
     if (rc) return rc;
     CK(h, launch_prefill_finish(w.hidden_f, w.last_row, w.h, dm.d, batch, st));
   }
   // root token: the greedy token after the prompt = argmax(lm_head h)
   CK(h, launch_cast_rows(dm.dtype, w.h, w.h_t, batch * dm.d, st));
-  rc = gemm(h, w.h_t, dm.d, h->w.lm_head, dm.V, dm.d, w.one_b, batch, ep_store(w.logits, dm.V), st);
+  GemmOut g;
+  rc = gemm(h, w.h_t, dm.d, h->w.lm_head, dm.V, dm.d, w.one_b, batch, w.logits, dm.V, &g, nullptr, st);
   if (rc) return rc;
-  CK(h, launch_argmax_rows(w.logits, dm.V, w.root, nullptr, w.one_b, batch, st));
+  CK(h, launch_argmax_rows(w.logits, g, dm.V, w.root, nullptr, w.one_b, batch, st));
   CKRT(h, cudaMemcpyAsync(w.ctx, prompt_len, batch * sizeof(int32_t), cudaMemcpyHostToDevice, st));
   h->prefilled = true;
   h->ctx_bound = longest;
@@ -647,11 +671,12 @@ int redrafter_ar_step(rd_handle* h, void* stream, int32_t* token) {
   const int B = h->batch;
   CK(h, launch_build_rows_ar(w.root, w.ctx, w.row_tok, w.row_seq, w.row_pos, w.row_slot, w.row_ncache, w.row_local,
                              w.row_out_index, w.seq_off, w.m_total, dm, B, w.status, st));
-  int rc = forward_layers(h, nullptr, B, B, 1, st);
+  int rc = forward_layers(h, nullptr, B, B, 1, h->w.lm_head, st);
   if (rc) return rc;
-  rc = gemm(h, w.hidden_t, dm.d, h->w.lm_head, dm.V, dm.d, w.m_total, B, ep_store(w.logits, dm.V), st);
+  GemmOut g;
+  rc = gemm(h, w.hidden_t, dm.d, h->w.lm_head, dm.V, dm.d, w.m_total, B, w.logits, dm.V, &g, h->wqkv[0], st);
   if (rc) return rc;
-  CK(h, launch_argmax_rows(w.logits, dm.V, w.argmax_c, nullptr, w.m_total, B, st));
+  CK(h, launch_argmax_rows(w.logits, g, dm.V, w.argmax_c, nullptr, w.m_total, B, st));
   CK(h, launch_ar_finish(w.argmax_c, w.hidden_f, w.ctx, w.root, w.h, token, dm, B, st));
   h->ctx_bound += 1;
   return RD_OK;

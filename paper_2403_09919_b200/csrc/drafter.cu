@@ -1,13 +1,15 @@
 // Beam search over the RNN drafter (Sections 3.1, 3.2): the small kernels around the
 // projections.  A drafter call t works on R = B*BW rows (call 1: B rows):
-//   rnn:   s_t = SiLU(U s_{t-1} + W e_t + b)            two projections with a fused epilogue
-//   head:  x <- x + SiLU(A_l x + c_l), x_0 = [s_t, h]   one projection per layer, fused epilogue
+//   rnn:   s_t = SiLU([U W] [s_{t-1}; e_t] + b)        one projection over the concatenated input,
+//                                                       finished by act_kernel
+//   head:  x <- x + SiLU(A_l x + c_l), x_0 = [s_t, h]   one projection per layer, finished by act_kernel
 //   out:   logits = O x                                  one projection
 //   row_topk:   per row, log-sum-exp and the BW best logits (value desc, index asc)
 //   beam_merge: per sequence, score_r + logit - lse_r over the BW*BW survivors, best BW in
 //               (score desc, flat index r*V + v asc) order; reorders histories and states and
-//               gathers the next call's inputs (e_{t+1} = E[token], s_t of the parent).
+//               gathers the next call's input [s_t of the parent ; E[token]].
 #include "rd_internal.cuh"
+#include "gemm_out.cuh"
 #include "pdl.cuh"
 
 namespace rd {
@@ -17,10 +19,11 @@ namespace rd {
   else { using T = __nv_bfloat16; __VA_ARGS__; }
 
 // ---------------------------------------------------------------- call-1 input and s_1
-// x[b] = [E[g_b], h_b] for the first call; sprev[r] = E[g_b] = s_1 for every beam row of b.
+// x[b] = [E[g_b], h_b] for the first call; the state half of se[r] = [s ; e] is E[g_b] = s_1 for
+// every beam row r of b.
 template <typename T>
 __global__ void draft_init_kernel(const T* __restrict__ emb, const int32_t* __restrict__ root, const float* __restrict__ h,
-                                  T* __restrict__ x_t, float* __restrict__ x_f, T* __restrict__ sprev_t, Dims dm,
+                                  T* __restrict__ x_t, float* __restrict__ x_f, T* __restrict__ se_t, Dims dm,
                                   int* status) {
   pdl_enter();
   const int b = blockIdx.x;
@@ -37,13 +40,13 @@ __global__ void draft_init_kernel(const T* __restrict__ emb, const int32_t* __re
     const float hv = h[(size_t)b * d + i];
     x_t[(size_t)b * dm.dh + dm.dr + i] = from_f<T>(hv);
     x_f[(size_t)b * dm.dh + dm.dr + i] = hv;
-    for (int k = 0; k < dm.BW; ++k) sprev_t[((size_t)b * dm.BW + k) * dm.dr + i] = e;
+    for (int k = 0; k < dm.BW; ++k) se_t[((size_t)b * dm.BW + k) * (dm.dr + dm.d) + i] = e;
   }
 }
 
 cudaError_t launch_draft_init(int dtype, const void* emb, const int32_t* root, const float* h, void* x_t, float* x_f,
-                              void* sprev_t, const Dims& dm, int B, int* status, cudaStream_t st) {
-  RD_DISPATCH(dtype, launch_pdl(draft_init_kernel<T>, B, 256, 0, st, (const T*)emb, root, h, (T*)x_t, x_f, (T*)sprev_t, dm, status));
+                              void* se_t, const Dims& dm, int B, int* status, cudaStream_t st) {
+  RD_DISPATCH(dtype, launch_pdl(draft_init_kernel<T>, B, 256, 0, st, (const T*)emb, root, h, (T*)x_t, x_f, (T*)se_t, dm, status));
   return cudaGetLastError();
 }
 
@@ -61,6 +64,39 @@ __global__ void fill_h_kernel(const float* __restrict__ h, T* __restrict__ x_t, 
 
 cudaError_t launch_fill_h(int dtype, const float* h, void* x_t, float* x_f, const Dims& dm, int B, cudaStream_t st) {
   RD_DISPATCH(dtype, launch_pdl(fill_h_kernel<T>, B * dm.BW, 256, 0, st, h, (T*)x_t, x_f, dm));
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- finish of a drafter projection
+// out[m][n] = (resid ? resid[m][n] : 0) + SiLU(proj[m][n] + bias[n]), written as fp32 and in the
+// storage type (the next projection's input).  Used for the RNN cell (no residual) and for the
+// head's residual layers.
+template <typename T>
+__global__ void act_kernel(GemmOut proj, const T* __restrict__ bias, const float* __restrict__ resid, int ld_resid,
+                           float* __restrict__ out_f, T* __restrict__ out_t, int ld_out, int N,
+                           const int32_t* __restrict__ m_total) {
+  pdl_enter();
+  const int m = blockIdx.y;
+  const int M = *m_total;
+  if (m >= M) return;
+  const int n = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (n >= N) return;
+  const float4 q = gemm_value4(proj, gemm_m_tiles(proj, M), m, n);
+  float v[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    v[k] = silu_f(v[k] + to_f<T>(bias[n + k]));
+    if (resid) v[k] += resid[(size_t)m * ld_resid + n + k];
+    out_f[(size_t)m * ld_out + n + k] = v[k];
+    out_t[(size_t)m * ld_out + n + k] = from_f<T>(v[k]);
+  }
+}
+
+cudaError_t launch_act(int dtype, const GemmOut& proj, const void* bias, const float* resid, int ld_resid, float* out_f,
+                       void* out_t, int ld_out, int N, const int32_t* m_total, int m_max, cudaStream_t st) {
+  dim3 grid((N / 4 + 255) / 256, m_max);
+  RD_DISPATCH(dtype, launch_pdl(act_kernel<T>, grid, 256, 0, st, proj, (const T*)bias, resid, ld_resid, out_f, (T*)out_t,
+                                ld_out, N, m_total));
   return cudaGetLastError();
 }
 
@@ -103,21 +139,25 @@ __device__ __forceinline__ Cand block_best(Cand c, Cand* sh) {
 constexpr int TOPK_THREADS = 1024;
 constexpr int TOPK_PER_THREAD = 32;  // V <= 32768
 
-__global__ void __launch_bounds__(TOPK_THREADS) row_topk_kernel(const float* __restrict__ logits, int V, int BW,
-                                                                 float* __restrict__ lse, float* __restrict__ val,
-                                                                 int32_t* __restrict__ idx) {
+__global__ void __launch_bounds__(TOPK_THREADS) row_topk_kernel(GemmOut proj, int V, int BW, float* __restrict__ lse,
+                                                                 float* __restrict__ val, int32_t* __restrict__ idx,
+                                                                 const int32_t* __restrict__ m_total) {
   pdl_enter();
   __shared__ Cand sh[32];
   __shared__ float shf[32];
   const int r = blockIdx.x;
-  const float* z = logits + (size_t)r * V;
+  const int m_tiles = gemm_m_tiles(proj, *m_total);
+  // element (k, e) of this thread is column 4 * (threadIdx.x + (k / 4) * TOPK_THREADS) + k % 4
   float v[TOPK_PER_THREAD];
   Cand c{-INFINITY, 0x7fffffff};
 #pragma unroll
-  for (int k = 0; k < TOPK_PER_THREAD; ++k) {
-    const int i = threadIdx.x + k * TOPK_THREADS;
-    v[k] = i < V ? z[i] : -INFINITY;
-    c = cand_best(c, Cand{v[k], i < V ? i : 0x7fffffff});
+  for (int k4 = 0; k4 < TOPK_PER_THREAD / 4; ++k4) {
+    const int i = 4 * (threadIdx.x + k4 * TOPK_THREADS);
+    float4 q = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    if (i < V) q = gemm_value4(proj, m_tiles, r, i);   // V is a multiple of 4
+    v[4 * k4] = q.x; v[4 * k4 + 1] = q.y; v[4 * k4 + 2] = q.z; v[4 * k4 + 3] = q.w;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) c = cand_best(c, Cand{v[4 * k4 + e], i < V ? i + e : 0x7fffffff});
   }
   const Cand top = block_best(c, sh);
   float s = 0.f;
@@ -144,7 +184,7 @@ __global__ void __launch_bounds__(TOPK_THREADS) row_topk_kernel(const float* __r
     Cand best{-INFINITY, 0x7fffffff};
 #pragma unroll
     for (int k = 0; k < TOPK_PER_THREAD; ++k) {
-      const int i = threadIdx.x + k * TOPK_THREADS;
+      const int i = 4 * (threadIdx.x + (k >> 2) * TOPK_THREADS) + (k & 3);
       if (i < V && cand_before(prev.v, prev.i, v[k], i)) best = cand_best(best, Cand{v[k], i});
     }
     best = block_best(best, sh);
@@ -156,24 +196,24 @@ __global__ void __launch_bounds__(TOPK_THREADS) row_topk_kernel(const float* __r
   }
 }
 
-cudaError_t launch_row_topk(const float* logits, int V, int BW, float* lse, float* val, int32_t* idx, int rows,
-                            cudaStream_t st) {
+cudaError_t launch_row_topk(const GemmOut& proj, int V, int BW, float* lse, float* val, int32_t* idx, int rows,
+                            const int32_t* m_total, cudaStream_t st) {
   if (V > TOPK_THREADS * TOPK_PER_THREAD) return cudaErrorInvalidValue;
-  launch_pdl(row_topk_kernel, rows, TOPK_THREADS, 0, st, logits, V, BW, lse, val, idx);
+  launch_pdl(row_topk_kernel, rows, TOPK_THREADS, 0, st, proj, V, BW, lse, val, idx, m_total);
   return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------- cross-row merge + reorder + gather
 // call == 1: the single row's top-BW become the beams.  call >= 2: best BW of the BW*BW survivors.  Writes score_out[k], hist_out[k][0..call-1], and the next call's inputs
-// sprev_t[k] = s_t of the parent (read from s_new_f with row stride ld_s; skipped for call 1, where
-// every beam keeps s_1) and e_t[k] = E[token_k].  On the last call also the public outputs.
+// se_t[k] = [s_t of the parent (read from s_new_f with row stride ld_s; skipped for call 1, where every
+// beam keeps s_1) ; E[token_k]].  On the last call also the public outputs.
 template <typename T>
 __global__ void __launch_bounds__(256) beam_merge_kernel(int call, const float* __restrict__ lse,
                                                           const float* __restrict__ val, const int32_t* __restrict__ idx,
                                                           const float* __restrict__ score_in, float* __restrict__ score_out,
                                                           const int32_t* __restrict__ hist_in, int32_t* __restrict__ hist_out,
                                                           const T* __restrict__ emb, const float* __restrict__ s_new_f,
-                                                          int ld_s, T* __restrict__ sprev_t, T* __restrict__ e_t, Dims dm,
+                                                          int ld_s, T* __restrict__ se_t, Dims dm,
                                                           int32_t* __restrict__ beams_out, float* __restrict__ scores_out) {
   pdl_enter();
   // grid = B * BW: every CTA of a sequence repeats the (tiny) selection over the BW*BW survivors and
@@ -221,13 +261,15 @@ __global__ void __launch_bounds__(256) beam_merge_kernel(int call, const float* 
   }
   if (call < L) {
     // gathers with 128-bit accesses (rows are 16-byte aligned: d is a multiple of 8)
+    // next call's input row [s of the parent ; E[token]]
     constexpr int EV = 16 / sizeof(T);
+    T* se = se_t + (size_t)orow * (dm.dr + dm.d);
     const uint4* e = reinterpret_cast<const uint4*>(emb + (size_t)tok * dm.d);
-    uint4* eo = reinterpret_cast<uint4*>(e_t + (size_t)orow * dm.d);
+    uint4* eo = reinterpret_cast<uint4*>(se + dm.dr);
     for (int i = threadIdx.x; i < dm.d / EV; i += blockDim.x) eo[i] = e[i];
     if (call > 1) {
       const float4* s = reinterpret_cast<const float4*>(s_new_f + (size_t)prow * ld_s);
-      T* so = sprev_t + (size_t)orow * dm.dr;
+      T* so = se;
       for (int i = threadIdx.x; i < dm.dr / 4; i += blockDim.x) {
         const float4 v = s[i];
         so[4 * i] = from_f<T>(v.x); so[4 * i + 1] = from_f<T>(v.y); so[4 * i + 2] = from_f<T>(v.z); so[4 * i + 3] = from_f<T>(v.w);
@@ -238,10 +280,10 @@ __global__ void __launch_bounds__(256) beam_merge_kernel(int call, const float* 
 
 cudaError_t launch_beam_merge(int dtype, int call, const float* lse, const float* val, const int32_t* idx,
                               const float* score_in, float* score_out, const int32_t* hist_in, int32_t* hist_out,
-                              const void* emb, const float* s_new_f, int ld_s, void* sprev_t, void* e_t,
-                              const Dims& dm, int B, int32_t* beams_out, float* scores_out, cudaStream_t st) {
+                              const void* emb, const float* s_new_f, int ld_s, void* se_t, const Dims& dm, int B,
+                              int32_t* beams_out, float* scores_out, cudaStream_t st) {
   RD_DISPATCH(dtype, launch_pdl(beam_merge_kernel<T>, B * dm.BW, 256, 0, st, call, lse, val, idx, score_in, score_out, hist_in, hist_out,
-                                                           (const T*)emb, s_new_f, ld_s, (T*)sprev_t, (T*)e_t, dm,
+                                                           (const T*)emb, s_new_f, ld_s, (T*)se_t, dm,
                                                            beams_out, scores_out));
   return cudaGetLastError();
 }

@@ -2,6 +2,7 @@
 // rotary embedding + KV-cache write, SwiGLU, row argmax, row tables.  All are bandwidth-trivial
 // (activations of at most a few MB that stay in L2); they exist to feed the projections.
 #include "rd_internal.cuh"
+#include "gemm_out.cuh"
 #include "pdl.cuh"
 
 namespace rd {
@@ -53,19 +54,22 @@ cudaError_t launch_embed(int dtype, const void* emb, const int32_t* tok, float* 
 // ---------------------------------------------------------------- RMSNorm
 // y = x / sqrt(mean(x^2) + eps) * gain, one block per row.  The row is read once with 128-bit loads
 // and kept in registers between the reduction and the scaling (d <= 8192).
-constexpr int NORM_THREADS = 256;
-constexpr int NORM_MAXV = 8;
+constexpr int NORM_THREADS = 1024;
+constexpr int NORM_MAXV = 2;
 
 template <typename T>
-__global__ void __launch_bounds__(NORM_THREADS) rmsnorm_kernel(const float* __restrict__ x, const T* __restrict__ gain,
+__global__ void __launch_bounds__(NORM_THREADS) rmsnorm_kernel(float* __restrict__ x, GemmOut proj, const T* __restrict__ gain,
                                                                 T* __restrict__ out_t, float* __restrict__ out_f, int d,
                                                                 float eps, const int32_t* __restrict__ m_total) {
   pdl_enter();
   __shared__ float sh[32];
   const int m = blockIdx.x;
-  if (m >= *m_total) return;
-  const float4* xr = reinterpret_cast<const float4*>(x + (size_t)m * d);
+  const int M = *m_total;
+  if (m >= M) return;
+  float4* xr = reinterpret_cast<float4*>(x + (size_t)m * d);
   const int nvec = d >> 2;
+  const bool add = proj.raw != nullptr;   // x += the projection that ends the previous block (O or down)
+  const int m_tiles = add ? gemm_m_tiles(proj, M) : 1;
   float4 v[NORM_MAXV];
   float ss = 0.f;
 #pragma unroll
@@ -73,6 +77,11 @@ __global__ void __launch_bounds__(NORM_THREADS) rmsnorm_kernel(const float* __re
     const int i = threadIdx.x + k * NORM_THREADS;
     if (i < nvec) {
       v[k] = xr[i];
+      if (add) {
+        const float4 q = gemm_value4(proj, m_tiles, m, 4 * i);
+        v[k].x += q.x; v[k].y += q.y; v[k].z += q.z; v[k].w += q.w;
+        xr[i] = v[k];
+      }
       ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
     }
   }
@@ -92,10 +101,13 @@ __global__ void __launch_bounds__(NORM_THREADS) rmsnorm_kernel(const float* __re
   }
 }
 
-cudaError_t launch_rmsnorm(int dtype, const float* x, const void* gain, void* out_t, float* out_f32, int d, float eps,
-                           const int32_t* m_total, int m_max, cudaStream_t st) {
+// x: residual stream (updated in place when proj != nullptr: x += proj).
+cudaError_t launch_rmsnorm(int dtype, float* x, const GemmOut* proj, const void* gain, void* out_t, float* out_f32, int d,
+                           float eps, const int32_t* m_total, int m_max, cudaStream_t st) {
   if (d > 4 * NORM_THREADS * NORM_MAXV || (d & 3)) return cudaErrorInvalidValue;
-  RD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T>, m_max, NORM_THREADS, 0, st, x, (const T*)gain, (T*)out_t, out_f32, d, eps, m_total));
+  GemmOut g{};
+  if (proj) g = *proj;
+  RD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T>, m_max, NORM_THREADS, 0, st, x, g, (const T*)gain, (T*)out_t, out_f32, d, eps, m_total));
   return cudaGetLastError();
 }
 
@@ -126,76 +138,94 @@ cudaError_t launch_rope_table(const int32_t* pos, float* table, int hd, float th
 // ---------------------------------------------------------------- rotary embedding + KV write
 // qkv: [M][3d] fp32 (Q | K | V).  Q is rotated in place; rotated K and V go to the cache slot of
 // the row.  Pairing (i, i + hd/2).
+constexpr int ROPE_SPLIT = 8;  // CTAs per row
+
 template <typename T>
-__global__ void rope_kv_kernel(float* __restrict__ qkv, T* __restrict__ kc, T* __restrict__ vc,
+__global__ void rope_kv_kernel(float* __restrict__ qkv, GemmOut proj, T* __restrict__ kc, T* __restrict__ vc,
                                const float2* __restrict__ table, RowTables rt, Dims dm, int* status) {
   pdl_enter();
   const int m = blockIdx.x;
-  if (m >= *rt.m_total) return;
+  const int M = *rt.m_total;
+  if (m >= M) return;
   const int b = rt.seq[m], slot = rt.slot[m];
   const int d = dm.d, hd = dm.hd, half = hd >> 1;
   const bool slot_ok = slot >= 0 && slot < dm.max_ctx;
-  if (!slot_ok && threadIdx.x == 0) atomicOr(status, DEV_ERR_CAPACITY);
+  if (!slot_ok && threadIdx.x == 0 && blockIdx.y == 0) atomicOr(status, DEV_ERR_CAPACITY);
+  const int m_tiles = gemm_m_tiles(proj, M);
   float* row = qkv + (size_t)m * 3 * d;
-  for (int idx = threadIdx.x; idx < dm.H * half; idx += blockDim.x) {
+  for (int idx = blockIdx.y * blockDim.x + threadIdx.x; idx < dm.H * half; idx += blockDim.x * gridDim.y) {
     const int h = idx / half, i = idx - h * half;
     const float2 cs = table[(size_t)m * half + i];
     const float c = cs.x, s = cs.y;
     const int o = h * hd + i;
-    const float q1 = row[o], q2 = row[o + half];
-    row[o] = q1 * c - q2 * s;
+    const float q1 = gemm_value(proj, m_tiles, m, o), q2 = gemm_value(proj, m_tiles, m, o + half);
+    const float k1 = gemm_value(proj, m_tiles, m, d + o), k2 = gemm_value(proj, m_tiles, m, d + o + half);
+    const float v1 = gemm_value(proj, m_tiles, m, 2 * d + o), v2 = gemm_value(proj, m_tiles, m, 2 * d + o + half);
+    row[o] = q1 * c - q2 * s;            // the attention kernel reads the rotated Q from here
     row[o + half] = q2 * c + q1 * s;
-    const float k1 = row[d + o], k2 = row[d + o + half];
     if (slot_ok) {
       const size_t base = (((size_t)b * dm.H + h) * dm.max_ctx + slot) * hd + i;
       kc[base] = from_f<T>(k1 * c - k2 * s);
       kc[base + half] = from_f<T>(k2 * c + k1 * s);
-      vc[base] = from_f<T>(row[2 * d + o]);
-      vc[base + half] = from_f<T>(row[2 * d + o + half]);
+      vc[base] = from_f<T>(v1);
+      vc[base + half] = from_f<T>(v2);
     }
   }
 }
 
-cudaError_t launch_rope_kv(int dtype, float* qkv, void* kcache, void* vcache, const float* table, const RowTables& rt,
-                           const Dims& dm, int m_max, int* status, cudaStream_t st) {
-  RD_DISPATCH(dtype, launch_pdl(rope_kv_kernel<T>, m_max, 256, 0, st, qkv, (T*)kcache, (T*)vcache,
-                                                            reinterpret_cast<const float2*>(table), rt, dm, status));
+cudaError_t launch_rope_kv(int dtype, float* qkv, const GemmOut& proj, void* kcache, void* vcache, const float* table,
+                           const RowTables& rt, const Dims& dm, int m_max, int* status, cudaStream_t st) {
+  dim3 grid(m_max, ROPE_SPLIT);
+  RD_DISPATCH(dtype, launch_pdl(rope_kv_kernel<T>, grid, 256, 0, st, qkv, proj, (T*)kcache, (T*)vcache,
+                                reinterpret_cast<const float2*>(table), rt, dm, status));
   return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------- SwiGLU
 template <typename T>
-__global__ void swiglu_kernel(const float* __restrict__ gu, T* __restrict__ out, int F, const int32_t* __restrict__ m_total) {
+__global__ void swiglu_kernel(GemmOut proj, T* __restrict__ out, int F, const int32_t* __restrict__ m_total) {
   pdl_enter();
   const int m = blockIdx.y;
-  if (m >= *m_total) return;
-  const int f = blockIdx.x * blockDim.x + threadIdx.x;
+  const int M = *m_total;
+  if (m >= M) return;
+  const int f = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (f >= F) return;
-  const float g = gu[(size_t)m * 2 * F + f], u = gu[(size_t)m * 2 * F + F + f];
-  out[(size_t)m * F + f] = from_f<T>(silu_f(g) * u);
+  const int m_tiles = gemm_m_tiles(proj, M);
+  const float4 g = gemm_value4(proj, m_tiles, m, f), u = gemm_value4(proj, m_tiles, m, F + f);
+  T* o = out + (size_t)m * F + f;
+  o[0] = from_f<T>(silu_f(g.x) * u.x); o[1] = from_f<T>(silu_f(g.y) * u.y);
+  o[2] = from_f<T>(silu_f(g.z) * u.z); o[3] = from_f<T>(silu_f(g.w) * u.w);
 }
 
-cudaError_t launch_swiglu(int dtype, const float* gu, void* out_t, int F, const int32_t* m_total, int m_max,
+// proj: the gate|up projection [M][2F]; out: [M][F].  F must be a multiple of 4.
+cudaError_t launch_swiglu(int dtype, const GemmOut& proj, void* out_t, int F, const int32_t* m_total, int m_max,
                           cudaStream_t st) {
-  dim3 grid((F + 255) / 256, m_max);
-  RD_DISPATCH(dtype, launch_pdl(swiglu_kernel<T>, grid, 256, 0, st, gu, (T*)out_t, F, m_total));
+  dim3 grid((F / 4 + 255) / 256, m_max);
+  RD_DISPATCH(dtype, launch_pdl(swiglu_kernel<T>, grid, 256, 0, st, proj, (T*)out_t, F, m_total));
   return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------- row argmax (lowest index on ties)
-__global__ void argmax_rows_kernel(const float* __restrict__ logits, int V, int32_t* __restrict__ out,
+__global__ void argmax_rows_kernel(float* __restrict__ logits, GemmOut proj, int V, int32_t* __restrict__ out,
                                    const int32_t* __restrict__ out_index, const int32_t* __restrict__ m_total) {
   pdl_enter();
   __shared__ float sv[32];
   __shared__ int si[32];
   const int m = blockIdx.x;
-  if (m >= *m_total) return;
-  const float* r = logits + (size_t)m * V;
+  const int M = *m_total;
+  if (m >= M) return;
+  float* r = logits + (size_t)m * V;
+  const int m_tiles = gemm_m_tiles(proj, M);
   float bv = -INFINITY;
   int bi = 0x7fffffff;
-  for (int i = threadIdx.x; i < V; i += blockDim.x) {
-    const float v = r[i];
-    if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+  // the complete logits are written back in place (later readers of the buffer see final values)
+  for (int i = threadIdx.x * 4; i < V; i += blockDim.x * 4) {
+    const float4 q = gemm_value4(proj, m_tiles, m, i);
+    *reinterpret_cast<float4*>(r + i) = q;
+    const float e[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (e[k] > bv || (e[k] == bv && i + k < bi)) { bv = e[k]; bi = i + k; }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
@@ -220,9 +250,10 @@ __global__ void argmax_rows_kernel(const float* __restrict__ logits, int V, int3
   }
 }
 
-cudaError_t launch_argmax_rows(const float* logits, int V, int32_t* out, const int32_t* out_index,
+// logits: the projection's output buffer [M][V] (V a multiple of 4), completed in place.
+cudaError_t launch_argmax_rows(float* logits, const GemmOut& proj, int V, int32_t* out, const int32_t* out_index,
                                const int32_t* m_total, int m_max, cudaStream_t st) {
-  launch_pdl(argmax_rows_kernel, m_max, 512, 0, st, logits, V, out, out_index, m_total);
+  launch_pdl(argmax_rows_kernel, m_max, 512, 0, st, logits, proj, V, out, out_index, m_total);
   return cudaGetLastError();
 }
 

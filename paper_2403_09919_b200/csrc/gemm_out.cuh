@@ -1,0 +1,115 @@
+// Where a projection's result lives until its consumer folds it.
+//
+// The tensor-core projection is a stream-K kernel: CTA c owns the contiguous unit range
+// [c*U/G, (c+1)*U/G) of the (tile, k-block) list, so a tile's k-range may be cut among several
+// CTAs.  The kernel applies no epilogue and does no cross-CTA reduction.  The contributor that
+// holds a tile's first k-block writes its sum to the fp32 output `raw`; every other contributor
+// (its range then starts inside that tile, so it has exactly one such segment) writes its sum to
+// its own slot of `partial`.  The kernel that consumes the projection (norm, rotary, SwiGLU,
+// argmax, ...) adds the slots to `raw` in CTA order -- a fixed order, so results are
+// deterministic -- while it does its own work.  This keeps fences, atomics and the serial
+// reduction out of the weight-streaming kernel.
+#pragma once
+#include <stdint.h>
+
+namespace rd {
+
+struct GemmOut {
+  const float* raw;      // [M][ld]
+  const float* partial;  // [grid][mt * 128], nullptr when nothing is cut (CUDA-core path)
+  int ld;
+  int nkb, n_tiles, mt, grid, m_tiles_max;
+  int all_work;          // every CTA has a non-empty range for any row count (units >= CTAs)
+};
+
+// Unit range of CTA c: [c*U/G, (c+1)*U/G).
+__host__ __device__ __forceinline__ long long gemm_range_begin(long long c, long long U, long long G) { return c * U / G; }
+// The CTA whose range holds unit u (the largest c with range_begin(c) <= u).
+__host__ __device__ __forceinline__ int gemm_cta_of_unit(long long u, long long U, long long G) {
+  const long long c = ((u + 1) * G - 1) / U;
+  return (int)(c > G - 1 ? G - 1 : c);
+}
+
+// Number of row tiles of a launch over M rows.
+__device__ __forceinline__ int gemm_m_tiles(const GemmOut& g, int M) { return g.m_tiles_max == 1 ? 1 : (M + g.mt - 1) / g.mt; }
+
+// Contributors of the tile that holds (m, n) other than the first: CTAs c_first+1 .. c_last.
+struct GemmFold {
+  int c_next, c_last;   // first non-first contributor, last contributor
+  size_t off;           // element offset of (m, n) inside a slot
+};
+__device__ __forceinline__ GemmFold gemm_fold(const GemmOut& g, int m_tiles, int m, int n) {
+  const int n_tile = n >> 7, row = n & 127;
+  GemmFold f;
+  if (g.m_tiles_max == 1) {
+    // one row tile (the decode-time case): 32-bit arithmetic, (units + 1) * CTAs stays far below 2^31
+    const uint32_t U = (uint32_t)g.n_tiles * g.nkb, G = g.grid, tu0 = (uint32_t)n_tile * g.nkb;
+    const uint32_t cf = ((tu0 + 1) * G - 1) / U, cl = ((tu0 + g.nkb) * G - 1) / U;
+    f.c_next = (int)(cf > G - 1 ? G - 1 : cf) + 1;
+    f.c_last = (int)(cl > G - 1 ? G - 1 : cl);
+    f.off = (size_t)m * 128 + row;
+    return f;
+  }
+  const int m_tile = m / g.mt, col = m - m_tile * g.mt;
+  const long long t = (long long)n_tile * m_tiles + m_tile;
+  const long long U = (long long)g.n_tiles * m_tiles * g.nkb, G = g.grid;
+  const long long tu0 = t * g.nkb;
+  f.c_next = gemm_cta_of_unit(tu0, U, G) + 1;
+  f.c_last = gemm_cta_of_unit(tu0 + g.nkb - 1, U, G);
+  f.off = (size_t)col * 128 + row;
+  return f;
+}
+// True when CTA c has work (with fewer units than CTAs some ranges are empty).
+__device__ __forceinline__ bool gemm_has_work(const GemmOut& g, int m_tiles, int c) {
+  if (g.all_work) return true;
+  const long long U = (long long)g.n_tiles * m_tiles * g.nkb, G = g.grid;
+  return gemm_range_begin(c, U, G) < gemm_range_begin(c + 1, U, G);
+}
+
+constexpr int GEMM_FOLD_UNROLL = 8;  // slots loaded together (a tile rarely has more contributors)
+
+// The complete value of output element (m, n): all slot loads are issued together, the sum is taken
+// in CTA order.
+__device__ __forceinline__ float gemm_value(const GemmOut& g, int m_tiles, int m, int n) {
+  float v = g.raw[(size_t)m * g.ld + n];
+  if (g.partial == nullptr) return v;
+  const GemmFold f = gemm_fold(g, m_tiles, m, n);
+  const size_t slot = (size_t)g.mt * 128;
+  float q[GEMM_FOLD_UNROLL];
+#pragma unroll
+  for (int j = 0; j < GEMM_FOLD_UNROLL; ++j) {
+    const int c = f.c_next + j;
+    q[j] = (c <= f.c_last && gemm_has_work(g, m_tiles, c)) ? __ldcg(g.partial + (size_t)c * slot + f.off) : 0.f;
+  }
+#pragma unroll
+  for (int j = 0; j < GEMM_FOLD_UNROLL; ++j) v += q[j];
+  for (int c = f.c_next + GEMM_FOLD_UNROLL; c <= f.c_last; ++c)
+    if (gemm_has_work(g, m_tiles, c)) v += __ldcg(g.partial + (size_t)c * slot + f.off);
+  return v;
+}
+
+// Four consecutive columns n .. n+3 (n a multiple of 4: they share a tile and the slots' alignment).
+__device__ __forceinline__ float4 gemm_value4(const GemmOut& g, int m_tiles, int m, int n) {
+  float4 v = *reinterpret_cast<const float4*>(g.raw + (size_t)m * g.ld + n);
+  if (g.partial == nullptr) return v;
+  const GemmFold f = gemm_fold(g, m_tiles, m, n);
+  const size_t slot = (size_t)g.mt * 128;
+  float4 q[GEMM_FOLD_UNROLL];
+#pragma unroll
+  for (int j = 0; j < GEMM_FOLD_UNROLL; ++j) {
+    const int c = f.c_next + j;
+    q[j] = (c <= f.c_last && gemm_has_work(g, m_tiles, c))
+               ? __ldcg(reinterpret_cast<const float4*>(g.partial + (size_t)c * slot + f.off))
+               : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+#pragma unroll
+  for (int j = 0; j < GEMM_FOLD_UNROLL; ++j) { v.x += q[j].x; v.y += q[j].y; v.z += q[j].z; v.w += q[j].w; }
+  for (int c = f.c_next + GEMM_FOLD_UNROLL; c <= f.c_last; ++c) {
+    if (!gemm_has_work(g, m_tiles, c)) continue;
+    const float4 t = __ldcg(reinterpret_cast<const float4*>(g.partial + (size_t)c * slot + f.off));
+    v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
+  }
+  return v;
+}
+
+}  // namespace rd

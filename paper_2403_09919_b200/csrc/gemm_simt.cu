@@ -1,4 +1,4 @@
-// CUDA-core projection Y[m][n] = sum_k A[m][k] W[n][k] with the fused epilogue.
+// CUDA-core projection Y[m][n] = sum_k A[m][k] W[n][k] (fp32 result; the consumer applies the epilogue).
 //
 // Used for the fp32 configuration (no tensor-core path for fp32 operands is wanted there: the
 // point of that configuration is tight parity) and for very small M (the autoregressive
@@ -7,7 +7,7 @@
 // sums, so the weight is read exactly once per MT rows.
 #include "rd_internal.cuh"
 #include "pdl.cuh"
-#include "epilogue.cuh"
+#include "gemm_out.cuh"
 
 namespace rd {
 
@@ -44,7 +44,8 @@ template <> struct Vec<__nv_bfloat16> {
 // grid (ceil(N / 8), ceil(m_max / MT)), block 256 = 8 warps, one weight row per warp.
 template <typename T, int MT>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ A, int lda, const T* __restrict__ W, int N,
-                                                        int K, const int32_t* __restrict__ m_total, Epilogue ep) {
+                                                        int K, const int32_t* __restrict__ m_total, float* __restrict__ raw,
+                                                        int ld_raw) {
   pdl_enter();
   constexpr int VN = Vec<T>::N;
   const int M = *m_total;
@@ -78,26 +79,30 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ A,
   }
 #pragma unroll
   for (int r = 0; r < MT; ++r)
-    if (lane == r && r < rows) apply_epilogue<T>(ep, m0 + r, n, acc[r]);
+    if (lane == r && r < rows) raw[(size_t)(m0 + r) * ld_raw + n] = acc[r];
 }
 
 cudaError_t launch_gemm_simt(int dtype, const void* A, int lda, const void* W, int N, int K, const int32_t* m_total,
-                             int m_max, const Epilogue& ep, cudaStream_t st) {
+                             int m_max, float* raw, int ld_raw, GemmOut* out_desc, cudaStream_t st) {
+  if (out_desc) {
+    out_desc->raw = raw; out_desc->partial = nullptr; out_desc->ld = ld_raw; out_desc->nkb = 1; out_desc->n_tiles = 1;
+    out_desc->mt = 1; out_desc->grid = 1; out_desc->m_tiles_max = 1; out_desc->all_work = 1;
+  }
   if (m_max <= 0) return cudaSuccess;
   if (m_max <= 2) {
     dim3 grid((N + 7) / 8, (m_max + 1) / 2);
     if (dtype == RD_DTYPE_FP32)
-      launch_pdl(gemm_simt_kernel<float, 2>, grid, 256, 0, st, (const float*)A, lda, (const float*)W, N, K, m_total, ep);
+      launch_pdl(gemm_simt_kernel<float, 2>, grid, 256, 0, st, (const float*)A, lda, (const float*)W, N, K, m_total, raw, ld_raw);
     else
-      launch_pdl(gemm_simt_kernel<__nv_bfloat16, 2>, grid, 256, 0, st, (const __nv_bfloat16*)A, lda, (const __nv_bfloat16*)W, N,
-                                                                K, m_total, ep);
+      launch_pdl(gemm_simt_kernel<__nv_bfloat16, 2>, grid, 256, 0, st, (const __nv_bfloat16*)A, lda,
+                 (const __nv_bfloat16*)W, N, K, m_total, raw, ld_raw);
   } else {
     dim3 grid((N + 7) / 8, (m_max + 7) / 8);
     if (dtype == RD_DTYPE_FP32)
-      launch_pdl(gemm_simt_kernel<float, 8>, grid, 256, 0, st, (const float*)A, lda, (const float*)W, N, K, m_total, ep);
+      launch_pdl(gemm_simt_kernel<float, 8>, grid, 256, 0, st, (const float*)A, lda, (const float*)W, N, K, m_total, raw, ld_raw);
     else
-      launch_pdl(gemm_simt_kernel<__nv_bfloat16, 8>, grid, 256, 0, st, (const __nv_bfloat16*)A, lda, (const __nv_bfloat16*)W, N,
-                                                                K, m_total, ep);
+      launch_pdl(gemm_simt_kernel<__nv_bfloat16, 8>, grid, 256, 0, st, (const __nv_bfloat16*)A, lda,
+                 (const __nv_bfloat16*)W, N, K, m_total, raw, ld_raw);
   }
   return cudaGetLastError();
 }

@@ -10,11 +10,11 @@
 // Schedule: persistent, one CTA per SM, stream-K.  The work is the list of (tile, k-block) units,
 // tile = (128 weight rows) x (MT activation rows), k-block = 64 columns; CTA c owns the contiguous
 // unit range [c*U/G, (c+1)*U/G), so every SM streams the same number of weight bytes whatever the
-// shape.  A CTA whose range cuts a tile writes its fp32 partial to scratch; the last contributor
-// of that tile (found with an atomic counter, never by waiting) adds the partials in CTA order --
-// a fixed order, so results are deterministic -- and applies the epilogue.
+// shape.  No epilogue and no cross-CTA reduction happen here: the segment that holds a tile's first
+// k-block stores its fp32 sums to the output, any other segment to the CTA's partial slot, and the
+// consuming kernel folds them in CTA order (gemm_out.cuh).
 //
-// Roles: warp 0 = TMA producer (weights 128x64 per stage, activations MT x 64 as 16-row boxes),
+// Roles: warp 0 = TMA producer (one 128x64 weight box and one MTx64 activation box per stage),
 // warp 1 = MMA issuer and TMEM owner, warps 2..5 = epilogue (tcgen05.ld, one TMEM lane quarter
 // each).  Two TMEM accumulators alternate so the epilogue of one segment overlaps the MMAs of the
 // next; the smem ring (full/empty mbarriers) never drains between tiles.
@@ -23,8 +23,9 @@
 // status word, lets its copies land, frees its TMEM and exits; later launches see the flag and
 // return at once.
 #include <cuda.h>
+#include <stdlib.h>
 
-#include "epilogue.cuh"
+#include "gemm_out.cuh"
 #include "pdl.cuh"
 #include "rd_internal.cuh"
 
@@ -35,19 +36,20 @@ namespace {
 constexpr int TILE_N = 128;       // weight rows per tile (MMA M)
 constexpr int TILE_K = 64;        // bf16 per k-block = one 128-byte swizzle row
 constexpr int W_STAGE_BYTES = TILE_N * TILE_K * 2;
-constexpr int A_BOX_ROWS = 16;
-constexpr int A_BOX_BYTES = A_BOX_ROWS * TILE_K * 2;
 constexpr int NUM_THREADS = 192;
 constexpr unsigned long long WAIT_LIMIT_NS = 1000000000ull;
+constexpr long long L2_PREFETCH_BYTES = 0;  // of the next projection's weights into L2; measured: any amount slows the step
 
 struct TcParams {
   int N, K, nkb, n_tiles, mt, m_tiles_max, stages, tmem_cols;
   const int32_t* m_total;
-  float* partial;     // [2 * gridDim.x][mt * 128]
-  int32_t* counters;  // [n_tiles * m_tiles_max], zero between launches
+  float* raw;         // [M][ld_raw] fp32 output
+  int ld_raw;
+  float* partial;     // [gridDim.x][mt * 128]
   int32_t* status;
   unsigned long long* trace;  // 8 timestamps of this launch (see redrafter_trace_read) or nullptr
-  Epilogue ep;
+  // L2 prefetch of the weights the NEXT projection will read first (0 units = none)
+  int next_nkb, next_n_tiles, pf_units;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -96,6 +98,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* map, int x, int y) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y) : "memory");
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
@@ -134,16 +140,9 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-// Unit range of CTA c: [c*U/G, (c+1)*U/G).
-__device__ __forceinline__ long long range_begin(long long c, long long U, long long G) { return c * U / G; }
-// The CTA whose range holds unit u (the largest c with range_begin(c) <= u).
-__device__ __forceinline__ int cta_of_unit(long long u, long long U, long long G) {
-  long long c = ((u + 1) * G - 1) / U;
-  return (int)(c > G - 1 ? G - 1 : c);
-}
-
 __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
                                                                  const __grid_constant__ CUtensorMap map_a,
+                                                                 const __grid_constant__ CUtensorMap map_next,
                                                                  const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   pdl_launch_dependents();  // the next kernel may start its own prologue now
@@ -163,7 +162,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
   const int m_tiles = early ? 1 : (*p.m_total + p.mt - 1) / p.mt;
   const long long G = gridDim.x;
   const long long U = (long long)p.n_tiles * m_tiles * p.nkb;
-  const long long u0 = range_begin(blockIdx.x, U, G), u1 = range_begin(blockIdx.x + 1, U, G);
+  const long long u0 = gemm_range_begin(blockIdx.x, U, G), u1 = gemm_range_begin(blockIdx.x + 1, U, G);
 
   // ---- shared memory carve-up (stage buffers 1024-byte aligned for the 128-byte swizzle)
   const uint32_t raw = smem_u32(smem_raw);
@@ -178,14 +177,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
   uint8_t* misc = smem_raw + (bar_base - raw) + 8u * (2 * p.stages + 4);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
-  volatile int* last_flag = reinterpret_cast<volatile int*>(misc + 8);
   volatile int* epi_ok = reinterpret_cast<volatile int*>(misc + 12);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
     *abort_flag = 0;
-    *last_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -217,9 +214,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
         const int t = (int)(u / p.nkb), kb = (int)(u - (long long)t * p.nkb);
         const int s = i % p.stages;
         const int m_tile = t - (t / m_tiles) * m_tiles;
-        for (int j = 0; j < p.mt / A_BOX_ROWS; ++j)
-          tma_load_2d(base + s * stage_bytes + W_STAGE_BYTES + j * A_BOX_BYTES, &map_a, full_bar(s), kb * TILE_K,
-                      m_tile * p.mt + j * A_BOX_ROWS);
+        // one box of MT rows: the TMA unit's cost is per operation, not per byte, at these sizes
+        tma_load_2d(base + s * stage_bytes + W_STAGE_BYTES, &map_a, full_bar(s), kb * TILE_K, m_tile * p.mt);
       };
       // weights of the first ring-full of k-blocks do not depend on the preceding kernels
       for (uint32_t i = 0; i < pre; ++i) issue_w(i);
@@ -233,6 +229,18 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
         if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
         issue_w(i);
         issue_a(i);
+      }
+      // The decode step is a fixed chain of projections separated by short kernels.  Once this CTA's own
+      // loads are issued it asks the L2 (126 MB) for the tiles the same CTA index will read first in the
+      // NEXT projection, so HBM keeps streaming weights through this kernel's tail and the gap behind it.
+      if (ok && p.pf_units > 0) {
+        const long long Un = (long long)p.next_n_tiles * p.next_nkb;
+        const long long v0 = gemm_range_begin(blockIdx.x, Un, G);
+        const long long v1 = min(gemm_range_begin(blockIdx.x + 1, Un, G), v0 + p.pf_units);
+        for (long long v = v0; v < v1; ++v) {
+          const int t = (int)(v / p.next_nkb), kb = (int)(v - (long long)t * p.next_nkb);
+          tma_prefetch_l2_2d(&map_next, kb * TILE_K, t * TILE_N);
+        }
       }
       if (!ok) {  // give the copies already issued time to land before the CTA's shared memory is released
         const unsigned long long t0 = globaltimer();
@@ -283,7 +291,6 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
       const int kb1 = (int)min((long long)p.nkb, kb0 + (u1 - u));
       const int n_tile = t / m_tiles, m_tile = t - n_tile * m_tiles;
       const uint32_t a = seg & 1u, aph = (seg >> 1) & 1u;
-      const bool complete = (kb0 == 0 && kb1 == p.nkb);
       const int n = n_tile * TILE_N + row;
       const int m_base = m_tile * p.mt;
       // one thread does the bounded wait and tells the others, so that all 128 take the same branch
@@ -292,67 +299,27 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
       if (!*epi_ok) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * (uint32_t)p.mt;
-      // slot 0 = this CTA's first segment, slot 1 = its last (a range has at most two cut tiles)
-      float* my_partial = p.partial + ((size_t)blockIdx.x * 2 + (u == u0 ? 0 : 1)) * ((size_t)p.mt * TILE_N);
+      float* my_partial = p.partial + (size_t)blockIdx.x * ((size_t)p.mt * TILE_N);
       for (int c0 = 0; c0 < p.mt; c0 += 16) {
         uint32_t r[16];
         tmem_ld16(taddr + c0, r);
-        if (complete) {
-          float v[16];
+        if (kb0 == 0) {
+          // this segment holds the tile's first k-block: its sums go to the output
+          if (n < p.N) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
-          if (n < p.N) apply_epilogue16<__nv_bfloat16>(p.ep, m_base + c0, M, n, v);
+            for (int j = 0; j < 16; ++j) {
+              const int m = m_base + c0 + j;
+              if (m < M) p.raw[(size_t)m * p.ld_raw + n] = __uint_as_float(r[j]);
+            }
+          }
         } else {
+          // the range starts inside this tile: at most one such segment per CTA
 #pragma unroll
           for (int j = 0; j < 16; ++j) my_partial[(size_t)(c0 + j) * TILE_N + row] = __uint_as_float(r[j]);
         }
       }
       tc_fence_before();
       mbar_arrive(tempty_bar(a));  // the accumulator may be overwritten
-      if (!complete) {
-        // publish the partial, then find out whether this CTA is the tile's last contributor
-        __threadfence();
-        epi_bar_sync();
-        const long long tu0 = (long long)t * p.nkb, tu1 = tu0 + p.nkb;
-        const int c_first = cta_of_unit(tu0, U, G), c_last = cta_of_unit(tu1 - 1, U, G);
-        if (et == 0) {
-          int contributors = 0;
-          for (int c = c_first; c <= c_last; ++c) contributors += range_begin(c, U, G) < range_begin(c + 1, U, G) ? 1 : 0;
-          const int old = atomicAdd(p.counters + t, 1);
-          *last_flag = (old == contributors - 1) ? 1 : 0;
-          if (old == contributors - 1) p.counters[t] = 0;  // ready for the next launch
-        }
-        epi_bar_sync();
-        if (*last_flag) {
-          __threadfence();
-          // address of contributor c's partial for this tile (nullptr for a CTA with an empty range)
-          auto partial_of = [&](int c) -> const float* {
-            const long long cb = range_begin(c, U, G), ce = range_begin(c + 1, U, G);
-            if (cb >= ce) return nullptr;
-            const int slot = (cb / p.nkb == t) ? 0 : 1;
-            return p.partial + ((size_t)c * 2 + slot) * ((size_t)p.mt * TILE_N) + row;
-          };
-          for (int c0 = 0; c0 < p.mt; c0 += 16) {
-            float acc[16];
-#pragma unroll
-            for (int j = 0; j < 16; ++j) acc[j] = 0.f;
-            // two contributors per round so that 32 loads are in flight; the sums stay in CTA order
-            for (int c = c_first; c <= c_last; c += 2) {
-              const float* pa = partial_of(c);
-              const float* pb = (c + 1 <= c_last) ? partial_of(c + 1) : nullptr;
-              float ta[16], tb[16];
-#pragma unroll
-              for (int j = 0; j < 16; ++j) ta[j] = pa ? __ldcg(pa + (size_t)(c0 + j) * TILE_N) : 0.f;
-#pragma unroll
-              for (int j = 0; j < 16; ++j) tb[j] = pb ? __ldcg(pb + (size_t)(c0 + j) * TILE_N) : 0.f;
-#pragma unroll
-              for (int j = 0; j < 16; ++j) acc[j] = (acc[j] + ta[j]) + tb[j];
-            }
-            if (n < p.N) apply_epilogue16<__nv_bfloat16>(p.ep, m_base + c0, M, n, acc);
-          }
-        }
-        epi_bar_sync();  // last_flag is rewritten by the next cut segment
-      }
       u += kb1 - kb0;
     }
   }
@@ -403,7 +370,6 @@ int tc_make_map(void* out_map, const void* ptr, uint64_t rows, uint64_t cols, ui
 }
 
 int tc_weight_box_rows() { return TILE_N; }
-int tc_act_box_rows() { return A_BOX_ROWS; }
 
 // Activation rows per tile for a launch whose row count is at most m_max.
 int tc_pick_mt(int m_max) {
@@ -413,8 +379,7 @@ int tc_pick_mt(int m_max) {
   return mt < 16 ? 16 : mt;
 }
 
-size_t tc_partial_floats(int grid, int mt) { return (size_t)2 * grid * mt * TILE_N; }
-size_t tc_counter_ints(int N, int m_max) { return (size_t)((N + TILE_N - 1) / TILE_N) * ((m_max + 15) / 16); }
+size_t tc_partial_floats(int grid, int mt) { return (size_t)grid * mt * TILE_N; }
 
 cudaError_t tc_prepare(int* smem_limit_out) {
   int dev = 0, lim = 0;
@@ -432,25 +397,45 @@ cudaError_t tc_prepare(int* smem_limit_out) {
 }
 
 cudaError_t launch_gemm_tc(const void* map_w, const void* map_a, int N, int K, const int32_t* m_total, int m_max,
-                           const Epilogue& ep, float* partial, int32_t* counters, int32_t* status, int grid,
-                           int smem_limit, unsigned long long* trace, cudaStream_t st) {
-  if (m_max <= 0) return cudaSuccess;
+                           float* raw, int ld_raw, float* partial, int32_t* status, int grid, int smem_limit,
+                           unsigned long long* trace, const void* map_next, int next_N, int next_K, GemmOut* out_desc,
+                           cudaStream_t st) {
   TcParams p;
   p.N = N; p.K = K; p.nkb = (K + TILE_K - 1) / TILE_K; p.n_tiles = (N + TILE_N - 1) / TILE_N;
-  p.mt = tc_pick_mt(m_max);
-  p.m_tiles_max = (m_max + p.mt - 1) / p.mt;
+  p.mt = tc_pick_mt(m_max > 0 ? m_max : 1);
+  p.m_tiles_max = m_max > 0 ? (m_max + p.mt - 1) / p.mt : 1;
+  if (out_desc) {
+    out_desc->raw = raw; out_desc->partial = partial; out_desc->ld = ld_raw; out_desc->nkb = p.nkb;
+    out_desc->n_tiles = p.n_tiles; out_desc->mt = p.mt; out_desc->grid = grid; out_desc->m_tiles_max = p.m_tiles_max;
+    out_desc->all_work = ((long long)p.n_tiles * p.nkb >= grid) ? 1 : 0;
+  }
+  if (m_max <= 0) return cudaSuccess;
   const int stage_bytes = W_STAGE_BYTES + p.mt * TILE_K * 2;
   const int overhead = 1024 + 8 * (2 * 16 + 4) + 64;
-  int stages = (smem_limit - overhead) / stage_bytes;
+  // Skinny launches (the decode step) leave about 70 KB of the SM's shared memory to the small kernels
+  // that run between projections, so that this kernel can become resident, and start its weight
+  // stream, while they are still running.
+  static const int cap_kb = getenv("RD_TC_SMEM_KB") ? atoi(getenv("RD_TC_SMEM_KB")) : 160;   // tuning toggles
+  static const long long pf_bytes = getenv("RD_TC_PREFETCH_MB") ? (long long)atoi(getenv("RD_TC_PREFETCH_MB")) << 20 : L2_PREFETCH_BYTES;
+  const int budget = p.mt <= 64 ? (smem_limit < cap_kb * 1024 ? smem_limit : cap_kb * 1024) : smem_limit;
+  int stages = (budget - overhead) / stage_bytes;
   if (stages > 16) stages = 16;
   if (stages < 2) return cudaErrorInvalidConfiguration;
   p.stages = stages;
   int cols = 32;
   while (cols < 2 * p.mt) cols <<= 1;
   p.tmem_cols = cols;
-  p.m_total = m_total; p.partial = partial; p.counters = counters; p.status = status; p.ep = ep; p.trace = trace;
+  p.m_total = m_total; p.raw = raw; p.ld_raw = ld_raw; p.partial = partial; p.status = status; p.trace = trace;
+  p.next_nkb = 0; p.next_n_tiles = 0; p.pf_units = 0;
+  if (map_next) {
+    p.next_nkb = (next_K + TILE_K - 1) / TILE_K;
+    p.next_n_tiles = (next_N + TILE_N - 1) / TILE_N;
+    const long long per_cta = (pf_bytes / W_STAGE_BYTES) / grid;
+    p.pf_units = (int)per_cta;
+  }
   const size_t smem = (size_t)stages * stage_bytes + overhead;
-  launch_pdl(gemm_tc_kernel, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, *(const CUtensorMap*)map_a, p);
+  launch_pdl(gemm_tc_kernel, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, *(const CUtensorMap*)map_a,
+             *(const CUtensorMap*)(map_next ? map_next : map_w), p);
   return cudaGetLastError();
 }
 

@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "gemm_out.cuh"
 #include "redrafter.h"
 
 namespace rd {
@@ -40,17 +41,6 @@ struct RowTables {
   const int32_t* m_total;     // [1] number of valid rows (device)
 };
 
-// Epilogue of every projection: v = acc (+ addend) (+ bias[n]) -> act -> (+ resid) -> out.
-struct Epilogue {
-  const float* addend;   // [M][ld_addend] or nullptr
-  const void* bias;      // [N] in weight dtype or nullptr
-  const float* resid;    // [M][ld_resid] or nullptr (may alias out_f32)
-  float* out_f32;        // [M][ld_out_f32] or nullptr
-  void* out_t;           // [M][ld_out_t] in activation dtype, or nullptr
-  int ld_addend, ld_resid, ld_out_f32, ld_out_t;
-  int silu;              // apply SiLU after bias
-};
-
 struct Dims {
   int n_layers, d, H, hd, F, V, dr, dh, n_head_layers;
   int B, max_ctx, BW, L, NMAX, MW;
@@ -59,30 +49,29 @@ struct Dims {
 };
 
 // ---- launchers (definitions in the .cu files; all enqueue on `st`, return cudaGetLastError) ----
-// Y[m][n] = sum_k A[m][k] W[n][k], M rows given by *m_total (<= m_max), on CUDA cores.
+// Y[m][n] = sum_k A[m][k] W[n][k], M rows given by *m_total (<= m_max), on CUDA cores.  Fills *out_desc.
 cudaError_t launch_gemm_simt(int dtype, const void* A, int lda, const void* W, int N, int K, const int32_t* m_total,
-                             int m_max, const Epilogue& ep, cudaStream_t st);
+                             int m_max, float* raw, int ld_raw, GemmOut* out_desc, cudaStream_t st);
 
 // Tensor-core (tcgen05) projection, bf16 only.  Operands are passed as TMA descriptors.
 int tc_make_map(void* out_map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows);
 int tc_weight_box_rows();
-int tc_act_box_rows();
 int tc_pick_mt(int m_max);
 size_t tc_partial_floats(int grid, int mt);
-size_t tc_counter_ints(int N, int m_max);
 cudaError_t tc_prepare(int* smem_limit_out);
 cudaError_t launch_gemm_tc(const void* map_w, const void* map_a, int N, int K, const int32_t* m_total, int m_max,
-                           const Epilogue& ep, float* partial, int32_t* counters, int32_t* status, int grid,
-                           int smem_limit, unsigned long long* trace, cudaStream_t st);
+                           float* raw, int ld_raw, float* partial, int32_t* status, int grid, int smem_limit,
+                           unsigned long long* trace, const void* map_next, int next_N, int next_K, GemmOut* out_desc,
+                           cudaStream_t st);
 
 cudaError_t launch_embed(int dtype, const void* emb, const int32_t* tok, float* x, int d, int V, const int32_t* m_total,
                          int m_max, int* status, cudaStream_t st);
-cudaError_t launch_rmsnorm(int dtype, const float* x, const void* gain, void* out_t, float* out_f32, int d, float eps,
-                           const int32_t* m_total, int m_max, cudaStream_t st);
+cudaError_t launch_rmsnorm(int dtype, float* x, const GemmOut* proj, const void* gain, void* out_t, float* out_f32, int d,
+                           float eps, const int32_t* m_total, int m_max, cudaStream_t st);
 cudaError_t launch_rope_table(const int32_t* pos, float* table, int hd, float theta, const int32_t* m_total, int m_max,
                               cudaStream_t st);
-cudaError_t launch_rope_kv(int dtype, float* qkv, void* kcache, void* vcache, const float* table, const RowTables& rt,
-                           const Dims& dm, int m_max, int* status, cudaStream_t st);
+cudaError_t launch_rope_kv(int dtype, float* qkv, const GemmOut& proj, void* kcache, void* vcache, const float* table,
+                           const RowTables& rt, const Dims& dm, int m_max, int* status, cudaStream_t st);
 cudaError_t launch_attention(int dtype, const float* qkv, const void* kcache, const void* vcache, void* out_t,
                              const RowTables& rt, const Dims& dm, int m_max, cudaStream_t st);
 // Tensor-core attention (bf16): KV tiles staged through shared memory, split over the keys.
@@ -92,20 +81,22 @@ cudaError_t attn_tc_prepare(int hd, int MW);
 cudaError_t launch_attention_tc(const float* qkv, const void* kcache, const void* vcache, void* out, const RowTables& rt,
                                 const int32_t* seq_off, const Dims& dm, int n_seq, int row_blocks, int n_splits,
                                 float* scratch, int32_t* counters, cudaStream_t st);
-cudaError_t launch_swiglu(int dtype, const float* gu, void* out_t, int F, const int32_t* m_total, int m_max,
+cudaError_t launch_swiglu(int dtype, const GemmOut& proj, void* out_t, int F, const int32_t* m_total, int m_max,
                           cudaStream_t st);
-cudaError_t launch_argmax_rows(const float* logits, int V, int32_t* out, const int32_t* out_index,
+cudaError_t launch_argmax_rows(float* logits, const GemmOut& proj, int V, int32_t* out, const int32_t* out_index,
                                const int32_t* m_total, int m_max, cudaStream_t st);
 
 // drafter
 cudaError_t launch_draft_init(int dtype, const void* emb, const int32_t* root, const float* h, void* x_t, float* x_f,
-                              void* sprev_t, const Dims& dm, int B, int* status, cudaStream_t st);
-cudaError_t launch_row_topk(const float* logits, int V, int BW, float* lse, float* val, int32_t* idx, int rows,
-                            cudaStream_t st);
+                              void* se_t, const Dims& dm, int B, int* status, cudaStream_t st);
+cudaError_t launch_act(int dtype, const GemmOut& proj, const void* bias, const float* resid, int ld_resid, float* out_f,
+                       void* out_t, int ld_out, int N, const int32_t* m_total, int m_max, cudaStream_t st);
+cudaError_t launch_row_topk(const GemmOut& proj, int V, int BW, float* lse, float* val, int32_t* idx, int rows,
+                            const int32_t* m_total, cudaStream_t st);
 cudaError_t launch_beam_merge(int dtype, int call, const float* lse, const float* val, const int32_t* idx,
                               const float* score_in, float* score_out, const int32_t* hist_in, int32_t* hist_out,
-                              const void* emb, const float* s_new_f, int ld_s, void* sprev_t, void* e_t,
-                              const Dims& dm, int B, int32_t* beams_out, float* scores_out, cudaStream_t st);
+                              const void* emb, const float* s_new_f, int ld_s, void* se_t, const Dims& dm, int B,
+                              int32_t* beams_out, float* scores_out, cudaStream_t st);
 cudaError_t launch_fill_h(int dtype, const float* h, void* x_t, float* x_f, const Dims& dm, int B, cudaStream_t st);
 
 // pack / accept
