@@ -49,7 +49,7 @@ struct Workspace {
   // tensor-core projection scratch
   float* tc_partial;
   // tensor-core attention scratch
-  int32_t* att_counters;
+  int32_t *att_counters, *sel_counters;
   float* att_scratch;
   unsigned long long* trace;  // [TRACE_SLOTS][8] timestamps of traced projection launches
 };
@@ -163,6 +163,7 @@ void carve(Bump& bp, const Dims& dm, int m_cap, Workspace* w) {
   w->one_b = bp.take<int32_t>(4); w->one_r = bp.take<int32_t>(4);
   w->seq_off = bp.take<int32_t>(B + 1);
   w->att_counters = bp.take<int32_t>(ATT_MAX_SPLIT_BLOCKS);
+  w->sel_counters = bp.take<int32_t>(B);
   w->x = bp.take<float>((size_t)m_cap * dm.d);
   w->qkv = bp.take<float>((size_t)m_cap * 3 * dm.d);
   w->proj_d = bp.take<float>((size_t)m_cap * dm.d);
@@ -378,9 +379,9 @@ int do_draft(rd_handle* h, cudaStream_t st, int32_t* beams, float* scores) {
     int rc = gemm(h, xin_t, dm.dh, h->w.draft_out, dm.V, dm.dh, mt, rows, w.dlogits, dm.V, &g,
                   call < dm.L ? (const void*)w.uw : h->wqkv[0], st);
     if (rc) return rc;
-    CKP(h, PROF_DRAFT_SMALL, launch_row_topk(g, dm.V, dm.BW, w.lse, w.cand_val, w.cand_idx, rows, mt, st));
-    CKP(h, PROF_DRAFT_SMALL, launch_beam_merge(dm.dtype, call, w.lse, w.cand_val, w.cand_idx, sc_in, sc_out, hi_in, hi_out,
-                                               h->w.tok_emb, w.x0_f, dm.dh, w.se_t, dm, B, beams, scores, st));
+    CKP(h, PROF_DRAFT_SMALL, launch_draft_select(dm.dtype, g, call, w.lse, w.cand_val, w.cand_idx, sc_in, sc_out, hi_in, hi_out,
+                                                 h->w.tok_emb, w.x0_f, dm.dh, w.se_t, dm, B, beams, scores, w.sel_counters, mt,
+                                                 (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) ? w.trace + (size_t)8 * h->trace_next++ : nullptr, st));
     float* tf = sc_in; sc_in = sc_out; sc_out = tf;
     int32_t* ti = hi_in; hi_in = hi_out; hi_out = ti;
   }

@@ -100,9 +100,9 @@ cudaError_t launch_act(int dtype, const GemmOut& proj, const void* bias, const f
   return cudaGetLastError();
 }
 
-// ---------------------------------------------------------------- per-row log-sum-exp + top-BW
-// Ordering (value desc, index asc).  Selection is stateless: pass p picks the best element that
-// comes strictly after the element picked by pass p-1, so nothing is marked or modified.
+// ---------------------------------------------------------------- selection: log-softmax, top-BW, beam pruning
+// Ordering of candidates: (value desc, index asc).  Selection is stateless: round p picks the best
+// element that comes strictly after the one picked by round p-1, so nothing is marked or modified.
 struct Cand {
   float v;
   int i;
@@ -111,8 +111,7 @@ __device__ __forceinline__ bool cand_before(float va, int ia, float vb, int ib) 
   return va > vb || (va == vb && ia < ib);
 }
 __device__ __forceinline__ Cand cand_best(Cand a, Cand b) { return cand_before(a.v, a.i, b.v, b.i) ? a : b; }
-__device__ __forceinline__ Cand block_best(Cand c, Cand* sh) {
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+__device__ __forceinline__ Cand warp_best(Cand c) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     Cand t;
@@ -120,171 +119,268 @@ __device__ __forceinline__ Cand block_best(Cand c, Cand* sh) {
     t.i = __shfl_xor_sync(0xffffffffu, c.i, o);
     c = cand_best(c, t);
   }
+  return c;  // identical in every lane
+}
+__device__ __forceinline__ float block_reduce_sum(float s, float* sh) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
   __syncthreads();
-  if (lane == 0) sh[w] = c;
+  if (lane == 0) sh[w] = s;
   __syncthreads();
-  Cand r = lane < nw ? sh[lane] : Cand{-INFINITY, 0x7fffffff};
+  s = lane < nw ? sh[lane] : 0.f;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    Cand t;
-    t.v = __shfl_xor_sync(0xffffffffu, r.v, o);
-    t.i = __shfl_xor_sync(0xffffffffu, r.i, o);
-    r = cand_best(r, t);
-  }
-  return r;  // identical in every thread
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  return s;
 }
 
-// One CTA per row.  The row is read once into registers (TOPK_PER_THREAD values per thread); the BW
-// selection passes then work on registers plus one block reduction each.
-constexpr int TOPK_THREADS = 1024;
-constexpr int TOPK_PER_THREAD = 32;  // V <= 32768
+constexpr int SEL_THREADS = 1024;
+constexpr int SEL_MAX_BW = 128;
+constexpr int SEL_LIST_CAP = 1024;  // elements at or above the selection threshold
 
-__global__ void __launch_bounds__(TOPK_THREADS) row_topk_kernel(GemmOut proj, int V, int BW, float* __restrict__ lse,
-                                                                 float* __restrict__ val, int32_t* __restrict__ idx,
-                                                                 const int32_t* __restrict__ m_total) {
-  pdl_enter();
-  __shared__ Cand sh[32];
-  __shared__ float shf[32];
-  const int r = blockIdx.x;
-  const int m_tiles = gemm_m_tiles(proj, *m_total);
-  // element (k, e) of this thread is column 4 * (threadIdx.x + (k / 4) * TOPK_THREADS) + k % 4
-  float v[TOPK_PER_THREAD];
-  Cand c{-INFINITY, 0x7fffffff};
-#pragma unroll
-  for (int k4 = 0; k4 < TOPK_PER_THREAD / 4; ++k4) {
-    const int i = 4 * (threadIdx.x + k4 * TOPK_THREADS);
-    float4 q = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-    if (i < V) q = gemm_value4(proj, m_tiles, r, i);   // V is a multiple of 4
-    v[4 * k4] = q.x; v[4 * k4 + 1] = q.y; v[4 * k4 + 2] = q.z; v[4 * k4 + 3] = q.w;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) c = cand_best(c, Cand{v[4 * k4 + e], i < V ? i + e : 0x7fffffff});
-  }
-  const Cand top = block_best(c, sh);
-  float s = 0.f;
-#pragma unroll
-  for (int k = 0; k < TOPK_PER_THREAD; ++k) s += expf(v[k] - top.v);  // exp(-inf) = 0 for the padding
-  {
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    __syncthreads();
-    if (lane == 0) shf[w] = s;
-    __syncthreads();
-    s = lane < nw ? shf[lane] : 0.f;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-  }
-  if (threadIdx.x == 0) {
-    lse[r] = top.v + logf(s);
-    val[(size_t)r * BW] = top.v;
-    idx[(size_t)r * BW] = top.i;
-  }
-  Cand prev = top;
-  for (int p = 1; p < BW; ++p) {
-    Cand best{-INFINITY, 0x7fffffff};
-#pragma unroll
-    for (int k = 0; k < TOPK_PER_THREAD; ++k) {
-      const int i = 4 * (threadIdx.x + (k >> 2) * TOPK_THREADS) + (k & 3);
-      if (i < V && cand_before(prev.v, prev.i, v[k], i)) best = cand_best(best, Cand{v[k], i});
-    }
-    best = block_best(best, sh);
-    if (threadIdx.x == 0) {
-      val[(size_t)r * BW + p] = best.v;
-      idx[(size_t)r * BW + p] = best.i == 0x7fffffff ? 0 : best.i;
-    }
-    prev = best;
-  }
-}
-
-cudaError_t launch_row_topk(const GemmOut& proj, int V, int BW, float* lse, float* val, int32_t* idx, int rows,
-                            const int32_t* m_total, cudaStream_t st) {
-  if (V > TOPK_THREADS * TOPK_PER_THREAD) return cudaErrorInvalidValue;
-  launch_pdl(row_topk_kernel, rows, TOPK_THREADS, 0, st, proj, V, BW, lse, val, idx, m_total);
-  return cudaGetLastError();
-}
-
-// ---------------------------------------------------------------- cross-row merge + reorder + gather
-// call == 1: the single row's top-BW become the beams.  call >= 2: best BW of the BW*BW survivors.  Writes score_out[k], hist_out[k][0..call-1], and the next call's inputs
-// se_t[k] = [s_t of the parent (read from s_new_f with row stride ld_s; skipped for call 1, where every
-// beam keeps s_1) ; E[token_k]].  On the last call also the public outputs.
+// One CTA per drafter row r (a live beam, or the single row of call 1).
+//  1. the row's logits (projection output + partial slots) into registers, 32 per thread;
+//  2. log-sum-exp of the row; a threshold that at least BW values reach (the BW-th largest per-thread
+//     maximum, found with warp shuffles); the few values at or above it go to a shared list that warp 0
+//     ranks.  Each value is touched a constant number of times, whatever BW is;
+//  3. the last CTA of a sequence to finish (atomic counter, no waiting) prunes the BW x BW survivors
+//     score_r + logit - lse_r to the BW best in (score desc, flat index r*V + v asc) order, writes the
+//     new scores and histories, and gathers the next call's input rows [s_t of the parent ; E[token]].
 template <typename T>
-__global__ void __launch_bounds__(256) beam_merge_kernel(int call, const float* __restrict__ lse,
-                                                          const float* __restrict__ val, const int32_t* __restrict__ idx,
-                                                          const float* __restrict__ score_in, float* __restrict__ score_out,
-                                                          const int32_t* __restrict__ hist_in, int32_t* __restrict__ hist_out,
-                                                          const T* __restrict__ emb, const float* __restrict__ s_new_f,
-                                                          int ld_s, T* __restrict__ se_t, Dims dm,
-                                                          int32_t* __restrict__ beams_out, float* __restrict__ scores_out) {
+__global__ void __launch_bounds__(SEL_THREADS) draft_select_kernel(
+    GemmOut proj, int call, float* __restrict__ lse, float* __restrict__ val, int32_t* __restrict__ idx,
+    const float* __restrict__ score_in, float* __restrict__ score_out, const int32_t* __restrict__ hist_in,
+    int32_t* __restrict__ hist_out, const T* __restrict__ emb, const float* __restrict__ s_new_f, int ld_s,
+    T* __restrict__ se_t, Dims dm, int32_t* __restrict__ beams_out, float* __restrict__ scores_out,
+    int32_t* __restrict__ counters, const int32_t* __restrict__ m_total, unsigned long long* dbg) {
+  unsigned long long t_dbg[8];
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[0]));
   pdl_enter();
-  // grid = B * BW: every CTA of a sequence repeats the (tiny) selection over the BW*BW survivors and
-  // then writes the outputs of ONE new beam, so the reorder/gather work is spread over BW CTAs.
-  __shared__ Cand sh[32];
-  __shared__ int sel_parent[128], sel_tok[128];
-  __shared__ float sel_score[128];
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[1]));
+  extern __shared__ __align__(16) uint8_t sel_smem[];
+  Cand* wl = reinterpret_cast<Cand*>(sel_smem);            // [32 warps][BW] per-warp survivors; reused by the pruning
+  __shared__ float shf[32];
+  __shared__ Cand sh_top[SEL_MAX_BW];
+  __shared__ int sel_parent[SEL_MAX_BW], sel_tok[SEL_MAX_BW];
+  __shared__ float sel_score[SEL_MAX_BW];
+  __shared__ int s_last, s_count;
+  __shared__ float s_tau;
   const int BW = dm.BW, L = dm.L, V = dm.V;
-  const int b = blockIdx.x / BW, k = blockIdx.x - b * BW;
-  const int rows = call == 1 ? 1 : BW;
-  const int row0 = call == 1 ? b : b * BW;
-  const int n_cand = rows * BW;
-  Cand prev{INFINITY, -1};
-  for (int p = 0; p <= k; ++p) {  // beams are ranked: beam k needs the first k+1 picks only
-    Cand best{-INFINITY, 0x7fffffff};
-    for (int c = threadIdx.x; c < n_cand; c += blockDim.x) {
-      const int r = c / BW;
-      const size_t o = (size_t)(row0 + r) * BW + (c - r * BW);
-      const float base = call == 1 ? 0.f : score_in[row0 + r];
-      const float sc = base + (val[o] - lse[row0 + r]);
-      const int flat = r * V + idx[o];
-      if (cand_before(prev.v, prev.i, sc, flat)) best = cand_best(best, Cand{sc, flat});
+  const int r = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int m_tiles = gemm_m_tiles(proj, *m_total);
+  Cand* cl = wl + 32 * BW;   // [SEL_LIST_CAP] values at or above the threshold
+  // ---- 1. logits into shared memory (compact loops from here on: the kernel runs once per launch,
+  // so straight-line code would be bound by instruction fetch)
+  float* zrow = reinterpret_cast<float*>(cl + SEL_LIST_CAP);   // [V]
+  float tmax = -INFINITY;
+#pragma unroll 4
+  for (int i = 4 * threadIdx.x; i < V; i += 4 * SEL_THREADS) {
+    const float4 q = gemm_value4<2>(proj, m_tiles, r, i);   // V is a multiple of 4
+    *reinterpret_cast<float4*>(zrow + i) = q;
+    tmax = fmaxf(tmax, fmaxf(fmaxf(q.x, q.y), fmaxf(q.z, q.w)));
+  }
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[2]));
+  // ---- 2a. a threshold that at least BW elements reach: the BW-th largest of the 1024 per-thread maxima
+  // (per warp BW rounds over one value per lane, then warp 0 over the 32 x BW survivors)
+  {
+    Cand prev{INFINITY, -1};
+    for (int p = 0; p < BW; ++p) {
+      Cand best{-INFINITY, 0x7fffffff};
+      if (cand_before(prev.v, prev.i, tmax, lane)) best = Cand{tmax, lane};
+      best = warp_best(best);
+      if (lane == 0) wl[warp * BW + p] = best;   // index unused below
+      prev = best;
     }
-    best = block_best(best, sh);
-    if (threadIdx.x == 0) {
-      sel_parent[p] = best.i / V;
-      sel_tok[p] = best.i - (best.i / V) * V;
-      sel_score[p] = best.v;
+  }
+  // ---- 2b. log-sum-exp of the row
+  float wmax = tmax;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) wmax = fmaxf(wmax, __shfl_xor_sync(0xffffffffu, wmax, o));
+  __syncthreads();
+  if (lane == 0) shf[warp] = wmax;
+  if (threadIdx.x == 0) s_count = 0;
+  __syncthreads();
+  float rmax = shf[lane];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, o));
+  float s = 0.f;
+#pragma unroll 4
+  for (int i = 4 * threadIdx.x; i < V; i += 4 * SEL_THREADS) {
+    const float4 q = *reinterpret_cast<const float4*>(zrow + i);
+    s += __expf(q.x - rmax) + __expf(q.y - rmax) + __expf(q.z - rmax) + __expf(q.w - rmax);
+  }
+  s = block_reduce_sum(s, shf);   // also orders the wl writes before warp 0 reads them
+  const float row_lse = rmax + logf(s);
+  if (warp == 0) {
+    Cand pv{INFINITY, -1};
+    for (int p = 0; p < BW; ++p) {
+      Cand best{-INFINITY, 0x7fffffff};
+      for (int c = lane; c < 32 * BW; c += 32) {
+        const float x = wl[c].v;
+        if (cand_before(pv.v, pv.i, x, c)) best = cand_best(best, Cand{x, c});
+      }
+      best = warp_best(best);
+      pv = best;
     }
-    prev = best;
+    if (lane == 0) s_tau = pv.v;   // -inf when the row has fewer than BW values
   }
   __syncthreads();
-  const int orow = b * BW + k;
-  const int prow = b * BW + sel_parent[k];
-  const int tok = sel_tok[k];
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[3]));
+  // ---- 2c. every element that reaches the threshold goes to a short list; warp 0 ranks the list
+  const float tau = s_tau;
+#pragma unroll 4
+  for (int i = 4 * threadIdx.x; i < V; i += 4 * SEL_THREADS) {
+    const float4 q = *reinterpret_cast<const float4*>(zrow + i);
+    const float e[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (e[k] >= tau) {
+        const int slot = atomicAdd(&s_count, 1);
+        if (slot < SEL_LIST_CAP) cl[slot] = Cand{e[k], i + k};
+      }
+    }
+  }
+  __syncthreads();
+  const int n_list = s_count;
+  if (n_list <= SEL_LIST_CAP) {
+    if (warp == 0) {
+      Cand pv{INFINITY, -1};
+      for (int p = 0; p < BW; ++p) {
+        Cand best{-INFINITY, 0x7fffffff};
+        for (int c = lane; c < n_list; c += 32) {
+          const Cand x = cl[c];
+          if (cand_before(pv.v, pv.i, x.v, x.i)) best = cand_best(best, x);
+        }
+        best = warp_best(best);
+        if (lane == 0) {
+          val[(size_t)r * BW + p] = best.v;
+          idx[(size_t)r * BW + p] = best.i == 0x7fffffff ? 0 : best.i;
+        }
+        pv = best;
+      }
+    }
+  } else {
+    // more ties at the threshold than the list holds: rank by rounds over all values (slow, exact)
+    Cand prev{INFINITY, -1};
+    for (int p = 0; p < BW; ++p) {
+      Cand best{-INFINITY, 0x7fffffff};
+      for (int i = threadIdx.x; i < V; i += SEL_THREADS)
+        if (cand_before(prev.v, prev.i, zrow[i], i)) best = cand_best(best, Cand{zrow[i], i});
+      best = warp_best(best);
+      __syncthreads();
+      if (lane == 0) wl[warp] = best;
+      __syncthreads();
+      best = warp_best(wl[lane]);
+      if (threadIdx.x == 0) {
+        val[(size_t)r * BW + p] = best.v;
+        idx[(size_t)r * BW + p] = best.i == 0x7fffffff ? 0 : best.i;
+      }
+      prev = best;
+    }
+  }
+  if (threadIdx.x == 0) lse[r] = row_lse;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[4]));
+  // ---- 3. pruning by the sequence's last CTA
+  const int rows = call == 1 ? 1 : BW;
+  const int b = call == 1 ? r : r / BW;
+  const int row0 = call == 1 ? b : b * BW;
+  __threadfence();
+  __syncthreads();
   if (threadIdx.x == 0) {
-    score_out[orow] = sel_score[k];
+    const int old = atomicAdd(counters + b, 1);
+    s_last = (old == rows - 1) ? 1 : 0;
+    if (old == rows - 1) counters[b] = 0;
+  }
+  __syncthreads();
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[5]));
+  if (!s_last) return;
+  __threadfence();
+  const int n_cand = rows * BW;
+  // candidates into shared memory: score and flat index
+  for (int c = threadIdx.x; c < n_cand; c += blockDim.x) {
+    const int rr = c / BW;
+    const size_t o = (size_t)(row0 + rr) * BW + (c - rr * BW);
+    const float base = call == 1 ? 0.f : score_in[row0 + rr];
+    wl[c] = Cand{base + (__ldcg(val + o) - __ldcg(lse + row0 + rr)), rr * V + __ldcg(idx + o)};
+  }
+  __syncthreads();
+  if (warp == 0) {
+    Cand pv{INFINITY, -1};
+    for (int p = 0; p < BW; ++p) {
+      Cand best{-INFINITY, 0x7fffffff};
+      for (int c = lane; c < n_cand; c += 32) {
+        const Cand x = wl[c];
+        if (cand_before(pv.v, pv.i, x.v, x.i)) best = cand_best(best, x);
+      }
+      best = warp_best(best);
+      if (lane == 0) sh_top[p] = best;
+      pv = best;
+    }
+  }
+  __syncthreads();
+  for (int k = threadIdx.x; k < BW; k += blockDim.x) {
+    const Cand c = sh_top[k];
+    const int parent = c.i / V, tok = c.i - parent * V;
+    sel_parent[k] = parent; sel_tok[k] = tok; sel_score[k] = c.v;
+    const int orow = b * BW + k, prow = b * BW + parent;
+    score_out[orow] = c.v;
     for (int t = 0; t < call - 1; ++t) hist_out[(size_t)orow * L + t] = hist_in[(size_t)prow * L + t];
     hist_out[(size_t)orow * L + call - 1] = tok;
     if (call == L) {
       for (int t = 0; t < L - 1; ++t) beams_out[(size_t)orow * L + t] = hist_in[(size_t)prow * L + t];
       beams_out[(size_t)orow * L + L - 1] = tok;
-      if (scores_out) scores_out[orow] = sel_score[k];
+      if (scores_out) scores_out[orow] = c.v;
     }
   }
+  __syncthreads();
   if (call < L) {
-    // gathers with 128-bit accesses (rows are 16-byte aligned: d is a multiple of 8)
-    // next call's input row [s of the parent ; E[token]]
+    // next call's input rows [s of the parent ; E[token]], 128-bit accesses (d, d_rnn multiples of 8)
     constexpr int EV = 16 / sizeof(T);
-    T* se = se_t + (size_t)orow * (dm.dr + dm.d);
-    const uint4* e = reinterpret_cast<const uint4*>(emb + (size_t)tok * dm.d);
-    uint4* eo = reinterpret_cast<uint4*>(se + dm.dr);
-    for (int i = threadIdx.x; i < dm.d / EV; i += blockDim.x) eo[i] = e[i];
+    const int ev = dm.d / EV, sv = dm.dr / 4;
+    for (int item = threadIdx.x; item < BW * ev; item += blockDim.x) {
+      const int k = item / ev, i = item - k * ev;
+      const uint4* e = reinterpret_cast<const uint4*>(emb + (size_t)sel_tok[k] * dm.d);
+      reinterpret_cast<uint4*>(se_t + (size_t)(b * BW + k) * (dm.dr + dm.d) + dm.dr)[i] = e[i];
+    }
     if (call > 1) {
-      const float4* s = reinterpret_cast<const float4*>(s_new_f + (size_t)prow * ld_s);
-      T* so = se;
-      for (int i = threadIdx.x; i < dm.dr / 4; i += blockDim.x) {
-        const float4 v = s[i];
-        so[4 * i] = from_f<T>(v.x); so[4 * i + 1] = from_f<T>(v.y); so[4 * i + 2] = from_f<T>(v.z); so[4 * i + 3] = from_f<T>(v.w);
+      for (int item = threadIdx.x; item < BW * sv; item += blockDim.x) {
+        const int k = item / sv, i = item - k * sv;
+        const float4 q = reinterpret_cast<const float4*>(s_new_f + (size_t)(b * BW + sel_parent[k]) * ld_s)[i];
+        T* so = se_t + (size_t)(b * BW + k) * (dm.dr + dm.d) + 4 * i;
+        so[0] = from_f<T>(q.x); so[1] = from_f<T>(q.y); so[2] = from_f<T>(q.z); so[3] = from_f<T>(q.w);
       }
     }
   }
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[6]));
+  if (dbg && threadIdx.x == 0) {
+    for (int i = 0; i < 7; ++i) dbg[i] = t_dbg[i];
+  }
 }
 
-cudaError_t launch_beam_merge(int dtype, int call, const float* lse, const float* val, const int32_t* idx,
-                              const float* score_in, float* score_out, const int32_t* hist_in, int32_t* hist_out,
-                              const void* emb, const float* s_new_f, int ld_s, void* se_t, const Dims& dm, int B,
-                              int32_t* beams_out, float* scores_out, cudaStream_t st) {
-  RD_DISPATCH(dtype, launch_pdl(beam_merge_kernel<T>, B * dm.BW, 256, 0, st, call, lse, val, idx, score_in, score_out, hist_in, hist_out,
-                                                           (const T*)emb, s_new_f, ld_s, (T*)se_t, dm,
-                                                           beams_out, scores_out));
+// rows = B (call 1) or B * BW.  counters: [B] zero between launches.
+cudaError_t launch_draft_select(int dtype, const GemmOut& proj, int call, float* lse, float* val, int32_t* idx,
+                                const float* score_in, float* score_out, const int32_t* hist_in, int32_t* hist_out,
+                                const void* emb, const float* s_new_f, int ld_s, void* se_t, const Dims& dm, int B,
+                                int32_t* beams_out, float* scores_out, int32_t* counters, const int32_t* m_total,
+                                unsigned long long* dbg, cudaStream_t st) {
+  if (dm.BW > SEL_MAX_BW) return cudaErrorInvalidValue;
+  const int rows = call == 1 ? B : B * dm.BW;
+  const size_t select = ((size_t)32 * dm.BW + SEL_LIST_CAP) * sizeof(Cand) + (size_t)dm.V * sizeof(float);
+  const size_t prune = (size_t)dm.BW * dm.BW * sizeof(Cand);
+  const size_t smem = select > prune ? select : prune;
+  if (smem > 200 * 1024) return cudaErrorInvalidValue;   // vocabulary too large for the shared-memory row
+  static bool attr_set[2] = {false, false};
+  if (!attr_set[dtype == RD_DTYPE_FP32 ? 0 : 1]) {
+    cudaError_t e = dtype == RD_DTYPE_FP32
+                        ? cudaFuncSetAttribute(draft_select_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)
+                        : cudaFuncSetAttribute(draft_select_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_set[dtype == RD_DTYPE_FP32 ? 0 : 1] = true;
+  }
+  RD_DISPATCH(dtype, launch_pdl(draft_select_kernel<T>, rows, SEL_THREADS, smem, st, proj, call, lse, val, idx, score_in,
+                                score_out, hist_in, hist_out, (const T*)emb, s_new_f, ld_s, (T*)se_t, dm, beams_out,
+                                scores_out, counters, m_total, dbg));
   return cudaGetLastError();
 }
 

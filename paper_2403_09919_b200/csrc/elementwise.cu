@@ -54,10 +54,9 @@ cudaError_t launch_embed(int dtype, const void* emb, const int32_t* tok, float* 
 // ---------------------------------------------------------------- RMSNorm
 // y = x / sqrt(mean(x^2) + eps) * gain, one block per row.  The row is read once with 128-bit loads
 // and kept in registers between the reduction and the scaling (d <= 8192).
-constexpr int NORM_THREADS = 1024;
-constexpr int NORM_MAXV = 2;
+constexpr int NORM_THREADS = 512;
 
-template <typename T>
+template <typename T, int NORM_MAXV>
 __global__ void __launch_bounds__(NORM_THREADS) rmsnorm_kernel(float* __restrict__ x, GemmOut proj, const T* __restrict__ gain,
                                                                 T* __restrict__ out_t, float* __restrict__ out_f, int d,
                                                                 float eps, const int32_t* __restrict__ m_total) {
@@ -71,14 +70,23 @@ __global__ void __launch_bounds__(NORM_THREADS) rmsnorm_kernel(float* __restrict
   const bool add = proj.raw != nullptr;   // x += the projection that ends the previous block (O or down)
   const int m_tiles = add ? gemm_m_tiles(proj, M) : 1;
   float4 v[NORM_MAXV];
+  GemmPending4<6> pend[NORM_MAXV];
   float ss = 0.f;
+  // every load first (residual row, projection output, partial slots), then the arithmetic
 #pragma unroll
   for (int k = 0; k < NORM_MAXV; ++k) {
     const int i = threadIdx.x + k * NORM_THREADS;
     if (i < nvec) {
       v[k] = xr[i];
+      if (add) pend[k] = gemm_issue4<6>(proj, m_tiles, m, 4 * i);
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < NORM_MAXV; ++k) {
+    const int i = threadIdx.x + k * NORM_THREADS;
+    if (i < nvec) {
       if (add) {
-        const float4 q = gemm_value4(proj, m_tiles, m, 4 * i);
+        const float4 q = gemm_finish4(proj, m_tiles, pend[k]);
         v[k].x += q.x; v[k].y += q.y; v[k].z += q.z; v[k].w += q.w;
         xr[i] = v[k];
       }
@@ -104,10 +112,14 @@ __global__ void __launch_bounds__(NORM_THREADS) rmsnorm_kernel(float* __restrict
 // x: residual stream (updated in place when proj != nullptr: x += proj).
 cudaError_t launch_rmsnorm(int dtype, float* x, const GemmOut* proj, const void* gain, void* out_t, float* out_f32, int d,
                            float eps, const int32_t* m_total, int m_max, cudaStream_t st) {
-  if (d > 4 * NORM_THREADS * NORM_MAXV || (d & 3)) return cudaErrorInvalidValue;
+  if (d > 4 * NORM_THREADS * 4 || (d & 3)) return cudaErrorInvalidValue;
   GemmOut g{};
   if (proj) g = *proj;
-  RD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T>, m_max, NORM_THREADS, 0, st, x, g, (const T*)gain, (T*)out_t, out_f32, d, eps, m_total));
+  if (d <= 4 * NORM_THREADS * 2) {
+    RD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 2>, m_max, NORM_THREADS, 0, st, x, g, (const T*)gain, (T*)out_t, out_f32, d, eps, m_total));
+  } else {
+    RD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 4>, m_max, NORM_THREADS, 0, st, x, g, (const T*)gain, (T*)out_t, out_f32, d, eps, m_total));
+  }
   return cudaGetLastError();
 }
 
@@ -158,9 +170,12 @@ __global__ void rope_kv_kernel(float* __restrict__ qkv, GemmOut proj, T* __restr
     const float2 cs = table[(size_t)m * half + i];
     const float c = cs.x, s = cs.y;
     const int o = h * hd + i;
-    const float q1 = gemm_value(proj, m_tiles, m, o), q2 = gemm_value(proj, m_tiles, m, o + half);
-    const float k1 = gemm_value(proj, m_tiles, m, d + o), k2 = gemm_value(proj, m_tiles, m, d + o + half);
-    const float v1 = gemm_value(proj, m_tiles, m, 2 * d + o), v2 = gemm_value(proj, m_tiles, m, 2 * d + o + half);
+    const auto pq1 = gemm_issue<4>(proj, m_tiles, m, o), pq2 = gemm_issue<4>(proj, m_tiles, m, o + half);
+    const auto pk1 = gemm_issue<4>(proj, m_tiles, m, d + o), pk2 = gemm_issue<4>(proj, m_tiles, m, d + o + half);
+    const auto pv1 = gemm_issue<4>(proj, m_tiles, m, 2 * d + o), pv2 = gemm_issue<4>(proj, m_tiles, m, 2 * d + o + half);
+    const float q1 = gemm_finish(proj, m_tiles, pq1), q2 = gemm_finish(proj, m_tiles, pq2);
+    const float k1 = gemm_finish(proj, m_tiles, pk1), k2 = gemm_finish(proj, m_tiles, pk2);
+    const float v1 = gemm_finish(proj, m_tiles, pv1), v2 = gemm_finish(proj, m_tiles, pv2);
     row[o] = q1 * c - q2 * s;            // the attention kernel reads the rotated Q from here
     row[o + half] = q2 * c + q1 * s;
     if (slot_ok) {
@@ -191,7 +206,8 @@ __global__ void swiglu_kernel(GemmOut proj, T* __restrict__ out, int F, const in
   const int f = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (f >= F) return;
   const int m_tiles = gemm_m_tiles(proj, M);
-  const float4 g = gemm_value4(proj, m_tiles, m, f), u = gemm_value4(proj, m_tiles, m, F + f);
+  const auto pg = gemm_issue4<4>(proj, m_tiles, m, f), pu = gemm_issue4<4>(proj, m_tiles, m, F + f);
+  const float4 g = gemm_finish4(proj, m_tiles, pg), u = gemm_finish4(proj, m_tiles, pu);
   T* o = out + (size_t)m * F + f;
   o[0] = from_f<T>(silu_f(g.x) * u.x); o[1] = from_f<T>(silu_f(g.y) * u.y);
   o[2] = from_f<T>(silu_f(g.z) * u.z); o[3] = from_f<T>(silu_f(g.w) * u.w);

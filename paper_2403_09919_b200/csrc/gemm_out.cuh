@@ -68,48 +68,85 @@ __device__ __forceinline__ bool gemm_has_work(const GemmOut& g, int m_tiles, int
 
 constexpr int GEMM_FOLD_UNROLL = 8;  // slots loaded together (a tile rarely has more contributors)
 
-// The complete value of output element (m, n): all slot loads are issued together, the sum is taken
-// in CTA order.
-__device__ __forceinline__ float gemm_value(const GemmOut& g, int m_tiles, int m, int n) {
-  float v = g.raw[(size_t)m * g.ld + n];
-  if (g.partial == nullptr) return v;
-  const GemmFold f = gemm_fold(g, m_tiles, m, n);
+// Two-phase read of a projection value: gemm_issue starts every load (output element and up to U
+// partial slots) without consuming any of them, gemm_finish sums them in CTA order.  A kernel that
+// needs several values issues all of them first, so the loads overlap instead of forming a chain
+// of L2 round trips.  Tiles with more than U extra contributors take a (rare) loop in gemm_finish.
+template <int U>
+struct GemmPending {
+  float raw;
+  float q[U];
+  GemmFold f;
+};
+template <int U>
+struct GemmPending4 {
+  float4 raw;
+  float4 q[U];
+  GemmFold f;
+};
+
+template <int U>
+__device__ __forceinline__ GemmPending<U> gemm_issue(const GemmOut& g, int m_tiles, int m, int n) {
+  GemmPending<U> p;
+  p.raw = g.raw[(size_t)m * g.ld + n];
+  p.f.c_next = 1; p.f.c_last = 0; p.f.off = 0;
+  if (g.partial != nullptr) p.f = gemm_fold(g, m_tiles, m, n);
   const size_t slot = (size_t)g.mt * 128;
-  float q[GEMM_FOLD_UNROLL];
 #pragma unroll
-  for (int j = 0; j < GEMM_FOLD_UNROLL; ++j) {
-    const int c = f.c_next + j;
-    q[j] = (c <= f.c_last && gemm_has_work(g, m_tiles, c)) ? __ldcg(g.partial + (size_t)c * slot + f.off) : 0.f;
+  for (int j = 0; j < U; ++j) {
+    const int c = p.f.c_next + j;
+    p.q[j] = (c <= p.f.c_last && gemm_has_work(g, m_tiles, c)) ? __ldcg(g.partial + (size_t)c * slot + p.f.off) : 0.f;
   }
+  return p;
+}
+template <int U>
+__device__ __forceinline__ float gemm_finish(const GemmOut& g, int m_tiles, const GemmPending<U>& p) {
+  float v = p.raw;
 #pragma unroll
-  for (int j = 0; j < GEMM_FOLD_UNROLL; ++j) v += q[j];
-  for (int c = f.c_next + GEMM_FOLD_UNROLL; c <= f.c_last; ++c)
-    if (gemm_has_work(g, m_tiles, c)) v += __ldcg(g.partial + (size_t)c * slot + f.off);
+  for (int j = 0; j < U; ++j) v += p.q[j];
+  const size_t slot = (size_t)g.mt * 128;
+  for (int c = p.f.c_next + U; c <= p.f.c_last; ++c)
+    if (gemm_has_work(g, m_tiles, c)) v += __ldcg(g.partial + (size_t)c * slot + p.f.off);
   return v;
 }
-
 // Four consecutive columns n .. n+3 (n a multiple of 4: they share a tile and the slots' alignment).
-__device__ __forceinline__ float4 gemm_value4(const GemmOut& g, int m_tiles, int m, int n) {
-  float4 v = *reinterpret_cast<const float4*>(g.raw + (size_t)m * g.ld + n);
-  if (g.partial == nullptr) return v;
-  const GemmFold f = gemm_fold(g, m_tiles, m, n);
+template <int U>
+__device__ __forceinline__ GemmPending4<U> gemm_issue4(const GemmOut& g, int m_tiles, int m, int n) {
+  GemmPending4<U> p;
+  p.raw = *reinterpret_cast<const float4*>(g.raw + (size_t)m * g.ld + n);
+  p.f.c_next = 1; p.f.c_last = 0; p.f.off = 0;
+  if (g.partial != nullptr) p.f = gemm_fold(g, m_tiles, m, n);
   const size_t slot = (size_t)g.mt * 128;
-  float4 q[GEMM_FOLD_UNROLL];
 #pragma unroll
-  for (int j = 0; j < GEMM_FOLD_UNROLL; ++j) {
-    const int c = f.c_next + j;
-    q[j] = (c <= f.c_last && gemm_has_work(g, m_tiles, c))
-               ? __ldcg(reinterpret_cast<const float4*>(g.partial + (size_t)c * slot + f.off))
-               : make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int j = 0; j < U; ++j) {
+    const int c = p.f.c_next + j;
+    p.q[j] = (c <= p.f.c_last && gemm_has_work(g, m_tiles, c))
+                 ? __ldcg(reinterpret_cast<const float4*>(g.partial + (size_t)c * slot + p.f.off))
+                 : make_float4(0.f, 0.f, 0.f, 0.f);
   }
+  return p;
+}
+template <int U>
+__device__ __forceinline__ float4 gemm_finish4(const GemmOut& g, int m_tiles, const GemmPending4<U>& p) {
+  float4 v = p.raw;
 #pragma unroll
-  for (int j = 0; j < GEMM_FOLD_UNROLL; ++j) { v.x += q[j].x; v.y += q[j].y; v.z += q[j].z; v.w += q[j].w; }
-  for (int c = f.c_next + GEMM_FOLD_UNROLL; c <= f.c_last; ++c) {
+  for (int j = 0; j < U; ++j) { v.x += p.q[j].x; v.y += p.q[j].y; v.z += p.q[j].z; v.w += p.q[j].w; }
+  const size_t slot = (size_t)g.mt * 128;
+  for (int c = p.f.c_next + U; c <= p.f.c_last; ++c) {
     if (!gemm_has_work(g, m_tiles, c)) continue;
-    const float4 t = __ldcg(reinterpret_cast<const float4*>(g.partial + (size_t)c * slot + f.off));
+    const float4 t = __ldcg(reinterpret_cast<const float4*>(g.partial + (size_t)c * slot + p.f.off));
     v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
   }
   return v;
+}
+
+// One-shot forms.
+__device__ __forceinline__ float gemm_value(const GemmOut& g, int m_tiles, int m, int n) {
+  return gemm_finish(g, m_tiles, gemm_issue<GEMM_FOLD_UNROLL>(g, m_tiles, m, n));
+}
+template <int U = GEMM_FOLD_UNROLL>
+__device__ __forceinline__ float4 gemm_value4(const GemmOut& g, int m_tiles, int m, int n) {
+  return gemm_finish4(g, m_tiles, gemm_issue4<U>(g, m_tiles, m, n));
 }
 
 }  // namespace rd
