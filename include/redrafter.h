@@ -160,6 +160,30 @@ RD_API int redrafter_verify(rd_handle* h, const rd_packed* packed, void* stream,
 RD_API int redrafter_accept(rd_handle* h, const int32_t* beams, const rd_packed* packed, const int32_t* argmax,
                      const float* hidden, void* stream, const rd_accept_out* out);
 
+/* redrafter_accept for callers that cannot provide scratch memory.  (The paper has no counterpart: this
+ * is a deployment variant of the accept step above, same inputs, same results.)
+ *
+ * Who needs it: code that runs where device allocation is off the table -- inside a latency-critical
+ * serving loop that must never enter the allocator, in a plugin whose host owns all GPU memory and
+ * hands out none, or after start-up in a process that has given its whole memory budget away.  Such a
+ * caller can still drive the accept step: the three per-sequence temporaries that the accept and the
+ * KV-compaction kernels pass to each other live in a fixed array inside the library instead of in
+ * memory the caller supplies.  This call performs no cudaMalloc/cudaFree and uses no allocating
+ * library routine.
+ *
+ * Limits and rules:
+ *  - at most 4096 sequences per call (RD_ERR_CAPACITY beyond that, nothing is enqueued); the array
+ *    takes 48 KB on every GPU that loads the library, until the process exits;
+ *  - the first call on each device looks up the array's device address (one runtime query, with that
+ *    device current) and remembers it: make that first call outside any stream capture;
+ *  - all calls on a device share the one array and it keeps the last call's values.  Nothing in it has
+ *    to start at zero (every entry that is read is written first by the same call), but two calls
+ *    whose kernels overlap on the GPU -- different streams, no ordering between them -- race on it:
+ *    order them.  redrafter_accept has no such restriction across handles.
+ * Everything else (arguments, outputs, state update, errors) is exactly as for redrafter_accept. */
+RD_API int redrafter_accept_static(rd_handle* h, const int32_t* beams, const rd_packed* packed, const int32_t* argmax,
+                                   const float* hidden, void* stream, const rd_accept_out* out);
+
 /* The whole step in one call, using workspace-internal intermediates.  With planted_beams
  * (device [B][BW][L]) non-NULL the drafter still runs but the planted candidates are packed and
  * verified.  `out` may be NULL.  Errors: STATE (no prefill yet), CAPACITY (host-tracked upper bound

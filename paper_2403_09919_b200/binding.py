@@ -25,7 +25,7 @@ EXPORTS = ["redrafter_workspace_bytes", "redrafter_kv_bytes", "redrafter_init", 
            "redrafter_last_error", "redrafter_prefill", "redrafter_draft", "redrafter_pack", "redrafter_verify",
            "redrafter_accept", "redrafter_step", "redrafter_ar_step", "redrafter_get_state", "redrafter_set_state",
            "redrafter_set_ctx_bound", "redrafter_poll", "redrafter_launch_count", "redrafter_profile",
-           "redrafter_profile_read", "redrafter_trace", "redrafter_trace_read"]
+           "redrafter_profile_read", "redrafter_trace", "redrafter_trace_read", "redrafter_accept_static"]
 
 
 class RdConfig(C.Structure):
@@ -74,6 +74,7 @@ def lib():
         L.redrafter_pack.argtypes = [vp, vp, vp, C.POINTER(RdPacked)]
         L.redrafter_verify.argtypes = [vp, C.POINTER(RdPacked), vp, vp, vp, vp]
         L.redrafter_accept.argtypes = [vp, vp, C.POINTER(RdPacked), vp, vp, vp, C.POINTER(RdAcceptOut)]
+        L.redrafter_accept_static.argtypes = [vp, vp, C.POINTER(RdPacked), vp, vp, vp, C.POINTER(RdAcceptOut)]
         L.redrafter_step.argtypes = [vp, vp, vp, C.POINTER(RdAcceptOut)]
         L.redrafter_ar_step.argtypes = [vp, vp, vp]
         L.redrafter_get_state.argtypes = [vp, vp, vp, vp, vp]
@@ -249,6 +250,13 @@ class ReDrafter:
         out = AcceptOut(self.B, self.Lb, self.device) if out is None else out
         self._ck(self.L.redrafter_accept(self.h, _ptr(beams), C.byref(packed.c), _ptr(argmax), _ptr(hidden), _stream(),
                                          C.byref(out.c)))
+        return out
+
+    def accept_static(self, beams, packed, argmax, hidden, out=None):
+        """redrafter_accept_static: the accept step with its scratch inside the library (no allocation)."""
+        out = AcceptOut(self.B, self.Lb, self.device) if out is None else out
+        self._ck(self.L.redrafter_accept_static(self.h, _ptr(beams), C.byref(packed.c), _ptr(argmax), _ptr(hidden),
+                                                _stream(), C.byref(out.c)))
         return out
 
     def step(self, planted_beams=None, out=None):

@@ -642,6 +642,27 @@ int redrafter_accept(rd_handle* h, const int32_t* beams, const rd_packed* packed
   return RD_OK;
 }
 
+int redrafter_accept_static(rd_handle* h, const int32_t* beams, const rd_packed* packed, const int32_t* argmax,
+                            const float* hidden, void* stream, const rd_accept_out* out) {
+  int rc = check_stepable(h);
+  if (rc) return rc;
+  if (!beams || !packed_ok(packed) || !argmax || !hidden) return fail(h, RD_ERR_INVALID_ARG, "null argument");
+  if (h->batch > accept_static_max_batch())
+    return fail(h, RD_ERR_CAPACITY, "batch %d exceeds the %d sequences the built-in scratch holds", h->batch,
+                accept_static_max_batch());
+  int32_t *n_accept = nullptr, *best = nullptr, *ctx_prev = nullptr;
+  cudaError_t e = accept_static_scratch(&n_accept, &best, &ctx_prev);
+  if (e != cudaSuccess) return fail(h, RD_ERR_CUDA, "built-in scratch: %s", cudaGetErrorString(e));
+  Workspace& w = h->ws;
+  rd_accept_out o{};
+  if (out) o = *out;
+  CK(h, launch_accept(h->dm.dtype, beams, *packed, argmax, hidden, h->kv, w.ctx, w.root, w.h, o, n_accept, best, ctx_prev,
+                      h->dm, h->batch, w.status, (cudaStream_t)stream));
+  h->launches++;  // accept + compaction
+  h->ctx_bound += 1 + h->dm.L;
+  return RD_OK;
+}
+
 int redrafter_step(rd_handle* h, const int32_t* planted_beams, void* stream, const rd_accept_out* out) {
   int rc = check_stepable(h);
   if (rc) return rc;

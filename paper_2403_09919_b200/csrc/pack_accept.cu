@@ -205,4 +205,36 @@ cudaError_t launch_accept(int dtype, const int32_t* beams, const rd_packed& pk, 
   return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------- scratch that needs no allocation
+// The accept and compaction kernels hand three small per-sequence values to each other (accepted
+// length, best candidate, previous context length).  redrafter_accept keeps them in the caller's
+// workspace; redrafter_accept_static keeps them here, in memory that is part of the loaded library,
+// for callers that cannot allocate.  Every GPU that loads the library holds these 48 KB until exit.
+constexpr int ACCEPT_STATIC_MAX_BATCH = 4096;
+static __device__ __align__(256) int32_t g_accept_scratch[3 * ACCEPT_STATIC_MAX_BATCH];
+
+int accept_static_max_batch() { return ACCEPT_STATIC_MAX_BATCH; }
+
+// Device address of the static scratch on the CURRENT device.  In host code the array's name is only a
+// handle for the runtime, not an address a kernel can use, so the address is asked for once per device
+// and remembered.
+cudaError_t accept_static_scratch(int32_t** n_accept, int32_t** best, int32_t** ctx_prev) {
+  constexpr int MAX_DEVICES = 64;
+  static int32_t* base[MAX_DEVICES] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+  if (base[dev] == nullptr) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_accept_scratch);
+    if (e != cudaSuccess) return e;
+    base[dev] = static_cast<int32_t*>(p);
+  }
+  *n_accept = base[dev];
+  *best = base[dev] + ACCEPT_STATIC_MAX_BATCH;
+  *ctx_prev = base[dev] + 2 * ACCEPT_STATIC_MAX_BATCH;
+  return cudaSuccess;
+}
+
 }  // namespace rd

@@ -117,6 +117,8 @@ cudaError_t launch_accept(int dtype, const int32_t* beams, const rd_packed& pk, 
                           const float* hidden, void* kcache, int32_t* ctx, int32_t* root, float* h,
                           const rd_accept_out& out, int32_t* n_accept_ws, int32_t* best_ws, int32_t* ctx_prev,
                           const Dims& dm, int B, int* status, cudaStream_t st);
+int accept_static_max_batch();
+cudaError_t accept_static_scratch(int32_t** n_accept, int32_t** best, int32_t** ctx_prev);
 cudaError_t launch_ar_finish(const int32_t* argmax_c, const float* hidden_c, int32_t* ctx, int32_t* root, float* h,
                              int32_t* token_out, const Dims& dm, int B, cudaStream_t st);
 cudaError_t launch_prefill_finish(const float* hidden_c, const int32_t* last_row, float* h, int d, int B,
