@@ -220,10 +220,15 @@ RD_API int redrafter_poll(rd_handle* h, void* stream);
 RD_API int redrafter_profile(rd_handle* h, int enable);
 RD_API int redrafter_profile_read(rd_handle* h, int32_t cls, double* ms, double* bytes, int64_t* launches);
 
-/* In-kernel timeline of the tensor-core projection launches, for measurement only.  After
- * redrafter_trace(h, 1, stream) the next launches (up to 512) each record eight %globaltimer
- * values in ns: [0] first CTA entered, [1]/[2] first/last producer past its dependency wait,
- * [3]/[4] first/last MMA issuer done, [5]/[6] first/last CTA done, [7] unused.
+/* In-kernel timeline, for measurement only.  After redrafter_trace(h, 1, stream) the next launches of
+ * the traced kernels (up to 512, in launch order) each record eight %globaltimer values in ns:
+ *   tensor-core projection: [0] first CTA entered, [1]/[2] first/last producer past its dependency wait,
+ *                           [3]/[4] first/last MMA issuer done, [5]/[6] first/last CTA done;
+ *   tensor-core attention (CTA of head 0, sequence 0, split 0): [0] entered, [1] past its dependency
+ *                           wait, [2] Q and masks loaded, [3] key chunks done, [4] partial published,
+ *                           [6] merge by the last split done;
+ *   drafter selection (last CTA): [0] entered, [1] past the wait, [2] logits in shared memory,
+ *                           [3] threshold found, [4] row ranked, [5] arrival counted, [6] pruning done.
  * redrafter_trace_read synchronises the stream, copies the records of the launches traced so far to
  * the HOST buffer out[max_launches][8] and returns their number (or a negative rd_status). */
 RD_API int redrafter_trace(rd_handle* h, int enable, void* stream);

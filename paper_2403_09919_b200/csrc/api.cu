@@ -297,7 +297,7 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
     const int rpb = attn_tc_rows_per_block();
     row_blocks = (rows_per_seq_max + rpb - 1) / rpb;
     const int blocks = dm.H * n_seq * row_blocks;
-    n_splits = (h->tc_grid + blocks - 1) / blocks;  // about one CTA per SM
+    n_splits = h->tc_grid / blocks;  // at most one CTA per SM: a second wave would double the time
     const int max_chunks = (h->ctx_bound + rows_per_seq_max + 63) / 64;
     if (n_splits > max_chunks) n_splits = max_chunks;
     if (n_splits > 16) n_splits = 16;
@@ -317,7 +317,8 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
       ProfScope ps(h, 1, 0.0, st);
       if (h->use_tc)
         CK(h, launch_attention_tc(w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.attn_t, rt, w.seq_off, dm, n_seq,
-                                  row_blocks, n_splits, w.att_scratch, w.att_counters, st));
+                                  row_blocks, n_splits, w.att_scratch, w.att_counters,
+                                  (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) ? w.trace + (size_t)8 * h->trace_next++ : nullptr, st));
       else
         CK(h, launch_attention(dm.dtype, w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.attn_t, rt, dm, m_max, st));
     }

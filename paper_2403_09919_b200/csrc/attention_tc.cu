@@ -46,16 +46,21 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
                                                            __nv_bfloat16* __restrict__ out, RowTables rt,
                                                            const int32_t* __restrict__ seq_off, Dims dm, int row_blocks,
                                                            int n_splits, float* __restrict__ scratch,
-                                                           int32_t* __restrict__ counters) {
+                                                           int32_t* __restrict__ counters, unsigned long long* dbg) {
+  unsigned long long t_dbg[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#define RD_STAMP(i) asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[i]))
+#define RD_DUMP() do { if (dbg && threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0) { \
+    if (blockIdx.z == 0) { for (int i_ = 0; i_ < 5; ++i_) dbg[i_] = t_dbg[i_]; } \
+    if (t_dbg[5]) atomicMax(dbg + 6, t_dbg[5]); } } while (0)
+  RD_STAMP(0);
   pdl_enter();
+  RD_STAMP(1);
   constexpr int LD = HD + PAD;           // shared row stride in bf16
   constexpr int NT = HD / 8;             // output n-tiles per warp
   constexpr int KS = HD / 16;            // k-steps of Q K^T
   extern __shared__ __align__(16) uint8_t smem[];
-  __nv_bfloat16* sQ = reinterpret_cast<__nv_bfloat16*>(smem);      // [ROWS][LD]
-  __nv_bfloat16* sK = sQ + ROWS * LD;                               // [KEYS][LD]
-  __nv_bfloat16* sV = sK + KEYS * LD;                               // [KEYS][LD]
-  int32_t* s_ncache = reinterpret_cast<int32_t*>(sV + KEYS * LD);  // [ROWS]
+  __nv_bfloat16* sKV = reinterpret_cast<__nv_bfloat16*>(smem);          // [2 buffers][K | V][KEYS][LD]
+  int32_t* s_ncache = reinterpret_cast<int32_t*>(sKV + 4 * KEYS * LD);  // [ROWS]
   uint32_t* s_mask = reinterpret_cast<uint32_t*>(s_ncache + ROWS);  // [ROWS][MW]
   __shared__ int s_last;
 
@@ -70,12 +75,56 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
   const int MW = dm.MW;
   const bool tree = rt.mask != nullptr;
 
-  // ---- Q (bf16) and per-row metadata to shared memory
-  for (int idx = tid; idx < ROWS * (HD / 2); idx += 128) {
-    const int r = idx / (HD / 2), c = (idx - r * (HD / 2)) * 2;
-    float2 q = make_float2(0.f, 0.f);
-    if (r < nrows) q = *reinterpret_cast<const float2*>(qkv + (size_t)(row0 + r) * 3 * dm.d + h * HD + c);
-    *reinterpret_cast<uint32_t*>(sQ + r * LD + c) = pack_bf16(q.x, q.y);
+  // ---- key extent of the block (the largest key index any of its rows may attend, plus one) and this
+  // split's chunk range.  Tree mode: every row of the sequence has the same n_cache and the tree rows
+  // follow it.  Causal mode: rows are in position order, the last one reaches furthest.
+  const int tree_base = rt.n_cache[row0];
+  int kext = tree ? tree_base + seq_rows : rt.n_cache[row0 + nrows - 1];
+  kext = min(kext, dm.max_ctx);
+  const int n_chunks = (kext + KEYS - 1) / KEYS;
+  const int c_begin = (int)((long long)z * n_chunks / n_splits), c_end = (int)((long long)(z + 1) * n_chunks / n_splits);
+
+  const size_t head_base = ((size_t)b * dm.H + h) * (size_t)dm.max_ctx * HD;
+  const uint32_t sKV_u = (uint32_t)__cvta_generic_to_shared(sKV);
+  constexpr uint32_t TILE_BYTES = KEYS * LD * 2;
+  // asynchronous copy of one chunk's K and V tiles into buffer `buf` (keys past the extent are zero-filled)
+  auto load_chunk = [&](int ch, int buf) {
+    const int k0 = ch * KEYS;
+    for (int idx = tid; idx < KEYS * (HD / 8); idx += 128) {
+      const int kr = idx / (HD / 8), c8 = (idx - kr * (HD / 8)) * 8;
+      const int key = k0 + kr;
+      const bool valid = key < kext;
+      const size_t off = head_base + (size_t)(valid ? key : 0) * HD + c8;
+      cp_async16(sKV_u + (2 * buf) * TILE_BYTES + (kr * LD + c8) * 2, kc + off, valid);
+      cp_async16(sKV_u + (2 * buf + 1) * TILE_BYTES + (kr * LD + c8) * 2, vc + off, valid);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  if (c_begin < c_end) load_chunk(c_begin, 0);   // in flight while Q and the masks are fetched
+
+  // ---- this warp's Q fragments (rows warp*16 + g, +8) straight from global memory into registers: 32
+  // independent 8-byte loads per thread, one round trip
+  const int r_lo = warp * 16 + g, r_hi = r_lo + 8;
+  uint32_t qf[KS][4];
+  {
+    const float* q_lo = qkv + (size_t)(row0 + (r_lo < nrows ? r_lo : 0)) * 3 * dm.d + h * HD + t4 * 2;
+    const float* q_hi = qkv + (size_t)(row0 + (r_hi < nrows ? r_hi : 0)) * 3 * dm.d + h * HD + t4 * 2;
+    float2 a[KS][4];
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      a[ks][0] = *reinterpret_cast<const float2*>(q_lo + ks * 16);
+      a[ks][1] = *reinterpret_cast<const float2*>(q_hi + ks * 16);
+      a[ks][2] = *reinterpret_cast<const float2*>(q_lo + ks * 16 + 8);
+      a[ks][3] = *reinterpret_cast<const float2*>(q_hi + ks * 16 + 8);
+    }
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const bool ok = ((e & 1) ? r_hi : r_lo) < nrows;
+        qf[ks][e] = ok ? pack_bf16(a[ks][e].x, a[ks][e].y) : 0u;
+      }
+    }
   }
   for (int r = tid; r < ROWS; r += 128) s_ncache[r] = r < nrows ? rt.n_cache[row0 + r] : 0;
   if (tree) {
@@ -85,28 +134,7 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
     }
   }
   __syncthreads();
-  // key extent of the block: the largest key index any of its rows may attend, plus one
-  int kext = 0;
-  for (int r = 0; r < nrows; ++r) kext = max(kext, s_ncache[r]);   // small loop, identical in every thread
-  const int tree_base = s_ncache[0];                                // tree mode: every row of a sequence has the same n_cache
-  if (tree) kext = tree_base + seq_rows;
-  kext = min(kext, dm.max_ctx);
-  const int n_chunks = (kext + KEYS - 1) / KEYS;
-  const int c_begin = (int)((long long)z * n_chunks / n_splits), c_end = (int)((long long)(z + 1) * n_chunks / n_splits);
-
-  // ---- this warp's Q fragments (rows warp*16 + g, +8), kept in registers
-  uint32_t qf[KS][4];
-  {
-    const __nv_bfloat16* q0 = sQ + (warp * 16 + g) * LD + t4 * 2;
-#pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
-      qf[ks][0] = *reinterpret_cast<const uint32_t*>(q0 + ks * 16);
-      qf[ks][1] = *reinterpret_cast<const uint32_t*>(q0 + 8 * LD + ks * 16);
-      qf[ks][2] = *reinterpret_cast<const uint32_t*>(q0 + ks * 16 + 8);
-      qf[ks][3] = *reinterpret_cast<const uint32_t*>(q0 + 8 * LD + ks * 16 + 8);
-    }
-  }
-  const int r_lo = warp * 16 + g, r_hi = r_lo + 8;
+  RD_STAMP(2);
   const int nc_lo = s_ncache[r_lo], nc_hi = s_ncache[r_hi];
   const float scale = rsqrtf((float)HD);
   float o[NT][4];
@@ -114,23 +142,20 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
   for (int i = 0; i < NT; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
   float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
 
-  const size_t head_base = ((size_t)b * dm.H + h) * (size_t)dm.max_ctx * HD;
-  const uint32_t sK_u = (uint32_t)__cvta_generic_to_shared(sK), sV_u = (uint32_t)__cvta_generic_to_shared(sV);
-
   for (int ch = c_begin; ch < c_end; ++ch) {
     const int k0 = ch * KEYS;
-    __syncthreads();  // the previous chunk's tiles are no longer read
-    for (int idx = tid; idx < KEYS * (HD / 8); idx += 128) {
-      const int kr = idx / (HD / 8), c8 = (idx - kr * (HD / 8)) * 8;
-      const int key = k0 + kr;
-      const bool valid = key < kext;
-      const size_t off = head_base + (size_t)(valid ? key : 0) * HD + c8;
-      cp_async16(sK_u + (kr * LD + c8) * 2, kc + off, valid);
-      cp_async16(sV_u + (kr * LD + c8) * 2, vc + off, valid);
+    const int buf = (ch - c_begin) & 1;
+    // the next chunk streams in while this one is used (its buffer was released by the barrier that
+    // ended the previous iteration)
+    if (ch + 1 < c_end) {
+      load_chunk(ch + 1, buf ^ 1);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
+    const __nv_bfloat16* sK = sKV + (size_t)(2 * buf) * KEYS * LD;
+    const uint32_t sV_u = sKV_u + (2 * buf + 1) * TILE_BYTES;
 
     // ---- S = Q K^T for this warp's 16 rows x 64 keys
     float s[KEYS / 8][4];
@@ -208,8 +233,10 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
         mma_bf16(o[np * 2 + 1], pf[kk], vb[2], vb[3]);
       }
     }
+    __syncthreads();  // every warp is done with this buffer
   }
 
+  RD_STAMP(3);
   // ---- results
   if (n_splits == 1) {
     const float inv_lo = l_lo > 0.f ? 1.f / l_lo : 0.f, inv_hi = l_hi > 0.f ? 1.f / l_hi : 0.f;
@@ -243,13 +270,14 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
     if (old == n_splits - 1) counters[blk] = 0;  // ready for the next launch
   }
   __syncthreads();
-  if (!s_last) return;
+  RD_STAMP(4);
+  if (!s_last) { RD_DUMP(); return; }
   __threadfence();
   // ---- merge of the splits, in split order.  Weights of every (row, split) first (into the shared
   // memory the K tile no longer needs), then each thread folds four columns of a row with all its
   // loads in flight at once.
   const float* all = scratch + (size_t)blk * n_splits * ROWS * PW;
-  float* s_w = reinterpret_cast<float*>(sK);            // [ROWS][MAX_SPLITS] weight / L of the row
+  float* s_w = reinterpret_cast<float*>(sKV);           // [ROWS][MAX_SPLITS] weight / L of the row
   constexpr int MAX_SPLITS = 16;
   for (int r = tid; r < nrows; r += 128) {
     float gm = -INFINITY;
@@ -273,28 +301,44 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
     for (int zz = 0; zz < MAX_SPLITS; ++zz) s_w[r * MAX_SPLITS + zz] = mz[zz] * inv;
   }
   __syncthreads();
-  for (int idx = tid; idx < nrows * (HD / 4); idx += 128) {
-    const int r = idx / (HD / 4), c = (idx - r * (HD / 4)) * 4;
-    float4 ov[MAX_SPLITS];
+  // four items per thread and iteration, every load of the iteration in flight together
+  const int n_items = nrows * (HD / 4);
+  for (int base_idx = tid; base_idx < n_items; base_idx += 128 * 4) {
+    float4 acc[4];
 #pragma unroll
-    for (int zz = 0; zz < MAX_SPLITS; ++zz)
-      if (zz < n_splits) ov[zz] = __ldcg(reinterpret_cast<const float4*>(all + ((size_t)zz * ROWS + r) * PW + c));
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int zz = 0; zz < n_splits; ++zz) {
+      float4 ov[4];
+      float wgt[4];
 #pragma unroll
-    for (int zz = 0; zz < MAX_SPLITS; ++zz) {
-      if (zz < n_splits) {
-        const float wgt = s_w[r * MAX_SPLITS + zz];
-        a0 += ov[zz].x * wgt; a1 += ov[zz].y * wgt; a2 += ov[zz].z * wgt; a3 += ov[zz].w * wgt;
+      for (int u = 0; u < 4; ++u) {
+        const int idx = base_idx + u * 128;
+        const int r = idx < n_items ? idx / (HD / 4) : 0, c = idx < n_items ? (idx - r * (HD / 4)) * 4 : 0;
+        ov[u] = __ldcg(reinterpret_cast<const float4*>(all + ((size_t)zz * ROWS + r) * PW + c));
+        wgt[u] = s_w[r * MAX_SPLITS + zz];
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        acc[u].x += ov[u].x * wgt[u]; acc[u].y += ov[u].y * wgt[u]; acc[u].z += ov[u].z * wgt[u]; acc[u].w += ov[u].w * wgt[u];
       }
     }
-    uint2 packed = make_uint2(pack_bf16(a0, a1), pack_bf16(a2, a3));
-    *reinterpret_cast<uint2*>(out + (size_t)(row0 + r) * dm.d + h * HD + c) = packed;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int idx = base_idx + u * 128;
+      if (idx < n_items) {
+        const int r = idx / (HD / 4), c = (idx - r * (HD / 4)) * 4;
+        uint2 packed = make_uint2(pack_bf16(acc[u].x, acc[u].y), pack_bf16(acc[u].z, acc[u].w));
+        *reinterpret_cast<uint2*>(out + (size_t)(row0 + r) * dm.d + h * HD + c) = packed;
+      }
+    }
   }
+  RD_STAMP(5);
+  RD_DUMP();
 }
 
 template <int HD>
 size_t smem_bytes(int MW) {
-  return (size_t)(ROWS + 2 * KEYS) * (HD + PAD) * 2 + ROWS * 4 + (size_t)ROWS * MW * 4;
+  return (size_t)(4 * KEYS) * (HD + PAD) * 2 + ROWS * 4 + (size_t)ROWS * MW * 4;
 }
 
 }  // namespace
@@ -313,16 +357,16 @@ cudaError_t attn_tc_prepare(int hd, int MW) {
 // grid (H, sequences * row_blocks, n_splits)
 cudaError_t launch_attention_tc(const float* qkv, const void* kcache, const void* vcache, void* out, const RowTables& rt,
                                 const int32_t* seq_off, const Dims& dm, int n_seq, int row_blocks, int n_splits,
-                                float* scratch, int32_t* counters, cudaStream_t st) {
+                                float* scratch, int32_t* counters, unsigned long long* dbg, cudaStream_t st) {
   dim3 grid(dm.H, n_seq * row_blocks, n_splits);
   if (dm.hd == 128)
     launch_pdl(attention_tc_kernel<128>, grid, 128, smem_bytes<128>(dm.MW), st, 
         qkv, (const __nv_bfloat16*)kcache, (const __nv_bfloat16*)vcache, (__nv_bfloat16*)out, rt, seq_off, dm, row_blocks,
-        n_splits, scratch, counters);
+        n_splits, scratch, counters, dbg);
   else if (dm.hd == 64)
     launch_pdl(attention_tc_kernel<64>, grid, 128, smem_bytes<64>(dm.MW), st, 
         qkv, (const __nv_bfloat16*)kcache, (const __nv_bfloat16*)vcache, (__nv_bfloat16*)out, rt, seq_off, dm, row_blocks,
-        n_splits, scratch, counters);
+        n_splits, scratch, counters, dbg);
   else
     return cudaErrorInvalidValue;
   return cudaGetLastError();

@@ -415,7 +415,7 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* map_a, int N, int K, c
   // Skinny launches (the decode step) leave about 70 KB of the SM's shared memory to the small kernels
   // that run between projections, so that this kernel can become resident, and start its weight
   // stream, while they are still running.
-  static const int cap_kb = getenv("RD_TC_SMEM_KB") ? atoi(getenv("RD_TC_SMEM_KB")) : 160;   // tuning toggles
+  static const int cap_kb = getenv("RD_TC_SMEM_KB") ? atoi(getenv("RD_TC_SMEM_KB")) : 152;   // tuning toggles
   static const long long pf_bytes = getenv("RD_TC_PREFETCH_MB") ? (long long)atoi(getenv("RD_TC_PREFETCH_MB")) << 20 : L2_PREFETCH_BYTES;
   const int budget = p.mt <= 64 ? (smem_limit < cap_kb * 1024 ? smem_limit : cap_kb * 1024) : smem_limit;
   int stages = (budget - overhead) / stage_bytes;
