@@ -214,7 +214,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--oracle-layers", type=int, default=2)
     ap.add_argument("--reference-max-steps", type=int, default=8)
-    ap.add_argument("--cpu-steps", type=int, default=6)
+    ap.add_argument("--cpu-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the planted-beam and autoregressive comparison legs")
     args = ap.parse_args()
