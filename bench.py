@@ -191,6 +191,25 @@ def workload_config(args, cfg):
             "parallelism": "replicas only (no collective)"}
 
 
+# --------------------------------------------------------------------------- replicas (N > 1)
+def reduce_over_ranks(ms, tokens, device):
+    """Whole-job figures of N independent replicas: the slowest rank's time and the sum of the tokens.
+    No-op without an initialised process group.  Works on any backend (tests run it over gloo)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return ms, tokens
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    tk = torch.tensor([tokens], device=device, dtype=torch.int64)
+    dist.all_reduce(tk, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(tk.item())
+
+
+def shard_of_rank(rank):
+    """Replicas share nothing: each rank decodes its own prompts (seed offset) with its own copy of the weights."""
+    return {"prompt_seed_offset": 100 * rank}
+
+
 # --------------------------------------------------------------------------- GPU legs
 def timed_loop(eng, n, fn):
     """n calls of fn between two events on the current stream; returns ms."""
@@ -244,7 +263,7 @@ def main():
                          + need * (L + 1) + 2 + BW * L)
     w = synth.make_weights(cfg, device)
     eng = binding.ReDrafter(cfg, w, device=device)
-    prompts = synth.make_prompts(cfg, B, seed=cfg.get("seed", 0) + 100 * rank)
+    prompts = synth.make_prompts(cfg, B, seed=cfg.get("seed", 0) + shard_of_rank(rank)["prompt_seed_offset"])
     out = binding.AcceptOut(B, L, device)
 
     def barrier():
@@ -274,13 +293,7 @@ def main():
     tokens = int(n_acc.sum().item()) + args.steps * B
     ctx_end, _, _ = eng.get_state()
     ctx_mid = float(ctx_end.float().mean().item()) - 0.5 * tokens / B
-    if dist is not None:
-        t = torch.tensor([ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-        tk = torch.tensor([tokens], device=device, dtype=torch.int64)
-        dist.all_reduce(tk)
-        tokens = int(tk.item())
+    ms, tokens = reduce_over_ranks(ms, tokens, device)
     value = tokens / (ms * 1e-3)
     ms_per_step = ms / args.steps
 
@@ -300,13 +313,7 @@ def main():
         eng.step(None, out)
     barrier()
     ms_e2e = timed_loop(eng, args.steps, one_e2e)
-    if dist is not None:
-        t = torch.tensor([ms_e2e], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-        tk = torch.tensor([e2e_tokens[0]], device=device, dtype=torch.int64)
-        dist.all_reduce(tk)
-        e2e_tokens[0] = int(tk.item())
+    ms_e2e, e2e_tokens[0] = reduce_over_ranks(ms_e2e, e2e_tokens[0], device)
     e2e = {"value": e2e_tokens[0] / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 0,
            "d2h_bytes_per_step": int(B * (L + 2) * 4), "ms_per_step": ms_e2e / args.steps,
            "note": "redrafter_step through the C ABI; the accepted tokens are copied to pinned host memory and the stream "
