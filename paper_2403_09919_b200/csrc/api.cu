@@ -290,16 +290,17 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
   RowTables rt{w.row_tok, w.row_seq, w.row_pos, w.row_slot, w.row_ncache, w.row_local, mask, w.m_total};
   CKP(h, PROF_MISC, launch_embed(dm.dtype, h->w.tok_emb, w.row_tok, w.x, dm.d, dm.V, w.m_total, m_max, w.status, st));
   CKP(h, PROF_MISC, launch_rope_table(w.row_pos, w.rope_tab, dm.hd, dm.theta, w.m_total, m_max, st));
-  // attention launch geometry (tensor-core path): blocks of 64 rows per sequence, keys split so that
-  // every SM gets a CTA, at least one 64-key chunk per split
+  // attention launch geometry (tensor-core path): tiles of 16 rows per sequence; keys split over CTAs only
+  // for long contexts with few tiles
   int row_blocks = 1, n_splits = 1;
   if (h->use_tc) {
     const int rpb = attn_tc_rows_per_block();
     row_blocks = (rows_per_seq_max + rpb - 1) / rpb;
     const int blocks = dm.H * n_seq * row_blocks;
     n_splits = h->tc_grid / blocks;  // at most one CTA per SM: a second wave would double the time
+    // ... and only when a CTA would otherwise walk many chunks: the cross-CTA merge costs several microseconds
     const int max_chunks = (h->ctx_bound + rows_per_seq_max + 63) / 64;
-    if (n_splits > max_chunks) n_splits = max_chunks;
+    if (n_splits > (max_chunks + 7) / 8) n_splits = (max_chunks + 7) / 8;
     if (n_splits > 16) n_splits = 16;
     if (n_splits < 1) n_splits = 1;
     while (n_splits > 1 && (long long)blocks * n_splits > ATT_MAX_SPLIT_BLOCKS) --n_splits;
