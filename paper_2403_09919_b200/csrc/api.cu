@@ -50,6 +50,7 @@ struct Workspace {
   float* tc_partial;
   // tensor-core attention scratch
   int32_t *att_counters, *sel_counters;
+  unsigned int* chain_ctr;  // counters of the launch-to-launch hand-off
   float* att_scratch;
   unsigned long long* trace;  // [TRACE_SLOTS][8] timestamps of traced projection launches
 };
@@ -84,6 +85,7 @@ struct rd_handle {
   bool use_tc;
   int trace_next;  // next trace slot, -1 = tracing off
   int tc_grid, tc_smem;
+  Chain chain;  // counter hand-off between the launches of a forward pass
   std::unordered_map<const void*, TensorMapBox> maps;               // weights
   std::unordered_map<const void*, std::pair<int, int>> act_shape;   // activation buffers: rows, cols
   std::map<std::pair<const void*, int>, TensorMapBox> act_maps;     // by (buffer, rows per box), made on first use
@@ -164,6 +166,7 @@ void carve(Bump& bp, const Dims& dm, int m_cap, Workspace* w) {
   w->seq_off = bp.take<int32_t>(B + 1);
   w->att_counters = bp.take<int32_t>(ATT_MAX_SPLIT_BLOCKS);
   w->sel_counters = bp.take<int32_t>(B);
+  w->chain_ctr = bp.take<unsigned int>(CHAIN_SLOTS);
   w->x = bp.take<float>((size_t)m_cap * dm.d);
   w->qkv = bp.take<float>((size_t)m_cap * 3 * dm.d);
   w->proj_d = bp.take<float>((size_t)m_cap * dm.d);
@@ -242,10 +245,8 @@ struct ProfScope {
   } while (0)
 
 // One projection Y = A W^T into the fp32 buffer `raw` (row stride ld_raw); fills `out` for the consumer.
-// `next_w`: the weight matrix of the projection that follows in the step (its first tiles are prefetched
-// into L2), or nullptr.
 int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, const int32_t* m_total, int m_max, float* raw,
-         int ld_raw, GemmOut* out, const void* next_w, cudaStream_t st) {
+         int ld_raw, GemmOut* out, Chain* chain, cudaStream_t st) {
   ProfScope ps(h, 0, (double)N * K * esize(h->dm.dtype), st);
   if (h->use_tc) {
     auto iw = h->maps.find(W);
@@ -264,15 +265,11 @@ int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, cons
     }
     unsigned long long* tr = nullptr;
     if (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) tr = h->ws.trace + (size_t)8 * h->trace_next++;
-    const TensorMapBox* nx = nullptr;
-    if (next_w) {
-      auto in = h->maps.find(next_w);
-      if (in != h->maps.end()) nx = &in->second;
-    }
     CK(h, launch_gemm_tc(&iw->second, &ia->second, N, K, m_total, m_max, raw, ld_raw, h->ws.tc_partial, h->ws.status,
-                         h->tc_grid, h->tc_smem, tr, nx, nx ? nx->rows : 0, nx ? nx->cols : 0, out, st));
+                         h->tc_grid, h->tc_smem, tr, out, chain, st));
     return RD_OK;
   }
+  if (chain) chain->cut();
   CK(h, launch_gemm_simt(h->dm.dtype, A, lda, W, N, K, m_total, m_max, raw, ld_raw, out, st));
   return RD_OK;
 }
@@ -306,36 +303,40 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
     while (n_splits > 1 && (long long)blocks * n_splits > ATT_MAX_SPLIT_BLOCKS) --n_splits;
   }
   GemmOut g_qkv, g_o, g_gu, g_dn;
+  // inside the layer loop every launch hands over to the next through a counter; the launches before
+  // and after it use the grid dependency
+  Chain* ch = h->use_tc ? &h->chain : nullptr;
+  h->chain.cut();
   for (int l = 0; l < dm.n_layers; ++l) {
     // attention block: (x += down of the previous layer) -> norm -> QKV -> rotary + KV write -> attention -> O
     CKP(h, PROF_NORM, launch_rmsnorm(dm.dtype, w.x, l ? &g_dn : nullptr, h->attn_norm[l], w.a_t, nullptr, dm.d, dm.eps,
-                                     w.m_total, m_max, st));
-    int rc = gemm(h, w.a_t, dm.d, h->wqkv[l], 3 * dm.d, dm.d, w.m_total, m_max, w.qkv, 3 * dm.d, &g_qkv, h->wo[l], st);
+                                     w.m_total, m_max, ch, st));
+    int rc = gemm(h, w.a_t, dm.d, h->wqkv[l], 3 * dm.d, dm.d, w.m_total, m_max, w.qkv, 3 * dm.d, &g_qkv, ch, st);
     if (rc) return rc;
     CKP(h, PROF_ROPE, launch_rope_kv(dm.dtype, w.qkv, g_qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.rope_tab, rt, dm,
-                                     m_max, w.status, st));
+                                     m_max, w.status, ch, st));
     {
       ProfScope ps(h, 1, 0.0, st);
       if (h->use_tc)
         CK(h, launch_attention_tc(w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.attn_t, rt, w.seq_off, dm, n_seq,
                                   row_blocks, n_splits, w.att_scratch, w.att_counters,
-                                  (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) ? w.trace + (size_t)8 * h->trace_next++ : nullptr, st));
+                                  (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) ? w.trace + (size_t)8 * h->trace_next++ : nullptr, ch, st));
       else
         CK(h, launch_attention(dm.dtype, w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.attn_t, rt, dm, m_max, st));
     }
-    rc = gemm(h, w.attn_t, dm.d, h->wo[l], dm.d, dm.d, w.m_total, m_max, w.proj_d, dm.d, &g_o, h->w_gate_up[l], st);
+    rc = gemm(h, w.attn_t, dm.d, h->wo[l], dm.d, dm.d, w.m_total, m_max, w.proj_d, dm.d, &g_o, ch, st);
     if (rc) return rc;
     // FFN block: (x += O) -> norm -> gate|up -> SwiGLU -> down
-    CKP(h, PROF_NORM, launch_rmsnorm(dm.dtype, w.x, &g_o, h->ffn_norm[l], w.a_t, nullptr, dm.d, dm.eps, w.m_total, m_max, st));
-    rc = gemm(h, w.a_t, dm.d, h->w_gate_up[l], 2 * dm.F, dm.d, w.m_total, m_max, w.gu, 2 * dm.F, &g_gu, h->w_down[l], st);
+    CKP(h, PROF_NORM, launch_rmsnorm(dm.dtype, w.x, &g_o, h->ffn_norm[l], w.a_t, nullptr, dm.d, dm.eps, w.m_total, m_max, ch, st));
+    rc = gemm(h, w.a_t, dm.d, h->w_gate_up[l], 2 * dm.F, dm.d, w.m_total, m_max, w.gu, 2 * dm.F, &g_gu, ch, st);
     if (rc) return rc;
-    CKP(h, PROF_SWIGLU, launch_swiglu(dm.dtype, g_gu, w.act_t, dm.F, w.m_total, m_max, st));
-    rc = gemm(h, w.act_t, dm.F, h->w_down[l], dm.d, dm.F, w.m_total, m_max, w.proj_d, dm.d, &g_dn,
-              l + 1 < dm.n_layers ? h->wqkv[l + 1] : after_w, st);
+    CKP(h, PROF_SWIGLU, launch_swiglu(dm.dtype, g_gu, w.act_t, dm.F, w.m_total, m_max, ch, st));
+    rc = gemm(h, w.act_t, dm.F, h->w_down[l], dm.d, dm.F, w.m_total, m_max, w.proj_d, dm.d, &g_dn, ch, st);
     if (rc) return rc;
   }
   CKP(h, PROF_NORM, launch_rmsnorm(dm.dtype, w.x, &g_dn, h->w.final_norm, w.hidden_t, w.hidden_f, dm.d, dm.eps, w.m_total,
-                                   m_max, st));
+                                   m_max, ch, st));
+  h->chain.cut();
   return RD_OK;
 }
 
@@ -364,22 +365,19 @@ int do_draft(rd_handle* h, cudaStream_t st, int32_t* beams, float* scores) {
     const float* xin_f = call == 1 ? w.xc_f : w.x0_f;
     if (call > 1) {
       // s_t = SiLU([U W][s_{t-1}; e_t] + b), written into the first d_rnn columns of x0 = [s_t, h]
-      int rc = gemm(h, w.se_t, dm.dr + dm.d, w.uw, dm.dr, dm.dr + dm.d, mt, rows, w.sraw, dm.dr, &g,
-                    dm.n_head_layers ? h->head_w[0] : h->w.draft_out, st);
+      int rc = gemm(h, w.se_t, dm.dr + dm.d, w.uw, dm.dr, dm.dr + dm.d, mt, rows, w.sraw, dm.dr, &g, nullptr, st);
       if (rc) return rc;
       CKP(h, PROF_DRAFT_SMALL, launch_act(dm.dtype, g, h->w.rnn_b, nullptr, 0, w.x0_f, w.x0_t, dm.dh, dm.dr, mt, rows, st));
     }
     for (int l = 0; l < dm.n_head_layers; ++l) {
       float* of = (l & 1) ? w.x2_f : w.x1_f;
       void* ot = (l & 1) ? w.x2_t : w.x1_t;
-      int rc = gemm(h, xin_t, dm.dh, h->head_w[l], dm.dh, dm.dh, mt, rows, w.hraw, dm.dh, &g,
-                    l + 1 < dm.n_head_layers ? h->head_w[l + 1] : h->w.draft_out, st);
+      int rc = gemm(h, xin_t, dm.dh, h->head_w[l], dm.dh, dm.dh, mt, rows, w.hraw, dm.dh, &g, nullptr, st);
       if (rc) return rc;
       CKP(h, PROF_DRAFT_SMALL, launch_act(dm.dtype, g, h->head_b[l], xin_f, dm.dh, of, ot, dm.dh, dm.dh, mt, rows, st));
       xin_t = ot; xin_f = of;
     }
-    int rc = gemm(h, xin_t, dm.dh, h->w.draft_out, dm.V, dm.dh, mt, rows, w.dlogits, dm.V, &g,
-                  call < dm.L ? (const void*)w.uw : h->wqkv[0], st);
+    int rc = gemm(h, xin_t, dm.dh, h->w.draft_out, dm.V, dm.dh, mt, rows, w.dlogits, dm.V, &g, nullptr, st);
     if (rc) return rc;
     CKP(h, PROF_DRAFT_SMALL, launch_draft_select(dm.dtype, g, call, w.lse, w.cand_val, w.cand_idx, sc_in, sc_out, hi_in, hi_out,
                                                  h->w.tok_emb, w.x0_f, dm.dh, w.se_t, dm, B, beams, scores, w.sel_counters, mt,
@@ -399,8 +397,7 @@ int do_verify(rd_handle* h, const rd_packed& pk, cudaStream_t st, int32_t* argma
   int rc = forward_layers(h, pk.mask, m_max, B, dm.NMAX, h->w.lm_head, st);
   if (rc) return rc;
   GemmOut g;
-  rc = gemm(h, w.hidden_t, dm.d, h->w.lm_head, dm.V, dm.d, w.m_total, m_max, w.logits, dm.V, &g,
-            dm.n_head_layers ? h->head_w[0] : h->w.draft_out, st);  // the next step starts with the drafter
+  rc = gemm(h, w.hidden_t, dm.d, h->w.lm_head, dm.V, dm.d, w.m_total, m_max, w.logits, dm.V, &g, nullptr, st);
   if (rc) return rc;
   CKP(h, PROF_MISC, launch_fill_i32(argmax, -1, B * dm.NMAX, st));
   CKP(h, PROF_MISC, launch_argmax_rows(w.logits, g, dm.V, argmax, w.row_out_index, w.m_total, m_max, st));
@@ -501,6 +498,9 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
   h->prefilled = false; h->batch = dm.B; h->ctx_bound = 0; h->launches = 0; h->err[0] = 0;
   h->profiling = false;
   h->trace_next = -1;
+  h->chain.ctr = h->ws.chain_ctr; h->chain.status = h->ws.status;
+  h->chain.trace_base = h->ws.trace; h->chain.trace_next = &h->trace_next; h->chain.trace_cap = TRACE_SLOTS;
+  h->chain.enabled = !(getenv("RD_CHAIN") && atoi(getenv("RD_CHAIN")) == 0);
   for (int c = 0; c < PROF_CLASSES; ++c) { h->ev_used[c] = 0; h->prof_ms[c] = 0; h->prof_bytes[c] = 0; h->prof_n[c] = 0; }
   // clear the state and the constants the kernels read from device memory
   cudaError_t e = cudaMemsetAsync(workspace, 0, (size_t)((char*)h->ws.x - (char*)workspace), 0);
@@ -698,7 +698,7 @@ int redrafter_ar_step(rd_handle* h, void* stream, int32_t* token) {
   int rc = forward_layers(h, nullptr, B, B, 1, h->w.lm_head, st);
   if (rc) return rc;
   GemmOut g;
-  rc = gemm(h, w.hidden_t, dm.d, h->w.lm_head, dm.V, dm.d, w.m_total, B, w.logits, dm.V, &g, h->wqkv[0], st);
+  rc = gemm(h, w.hidden_t, dm.d, h->w.lm_head, dm.V, dm.d, w.m_total, B, w.logits, dm.V, &g, nullptr, st);
   if (rc) return rc;
   CK(h, launch_argmax_rows(w.logits, g, dm.V, w.argmax_c, nullptr, w.m_total, B, st));
   CK(h, launch_ar_finish(w.argmax_c, w.hidden_f, w.ctx, w.root, w.h, token, dm, B, st));

@@ -54,10 +54,10 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
                                                            __nv_bfloat16* __restrict__ out, RowTables rt,
                                                            const int32_t* __restrict__ seq_off, Dims dm, int row_tiles,
                                                            int n_splits, float* __restrict__ scratch,
-                                                           int32_t* __restrict__ counters, unsigned long long* dbg) {
+                                                           int32_t* __restrict__ counters, unsigned long long* dbg, ChainSync cs) {
   unsigned long long t_dbg[6] = {0, 0, 0, 0, 0, 0};
   RD_STAMP(0);
-  pdl_enter();
+  chain_enter(cs);
   RD_STAMP(1);
   constexpr int LD = HD + PAD;           // shared row stride in bf16
   constexpr int NT = HD / 8;             // output n-tiles
@@ -75,7 +75,10 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
   const int seq_row0 = seq_off[b], seq_rows = seq_off[b + 1] - seq_row0;
   const int row0 = seq_row0 + rb * ROWS;
   const int nrows = min(ROWS, seq_rows - rb * ROWS);
-  if (nrows <= 0) return;  // the same for every split and head of this row tile
+  if (nrows <= 0) {  // the same for every split and head of this row tile
+    chain_exit(cs);
+    return;
+  }
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t4 = lane & 3;
   const int MW = dm.MW;
   const bool tree = rt.mask != nullptr;
@@ -89,10 +92,10 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
     const float* q_hi = qkv + (size_t)(row0 + (r_hi < nrows ? r_hi : 0)) * 3 * dm.d + h * HD + t4 * 2;
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) {
-      qraw[ks][0] = *reinterpret_cast<const float2*>(q_lo + ks * 16);
-      qraw[ks][1] = *reinterpret_cast<const float2*>(q_hi + ks * 16);
-      qraw[ks][2] = *reinterpret_cast<const float2*>(q_lo + ks * 16 + 8);
-      qraw[ks][3] = *reinterpret_cast<const float2*>(q_hi + ks * 16 + 8);
+      qraw[ks][0] = __ldcg(reinterpret_cast<const float2*>(q_lo + ks * 16));
+      qraw[ks][1] = __ldcg(reinterpret_cast<const float2*>(q_hi + ks * 16));
+      qraw[ks][2] = __ldcg(reinterpret_cast<const float2*>(q_lo + ks * 16 + 8));
+      qraw[ks][3] = __ldcg(reinterpret_cast<const float2*>(q_hi + ks * 16 + 8));
     }
   }
   const int nc_first = rt.n_cache[row0], nc_last = rt.n_cache[row0 + nrows - 1];
@@ -291,6 +294,7 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
   RD_STAMP(4);
   if (n_splits == 1) {
     if (dbg && tid == 0 && blk == 0) { for (int i = 0; i < 5; ++i) dbg[i] = t_dbg[i]; dbg[6] = t_dbg[4]; }
+    chain_exit(cs);
     return;
   }
 
@@ -304,7 +308,10 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
   }
   __syncthreads();
   if (dbg && tid == 0 && blk == 0 && z == 0) { for (int i = 0; i < 5; ++i) dbg[i] = t_dbg[i]; }
-  if (!s_last) return;
+  if (!s_last) {
+    chain_exit(cs);
+    return;
+  }
   __threadfence();
   const float* all = scratch + (size_t)blk * n_splits * ROWS * PW;
   if (tid < nrows) {
@@ -348,6 +355,7 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
         make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
   }
   if (dbg && tid == 0 && blk == 0) { RD_STAMP(5); atomicMax(dbg + 6, t_dbg[5]); }
+  chain_exit(cs);
 }
 
 template <int HD>
@@ -371,14 +379,15 @@ cudaError_t attn_tc_prepare(int hd, int MW) {
 // grid (H, sequences * row_tiles, n_splits)
 cudaError_t launch_attention_tc(const float* qkv, const void* kcache, const void* vcache, void* out, const RowTables& rt,
                                 const int32_t* seq_off, const Dims& dm, int n_seq, int row_tiles, int n_splits,
-                                float* scratch, int32_t* counters, unsigned long long* dbg, cudaStream_t st) {
+                                float* scratch, int32_t* counters, unsigned long long* dbg, Chain* chain, cudaStream_t st) {
   dim3 grid(dm.H, n_seq * row_tiles, n_splits);
+  const ChainSync cs = chain ? chain->link(grid.x * grid.y * grid.z) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
   if (dm.hd == 128)
     launch_pdl(attention_tc_kernel<128>, grid, 128, smem_bytes<128>(dm.MW), st, qkv, (const __nv_bfloat16*)kcache,
-               (const __nv_bfloat16*)vcache, (__nv_bfloat16*)out, rt, seq_off, dm, row_tiles, n_splits, scratch, counters, dbg);
+               (const __nv_bfloat16*)vcache, (__nv_bfloat16*)out, rt, seq_off, dm, row_tiles, n_splits, scratch, counters, dbg, cs);
   else if (dm.hd == 64)
     launch_pdl(attention_tc_kernel<64>, grid, 128, smem_bytes<64>(dm.MW), st, qkv, (const __nv_bfloat16*)kcache,
-               (const __nv_bfloat16*)vcache, (__nv_bfloat16*)out, rt, seq_off, dm, row_tiles, n_splits, scratch, counters, dbg);
+               (const __nv_bfloat16*)vcache, (__nv_bfloat16*)out, rt, seq_off, dm, row_tiles, n_splits, scratch, counters, dbg, cs);
   else
     return cudaErrorInvalidValue;
   return cudaGetLastError();

@@ -51,35 +51,80 @@ cudaError_t launch_embed(int dtype, const void* emb, const int32_t* tok, float* 
   return cudaGetLastError();
 }
 
+// Four consecutive outputs in the activation type (16- or 8-byte store; the address is that much aligned).
+__device__ __forceinline__ void store4(float* p, float a, float b, float c, float d) { *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d); }
+__device__ __forceinline__ void store4(__nv_bfloat16* p, float a, float b, float c, float d) {
+  const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+  uint2 u;
+  u.x = *reinterpret_cast<const uint32_t*>(&lo);
+  u.y = *reinterpret_cast<const uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(p) = u;
+}
+
 // ---------------------------------------------------------------- RMSNorm
 // y = x / sqrt(mean(x^2) + eps) * gain, one block per row.  The row is read once with 128-bit loads
 // and kept in registers between the reduction and the scaling (d <= 8192).
 constexpr int NORM_THREADS = 512;
 
+// Packed gain values of one float4 of the row.
+template <typename T> struct Gain4;
+template <> struct Gain4<float> {
+  float4 g;
+  __device__ __forceinline__ void load(const float* p) { g = *reinterpret_cast<const float4*>(p); }
+  __device__ __forceinline__ float4 get() const { return g; }
+};
+template <> struct Gain4<__nv_bfloat16> {
+  uint2 g;
+  __device__ __forceinline__ void load(const __nv_bfloat16* p) { g = *reinterpret_cast<const uint2*>(p); }
+  __device__ __forceinline__ float4 get() const {
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&g.x));
+    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&g.y));
+    return make_float4(a.x, a.y, b.x, b.y);
+  }
+};
+
+// At most 96 registers per thread: one CTA of this kernel (512 threads) and one CTA of the projection that
+// follows it then fit the SM's register file together, so the projection is resident and has its first
+// weight tiles in flight while the norm still runs.
 template <typename T, int NORM_MAXV>
-__global__ void __launch_bounds__(NORM_THREADS) rmsnorm_kernel(float* __restrict__ x, GemmOut proj, const T* __restrict__ gain,
-                                                                T* __restrict__ out_t, float* __restrict__ out_f, int d,
-                                                                float eps, const int32_t* __restrict__ m_total) {
-  pdl_enter();
+__global__ void __maxnreg__(88)
+    rmsnorm_kernel(float* __restrict__ x, GemmOut proj, const T* __restrict__ gain, T* __restrict__ out_t,
+                   float* __restrict__ out_f, int d, float eps, const int32_t* __restrict__ m_total, ChainSync cs) {
+  chain_begin(cs);
   __shared__ float sh[32];
   const int m = blockIdx.x;
-  const int M = *m_total;
-  if (m >= M) return;
-  float4* xr = reinterpret_cast<float4*>(x + (size_t)m * d);
   const int nvec = d >> 2;
+  // the gain is a weight: requested before the wait, it has arrived when the row has
+  Gain4<T> gn[NORM_MAXV];
+#pragma unroll
+  for (int k = 0; k < NORM_MAXV; ++k) {
+    const int i = threadIdx.x + k * NORM_THREADS;
+    if (i < nvec) gn[k].load(gain + 4 * i);
+  }
+  chain_wait_cta(cs);
+  float4* xr = reinterpret_cast<float4*>(x + (size_t)m * d);
   const bool add = proj.raw != nullptr;   // x += the projection that ends the previous block (O or down)
-  const int m_tiles = add ? gemm_m_tiles(proj, M) : 1;
+  // Decode-time launches have one row tile whatever the row count: the row's loads then do not wait for the
+  // row count (rows past it exist in memory and are simply not written back).
+  const volatile int32_t* mt_ptr = m_total;
+  int M = -1, m_tiles = 1;
+  if (add && proj.m_tiles_max != 1) { M = *mt_ptr; m_tiles = gemm_m_tiles(proj, M); }
   float4 v[NORM_MAXV];
-  GemmPending4<6> pend[NORM_MAXV];
+  GemmPending4<5> pend[NORM_MAXV];
   float ss = 0.f;
   // every load first (residual row, projection output, partial slots), then the arithmetic
 #pragma unroll
   for (int k = 0; k < NORM_MAXV; ++k) {
     const int i = threadIdx.x + k * NORM_THREADS;
     if (i < nvec) {
-      v[k] = xr[i];
-      if (add) pend[k] = gemm_issue4<6>(proj, m_tiles, m, 4 * i);
+      v[k] = __ldcg(xr + i);
+      if (add) pend[k] = gemm_issue4<5>(proj, m_tiles, m, 4 * i);
     }
+  }
+  if (M < 0) M = *mt_ptr;
+  if (m >= M) {
+    chain_exit(cs);
+    return;
   }
 #pragma unroll
   for (int k = 0; k < NORM_MAXV; ++k) {
@@ -99,26 +144,27 @@ __global__ void __launch_bounds__(NORM_THREADS) rmsnorm_kernel(float* __restrict
   for (int k = 0; k < NORM_MAXV; ++k) {
     const int i = threadIdx.x + k * NORM_THREADS;
     if (i < nvec) {
-      const float g0 = to_f<T>(gain[4 * i]), g1 = to_f<T>(gain[4 * i + 1]), g2 = to_f<T>(gain[4 * i + 2]),
-                  g3 = to_f<T>(gain[4 * i + 3]);
-      const float y0 = v[k].x * r * g0, y1 = v[k].y * r * g1, y2 = v[k].z * r * g2, y3 = v[k].w * r * g3;
+      const float4 g = gn[k].get();
+      const float y0 = v[k].x * r * g.x, y1 = v[k].y * r * g.y, y2 = v[k].z * r * g.z, y3 = v[k].w * r * g.w;
       const size_t o = (size_t)m * d + 4 * i;
-      if (out_t) { out_t[o] = from_f<T>(y0); out_t[o + 1] = from_f<T>(y1); out_t[o + 2] = from_f<T>(y2); out_t[o + 3] = from_f<T>(y3); }
+      if (out_t) store4(out_t + o, y0, y1, y2, y3);
       if (out_f) *reinterpret_cast<float4*>(out_f + o) = make_float4(y0, y1, y2, y3);
     }
   }
+  chain_exit(cs);
 }
 
 // x: residual stream (updated in place when proj != nullptr: x += proj).
 cudaError_t launch_rmsnorm(int dtype, float* x, const GemmOut* proj, const void* gain, void* out_t, float* out_f32, int d,
-                           float eps, const int32_t* m_total, int m_max, cudaStream_t st) {
+                           float eps, const int32_t* m_total, int m_max, Chain* chain, cudaStream_t st) {
   if (d > 4 * NORM_THREADS * 4 || (d & 3)) return cudaErrorInvalidValue;
   GemmOut g{};
   if (proj) g = *proj;
+  const ChainSync cs = chain ? chain->link((unsigned)m_max, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
   if (d <= 4 * NORM_THREADS * 2) {
-    RD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 2>, m_max, NORM_THREADS, 0, st, x, g, (const T*)gain, (T*)out_t, out_f32, d, eps, m_total));
+    RD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 2>, m_max, NORM_THREADS, 0, st, x, g, (const T*)gain, (T*)out_t, out_f32, d, eps, m_total, cs));
   } else {
-    RD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 4>, m_max, NORM_THREADS, 0, st, x, g, (const T*)gain, (T*)out_t, out_f32, d, eps, m_total));
+    RD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 4>, m_max, NORM_THREADS, 0, st, x, g, (const T*)gain, (T*)out_t, out_f32, d, eps, m_total, cs));
   }
   return cudaGetLastError();
 }
@@ -154,11 +200,14 @@ constexpr int ROPE_SPLIT = 8;  // CTAs per row
 
 template <typename T>
 __global__ void rope_kv_kernel(float* __restrict__ qkv, GemmOut proj, T* __restrict__ kc, T* __restrict__ vc,
-                               const float2* __restrict__ table, RowTables rt, Dims dm, int* status) {
-  pdl_enter();
+                               const float2* __restrict__ table, RowTables rt, Dims dm, int* status, ChainSync cs) {
+  chain_enter(cs);
   const int m = blockIdx.x;
   const int M = *rt.m_total;
-  if (m >= M) return;
+  if (m >= M) {
+    chain_exit(cs);
+    return;
+  }
   const int b = rt.seq[m], slot = rt.slot[m];
   const int d = dm.d, hd = dm.hd, half = hd >> 1;
   const bool slot_ok = slot >= 0 && slot < dm.max_ctx;
@@ -186,38 +235,42 @@ __global__ void rope_kv_kernel(float* __restrict__ qkv, GemmOut proj, T* __restr
       vc[base + half] = from_f<T>(v2);
     }
   }
+  chain_exit(cs);
 }
 
 cudaError_t launch_rope_kv(int dtype, float* qkv, const GemmOut& proj, void* kcache, void* vcache, const float* table,
-                           const RowTables& rt, const Dims& dm, int m_max, int* status, cudaStream_t st) {
+                           const RowTables& rt, const Dims& dm, int m_max, int* status, Chain* chain, cudaStream_t st) {
   dim3 grid(m_max, ROPE_SPLIT);
+  const ChainSync cs = chain ? chain->link((unsigned)m_max * ROPE_SPLIT, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
   RD_DISPATCH(dtype, launch_pdl(rope_kv_kernel<T>, grid, 256, 0, st, qkv, proj, (T*)kcache, (T*)vcache,
-                                reinterpret_cast<const float2*>(table), rt, dm, status));
+                                reinterpret_cast<const float2*>(table), rt, dm, status, cs));
   return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------- SwiGLU
 template <typename T>
-__global__ void swiglu_kernel(GemmOut proj, T* __restrict__ out, int F, const int32_t* __restrict__ m_total) {
-  pdl_enter();
+__global__ void swiglu_kernel(GemmOut proj, T* __restrict__ out, int F, const int32_t* __restrict__ m_total, ChainSync cs) {
+  chain_enter(cs);
   const int m = blockIdx.y;
   const int M = *m_total;
-  if (m >= M) return;
   const int f = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
-  if (f >= F) return;
-  const int m_tiles = gemm_m_tiles(proj, M);
-  const auto pg = gemm_issue4<4>(proj, m_tiles, m, f), pu = gemm_issue4<4>(proj, m_tiles, m, F + f);
-  const float4 g = gemm_finish4(proj, m_tiles, pg), u = gemm_finish4(proj, m_tiles, pu);
-  T* o = out + (size_t)m * F + f;
-  o[0] = from_f<T>(silu_f(g.x) * u.x); o[1] = from_f<T>(silu_f(g.y) * u.y);
-  o[2] = from_f<T>(silu_f(g.z) * u.z); o[3] = from_f<T>(silu_f(g.w) * u.w);
+  if (m < M && f < F) {
+    const int m_tiles = gemm_m_tiles(proj, M);
+    const auto pg = gemm_issue4<4>(proj, m_tiles, m, f), pu = gemm_issue4<4>(proj, m_tiles, m, F + f);
+    const float4 g = gemm_finish4(proj, m_tiles, pg), u = gemm_finish4(proj, m_tiles, pu);
+    T* o = out + (size_t)m * F + f;
+    o[0] = from_f<T>(silu_f(g.x) * u.x); o[1] = from_f<T>(silu_f(g.y) * u.y);
+    o[2] = from_f<T>(silu_f(g.z) * u.z); o[3] = from_f<T>(silu_f(g.w) * u.w);
+  }
+  chain_exit(cs);
 }
 
 // proj: the gate|up projection [M][2F]; out: [M][F].  F must be a multiple of 4.
 cudaError_t launch_swiglu(int dtype, const GemmOut& proj, void* out_t, int F, const int32_t* m_total, int m_max,
-                          cudaStream_t st) {
+                          Chain* chain, cudaStream_t st) {
   dim3 grid((F / 4 + 255) / 256, m_max);
-  RD_DISPATCH(dtype, launch_pdl(swiglu_kernel<T>, grid, 256, 0, st, proj, (T*)out_t, F, m_total));
+  const ChainSync cs = chain ? chain->link(grid.x * grid.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
+  RD_DISPATCH(dtype, launch_pdl(swiglu_kernel<T>, grid, 256, 0, st, proj, (T*)out_t, F, m_total, cs));
   return cudaGetLastError();
 }
 

@@ -38,7 +38,6 @@ constexpr int TILE_K = 64;        // bf16 per k-block = one 128-byte swizzle row
 constexpr int W_STAGE_BYTES = TILE_N * TILE_K * 2;
 constexpr int NUM_THREADS = 192;
 constexpr unsigned long long WAIT_LIMIT_NS = 1000000000ull;
-constexpr long long L2_PREFETCH_BYTES = 0;  // of the next projection's weights into L2; measured: any amount slows the step
 
 struct TcParams {
   int N, K, nkb, n_tiles, mt, m_tiles_max, stages, tmem_cols;
@@ -48,8 +47,7 @@ struct TcParams {
   float* partial;     // [gridDim.x][mt * 128]
   int32_t* status;
   unsigned long long* trace;  // 8 timestamps of this launch (see redrafter_trace_read) or nullptr
-  // L2 prefetch of the weights the NEXT projection will read first (0 units = none)
-  int next_nkb, next_n_tiles, pf_units;
+  ChainSync cs;       // counter hand-off with the launches before and after this one
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -98,8 +96,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
-__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* map, int x, int y) {
-  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y) : "memory");
+// Weight tiles are read once per step: they are marked evict-first so that the stream (hundreds of MB per
+// layer) does not push the step's small working set -- residual stream, row tables, rotary table, norm gains'
+// neighbours, partial sums -- out of the L2 between two uses.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;" ::"r"(dst),
+      "l"(map), "r"(bar), "r"(x), "r"(y), "l"(pol)
+      : "memory");
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
@@ -142,23 +151,19 @@ __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;"
 
 __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
                                                                  const __grid_constant__ CUtensorMap map_a,
-                                                                 const __grid_constant__ CUtensorMap map_next,
                                                                  const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   pdl_launch_dependents();  // the next kernel may start its own prologue now
-  if (p.trace && threadIdx.x == 0) atomicMin(p.trace + 0, globaltimer());   // first CTA entered
-  // leave at once when an earlier launch already timed out; one thread reads the flag so that the
-  // whole CTA takes the same branch
-  __shared__ int skip_launch;
-  if (threadIdx.x == 0) skip_launch = (*(volatile int32_t*)p.status & DEV_ERR_TIMEOUT) ? 1 : 0;
-  __syncthreads();
-  if (skip_launch) return;
+  if (p.trace && threadIdx.x == 0) { atomicMin(p.trace + 0, globaltimer()); }
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // With a single row tile the work split does not depend on the row count, so the weight stream can
   // start before the preceding kernels have finished (they produce the activations and the row count).
   const bool early = (p.m_tiles_max == 1);
-  if (!early) pdl_wait();
+  if (!early) {
+    if (threadIdx.x == 0) chain_wait_thread(p.cs);
+    __syncthreads();
+  }
   const int m_tiles = early ? 1 : (*p.m_total + p.mt - 1) / p.mt;
   const long long G = gridDim.x;
   const long long U = (long long)p.n_tiles * m_tiles * p.nkb;
@@ -179,11 +184,38 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
   volatile int* epi_ok = reinterpret_cast<volatile int*>(misc + 12);
 
+  // iteration i of this CTA = unit u0 + i = (tile, k-block) in tile-major order
+  const uint32_t n_it = (uint32_t)(u1 - u0);
+  const uint32_t pre = early ? min(n_it, (uint32_t)p.stages) : 0u;
+  const uint64_t pol_w = l2_policy_evict_first();
+  auto issue_w = [&](uint32_t i) {
+    const long long u = u0 + i;
+    const int t = (int)(u / p.nkb), kb = (int)(u - (long long)t * p.nkb);
+    const int s = i % p.stages;
+    mbar_expect_tx(full_bar(s), stage_bytes);
+    tma_load_2d_hint(base + s * stage_bytes, &map_w, full_bar(s), kb * TILE_K, (t / m_tiles) * TILE_N, pol_w);
+  };
+  auto issue_a = [&](uint32_t i) {
+    const long long u = u0 + i;
+    const int t = (int)(u / p.nkb), kb = (int)(u - (long long)t * p.nkb);
+    const int s = i % p.stages;
+    const int m_tile = t - (t / m_tiles) * m_tiles;
+    // one box of MT rows: the TMA unit's cost is per operation, not per byte, at these sizes
+    tma_load_2d(base + s * stage_bytes + W_STAGE_BYTES, &map_a, full_bar(s), kb * TILE_K, m_tile * p.mt);
+  };
+
   if (threadIdx.x == 0) {
+    // The producer thread sets the barriers up and starts the weight stream at once: the weights of the
+    // first ring-full of k-blocks depend on nothing in the step, and nothing of the CTA's remaining set-up
+    // (tensor-memory allocation, the other roles' start) needs to come first.
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
     for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    for (uint32_t i = 0; i < pre; ++i) issue_w(i);
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
@@ -199,28 +231,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
   if (warp == 0) {
     // ===================== TMA producer =====================
     if (lane == 0 && u0 < u1) {
-      // iteration i of this CTA = unit u0 + i = (tile, k-block) in tile-major order
-      const uint32_t n_it = (uint32_t)(u1 - u0);
-      const uint32_t pre = early ? min(n_it, (uint32_t)p.stages) : 0u;
-      auto issue_w = [&](uint32_t i) {
-        const long long u = u0 + i;
-        const int t = (int)(u / p.nkb), kb = (int)(u - (long long)t * p.nkb);
-        const int s = i % p.stages;
-        mbar_expect_tx(full_bar(s), stage_bytes);
-        tma_load_2d(base + s * stage_bytes, &map_w, full_bar(s), kb * TILE_K, (t / m_tiles) * TILE_N);
-      };
-      auto issue_a = [&](uint32_t i) {
-        const long long u = u0 + i;
-        const int t = (int)(u / p.nkb), kb = (int)(u - (long long)t * p.nkb);
-        const int s = i % p.stages;
-        const int m_tile = t - (t / m_tiles) * m_tiles;
-        // one box of MT rows: the TMA unit's cost is per operation, not per byte, at these sizes
-        tma_load_2d(base + s * stage_bytes + W_STAGE_BYTES, &map_a, full_bar(s), kb * TILE_K, m_tile * p.mt);
-      };
-      // weights of the first ring-full of k-blocks do not depend on the preceding kernels
-      for (uint32_t i = 0; i < pre; ++i) issue_w(i);
-      if (early) pdl_wait();
+      if (p.trace) atomicMax(p.trace + 7, globaltimer());   // last CTA ready to wait
+      if (early) chain_wait_thread(p.cs);
+      chain_fence_async_reads();  // the activations were written by ordinary stores of the preceding launch
       if (p.trace) { atomicMin(p.trace + 1, globaltimer()); atomicMax(p.trace + 2, globaltimer()); }   // dependency resolved
+      // an earlier launch of the step gave up on a wait: wind this one down through the roles' abort paths
+      if (*(volatile int32_t*)p.status & DEV_ERR_TIMEOUT) *abort_flag = 1;
       for (uint32_t i = 0; i < pre; ++i) issue_a(i);
       bool ok = true;
       for (uint32_t i = pre; i < n_it; ++i) {
@@ -230,19 +246,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
         issue_w(i);
         issue_a(i);
       }
-      // The decode step is a fixed chain of projections separated by short kernels.  Once this CTA's own
-      // loads are issued it asks the L2 (126 MB) for the tiles the same CTA index will read first in the
-      // NEXT projection, so HBM keeps streaming weights through this kernel's tail and the gap behind it.
-      if (ok && p.pf_units > 0) {
-        const long long Un = (long long)p.next_n_tiles * p.next_nkb;
-        const long long v0 = gemm_range_begin(blockIdx.x, Un, G);
-        const long long v1 = min(gemm_range_begin(blockIdx.x + 1, Un, G), v0 + p.pf_units);
-        for (long long v = v0; v < v1; ++v) {
-          const int t = (int)(v / p.next_nkb), kb = (int)(v - (long long)t * p.next_nkb);
-          tma_prefetch_l2_2d(&map_next, kb * TILE_K, t * TILE_N);
-        }
-      }
-      if (!ok) {  // give the copies already issued time to land before the CTA's shared memory is released
+      if (!ok || *abort_flag) {  // give the copies already issued time to land before the CTA's shared memory is released
         const unsigned long long t0 = globaltimer();
         while (globaltimer() - t0 < 2000000ull) __nanosleep(1000);
       }
@@ -279,7 +283,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
     }
   } else {
     // ===================== epilogue (warps 2..5) =====================
-    if (early) pdl_wait();                  // residual, addend and the row count come from preceding kernels
+    if (early) {                            // the row count comes from preceding kernels, and their readers of
+      if (threadIdx.x == 64) chain_wait_thread(p.cs);   // this launch's output buffers must be done
+      epi_bar_sync();
+    }
     const int M = *p.m_total;
     const int q = warp & 3;                 // TMEM lane quarter this warp may read
     const int row = q * 32 + lane;          // weight row inside the tile
@@ -328,6 +335,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
   tc_fence_before();
   __syncthreads();
   if (p.trace && threadIdx.x == 0) { atomicMin(p.trace + 5, globaltimer()); atomicMax(p.trace + 6, globaltimer()); }   // CTA done
+  chain_exit(p.cs);
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
@@ -398,8 +406,7 @@ cudaError_t tc_prepare(int* smem_limit_out) {
 
 cudaError_t launch_gemm_tc(const void* map_w, const void* map_a, int N, int K, const int32_t* m_total, int m_max,
                            float* raw, int ld_raw, float* partial, int32_t* status, int grid, int smem_limit,
-                           unsigned long long* trace, const void* map_next, int next_N, int next_K, GemmOut* out_desc,
-                           cudaStream_t st) {
+                           unsigned long long* trace, GemmOut* out_desc, Chain* chain, cudaStream_t st) {
   TcParams p;
   p.N = N; p.K = K; p.nkb = (K + TILE_K - 1) / TILE_K; p.n_tiles = (N + TILE_N - 1) / TILE_N;
   p.mt = tc_pick_mt(m_max > 0 ? m_max : 1);
@@ -416,7 +423,6 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* map_a, int N, int K, c
   // that run between projections, so that this kernel can become resident, and start its weight
   // stream, while they are still running.
   static const int cap_kb = getenv("RD_TC_SMEM_KB") ? atoi(getenv("RD_TC_SMEM_KB")) : 152;   // tuning toggles
-  static const long long pf_bytes = getenv("RD_TC_PREFETCH_MB") ? (long long)atoi(getenv("RD_TC_PREFETCH_MB")) << 20 : L2_PREFETCH_BYTES;
   const int budget = p.mt <= 64 ? (smem_limit < cap_kb * 1024 ? smem_limit : cap_kb * 1024) : smem_limit;
   int stages = (budget - overhead) / stage_bytes;
   if (stages > 16) stages = 16;
@@ -426,16 +432,9 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* map_a, int N, int K, c
   while (cols < 2 * p.mt) cols <<= 1;
   p.tmem_cols = cols;
   p.m_total = m_total; p.raw = raw; p.ld_raw = ld_raw; p.partial = partial; p.status = status; p.trace = trace;
-  p.next_nkb = 0; p.next_n_tiles = 0; p.pf_units = 0;
-  if (map_next) {
-    p.next_nkb = (next_K + TILE_K - 1) / TILE_K;
-    p.next_n_tiles = (next_N + TILE_N - 1) / TILE_N;
-    const long long per_cta = (pf_bytes / W_STAGE_BYTES) / grid;
-    p.pf_units = (int)per_cta;
-  }
+  p.cs = chain ? chain->link((unsigned)grid) : ChainSync{nullptr, 0u, nullptr, status, nullptr};
   const size_t smem = (size_t)stages * stage_bytes + overhead;
-  launch_pdl(gemm_tc_kernel, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, *(const CUtensorMap*)map_a,
-             *(const CUtensorMap*)(map_next ? map_next : map_w), p);
+  launch_pdl(gemm_tc_kernel, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, *(const CUtensorMap*)map_a, p);
   return cudaGetLastError();
 }
 

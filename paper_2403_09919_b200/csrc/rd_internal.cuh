@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "chain.cuh"
 #include "gemm_out.cuh"
 #include "redrafter.h"
 
@@ -61,17 +62,16 @@ size_t tc_partial_floats(int grid, int mt);
 cudaError_t tc_prepare(int* smem_limit_out);
 cudaError_t launch_gemm_tc(const void* map_w, const void* map_a, int N, int K, const int32_t* m_total, int m_max,
                            float* raw, int ld_raw, float* partial, int32_t* status, int grid, int smem_limit,
-                           unsigned long long* trace, const void* map_next, int next_N, int next_K, GemmOut* out_desc,
-                           cudaStream_t st);
+                           unsigned long long* trace, GemmOut* out_desc, Chain* chain, cudaStream_t st);
 
 cudaError_t launch_embed(int dtype, const void* emb, const int32_t* tok, float* x, int d, int V, const int32_t* m_total,
                          int m_max, int* status, cudaStream_t st);
 cudaError_t launch_rmsnorm(int dtype, float* x, const GemmOut* proj, const void* gain, void* out_t, float* out_f32, int d,
-                           float eps, const int32_t* m_total, int m_max, cudaStream_t st);
+                           float eps, const int32_t* m_total, int m_max, Chain* chain, cudaStream_t st);
 cudaError_t launch_rope_table(const int32_t* pos, float* table, int hd, float theta, const int32_t* m_total, int m_max,
                               cudaStream_t st);
 cudaError_t launch_rope_kv(int dtype, float* qkv, const GemmOut& proj, void* kcache, void* vcache, const float* table,
-                           const RowTables& rt, const Dims& dm, int m_max, int* status, cudaStream_t st);
+                           const RowTables& rt, const Dims& dm, int m_max, int* status, Chain* chain, cudaStream_t st);
 cudaError_t launch_attention(int dtype, const float* qkv, const void* kcache, const void* vcache, void* out_t,
                              const RowTables& rt, const Dims& dm, int m_max, cudaStream_t st);
 // Tensor-core attention (bf16): KV tiles staged through shared memory, split over the keys.
@@ -80,9 +80,9 @@ int attn_tc_rows_per_block();
 cudaError_t attn_tc_prepare(int hd, int MW);
 cudaError_t launch_attention_tc(const float* qkv, const void* kcache, const void* vcache, void* out, const RowTables& rt,
                                 const int32_t* seq_off, const Dims& dm, int n_seq, int row_blocks, int n_splits,
-                                float* scratch, int32_t* counters, unsigned long long* dbg, cudaStream_t st);
+                                float* scratch, int32_t* counters, unsigned long long* dbg, Chain* chain, cudaStream_t st);
 cudaError_t launch_swiglu(int dtype, const GemmOut& proj, void* out_t, int F, const int32_t* m_total, int m_max,
-                          cudaStream_t st);
+                          Chain* chain, cudaStream_t st);
 cudaError_t launch_argmax_rows(float* logits, const GemmOut& proj, int V, int32_t* out, const int32_t* out_index,
                                const int32_t* m_total, int m_max, cudaStream_t st);
 
