@@ -101,41 +101,66 @@ __global__ void __maxnreg__(88)
     const int i = threadIdx.x + k * NORM_THREADS;
     if (i < nvec) gn[k].load(gain + 4 * i);
   }
-  chain_wait_cta(cs);
   float4* xr = reinterpret_cast<float4*>(x + (size_t)m * d);
   const bool add = proj.raw != nullptr;   // x += the projection that ends the previous block (O or down)
-  // Decode-time launches have one row tile whatever the row count: the row's loads then do not wait for the
-  // row count (rows past it exist in memory and are simply not written back).
-  const volatile int32_t* mt_ptr = m_total;
-  int M = -1, m_tiles = 1;
-  if (add && proj.m_tiles_max != 1) { M = *mt_ptr; m_tiles = gemm_m_tiles(proj, M); }
-  float4 v[NORM_MAXV];
-  GemmPending4<5> pend[NORM_MAXV];
-  float ss = 0.f;
-  // every load first (residual row, projection output, partial slots), then the arithmetic
+  // Decode-time launches (one row tile, no idle CTA in the projection): every address is worked out while
+  // waiting, and the row's loads do not wait for the row count (rows past it exist in memory and are
+  // simply not written back).
+  const bool fast = add && proj.m_tiles_max == 1 && (proj.partial == nullptr || proj.all_work);
+  const size_t stride = add ? gemm_slot_stride(proj) : 0;
+  GemmSrc src[NORM_MAXV];
+  if (fast) {
 #pragma unroll
-  for (int k = 0; k < NORM_MAXV; ++k) {
-    const int i = threadIdx.x + k * NORM_THREADS;
-    if (i < nvec) {
-      v[k] = __ldcg(xr + i);
-      if (add) pend[k] = gemm_issue4<5>(proj, m_tiles, m, 4 * i);
+    for (int k = 0; k < NORM_MAXV; ++k) {
+      const int i = threadIdx.x + k * NORM_THREADS;
+      if (i < nvec) { src[k] = gemm_src(proj, 1, m, 4 * i); gemm_src_pin(src[k]); }
     }
+    asm volatile("" : "+l"(xr));
   }
-  if (M < 0) M = *mt_ptr;
-  if (m >= M) {
-    chain_exit(cs);
-    return;
-  }
+  chain_wait_cta(cs);
+  float4 v[NORM_MAXV];
+  float ss = 0.f;
+  if (fast) {
+    GemmData4<5> dat[NORM_MAXV];
+    const int M = *(const volatile int32_t*)m_total;
 #pragma unroll
-  for (int k = 0; k < NORM_MAXV; ++k) {
-    const int i = threadIdx.x + k * NORM_THREADS;
-    if (i < nvec) {
-      if (add) {
-        const float4 q = gemm_finish4(proj, m_tiles, pend[k]);
+    for (int k = 0; k < NORM_MAXV; ++k) {
+      const int i = threadIdx.x + k * NORM_THREADS;
+      if (i < nvec) { v[k] = __ldcg(xr + i); dat[k] = gemm_load4<5>(src[k], stride); }
+    }
+    if (m >= M) {
+      chain_exit(cs);
+      return;
+    }
+#pragma unroll
+    for (int k = 0; k < NORM_MAXV; ++k) {
+      const int i = threadIdx.x + k * NORM_THREADS;
+      if (i < nvec) {
+        const float4 q = gemm_sum4(src[k], stride, dat[k]);
         v[k].x += q.x; v[k].y += q.y; v[k].z += q.z; v[k].w += q.w;
         xr[i] = v[k];
+        ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
       }
-      ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
+    }
+  } else {
+    const int M = *m_total;
+    if (m >= M) {
+      chain_exit(cs);
+      return;
+    }
+    const int m_tiles = add ? gemm_m_tiles(proj, M) : 1;
+#pragma unroll
+    for (int k = 0; k < NORM_MAXV; ++k) {
+      const int i = threadIdx.x + k * NORM_THREADS;
+      if (i < nvec) {
+        v[k] = xr[i];
+        if (add) {
+          const float4 q = gemm_value4<5>(proj, m_tiles, m, 4 * i);
+          v[k].x += q.x; v[k].y += q.y; v[k].z += q.z; v[k].w += q.w;
+          xr[i] = v[k];
+        }
+        ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
+      }
     }
   }
   ss = block_sum(ss, sh);
@@ -196,43 +221,98 @@ cudaError_t launch_rope_table(const int32_t* pos, float* table, int hd, float th
 // ---------------------------------------------------------------- rotary embedding + KV write
 // qkv: [M][3d] fp32 (Q | K | V).  Q is rotated in place; rotated K and V go to the cache slot of
 // the row.  Pairing (i, i + hd/2).
-constexpr int ROPE_SPLIT = 8;  // CTAs per row
+// One thread per pair of adjacent rotary indices (i, i+1) of one head: it reads Q, K, V at columns i, i+1
+// and i+hd/2, i+hd/2+1 (one tile of the projection, one fold), all in a single batch of loads issued right
+// after the wait, together with the row's table entries -- one L2 round trip for the whole kernel.
+// What bounds the kernel is how fast ONE SM can pull its share out of the L2 (a few tens of GB/s), so the
+// rows are spread over as many SMs as possible: 256-thread CTAs, several per row, at no more than 88
+// registers so that they are all resident beside the projection that runs before them.
+constexpr int ROPE_THREADS = 256;
+constexpr int ROPE_FOLD = 2;   // partial slots loaded up front: a QKV tile (64+ k-blocks) is rarely cut in more than three
+
+__device__ __forceinline__ void store2(float* p, float a, float b) { *reinterpret_cast<float2*>(p) = make_float2(a, b); }
+__device__ __forceinline__ void store2(__nv_bfloat16* p, float a, float b) {
+  *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(a, b);
+}
 
 template <typename T>
-__global__ void rope_kv_kernel(float* __restrict__ qkv, GemmOut proj, T* __restrict__ kc, T* __restrict__ vc,
-                               const float2* __restrict__ table, RowTables rt, Dims dm, int* status, ChainSync cs) {
-  chain_enter(cs);
+__global__ void __maxnreg__(88) rope_kv_kernel(float* __restrict__ qkv, GemmOut proj, T* __restrict__ kc, T* __restrict__ vc,
+                                               const float2* __restrict__ table, RowTables rt, Dims dm, int* status,
+                                               ChainSync cs) {
+  chain_begin(cs);
   const int m = blockIdx.x;
-  const int M = *rt.m_total;
-  if (m >= M) {
-    chain_exit(cs);
-    return;
-  }
-  const int b = rt.seq[m], slot = rt.slot[m];
   const int d = dm.d, hd = dm.hd, half = hd >> 1;
-  const bool slot_ok = slot >= 0 && slot < dm.max_ctx;
-  if (!slot_ok && threadIdx.x == 0 && blockIdx.y == 0) atomicOr(status, DEV_ERR_CAPACITY);
-  const int m_tiles = gemm_m_tiles(proj, M);
+  const int n_items = dm.H * (half >> 1);
+  const int idx = blockIdx.y * ROPE_THREADS + threadIdx.x;   // the grid covers every item of the row once
+  const bool active = idx < n_items;
+  const int h = idx / (half >> 1), i = (idx - h * (half >> 1)) * 2;
+  const int o = h * hd + i;
   float* row = qkv + (size_t)m * 3 * d;
-  for (int idx = blockIdx.y * blockDim.x + threadIdx.x; idx < dm.H * half; idx += blockDim.x * gridDim.y) {
-    const int h = idx / half, i = idx - h * half;
-    const float2 cs = table[(size_t)m * half + i];
-    const float c = cs.x, s = cs.y;
-    const int o = h * hd + i;
-    const auto pq1 = gemm_issue<4>(proj, m_tiles, m, o), pq2 = gemm_issue<4>(proj, m_tiles, m, o + half);
-    const auto pk1 = gemm_issue<4>(proj, m_tiles, m, d + o), pk2 = gemm_issue<4>(proj, m_tiles, m, d + o + half);
-    const auto pv1 = gemm_issue<4>(proj, m_tiles, m, 2 * d + o), pv2 = gemm_issue<4>(proj, m_tiles, m, 2 * d + o + half);
-    const float q1 = gemm_finish(proj, m_tiles, pq1), q2 = gemm_finish(proj, m_tiles, pq2);
-    const float k1 = gemm_finish(proj, m_tiles, pk1), k2 = gemm_finish(proj, m_tiles, pk2);
-    const float v1 = gemm_finish(proj, m_tiles, pv1), v2 = gemm_finish(proj, m_tiles, pv2);
-    row[o] = q1 * c - q2 * s;            // the attention kernel reads the rotated Q from here
-    row[o + half] = q2 * c + q1 * s;
-    if (slot_ok) {
-      const size_t base = (((size_t)b * dm.H + h) * dm.max_ctx + slot) * hd + i;
-      kc[base] = from_f<T>(k1 * c - k2 * s);
-      kc[base + half] = from_f<T>(k2 * c + k1 * s);
-      vc[base] = from_f<T>(v1);
-      vc[base + half] = from_f<T>(v2);
+  // decode-time launches (one row tile, no idle CTA in the projection): every address is known before the
+  // projection has produced anything
+  const bool fast = proj.m_tiles_max == 1 && (proj.partial == nullptr || proj.all_work);
+  GemmSrc sq, sk, sv;
+  const size_t stride = gemm_slot_stride(proj);
+  const float2* tab = table + (size_t)m * half + i;
+  if (fast && active) {
+    sq = gemm_src(proj, 1, m, o); sk = gemm_src(proj, 1, m, d + o); sv = gemm_src(proj, 1, m, 2 * d + o);
+    gemm_src_pin(sq); gemm_src_pin(sk); gemm_src_pin(sv);
+    asm volatile("" : "+l"(tab), "+l"(row));
+  }
+  chain_wait_cta(cs);
+  if (fast) {
+    if (active) {
+      // one batch of loads (rows past the row count exist in memory), then the arithmetic
+      const int M = *(const volatile int32_t*)rt.m_total;
+      const int b = rt.seq[m], slot = rt.slot[m];
+      const float4 cs2 = *reinterpret_cast<const float4*>(tab);   // (cos, sin) of i and i+1
+      const auto dq1 = gemm_load2<ROPE_FOLD>(sq, stride), dq2 = gemm_load2<ROPE_FOLD>(sq, stride, half);
+      const auto dk1 = gemm_load2<ROPE_FOLD>(sk, stride), dk2 = gemm_load2<ROPE_FOLD>(sk, stride, half);
+      const auto dv1 = gemm_load2<ROPE_FOLD>(sv, stride), dv2 = gemm_load2<ROPE_FOLD>(sv, stride, half);
+      if (m < M) {
+        const bool slot_ok = slot >= 0 && slot < dm.max_ctx;
+        if (!slot_ok && idx == 0) atomicOr(status, DEV_ERR_CAPACITY);
+        const float2 q1 = gemm_sum2(sq, stride, dq1), q2 = gemm_sum2(sq, stride, dq2, half);
+        const float2 k1 = gemm_sum2(sk, stride, dk1), k2 = gemm_sum2(sk, stride, dk2, half);
+        const float2 v1 = gemm_sum2(sv, stride, dv1), v2 = gemm_sum2(sv, stride, dv2, half);
+        // the attention kernel reads the rotated Q from the projection's own buffer
+        store2(row + o, q1.x * cs2.x - q2.x * cs2.y, q1.y * cs2.z - q2.y * cs2.w);
+        store2(row + o + half, q2.x * cs2.x + q1.x * cs2.y, q2.y * cs2.z + q1.y * cs2.w);
+        if (slot_ok) {
+          const size_t base = (((size_t)b * dm.H + h) * dm.max_ctx + slot) * hd + i;
+          store2(kc + base, k1.x * cs2.x - k2.x * cs2.y, k1.y * cs2.z - k2.y * cs2.w);
+          store2(kc + base + half, k2.x * cs2.x + k1.x * cs2.y, k2.y * cs2.z + k1.y * cs2.w);
+          store2(vc + base, v1.x, v1.y);
+          store2(vc + base + half, v2.x, v2.y);
+        }
+      }
+    }
+  } else {
+    // prompt-sized launches (several row tiles) and projections shorter than the grid
+    const int M = *rt.m_total;
+    if (m < M && active) {
+      const int m_tiles = gemm_m_tiles(proj, M);
+      const int b = rt.seq[m], slot = rt.slot[m];
+      const bool slot_ok = slot >= 0 && slot < dm.max_ctx;
+      if (!slot_ok && idx == 0) atomicOr(status, DEV_ERR_CAPACITY);
+      const float4 cs2 = *reinterpret_cast<const float4*>(tab);
+      const GemmFold fq = gemm_fold_or_none(proj, m_tiles, m, o), fk = gemm_fold_or_none(proj, m_tiles, m, d + o),
+                     fv = gemm_fold_or_none(proj, m_tiles, m, 2 * d + o);
+      const auto pq1 = gemm_issue2<ROPE_FOLD>(proj, m_tiles, fq, m, o, 0), pq2 = gemm_issue2<ROPE_FOLD>(proj, m_tiles, fq, m, o + half, half);
+      const auto pk1 = gemm_issue2<ROPE_FOLD>(proj, m_tiles, fk, m, d + o, 0), pk2 = gemm_issue2<ROPE_FOLD>(proj, m_tiles, fk, m, d + o + half, half);
+      const auto pv1 = gemm_issue2<ROPE_FOLD>(proj, m_tiles, fv, m, 2 * d + o, 0), pv2 = gemm_issue2<ROPE_FOLD>(proj, m_tiles, fv, m, 2 * d + o + half, half);
+      const float2 q1 = gemm_finish2(proj, m_tiles, fq, 0, pq1), q2 = gemm_finish2(proj, m_tiles, fq, half, pq2);
+      const float2 k1 = gemm_finish2(proj, m_tiles, fk, 0, pk1), k2 = gemm_finish2(proj, m_tiles, fk, half, pk2);
+      const float2 v1 = gemm_finish2(proj, m_tiles, fv, 0, pv1), v2 = gemm_finish2(proj, m_tiles, fv, half, pv2);
+      store2(row + o, q1.x * cs2.x - q2.x * cs2.y, q1.y * cs2.z - q2.y * cs2.w);
+      store2(row + o + half, q2.x * cs2.x + q1.x * cs2.y, q2.y * cs2.z + q1.y * cs2.w);
+      if (slot_ok) {
+        const size_t base = (((size_t)b * dm.H + h) * dm.max_ctx + slot) * hd + i;
+        store2(kc + base, k1.x * cs2.x - k2.x * cs2.y, k1.y * cs2.z - k2.y * cs2.w);
+        store2(kc + base + half, k2.x * cs2.x + k1.x * cs2.y, k2.y * cs2.z + k1.y * cs2.w);
+        store2(vc + base, v1.x, v1.y);
+        store2(vc + base + half, v2.x, v2.y);
+      }
     }
   }
   chain_exit(cs);
@@ -240,27 +320,71 @@ __global__ void rope_kv_kernel(float* __restrict__ qkv, GemmOut proj, T* __restr
 
 cudaError_t launch_rope_kv(int dtype, float* qkv, const GemmOut& proj, void* kcache, void* vcache, const float* table,
                            const RowTables& rt, const Dims& dm, int m_max, int* status, Chain* chain, cudaStream_t st) {
-  dim3 grid(m_max, ROPE_SPLIT);
-  const ChainSync cs = chain ? chain->link((unsigned)m_max * ROPE_SPLIT, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
-  RD_DISPATCH(dtype, launch_pdl(rope_kv_kernel<T>, grid, 256, 0, st, qkv, proj, (T*)kcache, (T*)vcache,
+  const int n_items = dm.H * (dm.hd / 4);
+  dim3 grid(m_max, (n_items + ROPE_THREADS - 1) / ROPE_THREADS);
+  const ChainSync cs = chain ? chain->link(grid.x * grid.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
+  RD_DISPATCH(dtype, launch_pdl(rope_kv_kernel<T>, grid, ROPE_THREADS, 0, st, qkv, proj, (T*)kcache, (T*)vcache,
                                 reinterpret_cast<const float2*>(table), rt, dm, status, cs));
   return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------- SwiGLU
+// Two float4 items of the row per thread, every load of both issued before either is used.  Small CTAs
+// (128 threads), many per row: the kernel is bounded by the rate at which one SM pulls data out of the L2,
+// so the work is spread evenly over all SMs; at 88 registers they are all resident beside the gate|up
+// projection.
+constexpr int SWIGLU_THREADS = 128;
+constexpr int SWIGLU_ITEMS = 2;
+constexpr int SWIGLU_FOLD = 2;  // a gate|up tile is cut between two CTAs at most once the stream is longer than a tile per CTA
+
 template <typename T>
-__global__ void swiglu_kernel(GemmOut proj, T* __restrict__ out, int F, const int32_t* __restrict__ m_total, ChainSync cs) {
-  chain_enter(cs);
+__global__ void __maxnreg__(88) swiglu_kernel(GemmOut proj, T* __restrict__ out, int F, const int32_t* __restrict__ m_total,
+                                              ChainSync cs) {
+  chain_begin(cs);
   const int m = blockIdx.y;
-  const int M = *m_total;
-  const int f = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
-  if (m < M && f < F) {
-    const int m_tiles = gemm_m_tiles(proj, M);
-    const auto pg = gemm_issue4<4>(proj, m_tiles, m, f), pu = gemm_issue4<4>(proj, m_tiles, m, F + f);
-    const float4 g = gemm_finish4(proj, m_tiles, pg), u = gemm_finish4(proj, m_tiles, pu);
-    T* o = out + (size_t)m * F + f;
-    o[0] = from_f<T>(silu_f(g.x) * u.x); o[1] = from_f<T>(silu_f(g.y) * u.y);
-    o[2] = from_f<T>(silu_f(g.z) * u.z); o[3] = from_f<T>(silu_f(g.w) * u.w);
+  const bool fast = proj.m_tiles_max == 1 && (proj.partial == nullptr || proj.all_work);
+  const size_t stride = gemm_slot_stride(proj);
+  GemmSrc sg[SWIGLU_ITEMS], su[SWIGLU_ITEMS];
+  T* dst[SWIGLU_ITEMS];
+  bool act[SWIGLU_ITEMS];
+#pragma unroll
+  for (int k = 0; k < SWIGLU_ITEMS; ++k) {
+    const int f = ((blockIdx.x * SWIGLU_ITEMS + k) * SWIGLU_THREADS + threadIdx.x) * 4;
+    act[k] = f < F;
+    dst[k] = out + (size_t)m * F + f;
+    if (fast && act[k]) {
+      sg[k] = gemm_src(proj, 1, m, f); su[k] = gemm_src(proj, 1, m, F + f);
+      gemm_src_pin(sg[k]); gemm_src_pin(su[k]);
+      asm volatile("" : "+l"(dst[k]));
+    }
+  }
+  chain_wait_cta(cs);
+  if (fast) {
+    const int M = *(const volatile int32_t*)m_total;
+    GemmData4<SWIGLU_FOLD> dg[SWIGLU_ITEMS], du[SWIGLU_ITEMS];
+#pragma unroll
+    for (int k = 0; k < SWIGLU_ITEMS; ++k)
+      if (act[k]) { dg[k] = gemm_load4<SWIGLU_FOLD>(sg[k], stride); du[k] = gemm_load4<SWIGLU_FOLD>(su[k], stride); }
+    if (m < M) {
+#pragma unroll
+      for (int k = 0; k < SWIGLU_ITEMS; ++k)
+        if (act[k]) {
+          const float4 g = gemm_sum4(sg[k], stride, dg[k]), u = gemm_sum4(su[k], stride, du[k]);
+          store4(dst[k], silu_f(g.x) * u.x, silu_f(g.y) * u.y, silu_f(g.z) * u.z, silu_f(g.w) * u.w);
+        }
+    }
+  } else {
+    const int M = *m_total;
+    if (m < M) {
+      const int m_tiles = gemm_m_tiles(proj, M);
+      for (int k = 0; k < SWIGLU_ITEMS; ++k) {
+        const int f = ((blockIdx.x * SWIGLU_ITEMS + k) * SWIGLU_THREADS + threadIdx.x) * 4;
+        if (f < F) {
+          const float4 g = gemm_value4<SWIGLU_FOLD>(proj, m_tiles, m, f), u = gemm_value4<SWIGLU_FOLD>(proj, m_tiles, m, F + f);
+          store4(dst[k], silu_f(g.x) * u.x, silu_f(g.y) * u.y, silu_f(g.z) * u.z, silu_f(g.w) * u.w);
+        }
+      }
+    }
   }
   chain_exit(cs);
 }
@@ -268,9 +392,10 @@ __global__ void swiglu_kernel(GemmOut proj, T* __restrict__ out, int F, const in
 // proj: the gate|up projection [M][2F]; out: [M][F].  F must be a multiple of 4.
 cudaError_t launch_swiglu(int dtype, const GemmOut& proj, void* out_t, int F, const int32_t* m_total, int m_max,
                           Chain* chain, cudaStream_t st) {
-  dim3 grid((F / 4 + 255) / 256, m_max);
+  const int per_cta = SWIGLU_THREADS * SWIGLU_ITEMS * 4;
+  dim3 grid((F + per_cta - 1) / per_cta, m_max);
   const ChainSync cs = chain ? chain->link(grid.x * grid.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
-  RD_DISPATCH(dtype, launch_pdl(swiglu_kernel<T>, grid, 256, 0, st, proj, (T*)out_t, F, m_total, cs));
+  RD_DISPATCH(dtype, launch_pdl(swiglu_kernel<T>, grid, SWIGLU_THREADS, 0, st, proj, (T*)out_t, F, m_total, cs));
   return cudaGetLastError();
 }
 

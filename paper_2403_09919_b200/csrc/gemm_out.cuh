@@ -140,6 +140,129 @@ __device__ __forceinline__ float4 gemm_finish4(const GemmOut& g, int m_tiles, co
   return v;
 }
 
+// Two consecutive columns n, n+1 (n even) of row m, with the fold of a column of the same tile already
+// computed: `doff` is n minus the column the fold was made for.  Lets a kernel that reads several column
+// pairs of one tile (the two halves of a rotary pair) pay for the fold once.
+__device__ __forceinline__ GemmFold gemm_fold_or_none(const GemmOut& g, int m_tiles, int m, int n) {
+  GemmFold f;
+  f.c_next = 1; f.c_last = 0; f.off = 0;
+  if (g.partial != nullptr) f = gemm_fold(g, m_tiles, m, n);
+  return f;
+}
+template <int U>
+struct GemmPending2 {
+  float2 raw;
+  float2 q[U];
+};
+template <int U>
+__device__ __forceinline__ GemmPending2<U> gemm_issue2(const GemmOut& g, int m_tiles, const GemmFold& f, int m, int n, int doff) {
+  GemmPending2<U> p;
+  p.raw = __ldcg(reinterpret_cast<const float2*>(g.raw + (size_t)m * g.ld + n));
+  const size_t slot = (size_t)g.mt * 128;
+#pragma unroll
+  for (int j = 0; j < U; ++j) {
+    const int c = f.c_next + j;
+    p.q[j] = (c <= f.c_last && gemm_has_work(g, m_tiles, c))
+                 ? __ldcg(reinterpret_cast<const float2*>(g.partial + (size_t)c * slot + f.off + doff))
+                 : make_float2(0.f, 0.f);
+  }
+  return p;
+}
+template <int U>
+__device__ __forceinline__ float2 gemm_finish2(const GemmOut& g, int m_tiles, const GemmFold& f, int doff, const GemmPending2<U>& p) {
+  float2 v = p.raw;
+#pragma unroll
+  for (int j = 0; j < U; ++j) { v.x += p.q[j].x; v.y += p.q[j].y; }
+  const size_t slot = (size_t)g.mt * 128;
+  for (int c = f.c_next + U; c <= f.c_last; ++c) {
+    if (!gemm_has_work(g, m_tiles, c)) continue;
+    const float2 t = __ldcg(reinterpret_cast<const float2*>(g.partial + (size_t)c * slot + f.off + doff));
+    v.x += t.x; v.y += t.y;
+  }
+  return v;
+}
+
+// ---- addresses first, data later ---------------------------------------------------------------
+// The short kernels between two projections run once per layer with cold instruction caches, and what
+// they execute AFTER their predecessor has finished is the step's critical path.  Where a value lives
+// (output element, first partial slot, number of slots) depends only on launch constants, so a consumer
+// works it out while it is still waiting; afterwards it only loads and adds.
+struct GemmSrc {
+  const float* raw;    // &raw[m][n]
+  const float* part;   // the value's place in the first extra contributor's slot; slot j is at part + j * stride
+  int n_extra;         // contributors other than the first (0 when the tile is not cut or on the CUDA-core path)
+};
+__device__ __forceinline__ size_t gemm_slot_stride(const GemmOut& g) { return (size_t)g.mt * 128; }
+// Valid for launches where every CTA has work (all_work), which is every launch whose stream is at
+// least as long as the grid; callers fall back to gemm_value* otherwise.
+__device__ __forceinline__ GemmSrc gemm_src(const GemmOut& g, int m_tiles, int m, int n) {
+  GemmSrc s;
+  s.raw = g.raw + (size_t)m * g.ld + n;
+  s.part = g.partial;
+  s.n_extra = 0;
+  if (g.partial != nullptr) {
+    const GemmFold f = gemm_fold(g, m_tiles, m, n);
+    s.part = g.partial + (size_t)f.c_next * gemm_slot_stride(g) + f.off;
+    s.n_extra = f.c_last - f.c_next + 1;
+  }
+  return s;
+}
+// Keeps the compiler from sinking the address arithmetic below the wait.
+__device__ __forceinline__ void gemm_src_pin(GemmSrc& s) {
+  asm volatile("" : "+l"(s.raw), "+l"(s.part), "+r"(s.n_extra));
+}
+template <int U>
+struct GemmData4 {
+  float4 raw;
+  float4 q[U];
+};
+template <int U>
+struct GemmData2 {
+  float2 raw;
+  float2 q[U];
+};
+// `doff`: element offset from the column the source was made for (same tile, same row).
+template <int U>
+__device__ __forceinline__ GemmData4<U> gemm_load4(const GemmSrc& s, size_t stride, int doff = 0) {
+  GemmData4<U> p;
+  p.raw = __ldcg(reinterpret_cast<const float4*>(s.raw + doff));
+#pragma unroll
+  for (int j = 0; j < U; ++j)
+    p.q[j] = j < s.n_extra ? __ldcg(reinterpret_cast<const float4*>(s.part + j * stride + doff)) : make_float4(0.f, 0.f, 0.f, 0.f);
+  return p;
+}
+template <int U>
+__device__ __forceinline__ float4 gemm_sum4(const GemmSrc& s, size_t stride, const GemmData4<U>& p, int doff = 0) {
+  float4 v = p.raw;
+#pragma unroll
+  for (int j = 0; j < U; ++j) { v.x += p.q[j].x; v.y += p.q[j].y; v.z += p.q[j].z; v.w += p.q[j].w; }
+  for (int j = U; j < s.n_extra; ++j) {
+    const float4 t = __ldcg(reinterpret_cast<const float4*>(s.part + j * stride + doff));
+    v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
+  }
+  return v;
+}
+template <int U>
+__device__ __forceinline__ GemmData2<U> gemm_load2(const GemmSrc& s, size_t stride, int doff = 0) {
+  GemmData2<U> p;
+  p.raw = __ldcg(reinterpret_cast<const float2*>(s.raw + doff));
+#pragma unroll
+  for (int j = 0; j < U; ++j)
+    p.q[j] = j < s.n_extra ? __ldcg(reinterpret_cast<const float2*>(s.part + j * stride + doff)) : make_float2(0.f, 0.f);
+  return p;
+}
+template <int U>
+__device__ __forceinline__ float2 gemm_sum2(const GemmSrc& s, size_t stride, const GemmData2<U>& p, int doff = 0) {
+  float2 v = p.raw;
+#pragma unroll
+  for (int j = 0; j < U; ++j) { v.x += p.q[j].x; v.y += p.q[j].y; }
+  for (int j = U; j < s.n_extra; ++j) {
+    const float2 t = __ldcg(reinterpret_cast<const float2*>(s.part + j * stride + doff));
+    v.x += t.x; v.y += t.y;
+  }
+  return v;
+}
+
 // One-shot forms.
 __device__ __forceinline__ float gemm_value(const GemmOut& g, int m_tiles, int m, int n) {
   return gemm_finish(g, m_tiles, gemm_issue<GEMM_FOLD_UNROLL>(g, m_tiles, m, n));
