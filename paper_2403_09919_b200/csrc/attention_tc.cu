@@ -57,8 +57,12 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
                                                            int32_t* __restrict__ counters, unsigned long long* dbg, ChainSync cs) {
   unsigned long long t_dbg[6] = {0, 0, 0, 0, 0, 0};
   RD_STAMP(0);
-  chain_enter(cs);
-  RD_STAMP(1);
+  chain_begin(cs);
+  // Launched inside a chain, the kernel may read before its wait whatever the launches ahead of the chain
+  // wrote: the row tables, the tree mask and the cache entries of earlier steps.  Only Q and the K/V of
+  // this pass's own rows come from the kernel right before it.
+  const bool early = cs.signal_ptr != nullptr;
+  if (!early) chain_wait_cta(cs);
   constexpr int LD = HD + PAD;           // shared row stride in bf16
   constexpr int NT = HD / 8;             // output n-tiles
   constexpr int KS = HD / 16;            // k-steps of Q K^T
@@ -76,28 +80,17 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
   const int row0 = seq_row0 + rb * ROWS;
   const int nrows = min(ROWS, seq_rows - rb * ROWS);
   if (nrows <= 0) {  // the same for every split and head of this row tile
+    if (early) chain_wait_cta(cs);
     chain_exit(cs);
     return;
   }
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t4 = lane & 3;
   const int MW = dm.MW;
   const bool tree = rt.mask != nullptr;
-
-  // ---- round trip 2 (after seq_off): everything that only needs the tile's first row index is requested
-  // together -- raw Q (fp32), the rows' n_cache, the mask rows -- before any of it is used
   const int r_lo = g, r_hi = g + 8;
-  float2 qraw[KS][4];
-  {
-    const float* q_lo = qkv + (size_t)(row0 + (r_lo < nrows ? r_lo : 0)) * 3 * dm.d + h * HD + t4 * 2;
-    const float* q_hi = qkv + (size_t)(row0 + (r_hi < nrows ? r_hi : 0)) * 3 * dm.d + h * HD + t4 * 2;
-#pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
-      qraw[ks][0] = __ldcg(reinterpret_cast<const float2*>(q_lo + ks * 16));
-      qraw[ks][1] = __ldcg(reinterpret_cast<const float2*>(q_hi + ks * 16));
-      qraw[ks][2] = __ldcg(reinterpret_cast<const float2*>(q_lo + ks * 16 + 8));
-      qraw[ks][3] = __ldcg(reinterpret_cast<const float2*>(q_hi + ks * 16 + 8));
-    }
-  }
+
+  // ---- row tables and mask
+  const int nc_seq = rt.n_cache[seq_row0];   // first row of the sequence in this pass
   const int nc_first = rt.n_cache[row0], nc_last = rt.n_cache[row0 + nrows - 1];
   const int nc_mine = (tid < nrows) ? rt.n_cache[row0 + tid] : 0;
   if (tid < ROWS) s_ncache[tid] = nc_mine;
@@ -115,6 +108,9 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
   const int tree_base = nc_first;
   int kext = tree ? tree_base + seq_rows : nc_last;
   kext = min(kext, dm.max_ctx);
+  // keys below this index were written by earlier passes (tree: the context; causal: everything before the
+  // slot of the sequence's first row of this pass)
+  const int const_keys = tree ? tree_base : nc_seq - 1;
   const int n_chunks = (kext + KEYS - 1) / KEYS;
   const int c_begin = (int)((long long)z * n_chunks / n_splits), c_end = (int)((long long)(z + 1) * n_chunks / n_splits);
 
@@ -137,9 +133,30 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
-  // round trip 3: the first NSTAGE-1 chunks
+  // the first NSTAGE-1 chunks: those that hold only older keys start before the wait
+  int n_pre = 0;
+  if (early) {
+    while (n_pre < NSTAGE - 1 && (c_begin + n_pre + 1) * KEYS <= const_keys) {
+      load_chunk(c_begin + n_pre, n_pre);
+      ++n_pre;
+    }
+    chain_wait_cta(cs);
+  }
+  RD_STAMP(1);
+  // Q of the tile's rows (fp32, rotated by the preceding kernel)
+  float2 qraw[KS][4];
+  {
+    const float* q_lo = qkv + (size_t)(row0 + (r_lo < nrows ? r_lo : 0)) * 3 * dm.d + h * HD + t4 * 2;
+    const float* q_hi = qkv + (size_t)(row0 + (r_hi < nrows ? r_hi : 0)) * 3 * dm.d + h * HD + t4 * 2;
 #pragma unroll
-  for (int i = 0; i < NSTAGE - 1; ++i) load_chunk(c_begin + i, i);
+    for (int ks = 0; ks < KS; ++ks) {
+      qraw[ks][0] = __ldcg(reinterpret_cast<const float2*>(q_lo + ks * 16));
+      qraw[ks][1] = __ldcg(reinterpret_cast<const float2*>(q_hi + ks * 16));
+      qraw[ks][2] = __ldcg(reinterpret_cast<const float2*>(q_lo + ks * 16 + 8));
+      qraw[ks][3] = __ldcg(reinterpret_cast<const float2*>(q_hi + ks * 16 + 8));
+    }
+  }
+  for (int i = n_pre; i < NSTAGE - 1; ++i) load_chunk(c_begin + i, i);
 
   uint32_t qf[KS][4];
 #pragma unroll
@@ -293,7 +310,7 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
   }
   RD_STAMP(4);
   if (n_splits == 1) {
-    if (dbg && tid == 0 && blk == 0) { for (int i = 0; i < 5; ++i) dbg[i] = t_dbg[i]; dbg[6] = t_dbg[4]; }
+    if (dbg && tid == 0) { if (blk == 0) { for (int i = 0; i < 5; ++i) dbg[i] = t_dbg[i]; } atomicMax(dbg + 6, t_dbg[4]); }
     chain_exit(cs);
     return;
   }

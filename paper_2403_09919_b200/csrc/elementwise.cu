@@ -92,6 +92,9 @@ __global__ void __maxnreg__(88)
                    float* __restrict__ out_f, int d, float eps, const int32_t* __restrict__ m_total, ChainSync cs) {
   chain_begin(cs);
   __shared__ float sh[32];
+  // The first launch of a chain is ordered after everything before it; the later ones may read the row
+  // count (written ahead of the chain) before their wait.
+  const bool early = cs.signal_ptr != nullptr && cs.wait_ptr != nullptr;
   const int m = blockIdx.x;
   const int nvec = d >> 2;
   // the gain is a weight: requested before the wait, it has arrived when the row has
@@ -117,20 +120,21 @@ __global__ void __maxnreg__(88)
     }
     asm volatile("" : "+l"(xr));
   }
+  int M = early ? *m_total : 0;
   chain_wait_cta(cs);
+  if (!early) M = *m_total;
   float4 v[NORM_MAXV];
   float ss = 0.f;
   if (fast) {
     GemmData4<5> dat[NORM_MAXV];
-    const int M = *(const volatile int32_t*)m_total;
+    if (m >= M) {
+      chain_exit(cs);
+      return;
+    }
 #pragma unroll
     for (int k = 0; k < NORM_MAXV; ++k) {
       const int i = threadIdx.x + k * NORM_THREADS;
       if (i < nvec) { v[k] = __ldcg(xr + i); dat[k] = gemm_load4<5>(src[k], stride); }
-    }
-    if (m >= M) {
-      chain_exit(cs);
-      return;
     }
 #pragma unroll
     for (int k = 0; k < NORM_MAXV; ++k) {
@@ -143,7 +147,6 @@ __global__ void __maxnreg__(88)
       }
     }
   } else {
-    const int M = *m_total;
     if (m >= M) {
       chain_exit(cs);
       return;
@@ -185,12 +188,20 @@ cudaError_t launch_rmsnorm(int dtype, float* x, const GemmOut* proj, const void*
   if (d > 4 * NORM_THREADS * 4 || (d & 3)) return cudaErrorInvalidValue;
   GemmOut g{};
   if (proj) g = *proj;
+  // the first launch of a chain starts after everything before it has completed (see launch_ordered)
+  const bool first = chain && chain->enabled && chain->prev_ptr == nullptr;
   const ChainSync cs = chain ? chain->link((unsigned)m_max, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
+#define RD_NORM_LAUNCH(MAXV)                                                                                              \
+  RD_DISPATCH(dtype, if (first) launch_ordered(rmsnorm_kernel<T, MAXV>, m_max, NORM_THREADS, 0, st, x, g, (const T*)gain,  \
+                                               (T*)out_t, out_f32, d, eps, m_total, cs);                                  \
+              else launch_pdl(rmsnorm_kernel<T, MAXV>, m_max, NORM_THREADS, 0, st, x, g, (const T*)gain, (T*)out_t,        \
+                              out_f32, d, eps, m_total, cs))
   if (d <= 4 * NORM_THREADS * 2) {
-    RD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 2>, m_max, NORM_THREADS, 0, st, x, g, (const T*)gain, (T*)out_t, out_f32, d, eps, m_total, cs));
+    RD_NORM_LAUNCH(2);
   } else {
-    RD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 4>, m_max, NORM_THREADS, 0, st, x, g, (const T*)gain, (T*)out_t, out_f32, d, eps, m_total, cs));
+    RD_NORM_LAUNCH(4);
   }
+#undef RD_NORM_LAUNCH
   return cudaGetLastError();
 }
 
@@ -240,6 +251,9 @@ __global__ void __maxnreg__(88) rope_kv_kernel(float* __restrict__ qkv, GemmOut 
                                                const float2* __restrict__ table, RowTables rt, Dims dm, int* status,
                                                ChainSync cs) {
   chain_begin(cs);
+  // inside a chain the row tables and the rotary table (written ahead of the chain) may be read before the wait
+  const bool early = cs.signal_ptr != nullptr;
+  if (!early) chain_wait_cta(cs);
   const int m = blockIdx.x;
   const int d = dm.d, hd = dm.hd, half = hd >> 1;
   const int n_items = dm.H * (half >> 1);
@@ -259,17 +273,20 @@ __global__ void __maxnreg__(88) rope_kv_kernel(float* __restrict__ qkv, GemmOut 
     gemm_src_pin(sq); gemm_src_pin(sk); gemm_src_pin(sv);
     asm volatile("" : "+l"(tab), "+l"(row));
   }
-  chain_wait_cta(cs);
+  int M = 0, b = 0, slot = 0;
+  float4 cs2 = make_float4(0.f, 0.f, 0.f, 0.f);   // (cos, sin) of i and i+1
+  if (fast && active) {
+    M = *rt.m_total; b = rt.seq[m]; slot = rt.slot[m];
+    cs2 = *reinterpret_cast<const float4*>(tab);
+  }
+  if (early) chain_wait_cta(cs);
   if (fast) {
-    if (active) {
-      // one batch of loads (rows past the row count exist in memory), then the arithmetic
-      const int M = *(const volatile int32_t*)rt.m_total;
-      const int b = rt.seq[m], slot = rt.slot[m];
-      const float4 cs2 = *reinterpret_cast<const float4*>(tab);   // (cos, sin) of i and i+1
+    if (active && m < M) {
+      // one batch of loads, then the arithmetic
       const auto dq1 = gemm_load2<ROPE_FOLD>(sq, stride), dq2 = gemm_load2<ROPE_FOLD>(sq, stride, half);
       const auto dk1 = gemm_load2<ROPE_FOLD>(sk, stride), dk2 = gemm_load2<ROPE_FOLD>(sk, stride, half);
       const auto dv1 = gemm_load2<ROPE_FOLD>(sv, stride), dv2 = gemm_load2<ROPE_FOLD>(sv, stride, half);
-      if (m < M) {
+      {
         const bool slot_ok = slot >= 0 && slot < dm.max_ctx;
         if (!slot_ok && idx == 0) atomicOr(status, DEV_ERR_CAPACITY);
         const float2 q1 = gemm_sum2(sq, stride, dq1), q2 = gemm_sum2(sq, stride, dq2, half);
@@ -289,13 +306,13 @@ __global__ void __maxnreg__(88) rope_kv_kernel(float* __restrict__ qkv, GemmOut 
     }
   } else {
     // prompt-sized launches (several row tiles) and projections shorter than the grid
-    const int M = *rt.m_total;
+    M = *rt.m_total;
     if (m < M && active) {
       const int m_tiles = gemm_m_tiles(proj, M);
-      const int b = rt.seq[m], slot = rt.slot[m];
+      b = rt.seq[m]; slot = rt.slot[m];
       const bool slot_ok = slot >= 0 && slot < dm.max_ctx;
       if (!slot_ok && idx == 0) atomicOr(status, DEV_ERR_CAPACITY);
-      const float4 cs2 = *reinterpret_cast<const float4*>(tab);
+      cs2 = *reinterpret_cast<const float4*>(tab);
       const GemmFold fq = gemm_fold_or_none(proj, m_tiles, m, o), fk = gemm_fold_or_none(proj, m_tiles, m, d + o),
                      fv = gemm_fold_or_none(proj, m_tiles, m, 2 * d + o);
       const auto pq1 = gemm_issue2<ROPE_FOLD>(proj, m_tiles, fq, m, o, 0), pq2 = gemm_issue2<ROPE_FOLD>(proj, m_tiles, fq, m, o + half, half);
@@ -341,9 +358,12 @@ template <typename T>
 __global__ void __maxnreg__(88) swiglu_kernel(GemmOut proj, T* __restrict__ out, int F, const int32_t* __restrict__ m_total,
                                               ChainSync cs) {
   chain_begin(cs);
+  const bool early = cs.signal_ptr != nullptr;   // inside a chain the row count (written ahead of it) may be read now
+  if (!early) chain_wait_cta(cs);
   const int m = blockIdx.y;
   const bool fast = proj.m_tiles_max == 1 && (proj.partial == nullptr || proj.all_work);
   const size_t stride = gemm_slot_stride(proj);
+  const int M = *m_total;
   GemmSrc sg[SWIGLU_ITEMS], su[SWIGLU_ITEMS];
   T* dst[SWIGLU_ITEMS];
   bool act[SWIGLU_ITEMS];
@@ -358,14 +378,13 @@ __global__ void __maxnreg__(88) swiglu_kernel(GemmOut proj, T* __restrict__ out,
       asm volatile("" : "+l"(dst[k]));
     }
   }
-  chain_wait_cta(cs);
+  if (early) chain_wait_cta(cs);
   if (fast) {
-    const int M = *(const volatile int32_t*)m_total;
-    GemmData4<SWIGLU_FOLD> dg[SWIGLU_ITEMS], du[SWIGLU_ITEMS];
-#pragma unroll
-    for (int k = 0; k < SWIGLU_ITEMS; ++k)
-      if (act[k]) { dg[k] = gemm_load4<SWIGLU_FOLD>(sg[k], stride); du[k] = gemm_load4<SWIGLU_FOLD>(su[k], stride); }
     if (m < M) {
+      GemmData4<SWIGLU_FOLD> dg[SWIGLU_ITEMS], du[SWIGLU_ITEMS];
+#pragma unroll
+      for (int k = 0; k < SWIGLU_ITEMS; ++k)
+        if (act[k]) { dg[k] = gemm_load4<SWIGLU_FOLD>(sg[k], stride); du[k] = gemm_load4<SWIGLU_FOLD>(su[k], stride); }
 #pragma unroll
       for (int k = 0; k < SWIGLU_ITEMS; ++k)
         if (act[k]) {
@@ -374,7 +393,6 @@ __global__ void __maxnreg__(88) swiglu_kernel(GemmOut proj, T* __restrict__ out,
         }
     }
   } else {
-    const int M = *m_total;
     if (m < M) {
       const int m_tiles = gemm_m_tiles(proj, M);
       for (int k = 0; k < SWIGLU_ITEMS; ++k) {
