@@ -358,6 +358,9 @@ int do_draft(rd_handle* h, cudaStream_t st, int32_t* beams, float* scores) {
   float *sc_in = w.score_a, *sc_out = w.score_b;
   int32_t *hi_in = w.hist_a, *hi_out = w.hist_b;
   GemmOut g;
+  // the calls' launches hand over to each other through counters (tensor-core path)
+  Chain* ch = h->use_tc ? &h->chain : nullptr;
+  h->chain.cut();
   for (int call = 1; call <= dm.L; ++call) {
     const int rows = call == 1 ? B : R;
     const int32_t* mt = call == 1 ? w.one_b : w.one_r;
@@ -365,26 +368,27 @@ int do_draft(rd_handle* h, cudaStream_t st, int32_t* beams, float* scores) {
     const float* xin_f = call == 1 ? w.xc_f : w.x0_f;
     if (call > 1) {
       // s_t = SiLU([U W][s_{t-1}; e_t] + b), written into the first d_rnn columns of x0 = [s_t, h]
-      int rc = gemm(h, w.se_t, dm.dr + dm.d, w.uw, dm.dr, dm.dr + dm.d, mt, rows, w.sraw, dm.dr, &g, nullptr, st);
+      int rc = gemm(h, w.se_t, dm.dr + dm.d, w.uw, dm.dr, dm.dr + dm.d, mt, rows, w.sraw, dm.dr, &g, ch, st);
       if (rc) return rc;
-      CKP(h, PROF_DRAFT_SMALL, launch_act(dm.dtype, g, h->w.rnn_b, nullptr, 0, w.x0_f, w.x0_t, dm.dh, dm.dr, mt, rows, st));
+      CKP(h, PROF_DRAFT_SMALL, launch_act(dm.dtype, g, h->w.rnn_b, nullptr, 0, w.x0_f, w.x0_t, dm.dh, dm.dr, mt, rows, ch, st));
     }
     for (int l = 0; l < dm.n_head_layers; ++l) {
       float* of = (l & 1) ? w.x2_f : w.x1_f;
       void* ot = (l & 1) ? w.x2_t : w.x1_t;
-      int rc = gemm(h, xin_t, dm.dh, h->head_w[l], dm.dh, dm.dh, mt, rows, w.hraw, dm.dh, &g, nullptr, st);
+      int rc = gemm(h, xin_t, dm.dh, h->head_w[l], dm.dh, dm.dh, mt, rows, w.hraw, dm.dh, &g, ch, st);
       if (rc) return rc;
-      CKP(h, PROF_DRAFT_SMALL, launch_act(dm.dtype, g, h->head_b[l], xin_f, dm.dh, of, ot, dm.dh, dm.dh, mt, rows, st));
+      CKP(h, PROF_DRAFT_SMALL, launch_act(dm.dtype, g, h->head_b[l], xin_f, dm.dh, of, ot, dm.dh, dm.dh, mt, rows, ch, st));
       xin_t = ot; xin_f = of;
     }
-    int rc = gemm(h, xin_t, dm.dh, h->w.draft_out, dm.V, dm.dh, mt, rows, w.dlogits, dm.V, &g, nullptr, st);
+    int rc = gemm(h, xin_t, dm.dh, h->w.draft_out, dm.V, dm.dh, mt, rows, w.dlogits, dm.V, &g, ch, st);
     if (rc) return rc;
     CKP(h, PROF_DRAFT_SMALL, launch_draft_select(dm.dtype, g, call, w.lse, w.cand_val, w.cand_idx, sc_in, sc_out, hi_in, hi_out,
                                                  h->w.tok_emb, w.x0_f, dm.dh, w.se_t, dm, B, beams, scores, w.sel_counters, mt,
-                                                 (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) ? w.trace + (size_t)8 * h->trace_next++ : nullptr, st));
+                                                 (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) ? w.trace + (size_t)8 * h->trace_next++ : nullptr, ch, st));
     float* tf = sc_in; sc_in = sc_out; sc_out = tf;
     int32_t* ti = hi_in; hi_in = hi_out; hi_out = ti;
   }
+  h->chain.cut();
   return RD_OK;
 }
 

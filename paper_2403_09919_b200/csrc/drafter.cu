@@ -71,32 +71,77 @@ cudaError_t launch_fill_h(int dtype, const float* h, void* x_t, float* x_f, cons
 // out[m][n] = (resid ? resid[m][n] : 0) + SiLU(proj[m][n] + bias[n]), written as fp32 and in the
 // storage type (the next projection's input).  Used for the RNN cell (no residual) and for the
 // head's residual layers.
-template <typename T>
-__global__ void act_kernel(GemmOut proj, const T* __restrict__ bias, const float* __restrict__ resid, int ld_resid,
-                           float* __restrict__ out_f, T* __restrict__ out_t, int ld_out, int N,
-                           const int32_t* __restrict__ m_total) {
-  pdl_enter();
-  const int m = blockIdx.y;
-  const int M = *m_total;
-  if (m >= M) return;
-  const int n = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
-  if (n >= N) return;
-  const float4 q = gemm_value4(proj, gemm_m_tiles(proj, M), m, n);
-  float v[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    v[k] = silu_f(v[k] + to_f<T>(bias[n + k]));
-    if (resid) v[k] += resid[(size_t)m * ld_resid + n + k];
-    out_f[(size_t)m * ld_out + n + k] = v[k];
-    out_t[(size_t)m * ld_out + n + k] = from_f<T>(v[k]);
-  }
+constexpr int ACT_THREADS = 128;
+constexpr int ACT_FOLD = 5;   // partial slots loaded up front (a 128-k-block tile cut over 28-unit ranges has up to 5 extra)
+
+__device__ __forceinline__ void act_store4(float* p, float a, float b, float c, float d) { *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d); }
+__device__ __forceinline__ void act_store4(__nv_bfloat16* p, float a, float b, float c, float d) {
+  const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+  uint2 u;
+  u.x = *reinterpret_cast<const uint32_t*>(&lo);
+  u.y = *reinterpret_cast<const uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(p) = u;
+}
+template <typename T> __device__ __forceinline__ float4 act_bias4(const T* p);
+template <> __device__ __forceinline__ float4 act_bias4<float>(const float* p) { return *reinterpret_cast<const float4*>(p); }
+template <> __device__ __forceinline__ float4 act_bias4<__nv_bfloat16>(const __nv_bfloat16* p) {
+  const uint2 g = *reinterpret_cast<const uint2*>(p);
+  const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&g.x));
+  const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&g.y));
+  return make_float4(a.x, a.y, b.x, b.y);
 }
 
+// One float4 of one row per thread, small CTAs spread over all SMs (what bounds the kernel is the rate at
+// which one SM pulls data out of the L2).  The bias is a weight and every address is a launch constant: both
+// are dealt with before the wait; after it the thread loads, adds and stores.
+template <typename T>
+__global__ void __maxnreg__(88) act_kernel(GemmOut proj, const T* __restrict__ bias, const float* resid, int ld_resid,
+                                           float* __restrict__ out_f, T* __restrict__ out_t, int ld_out, int N,
+                                           const int32_t* __restrict__ m_total, ChainSync cs) {
+  chain_begin(cs);
+  const int m = blockIdx.y;
+  const int n = (blockIdx.x * ACT_THREADS + threadIdx.x) * 4;
+  const bool active = n < N;
+  const bool fast = proj.m_tiles_max == 1 && (proj.partial == nullptr || proj.all_work);
+  const size_t stride = gemm_slot_stride(proj);
+  GemmSrc src;
+  float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+  const float* rp = resid ? resid + (size_t)m * ld_resid + n : nullptr;
+  float* of = out_f + (size_t)m * ld_out + n;
+  T* ot = out_t + (size_t)m * ld_out + n;
+  if (active) {
+    bv = act_bias4<T>(bias + n);
+    if (fast) { src = gemm_src(proj, 1, m, n); gemm_src_pin(src); }
+    asm volatile("" : "+l"(rp), "+l"(of), "+l"(ot));
+  }
+  chain_wait_cta(cs);
+  const int M = *m_total;
+  if (m < M && active) {
+    float4 q;
+    float4 rv = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (fast) {
+      const auto dat = gemm_load4<ACT_FOLD>(src, stride);
+      if (rp) rv = __ldcg(reinterpret_cast<const float4*>(rp));
+      q = gemm_sum4(src, stride, dat);
+    } else {
+      if (rp) rv = __ldcg(reinterpret_cast<const float4*>(rp));
+      q = gemm_value4(proj, gemm_m_tiles(proj, M), m, n);
+    }
+    const float y0 = rv.x + silu_f(q.x + bv.x), y1 = rv.y + silu_f(q.y + bv.y), y2 = rv.z + silu_f(q.z + bv.z),
+                y3 = rv.w + silu_f(q.w + bv.w);
+    act_store4(of, y0, y1, y2, y3);
+    act_store4(ot, y0, y1, y2, y3);
+  }
+  chain_exit(cs);
+}
+
+// N, ld_resid, ld_out multiples of 4 (8 for bf16 outputs); bias 16-byte aligned.
 cudaError_t launch_act(int dtype, const GemmOut& proj, const void* bias, const float* resid, int ld_resid, float* out_f,
-                       void* out_t, int ld_out, int N, const int32_t* m_total, int m_max, cudaStream_t st) {
-  dim3 grid((N / 4 + 255) / 256, m_max);
-  RD_DISPATCH(dtype, launch_pdl(act_kernel<T>, grid, 256, 0, st, proj, (const T*)bias, resid, ld_resid, out_f, (T*)out_t,
-                                ld_out, N, m_total));
+                       void* out_t, int ld_out, int N, const int32_t* m_total, int m_max, Chain* chain, cudaStream_t st) {
+  dim3 grid((N / 4 + ACT_THREADS - 1) / ACT_THREADS, m_max);
+  const ChainSync cs = chain ? chain->link(grid.x * grid.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
+  RD_DISPATCH(dtype, launch_pdl(act_kernel<T>, grid, ACT_THREADS, 0, st, proj, (const T*)bias, resid, ld_resid, out_f,
+                                (T*)out_t, ld_out, N, m_total, cs));
   return cudaGetLastError();
 }
 
@@ -152,10 +197,10 @@ __global__ void __launch_bounds__(SEL_THREADS) draft_select_kernel(
     const float* __restrict__ score_in, float* __restrict__ score_out, const int32_t* __restrict__ hist_in,
     int32_t* __restrict__ hist_out, const T* __restrict__ emb, const float* __restrict__ s_new_f, int ld_s,
     T* __restrict__ se_t, Dims dm, int32_t* __restrict__ beams_out, float* __restrict__ scores_out,
-    int32_t* __restrict__ counters, const int32_t* __restrict__ m_total, unsigned long long* dbg) {
+    int32_t* __restrict__ counters, const int32_t* __restrict__ m_total, unsigned long long* dbg, ChainSync cs) {
   unsigned long long t_dbg[8];
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[0]));
-  pdl_enter();
+  chain_enter(cs);
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[1]));
   extern __shared__ __align__(16) uint8_t sel_smem[];
   Cand* wl = reinterpret_cast<Cand*>(sel_smem);            // [32 warps][BW] per-warp survivors; reused by the pruning
@@ -294,7 +339,10 @@ __global__ void __launch_bounds__(SEL_THREADS) draft_select_kernel(
   }
   __syncthreads();
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[5]));
-  if (!s_last) return;
+  if (!s_last) {
+    chain_exit(cs);
+    return;
+  }
   __threadfence();
   const int n_cand = rows * BW;
   // candidates into shared memory: score and flat index
@@ -356,6 +404,7 @@ __global__ void __launch_bounds__(SEL_THREADS) draft_select_kernel(
   if (dbg && threadIdx.x == 0) {
     for (int i = 0; i < 7; ++i) dbg[i] = t_dbg[i];
   }
+  chain_exit(cs);
 }
 
 // rows = B (call 1) or B * BW.  counters: [B] zero between launches.
@@ -363,7 +412,7 @@ cudaError_t launch_draft_select(int dtype, const GemmOut& proj, int call, float*
                                 const float* score_in, float* score_out, const int32_t* hist_in, int32_t* hist_out,
                                 const void* emb, const float* s_new_f, int ld_s, void* se_t, const Dims& dm, int B,
                                 int32_t* beams_out, float* scores_out, int32_t* counters, const int32_t* m_total,
-                                unsigned long long* dbg, cudaStream_t st) {
+                                unsigned long long* dbg, Chain* chain, cudaStream_t st) {
   if (dm.BW > SEL_MAX_BW) return cudaErrorInvalidValue;
   const int rows = call == 1 ? B : B * dm.BW;
   const size_t select = ((size_t)32 * dm.BW + SEL_LIST_CAP) * sizeof(Cand) + (size_t)dm.V * sizeof(float);
@@ -378,9 +427,10 @@ cudaError_t launch_draft_select(int dtype, const GemmOut& proj, int call, float*
     if (e != cudaSuccess) return e;
     attr_set[dtype == RD_DTYPE_FP32 ? 0 : 1] = true;
   }
+  const ChainSync cs = chain ? chain->link((unsigned)rows) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
   RD_DISPATCH(dtype, launch_pdl(draft_select_kernel<T>, rows, SEL_THREADS, smem, st, proj, call, lse, val, idx, score_in,
                                 score_out, hist_in, hist_out, (const T*)emb, s_new_f, ld_s, (T*)se_t, dm, beams_out,
-                                scores_out, counters, m_total, dbg));
+                                scores_out, counters, m_total, dbg, cs));
   return cudaGetLastError();
 }
 

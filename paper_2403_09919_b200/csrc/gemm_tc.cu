@@ -432,9 +432,14 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* map_a, int N, int K, c
   while (cols < 2 * p.mt) cols <<= 1;
   p.tmem_cols = cols;
   p.m_total = m_total; p.raw = raw; p.ld_raw = ld_raw; p.partial = partial; p.status = status; p.trace = trace;
+  // the first launch of a chain starts after everything before it has completed (see launch_ordered)
+  const bool first = chain && chain->enabled && chain->prev_ptr == nullptr;
   p.cs = chain ? chain->link((unsigned)grid) : ChainSync{nullptr, 0u, nullptr, status, nullptr};
   const size_t smem = (size_t)stages * stage_bytes + overhead;
-  launch_pdl(gemm_tc_kernel, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, *(const CUtensorMap*)map_a, p);
+  if (first)
+    launch_ordered(gemm_tc_kernel, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, *(const CUtensorMap*)map_a, p);
+  else
+    launch_pdl(gemm_tc_kernel, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, *(const CUtensorMap*)map_a, p);
   return cudaGetLastError();
 }
 
