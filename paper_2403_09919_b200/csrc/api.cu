@@ -46,6 +46,8 @@ struct Workspace {
   void *xc_t, *x0_t, *x1_t, *x2_t, *se_t, *uw;   // se_t: [R][d_rnn + d] = [s ; e]; uw: [d_rnn][d_rnn + d] = [U W]
   float *xc_f, *x0_f, *x1_f, *x2_f, *sraw, *hraw, *dlogits, *lse, *cand_val, *score_a, *score_b;
   int32_t *cand_idx, *hist_a, *hist_b, *one_b, *one_r;
+  float *seg_max, *seg_sum, *seg_val;   // two-kernel selection: per (row, segment) maximum, sum, candidates
+  int32_t* seg_idx;
   // tensor-core projection scratch
   float* tc_partial;
   // tensor-core attention scratch
@@ -194,6 +196,8 @@ void carve(Bump& bp, const Dims& dm, int m_cap, Workspace* w) {
   w->x1_f = bp.take<float>((size_t)R * dm.dh); w->x2_f = bp.take<float>((size_t)R * dm.dh);
   w->sraw = bp.take<float>((size_t)R * dm.dr); w->hraw = bp.take<float>((size_t)R * dm.dh);
   w->dlogits = bp.take<float>((size_t)R * dm.V);
+  w->seg_max = bp.take<float>((size_t)R * 32); w->seg_sum = bp.take<float>((size_t)R * 32);
+  w->seg_val = bp.take<float>((size_t)R * 512); w->seg_idx = bp.take<int32_t>((size_t)R * 512);
   w->lse = bp.take<float>(R); w->cand_val = bp.take<float>((size_t)R * dm.BW);
   w->score_a = bp.take<float>(R); w->score_b = bp.take<float>(R);
   w->cand_idx = bp.take<int32_t>((size_t)R * dm.BW); w->hist_a = bp.take<int32_t>((size_t)R * dm.L);
@@ -384,7 +388,9 @@ int do_draft(rd_handle* h, cudaStream_t st, int32_t* beams, float* scores) {
     if (rc) return rc;
     CKP(h, PROF_DRAFT_SMALL, launch_draft_select(dm.dtype, g, call, w.lse, w.cand_val, w.cand_idx, sc_in, sc_out, hi_in, hi_out,
                                                  h->w.tok_emb, w.x0_f, dm.dh, w.se_t, dm, B, beams, scores, w.sel_counters, mt,
-                                                 (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) ? w.trace + (size_t)8 * h->trace_next++ : nullptr, ch, st));
+                                                 (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) ? w.trace + (size_t)8 * h->trace_next++ : nullptr,
+                                                 SelectScratch{h->use_tc ? w.seg_max : nullptr, w.seg_sum, w.seg_val, w.seg_idx, h->tc_grid}, ch, st));
+    if (h->use_tc && draft_select_segments(dm, rows, h->tc_grid) > 0) h->launches++;   // that selection is two launches
     float* tf = sc_in; sc_in = sc_out; sc_out = tf;
     int32_t* ti = hi_in; hi_in = hi_out; hi_out = ti;
   }

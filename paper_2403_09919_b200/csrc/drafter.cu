@@ -407,14 +407,292 @@ __global__ void __launch_bounds__(SEL_THREADS) draft_select_kernel(
   chain_exit(cs);
 }
 
+// ---------------------------------------------------------------- selection in two short kernels (BW <= 32)
+// The one-CTA-per-row kernel above pulls a whole row of logits through one SM and ranks it there; with a
+// handful of rows that leaves most of the GPU idle for tens of microseconds.  Here every row is cut into S
+// segments (rows x S CTAs, about one per SM): a segment's CTA folds its logits, and reduces them to the
+// segment's maximum, its sum of exponentials and its BW best candidates.  A second kernel with one CTA per
+// surviving beam merges the segments of its sequence's rows (log-sum-exp, BW best per row), prunes the
+// BW x BW candidates in (score desc, flat index asc) order up to its own rank, and writes that beam's score,
+// history and next input row.  Both orders are the ones of the single-kernel path.
+// (value desc, index asc) as the unsigned order of one 64-bit key; 0 is below every candidate.
+__device__ __forceinline__ unsigned long long cand_key(float v, int i) {
+  uint32_t u = __float_as_uint(v);
+  u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  return ((unsigned long long)u << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)i);
+}
+__device__ __forceinline__ float key_value(unsigned long long k) {
+  if (k == 0ull) return -INFINITY;
+  const uint32_t u = (uint32_t)(k >> 32);
+  return __uint_as_float((u & 0x80000000u) ? (u ^ 0x80000000u) : ~u);
+}
+__device__ __forceinline__ int key_index(unsigned long long k) {
+  return k == 0ull ? 0x7fffffff : (int)(0xFFFFFFFFu - (uint32_t)(k & 0xFFFFFFFFull));
+}
+__device__ __forceinline__ unsigned long long warp_max_key(unsigned long long k) {
+  const uint32_t hi = (uint32_t)(k >> 32), lo = (uint32_t)k;
+  const uint32_t mh = __reduce_max_sync(0xffffffffu, hi);
+  const uint32_t ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
+  return ((unsigned long long)mh << 32) | ml;
+}
+
+constexpr int SEG_THREADS = 256;
+constexpr int SEG_ITEMS_MAX = 4;     // float4 per thread at most (the kernel is instantiated for 1, 2 and 4)
+constexpr int SEG_FOLD = 2;
+constexpr int SEG_MAX_CAND = 512;    // S * BW candidates per row at most
+constexpr int MRG_THREADS = 256;
+
+template <int SEG_ITEMS>
+__global__ void __maxnreg__(88) draft_seg_kernel(GemmOut proj, int V, int BW, int seg_len4, float* __restrict__ seg_max,
+                                                 float* __restrict__ seg_sum, float* __restrict__ seg_val,
+                                                 int32_t* __restrict__ seg_idx, const int32_t* __restrict__ m_total,
+                                                 ChainSync cs) {
+  chain_begin(cs);
+  __shared__ float shf[32];
+  __shared__ unsigned long long shk[2][SEG_THREADS / 32];
+  const int r = blockIdx.y, sgm = blockIdx.x, S = gridDim.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const bool fast = proj.m_tiles_max == 1 && (proj.partial == nullptr || proj.all_work);
+  const size_t stride = gemm_slot_stride(proj);
+  GemmSrc src[SEG_ITEMS];
+  int col[SEG_ITEMS];
+  bool ok[SEG_ITEMS];
+#pragma unroll
+  for (int k = 0; k < SEG_ITEMS; ++k) {
+    const int j = threadIdx.x + k * SEG_THREADS;
+    col[k] = 4 * (sgm * seg_len4 + j);
+    ok[k] = j < seg_len4 && col[k] < V;
+    if (fast && ok[k]) { src[k] = gemm_src(proj, 1, r, col[k]); gemm_src_pin(src[k]); }
+  }
+  chain_wait_cta(cs);
+  float v[SEG_ITEMS][4];
+  if (fast) {
+    GemmData4<SEG_FOLD> dat[SEG_ITEMS];
+#pragma unroll
+    for (int k = 0; k < SEG_ITEMS; ++k)
+      if (ok[k]) dat[k] = gemm_load4<SEG_FOLD>(src[k], stride);
+#pragma unroll
+    for (int k = 0; k < SEG_ITEMS; ++k) {
+      float4 q = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+      if (ok[k]) q = gemm_sum4(src[k], stride, dat[k]);
+      v[k][0] = q.x; v[k][1] = q.y; v[k][2] = q.z; v[k][3] = q.w;
+    }
+  } else {
+    const int m_tiles = gemm_m_tiles(proj, *m_total);
+#pragma unroll
+    for (int k = 0; k < SEG_ITEMS; ++k) {
+      float4 q = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+      if (ok[k]) q = gemm_value4<SEG_FOLD>(proj, m_tiles, r, col[k]);
+      v[k][0] = q.x; v[k][1] = q.y; v[k][2] = q.z; v[k][3] = q.w;
+    }
+  }
+  // ---- segment maximum and sum of exponentials
+  float tmax = -INFINITY;
+#pragma unroll
+  for (int k = 0; k < SEG_ITEMS; ++k)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) tmax = fmaxf(tmax, v[k][e]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+  if (lane == 0) shf[warp] = tmax;
+  __syncthreads();
+  float smax = lane < SEG_THREADS / 32 ? shf[lane] : -INFINITY;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) smax = fmaxf(smax, __shfl_xor_sync(0xffffffffu, smax, o));
+  float sum = 0.f;
+  if (smax > -INFINITY) {
+#pragma unroll
+    for (int k = 0; k < SEG_ITEMS; ++k)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) sum += __expf(v[k][e] - smax);   // exp(-inf) = 0 for the padding
+  }
+  sum = block_reduce_sum(sum, shf);
+  if (threadIdx.x == 0) { seg_max[(size_t)r * S + sgm] = smax; seg_sum[(size_t)r * S + sgm] = sum; }
+  // ---- the segment's BW best in (value desc, index asc) order.  Every candidate becomes one 64-bit key whose
+  // unsigned order is that order (ordered value bits, then the complemented index): keys are unique, so round
+  // p's winner is simply the largest key below round p-1's, and nothing is marked or removed.  One redux pair
+  // per warp, one barrier per round (the per-warp results alternate between two shared buffers).
+  unsigned long long key[SEG_ITEMS * 4];
+#pragma unroll
+  for (int k = 0; k < SEG_ITEMS; ++k)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) key[k * 4 + e] = ok[k] ? cand_key(v[k][e], col[k] + e) : 0ull;
+  unsigned long long prev = ~0ull;
+  for (int p = 0; p < BW; ++p) {
+    unsigned long long mine = 0ull;
+#pragma unroll
+    for (int q = 0; q < SEG_ITEMS * 4; ++q) mine = max(mine, key[q] < prev ? key[q] : 0ull);
+    mine = warp_max_key(mine);
+    if (lane == 0) shk[p & 1][warp] = mine;
+    __syncthreads();
+    unsigned long long best = 0ull;
+#pragma unroll
+    for (int w = 0; w < SEG_THREADS / 32; ++w) best = max(best, shk[p & 1][w]);
+    if (threadIdx.x == 0) {
+      seg_val[((size_t)r * S + sgm) * BW + p] = key_value(best);
+      seg_idx[((size_t)r * S + sgm) * BW + p] = key_index(best);
+    }
+    prev = best;
+  }
+  chain_exit(cs);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(MRG_THREADS) draft_merge_kernel(
+    int S, int call, const float* __restrict__ seg_max, const float* __restrict__ seg_sum, const float* __restrict__ seg_val,
+    const int32_t* __restrict__ seg_idx, const float* __restrict__ score_in, float* __restrict__ score_out,
+    const int32_t* __restrict__ hist_in, int32_t* __restrict__ hist_out, const T* __restrict__ emb,
+    const float* __restrict__ s_new_f, int ld_s, T* __restrict__ se_t, Dims dm, int32_t* __restrict__ beams_out,
+    float* __restrict__ scores_out, unsigned long long* dbg, ChainSync cs) {
+  unsigned long long t_dbg[4] = {0, 0, 0, 0};
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[0]));
+  chain_enter(cs);
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[1]));
+  __shared__ unsigned long long wbuf[MRG_THREADS / 32][SEG_MAX_CAND];
+  __shared__ unsigned long long top[32 * 32];
+  __shared__ Cand s_win;
+  const int BW = dm.BW, L = dm.L, V = dm.V;
+  const int kout = blockIdx.x, b = blockIdx.y;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int rows = call == 1 ? 1 : BW;
+  const int row0 = call == 1 ? b : b * BW;
+  const int n = S * BW;
+  for (int rr = warp; rr < rows; rr += MRG_THREADS / 32) {
+    const int r = row0 + rr;
+    // every load of the row first: segment maxima and sums (S <= 32: one per lane), candidates, the row's score
+    const float sm = lane < S ? __ldcg(seg_max + (size_t)r * S + lane) : -INFINITY;
+    const float ss = lane < S ? __ldcg(seg_sum + (size_t)r * S + lane) : 0.f;
+    const float base = call == 1 ? 0.f : __ldcg(score_in + r);
+    for (int c = lane; c < n; c += 32) {
+      const float cv = __ldcg(seg_val + (size_t)r * n + c);
+      const int ci = __ldcg(seg_idx + (size_t)r * n + c);
+      wbuf[warp][c] = ci == 0x7fffffff ? 0ull : cand_key(cv, ci);
+    }
+    // log-sum-exp of the row from its segments
+    float m = sm;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    float sum = sm > -INFINITY ? ss * __expf(sm - m) : 0.f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    const float row_lse = m + logf(sum);
+    __syncwarp();
+    unsigned long long pv = ~0ull;
+    for (int p = 0; p < BW; ++p) {
+      unsigned long long mine = 0ull;
+      for (int c = lane; c < n; c += 32) {
+        const unsigned long long x = wbuf[warp][c];
+        mine = max(mine, x < pv ? x : 0ull);
+      }
+      mine = warp_max_key(mine);
+      if (lane == 0) {
+        const int bi = key_index(mine);
+        top[rr * BW + p] = cand_key(base + (key_value(mine) - row_lse), rr * V + (bi == 0x7fffffff ? 0 : bi));
+      }
+      pv = mine;
+    }
+    __syncwarp();
+  }
+  __syncthreads();
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[2]));
+  // the beam of rank kout among the rows * BW candidates, (score desc, flat index asc)
+  if (warp == 0) {
+    const int n_cand = rows * BW;
+    unsigned long long pv = ~0ull;
+    for (int p = 0; p <= kout; ++p) {
+      unsigned long long mine = 0ull;
+      for (int c = lane; c < n_cand; c += 32) {
+        const unsigned long long x = top[c];
+        mine = max(mine, x < pv ? x : 0ull);
+      }
+      pv = warp_max_key(mine);
+    }
+    if (lane == 0) s_win = Cand{key_value(pv), key_index(pv)};
+  }
+  __syncthreads();
+  const Cand win = s_win;
+  const int parent = win.i / V, tok = win.i - parent * V;
+  const int orow = b * BW + kout, prow = b * BW + parent;
+  if (threadIdx.x == 0) {
+    score_out[orow] = win.v;
+    for (int t = 0; t < call - 1; ++t) hist_out[(size_t)orow * L + t] = __ldcg(hist_in + (size_t)prow * L + t);
+    hist_out[(size_t)orow * L + call - 1] = tok;
+    if (call == L) {
+      for (int t = 0; t < L - 1; ++t) beams_out[(size_t)orow * L + t] = __ldcg(hist_in + (size_t)prow * L + t);
+      beams_out[(size_t)orow * L + L - 1] = tok;
+      if (scores_out) scores_out[orow] = win.v;
+    }
+  }
+  if (call < L) {
+    // this beam's input row of the next call: [s of the parent ; E[token]], 128-bit accesses
+    constexpr int EV = 16 / sizeof(T);
+    const int ev = dm.d / EV, sv = dm.dr / 4;
+    const uint4* e = reinterpret_cast<const uint4*>(emb + (size_t)tok * dm.d);
+    uint4* eo = reinterpret_cast<uint4*>(se_t + (size_t)orow * (dm.dr + dm.d) + dm.dr);
+    for (int i = threadIdx.x; i < ev; i += MRG_THREADS) eo[i] = e[i];
+    if (call > 1) {
+      const float4* sp = reinterpret_cast<const float4*>(s_new_f + (size_t)prow * ld_s);
+      T* so = se_t + (size_t)orow * (dm.dr + dm.d);
+      for (int i = threadIdx.x; i < sv; i += MRG_THREADS) {
+        const float4 q = __ldcg(sp + i);
+        act_store4(so + 4 * i, q.x, q.y, q.z, q.w);
+      }
+    }
+  }
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[3]));
+  if (dbg && threadIdx.x == 0) {
+    atomicMin(dbg + 0, t_dbg[0]); atomicMin(dbg + 1, t_dbg[1]); atomicMax(dbg + 2, t_dbg[2]); atomicMax(dbg + 6, t_dbg[3]);
+  }
+  chain_exit(cs);
+}
+
+// Segments per row for the two-kernel selection, or 0 when the shape does not fit it.
+int draft_select_segments(const Dims& dm, int rows, int grid_hint) {
+  if (dm.BW > 32 || (dm.V & 3)) return 0;
+  int S = grid_hint / (rows > 0 ? rows : 1);
+  const int s_cap = SEG_MAX_CAND / dm.BW < 32 ? SEG_MAX_CAND / dm.BW : 32;
+  if (S > s_cap) S = s_cap;
+  const int v4 = dm.V / 4;
+  const int s_min = (v4 + SEG_THREADS * SEG_ITEMS_MAX - 1) / (SEG_THREADS * SEG_ITEMS_MAX);
+  if (S < s_min) S = s_min;
+  if (S < 1) S = 1;
+  if (S > s_cap) return 0;
+  return S;
+}
+
 // rows = B (call 1) or B * BW.  counters: [B] zero between launches.
 cudaError_t launch_draft_select(int dtype, const GemmOut& proj, int call, float* lse, float* val, int32_t* idx,
                                 const float* score_in, float* score_out, const int32_t* hist_in, int32_t* hist_out,
                                 const void* emb, const float* s_new_f, int ld_s, void* se_t, const Dims& dm, int B,
                                 int32_t* beams_out, float* scores_out, int32_t* counters, const int32_t* m_total,
-                                unsigned long long* dbg, Chain* chain, cudaStream_t st) {
+                                unsigned long long* dbg, const SelectScratch& sc, Chain* chain, cudaStream_t st) {
   if (dm.BW > SEL_MAX_BW) return cudaErrorInvalidValue;
   const int rows = call == 1 ? B : B * dm.BW;
+  const int S = sc.seg_max ? draft_select_segments(dm, rows, sc.grid_hint) : 0;
+  if (S > 0) {
+    const int seg_len4 = (dm.V / 4 + S - 1) / S;
+    dim3 g1(S, rows);
+    const ChainSync c1 = chain ? chain->link(g1.x * g1.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
+    const int items = (seg_len4 + SEG_THREADS - 1) / SEG_THREADS;
+    if (items <= 1)
+      launch_pdl(draft_seg_kernel<1>, g1, SEG_THREADS, 0, st, proj, dm.V, dm.BW, seg_len4, sc.seg_max, sc.seg_sum, sc.seg_val,
+                 sc.seg_idx, m_total, c1);
+    else if (items == 2)
+      launch_pdl(draft_seg_kernel<2>, g1, SEG_THREADS, 0, st, proj, dm.V, dm.BW, seg_len4, sc.seg_max, sc.seg_sum, sc.seg_val,
+                 sc.seg_idx, m_total, c1);
+    else
+      launch_pdl(draft_seg_kernel<4>, g1, SEG_THREADS, 0, st, proj, dm.V, dm.BW, seg_len4, sc.seg_max, sc.seg_sum, sc.seg_val,
+                 sc.seg_idx, m_total, c1);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    dim3 g2(dm.BW, B);
+    const ChainSync c2 = chain ? chain->link(g2.x * g2.y) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
+    RD_DISPATCH(dtype, launch_pdl(draft_merge_kernel<T>, g2, MRG_THREADS, 0, st, S, call, (const float*)sc.seg_max,
+                                  (const float*)sc.seg_sum, (const float*)sc.seg_val, (const int32_t*)sc.seg_idx, score_in,
+                                  score_out, hist_in, hist_out, (const T*)emb, s_new_f, ld_s, (T*)se_t, dm, beams_out,
+                                  scores_out, dbg, c2));
+    return cudaGetLastError();
+  }
   const size_t select = ((size_t)32 * dm.BW + SEL_LIST_CAP) * sizeof(Cand) + (size_t)dm.V * sizeof(float);
   const size_t prune = (size_t)dm.BW * dm.BW * sizeof(Cand);
   const size_t smem = select > prune ? select : prune;

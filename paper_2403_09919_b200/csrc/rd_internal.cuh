@@ -91,11 +91,18 @@ cudaError_t launch_draft_init(int dtype, const void* emb, const int32_t* root, c
                               void* se_t, const Dims& dm, int B, int* status, cudaStream_t st);
 cudaError_t launch_act(int dtype, const GemmOut& proj, const void* bias, const float* resid, int ld_resid, float* out_f,
                        void* out_t, int ld_out, int N, const int32_t* m_total, int m_max, Chain* chain, cudaStream_t st);
+// Scratch of the two-kernel selection (seg_max == nullptr: single-kernel selection only).
+struct SelectScratch {
+  float *seg_max, *seg_sum, *seg_val;   // [rows][32], [rows][32], [rows][512]
+  int32_t* seg_idx;                     // [rows][512]
+  int grid_hint;                        // CTAs to aim for (the SM count)
+};
+int draft_select_segments(const Dims& dm, int rows, int grid_hint);
 cudaError_t launch_draft_select(int dtype, const GemmOut& proj, int call, float* lse, float* val, int32_t* idx,
                                 const float* score_in, float* score_out, const int32_t* hist_in, int32_t* hist_out,
                                 const void* emb, const float* s_new_f, int ld_s, void* se_t, const Dims& dm, int B,
                                 int32_t* beams_out, float* scores_out, int32_t* counters, const int32_t* m_total,
-                                unsigned long long* dbg, Chain* chain, cudaStream_t st);
+                                unsigned long long* dbg, const SelectScratch& sc, Chain* chain, cudaStream_t st);
 cudaError_t launch_fill_h(int dtype, const float* h, void* x_t, float* x_f, const Dims& dm, int B, cudaStream_t st);
 
 // pack / accept
