@@ -258,18 +258,26 @@ int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, cons
     if (iw == h->maps.end() || is == h->act_shape.end() || lda != K || is->second.second != K)
       return fail(h, RD_ERR_STATE, "projection operand without a TMA descriptor");
     const int mt = tc_pick_mt(m_max > 0 ? m_max : 1);
-    auto key = std::make_pair(A, mt);
-    auto ia = h->act_maps.find(key);
-    if (ia == h->act_maps.end()) {
-      TensorMapBox box;
-      box.rows = is->second.first; box.cols = K;
-      const int rc = tc_make_map(&box, A, (uint64_t)box.rows, (uint64_t)K, (uint32_t)mt);
-      if (rc) return fail(h, RD_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d for an activation buffer", rc);
-      ia = h->act_maps.emplace(key, box).first;
+    // activation descriptors: box heights 16..mt in steps of 16 for skinny launches (the kernel picks by the
+    // actual row count), the launch's own height otherwise; made on first use
+    const void* amaps[4] = {nullptr, nullptr, nullptr, nullptr};
+    const int n_maps = mt <= 64 ? mt / 16 : 1;
+    for (int i = 0; i < n_maps; ++i) {
+      const int box_rows = mt <= 64 ? 16 * (i + 1) : mt;
+      auto key = std::make_pair(A, box_rows);
+      auto ia = h->act_maps.find(key);
+      if (ia == h->act_maps.end()) {
+        TensorMapBox box;
+        box.rows = is->second.first; box.cols = K;
+        const int rc = tc_make_map(&box, A, (uint64_t)box.rows, (uint64_t)K, (uint32_t)box_rows);
+        if (rc) return fail(h, RD_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d for an activation buffer", rc);
+        ia = h->act_maps.emplace(key, box).first;
+      }
+      amaps[i] = &ia->second;
     }
     unsigned long long* tr = nullptr;
     if (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) tr = h->ws.trace + (size_t)8 * h->trace_next++;
-    CK(h, launch_gemm_tc(&iw->second, &ia->second, N, K, m_total, m_max, raw, ld_raw, h->ws.tc_partial, h->ws.status,
+    CK(h, launch_gemm_tc(&iw->second, amaps, N, K, m_total, m_max, raw, ld_raw, h->ws.tc_partial, h->ws.status,
                          h->tc_grid, h->tc_smem, tr, out, chain, st));
     return RD_OK;
   }

@@ -39,6 +39,13 @@ constexpr int W_STAGE_BYTES = TILE_N * TILE_K * 2;
 constexpr int NUM_THREADS = 192;
 constexpr unsigned long long WAIT_LIMIT_NS = 1000000000ull;
 
+// Activation operand: one descriptor per box height.  Skinny launches (at most 64 rows) carry the descriptors
+// for 16, 32, 48 and 64 rows in m[0..3] and pick the smallest that holds the actual row count on the device;
+// taller launches use m[0] with the launch's own box height.
+struct ActMaps {
+  CUtensorMap m[4];
+};
+
 struct TcParams {
   int N, K, nkb, n_tiles, mt, m_tiles_max, stages, tmem_cols;
   const int32_t* m_total;
@@ -150,7 +157,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
-                                                                 const __grid_constant__ CUtensorMap map_a,
+                                                                 const __grid_constant__ ActMaps maps_a,
                                                                  const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   pdl_launch_dependents();  // the next kernel may start its own prologue now
@@ -168,12 +175,22 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
   const long long G = gridDim.x;
   const long long U = (long long)p.n_tiles * m_tiles * p.nkb;
   const long long u0 = gemm_range_begin(blockIdx.x, U, G), u1 = gemm_range_begin(blockIdx.x + 1, U, G);
+  // Rows actually present: the activation box, the MMA's N and the epilogue shrink to the next multiple of 16.
+  // Every byte of the activation operand is fetched once per weight tile, so at 48 rows it is more than a third
+  // of what an SM has to pull in; the row count is known before the chain starts, so it may be read at once.
+  int mt_eff = p.mt;
+  if (early && p.mt <= 64 && p.cs.signal_ptr != nullptr) {
+    const int M = *p.m_total;
+    mt_eff = min(p.mt, max(16, (M + 15) & ~15));
+  }
+  const CUtensorMap* map_a = &maps_a.m[p.mt <= 64 ? (mt_eff >> 4) - 1 : 0];
 
   // ---- shared memory carve-up (stage buffers 1024-byte aligned for the 128-byte swizzle)
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
-  const uint32_t a_stage_bytes = (uint32_t)p.mt * TILE_K * 2;
+  const uint32_t a_stage_bytes = (uint32_t)p.mt * TILE_K * 2;          // reserved
   const uint32_t stage_bytes = W_STAGE_BYTES + a_stage_bytes;
+  const uint32_t tx_bytes = W_STAGE_BYTES + (uint32_t)mt_eff * TILE_K * 2;   // arriving per stage
   const uint32_t bar_base = base + p.stages * stage_bytes;  // 8-byte aligned
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (p.stages + s); };
@@ -192,7 +209,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
     const long long u = u0 + i;
     const int t = (int)(u / p.nkb), kb = (int)(u - (long long)t * p.nkb);
     const int s = i % p.stages;
-    mbar_expect_tx(full_bar(s), stage_bytes);
+    mbar_expect_tx(full_bar(s), tx_bytes);
     tma_load_2d_hint(base + s * stage_bytes, &map_w, full_bar(s), kb * TILE_K, (t / m_tiles) * TILE_N, pol_w);
   };
   auto issue_a = [&](uint32_t i) {
@@ -201,7 +218,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
     const int s = i % p.stages;
     const int m_tile = t - (t / m_tiles) * m_tiles;
     // one box of MT rows: the TMA unit's cost is per operation, not per byte, at these sizes
-    tma_load_2d(base + s * stage_bytes + W_STAGE_BYTES, &map_a, full_bar(s), kb * TILE_K, m_tile * p.mt);
+    tma_load_2d(base + s * stage_bytes + W_STAGE_BYTES, map_a, full_bar(s), kb * TILE_K, m_tile * p.mt);
   };
 
   if (threadIdx.x == 0) {
@@ -209,7 +226,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
     // first ring-full of k-blocks depend on nothing in the step, and nothing of the CTA's remaining set-up
     // (tensor-memory allocation, the other roles' start) needs to come first.
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map_a) : "memory");
     for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
     *abort_flag = 0;
@@ -254,7 +271,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
     if (lane == 0 && u0 < u1) {
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.mt >> 3) << 17) | ((uint32_t)(TILE_N >> 4) << 24);
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(mt_eff >> 3) << 17) | ((uint32_t)(TILE_N >> 4) << 24);
       uint32_t it = 0, seg = 0;
       bool ok = true;
       for (long long u = u0; u < u1 && ok; ++seg) {
@@ -307,7 +324,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * (uint32_t)p.mt;
       float* my_partial = p.partial + (size_t)blockIdx.x * ((size_t)p.mt * TILE_N);
-      for (int c0 = 0; c0 < p.mt; c0 += 16) {
+      for (int c0 = 0; c0 < mt_eff; c0 += 16) {
         uint32_t r[16];
         tmem_ld16(taddr + c0, r);
         if (kb0 == 0) {
@@ -404,7 +421,7 @@ cudaError_t tc_prepare(int* smem_limit_out) {
   return e;
 }
 
-cudaError_t launch_gemm_tc(const void* map_w, const void* map_a, int N, int K, const int32_t* m_total, int m_max,
+cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[4], int N, int K, const int32_t* m_total, int m_max,
                            float* raw, int ld_raw, float* partial, int32_t* status, int grid, int smem_limit,
                            unsigned long long* trace, GemmOut* out_desc, Chain* chain, cudaStream_t st) {
   TcParams p;
@@ -436,10 +453,12 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* map_a, int N, int K, c
   const bool first = chain && chain->enabled && chain->prev_ptr == nullptr;
   p.cs = chain ? chain->link((unsigned)grid) : ChainSync{nullptr, 0u, nullptr, status, nullptr};
   const size_t smem = (size_t)stages * stage_bytes + overhead;
+  ActMaps am;
+  for (int i = 0; i < 4; ++i) am.m[i] = *(const CUtensorMap*)(map_a[i] ? map_a[i] : map_a[0]);
   if (first)
-    launch_ordered(gemm_tc_kernel, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, *(const CUtensorMap*)map_a, p);
+    launch_ordered(gemm_tc_kernel, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
   else
-    launch_pdl(gemm_tc_kernel, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, *(const CUtensorMap*)map_a, p);
+    launch_pdl(gemm_tc_kernel, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
   return cudaGetLastError();
 }
 
