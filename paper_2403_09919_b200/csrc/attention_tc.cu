@@ -119,16 +119,32 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
   constexpr uint32_t TILE_BYTES = KEYS * LD * 2;
   // asynchronous copy of one chunk's K and V tiles into ring slot `buf` (keys past the extent are
   // zero-filled); always closes a copy group, empty past the last chunk, so the group count is uniform
+  // per thread: 16-byte piece c8 of key rows tid/16 + 8j of a chunk (j = 0 .. KEYS/8 - 1 for HD = 128)
+  constexpr int PIECES = HD / 8;                 // 16-byte pieces per key row
+  constexpr int ROWS_PER_PASS = 128 / PIECES;    // key rows covered by one pass of the 128 threads
+  const int cp_row = tid / PIECES, cp_c8 = (tid % PIECES) * 8;
+  const __nv_bfloat16* cp_k = kc + head_base + (size_t)cp_row * HD + cp_c8;
+  const __nv_bfloat16* cp_v = vc + head_base + (size_t)cp_row * HD + cp_c8;
+  const uint32_t cp_dst = sKV_u + (cp_row * LD + cp_c8) * 2;
   auto load_chunk = [&](int ch, int buf) {
     if (ch < c_end) {
       const int k0 = ch * KEYS;
-      for (int idx = tid; idx < KEYS * (HD / 8); idx += 128) {
-        const int kr = idx / (HD / 8), c8 = (idx - kr * (HD / 8)) * 8;
-        const int key = k0 + kr;
-        const bool valid = key < kext;
-        const size_t off = head_base + (size_t)(valid ? key : 0) * HD + c8;
-        cp_async16(sKV_u + (2 * buf) * TILE_BYTES + (kr * LD + c8) * 2, kc + off, valid);
-        cp_async16(sKV_u + (2 * buf + 1) * TILE_BYTES + (kr * LD + c8) * 2, vc + off, valid);
+      const uint32_t dk = cp_dst + (2 * buf) * TILE_BYTES, dv = dk + TILE_BYTES;
+      if (k0 + KEYS <= kext) {
+#pragma unroll
+        for (int j = 0; j < KEYS / ROWS_PER_PASS; ++j) {
+          const size_t off = (size_t)(k0 + j * ROWS_PER_PASS) * HD;
+          cp_async16(dk + j * ROWS_PER_PASS * LD * 2, cp_k + off, true);
+          cp_async16(dv + j * ROWS_PER_PASS * LD * 2, cp_v + off, true);
+        }
+      } else {
+#pragma unroll 1
+        for (int j = 0; j < KEYS / ROWS_PER_PASS; ++j) {
+          const bool valid = k0 + j * ROWS_PER_PASS + cp_row < kext;
+          const size_t off = valid ? (size_t)(k0 + j * ROWS_PER_PASS) * HD : (size_t)0;
+          cp_async16(dk + j * ROWS_PER_PASS * LD * 2, cp_k + off, valid);
+          cp_async16(dv + j * ROWS_PER_PASS * LD * 2, cp_v + off, valid);
+        }
       }
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
@@ -170,6 +186,7 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
   __syncthreads();
   RD_STAMP(2);
   const int nc_lo = s_ncache[r_lo], nc_hi = s_ncache[r_hi];
+  const int nc_min = tree ? tree_base : nc_first;   // every valid row of the tile attends at least the keys below this
   const float scale = rsqrtf((float)HD);
   float o[NT][4];
 #pragma unroll
@@ -189,36 +206,60 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
 
     // ---- S = Q K^T: 16 rows x this warp's 16 keys
     float s[WKEYS / 8][4];
+    {
+      // two accumulators per key tile (even and odd k-steps): four independent MMA chains instead of two
+      float s2[WKEYS / 8][4];
 #pragma unroll
-    for (int nt = 0; nt < WKEYS / 8; ++nt) {
-      s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
-      const __nv_bfloat16* kp = sK + (nt * 8 + g) * LD + t4 * 2;
-#pragma unroll
-      for (int ks = 0; ks < KS; ++ks) {
-        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(kp + ks * 16);
-        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(kp + ks * 16 + 8);
-        mma_bf16(s[nt], qf[ks], b0, b1);
+      for (int nt = 0; nt < WKEYS / 8; ++nt) {
+        s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+        s2[nt][0] = s2[nt][1] = s2[nt][2] = s2[nt][3] = 0.f;
       }
+#pragma unroll
+      for (int ks = 0; ks < KS; ks += 2) {
+#pragma unroll
+        for (int nt = 0; nt < WKEYS / 8; ++nt) {
+          const __nv_bfloat16* kp = sK + (nt * 8 + g) * LD + t4 * 2;
+          const uint32_t b0 = *reinterpret_cast<const uint32_t*>(kp + ks * 16);
+          const uint32_t b1 = *reinterpret_cast<const uint32_t*>(kp + ks * 16 + 8);
+          const uint32_t b2 = *reinterpret_cast<const uint32_t*>(kp + ks * 16 + 16);
+          const uint32_t b3 = *reinterpret_cast<const uint32_t*>(kp + ks * 16 + 24);
+          mma_bf16(s[nt], qf[ks], b0, b1);
+          mma_bf16(s2[nt], qf[ks + 1], b2, b3);
+        }
+      }
+#pragma unroll
+      for (int nt = 0; nt < WKEYS / 8; ++nt) { s[nt][0] += s2[nt][0]; s[nt][1] += s2[nt][1]; s[nt][2] += s2[nt][2]; s[nt][3] += s2[nt][3]; }
     }
     // ---- scale, mask, online softmax (thread holds keys kw + nt*8 + t4*2 + {0,1} of rows r_lo, r_hi)
     float mx_lo = -INFINITY, mx_hi = -INFINITY;
+    if (ch * KEYS + KEYS <= nc_min) {
+      // every row of the tile attends every key of the chunk
 #pragma unroll
-    for (int nt = 0; nt < WKEYS / 8; ++nt) {
+      for (int nt = 0; nt < WKEYS / 8; ++nt) {
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int key = kw + nt * 8 + t4 * 2 + e;
-        bool v_lo = key < nc_lo, v_hi = key < nc_hi;
-        if (tree && key >= tree_base) {
-          const int tb = key - tree_base;
-          if (tb < seq_rows) {
-            v_lo = (s_mask[r_lo * MW + (tb >> 5)] >> (tb & 31)) & 1u;
-            v_hi = (s_mask[r_hi * MW + (tb >> 5)] >> (tb & 31)) & 1u;
+        for (int e = 0; e < 4; ++e) s[nt][e] *= scale;
+        mx_lo = fmaxf(mx_lo, fmaxf(s[nt][0], s[nt][1]));
+        mx_hi = fmaxf(mx_hi, fmaxf(s[nt][2], s[nt][3]));
+      }
+    } else {
+#pragma unroll
+      for (int nt = 0; nt < WKEYS / 8; ++nt) {
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int key = kw + nt * 8 + t4 * 2 + e;
+          bool v_lo = key < nc_lo, v_hi = key < nc_hi;
+          if (tree && key >= tree_base) {
+            const int tb = key - tree_base;
+            if (tb < seq_rows) {
+              v_lo = (s_mask[r_lo * MW + (tb >> 5)] >> (tb & 31)) & 1u;
+              v_hi = (s_mask[r_hi * MW + (tb >> 5)] >> (tb & 31)) & 1u;
+            }
           }
+          s[nt][e] = v_lo ? s[nt][e] * scale : -INFINITY;
+          s[nt][2 + e] = v_hi ? s[nt][2 + e] * scale : -INFINITY;
+          mx_lo = fmaxf(mx_lo, s[nt][e]);
+          mx_hi = fmaxf(mx_hi, s[nt][2 + e]);
         }
-        s[nt][e] = v_lo ? s[nt][e] * scale : -INFINITY;
-        s[nt][2 + e] = v_hi ? s[nt][2 + e] * scale : -INFINITY;
-        mx_lo = fmaxf(mx_lo, s[nt][e]);
-        mx_hi = fmaxf(mx_hi, s[nt][2 + e]);
       }
     }
     mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
