@@ -250,7 +250,7 @@ struct ProfScope {
 
 // One projection Y = A W^T into the fp32 buffer `raw` (row stride ld_raw); fills `out` for the consumer.
 int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, const int32_t* m_total, int m_max, float* raw,
-         int ld_raw, GemmOut* out, Chain* chain, cudaStream_t st) {
+         int ld_raw, GemmOut* out, Chain* chain, cudaStream_t st, int pair = 0) {
   ProfScope ps(h, 0, (double)N * K * esize(h->dm.dtype), st);
   if (h->use_tc) {
     auto iw = h->maps.find(W);
@@ -278,7 +278,7 @@ int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, cons
     unsigned long long* tr = nullptr;
     if (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) tr = h->ws.trace + (size_t)8 * h->trace_next++;
     CK(h, launch_gemm_tc(&iw->second, amaps, N, K, m_total, m_max, raw, ld_raw, h->ws.tc_partial, h->ws.status,
-                         h->tc_grid, h->tc_smem, tr, out, chain, st));
+                         h->tc_grid, h->tc_smem, tr, out, chain, pair, st));
     return RD_OK;
   }
   if (chain) chain->cut();
@@ -340,7 +340,7 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
     if (rc) return rc;
     // FFN block: (x += O) -> norm -> gate|up -> SwiGLU -> down
     CKP(h, PROF_NORM, launch_rmsnorm(dm.dtype, w.x, &g_o, h->ffn_norm[l], w.a_t, nullptr, dm.d, dm.eps, w.m_total, m_max, ch, st));
-    rc = gemm(h, w.a_t, dm.d, h->w_gate_up[l], 2 * dm.F, dm.d, w.m_total, m_max, w.gu, 2 * dm.F, &g_gu, ch, st);
+    rc = gemm(h, w.a_t, dm.d, h->w_gate_up[l], 2 * dm.F, dm.d, w.m_total, m_max, w.gu, 2 * dm.F, &g_gu, ch, st, /*pair=*/1);
     if (rc) return rc;
     CKP(h, PROF_SWIGLU, launch_swiglu(dm.dtype, g_gu, w.act_t, dm.F, w.m_total, m_max, ch, st));
     rc = gemm(h, w.act_t, dm.F, h->w_down[l], dm.d, dm.F, w.m_total, m_max, w.proj_d, dm.d, &g_dn, ch, st);
@@ -392,7 +392,7 @@ int do_draft(rd_handle* h, cudaStream_t st, int32_t* beams, float* scores) {
       CKP(h, PROF_DRAFT_SMALL, launch_act(dm.dtype, g, h->head_b[l], xin_f, dm.dh, of, ot, dm.dh, dm.dh, mt, rows, ch, st));
       xin_t = ot; xin_f = of;
     }
-    int rc = gemm(h, xin_t, dm.dh, h->w.draft_out, dm.V, dm.dh, mt, rows, w.dlogits, dm.V, &g, ch, st);
+    int rc = gemm(h, xin_t, dm.dh, h->w.draft_out, dm.V, dm.dh, mt, rows, w.dlogits, dm.V, &g, ch, st, /*pair=*/1);
     if (rc) return rc;
     CKP(h, PROF_DRAFT_SMALL, launch_draft_select(dm.dtype, g, call, w.lse, w.cand_val, w.cand_idx, sc_in, sc_out, hi_in, hi_out,
                                                  h->w.tok_emb, w.x0_f, dm.dh, w.se_t, dm, B, beams, scores, w.sel_counters, mt,
@@ -415,7 +415,7 @@ int do_verify(rd_handle* h, const rd_packed& pk, cudaStream_t st, int32_t* argma
   int rc = forward_layers(h, pk.mask, m_max, B, dm.NMAX, h->w.lm_head, st);
   if (rc) return rc;
   GemmOut g;
-  rc = gemm(h, w.hidden_t, dm.d, h->w.lm_head, dm.V, dm.d, w.m_total, m_max, w.logits, dm.V, &g, nullptr, st);
+  rc = gemm(h, w.hidden_t, dm.d, h->w.lm_head, dm.V, dm.d, w.m_total, m_max, w.logits, dm.V, &g, nullptr, st, /*pair=*/1);
   if (rc) return rc;
   CKP(h, PROF_MISC, launch_fill_i32(argmax, -1, B * dm.NMAX, st));
   CKP(h, PROF_MISC, launch_argmax_rows(w.logits, g, dm.V, argmax, w.row_out_index, w.m_total, m_max, st));

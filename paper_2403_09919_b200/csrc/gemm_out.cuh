@@ -20,7 +20,11 @@ struct GemmOut {
   int ld;
   int nkb, n_tiles, mt, grid, m_tiles_max;
   int all_work;          // every CTA has a non-empty range for any row count (units >= CTAs)
+  int pair;              // 1: a unit is (pair of adjacent tiles, k-block); a slot holds two tiles, even one first
 };
+
+// Floats per partial slot (one slot per CTA).
+__host__ __device__ __forceinline__ size_t gemm_slot_stride(const GemmOut& g) { return (size_t)g.mt * 128 * (g.pair ? 2 : 1); }
 
 // Unit range of CTA c: [c*U/G, (c+1)*U/G).
 __host__ __device__ __forceinline__ long long gemm_range_begin(long long c, long long U, long long G) { return c * U / G; }
@@ -43,11 +47,14 @@ __device__ __forceinline__ GemmFold gemm_fold(const GemmOut& g, int m_tiles, int
   GemmFold f;
   if (g.m_tiles_max == 1) {
     // one row tile (the decode-time case): 32-bit arithmetic, (units + 1) * CTAs stays far below 2^31
-    const uint32_t U = (uint32_t)g.n_tiles * g.nkb, G = g.grid, tu0 = (uint32_t)n_tile * g.nkb;
+    // (in pair mode the units run over pairs of tiles, and the odd tile sits in the second half of a slot)
+    const uint32_t group = g.pair ? (uint32_t)(n_tile >> 1) : (uint32_t)n_tile;
+    const uint32_t n_groups = g.pair ? (uint32_t)((g.n_tiles + 1) >> 1) : (uint32_t)g.n_tiles;
+    const uint32_t U = n_groups * g.nkb, G = g.grid, tu0 = group * g.nkb;
     const uint32_t cf = ((tu0 + 1) * G - 1) / U, cl = ((tu0 + g.nkb) * G - 1) / U;
     f.c_next = (int)(cf > G - 1 ? G - 1 : cf) + 1;
     f.c_last = (int)(cl > G - 1 ? G - 1 : cl);
-    f.off = (size_t)m * 128 + row;
+    f.off = (size_t)m * 128 + row + ((g.pair && (n_tile & 1)) ? (size_t)g.mt * 128 : 0);
     return f;
   }
   const int m_tile = m / g.mt, col = m - m_tile * g.mt;
@@ -62,7 +69,7 @@ __device__ __forceinline__ GemmFold gemm_fold(const GemmOut& g, int m_tiles, int
 // True when CTA c has work (with fewer units than CTAs some ranges are empty).
 __device__ __forceinline__ bool gemm_has_work(const GemmOut& g, int m_tiles, int c) {
   if (g.all_work) return true;
-  const long long U = (long long)g.n_tiles * m_tiles * g.nkb, G = g.grid;
+  const long long U = (g.pair ? (long long)((g.n_tiles + 1) >> 1) : (long long)g.n_tiles * m_tiles) * g.nkb, G = g.grid;
   return gemm_range_begin(c, U, G) < gemm_range_begin(c + 1, U, G);
 }
 
@@ -91,7 +98,7 @@ __device__ __forceinline__ GemmPending<U> gemm_issue(const GemmOut& g, int m_til
   p.raw = g.raw[(size_t)m * g.ld + n];
   p.f.c_next = 1; p.f.c_last = 0; p.f.off = 0;
   if (g.partial != nullptr) p.f = gemm_fold(g, m_tiles, m, n);
-  const size_t slot = (size_t)g.mt * 128;
+  const size_t slot = gemm_slot_stride(g);
 #pragma unroll
   for (int j = 0; j < U; ++j) {
     const int c = p.f.c_next + j;
@@ -104,7 +111,7 @@ __device__ __forceinline__ float gemm_finish(const GemmOut& g, int m_tiles, cons
   float v = p.raw;
 #pragma unroll
   for (int j = 0; j < U; ++j) v += p.q[j];
-  const size_t slot = (size_t)g.mt * 128;
+  const size_t slot = gemm_slot_stride(g);
   for (int c = p.f.c_next + U; c <= p.f.c_last; ++c)
     if (gemm_has_work(g, m_tiles, c)) v += __ldcg(g.partial + (size_t)c * slot + p.f.off);
   return v;
@@ -116,7 +123,7 @@ __device__ __forceinline__ GemmPending4<U> gemm_issue4(const GemmOut& g, int m_t
   p.raw = *reinterpret_cast<const float4*>(g.raw + (size_t)m * g.ld + n);
   p.f.c_next = 1; p.f.c_last = 0; p.f.off = 0;
   if (g.partial != nullptr) p.f = gemm_fold(g, m_tiles, m, n);
-  const size_t slot = (size_t)g.mt * 128;
+  const size_t slot = gemm_slot_stride(g);
 #pragma unroll
   for (int j = 0; j < U; ++j) {
     const int c = p.f.c_next + j;
@@ -131,7 +138,7 @@ __device__ __forceinline__ float4 gemm_finish4(const GemmOut& g, int m_tiles, co
   float4 v = p.raw;
 #pragma unroll
   for (int j = 0; j < U; ++j) { v.x += p.q[j].x; v.y += p.q[j].y; v.z += p.q[j].z; v.w += p.q[j].w; }
-  const size_t slot = (size_t)g.mt * 128;
+  const size_t slot = gemm_slot_stride(g);
   for (int c = p.f.c_next + U; c <= p.f.c_last; ++c) {
     if (!gemm_has_work(g, m_tiles, c)) continue;
     const float4 t = __ldcg(reinterpret_cast<const float4*>(g.partial + (size_t)c * slot + p.f.off));
@@ -158,7 +165,7 @@ template <int U>
 __device__ __forceinline__ GemmPending2<U> gemm_issue2(const GemmOut& g, int m_tiles, const GemmFold& f, int m, int n, int doff) {
   GemmPending2<U> p;
   p.raw = __ldcg(reinterpret_cast<const float2*>(g.raw + (size_t)m * g.ld + n));
-  const size_t slot = (size_t)g.mt * 128;
+  const size_t slot = gemm_slot_stride(g);
 #pragma unroll
   for (int j = 0; j < U; ++j) {
     const int c = f.c_next + j;
@@ -173,7 +180,7 @@ __device__ __forceinline__ float2 gemm_finish2(const GemmOut& g, int m_tiles, co
   float2 v = p.raw;
 #pragma unroll
   for (int j = 0; j < U; ++j) { v.x += p.q[j].x; v.y += p.q[j].y; }
-  const size_t slot = (size_t)g.mt * 128;
+  const size_t slot = gemm_slot_stride(g);
   for (int c = f.c_next + U; c <= f.c_last; ++c) {
     if (!gemm_has_work(g, m_tiles, c)) continue;
     const float2 t = __ldcg(reinterpret_cast<const float2*>(g.partial + (size_t)c * slot + f.off + doff));
@@ -192,7 +199,6 @@ struct GemmSrc {
   const float* part;   // the value's place in the first extra contributor's slot; slot j is at part + j * stride
   int n_extra;         // contributors other than the first (0 when the tile is not cut or on the CUDA-core path)
 };
-__device__ __forceinline__ size_t gemm_slot_stride(const GemmOut& g) { return (size_t)g.mt * 128; }
 // Valid for launches where every CTA has work (all_work), which is every launch whose stream is at
 // least as long as the grid; callers fall back to gemm_value* otherwise.
 __device__ __forceinline__ GemmSrc gemm_src(const GemmOut& g, int m_tiles, int m, int n) {

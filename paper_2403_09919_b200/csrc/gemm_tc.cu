@@ -55,6 +55,9 @@ struct TcParams {
   int32_t* status;
   unsigned long long* trace;  // 8 timestamps of this launch (see redrafter_trace_read) or nullptr
   ChainSync cs;       // counter hand-off with the launches before and after this one
+  // 1: a unit is (pair of adjacent weight tiles, k-block): both tiles of a stage are multiplied by ONE activation
+  // box, which halves what the activation operand costs an SM.  Single row tile only.
+  int pair;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -156,7 +159,8 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-__global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
+template <bool PAIR>
+__global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
                                                                  const __grid_constant__ ActMaps maps_a,
                                                                  const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -173,7 +177,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
   }
   const int m_tiles = early ? 1 : (*p.m_total + p.mt - 1) / p.mt;
   const long long G = gridDim.x;
-  const long long U = (long long)p.n_tiles * m_tiles * p.nkb;
+  const int n_groups = PAIR ? (p.n_tiles + 1) / 2 : p.n_tiles * m_tiles;   // unit = (group, k-block)
+  const long long U = (long long)n_groups * p.nkb;
   const long long u0 = gemm_range_begin(blockIdx.x, U, G), u1 = gemm_range_begin(blockIdx.x + 1, U, G);
   // Rows actually present: the activation box, the MMA's N and the epilogue shrink to the next multiple of 16.
   // Every byte of the activation operand is fetched once per weight tile, so at 48 rows it is more than a third
@@ -189,8 +194,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   const uint32_t a_stage_bytes = (uint32_t)p.mt * TILE_K * 2;          // reserved
-  const uint32_t stage_bytes = W_STAGE_BYTES + a_stage_bytes;
-  const uint32_t tx_bytes = W_STAGE_BYTES + (uint32_t)mt_eff * TILE_K * 2;   // arriving per stage
+  const uint32_t w_bytes = PAIR ? 2u * W_STAGE_BYTES : (uint32_t)W_STAGE_BYTES;
+  const uint32_t stage_bytes = w_bytes + a_stage_bytes;
+  const uint32_t tx_bytes = w_bytes + (uint32_t)mt_eff * TILE_K * 2;   // arriving per stage
   const uint32_t bar_base = base + p.stages * stage_bytes;  // 8-byte aligned
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (p.stages + s); };
@@ -210,15 +216,21 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
     const int t = (int)(u / p.nkb), kb = (int)(u - (long long)t * p.nkb);
     const int s = i % p.stages;
     mbar_expect_tx(full_bar(s), tx_bytes);
-    tma_load_2d_hint(base + s * stage_bytes, &map_w, full_bar(s), kb * TILE_K, (t / m_tiles) * TILE_N, pol_w);
+    if (PAIR) {
+      // tiles 2t and 2t+1 (the second may lie past the matrix: the copy then delivers zeros)
+      tma_load_2d_hint(base + s * stage_bytes, &map_w, full_bar(s), kb * TILE_K, (2 * t) * TILE_N, pol_w);
+      tma_load_2d_hint(base + s * stage_bytes + W_STAGE_BYTES, &map_w, full_bar(s), kb * TILE_K, (2 * t + 1) * TILE_N, pol_w);
+    } else {
+      tma_load_2d_hint(base + s * stage_bytes, &map_w, full_bar(s), kb * TILE_K, (t / m_tiles) * TILE_N, pol_w);
+    }
   };
   auto issue_a = [&](uint32_t i) {
     const long long u = u0 + i;
     const int t = (int)(u / p.nkb), kb = (int)(u - (long long)t * p.nkb);
     const int s = i % p.stages;
-    const int m_tile = t - (t / m_tiles) * m_tiles;
+    const int m_tile = PAIR ? 0 : t - (t / m_tiles) * m_tiles;
     // one box of MT rows: the TMA unit's cost is per operation, not per byte, at these sizes
-    tma_load_2d(base + s * stage_bytes + W_STAGE_BYTES, map_a, full_bar(s), kb * TILE_K, m_tile * p.mt);
+    tma_load_2d(base + s * stage_bytes + w_bytes, map_a, full_bar(s), kb * TILE_K, m_tile * p.mt);
   };
 
   if (threadIdx.x == 0) {
@@ -280,17 +292,24 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
         const uint32_t a = seg & 1u, aph = (seg >> 1) & 1u;
         if (!mbar_wait(tempty_bar(a), aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + a * (uint32_t)p.mt;
+        const uint32_t acc_cols = (uint32_t)p.mt * (PAIR ? 2u : 1u);   // columns of one accumulator buffer
+        const uint32_t d_tmem = tmem_base + a * acc_cols;
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % p.stages;
           const uint32_t ph = (it / p.stages) & 1u;
           if (!mbar_wait(full_bar(s), ph, abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
           const uint64_t wdesc = umma_desc(base + s * stage_bytes);
-          const uint64_t adesc = umma_desc(base + s * stage_bytes + W_STAGE_BYTES);
+          const uint64_t adesc = umma_desc(base + s * stage_bytes + w_bytes);
 #pragma unroll
           for (int k = 0; k < TILE_K / 16; ++k)
             umma_bf16(d_tmem, wdesc + 2 * k, adesc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+          if (PAIR) {   // the stage's second weight tile against the same activation box
+            const uint64_t wdesc2 = umma_desc(base + s * stage_bytes + W_STAGE_BYTES);
+#pragma unroll
+            for (int k = 0; k < TILE_K / 16; ++k)
+              umma_bf16(d_tmem + (uint32_t)p.mt, wdesc2 + 2 * k, adesc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+          }
           umma_commit(empty_bar(s));  // the stage is free once these MMAs have read it
         }
         if (ok) umma_commit(tfull_bar(a));
@@ -313,33 +332,37 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
     for (long long u = u0; u < u1 && ok; ++seg) {
       const int t = (int)(u / p.nkb), kb0 = (int)(u - (long long)t * p.nkb);
       const int kb1 = (int)min((long long)p.nkb, kb0 + (u1 - u));
-      const int n_tile = t / m_tiles, m_tile = t - n_tile * m_tiles;
+      const int n_tile0 = PAIR ? 2 * t : t / m_tiles, m_tile = PAIR ? 0 : t - (t / m_tiles) * m_tiles;
       const uint32_t a = seg & 1u, aph = (seg >> 1) & 1u;
-      const int n = n_tile * TILE_N + row;
       const int m_base = m_tile * p.mt;
       // one thread does the bounded wait and tells the others, so that all 128 take the same branch
       if (et == 0) *epi_ok = mbar_wait(tfull_bar(a), aph, abort_flag, p.status) ? 1 : 0;
       epi_bar_sync();
       if (!*epi_ok) { ok = false; break; }
       tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * (uint32_t)p.mt;
-      float* my_partial = p.partial + (size_t)blockIdx.x * ((size_t)p.mt * TILE_N);
-      for (int c0 = 0; c0 < mt_eff; c0 += 16) {
-        uint32_t r[16];
-        tmem_ld16(taddr + c0, r);
-        if (kb0 == 0) {
-          // this segment holds the tile's first k-block: its sums go to the output
-          if (n < p.N) {
+      const uint32_t acc_cols = (uint32_t)p.mt * (PAIR ? 2u : 1u);
+      const size_t slot_floats = (size_t)acc_cols * TILE_N;
+      for (int sub = 0; sub < (PAIR ? 2 : 1); ++sub) {
+        const int n = (n_tile0 + sub) * TILE_N + row;
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * acc_cols + (uint32_t)sub * (uint32_t)p.mt;
+        float* my_partial = p.partial + (size_t)blockIdx.x * slot_floats + (size_t)sub * p.mt * TILE_N;
+        for (int c0 = 0; c0 < mt_eff; c0 += 16) {
+          uint32_t r[16];
+          tmem_ld16(taddr + c0, r);
+          if (kb0 == 0) {
+            // this segment holds the tile's first k-block: its sums go to the output
+            if (n < p.N) {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const int m = m_base + c0 + j;
-              if (m < M) p.raw[(size_t)m * p.ld_raw + n] = __uint_as_float(r[j]);
+              for (int j = 0; j < 16; ++j) {
+                const int m = m_base + c0 + j;
+                if (m < M) p.raw[(size_t)m * p.ld_raw + n] = __uint_as_float(r[j]);
+              }
             }
-          }
-        } else {
-          // the range starts inside this tile: at most one such segment per CTA
+          } else {
+            // the range starts inside this tile: at most one such segment per CTA
 #pragma unroll
-          for (int j = 0; j < 16; ++j) my_partial[(size_t)(c0 + j) * TILE_N + row] = __uint_as_float(r[j]);
+            for (int j = 0; j < 16; ++j) my_partial[(size_t)(c0 + j) * TILE_N + row] = __uint_as_float(r[j]);
+          }
         }
       }
       tc_fence_before();
@@ -404,7 +427,7 @@ int tc_pick_mt(int m_max) {
   return mt < 16 ? 16 : mt;
 }
 
-size_t tc_partial_floats(int grid, int mt) { return (size_t)grid * mt * TILE_N; }
+size_t tc_partial_floats(int grid, int mt) { return (size_t)grid * mt * TILE_N * 2; }   // room for pair mode
 
 cudaError_t tc_prepare(int* smem_limit_out) {
   int dev = 0, lim = 0;
@@ -413,28 +436,33 @@ cudaError_t tc_prepare(int* smem_limit_out) {
   e = cudaDeviceGetAttribute(&lim, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   if (e != cudaSuccess) return e;
   cudaFuncAttributes fa;
-  e = cudaFuncGetAttributes(&fa, gemm_tc_kernel);
+  e = cudaFuncGetAttributes(&fa, gemm_tc_kernel<false>);
   if (e != cudaSuccess) return e;
   lim -= (int)fa.sharedSizeBytes;  // the opt-in limit covers static + dynamic shared memory
-  e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
+  e = cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
   if (smem_limit_out) *smem_limit_out = lim;
   return e;
 }
 
 cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[4], int N, int K, const int32_t* m_total, int m_max,
                            float* raw, int ld_raw, float* partial, int32_t* status, int grid, int smem_limit,
-                           unsigned long long* trace, GemmOut* out_desc, Chain* chain, cudaStream_t st) {
+                           unsigned long long* trace, GemmOut* out_desc, Chain* chain, int pair, cudaStream_t st) {
   TcParams p;
   p.N = N; p.K = K; p.nkb = (K + TILE_K - 1) / TILE_K; p.n_tiles = (N + TILE_N - 1) / TILE_N;
   p.mt = tc_pick_mt(m_max > 0 ? m_max : 1);
   p.m_tiles_max = m_max > 0 ? (m_max + p.mt - 1) / p.mt : 1;
+  static const int pair_ok = getenv("RD_TC_PAIR") ? atoi(getenv("RD_TC_PAIR")) : 1;   // tuning toggle
+  p.pair = (pair && pair_ok && p.m_tiles_max == 1 && p.mt <= 64 && p.n_tiles >= 2) ? 1 : 0;
+  const long long n_units = (long long)(p.pair ? (p.n_tiles + 1) / 2 : p.n_tiles) * p.nkb;
   if (out_desc) {
     out_desc->raw = raw; out_desc->partial = partial; out_desc->ld = ld_raw; out_desc->nkb = p.nkb;
     out_desc->n_tiles = p.n_tiles; out_desc->mt = p.mt; out_desc->grid = grid; out_desc->m_tiles_max = p.m_tiles_max;
-    out_desc->all_work = ((long long)p.n_tiles * p.nkb >= grid) ? 1 : 0;
+    out_desc->all_work = (n_units >= grid) ? 1 : 0;
+    out_desc->pair = p.pair;
   }
   if (m_max <= 0) return cudaSuccess;
-  const int stage_bytes = W_STAGE_BYTES + p.mt * TILE_K * 2;
+  const int stage_bytes = W_STAGE_BYTES * (p.pair ? 2 : 1) + p.mt * TILE_K * 2;
   const int overhead = 1024 + 8 * (2 * 16 + 4) + 64;
   // Skinny launches (the decode step) leave about 70 KB of the SM's shared memory to the small kernels
   // that run between projections, so that this kernel can become resident, and start its weight
@@ -446,7 +474,7 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[4], int N,
   if (stages < 2) return cudaErrorInvalidConfiguration;
   p.stages = stages;
   int cols = 32;
-  while (cols < 2 * p.mt) cols <<= 1;
+  while (cols < 2 * p.mt * (p.pair ? 2 : 1)) cols <<= 1;
   p.tmem_cols = cols;
   p.m_total = m_total; p.raw = raw; p.ld_raw = ld_raw; p.partial = partial; p.status = status; p.trace = trace;
   // the first launch of a chain starts after everything before it has completed (see launch_ordered)
@@ -455,10 +483,13 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[4], int N,
   const size_t smem = (size_t)stages * stage_bytes + overhead;
   ActMaps am;
   for (int i = 0; i < 4; ++i) am.m[i] = *(const CUtensorMap*)(map_a[i] ? map_a[i] : map_a[0]);
-  if (first)
-    launch_ordered(gemm_tc_kernel, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
-  else
-    launch_pdl(gemm_tc_kernel, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+  if (p.pair) {
+    if (first) launch_ordered(gemm_tc_kernel<true>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+    else launch_pdl(gemm_tc_kernel<true>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+  } else {
+    if (first) launch_ordered(gemm_tc_kernel<false>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+    else launch_pdl(gemm_tc_kernel<false>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+  }
   return cudaGetLastError();
 }
 

@@ -62,7 +62,7 @@ size_t tc_partial_floats(int grid, int mt);
 cudaError_t tc_prepare(int* smem_limit_out);
 cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[4], int N, int K, const int32_t* m_total, int m_max,
                            float* raw, int ld_raw, float* partial, int32_t* status, int grid, int smem_limit,
-                           unsigned long long* trace, GemmOut* out_desc, Chain* chain, cudaStream_t st);
+                           unsigned long long* trace, GemmOut* out_desc, Chain* chain, int pair, cudaStream_t st);
 
 cudaError_t launch_embed(int dtype, const void* emb, const int32_t* tok, float* x, int d, int V, const int32_t* m_total,
                          int m_max, int* status, cudaStream_t st);
