@@ -323,7 +323,7 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
     // attention block: (x += down of the previous layer) -> norm -> QKV -> rotary + KV write -> attention -> O
     CKP(h, PROF_NORM, launch_rmsnorm(dm.dtype, w.x, l ? &g_dn : nullptr, h->attn_norm[l], w.a_t, nullptr, dm.d, dm.eps,
                                      w.m_total, m_max, ch, st));
-    int rc = gemm(h, w.a_t, dm.d, h->wqkv[l], 3 * dm.d, dm.d, w.m_total, m_max, w.qkv, 3 * dm.d, &g_qkv, ch, st);
+    int rc = gemm(h, w.a_t, dm.d, h->wqkv[l], 3 * dm.d, dm.d, w.m_total, m_max, w.qkv, 3 * dm.d, &g_qkv, ch, st, /*pair=*/1);
     if (rc) return rc;
     CKP(h, PROF_ROPE, launch_rope_kv(dm.dtype, w.qkv, g_qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.rope_tab, rt, dm,
                                      m_max, w.status, ch, st));
@@ -387,7 +387,7 @@ int do_draft(rd_handle* h, cudaStream_t st, int32_t* beams, float* scores) {
     for (int l = 0; l < dm.n_head_layers; ++l) {
       float* of = (l & 1) ? w.x2_f : w.x1_f;
       void* ot = (l & 1) ? w.x2_t : w.x1_t;
-      int rc = gemm(h, xin_t, dm.dh, h->head_w[l], dm.dh, dm.dh, mt, rows, w.hraw, dm.dh, &g, ch, st);
+      int rc = gemm(h, xin_t, dm.dh, h->head_w[l], dm.dh, dm.dh, mt, rows, w.hraw, dm.dh, &g, ch, st, /*pair=*/1);
       if (rc) return rc;
       CKP(h, PROF_DRAFT_SMALL, launch_act(dm.dtype, g, h->head_b[l], xin_f, dm.dh, of, ot, dm.dh, dm.dh, mt, rows, ch, st));
       xin_t = ot; xin_f = of;

@@ -239,7 +239,7 @@ cudaError_t launch_rope_table(const int32_t* pos, float* table, int hd, float th
 // rows are spread over as many SMs as possible: 256-thread CTAs, several per row, at no more than 88
 // registers so that they are all resident beside the projection that runs before them.
 constexpr int ROPE_THREADS = 256;
-constexpr int ROPE_FOLD = 2;   // partial slots loaded up front: a QKV tile (64+ k-blocks) is rarely cut in more than three
+constexpr int ROPE_FOLD = 4;   // partial slots loaded up front: a QKV tile (64+ k-blocks) is rarely cut in more than three
 
 __device__ __forceinline__ void store2(float* p, float a, float b) { *reinterpret_cast<float2*>(p) = make_float2(a, b); }
 __device__ __forceinline__ void store2(__nv_bfloat16* p, float a, float b) {
