@@ -242,9 +242,14 @@ __device__ __forceinline__ float4 gemm_sum4(const GemmSrc& s, size_t stride, con
   float4 v = p.raw;
 #pragma unroll
   for (int j = 0; j < U; ++j) { v.x += p.q[j].x; v.y += p.q[j].y; v.z += p.q[j].z; v.w += p.q[j].w; }
-  for (int j = U; j < s.n_extra; ++j) {
-    const float4 t = __ldcg(reinterpret_cast<const float4*>(s.part + j * stride + doff));
-    v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
+  // more contributors than were loaded up front: the rest in batches of four loads (slot order is kept)
+  for (int j = U; j < s.n_extra; j += 4) {
+    float4 t[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      t[k] = j + k < s.n_extra ? __ldcg(reinterpret_cast<const float4*>(s.part + (j + k) * stride + doff)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) { v.x += t[k].x; v.y += t[k].y; v.z += t[k].z; v.w += t[k].w; }
   }
   return v;
 }
