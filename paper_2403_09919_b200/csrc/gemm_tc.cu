@@ -464,10 +464,11 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[4], int N,
   if (m_max <= 0) return cudaSuccess;
   const int stage_bytes = W_STAGE_BYTES * (p.pair ? 2 : 1) + p.mt * TILE_K * 2;
   const int overhead = 1024 + 8 * (2 * 16 + 4) + 64;
-  // Skinny launches (the decode step) leave about 70 KB of the SM's shared memory to the small kernels
-  // that run between projections, so that this kernel can become resident, and start its weight
-  // stream, while they are still running.
-  static const int cap_kb = getenv("RD_TC_SMEM_KB") ? atoi(getenv("RD_TC_SMEM_KB")) : 152;   // tuning toggles
+  // Skinny launches (the decode step) take 168 KB at most -- four stages of a pair of weight tiles plus the
+  // activation box -- and leave the rest of the SM's shared memory to the small kernels that run between
+  // projections, so that this kernel can become resident, and start its weight stream, while they are still
+  // running.  (Measured: a fifth stage does not pay.)
+  static const int cap_kb = getenv("RD_TC_SMEM_KB") ? atoi(getenv("RD_TC_SMEM_KB")) : 168;   // tuning toggles
   const int budget = p.mt <= 64 ? (smem_limit < cap_kb * 1024 ? smem_limit : cap_kb * 1024) : smem_limit;
   int stages = (budget - overhead) / stage_bytes;
   if (stages > 16) stages = 16;
