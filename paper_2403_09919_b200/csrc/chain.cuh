@@ -131,9 +131,9 @@ __device__ __forceinline__ void chain_exit(const ChainSync& cs) {
   const bool t0 = threadIdx.x == 0 && threadIdx.y == 0 && threadIdx.z == 0;
   if (cs.trace && t0) { const unsigned long long t = chain_now(); atomicMin(cs.trace + 5, t); atomicMax(cs.trace + 6, t); }
   if (cs.signal_ptr && t0) {
-    asm volatile("fence.proxy.async.global;" ::: "memory");  // consumers may read through the TMA unit
-    __threadfence();
-    atomicAdd(cs.signal_ptr, 1u);
+    // release: the CTA's stores (ordered before this thread by the barrier above) become visible before the
+    // increment; a consumer that hands the data to the TMA unit adds its own proxy fence after its acquire
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(cs.signal_ptr) : "memory");
   }
 }
 #endif
