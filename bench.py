@@ -344,13 +344,13 @@ def main():
         achieved = g_bytes / (g_ms * 1e-3) / 1e9 if g_ms > 0 else 0.0
         sb = step_bytes(cfg, ctx_mid)
         # DRAM traffic per launch: an ncu capture of six consecutive projection launches of this workload (summary
-        # under profiles/) read and wrote 1.022 x their algorithmic bytes in total (the surplus is the activation
+        # under profiles/) read and wrote 1.026 x their algorithmic bytes in total (the surplus is the activation
         # operand and the partial sums); traffic grows with the weight bytes, so that ratio scales the mean launch.
-        NCU_TRAFFIC_RATIO = 1.022
+        NCU_TRAFFIC_RATIO = 1.026
         traffic = NCU_TRAFFIC_RATIO * g_bytes / g_n if g_n else None
         line["roofline"] = {"bound": "hbm", "kernel": "projection (weight-streaming GEMM)", "achieved": achieved, "peak": peak,
                             "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
-                            "traffic_note": "bytes per launch: mean algorithmic bytes x 1.022, the DRAM read+write / algorithmic ratio of an ncu capture of six launches",
+                            "traffic_note": "bytes per launch: mean algorithmic bytes x 1.026, the DRAM read+write / algorithmic ratio of an ncu capture of six launches",
                             "algorithmic_bytes_per_launch": g_bytes / g_n if g_n else None, "peak_source": peak_src,
                             "launches_per_step": g_n / prof_steps, "ms_per_step_in_kernel": g_ms / prof_steps,
                             "attention_ms_per_step": at[0] / prof_steps,
