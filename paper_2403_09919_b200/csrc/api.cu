@@ -380,7 +380,7 @@ int do_draft(rd_handle* h, cudaStream_t st, int32_t* beams, float* scores) {
     const float* xin_f = call == 1 ? w.xc_f : w.x0_f;
     if (call > 1) {
       // s_t = SiLU([U W][s_{t-1}; e_t] + b), written into the first d_rnn columns of x0 = [s_t, h]
-      int rc = gemm(h, w.se_t, dm.dr + dm.d, w.uw, dm.dr, dm.dr + dm.d, mt, rows, w.sraw, dm.dr, &g, ch, st);
+      int rc = gemm(h, w.se_t, dm.dr + dm.d, w.uw, dm.dr, dm.dr + dm.d, mt, rows, w.sraw, dm.dr, &g, ch, st, /*pair=*/1);
       if (rc) return rc;
       CKP(h, PROF_DRAFT_SMALL, launch_act(dm.dtype, g, h->w.rnn_b, nullptr, 0, w.x0_f, w.x0_t, dm.dh, dm.dr, mt, rows, ch, st));
     }
