@@ -76,11 +76,14 @@ def test_verify_7b_shapes_two_layers():
     check_verify(Rig(cfg=synth.with_layers(dict(synth.CONFIGS["7b"], max_ctx=256), 2), oracle_dtype=np.float32))
 
 
-def test_tensor_core_path_matches_cuda_core_path():
+@pytest.mark.parametrize("vocab,d_ffn", [(1000, 1376), (1100, 1440)])
+def test_tensor_core_path_matches_cuda_core_path(vocab, d_ffn):
+    """The second shape gives the LM head 9 and the gate+up projection 23 weight tiles: odd counts, so the last
+    pair of tiles of a stage has a tile that lies past the matrix."""
     from paper_2403_09919_b200 import binding
     outs = []
     for flags in (0, binding.RD_FLAG_FORCE_SIMT):
-        r = Rig(cfg=RAGGED, flags=flags)
+        r = Rig(cfg=dict(RAGGED, vocab=vocab, d_ffn=d_ffn), flags=flags)
         prompt = np.random.default_rng(0).integers(0, 1000, size=96)
         r.eng.prefill([prompt])
         beams = np.random.default_rng(1).integers(0, 3, size=(1, 8, 5))
