@@ -11,7 +11,11 @@
  *   - The library allocates NO device memory: all scratch lives in the caller's workspace
  *     given to redrafter_init (size from redrafter_workspace_bytes).
  *   - Calls enqueue work on the given stream and return without synchronising it (the
- *     two exceptions, redrafter_prefill and redrafter_poll, say so).
+ *     two exceptions, redrafter_prefill and redrafter_poll, say so).  The calls on one handle
+ *     must be issued in stream order on one stream at a time: inside a call consecutive kernels
+ *     hand over through counters in the workspace (each is resident before its predecessor has
+ *     finished, and waits -- bounded, 1 s -> RD_ERR_TIMEOUT at the next poll -- for the
+ *     predecessor's last store), and the bookkeeping of those counters follows the call order.
  *   - Every call returns an rd_status.  Nothing throws, traps or asserts on the device;
  *     problems detected by kernels are recorded in a device status word (redrafter_poll).
  *   - Sizes: B = batch, BW = beam_width, L = beam_length (drafted tokens per candidate =
