@@ -223,6 +223,61 @@ def timed_loop(eng, n, fn):
     return e0.elapsed_time(e1)
 
 
+def run_sweep(args, cfg):
+    """Beam width x batch sweep at the workload's layer shapes (Section 4.2's trade-off on synthetic shapes): where a
+    step stops being a weight stream and becomes tensor-core work.  One line of JSON per point and a table on stderr.
+    Not part of the default run."""
+    from paper_2403_09919_b200 import binding
+    device = "cuda:0"
+    torch.cuda.set_device(device)
+    peak_bw, _ = measured_peaks()
+    peak_tf = 1411.0
+    try:
+        with open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "MEASURED_PEAKS.json")) as f:
+            peak_tf = float(json.load(f).get("bf16_tflops_sustained", peak_tf))
+    except Exception:
+        pass
+    w = synth.make_weights(cfg, device)
+    L = cfg["beam_length"]
+    rows = []
+    for BW in [int(x) for x in args.sweep_bw.split(",")]:
+        for B in [int(x) for x in args.sweep_batch.split(",")]:
+            c = dict(cfg, beam_width=BW, max_batch=B, prompt_len=args.sweep_prompt)
+            need = args.warmup + args.steps
+            c["max_ctx"] = args.sweep_prompt + (need + 2) * (L + 1) + 2 + BW * L
+            eng = binding.ReDrafter(c, w, device=device)
+            prompts = synth.make_prompts(c, B, seed=c.get("seed", 0))
+            out = binding.AcceptOut(B, L, device)
+            eng.prefill(prompts)
+            beams, _ = eng.draft()
+            n_rows = int(eng.pack(beams).n.sum().item())       # packed rows of a typical step (the drafter's own beams)
+            for _ in range(args.warmup):
+                eng.step(None, out)
+
+            def one(i):
+                eng.step(None, out)
+            ms = timed_loop(eng, args.steps, one) / args.steps
+            eng.poll()
+            ctx = args.sweep_prompt + (args.warmup + args.steps / 2) * 1.0
+            sb = step_bytes(c, ctx * B)
+            es = 2
+            flops = 2.0 * n_rows * (sb["llm"] / es) + 2.0 * (B * BW) * (sb["drafter"] / es) + 4.0 * n_rows * ctx * c["d_model"] * c["n_layers"]
+            t_bw, t_tc = sb["total"] / (peak_bw * 1e9) * 1e3, flops / (peak_tf * 1e12) * 1e3
+            row = {"sweep": True, "beam_width": BW, "batch": B, "packed_rows": n_rows, "ms_per_step": ms,
+                   "algorithmic_gb": sb["total"] / 1e9, "dense_tflop": flops / 1e12, "hbm_bound_ms": t_bw, "tensor_bound_ms": t_tc,
+                   "roofline_ms": max(t_bw, t_tc), "frac_of_roofline": max(t_bw, t_tc) / ms,
+                   "bound": "hbm" if t_bw >= t_tc else "tensor"}
+            rows.append(row)
+            print(json.dumps(row), flush=True)
+            eng.close()
+            del eng
+    print("| BW | batch | packed rows | ms/step | HBM-bound ms | tensor-bound ms | bound | roofline frac |", file=sys.stderr)
+    print("|---|---|---|---|---|---|---|---|", file=sys.stderr)
+    for r in rows:
+        print("| %d | %d | %d | %.2f | %.2f | %.2f | %s | %.2f |" % (r["beam_width"], r["batch"], r["packed_rows"], r["ms_per_step"],
+              r["hbm_bound_ms"], r["tensor_bound_ms"], r["bound"], r["frac_of_roofline"]), file=sys.stderr)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -236,12 +291,19 @@ def main():
     ap.add_argument("--cpu-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the planted-beam and autoregressive comparison legs")
+    ap.add_argument("--sweep", action="store_true", help="beam width x batch sweep instead of the benchmark line")
+    ap.add_argument("--sweep-bw", default="1,4,8,16,32")
+    ap.add_argument("--sweep-batch", default="1,2,4,8,16")
+    ap.add_argument("--sweep-prompt", type=int, default=256)
     args = ap.parse_args()
     cfg = dict(synth.CONFIGS[args.workload])
     if args.layers:
         cfg = synth.with_layers(cfg, args.layers)
     if args.impl == "reference":
         run_reference(args, cfg)
+        return
+    if args.sweep:
+        run_sweep(args, cfg)
         return
     if args.warmup < 3:
         args.warmup = 3

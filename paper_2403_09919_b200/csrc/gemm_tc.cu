@@ -39,11 +39,12 @@ constexpr int W_STAGE_BYTES = TILE_N * TILE_K * 2;
 constexpr int NUM_THREADS = 192;
 constexpr unsigned long long WAIT_LIMIT_NS = 1000000000ull;
 
-// Activation operand: one descriptor per box height.  Skinny launches (at most 64 rows) carry the descriptors
-// for 16, 32, 48 and 64 rows in m[0..3] and pick the smallest that holds the actual row count on the device;
-// taller launches use m[0] with the launch's own box height.
+// Activation operand: one descriptor per box height.  Launches with a single row tile (at most 256 rows) carry
+// the descriptors for 16, 32, ..., 256 rows in m[0..15] and pick the smallest that holds the actual row count on
+// the device; launches with several row tiles use m[0] with the launch's own box height.
+constexpr int ACT_MAPS = 16;
 struct ActMaps {
-  CUtensorMap m[4];
+  CUtensorMap m[ACT_MAPS];
 };
 
 struct TcParams {
@@ -184,11 +185,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
   // Every byte of the activation operand is fetched once per weight tile, so at 48 rows it is more than a third
   // of what an SM has to pull in; the row count is known before the chain starts, so it may be read at once.
   int mt_eff = p.mt;
-  if (early && p.mt <= 64 && p.cs.signal_ptr != nullptr) {
+  if (early && p.cs.signal_ptr != nullptr) {
     const int M = *p.m_total;
     mt_eff = min(p.mt, max(16, (M + 15) & ~15));
   }
-  const CUtensorMap* map_a = &maps_a.m[p.mt <= 64 ? (mt_eff >> 4) - 1 : 0];
+  const CUtensorMap* map_a = &maps_a.m[early ? (mt_eff >> 4) - 1 : 0];
 
   // ---- shared memory carve-up (stage buffers 1024-byte aligned for the 128-byte swizzle)
   const uint32_t raw = smem_u32(smem_raw);
@@ -445,7 +446,7 @@ cudaError_t tc_prepare(int* smem_limit_out) {
   return e;
 }
 
-cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[4], int N, int K, const int32_t* m_total, int m_max,
+cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[16], int N, int K, const int32_t* m_total, int m_max,
                            float* raw, int ld_raw, float* partial, int32_t* status, int grid, int smem_limit,
                            unsigned long long* trace, GemmOut* out_desc, Chain* chain, int pair, cudaStream_t st) {
   TcParams p;
@@ -453,7 +454,7 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[4], int N,
   p.mt = tc_pick_mt(m_max > 0 ? m_max : 1);
   p.m_tiles_max = m_max > 0 ? (m_max + p.mt - 1) / p.mt : 1;
   static const int pair_ok = getenv("RD_TC_PAIR") ? atoi(getenv("RD_TC_PAIR")) : 1;   // tuning toggle
-  p.pair = (pair && pair_ok && p.m_tiles_max == 1 && p.mt <= 64 && p.n_tiles >= 2) ? 1 : 0;
+  p.pair = (pair && pair_ok && p.m_tiles_max == 1 && p.mt <= 128 && p.n_tiles >= 2) ? 1 : 0;
   const long long n_units = (long long)(p.pair ? (p.n_tiles + 1) / 2 : p.n_tiles) * p.nkb;
   if (out_desc) {
     out_desc->raw = raw; out_desc->partial = partial; out_desc->ld = ld_raw; out_desc->nkb = p.nkb;
@@ -483,7 +484,7 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[4], int N,
   p.cs = chain ? chain->link((unsigned)grid) : ChainSync{nullptr, 0u, nullptr, status, nullptr};
   const size_t smem = (size_t)stages * stage_bytes + overhead;
   ActMaps am;
-  for (int i = 0; i < 4; ++i) am.m[i] = *(const CUtensorMap*)(map_a[i] ? map_a[i] : map_a[0]);
+  for (int i = 0; i < ACT_MAPS; ++i) am.m[i] = *(const CUtensorMap*)(map_a[i] ? map_a[i] : map_a[0]);
   if (p.pair) {
     if (first) launch_ordered(gemm_tc_kernel<true>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
     else launch_pdl(gemm_tc_kernel<true>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
