@@ -258,14 +258,13 @@ int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, cons
     if (iw == h->maps.end() || is == h->act_shape.end() || lda != K || is->second.second != K)
       return fail(h, RD_ERR_STATE, "projection operand without a TMA descriptor");
     const int mt = tc_pick_mt(m_max > 0 ? m_max : 1);
-    // activation descriptors: box heights 16..mt in steps of 16 for launches with one row tile (the kernel picks
-    // by the actual row count), the launch's own height otherwise; made on first use
+    // activation descriptors: box heights 16..mt in steps of 16 (a launch that has a single row tile picks by the
+    // actual row count); made on first use
     const void* amaps[16] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr,
                              nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
-    const bool one_tile = m_max <= mt;
-    const int n_maps = one_tile ? mt / 16 : 1;
+    const int n_maps = mt / 16;
     for (int i = 0; i < n_maps; ++i) {
-      const int box_rows = one_tile ? 16 * (i + 1) : mt;
+      const int box_rows = 16 * (i + 1);
       auto key = std::make_pair(A, box_rows);
       auto ia = h->act_maps.find(key);
       if (ia == h->act_maps.end()) {

@@ -39,9 +39,8 @@ constexpr int W_STAGE_BYTES = TILE_N * TILE_K * 2;
 constexpr int NUM_THREADS = 192;
 constexpr unsigned long long WAIT_LIMIT_NS = 1000000000ull;
 
-// Activation operand: one descriptor per box height.  Launches with a single row tile (at most 256 rows) carry
-// the descriptors for 16, 32, ..., 256 rows in m[0..15] and pick the smallest that holds the actual row count on
-// the device; launches with several row tiles use m[0] with the launch's own box height.
+// Activation operand: one descriptor per box height, 16, 32, ..., 256 rows in m[0..15] (up to the launch's own
+// height).  A launch that turns out to have a single row tile picks the smallest that holds the actual row count.
 constexpr int ACT_MAPS = 16;
 struct ActMaps {
   CUtensorMap m[ACT_MAPS];
@@ -185,11 +184,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
   // Every byte of the activation operand is fetched once per weight tile, so at 48 rows it is more than a third
   // of what an SM has to pull in; the row count is known before the chain starts, so it may be read at once.
   int mt_eff = p.mt;
-  if (early && p.cs.signal_ptr != nullptr) {
+  if ((early && p.cs.signal_ptr != nullptr) || (!early && m_tiles == 1)) {
     const int M = *p.m_total;
     mt_eff = min(p.mt, max(16, (M + 15) & ~15));
   }
-  const CUtensorMap* map_a = &maps_a.m[early ? (mt_eff >> 4) - 1 : 0];
+  const CUtensorMap* map_a = &maps_a.m[(mt_eff >> 4) - 1];
 
   // ---- shared memory carve-up (stage buffers 1024-byte aligned for the 128-byte swizzle)
   const uint32_t raw = smem_u32(smem_raw);
@@ -422,9 +421,10 @@ int tc_weight_box_rows() { return TILE_N; }
 
 // Activation rows per tile for a launch whose row count is at most m_max.
 int tc_pick_mt(int m_max) {
-  const int m_tiles = (m_max + 255) / 256;
-  const int per = (m_max + m_tiles - 1) / m_tiles;
-  int mt = (per + 15) / 16 * 16;
+  // One row tile up to 256 rows.  Beyond that the tiles are 256 rows: the bound is a host-side one (batch x rows per
+  // sequence) and the actual count is often below 256, in which case the kernel runs a single tile after all.
+  if (m_max > 256) return 256;
+  const int mt = (m_max + 15) / 16 * 16;
   return mt < 16 ? 16 : mt;
 }
 
