@@ -405,6 +405,27 @@ def main():
         g_ms, g_bytes, g_n = gm
         achieved = g_bytes / (g_ms * 1e-3) / 1e9 if g_ms > 0 else 0.0
         sb = step_bytes(cfg, ctx_mid)
+        # The per-launch event timing above serialises the launches: a projection timed alone cannot start its weight
+        # stream under its predecessor the way it does in the running step.  The in-kernel timeline of one traced step
+        # gives the rate in place: weight bytes / (last CTA done - last CTA past its dependency wait), summed over the
+        # step's projections.
+        in_step = None
+        try:
+            eng.trace(True)
+            eng.step(None, out)
+            torch.cuda.synchronize()
+            tr = eng.trace_read().astype(np.int64)
+            tb = eng.trace_bytes()
+            eng.trace(False)
+            sel = [i for i in range(len(tb)) if tb[i] > 0 and tr[i][6] > tr[i][2] > 0]
+            body_ns = float(sum(int(tr[i][6] - tr[i][2]) for i in sel))
+            if body_ns > 0:
+                in_step = {"gbs": float(sum(tb[i] for i in sel)) / body_ns, "launches": len(sel), "ms_per_step": body_ns * 1e-6,
+                           "note": "in-kernel %globaltimer records of one traced step (not CUDA events): weight bytes / time from "
+                                   "the last CTA's dependency wait to the last CTA's end, summed over the projections"}
+                in_step["frac_of_measured_peak"] = in_step["gbs"] / peak
+        except Exception as e:  # measurement aid only
+            in_step = {"error": str(e)}
         # DRAM traffic per launch: an ncu capture of six consecutive projection launches of this workload (summary
         # under profiles/) read and wrote 1.026 x their algorithmic bytes in total (the surplus is the activation
         # operand and the partial sums); traffic grows with the weight bytes, so that ratio scales the mean launch.
@@ -414,6 +435,7 @@ def main():
                             "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
                             "traffic_note": "bytes per launch: mean algorithmic bytes x 1.026, the DRAM read+write / algorithmic ratio of an ncu capture of six launches",
                             "algorithmic_bytes_per_launch": g_bytes / g_n if g_n else None, "peak_source": peak_src,
+                            "in_step": in_step,
                             "launches_per_step": g_n / prof_steps, "ms_per_step_in_kernel": g_ms / prof_steps,
                             "attention_ms_per_step": at[0] / prof_steps,
                             "other_ms_per_step": {n: round(o[0] / prof_steps, 4) for n, o in

@@ -225,18 +225,27 @@ RD_API int redrafter_profile(rd_handle* h, int enable);
 RD_API int redrafter_profile_read(rd_handle* h, int32_t cls, double* ms, double* bytes, int64_t* launches);
 
 /* In-kernel timeline, for measurement only.  After redrafter_trace(h, 1, stream) the next launches of
- * the traced kernels (up to 512, in launch order) each record eight %globaltimer values in ns:
+ * the traced kernels (up to 512, in launch order) each record eight %globaltimer values in ns
+ * (fields a kernel does not write keep their initial value: all ones in [0], [1], [3], [5], zero elsewhere):
  *   tensor-core projection: [0] first CTA entered, [1]/[2] first/last producer past its dependency wait,
- *                           [3]/[4] first/last MMA issuer done, [5]/[6] first/last CTA done;
- *   tensor-core attention (CTA of head 0, sequence 0, split 0): [0] entered, [1] past its dependency
- *                           wait, [2] Q and masks loaded, [3] key chunks done, [4] partial published,
- *                           [6] merge by the last split done;
- *   drafter selection (last CTA): [0] entered, [1] past the wait, [2] logits in shared memory,
- *                           [3] threshold found, [4] row ranked, [5] arrival counted, [6] pruning done.
+ *                           [3]/[4] first/last MMA issuer done, [5]/[6] first/last CTA done, [7] last producer
+ *                           ready to wait (its first ring of weight tiles requested);
+ *   short kernels of the chained loops (RMSNorm, rotary, SwiGLU, drafter activation, selection segments):
+ *                           [0]/[7] first/last CTA entered, [1]/[2] first/last CTA past its wait,
+ *                           [5]/[6] first/last CTA done;
+ *   tensor-core attention:  [0] entered, [1] past its wait, [2] Q loaded, [3] key chunks done (the CTA of head 0,
+ *                           sequence 0, split 0); [6] last CTA done;
+ *   selection, two-kernel form (its second kernel): [0] first CTA entered, [1] first past the wait, [2] last CTA's
+ *                           rows merged, [6] last CTA done;  single-kernel form (last CTA): [0] entered, [1] past
+ *                           the wait, [2] logits in shared memory, [3] threshold found, [4] row ranked,
+ *                           [5] arrival counted, [6] pruning done.
  * redrafter_trace_read synchronises the stream, copies the records of the launches traced so far to
- * the HOST buffer out[max_launches][8] and returns their number (or a negative rd_status). */
+ * the HOST buffer out[max_launches][8] and returns their number (or a negative rd_status).
+ * redrafter_trace_bytes fills the HOST buffer out[max_launches] with the weight bytes (N*K*element size) of each of
+ * those launches, 0 for the ones that are not projections, and returns the same number. */
 RD_API int redrafter_trace(rd_handle* h, int enable, void* stream);
 RD_API int redrafter_trace_read(rd_handle* h, void* stream, uint64_t* out, int32_t max_launches);
+RD_API int redrafter_trace_bytes(rd_handle* h, double* out, int32_t max_launches);
 
 /* Number of kernels this handle has launched since it was created (for launch accounting). */
 RD_API int64_t redrafter_launch_count(const rd_handle* h);

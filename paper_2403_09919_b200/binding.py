@@ -25,7 +25,8 @@ EXPORTS = ["redrafter_workspace_bytes", "redrafter_kv_bytes", "redrafter_init", 
            "redrafter_last_error", "redrafter_prefill", "redrafter_draft", "redrafter_pack", "redrafter_verify",
            "redrafter_accept", "redrafter_step", "redrafter_ar_step", "redrafter_get_state", "redrafter_set_state",
            "redrafter_set_ctx_bound", "redrafter_poll", "redrafter_launch_count", "redrafter_profile",
-           "redrafter_profile_read", "redrafter_trace", "redrafter_trace_read", "redrafter_accept_static"]
+           "redrafter_profile_read", "redrafter_trace", "redrafter_trace_read", "redrafter_trace_bytes",
+           "redrafter_accept_static"]
 
 
 class RdConfig(C.Structure):
@@ -88,6 +89,7 @@ def lib():
                                              C.POINTER(C.c_int64)]
         L.redrafter_trace.argtypes = [vp, C.c_int, vp]
         L.redrafter_trace_read.argtypes = [vp, vp, vp, i32]
+        L.redrafter_trace_bytes.argtypes = [vp, vp, i32]
         _lib = L
     return _lib
 
@@ -301,6 +303,15 @@ class ReDrafter:
         import numpy as np
         buf = np.zeros((max_launches, 8), dtype=np.uint64)
         n = self.L.redrafter_trace_read(self.h, _stream(), buf.ctypes.data, max_launches)
+        if n < 0:
+            self._ck(-n)
+        return buf[:n]
+
+    def trace_bytes(self, max_launches=512):
+        """Weight bytes of each traced launch (0 for launches that are not projections)."""
+        import numpy as np
+        buf = np.zeros(max_launches, dtype=np.float64)
+        n = self.L.redrafter_trace_bytes(self.h, buf.ctypes.data, max_launches)
         if n < 0:
             self._ck(-n)
         return buf[:n]

@@ -86,6 +86,7 @@ struct rd_handle {
   // tensor-core path (bf16): TMA descriptors by base pointer, launch geometry
   bool use_tc;
   int trace_next;  // next trace slot, -1 = tracing off
+  std::vector<double> trace_bytes;  // weight bytes of each traced launch (0: not a projection)
   int tc_grid, tc_smem;
   Chain chain;  // counter hand-off between the launches of a forward pass
   std::unordered_map<const void*, TensorMapBox> maps;               // weights
@@ -277,7 +278,11 @@ int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, cons
       amaps[i] = &ia->second;
     }
     unsigned long long* tr = nullptr;
-    if (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) tr = h->ws.trace + (size_t)8 * h->trace_next++;
+    if (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) {
+      if ((int)h->trace_bytes.size() < TRACE_SLOTS) h->trace_bytes.assign(TRACE_SLOTS, 0.0);
+      h->trace_bytes[h->trace_next] = (double)N * K * esize(h->dm.dtype);
+      tr = h->ws.trace + (size_t)8 * h->trace_next++;
+    }
     CK(h, launch_gemm_tc(&iw->second, amaps, N, K, m_total, m_max, raw, ld_raw, h->ws.tc_partial, h->ws.status,
                          h->tc_grid, h->tc_smem, tr, out, chain, pair, st));
     return RD_OK;
@@ -792,6 +797,7 @@ int redrafter_trace(rd_handle* h, int enable, void* stream) {
     CKRT(h, cudaMemcpyAsync(h->ws.trace, init.data(), init.size() * sizeof(unsigned long long), cudaMemcpyHostToDevice, st));
     CKRT(h, cudaStreamSynchronize(st));
     h->trace_next = 0;
+    h->trace_bytes.assign(TRACE_SLOTS, 0.0);
   } else {
     h->trace_next = -1;
   }
@@ -806,6 +812,14 @@ int redrafter_trace_read(rd_handle* h, void* stream, uint64_t* out, int32_t max_
   cudaError_t e = cudaMemcpyAsync(out, h->ws.trace, (size_t)n * 8 * sizeof(unsigned long long), cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) return -fail(h, RD_ERR_CUDA, "trace read: %s", cudaGetErrorString(e));
+  return n;
+}
+
+int redrafter_trace_bytes(rd_handle* h, double* out, int32_t max_launches) {
+  if (!h || !out || max_launches < 0) return -RD_ERR_INVALID_ARG;
+  int n = h->trace_next < 0 ? 0 : h->trace_next;
+  if (n > max_launches) n = max_launches;
+  for (int i = 0; i < n; ++i) out[i] = i < (int)h->trace_bytes.size() ? h->trace_bytes[i] : 0.0;
   return n;
 }
 
