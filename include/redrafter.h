@@ -247,6 +247,12 @@ RD_API int redrafter_trace(rd_handle* h, int enable, void* stream);
 RD_API int redrafter_trace_read(rd_handle* h, void* stream, uint64_t* out, int32_t max_launches);
 RD_API int redrafter_trace_bytes(rd_handle* h, double* out, int32_t max_launches);
 
+/* Self-test of the bounded device-side waits (the paper has no counterpart).  Enqueues one tiny kernel that waits on
+ * a hand-off counter value that nothing will ever produce: the wait gives up after its limit (about one second) and
+ * records it, the kernel returns, the context stays usable; the next redrafter_poll returns RD_ERR_TIMEOUT and clears
+ * the status word.  Nothing else of the handle's state is touched. */
+RD_API int redrafter_selftest_wait(rd_handle* h, void* stream);
+
 /* Number of kernels this handle has launched since it was created (for launch accounting). */
 RD_API int64_t redrafter_launch_count(const rd_handle* h);
 

@@ -26,7 +26,7 @@ EXPORTS = ["redrafter_workspace_bytes", "redrafter_kv_bytes", "redrafter_init", 
            "redrafter_accept", "redrafter_step", "redrafter_ar_step", "redrafter_get_state", "redrafter_set_state",
            "redrafter_set_ctx_bound", "redrafter_poll", "redrafter_launch_count", "redrafter_profile",
            "redrafter_profile_read", "redrafter_trace", "redrafter_trace_read", "redrafter_trace_bytes",
-           "redrafter_accept_static"]
+           "redrafter_accept_static", "redrafter_selftest_wait"]
 
 
 class RdConfig(C.Structure):
@@ -90,6 +90,7 @@ def lib():
         L.redrafter_trace.argtypes = [vp, C.c_int, vp]
         L.redrafter_trace_read.argtypes = [vp, vp, vp, i32]
         L.redrafter_trace_bytes.argtypes = [vp, vp, i32]
+        L.redrafter_selftest_wait.argtypes = [vp, vp]
         _lib = L
     return _lib
 
@@ -282,6 +283,9 @@ class ReDrafter:
         self.B = batch
         if ctx_bound is not None:
             self._ck(self.L.redrafter_set_ctx_bound(self.h, int(ctx_bound)))
+
+    def selftest_wait(self):
+        self._ck(self.L.redrafter_selftest_wait(self.h, _stream()))
 
     def poll(self):
         self._ck(self.L.redrafter_poll(self.h, _stream()))

@@ -432,6 +432,11 @@ int do_verify(rd_handle* h, const rd_packed& pk, cudaStream_t st, int32_t* argma
 
 }  // namespace
 
+// One warp whose first thread waits, bounded, on a hand-off counter value that no launch will ever produce.
+__global__ void selftest_wait_kernel(rd::ChainSync cs) {
+  if (threadIdx.x == 0) rd::chain_wait_thread(cs);
+}
+
 extern "C" {
 
 size_t redrafter_workspace_bytes(const rd_config* cfg) {
@@ -821,6 +826,15 @@ int redrafter_trace_bytes(rd_handle* h, double* out, int32_t max_launches) {
   if (n > max_launches) n = max_launches;
   for (int i = 0; i < n; ++i) out[i] = i < (int)h->trace_bytes.size() ? h->trace_bytes[i] : 0.0;
   return n;
+}
+
+int redrafter_selftest_wait(rd_handle* h, void* stream) {
+  if (!h) return RD_ERR_INVALID_ARG;
+  if (!h->chain.ctr) return fail(h, RD_ERR_STATE, "no hand-off counters in this workspace");
+  ChainSync cs{h->chain.ctr, h->chain.cum[0] + 0x40000000u, nullptr, h->ws.status, nullptr};
+  selftest_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(cs);
+  CK(h, cudaGetLastError());
+  return RD_OK;
 }
 
 int redrafter_poll(rd_handle* h, void* stream) {

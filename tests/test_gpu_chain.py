@@ -80,3 +80,28 @@ def test_fused_steps_repeat_bit_identically():
     for other in streams[1:]:
         for (na, ta), (nb, tb) in zip(streams[0], other):
             assert na == nb and (ta[:na + 1] == tb[:nb + 1]).all()
+
+
+def test_a_wait_that_nothing_satisfies_gives_up_and_is_reported():
+    """The device-side waits are bounded: one that can never be satisfied returns after about a second, the next
+    poll reports RD_ERR_TIMEOUT and clears it, and the engine keeps working."""
+    import time
+    r = make_rig(True)
+    rng = np.random.default_rng(3)
+    r.eng.prefill([rng.integers(0, r.cfg["vocab"], size=64)])
+    out = r.binding.AcceptOut(1, r.cfg["beam_length"], "cuda:0")
+    r.eng.step(None, out)
+    r.eng.poll()
+    ref_state = [s.clone() for s in r.eng.get_state()]
+    t0 = time.time()
+    r.eng.selftest_wait()
+    with pytest.raises(r.binding.RdError) as e:
+        r.eng.poll()
+    dt = time.time() - t0
+    assert e.value.code == 6 and 0.5 < dt < 10.0          # RD_ERR_TIMEOUT, after the wait's one-second limit
+    r.eng.poll()                                          # the status word was cleared
+    for a, b in zip(ref_state, r.eng.get_state()):
+        assert torch.equal(a, b)                          # nothing of the state was touched
+    r.eng.step(None, out)                                 # and the engine still decodes
+    r.eng.poll()
+    assert int(out.n_accept[0]) >= 0
