@@ -1,4 +1,4 @@
-"""Benchmark of one ReDrafter speculative decode step on B200 (see the design doc for the contract).
+"""Benchmark of one ReDrafter speculative decode step on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 7b] [--impl ours|reference]
 
