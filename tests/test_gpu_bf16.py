@@ -128,12 +128,15 @@ def run_steps(rig, n_steps, seed, p=0.3, rho=0.3):
         c_ctx, c_root, c_h = rig.eng.get_state()
         assert int(c_ctx[0]) == ctx + 1 + a and int(c_root[0]) == toks[-1]
         if (am == ref["argmax"]).all():
-            full_match += 1
             assert a == ref["n_accept"] and toks == ref["emitted"]
+        if a == ref["n_accept"] and toks == ref["emitted"]:
+            # same outcome as the oracle's step (rows off the accepted path may differ at near-ties): the handed-over
+            # hidden state and the compacted cache must then agree too
+            full_match += 1
             assert rel_err(c_h[0].cpu().numpy()[None], np.asarray(ref["h"])[None]) < REL
             kvg = rig.eng.kv_view()[:, 0, 0, :, :ref["ctx"]].float().cpu().numpy().transpose(0, 2, 1, 3)
             assert np.abs(kvg - kv.k[:, :ref["ctx"]]).max() < REL * np.abs(kv.k[:, :ref["ctx"]]).max()
-        elif a != ref["n_accept"]:
+        else:
             break                                     # an undecided row changed the outcome: stop here
         ctx, g, h = ref["ctx"], ref["g"], ref["h"]
         emitted.extend(ref["emitted"])
