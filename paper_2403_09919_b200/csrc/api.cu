@@ -308,10 +308,16 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
   // attention launch geometry (tensor-core path): tiles of 16 rows per sequence; keys split over CTAs only
   // for long contexts with few tiles
   int row_blocks = 1, n_splits = 1;
+  bool att_wide = false;
   if (h->use_tc) {
     const int rpb = attn_tc_rows_per_block();
     row_blocks = (rows_per_seq_max + rpb - 1) / rpb;
     const int blocks = dm.H * n_seq * row_blocks;
+    // The 16-row kernel runs one CTA per SM; past a few waves of them the 64-row kernel (three CTAs per SM, each
+    // K/V chunk staged once for four times the rows) takes over.
+    static const int wide_waves = getenv("RD_ATT_WIDE") ? atoi(getenv("RD_ATT_WIDE")) : 4;   // tuning toggle
+    att_wide = wide_waves < 0 || (wide_waves > 0 && blocks > wide_waves * h->tc_grid);   // negative: always
+    if (att_wide) row_blocks = (rows_per_seq_max + attn_wide_rows_per_block() - 1) / attn_wide_rows_per_block();
     n_splits = h->tc_grid / blocks;  // at most one CTA per SM: a second wave would double the time
     // ... and only when a CTA would otherwise walk many chunks: the cross-CTA merge costs several microseconds
     const int max_chunks = (h->ctx_bound + rows_per_seq_max + 63) / 64;
@@ -335,7 +341,10 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
                                      m_max, w.status, ch, st));
     {
       ProfScope ps(h, 1, 0.0, st);
-      if (h->use_tc)
+      if (h->use_tc && att_wide)
+        CK(h, launch_attention_wide(w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.attn_t, rt, w.seq_off, dm, n_seq,
+                                    row_blocks, ch, st));
+      else if (h->use_tc)
         CK(h, launch_attention_tc(w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.attn_t, rt, w.seq_off, dm, n_seq,
                                   row_blocks, n_splits, w.att_scratch, w.att_counters,
                                   (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) ? w.trace + (size_t)8 * h->trace_next++ : nullptr, ch, st));
@@ -494,6 +503,7 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
     if (ce == cudaSuccess) ce = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (ce == cudaSuccess) ce = tc_prepare(&h->tc_smem);
     if (ce == cudaSuccess) ce = attn_tc_prepare(dm.hd, dm.MW);
+    if (ce == cudaSuccess) ce = attn_wide_prepare(dm.hd, dm.MW);
     if (ce != cudaSuccess || sms <= 0)
       return init_fail(h, RD_ERR_CUDA, "tensor-core path set-up: %s", cudaGetErrorString(ce));
     h->tc_grid = sms < TC_MAX_GRID ? sms : TC_MAX_GRID;

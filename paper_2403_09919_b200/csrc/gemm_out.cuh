@@ -21,6 +21,7 @@ struct GemmOut {
   int nkb, n_tiles, mt, grid, m_tiles_max;
   int all_work;          // every CTA has a non-empty range for any row count (units >= CTAs)
   int pair;              // 1: a unit is (pair of adjacent tiles, k-block); a slot holds two tiles, even one first
+  int small32;           // (units + 1) * CTAs stays below 2^31 for any row count of the launch: 32-bit index arithmetic
 };
 
 // Floats per partial slot (one slot per CTA).
@@ -57,19 +58,28 @@ __device__ __forceinline__ GemmFold gemm_fold(const GemmOut& g, int m_tiles, int
     f.off = (size_t)m * 128 + row + ((g.pair && (n_tile & 1)) ? (size_t)g.mt * 128 : 0);
     return f;
   }
+  // several row tiles: units run over (tile or pair of tiles, row tile, k-block)
   const int m_tile = m / g.mt, col = m - m_tile * g.mt;
-  const long long t = (long long)n_tile * m_tiles + m_tile;
-  const long long U = (long long)g.n_tiles * m_tiles * g.nkb, G = g.grid;
+  const int group = g.pair ? (n_tile >> 1) : n_tile, n_groups = g.pair ? ((g.n_tiles + 1) >> 1) : g.n_tiles;
+  f.off = (size_t)col * 128 + row + ((g.pair && (n_tile & 1)) ? (size_t)g.mt * 128 : 0);
+  if (g.small32) {   // the usual case; 64-bit divisions cost the consuming kernels more than their loads
+    const uint32_t U = (uint32_t)n_groups * m_tiles * g.nkb, G = g.grid, tu0 = ((uint32_t)group * m_tiles + m_tile) * g.nkb;
+    const uint32_t cf = ((tu0 + 1) * G - 1) / U, cl = ((tu0 + g.nkb) * G - 1) / U;
+    f.c_next = (int)(cf > G - 1 ? G - 1 : cf) + 1;
+    f.c_last = (int)(cl > G - 1 ? G - 1 : cl);
+    return f;
+  }
+  const long long t = (long long)group * m_tiles + m_tile;
+  const long long U = (long long)n_groups * m_tiles * g.nkb, G = g.grid;
   const long long tu0 = t * g.nkb;
   f.c_next = gemm_cta_of_unit(tu0, U, G) + 1;
   f.c_last = gemm_cta_of_unit(tu0 + g.nkb - 1, U, G);
-  f.off = (size_t)col * 128 + row;
   return f;
 }
 // True when CTA c has work (with fewer units than CTAs some ranges are empty).
 __device__ __forceinline__ bool gemm_has_work(const GemmOut& g, int m_tiles, int c) {
   if (g.all_work) return true;
-  const long long U = (g.pair ? (long long)((g.n_tiles + 1) >> 1) : (long long)g.n_tiles * m_tiles) * g.nkb, G = g.grid;
+  const long long U = (long long)(g.pair ? ((g.n_tiles + 1) >> 1) : g.n_tiles) * m_tiles * g.nkb, G = g.grid;
   return gemm_range_begin(c, U, G) < gemm_range_begin(c + 1, U, G);
 }
 

@@ -86,7 +86,7 @@ cudaError_t launch_gemm_simt(int dtype, const void* A, int lda, const void* W, i
                              int m_max, float* raw, int ld_raw, GemmOut* out_desc, cudaStream_t st) {
   if (out_desc) {
     out_desc->raw = raw; out_desc->partial = nullptr; out_desc->ld = ld_raw; out_desc->nkb = 1; out_desc->n_tiles = 1;
-    out_desc->mt = 1; out_desc->grid = 1; out_desc->m_tiles_max = 1; out_desc->all_work = 1; out_desc->pair = 0;
+    out_desc->mt = 1; out_desc->grid = 1; out_desc->m_tiles_max = 1; out_desc->all_work = 1; out_desc->pair = 0; out_desc->small32 = 0;
   }
   if (m_max <= 0) return cudaSuccess;
   if (m_max <= 2) {

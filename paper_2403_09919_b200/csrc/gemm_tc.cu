@@ -159,10 +159,17 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-template <bool PAIR>
+// MODE 0: one weight tile and one activation box per stage.  MODE 1 (one row tile of at most 128 rows): two adjacent
+// weight tiles per stage share one activation box, with two accumulator buffers of two tiles each.  MODE 2 (row tiles
+// of up to 256 rows, any number of them): the same pairing, a 256 x 256 output tile per unit -- the squarest tile the
+// 512 TMEM columns can hold and so the fewest operand bytes per multiply-add an SM has to pull in; its two
+// accumulators fill the tensor memory, so they are not double buffered.
+template <int MODE>
 __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
                                                                  const __grid_constant__ ActMaps maps_a,
                                                                  const TcParams p) {
+  constexpr bool PAIR = MODE >= 1, WIDE = MODE == 2;
+  constexpr uint32_t NBUF = WIDE ? 1u : 2u;   // accumulator buffers
   extern __shared__ uint8_t smem_raw[];
   pdl_launch_dependents();  // the next kernel may start its own prologue now
   if (p.trace && threadIdx.x == 0) { atomicMin(p.trace + 0, globaltimer()); }
@@ -177,7 +184,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
   }
   const int m_tiles = early ? 1 : (*p.m_total + p.mt - 1) / p.mt;
   const long long G = gridDim.x;
-  const int n_groups = PAIR ? (p.n_tiles + 1) / 2 : p.n_tiles * m_tiles;   // unit = (group, k-block)
+  const int n_groups = (PAIR ? (p.n_tiles + 1) / 2 : p.n_tiles) * m_tiles;   // unit = (tile or tile pair, row tile, k-block)
   const long long U = (long long)n_groups * p.nkb;
   const long long u0 = gemm_range_begin(blockIdx.x, U, G), u1 = gemm_range_begin(blockIdx.x + 1, U, G);
   // Rows actually present: the activation box, the MMA's N and the epilogue shrink to the next multiple of 16.
@@ -217,9 +224,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
     const int s = i % p.stages;
     mbar_expect_tx(full_bar(s), tx_bytes);
     if (PAIR) {
-      // tiles 2t and 2t+1 (the second may lie past the matrix: the copy then delivers zeros)
-      tma_load_2d_hint(base + s * stage_bytes, &map_w, full_bar(s), kb * TILE_K, (2 * t) * TILE_N, pol_w);
-      tma_load_2d_hint(base + s * stage_bytes + W_STAGE_BYTES, &map_w, full_bar(s), kb * TILE_K, (2 * t + 1) * TILE_N, pol_w);
+      // tiles 2g and 2g+1 (the second may lie past the matrix: the copy then delivers zeros)
+      const int g = WIDE ? t / m_tiles : t;
+      tma_load_2d_hint(base + s * stage_bytes, &map_w, full_bar(s), kb * TILE_K, (2 * g) * TILE_N, pol_w);
+      tma_load_2d_hint(base + s * stage_bytes + W_STAGE_BYTES, &map_w, full_bar(s), kb * TILE_K, (2 * g + 1) * TILE_N, pol_w);
     } else {
       tma_load_2d_hint(base + s * stage_bytes, &map_w, full_bar(s), kb * TILE_K, (t / m_tiles) * TILE_N, pol_w);
     }
@@ -228,7 +236,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
     const long long u = u0 + i;
     const int t = (int)(u / p.nkb), kb = (int)(u - (long long)t * p.nkb);
     const int s = i % p.stages;
-    const int m_tile = PAIR ? 0 : t - (t / m_tiles) * m_tiles;
+    const int m_tile = (PAIR && !WIDE) ? 0 : t - (t / m_tiles) * m_tiles;
     // one box of MT rows: the TMA unit's cost is per operation, not per byte, at these sizes
     tma_load_2d(base + s * stage_bytes + w_bytes, map_a, full_bar(s), kb * TILE_K, m_tile * p.mt);
   };
@@ -289,7 +297,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
       for (long long u = u0; u < u1 && ok; ++seg) {
         const int t = (int)(u / p.nkb), kb0 = (int)(u - (long long)t * p.nkb);
         const int kb1 = (int)min((long long)p.nkb, kb0 + (u1 - u));
-        const uint32_t a = seg & 1u, aph = (seg >> 1) & 1u;
+        const uint32_t a = NBUF == 2u ? (seg & 1u) : 0u, aph = NBUF == 2u ? ((seg >> 1) & 1u) : (seg & 1u);
         if (!mbar_wait(tempty_bar(a), aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t acc_cols = (uint32_t)p.mt * (PAIR ? 2u : 1u);   // columns of one accumulator buffer
@@ -332,9 +340,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
     for (long long u = u0; u < u1 && ok; ++seg) {
       const int t = (int)(u / p.nkb), kb0 = (int)(u - (long long)t * p.nkb);
       const int kb1 = (int)min((long long)p.nkb, kb0 + (u1 - u));
-      const int n_tile0 = PAIR ? 2 * t : t / m_tiles, m_tile = PAIR ? 0 : t - (t / m_tiles) * m_tiles;
-      const uint32_t a = seg & 1u, aph = (seg >> 1) & 1u;
+      const int grp = (PAIR && !WIDE) ? t : t / m_tiles, m_tile = (PAIR && !WIDE) ? 0 : t - grp * m_tiles;
+      const int n_tile0 = PAIR ? 2 * grp : grp;
       const int m_base = m_tile * p.mt;
+      const int c_end = min(mt_eff, ((M - m_base) + 15) & ~15);   // accumulator columns that hold rows of the launch
+      const uint32_t a = NBUF == 2u ? (seg & 1u) : 0u, aph = NBUF == 2u ? ((seg >> 1) & 1u) : (seg & 1u);
       // one thread does the bounded wait and tells the others, so that all 128 take the same branch
       if (et == 0) *epi_ok = mbar_wait(tfull_bar(a), aph, abort_flag, p.status) ? 1 : 0;
       epi_bar_sync();
@@ -346,7 +356,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
         const int n = (n_tile0 + sub) * TILE_N + row;
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * acc_cols + (uint32_t)sub * (uint32_t)p.mt;
         float* my_partial = p.partial + (size_t)blockIdx.x * slot_floats + (size_t)sub * p.mt * TILE_N;
-        for (int c0 = 0; c0 < mt_eff; c0 += 16) {
+        for (int c0 = 0; c0 < c_end; c0 += 16) {
           uint32_t r[16];
           tmem_ld16(taddr + c0, r);
           if (kb0 == 0) {
@@ -437,11 +447,12 @@ cudaError_t tc_prepare(int* smem_limit_out) {
   e = cudaDeviceGetAttribute(&lim, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   if (e != cudaSuccess) return e;
   cudaFuncAttributes fa;
-  e = cudaFuncGetAttributes(&fa, gemm_tc_kernel<false>);
+  e = cudaFuncGetAttributes(&fa, gemm_tc_kernel<0>);
   if (e != cudaSuccess) return e;
   lim -= (int)fa.sharedSizeBytes;  // the opt-in limit covers static + dynamic shared memory
-  e = cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
+  e = cudaFuncSetAttribute(gemm_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
   if (smem_limit_out) *smem_limit_out = lim;
   return e;
 }
@@ -453,14 +464,16 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[16], int N
   p.N = N; p.K = K; p.nkb = (K + TILE_K - 1) / TILE_K; p.n_tiles = (N + TILE_N - 1) / TILE_N;
   p.mt = tc_pick_mt(m_max > 0 ? m_max : 1);
   p.m_tiles_max = m_max > 0 ? (m_max + p.mt - 1) / p.mt : 1;
-  static const int pair_ok = getenv("RD_TC_PAIR") ? atoi(getenv("RD_TC_PAIR")) : 1;   // tuning toggle
-  p.pair = (pair && pair_ok && p.m_tiles_max == 1 && p.mt <= 128 && p.n_tiles >= 2) ? 1 : 0;
+  static const int pair_ok = getenv("RD_TC_PAIR") ? atoi(getenv("RD_TC_PAIR")) : 2;   // tuning toggle: 0 off, 1 narrow only
+  const bool wide = p.m_tiles_max > 1 || p.mt > 128;   // the accumulators of a tile pair then fill the tensor memory
+  p.pair = (pair && p.n_tiles >= 2 && pair_ok >= (wide ? 2 : 1)) ? (wide ? 2 : 1) : 0;
   const long long n_units = (long long)(p.pair ? (p.n_tiles + 1) / 2 : p.n_tiles) * p.nkb;
   if (out_desc) {
     out_desc->raw = raw; out_desc->partial = partial; out_desc->ld = ld_raw; out_desc->nkb = p.nkb;
     out_desc->n_tiles = p.n_tiles; out_desc->mt = p.mt; out_desc->grid = grid; out_desc->m_tiles_max = p.m_tiles_max;
     out_desc->all_work = (n_units >= grid) ? 1 : 0;
-    out_desc->pair = p.pair;
+    out_desc->pair = p.pair ? 1 : 0;
+    out_desc->small32 = ((n_units * p.m_tiles_max + 1) * grid < (1ll << 31)) ? 1 : 0;
   }
   if (m_max <= 0) return cudaSuccess;
   const int stage_bytes = W_STAGE_BYTES * (p.pair ? 2 : 1) + p.mt * TILE_K * 2;
@@ -476,7 +489,7 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[16], int N
   if (stages < 2) return cudaErrorInvalidConfiguration;
   p.stages = stages;
   int cols = 32;
-  while (cols < 2 * p.mt * (p.pair ? 2 : 1)) cols <<= 1;
+  while (cols < (p.pair == 2 ? 2 * p.mt : 2 * p.mt * (p.pair ? 2 : 1))) cols <<= 1;
   p.tmem_cols = cols;
   p.m_total = m_total; p.raw = raw; p.ld_raw = ld_raw; p.partial = partial; p.status = status; p.trace = trace;
   // the first launch of a chain starts after everything before it has completed (see launch_ordered)
@@ -485,12 +498,15 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[16], int N
   const size_t smem = (size_t)stages * stage_bytes + overhead;
   ActMaps am;
   for (int i = 0; i < ACT_MAPS; ++i) am.m[i] = *(const CUtensorMap*)(map_a[i] ? map_a[i] : map_a[0]);
-  if (p.pair) {
-    if (first) launch_ordered(gemm_tc_kernel<true>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
-    else launch_pdl(gemm_tc_kernel<true>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+  if (p.pair == 1) {
+    if (first) launch_ordered(gemm_tc_kernel<1>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+    else launch_pdl(gemm_tc_kernel<1>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+  } else if (p.pair == 2) {
+    if (first) launch_ordered(gemm_tc_kernel<2>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+    else launch_pdl(gemm_tc_kernel<2>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
   } else {
-    if (first) launch_ordered(gemm_tc_kernel<false>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
-    else launch_pdl(gemm_tc_kernel<false>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+    if (first) launch_ordered(gemm_tc_kernel<0>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+    else launch_pdl(gemm_tc_kernel<0>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
   }
   return cudaGetLastError();
 }

@@ -76,6 +76,11 @@ cudaError_t launch_attention(int dtype, const float* qkv, const void* kcache, co
                              const RowTables& rt, const Dims& dm, int m_max, cudaStream_t st);
 // Tensor-core attention (bf16): KV tiles staged through shared memory, split over the keys.
 size_t attn_tc_scratch_floats(int blocks, int n_splits, int hd);
+// many rows per sequence (prompts, wide beams, large batches): tiles of 64 rows, a warp per 16 of them
+int attn_wide_rows_per_block();
+cudaError_t attn_wide_prepare(int hd, int MW);
+cudaError_t launch_attention_wide(const float* qkv, const void* kcache, const void* vcache, void* out, const RowTables& rt,
+                                  const int32_t* seq_off, const Dims& dm, int n_seq, int row_tiles, Chain* chain, cudaStream_t st);
 int attn_tc_rows_per_block();
 cudaError_t attn_tc_prepare(int hd, int MW);
 cudaError_t launch_attention_tc(const float* qkv, const void* kcache, const void* vcache, void* out, const RowTables& rt,
