@@ -213,7 +213,7 @@ __global__ void __launch_bounds__(SEL_THREADS) draft_select_kernel(
   const int BW = dm.BW, L = dm.L, V = dm.V;
   const int r = blockIdx.x;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int m_tiles = gemm_m_tiles(proj, *m_total);
+  const GemmRows m_tiles = gemm_m_tiles(proj, *m_total);
   Cand* cl = wl + 32 * BW;   // [SEL_LIST_CAP] values at or above the threshold
   // ---- 1. logits into shared memory (compact loops from here on: the kernel runs once per launch,
   // so straight-line code would be bound by instruction fetch)
@@ -478,7 +478,7 @@ __global__ void __maxnreg__(88) draft_seg_kernel(GemmOut proj, int V, int BW, in
       v[k][0] = q.x; v[k][1] = q.y; v[k][2] = q.z; v[k][3] = q.w;
     }
   } else {
-    const int m_tiles = gemm_m_tiles(proj, *m_total);
+    const GemmRows m_tiles = gemm_m_tiles(proj, *m_total);
 #pragma unroll
     for (int k = 0; k < SEG_ITEMS; ++k) {
       float4 q = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);

@@ -151,7 +151,7 @@ __global__ void __maxnreg__(88)
       chain_exit(cs);
       return;
     }
-    const int m_tiles = add ? gemm_m_tiles(proj, M) : 1;
+    const GemmRows m_tiles = add ? gemm_m_tiles(proj, M) : GemmRows();
 #pragma unroll
     for (int k = 0; k < NORM_MAXV; ++k) {
       const int i = threadIdx.x + k * NORM_THREADS;
@@ -182,6 +182,77 @@ __global__ void __maxnreg__(88)
   chain_exit(cs);
 }
 
+
+// Launches of more than one row tile (prompts, wide beams, large batches).  The kernels above are built around the
+// latency of a single short pass per CTA; with thousands of rows that becomes wave after wave of CTAs that each pay
+// the hand-off poll, the row-count load and one round trip for their data.  The *_wide variants fill the SMs once
+// and walk the rows in a loop, every load of a row in flight before the first is used.
+static int wide_sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+// Partial slots loaded up front (a longer list takes the tail loop).  With more (tile pair, row tile) groups than CTAs a
+// tile is cut at most once: gate|up always, QKV mostly; O and down have few tiles, cut among several CTAs each.
+constexpr int WIDE_FOLD_NORM = 2, WIDE_FOLD_ROPE = 2, WIDE_FOLD_SWIGLU = 1;
+
+template <typename T, int NORM_MAXV>
+__global__ void __launch_bounds__(NORM_THREADS, NORM_MAXV <= 2 ? 2 : 1)
+    rmsnorm_wide_kernel(float* __restrict__ x, GemmOut proj, const T* __restrict__ gain, T* __restrict__ out_t,
+                        float* __restrict__ out_f, int d, float eps, const int32_t* __restrict__ m_total, ChainSync cs) {
+  chain_enter(cs);
+  __shared__ float sh[32];
+  const int M = *m_total;
+  const int nvec = d >> 2;
+  const bool add = proj.raw != nullptr;   // x += the projection that ends the previous block (O or down)
+  const GemmRows m_tiles = add ? gemm_m_tiles(proj, M) : GemmRows();
+  for (int m = blockIdx.x; m < M; m += gridDim.x) {
+    float4* xr = reinterpret_cast<float4*>(x + (size_t)m * d);
+    float4 v[NORM_MAXV];
+    GemmPending4<WIDE_FOLD_NORM> pd[NORM_MAXV];
+#pragma unroll
+    for (int k = 0; k < NORM_MAXV; ++k) {
+      const int i = threadIdx.x + k * NORM_THREADS;
+      if (i < nvec) {
+        v[k] = __ldcg(xr + i);
+        if (add) pd[k] = gemm_issue4<WIDE_FOLD_NORM>(proj, m_tiles, m, 4 * i);
+      }
+    }
+    float ss = 0.f;
+#pragma unroll
+    for (int k = 0; k < NORM_MAXV; ++k) {
+      const int i = threadIdx.x + k * NORM_THREADS;
+      if (i < nvec) {
+        if (add) {
+          const float4 q = gemm_finish4(proj, m_tiles, pd[k]);
+          v[k].x += q.x; v[k].y += q.y; v[k].z += q.z; v[k].w += q.w;
+          xr[i] = v[k];
+        }
+        ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
+      }
+    }
+    ss = block_sum(ss, sh);
+    const float r = rsqrtf(ss / (float)d + eps);
+#pragma unroll
+    for (int k = 0; k < NORM_MAXV; ++k) {
+      const int i = threadIdx.x + k * NORM_THREADS;
+      if (i < nvec) {
+        Gain4<T> gn;
+        gn.load(gain + 4 * i);
+        const float4 g = gn.get();
+        const float y0 = v[k].x * r * g.x, y1 = v[k].y * r * g.y, y2 = v[k].z * r * g.z, y3 = v[k].w * r * g.w;
+        const size_t o = (size_t)m * d + 4 * i;
+        if (out_t) store4(out_t + o, y0, y1, y2, y3);
+        if (out_f) *reinterpret_cast<float4*>(out_f + o) = make_float4(y0, y1, y2, y3);
+      }
+    }
+  }
+  chain_exit(cs);
+}
+
 // x: residual stream (updated in place when proj != nullptr: x += proj).
 cudaError_t launch_rmsnorm(int dtype, float* x, const GemmOut* proj, const void* gain, void* out_t, float* out_f32, int d,
                            float eps, const int32_t* m_total, int m_max, Chain* chain, cudaStream_t st) {
@@ -190,6 +261,22 @@ cudaError_t launch_rmsnorm(int dtype, float* x, const GemmOut* proj, const void*
   if (proj) g = *proj;
   // the first launch of a chain starts after everything before it has completed (see launch_ordered)
   const bool first = chain && chain->enabled && chain->prev_ptr == nullptr;
+  if (m_max > 256) {   // several row tiles
+    const int grid = m_max < 4 * wide_sm_count() ? m_max : 4 * wide_sm_count();
+    const ChainSync cs = chain ? chain->link((unsigned)grid, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
+#define RD_NORM_WIDE(MAXV)                                                                                                \
+  RD_DISPATCH(dtype, if (first) launch_ordered(rmsnorm_wide_kernel<T, MAXV>, grid, NORM_THREADS, 0, st, x, g, (const T*)gain, \
+                                               (T*)out_t, out_f32, d, eps, m_total, cs);                                  \
+              else launch_pdl(rmsnorm_wide_kernel<T, MAXV>, grid, NORM_THREADS, 0, st, x, g, (const T*)gain, (T*)out_t,    \
+                              out_f32, d, eps, m_total, cs))
+    if (d <= 4 * NORM_THREADS * 2) {
+      RD_NORM_WIDE(2);
+    } else {
+      RD_NORM_WIDE(4);
+    }
+#undef RD_NORM_WIDE
+    return cudaGetLastError();
+  }
   const ChainSync cs = chain ? chain->link((unsigned)m_max, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
 #define RD_NORM_LAUNCH(MAXV)                                                                                              \
   RD_DISPATCH(dtype, if (first) launch_ordered(rmsnorm_kernel<T, MAXV>, m_max, NORM_THREADS, 0, st, x, g, (const T*)gain,  \
@@ -308,7 +395,7 @@ __global__ void __maxnreg__(88) rope_kv_kernel(float* __restrict__ qkv, GemmOut 
     // prompt-sized launches (several row tiles) and projections shorter than the grid
     M = *rt.m_total;
     if (m < M && active) {
-      const int m_tiles = gemm_m_tiles(proj, M);
+      const GemmRows m_tiles = gemm_m_tiles(proj, M);
       b = rt.seq[m]; slot = rt.slot[m];
       const bool slot_ok = slot >= 0 && slot < dm.max_ctx;
       if (!slot_ok && idx == 0) atomicOr(status, DEV_ERR_CAPACITY);
@@ -335,10 +422,71 @@ __global__ void __maxnreg__(88) rope_kv_kernel(float* __restrict__ qkv, GemmOut 
   chain_exit(cs);
 }
 
+
+// Rows in a loop (see rmsnorm_wide_kernel): blockIdx.y picks the items of a row, blockIdx.x the first row.
+template <typename T>
+__global__ void __launch_bounds__(ROPE_THREADS, 2)
+    rope_kv_wide_kernel(float* __restrict__ qkv, GemmOut proj, T* __restrict__ kc, T* __restrict__ vc,
+                        const float2* __restrict__ table, RowTables rt, Dims dm, int* status, ChainSync cs) {
+  chain_enter(cs);
+  const int d = dm.d, hd = dm.hd, half = hd >> 1;
+  const int n_items = dm.H * (half >> 1);
+  const int idx = blockIdx.y * ROPE_THREADS + threadIdx.x;
+  const int h = idx / (half >> 1), i = (idx - h * (half >> 1)) * 2;
+  const int o = h * hd + i;
+  const int M = *rt.m_total;
+  const GemmRows m_tiles = gemm_m_tiles(proj, M);
+  if (idx < n_items) {
+    // each CTA takes a contiguous run of rows; the fold of a column changes only from one row tile to the next
+    const int m_end = gemm_rows_begin(M, gridDim.x, blockIdx.x + 1);
+    int cur_tile = -1;
+    GemmFold fq, fk, fv;
+    for (int m = gemm_rows_begin(M, gridDim.x, blockIdx.x); m < m_end; ++m) {
+      float* row = qkv + (size_t)m * 3 * d;
+      const int b = rt.seq[m], slot = rt.slot[m];
+      const float4 cs2 = *reinterpret_cast<const float4*>(table + (size_t)m * half + i);   // (cos, sin) of i and i+1
+      const int m_tile = m / m_tiles.rows;
+      const int r0 = (m - m_tile * m_tiles.rows) * 128, r1 = r0 + half;
+      if (m_tile != cur_tile) {
+        cur_tile = m_tile;
+        fq = gemm_fold_or_none(proj, m_tiles, m_tile * m_tiles.rows, o);
+        fk = gemm_fold_or_none(proj, m_tiles, m_tile * m_tiles.rows, d + o);
+        fv = gemm_fold_or_none(proj, m_tiles, m_tile * m_tiles.rows, 2 * d + o);
+      }
+      const auto pq1 = gemm_issue2<WIDE_FOLD_ROPE>(proj, m_tiles, fq, m, o, r0), pq2 = gemm_issue2<WIDE_FOLD_ROPE>(proj, m_tiles, fq, m, o + half, r1);
+      const auto pk1 = gemm_issue2<WIDE_FOLD_ROPE>(proj, m_tiles, fk, m, d + o, r0), pk2 = gemm_issue2<WIDE_FOLD_ROPE>(proj, m_tiles, fk, m, d + o + half, r1);
+      const auto pv1 = gemm_issue2<WIDE_FOLD_ROPE>(proj, m_tiles, fv, m, 2 * d + o, r0), pv2 = gemm_issue2<WIDE_FOLD_ROPE>(proj, m_tiles, fv, m, 2 * d + o + half, r1);
+      const bool slot_ok = slot >= 0 && slot < dm.max_ctx;
+      if (!slot_ok && idx == 0) atomicOr(status, DEV_ERR_CAPACITY);
+      const float2 q1 = gemm_finish2(proj, m_tiles, fq, r0, pq1), q2 = gemm_finish2(proj, m_tiles, fq, r1, pq2);
+      const float2 k1 = gemm_finish2(proj, m_tiles, fk, r0, pk1), k2 = gemm_finish2(proj, m_tiles, fk, r1, pk2);
+      const float2 v1 = gemm_finish2(proj, m_tiles, fv, r0, pv1), v2 = gemm_finish2(proj, m_tiles, fv, r1, pv2);
+      store2(row + o, q1.x * cs2.x - q2.x * cs2.y, q1.y * cs2.z - q2.y * cs2.w);
+      store2(row + o + half, q2.x * cs2.x + q1.x * cs2.y, q2.y * cs2.z + q1.y * cs2.w);
+      if (slot_ok) {
+        const size_t base = (((size_t)b * dm.H + h) * dm.max_ctx + slot) * hd + i;
+        store2(kc + base, k1.x * cs2.x - k2.x * cs2.y, k1.y * cs2.z - k2.y * cs2.w);
+        store2(kc + base + half, k2.x * cs2.x + k1.x * cs2.y, k2.y * cs2.z + k1.y * cs2.w);
+        store2(vc + base, v1.x, v1.y);
+        store2(vc + base + half, v2.x, v2.y);
+      }
+    }
+  }
+  chain_exit(cs);
+}
+
 cudaError_t launch_rope_kv(int dtype, float* qkv, const GemmOut& proj, void* kcache, void* vcache, const float* table,
                            const RowTables& rt, const Dims& dm, int m_max, int* status, Chain* chain, cudaStream_t st) {
   const int n_items = dm.H * (dm.hd / 4);
   dim3 grid(m_max, (n_items + ROPE_THREADS - 1) / ROPE_THREADS);
+  if (m_max > 256) {   // several row tiles: about four CTAs per SM walk the rows
+    const int gx = (4 * wide_sm_count() + (int)grid.y - 1) / (int)grid.y;
+    if (gx < m_max) grid.x = gx;
+    const ChainSync cs = chain ? chain->link(grid.x * grid.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
+    RD_DISPATCH(dtype, launch_pdl(rope_kv_wide_kernel<T>, grid, ROPE_THREADS, 0, st, qkv, proj, (T*)kcache, (T*)vcache,
+                                  reinterpret_cast<const float2*>(table), rt, dm, status, cs));
+    return cudaGetLastError();
+  }
   const ChainSync cs = chain ? chain->link(grid.x * grid.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
   RD_DISPATCH(dtype, launch_pdl(rope_kv_kernel<T>, grid, ROPE_THREADS, 0, st, qkv, proj, (T*)kcache, (T*)vcache,
                                 reinterpret_cast<const float2*>(table), rt, dm, status, cs));
@@ -394,7 +542,7 @@ __global__ void __maxnreg__(88) swiglu_kernel(GemmOut proj, T* __restrict__ out,
     }
   } else {
     if (m < M) {
-      const int m_tiles = gemm_m_tiles(proj, M);
+      const GemmRows m_tiles = gemm_m_tiles(proj, M);
       for (int k = 0; k < SWIGLU_ITEMS; ++k) {
         const int f = ((blockIdx.x * SWIGLU_ITEMS + k) * SWIGLU_THREADS + threadIdx.x) * 4;
         if (f < F) {
@@ -407,11 +555,60 @@ __global__ void __maxnreg__(88) swiglu_kernel(GemmOut proj, T* __restrict__ out,
   chain_exit(cs);
 }
 
+
+// Rows in a loop (see rmsnorm_wide_kernel): blockIdx.x picks the columns, blockIdx.y the first row.
+template <typename T>
+__global__ void __launch_bounds__(SWIGLU_THREADS, 6)
+    swiglu_wide_kernel(GemmOut proj, T* __restrict__ out, int F, const int32_t* __restrict__ m_total, ChainSync cs) {
+  chain_enter(cs);
+  const int M = *m_total;
+  const GemmRows m_tiles = gemm_m_tiles(proj, M);
+  const int f0 = (blockIdx.x * SWIGLU_ITEMS * SWIGLU_THREADS + threadIdx.x) * 4;
+  // each CTA takes a contiguous run of rows; the fold of a column changes only from one row tile to the next
+  const int m_end = gemm_rows_begin(M, gridDim.y, blockIdx.y + 1);
+  int cur_tile = -1;
+  GemmFold fg[SWIGLU_ITEMS], fu[SWIGLU_ITEMS];
+  for (int m = gemm_rows_begin(M, gridDim.y, blockIdx.y); m < m_end; ++m) {
+    GemmPending4f<WIDE_FOLD_SWIGLU> pg[SWIGLU_ITEMS], pu[SWIGLU_ITEMS];
+    const int m_tile = m / m_tiles.rows;
+    const size_t doff = (size_t)(m - m_tile * m_tiles.rows) * 128;
+    if (m_tile != cur_tile) {
+      cur_tile = m_tile;
+#pragma unroll
+      for (int k = 0; k < SWIGLU_ITEMS; ++k) {
+        const int f = f0 + k * SWIGLU_THREADS * 4;
+        if (f < F) { fg[k] = gemm_fold_or_none(proj, m_tiles, m_tile * m_tiles.rows, f); fu[k] = gemm_fold_or_none(proj, m_tiles, m_tile * m_tiles.rows, F + f); }
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < SWIGLU_ITEMS; ++k) {
+      const int f = f0 + k * SWIGLU_THREADS * 4;
+      if (f < F) { pg[k] = gemm_issue4f<WIDE_FOLD_SWIGLU>(proj, m_tiles, fg[k], m, f, doff); pu[k] = gemm_issue4f<WIDE_FOLD_SWIGLU>(proj, m_tiles, fu[k], m, F + f, doff); }
+    }
+#pragma unroll
+    for (int k = 0; k < SWIGLU_ITEMS; ++k) {
+      const int f = f0 + k * SWIGLU_THREADS * 4;
+      if (f < F) {
+        const float4 g = gemm_finish4f(proj, m_tiles, fg[k], doff, pg[k]), u = gemm_finish4f(proj, m_tiles, fu[k], doff, pu[k]);
+        store4(out + (size_t)m * F + f, silu_f(g.x) * u.x, silu_f(g.y) * u.y, silu_f(g.z) * u.z, silu_f(g.w) * u.w);
+      }
+    }
+  }
+  chain_exit(cs);
+}
+
 // proj: the gate|up projection [M][2F]; out: [M][F].  F must be a multiple of 4.
 cudaError_t launch_swiglu(int dtype, const GemmOut& proj, void* out_t, int F, const int32_t* m_total, int m_max,
                           Chain* chain, cudaStream_t st) {
   const int per_cta = SWIGLU_THREADS * SWIGLU_ITEMS * 4;
   dim3 grid((F + per_cta - 1) / per_cta, m_max);
+  if (m_max > 256) {   // several row tiles: about sixteen CTAs per SM walk the rows
+    const int gy = (16 * wide_sm_count() + (int)grid.x - 1) / (int)grid.x;
+    if (gy < m_max) grid.y = gy;
+    const ChainSync cs = chain ? chain->link(grid.x * grid.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
+    RD_DISPATCH(dtype, launch_pdl(swiglu_wide_kernel<T>, grid, SWIGLU_THREADS, 0, st, proj, (T*)out_t, F, m_total, cs));
+    return cudaGetLastError();
+  }
   const ChainSync cs = chain ? chain->link(grid.x * grid.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
   RD_DISPATCH(dtype, launch_pdl(swiglu_kernel<T>, grid, SWIGLU_THREADS, 0, st, proj, (T*)out_t, F, m_total, cs));
   return cudaGetLastError();
@@ -427,7 +624,7 @@ __global__ void argmax_rows_kernel(float* __restrict__ logits, GemmOut proj, int
   const int M = *m_total;
   if (m >= M) return;
   float* r = logits + (size_t)m * V;
-  const int m_tiles = gemm_m_tiles(proj, M);
+  const GemmRows m_tiles = gemm_m_tiles(proj, M);
   float bv = -INFINITY;
   int bi = 0x7fffffff;
   // the complete logits are written back in place (later readers of the buffer see final values)

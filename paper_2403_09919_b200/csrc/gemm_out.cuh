@@ -35,15 +35,30 @@ __host__ __device__ __forceinline__ int gemm_cta_of_unit(long long u, long long 
   return (int)(c > G - 1 ? G - 1 : c);
 }
 
-// Number of row tiles of a launch over M rows.
-__device__ __forceinline__ int gemm_m_tiles(const GemmOut& g, int M) { return g.m_tiles_max == 1 ? 1 : (M + g.mt - 1) / g.mt; }
+// Row tiles of a launch over M rows: their number and the rows of each.  A launch laid out for several row tiles of
+// at most g.mt rows uses the fewest tiles that hold M rows and makes them equal (a multiple of 16 rows), so that no
+// tile is mostly padding.
+struct GemmRows {
+  int n, rows;
+  __host__ __device__ GemmRows(int n_ = 1, int rows_ = 0) : n(n_), rows(rows_) {}
+};
+__host__ __device__ __forceinline__ GemmRows gemm_row_tiles(int mt, int m_tiles_max, int M) {
+  if (m_tiles_max == 1) return GemmRows(1, mt);
+  int n = (M + mt - 1) / mt;
+  if (n < 1) n = 1;
+  int rows = ((M + n - 1) / n + 15) & ~15;
+  if (rows < 16) rows = 16;
+  if (rows > mt) rows = mt;
+  return GemmRows(n, rows);
+}
+__device__ __forceinline__ GemmRows gemm_m_tiles(const GemmOut& g, int M) { return gemm_row_tiles(g.mt, g.m_tiles_max, M); }
 
 // Contributors of the tile that holds (m, n) other than the first: CTAs c_first+1 .. c_last.
 struct GemmFold {
   int c_next, c_last;   // first non-first contributor, last contributor
   size_t off;           // element offset of (m, n) inside a slot
 };
-__device__ __forceinline__ GemmFold gemm_fold(const GemmOut& g, int m_tiles, int m, int n) {
+__device__ __forceinline__ GemmFold gemm_fold(const GemmOut& g, GemmRows m_tiles, int m, int n) {
   const int n_tile = n >> 7, row = n & 127;
   GemmFold f;
   if (g.m_tiles_max == 1) {
@@ -59,27 +74,27 @@ __device__ __forceinline__ GemmFold gemm_fold(const GemmOut& g, int m_tiles, int
     return f;
   }
   // several row tiles: units run over (tile or pair of tiles, row tile, k-block)
-  const int m_tile = m / g.mt, col = m - m_tile * g.mt;
+  const int m_tile = m / m_tiles.rows, col = m - m_tile * m_tiles.rows;
   const int group = g.pair ? (n_tile >> 1) : n_tile, n_groups = g.pair ? ((g.n_tiles + 1) >> 1) : g.n_tiles;
   f.off = (size_t)col * 128 + row + ((g.pair && (n_tile & 1)) ? (size_t)g.mt * 128 : 0);
   if (g.small32) {   // the usual case; 64-bit divisions cost the consuming kernels more than their loads
-    const uint32_t U = (uint32_t)n_groups * m_tiles * g.nkb, G = g.grid, tu0 = ((uint32_t)group * m_tiles + m_tile) * g.nkb;
+    const uint32_t U = (uint32_t)n_groups * m_tiles.n * g.nkb, G = g.grid, tu0 = ((uint32_t)group * m_tiles.n + m_tile) * g.nkb;
     const uint32_t cf = ((tu0 + 1) * G - 1) / U, cl = ((tu0 + g.nkb) * G - 1) / U;
     f.c_next = (int)(cf > G - 1 ? G - 1 : cf) + 1;
     f.c_last = (int)(cl > G - 1 ? G - 1 : cl);
     return f;
   }
-  const long long t = (long long)group * m_tiles + m_tile;
-  const long long U = (long long)n_groups * m_tiles * g.nkb, G = g.grid;
+  const long long t = (long long)group * m_tiles.n + m_tile;
+  const long long U = (long long)n_groups * m_tiles.n * g.nkb, G = g.grid;
   const long long tu0 = t * g.nkb;
   f.c_next = gemm_cta_of_unit(tu0, U, G) + 1;
   f.c_last = gemm_cta_of_unit(tu0 + g.nkb - 1, U, G);
   return f;
 }
 // True when CTA c has work (with fewer units than CTAs some ranges are empty).
-__device__ __forceinline__ bool gemm_has_work(const GemmOut& g, int m_tiles, int c) {
+__device__ __forceinline__ bool gemm_has_work(const GemmOut& g, GemmRows m_tiles, int c) {
   if (g.all_work) return true;
-  const long long U = (long long)(g.pair ? ((g.n_tiles + 1) >> 1) : g.n_tiles) * m_tiles * g.nkb, G = g.grid;
+  const long long U = (long long)(g.pair ? ((g.n_tiles + 1) >> 1) : g.n_tiles) * m_tiles.n * g.nkb, G = g.grid;
   return gemm_range_begin(c, U, G) < gemm_range_begin(c + 1, U, G);
 }
 
@@ -103,7 +118,7 @@ struct GemmPending4 {
 };
 
 template <int U>
-__device__ __forceinline__ GemmPending<U> gemm_issue(const GemmOut& g, int m_tiles, int m, int n) {
+__device__ __forceinline__ GemmPending<U> gemm_issue(const GemmOut& g, GemmRows m_tiles, int m, int n) {
   GemmPending<U> p;
   p.raw = g.raw[(size_t)m * g.ld + n];
   p.f.c_next = 1; p.f.c_last = 0; p.f.off = 0;
@@ -117,7 +132,7 @@ __device__ __forceinline__ GemmPending<U> gemm_issue(const GemmOut& g, int m_til
   return p;
 }
 template <int U>
-__device__ __forceinline__ float gemm_finish(const GemmOut& g, int m_tiles, const GemmPending<U>& p) {
+__device__ __forceinline__ float gemm_finish(const GemmOut& g, GemmRows m_tiles, const GemmPending<U>& p) {
   float v = p.raw;
 #pragma unroll
   for (int j = 0; j < U; ++j) v += p.q[j];
@@ -128,7 +143,7 @@ __device__ __forceinline__ float gemm_finish(const GemmOut& g, int m_tiles, cons
 }
 // Four consecutive columns n .. n+3 (n a multiple of 4: they share a tile and the slots' alignment).
 template <int U>
-__device__ __forceinline__ GemmPending4<U> gemm_issue4(const GemmOut& g, int m_tiles, int m, int n) {
+__device__ __forceinline__ GemmPending4<U> gemm_issue4(const GemmOut& g, GemmRows m_tiles, int m, int n) {
   GemmPending4<U> p;
   p.raw = *reinterpret_cast<const float4*>(g.raw + (size_t)m * g.ld + n);
   p.f.c_next = 1; p.f.c_last = 0; p.f.off = 0;
@@ -144,7 +159,7 @@ __device__ __forceinline__ GemmPending4<U> gemm_issue4(const GemmOut& g, int m_t
   return p;
 }
 template <int U>
-__device__ __forceinline__ float4 gemm_finish4(const GemmOut& g, int m_tiles, const GemmPending4<U>& p) {
+__device__ __forceinline__ float4 gemm_finish4(const GemmOut& g, GemmRows m_tiles, const GemmPending4<U>& p) {
   float4 v = p.raw;
 #pragma unroll
   for (int j = 0; j < U; ++j) { v.x += p.q[j].x; v.y += p.q[j].y; v.z += p.q[j].z; v.w += p.q[j].w; }
@@ -160,7 +175,7 @@ __device__ __forceinline__ float4 gemm_finish4(const GemmOut& g, int m_tiles, co
 // Two consecutive columns n, n+1 (n even) of row m, with the fold of a column of the same tile already
 // computed: `doff` is n minus the column the fold was made for.  Lets a kernel that reads several column
 // pairs of one tile (the two halves of a rotary pair) pay for the fold once.
-__device__ __forceinline__ GemmFold gemm_fold_or_none(const GemmOut& g, int m_tiles, int m, int n) {
+__device__ __forceinline__ GemmFold gemm_fold_or_none(const GemmOut& g, GemmRows m_tiles, int m, int n) {
   GemmFold f;
   f.c_next = 1; f.c_last = 0; f.off = 0;
   if (g.partial != nullptr) f = gemm_fold(g, m_tiles, m, n);
@@ -172,7 +187,7 @@ struct GemmPending2 {
   float2 q[U];
 };
 template <int U>
-__device__ __forceinline__ GemmPending2<U> gemm_issue2(const GemmOut& g, int m_tiles, const GemmFold& f, int m, int n, int doff) {
+__device__ __forceinline__ GemmPending2<U> gemm_issue2(const GemmOut& g, GemmRows m_tiles, const GemmFold& f, int m, int n, int doff) {
   GemmPending2<U> p;
   p.raw = __ldcg(reinterpret_cast<const float2*>(g.raw + (size_t)m * g.ld + n));
   const size_t slot = gemm_slot_stride(g);
@@ -186,7 +201,7 @@ __device__ __forceinline__ GemmPending2<U> gemm_issue2(const GemmOut& g, int m_t
   return p;
 }
 template <int U>
-__device__ __forceinline__ float2 gemm_finish2(const GemmOut& g, int m_tiles, const GemmFold& f, int doff, const GemmPending2<U>& p) {
+__device__ __forceinline__ float2 gemm_finish2(const GemmOut& g, GemmRows m_tiles, const GemmFold& f, int doff, const GemmPending2<U>& p) {
   float2 v = p.raw;
 #pragma unroll
   for (int j = 0; j < U; ++j) { v.x += p.q[j].x; v.y += p.q[j].y; }
@@ -211,7 +226,7 @@ struct GemmSrc {
 };
 // Valid for launches where every CTA has work (all_work), which is every launch whose stream is at
 // least as long as the grid; callers fall back to gemm_value* otherwise.
-__device__ __forceinline__ GemmSrc gemm_src(const GemmOut& g, int m_tiles, int m, int n) {
+__device__ __forceinline__ GemmSrc gemm_src(const GemmOut& g, GemmRows m_tiles, int m, int n) {
   GemmSrc s;
   s.raw = g.raw + (size_t)m * g.ld + n;
   s.part = g.partial;
@@ -285,12 +300,49 @@ __device__ __forceinline__ float2 gemm_sum2(const GemmSrc& s, size_t stride, con
 }
 
 // One-shot forms.
-__device__ __forceinline__ float gemm_value(const GemmOut& g, int m_tiles, int m, int n) {
+__device__ __forceinline__ float gemm_value(const GemmOut& g, GemmRows m_tiles, int m, int n) {
   return gemm_finish(g, m_tiles, gemm_issue<GEMM_FOLD_UNROLL>(g, m_tiles, m, n));
 }
 template <int U = GEMM_FOLD_UNROLL>
-__device__ __forceinline__ float4 gemm_value4(const GemmOut& g, int m_tiles, int m, int n) {
+__device__ __forceinline__ float4 gemm_value4(const GemmOut& g, GemmRows m_tiles, int m, int n) {
   return gemm_finish4(g, m_tiles, gemm_issue4<U>(g, m_tiles, m, n));
 }
+
+// Four consecutive columns with the fold worked out by the caller (a kernel that walks the rows of one row tile
+// computes it once per tile: only the offset inside the slot, doff, changes from row to row).
+template <int U>
+struct GemmPending4f {
+  float4 raw;
+  float4 q[U];
+};
+template <int U>
+__device__ __forceinline__ GemmPending4f<U> gemm_issue4f(const GemmOut& g, GemmRows m_tiles, const GemmFold& f, int m, int n, size_t doff) {
+  GemmPending4f<U> p;
+  p.raw = __ldcg(reinterpret_cast<const float4*>(g.raw + (size_t)m * g.ld + n));
+  const size_t slot = gemm_slot_stride(g);
+#pragma unroll
+  for (int j = 0; j < U; ++j) {
+    const int c = f.c_next + j;
+    p.q[j] = (c <= f.c_last && gemm_has_work(g, m_tiles, c))
+                 ? __ldcg(reinterpret_cast<const float4*>(g.partial + (size_t)c * slot + f.off + doff))
+                 : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  return p;
+}
+template <int U>
+__device__ __forceinline__ float4 gemm_finish4f(const GemmOut& g, GemmRows m_tiles, const GemmFold& f, size_t doff, const GemmPending4f<U>& p) {
+  float4 v = p.raw;
+#pragma unroll
+  for (int j = 0; j < U; ++j) { v.x += p.q[j].x; v.y += p.q[j].y; v.z += p.q[j].z; v.w += p.q[j].w; }
+  const size_t slot = gemm_slot_stride(g);
+  for (int c = f.c_next + U; c <= f.c_last; ++c) {
+    if (!gemm_has_work(g, m_tiles, c)) continue;
+    const float4 t = __ldcg(reinterpret_cast<const float4*>(g.partial + (size_t)c * slot + f.off + doff));
+    v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
+  }
+  return v;
+}
+// Rows [begin, end) of a kernel that splits M rows evenly over `parts` CTAs, part `i`.
+__device__ __forceinline__ int gemm_rows_begin(int M, int parts, int i) { return (int)((long long)M * i / parts); }
 
 }  // namespace rd

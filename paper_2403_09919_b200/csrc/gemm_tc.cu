@@ -182,7 +182,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
     if (threadIdx.x == 0) chain_wait_thread(p.cs);
     __syncthreads();
   }
-  const int m_tiles = early ? 1 : (*p.m_total + p.mt - 1) / p.mt;
+  const GemmRows rows = early ? GemmRows(1, p.mt) : gemm_row_tiles(p.mt, p.m_tiles_max, *p.m_total);
+  const int m_tiles = rows.n;
   const long long G = gridDim.x;
   const int n_groups = (PAIR ? (p.n_tiles + 1) / 2 : p.n_tiles) * m_tiles;   // unit = (tile or tile pair, row tile, k-block)
   const long long U = (long long)n_groups * p.nkb;
@@ -190,8 +191,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
   // Rows actually present: the activation box, the MMA's N and the epilogue shrink to the next multiple of 16.
   // Every byte of the activation operand is fetched once per weight tile, so at 48 rows it is more than a third
   // of what an SM has to pull in; the row count is known before the chain starts, so it may be read at once.
+  // Several row tiles are made equal (the fewest tiles that hold the rows, each a multiple of 16 rows).
   int mt_eff = p.mt;
-  if ((early && p.cs.signal_ptr != nullptr) || (!early && m_tiles == 1)) {
+  if (!early) {
+    mt_eff = rows.rows;
+  } else if (p.cs.signal_ptr != nullptr) {
     const int M = *p.m_total;
     mt_eff = min(p.mt, max(16, (M + 15) & ~15));
   }
@@ -218,27 +222,43 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
   const uint32_t n_it = (uint32_t)(u1 - u0);
   const uint32_t pre = early ? min(n_it, (uint32_t)p.stages) : 0u;
   const uint64_t pol_w = l2_policy_evict_first();
-  auto issue_w = [&](uint32_t i) {
-    const long long u = u0 + i;
-    const int t = (int)(u / p.nkb), kb = (int)(u - (long long)t * p.nkb);
-    const int s = i % p.stages;
-    mbar_expect_tx(full_bar(s), tx_bytes);
+  // Position of the producer in its unit range, advanced without divisions: the producer is a single thread, and
+  // a division by a run-time value is a chain of a hundred dependent instructions -- several of them per stage
+  // would bound the rate at which stages are issued.
+  struct UnitPos {
+    int g, m_tile, kb;     // weight tile (or tile pair), row tile, k-block
+    uint32_t s, ph;        // ring slot and the parity of its current use
+  };
+  auto pos_at = [&](long long u) {
+    UnitPos q;
+    const int t = (int)(u / p.nkb);
+    q.kb = (int)(u - (long long)t * p.nkb);
+    q.g = (PAIR && !WIDE) ? t : t / m_tiles;
+    q.m_tile = (PAIR && !WIDE) ? 0 : t - q.g * m_tiles;
+    q.s = 0; q.ph = 0;
+    return q;
+  };
+  auto advance = [&](UnitPos& q) {
+    if (++q.kb == p.nkb) {
+      q.kb = 0;
+      if ((PAIR && !WIDE) || ++q.m_tile == m_tiles) { q.m_tile = 0; ++q.g; }
+    }
+    if (++q.s == (uint32_t)p.stages) { q.s = 0; q.ph ^= 1u; }
+  };
+  auto issue_w = [&](const UnitPos& q) {
+    const uint32_t dst = base + q.s * stage_bytes;
+    mbar_expect_tx(full_bar(q.s), tx_bytes);
     if (PAIR) {
       // tiles 2g and 2g+1 (the second may lie past the matrix: the copy then delivers zeros)
-      const int g = WIDE ? t / m_tiles : t;
-      tma_load_2d_hint(base + s * stage_bytes, &map_w, full_bar(s), kb * TILE_K, (2 * g) * TILE_N, pol_w);
-      tma_load_2d_hint(base + s * stage_bytes + W_STAGE_BYTES, &map_w, full_bar(s), kb * TILE_K, (2 * g + 1) * TILE_N, pol_w);
+      tma_load_2d_hint(dst, &map_w, full_bar(q.s), q.kb * TILE_K, (2 * q.g) * TILE_N, pol_w);
+      tma_load_2d_hint(dst + W_STAGE_BYTES, &map_w, full_bar(q.s), q.kb * TILE_K, (2 * q.g + 1) * TILE_N, pol_w);
     } else {
-      tma_load_2d_hint(base + s * stage_bytes, &map_w, full_bar(s), kb * TILE_K, (t / m_tiles) * TILE_N, pol_w);
+      tma_load_2d_hint(dst, &map_w, full_bar(q.s), q.kb * TILE_K, q.g * TILE_N, pol_w);
     }
   };
-  auto issue_a = [&](uint32_t i) {
-    const long long u = u0 + i;
-    const int t = (int)(u / p.nkb), kb = (int)(u - (long long)t * p.nkb);
-    const int s = i % p.stages;
-    const int m_tile = (PAIR && !WIDE) ? 0 : t - (t / m_tiles) * m_tiles;
+  auto issue_a = [&](const UnitPos& q) {
     // one box of MT rows: the TMA unit's cost is per operation, not per byte, at these sizes
-    tma_load_2d(base + s * stage_bytes + w_bytes, map_a, full_bar(s), kb * TILE_K, m_tile * p.mt);
+    tma_load_2d(base + q.s * stage_bytes + w_bytes, map_a, full_bar(q.s), q.kb * TILE_K, q.m_tile * mt_eff);
   };
 
   if (threadIdx.x == 0) {
@@ -252,7 +272,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    for (uint32_t i = 0; i < pre; ++i) issue_w(i);
+    UnitPos q = pos_at(u0);
+    for (uint32_t i = 0; i < pre; ++i) { issue_w(q); advance(q); }
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
@@ -274,14 +295,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
       if (p.trace) { atomicMin(p.trace + 1, globaltimer()); atomicMax(p.trace + 2, globaltimer()); }   // dependency resolved
       // an earlier launch of the step gave up on a wait: wind this one down through the roles' abort paths
       if (*(volatile int32_t*)p.status & DEV_ERR_TIMEOUT) *abort_flag = 1;
-      for (uint32_t i = 0; i < pre; ++i) issue_a(i);
+      UnitPos q = pos_at(u0);
+      for (uint32_t i = 0; i < pre; ++i) { issue_a(q); advance(q); }
       bool ok = true;
       for (uint32_t i = pre; i < n_it; ++i) {
-        const int s = i % p.stages;
-        const uint32_t ph = (i / p.stages) & 1u;
-        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-        issue_w(i);
-        issue_a(i);
+        if (!mbar_wait(empty_bar(q.s), q.ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        issue_w(q);
+        issue_a(q);
+        advance(q);
       }
       if (!ok || *abort_flag) {  // give the copies already issued time to land before the CTA's shared memory is released
         const unsigned long long t0 = globaltimer();
@@ -292,7 +313,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
     // ===================== MMA issuer =====================
     if (lane == 0 && u0 < u1) {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(mt_eff >> 3) << 17) | ((uint32_t)(TILE_N >> 4) << 24);
-      uint32_t it = 0, seg = 0;
+      uint32_t seg = 0, s = 0, ph = 0;   // ring slot and parity, advanced without divisions
       bool ok = true;
       for (long long u = u0; u < u1 && ok; ++seg) {
         const int t = (int)(u / p.nkb), kb0 = (int)(u - (long long)t * p.nkb);
@@ -302,9 +323,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
         tc_fence_after();
         const uint32_t acc_cols = (uint32_t)p.mt * (PAIR ? 2u : 1u);   // columns of one accumulator buffer
         const uint32_t d_tmem = tmem_base + a * acc_cols;
-        for (int kb = kb0; kb < kb1; ++kb, ++it) {
-          const int s = it % p.stages;
-          const uint32_t ph = (it / p.stages) & 1u;
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full_bar(s), ph, abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
           const uint64_t wdesc = umma_desc(base + s * stage_bytes);
@@ -319,6 +338,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
               umma_bf16(d_tmem + (uint32_t)p.mt, wdesc2 + 2 * k, adesc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
           }
           umma_commit(empty_bar(s));  // the stage is free once these MMAs have read it
+          if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; }
         }
         if (ok) umma_commit(tfull_bar(a));
         u += kb1 - kb0;
@@ -342,7 +362,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
       const int kb1 = (int)min((long long)p.nkb, kb0 + (u1 - u));
       const int grp = (PAIR && !WIDE) ? t : t / m_tiles, m_tile = (PAIR && !WIDE) ? 0 : t - grp * m_tiles;
       const int n_tile0 = PAIR ? 2 * grp : grp;
-      const int m_base = m_tile * p.mt;
+      const int m_base = m_tile * mt_eff;
       const int c_end = min(mt_eff, ((M - m_base) + 15) & ~15);   // accumulator columns that hold rows of the launch
       const uint32_t a = NBUF == 2u ? (seg & 1u) : 0u, aph = NBUF == 2u ? ((seg >> 1) & 1u) : (seg & 1u);
       // one thread does the bounded wait and tells the others, so that all 128 take the same branch
