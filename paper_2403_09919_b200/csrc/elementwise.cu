@@ -109,18 +109,21 @@ __global__ void __maxnreg__(88)
   // Decode-time launches (one row tile, no idle CTA in the projection): every address is worked out while
   // waiting, and the row's loads do not wait for the row count (rows past it exist in memory and are
   // simply not written back).
-  const bool fast = add && proj.m_tiles_max == 1 && (proj.partial == nullptr || proj.all_work);
+  // (A launch laid out for several row tiles whose rows fit one after all is a single-tile launch; inside a
+  // chain the row count is known up front.)
+  int M = early ? *m_total : 0;
+  const bool single = proj.m_tiles_max == 1 || (early && M <= proj.mt);
+  const bool fast = add && single && (proj.partial == nullptr || proj.all_work);
   const size_t stride = add ? gemm_slot_stride(proj) : 0;
   GemmSrc src[NORM_MAXV];
   if (fast) {
 #pragma unroll
     for (int k = 0; k < NORM_MAXV; ++k) {
       const int i = threadIdx.x + k * NORM_THREADS;
-      if (i < nvec) { src[k] = gemm_src(proj, 1, m, 4 * i); gemm_src_pin(src[k]); }
+      if (i < nvec) { src[k] = gemm_src(proj, GemmRows(1, proj.mt), m, 4 * i); gemm_src_pin(src[k]); }
     }
     asm volatile("" : "+l"(xr));
   }
-  int M = early ? *m_total : 0;
   chain_wait_cta(cs);
   if (!early) M = *m_total;
   float4 v[NORM_MAXV];
@@ -187,6 +190,9 @@ __global__ void __maxnreg__(88)
 // latency of a single short pass per CTA; with thousands of rows that becomes wave after wave of CTAs that each pay
 // the hand-off poll, the row-count load and one round trip for their data.  The *_wide variants fill the SMs once
 // and walk the rows in a loop, every load of a row in flight before the first is used.
+// The row-loop variants take over where the host-side bound on the rows exceeds one and a half row tiles: below that the
+// rows actually present mostly fit a single tile, which the kernels above handle on their fast path.
+constexpr int WIDE_ROWS_MIN = 384;
 static int wide_sm_count() {
   static int n = 0;
   if (!n) {
@@ -261,7 +267,7 @@ cudaError_t launch_rmsnorm(int dtype, float* x, const GemmOut* proj, const void*
   if (proj) g = *proj;
   // the first launch of a chain starts after everything before it has completed (see launch_ordered)
   const bool first = chain && chain->enabled && chain->prev_ptr == nullptr;
-  if (m_max > 256) {   // several row tiles
+  if (m_max > WIDE_ROWS_MIN) {   // several row tiles
     const int grid = m_max < 4 * wide_sm_count() ? m_max : 4 * wide_sm_count();
     const ChainSync cs = chain ? chain->link((unsigned)grid, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
 #define RD_NORM_WIDE(MAXV)                                                                                                \
@@ -351,12 +357,13 @@ __global__ void __maxnreg__(88) rope_kv_kernel(float* __restrict__ qkv, GemmOut 
   float* row = qkv + (size_t)m * 3 * d;
   // decode-time launches (one row tile, no idle CTA in the projection): every address is known before the
   // projection has produced anything
-  const bool fast = proj.m_tiles_max == 1 && (proj.partial == nullptr || proj.all_work);
+  const bool single = proj.m_tiles_max == 1 || (early && *rt.m_total <= proj.mt);   // rows that fit one row tile after all
+  const bool fast = single && (proj.partial == nullptr || proj.all_work);
   GemmSrc sq, sk, sv;
   const size_t stride = gemm_slot_stride(proj);
   const float2* tab = table + (size_t)m * half + i;
   if (fast && active) {
-    sq = gemm_src(proj, 1, m, o); sk = gemm_src(proj, 1, m, d + o); sv = gemm_src(proj, 1, m, 2 * d + o);
+    sq = gemm_src(proj, GemmRows(1, proj.mt), m, o); sk = gemm_src(proj, GemmRows(1, proj.mt), m, d + o); sv = gemm_src(proj, GemmRows(1, proj.mt), m, 2 * d + o);
     gemm_src_pin(sq); gemm_src_pin(sk); gemm_src_pin(sv);
     asm volatile("" : "+l"(tab), "+l"(row));
   }
@@ -479,7 +486,7 @@ cudaError_t launch_rope_kv(int dtype, float* qkv, const GemmOut& proj, void* kca
                            const RowTables& rt, const Dims& dm, int m_max, int* status, Chain* chain, cudaStream_t st) {
   const int n_items = dm.H * (dm.hd / 4);
   dim3 grid(m_max, (n_items + ROPE_THREADS - 1) / ROPE_THREADS);
-  if (m_max > 256) {   // several row tiles: about four CTAs per SM walk the rows
+  if (m_max > WIDE_ROWS_MIN) {   // several row tiles: about four CTAs per SM walk the rows
     const int gx = (4 * wide_sm_count() + (int)grid.y - 1) / (int)grid.y;
     if (gx < m_max) grid.x = gx;
     const ChainSync cs = chain ? chain->link(grid.x * grid.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
@@ -509,9 +516,10 @@ __global__ void __maxnreg__(88) swiglu_kernel(GemmOut proj, T* __restrict__ out,
   const bool early = cs.signal_ptr != nullptr;   // inside a chain the row count (written ahead of it) may be read now
   if (!early) chain_wait_cta(cs);
   const int m = blockIdx.y;
-  const bool fast = proj.m_tiles_max == 1 && (proj.partial == nullptr || proj.all_work);
   const size_t stride = gemm_slot_stride(proj);
   const int M = *m_total;
+  const bool single = proj.m_tiles_max == 1 || M <= proj.mt;   // rows that fit one row tile after all
+  const bool fast = single && (proj.partial == nullptr || proj.all_work);
   GemmSrc sg[SWIGLU_ITEMS], su[SWIGLU_ITEMS];
   T* dst[SWIGLU_ITEMS];
   bool act[SWIGLU_ITEMS];
@@ -521,7 +529,7 @@ __global__ void __maxnreg__(88) swiglu_kernel(GemmOut proj, T* __restrict__ out,
     act[k] = f < F;
     dst[k] = out + (size_t)m * F + f;
     if (fast && act[k]) {
-      sg[k] = gemm_src(proj, 1, m, f); su[k] = gemm_src(proj, 1, m, F + f);
+      sg[k] = gemm_src(proj, GemmRows(1, proj.mt), m, f); su[k] = gemm_src(proj, GemmRows(1, proj.mt), m, F + f);
       gemm_src_pin(sg[k]); gemm_src_pin(su[k]);
       asm volatile("" : "+l"(dst[k]));
     }
@@ -602,7 +610,7 @@ cudaError_t launch_swiglu(int dtype, const GemmOut& proj, void* out_t, int F, co
                           Chain* chain, cudaStream_t st) {
   const int per_cta = SWIGLU_THREADS * SWIGLU_ITEMS * 4;
   dim3 grid((F + per_cta - 1) / per_cta, m_max);
-  if (m_max > 256) {   // several row tiles: about sixteen CTAs per SM walk the rows
+  if (m_max > WIDE_ROWS_MIN) {   // several row tiles: about sixteen CTAs per SM walk the rows
     const int gy = (16 * wide_sm_count() + (int)grid.x - 1) / (int)grid.x;
     if (gy < m_max) grid.y = gy;
     const ChainSync cs = chain ? chain->link(grid.x * grid.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};

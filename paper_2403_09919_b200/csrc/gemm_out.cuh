@@ -61,7 +61,7 @@ struct GemmFold {
 __device__ __forceinline__ GemmFold gemm_fold(const GemmOut& g, GemmRows m_tiles, int m, int n) {
   const int n_tile = n >> 7, row = n & 127;
   GemmFold f;
-  if (g.m_tiles_max == 1) {
+  if (m_tiles.n == 1) {
     // one row tile (the decode-time case): 32-bit arithmetic, (units + 1) * CTAs stays far below 2^31
     // (in pair mode the units run over pairs of tiles, and the odd tile sits in the second half of a slot)
     const uint32_t group = g.pair ? (uint32_t)(n_tile >> 1) : (uint32_t)n_tile;

@@ -159,17 +159,14 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-// MODE 0: one weight tile and one activation box per stage.  MODE 1 (one row tile of at most 128 rows): two adjacent
-// weight tiles per stage share one activation box, with two accumulator buffers of two tiles each.  MODE 2 (row tiles
-// of up to 256 rows, any number of them): the same pairing, a 256 x 256 output tile per unit -- the squarest tile the
-// 512 TMEM columns can hold and so the fewest operand bytes per multiply-add an SM has to pull in; its two
-// accumulators fill the tensor memory, so they are not double buffered.
-template <int MODE>
+// PAIR (one row tile of at most 128 rows): two adjacent weight tiles per stage share one activation box, and an
+// accumulator buffer holds both tiles.  Measured and dropped: the same pairing at up to 256 rows and with several
+// row tiles (a 256 x 256 output tile per unit).  Its two accumulators fill the tensor memory, so the epilogue no
+// longer overlaps the next tile's MMAs, and that costs what the shared activation box saves.
+template <bool PAIR>
 __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
                                                                  const __grid_constant__ ActMaps maps_a,
                                                                  const TcParams p) {
-  constexpr bool PAIR = MODE >= 1, WIDE = MODE == 2;
-  constexpr uint32_t NBUF = WIDE ? 1u : 2u;   // accumulator buffers
   extern __shared__ uint8_t smem_raw[];
   pdl_launch_dependents();  // the next kernel may start its own prologue now
   if (p.trace && threadIdx.x == 0) { atomicMin(p.trace + 0, globaltimer()); }
@@ -177,28 +174,27 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // With a single row tile the work split does not depend on the row count, so the weight stream can
   // start before the preceding kernels have finished (they produce the activations and the row count).
-  const bool early = (p.m_tiles_max == 1);
+  // Inside a chain the row count was written ahead of the chain's first launch and may be read at once,
+  // so the same holds for any number of row tiles.
+  const bool chained = p.cs.signal_ptr != nullptr;
+  const bool early = (p.m_tiles_max == 1) || chained;
   if (!early) {
     if (threadIdx.x == 0) chain_wait_thread(p.cs);
     __syncthreads();
   }
-  const GemmRows rows = early ? GemmRows(1, p.mt) : gemm_row_tiles(p.mt, p.m_tiles_max, *p.m_total);
+  // Rows actually present: the activation box, the MMA's N and the epilogue shrink to the next multiple of 16.
+  // Every byte of the activation operand is fetched once per weight tile, so at 48 rows it is more than a third
+  // of what an SM has to pull in.  (A single row tile outside a chain keeps the full box: its row count is not
+  // known yet.)
+  GemmRows rows(1, p.mt);
+  if (p.m_tiles_max > 1) rows = gemm_row_tiles(p.mt, p.m_tiles_max, *p.m_total);
+  else if (chained) rows.rows = min(p.mt, max(16, (*p.m_total + 15) & ~15));
   const int m_tiles = rows.n;
   const long long G = gridDim.x;
   const int n_groups = (PAIR ? (p.n_tiles + 1) / 2 : p.n_tiles) * m_tiles;   // unit = (tile or tile pair, row tile, k-block)
   const long long U = (long long)n_groups * p.nkb;
   const long long u0 = gemm_range_begin(blockIdx.x, U, G), u1 = gemm_range_begin(blockIdx.x + 1, U, G);
-  // Rows actually present: the activation box, the MMA's N and the epilogue shrink to the next multiple of 16.
-  // Every byte of the activation operand is fetched once per weight tile, so at 48 rows it is more than a third
-  // of what an SM has to pull in; the row count is known before the chain starts, so it may be read at once.
-  // Several row tiles are made equal (the fewest tiles that hold the rows, each a multiple of 16 rows).
-  int mt_eff = p.mt;
-  if (!early) {
-    mt_eff = rows.rows;
-  } else if (p.cs.signal_ptr != nullptr) {
-    const int M = *p.m_total;
-    mt_eff = min(p.mt, max(16, (M + 15) & ~15));
-  }
+  const int mt_eff = rows.rows;   // several row tiles are equal: the fewest that hold the rows, each a multiple of 16 rows
   const CUtensorMap* map_a = &maps_a.m[(mt_eff >> 4) - 1];
 
   // ---- shared memory carve-up (stage buffers 1024-byte aligned for the 128-byte swizzle)
@@ -233,15 +229,15 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
     UnitPos q;
     const int t = (int)(u / p.nkb);
     q.kb = (int)(u - (long long)t * p.nkb);
-    q.g = (PAIR && !WIDE) ? t : t / m_tiles;
-    q.m_tile = (PAIR && !WIDE) ? 0 : t - q.g * m_tiles;
+    q.g = PAIR ? t : t / m_tiles;
+    q.m_tile = PAIR ? 0 : t - q.g * m_tiles;
     q.s = 0; q.ph = 0;
     return q;
   };
   auto advance = [&](UnitPos& q) {
     if (++q.kb == p.nkb) {
       q.kb = 0;
-      if ((PAIR && !WIDE) || ++q.m_tile == m_tiles) { q.m_tile = 0; ++q.g; }
+      if (PAIR || ++q.m_tile == m_tiles) { q.m_tile = 0; ++q.g; }
     }
     if (++q.s == (uint32_t)p.stages) { q.s = 0; q.ph ^= 1u; }
   };
@@ -318,7 +314,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
       for (long long u = u0; u < u1 && ok; ++seg) {
         const int t = (int)(u / p.nkb), kb0 = (int)(u - (long long)t * p.nkb);
         const int kb1 = (int)min((long long)p.nkb, kb0 + (u1 - u));
-        const uint32_t a = NBUF == 2u ? (seg & 1u) : 0u, aph = NBUF == 2u ? ((seg >> 1) & 1u) : (seg & 1u);
+        const uint32_t a = seg & 1u, aph = (seg >> 1) & 1u;
         if (!mbar_wait(tempty_bar(a), aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t acc_cols = (uint32_t)p.mt * (PAIR ? 2u : 1u);   // columns of one accumulator buffer
@@ -360,11 +356,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
     for (long long u = u0; u < u1 && ok; ++seg) {
       const int t = (int)(u / p.nkb), kb0 = (int)(u - (long long)t * p.nkb);
       const int kb1 = (int)min((long long)p.nkb, kb0 + (u1 - u));
-      const int grp = (PAIR && !WIDE) ? t : t / m_tiles, m_tile = (PAIR && !WIDE) ? 0 : t - grp * m_tiles;
+      const int grp = PAIR ? t : t / m_tiles, m_tile = PAIR ? 0 : t - grp * m_tiles;
       const int n_tile0 = PAIR ? 2 * grp : grp;
       const int m_base = m_tile * mt_eff;
       const int c_end = min(mt_eff, ((M - m_base) + 15) & ~15);   // accumulator columns that hold rows of the launch
-      const uint32_t a = NBUF == 2u ? (seg & 1u) : 0u, aph = NBUF == 2u ? ((seg >> 1) & 1u) : (seg & 1u);
+      const uint32_t a = seg & 1u, aph = (seg >> 1) & 1u;
       // one thread does the bounded wait and tells the others, so that all 128 take the same branch
       if (et == 0) *epi_ok = mbar_wait(tfull_bar(a), aph, abort_flag, p.status) ? 1 : 0;
       epi_bar_sync();
@@ -467,12 +463,11 @@ cudaError_t tc_prepare(int* smem_limit_out) {
   e = cudaDeviceGetAttribute(&lim, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   if (e != cudaSuccess) return e;
   cudaFuncAttributes fa;
-  e = cudaFuncGetAttributes(&fa, gemm_tc_kernel<0>);
+  e = cudaFuncGetAttributes(&fa, gemm_tc_kernel<false>);
   if (e != cudaSuccess) return e;
   lim -= (int)fa.sharedSizeBytes;  // the opt-in limit covers static + dynamic shared memory
-  e = cudaFuncSetAttribute(gemm_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
+  e = cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
   if (smem_limit_out) *smem_limit_out = lim;
   return e;
 }
@@ -484,9 +479,8 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[16], int N
   p.N = N; p.K = K; p.nkb = (K + TILE_K - 1) / TILE_K; p.n_tiles = (N + TILE_N - 1) / TILE_N;
   p.mt = tc_pick_mt(m_max > 0 ? m_max : 1);
   p.m_tiles_max = m_max > 0 ? (m_max + p.mt - 1) / p.mt : 1;
-  static const int pair_ok = getenv("RD_TC_PAIR") ? atoi(getenv("RD_TC_PAIR")) : 2;   // tuning toggle: 0 off, 1 narrow only
-  const bool wide = p.m_tiles_max > 1 || p.mt > 128;   // the accumulators of a tile pair then fill the tensor memory
-  p.pair = (pair && p.n_tiles >= 2 && pair_ok >= (wide ? 2 : 1)) ? (wide ? 2 : 1) : 0;
+  static const int pair_ok = getenv("RD_TC_PAIR") ? atoi(getenv("RD_TC_PAIR")) : 1;   // tuning toggle
+  p.pair = (pair && pair_ok && p.m_tiles_max == 1 && p.mt <= 128 && p.n_tiles >= 2) ? 1 : 0;
   const long long n_units = (long long)(p.pair ? (p.n_tiles + 1) / 2 : p.n_tiles) * p.nkb;
   if (out_desc) {
     out_desc->raw = raw; out_desc->partial = partial; out_desc->ld = ld_raw; out_desc->nkb = p.nkb;
@@ -509,7 +503,7 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[16], int N
   if (stages < 2) return cudaErrorInvalidConfiguration;
   p.stages = stages;
   int cols = 32;
-  while (cols < (p.pair == 2 ? 2 * p.mt : 2 * p.mt * (p.pair ? 2 : 1))) cols <<= 1;
+  while (cols < 2 * p.mt * (p.pair ? 2 : 1)) cols <<= 1;
   p.tmem_cols = cols;
   p.m_total = m_total; p.raw = raw; p.ld_raw = ld_raw; p.partial = partial; p.status = status; p.trace = trace;
   // the first launch of a chain starts after everything before it has completed (see launch_ordered)
@@ -518,15 +512,12 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[16], int N
   const size_t smem = (size_t)stages * stage_bytes + overhead;
   ActMaps am;
   for (int i = 0; i < ACT_MAPS; ++i) am.m[i] = *(const CUtensorMap*)(map_a[i] ? map_a[i] : map_a[0]);
-  if (p.pair == 1) {
-    if (first) launch_ordered(gemm_tc_kernel<1>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
-    else launch_pdl(gemm_tc_kernel<1>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
-  } else if (p.pair == 2) {
-    if (first) launch_ordered(gemm_tc_kernel<2>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
-    else launch_pdl(gemm_tc_kernel<2>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+  if (p.pair) {
+    if (first) launch_ordered(gemm_tc_kernel<true>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+    else launch_pdl(gemm_tc_kernel<true>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
   } else {
-    if (first) launch_ordered(gemm_tc_kernel<0>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
-    else launch_pdl(gemm_tc_kernel<0>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+    if (first) launch_ordered(gemm_tc_kernel<false>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+    else launch_pdl(gemm_tc_kernel<false>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
   }
   return cudaGetLastError();
 }
