@@ -15,7 +15,7 @@ namespace {
 constexpr int WROWS = 64;    // rows per CTA
 constexpr int KEYS = 64;     // keys per chunk
 constexpr int PAD = 8;       // bf16 padding of a shared-memory row (keeps 32-bit and ldmatrix accesses conflict free)
-constexpr int NSTAGE = 2;    // K/V chunks in flight per CTA
+constexpr int NSTAGE = 3;    // K/V chunks in flight per CTA
 
 __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile(
@@ -43,7 +43,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 template <int HD>
-__global__ void __launch_bounds__(128, 3) attention_wide_kernel(const float* __restrict__ qkv,
+__global__ void __launch_bounds__(128, 2) attention_wide_kernel(const float* __restrict__ qkv,
                                                              const __nv_bfloat16* __restrict__ kc,
                                                              const __nv_bfloat16* __restrict__ vc,
                                                              __nv_bfloat16* __restrict__ out, RowTables rt,
@@ -126,7 +126,8 @@ __global__ void __launch_bounds__(128, 3) attention_wide_kernel(const float* __r
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
   if (early) chain_wait_cta(cs);
-  load_chunk(0, 0);
+#pragma unroll
+  for (int i = 0; i < NSTAGE - 1; ++i) load_chunk(i, i);
 
   // Q of this warp's rows (fp32, rotated by the preceding kernel) as bf16 A fragments
   uint32_t qf[KS][4];
@@ -158,7 +159,7 @@ __global__ void __launch_bounds__(128, 3) attention_wide_kernel(const float* __r
   for (int ch = 0; ch < n_chunks; ++ch) {
     const int k0 = ch * KEYS;
     const int buf = ch % NSTAGE;
-    load_chunk(ch + 1, (ch + 1) % NSTAGE);   // into the slot the previous iteration released
+    load_chunk(ch + NSTAGE - 1, (ch + NSTAGE - 1) % NSTAGE);   // into the slot the previous iteration released
     asm volatile("cp.async.wait_group %0;" ::"n"(NSTAGE - 1) : "memory");
     __syncthreads();
     if (k0 < wext) {

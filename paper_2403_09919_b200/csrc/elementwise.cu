@@ -1,6 +1,7 @@
 // Small row-wise kernels of the verification forward (Section 3.4): embedding gather, RMSNorm,
 // rotary embedding + KV-cache write, SwiGLU, row argmax, row tables.  All are bandwidth-trivial
 // (activations of at most a few MB that stay in L2); they exist to feed the projections.
+#include <cstdlib>
 #include "rd_internal.cuh"
 #include "gemm_out.cuh"
 #include "pdl.cuh"
@@ -209,9 +210,13 @@ template <typename T, int NORM_MAXV>
 __global__ void __launch_bounds__(NORM_THREADS, NORM_MAXV <= 2 ? 2 : 1)
     rmsnorm_wide_kernel(float* __restrict__ x, GemmOut proj, const T* __restrict__ gain, T* __restrict__ out_t,
                         float* __restrict__ out_f, int d, float eps, const int32_t* __restrict__ m_total, ChainSync cs) {
-  chain_enter(cs);
+  chain_begin(cs);
   __shared__ float sh[32];
-  const int M = *m_total;
+  // inside a chain (but not as its first launch) the row count, written ahead of the chain, may be read before the wait
+  const bool early = cs.signal_ptr != nullptr && cs.wait_ptr != nullptr;
+  int M = early ? *m_total : 0;
+  chain_wait_cta(cs);
+  if (!early) M = *m_total;
   const int nvec = d >> 2;
   const bool add = proj.raw != nullptr;   // x += the projection that ends the previous block (O or down)
   const GemmRows m_tiles = add ? gemm_m_tiles(proj, M) : GemmRows();
@@ -268,7 +273,8 @@ cudaError_t launch_rmsnorm(int dtype, float* x, const GemmOut* proj, const void*
   // the first launch of a chain starts after everything before it has completed (see launch_ordered)
   const bool first = chain && chain->enabled && chain->prev_ptr == nullptr;
   if (m_max > WIDE_ROWS_MIN) {   // several row tiles
-    const int grid = m_max < 4 * wide_sm_count() ? m_max : 4 * wide_sm_count();
+    const int per_sm = (d <= 4 * NORM_THREADS * 2) ? 2 : 1;   // resident CTAs per SM: one wave walks all rows
+    const int grid = m_max < per_sm * wide_sm_count() ? m_max : per_sm * wide_sm_count();
     const ChainSync cs = chain ? chain->link((unsigned)grid, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
 #define RD_NORM_WIDE(MAXV)                                                                                                \
   RD_DISPATCH(dtype, if (first) launch_ordered(rmsnorm_wide_kernel<T, MAXV>, grid, NORM_THREADS, 0, st, x, g, (const T*)gain, \
@@ -435,13 +441,17 @@ template <typename T>
 __global__ void __launch_bounds__(ROPE_THREADS, 2)
     rope_kv_wide_kernel(float* __restrict__ qkv, GemmOut proj, T* __restrict__ kc, T* __restrict__ vc,
                         const float2* __restrict__ table, RowTables rt, Dims dm, int* status, ChainSync cs) {
-  chain_enter(cs);
+  chain_begin(cs);
   const int d = dm.d, hd = dm.hd, half = hd >> 1;
   const int n_items = dm.H * (half >> 1);
   const int idx = blockIdx.y * ROPE_THREADS + threadIdx.x;
   const int h = idx / (half >> 1), i = (idx - h * (half >> 1)) * 2;
   const int o = h * hd + i;
-  const int M = *rt.m_total;
+  // inside a chain the row count, written ahead of the chain, may be read before the wait
+  const bool early = cs.signal_ptr != nullptr && cs.wait_ptr != nullptr;
+  int M = early ? *rt.m_total : 0;
+  chain_wait_cta(cs);
+  if (!early) M = *rt.m_total;
   const GemmRows m_tiles = gemm_m_tiles(proj, M);
   if (idx < n_items) {
     // each CTA takes a contiguous run of rows; the fold of a column changes only from one row tile to the next
@@ -486,8 +496,8 @@ cudaError_t launch_rope_kv(int dtype, float* qkv, const GemmOut& proj, void* kca
                            const RowTables& rt, const Dims& dm, int m_max, int* status, Chain* chain, cudaStream_t st) {
   const int n_items = dm.H * (dm.hd / 4);
   dim3 grid(m_max, (n_items + ROPE_THREADS - 1) / ROPE_THREADS);
-  if (m_max > WIDE_ROWS_MIN) {   // several row tiles: about four CTAs per SM walk the rows
-    const int gx = (4 * wide_sm_count() + (int)grid.y - 1) / (int)grid.y;
+  if (m_max > WIDE_ROWS_MIN) {   // several row tiles
+    const int gx = (2 * wide_sm_count() + (int)grid.y - 1) / (int)grid.y;   // two resident CTAs per SM: one wave walks all rows
     if (gx < m_max) grid.x = gx;
     const ChainSync cs = chain ? chain->link(grid.x * grid.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
     RD_DISPATCH(dtype, launch_pdl(rope_kv_wide_kernel<T>, grid, ROPE_THREADS, 0, st, qkv, proj, (T*)kcache, (T*)vcache,
@@ -568,8 +578,12 @@ __global__ void __maxnreg__(88) swiglu_kernel(GemmOut proj, T* __restrict__ out,
 template <typename T>
 __global__ void __launch_bounds__(SWIGLU_THREADS, 6)
     swiglu_wide_kernel(GemmOut proj, T* __restrict__ out, int F, const int32_t* __restrict__ m_total, ChainSync cs) {
-  chain_enter(cs);
-  const int M = *m_total;
+  chain_begin(cs);
+  // inside a chain the row count, written ahead of the chain, may be read before the wait
+  const bool early = cs.signal_ptr != nullptr && cs.wait_ptr != nullptr;
+  int M = early ? *m_total : 0;
+  chain_wait_cta(cs);
+  if (!early) M = *m_total;
   const GemmRows m_tiles = gemm_m_tiles(proj, M);
   const int f0 = (blockIdx.x * SWIGLU_ITEMS * SWIGLU_THREADS + threadIdx.x) * 4;
   // each CTA takes a contiguous run of rows; the fold of a column changes only from one row tile to the next
@@ -610,8 +624,9 @@ cudaError_t launch_swiglu(int dtype, const GemmOut& proj, void* out_t, int F, co
                           Chain* chain, cudaStream_t st) {
   const int per_cta = SWIGLU_THREADS * SWIGLU_ITEMS * 4;
   dim3 grid((F + per_cta - 1) / per_cta, m_max);
-  if (m_max > WIDE_ROWS_MIN) {   // several row tiles: about sixteen CTAs per SM walk the rows
-    const int gy = (16 * wide_sm_count() + (int)grid.x - 1) / (int)grid.x;
+  if (m_max > WIDE_ROWS_MIN) {   // several row tiles
+    // four CTAs per SM: they share the SM with a CTA of the projection before and of the one after (measured: 3 to 6 alike)
+    const int gy = (4 * wide_sm_count() + (int)grid.x - 1) / (int)grid.x;
     if (gy < m_max) grid.y = gy;
     const ChainSync cs = chain ? chain->link(grid.x * grid.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
     RD_DISPATCH(dtype, launch_pdl(swiglu_wide_kernel<T>, grid, SWIGLU_THREADS, 0, st, proj, (T*)out_t, F, m_total, cs));

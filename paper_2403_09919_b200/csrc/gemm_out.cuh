@@ -73,18 +73,18 @@ __device__ __forceinline__ GemmFold gemm_fold(const GemmOut& g, GemmRows m_tiles
     f.off = (size_t)m * 128 + row + ((g.pair && (n_tile & 1)) ? (size_t)g.mt * 128 : 0);
     return f;
   }
-  // several row tiles: units run over (tile or pair of tiles, row tile, k-block)
+  // several row tiles: units run over (row tile, tile or pair of tiles, k-block)
   const int m_tile = m / m_tiles.rows, col = m - m_tile * m_tiles.rows;
   const int group = g.pair ? (n_tile >> 1) : n_tile, n_groups = g.pair ? ((g.n_tiles + 1) >> 1) : g.n_tiles;
   f.off = (size_t)col * 128 + row + ((g.pair && (n_tile & 1)) ? (size_t)g.mt * 128 : 0);
   if (g.small32) {   // the usual case; 64-bit divisions cost the consuming kernels more than their loads
-    const uint32_t U = (uint32_t)n_groups * m_tiles.n * g.nkb, G = g.grid, tu0 = ((uint32_t)group * m_tiles.n + m_tile) * g.nkb;
+    const uint32_t U = (uint32_t)n_groups * m_tiles.n * g.nkb, G = g.grid, tu0 = ((uint32_t)m_tile * n_groups + group) * g.nkb;
     const uint32_t cf = ((tu0 + 1) * G - 1) / U, cl = ((tu0 + g.nkb) * G - 1) / U;
     f.c_next = (int)(cf > G - 1 ? G - 1 : cf) + 1;
     f.c_last = (int)(cl > G - 1 ? G - 1 : cl);
     return f;
   }
-  const long long t = (long long)group * m_tiles.n + m_tile;
+  const long long t = (long long)m_tile * n_groups + group;
   const long long U = (long long)n_groups * m_tiles.n * g.nkb, G = g.grid;
   const long long tu0 = t * g.nkb;
   f.c_next = gemm_cta_of_unit(tu0, U, G) + 1;

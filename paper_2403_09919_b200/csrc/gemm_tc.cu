@@ -191,7 +191,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
   else if (chained) rows.rows = min(p.mt, max(16, (*p.m_total + 15) & ~15));
   const int m_tiles = rows.n;
   const long long G = gridDim.x;
-  const int n_groups = (PAIR ? (p.n_tiles + 1) / 2 : p.n_tiles) * m_tiles;   // unit = (tile or tile pair, row tile, k-block)
+  // unit = (row tile, weight tile or tile pair, k-block), row tile slowest: the CTAs of each row tile then walk the
+  // weight tiles abreast of the other row tiles' CTAs, and a weight tile leaves device memory once for all of them
+  const int n_wt = PAIR ? (p.n_tiles + 1) / 2 : p.n_tiles;
+  const int n_groups = n_wt * m_tiles;
   const long long U = (long long)n_groups * p.nkb;
   const long long u0 = gemm_range_begin(blockIdx.x, U, G), u1 = gemm_range_begin(blockIdx.x + 1, U, G);
   const int mt_eff = rows.rows;   // several row tiles are equal: the fewest that hold the rows, each a multiple of 16 rows
@@ -229,15 +232,15 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
     UnitPos q;
     const int t = (int)(u / p.nkb);
     q.kb = (int)(u - (long long)t * p.nkb);
-    q.g = PAIR ? t : t / m_tiles;
-    q.m_tile = PAIR ? 0 : t - q.g * m_tiles;
+    q.m_tile = PAIR ? 0 : t / n_wt;
+    q.g = t - q.m_tile * n_wt;
     q.s = 0; q.ph = 0;
     return q;
   };
   auto advance = [&](UnitPos& q) {
     if (++q.kb == p.nkb) {
       q.kb = 0;
-      if (PAIR || ++q.m_tile == m_tiles) { q.m_tile = 0; ++q.g; }
+      if (++q.g == n_wt) { q.g = 0; ++q.m_tile; }
     }
     if (++q.s == (uint32_t)p.stages) { q.s = 0; q.ph ^= 1u; }
   };
@@ -356,7 +359,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
     for (long long u = u0; u < u1 && ok; ++seg) {
       const int t = (int)(u / p.nkb), kb0 = (int)(u - (long long)t * p.nkb);
       const int kb1 = (int)min((long long)p.nkb, kb0 + (u1 - u));
-      const int grp = PAIR ? t : t / m_tiles, m_tile = PAIR ? 0 : t - grp * m_tiles;
+      const int m_tile = PAIR ? 0 : t / n_wt, grp = t - m_tile * n_wt;
       const int n_tile0 = PAIR ? 2 * grp : grp;
       const int m_base = m_tile * mt_eff;
       const int c_end = min(mt_eff, ((M - m_base) + 15) & ~15);   // accumulator columns that hold rows of the launch
