@@ -308,7 +308,7 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
   // attention launch geometry (tensor-core path): tiles of 16 rows per sequence; keys split over CTAs only
   // for long contexts with few tiles
   int row_blocks = 1, n_splits = 1;
-  bool att_wide = false;
+  bool att_wide = false, att_shallow = false;
   if (h->use_tc) {
     const int rpb = attn_tc_rows_per_block();
     row_blocks = (rows_per_seq_max + rpb - 1) / rpb;
@@ -318,6 +318,9 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
     static const int wide_waves = getenv("RD_ATT_WIDE") ? atoi(getenv("RD_ATT_WIDE")) : 4;   // tuning toggle
     att_wide = wide_waves < 0 || (wide_waves > 0 && blocks > wide_waves * h->tc_grid);   // negative: always
     if (att_wide) row_blocks = (rows_per_seq_max + attn_wide_rows_per_block() - 1) / attn_wide_rows_per_block();
+    // more 16-row CTAs than SMs (many sequences of a few rows): a two-chunk ring so that three CTAs share an SM
+    static const int shallow_ok = getenv("RD_ATT_SHALLOW") ? atoi(getenv("RD_ATT_SHALLOW")) : 1;   // tuning toggle
+    att_shallow = shallow_ok && !att_wide && blocks > h->tc_grid;
     n_splits = h->tc_grid / blocks;  // at most one CTA per SM: a second wave would double the time
     // ... and only when a CTA would otherwise walk many chunks: the cross-CTA merge costs several microseconds
     const int max_chunks = (h->ctx_bound + rows_per_seq_max + 63) / 64;
@@ -347,7 +350,8 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
       else if (h->use_tc)
         CK(h, launch_attention_tc(w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.attn_t, rt, w.seq_off, dm, n_seq,
                                   row_blocks, n_splits, w.att_scratch, w.att_counters,
-                                  (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) ? w.trace + (size_t)8 * h->trace_next++ : nullptr, ch, st));
+                                  (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) ? w.trace + (size_t)8 * h->trace_next++ : nullptr, ch,
+                                  att_shallow ? 1 : 0, st));
       else
         CK(h, launch_attention(dm.dtype, w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.attn_t, rt, dm, m_max, st));
     }

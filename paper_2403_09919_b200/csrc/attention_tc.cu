@@ -23,7 +23,8 @@ constexpr int KEYS = 64;     // keys per chunk
 constexpr int WKEYS = 16;    // keys of a chunk per warp
 constexpr int PAD = 8;       // bf16 padding of a shared-memory row (keeps 32-bit and ldmatrix accesses conflict free)
 constexpr int MAX_SPLITS = 16;
-constexpr int NSTAGE = 4;     // K/V chunks in flight per CTA
+constexpr int NSTAGE_DEEP = 4;     // K/V chunks in flight per CTA: one CTA per SM (139 KB), the decode-time case
+constexpr int NSTAGE_SHALLOW = 2;  // ... three CTAs per SM (70 KB each), for launches of more CTAs than SMs
 
 __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile(
@@ -47,7 +48,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 #define RD_STAMP(i) asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[i]))
 
-template <int HD>
+template <int HD, int NSTAGE>
 __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restrict__ qkv,
                                                            const __nv_bfloat16* __restrict__ kc,
                                                            const __nv_bfloat16* __restrict__ vc,
@@ -416,9 +417,12 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
   chain_exit(cs);
 }
 
-template <int HD>
+template <int HD, int NSTAGE>
 size_t smem_bytes(int MW) {
-  return (size_t)(2 * NSTAGE * KEYS) * (HD + PAD) * 2 + ROWS * 4 + (size_t)ROWS * MW * 4;
+  size_t ring = (size_t)(2 * NSTAGE * KEYS) * (HD + PAD) * 2;
+  const size_t merge = (size_t)(4 * ROWS * (HD + 4) + ROWS * MAX_SPLITS) * 4;   // the warps' partials reuse the ring
+  if (ring < merge) ring = merge;
+  return ring + ROWS * 4 + (size_t)ROWS * MW * 4;
 }
 
 }  // namespace
@@ -427,27 +431,36 @@ size_t attn_tc_scratch_floats(int blocks, int n_splits, int hd) { return (size_t
 int attn_tc_rows_per_block() { return ROWS; }
 
 cudaError_t attn_tc_prepare(int hd, int MW) {
-  if (hd == 128)
-    return cudaFuncSetAttribute(attention_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes<128>(MW));
-  if (hd == 64)
-    return cudaFuncSetAttribute(attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes<64>(MW));
-  return cudaErrorInvalidValue;
+  cudaError_t e = cudaErrorInvalidValue;
+  if (hd == 128) {
+    e = cudaFuncSetAttribute(attention_tc_kernel<128, NSTAGE_DEEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes<128, NSTAGE_DEEP>(MW));
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(attention_tc_kernel<128, NSTAGE_SHALLOW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes<128, NSTAGE_SHALLOW>(MW));
+  } else if (hd == 64) {
+    e = cudaFuncSetAttribute(attention_tc_kernel<64, NSTAGE_DEEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes<64, NSTAGE_DEEP>(MW));
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(attention_tc_kernel<64, NSTAGE_SHALLOW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes<64, NSTAGE_SHALLOW>(MW));
+  }
+  return e;
 }
 
-// grid (H, sequences * row_tiles, n_splits)
+// grid (H, sequences * row_tiles, n_splits); `shallow`: more CTAs than SMs, so several should share an SM
 cudaError_t launch_attention_tc(const float* qkv, const void* kcache, const void* vcache, void* out, const RowTables& rt,
                                 const int32_t* seq_off, const Dims& dm, int n_seq, int row_tiles, int n_splits,
-                                float* scratch, int32_t* counters, unsigned long long* dbg, Chain* chain, cudaStream_t st) {
+                                float* scratch, int32_t* counters, unsigned long long* dbg, Chain* chain, int shallow, cudaStream_t st) {
   dim3 grid(dm.H, n_seq * row_tiles, n_splits);
   const ChainSync cs = chain ? chain->link(grid.x * grid.y * grid.z) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
-  if (dm.hd == 128)
-    launch_pdl(attention_tc_kernel<128>, grid, 128, smem_bytes<128>(dm.MW), st, qkv, (const __nv_bfloat16*)kcache,
-               (const __nv_bfloat16*)vcache, (__nv_bfloat16*)out, rt, seq_off, dm, row_tiles, n_splits, scratch, counters, dbg, cs);
-  else if (dm.hd == 64)
-    launch_pdl(attention_tc_kernel<64>, grid, 128, smem_bytes<64>(dm.MW), st, qkv, (const __nv_bfloat16*)kcache,
-               (const __nv_bfloat16*)vcache, (__nv_bfloat16*)out, rt, seq_off, dm, row_tiles, n_splits, scratch, counters, dbg, cs);
-  else
+#define RD_ATT_LAUNCH(HD, NST)                                                                                              \
+  launch_pdl(attention_tc_kernel<HD, NST>, grid, 128, smem_bytes<HD, NST>(dm.MW), st, qkv, (const __nv_bfloat16*)kcache,    \
+             (const __nv_bfloat16*)vcache, (__nv_bfloat16*)out, rt, seq_off, dm, row_tiles, n_splits, scratch, counters, dbg, cs)
+  if (dm.hd == 128) {
+    if (shallow) RD_ATT_LAUNCH(128, NSTAGE_SHALLOW); else RD_ATT_LAUNCH(128, NSTAGE_DEEP);
+  } else if (dm.hd == 64) {
+    if (shallow) RD_ATT_LAUNCH(64, NSTAGE_SHALLOW); else RD_ATT_LAUNCH(64, NSTAGE_DEEP);
+  } else {
     return cudaErrorInvalidValue;
+  }
+#undef RD_ATT_LAUNCH
   return cudaGetLastError();
 }
 
