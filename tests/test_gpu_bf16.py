@@ -178,6 +178,45 @@ def test_wide_beam_two_row_tiles():
     check_verify(rig, beams_alphabet=40)
 
 
+def test_long_prompts_many_row_tiles():
+    """Prompts of 700 and 450 tokens in one prefill of an engine sized for 16 sequences (passes of up to 656 rows: the
+    first holds 656 rows of one sequence, the second its last 44 and the whole other prompt): three row tiles in the
+    projections, the row-loop kernels, and 64-row causal attention tiles in which the warps' key ranges differ and
+    start past the keys of an earlier pass.  The handed-over state (context length, last hidden vector) and a
+    verification on top of the two caches must match the oracle."""
+    # 16 heads of 64: 16 x 2 x 41 sixteen-row tiles would be several waves of CTAs, so the 64-row attention kernel runs
+    cfg = dict(RAGGED, d_model=1024, n_heads=16, d_rnn=1024, max_batch=16, max_ctx=800)
+    rig = Rig(cfg=cfg)
+    rng = np.random.default_rng(11)
+    prompts = [rng.integers(0, 1000, size=700), rng.integers(0, 1000, size=450)]
+    rig.eng.prefill(prompts)
+    rig.eng.poll()
+    c_ctx, c_root, c_h = rig.eng.get_state()
+    refs = []
+    for b, pr in enumerate(prompts):
+        kv = rig.new_kv()
+        ctx, g, h = ora.prefill(rig.W, cfg, pr, kv)
+        assert int(c_ctx[b]) == ctx
+        assert rel_err(c_h[b].cpu().numpy()[None], np.asarray(h)[None]) < REL
+        refs.append((kv, ctx, g, h))
+    roots = np.array([r[2] for r in refs])
+    hs = np.stack([np.asarray(r[3]) for r in refs]).astype(np.float32)
+    rig.eng.set_state(None, dev(roots), dev(hs, torch.float32))
+    beams = rng.integers(0, 4, size=(2, 8, 5))
+    pk = rig.eng.pack(dev(beams))
+    argmax, hidden, logits = rig.eng.verify(pk, want_logits=True)
+    rig.eng.poll()
+    for b, (kv, ctx, g, h) in enumerate(refs):
+        aug = np.concatenate([np.full((8, 1), g), beams[b]], axis=1)
+        p = ora.pack_beam(aug, ctx)
+        n = p["n"]
+        assert int(pk.n[b]) == n
+        rh, rl = ora.llm_forward(rig.W, cfg, p["tokens"], p["pos"], p["mask"], kv, ctx)
+        assert rel_err(logits[b, :n].cpu().numpy(), rl) < REL
+        sure = decided(rl)
+        assert (argmax[b, :n].cpu().numpy()[sure] == rl.argmax(1)[sure]).all()
+
+
 def test_batched_ragged_many_rows():
     """Batch 16 x beam width 16: up to 1296 compact rows, six activation tiles, per-sequence contexts."""
     cfg = dict(RAGGED, max_batch=16, beam_width=16, beam_length=5, max_ctx=260)
