@@ -1,8 +1,8 @@
 // Where a projection's result lives until its consumer folds it.
 //
 // The tensor-core projection is a stream-K kernel: CTA c owns the contiguous unit range
-// [c*U/G, (c+1)*U/G) of the (tile, k-block) list, so a tile's k-range may be cut among several
-// CTAs.  The kernel applies no epilogue and does no cross-CTA reduction.  The contributor that
+// [c*U/G, (c+1)*U/G) of the (row tile, weight tile or tile pair, k-block) list, so a tile's k-range
+// may be cut among several CTAs.  The kernel applies no epilogue and does no cross-CTA reduction.  The contributor that
 // holds a tile's first k-block writes its sum to the fp32 output `raw`; every other contributor
 // (its range then starts inside that tile, so it has exactly one such segment) writes its sum to
 // its own slot of `partial`.  The kernel that consumes the projection (norm, rotary, SwiGLU,
@@ -16,9 +16,9 @@ namespace rd {
 
 struct GemmOut {
   const float* raw;      // [M][ld]
-  const float* partial;  // [grid][mt * 128], nullptr when nothing is cut (CUDA-core path)
+  const float* partial;  // [grid][mt * 128 (x 2 in pair mode)], nullptr when nothing is cut (CUDA-core path)
   int ld;
-  int nkb, n_tiles, mt, grid, m_tiles_max;
+  int nkb, n_tiles, mt, grid, m_tiles_max;   // mt: most rows of a row tile; m_tiles_max: most row tiles of the launch
   int all_work;          // every CTA has a non-empty range for any row count (units >= CTAs)
   int pair;              // 1: a unit is (pair of adjacent tiles, k-block); a slot holds two tiles, even one first
   int small32;           // (units + 1) * CTAs stays below 2^31 for any row count of the launch: 32-bit index arithmetic

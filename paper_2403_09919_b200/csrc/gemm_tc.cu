@@ -7,17 +7,23 @@
 // activations are the MMA "B" operand, N_mma = MT rows (a multiple of 16, at most 256).  The
 // accumulator D[n][m] lives in TMEM: lane = weight row, column = activation row.
 //
-// Schedule: persistent, one CTA per SM, stream-K.  The work is the list of (tile, k-block) units,
-// tile = (128 weight rows) x (MT activation rows), k-block = 64 columns; CTA c owns the contiguous
-// unit range [c*U/G, (c+1)*U/G), so every SM streams the same number of weight bytes whatever the
-// shape.  No epilogue and no cross-CTA reduction happen here: the segment that holds a tile's first
-// k-block stores its fp32 sums to the output, any other segment to the CTA's partial slot, and the
-// consuming kernel folds them in CTA order (gemm_out.cuh).
+// Schedule: persistent, one CTA per SM, stream-K.  The work is the list of (row tile, weight tile,
+// k-block) units, row tile slowest; tile = (128 weight rows) x (MT activation rows), k-block = 64
+// columns; CTA c owns the contiguous unit range [c*U/G, (c+1)*U/G), so every SM streams the same
+// number of weight bytes whatever the shape, and with several row tiles the CTAs of all row tiles
+// walk the weight tiles abreast (a tile leaves device memory once).  With one row tile of at most
+// 128 rows a unit is a PAIR of adjacent weight tiles sharing one activation box.  The rows of a
+// launch are a device-side count: the box height, the MMA's N and the number of (equal) row tiles
+// follow it (gemm_row_tiles).  No epilogue and no cross-CTA reduction happen here: the segment that
+// holds a tile's first k-block stores its fp32 sums to the output, any other segment to the CTA's
+// partial slot, and the consuming kernel folds them in CTA order (gemm_out.cuh).
 //
-// Roles: warp 0 = TMA producer (one 128x64 weight box and one MTx64 activation box per stage),
+// Roles: warp 0 = TMA producer (one or two 128x64 weight boxes and one activation box per stage),
 // warp 1 = MMA issuer and TMEM owner, warps 2..5 = epilogue (tcgen05.ld, one TMEM lane quarter
-// each).  Two TMEM accumulators alternate so the epilogue of one segment overlaps the MMAs of the
-// next; the smem ring (full/empty mbarriers) never drains between tiles.
+// each).  Two TMEM accumulator buffers alternate so the epilogue of one segment overlaps the MMAs
+// of the next; the smem ring (full/empty mbarriers) never drains between tiles.  The producer and
+// the MMA issuer are single threads: their loops carry their positions along and contain no
+// division (a division by a run-time value per stage was what bounded the stream).
 //
 // Every mbarrier wait is bounded (one second); on expiry the CTA raises DEV_ERR_TIMEOUT in the
 // status word, lets its copies land, frees its TMEM and exits; later launches see the flag and
@@ -217,7 +223,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
   volatile int* epi_ok = reinterpret_cast<volatile int*>(misc + 12);
 
-  // iteration i of this CTA = unit u0 + i = (tile, k-block) in tile-major order
+  // iteration i of this CTA = unit u0 + i
   const uint32_t n_it = (uint32_t)(u1 - u0);
   const uint32_t pre = early ? min(n_it, (uint32_t)p.stages) : 0u;
   const uint64_t pol_w = l2_policy_evict_first();
