@@ -217,6 +217,15 @@ def test_long_prompts_many_row_tiles():
         assert (argmax[b, :n].cpu().numpy()[sure] == rl.argmax(1)[sure]).all()
 
 
+def test_wide_beam_whose_rows_fit_one_tile_after_all():
+    """Beam width 64 with heavily shared prefixes: the host-side bound is 321 rows (two row tiles), the packed rows are
+    about 170, so the projections run a single tile and their consumers take the single-tile path of a launch that was
+    laid out for two."""
+    cfg = dict(RAGGED, beam_width=64, beam_length=5, max_ctx=500)
+    rig = Rig(cfg=cfg)
+    check_verify(rig, beams_alphabet=3)
+
+
 def test_batched_ragged_many_rows():
     """Batch 16 x beam width 16: up to 1296 compact rows, six activation tiles, per-sequence contexts."""
     cfg = dict(RAGGED, max_batch=16, beam_width=16, beam_length=5, max_ctx=260)
