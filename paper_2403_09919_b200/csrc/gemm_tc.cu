@@ -295,11 +295,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
     // ===================== TMA producer =====================
     if (lane == 0 && u0 < u1) {
       if (p.trace) atomicMax(p.trace + 7, globaltimer());   // last CTA ready to wait
+      // An earlier launch of the step gave up on a wait: wind this one down through the roles' abort paths.  The
+      // status word is requested BEFORE the wait (a load right after it would put an L2 round trip between the
+      // dependency and the first activation copy); a time-out raised while this thread waits ends the wait itself.
+      const int32_t status_before = *(volatile int32_t*)p.status;
       if (early) chain_wait_thread(p.cs);
       chain_fence_async_reads();  // the activations were written by ordinary stores of the preceding launch
       if (p.trace) { atomicMin(p.trace + 1, globaltimer()); atomicMax(p.trace + 2, globaltimer()); }   // dependency resolved
-      // an earlier launch of the step gave up on a wait: wind this one down through the roles' abort paths
-      if (*(volatile int32_t*)p.status & DEV_ERR_TIMEOUT) *abort_flag = 1;
+      if (status_before & DEV_ERR_TIMEOUT) *abort_flag = 1;
       UnitPos q = pos_at(u0);
       for (uint32_t i = 0; i < pre; ++i) { issue_a(q); advance(q); }
       bool ok = true;
