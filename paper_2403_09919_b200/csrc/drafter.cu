@@ -114,8 +114,11 @@ __global__ void __maxnreg__(88) act_kernel(GemmOut proj, const T* __restrict__ b
     if (fast) { src = gemm_src(proj, 1, m, n); gemm_src_pin(src); }
     asm volatile("" : "+l"(rp), "+l"(of), "+l"(ot));
   }
+  // inside a chain the row count, written ahead of the chain, is requested before the wait
+  const bool early = cs.signal_ptr != nullptr && cs.wait_ptr != nullptr;
+  int M = early ? *m_total : 0;
   chain_wait_cta(cs);
-  const int M = *m_total;
+  if (!early) M = *m_total;
   if (m < M && active) {
     float4 q;
     float4 rv = make_float4(0.f, 0.f, 0.f, 0.f);
