@@ -638,7 +638,7 @@ cudaError_t launch_swiglu(int dtype, const GemmOut& proj, void* out_t, int F, co
 }
 
 // ---------------------------------------------------------------- row argmax (lowest index on ties)
-__global__ void argmax_rows_kernel(float* __restrict__ logits, GemmOut proj, int V, int32_t* __restrict__ out,
+__global__ void __launch_bounds__(512) argmax_rows_kernel(float* __restrict__ logits, GemmOut proj, int V, int32_t* __restrict__ out,
                                    const int32_t* __restrict__ out_index, const int32_t* __restrict__ m_total) {
   pdl_enter();
   __shared__ float sv[32];
@@ -650,14 +650,28 @@ __global__ void argmax_rows_kernel(float* __restrict__ logits, GemmOut proj, int
   const GemmRows m_tiles = gemm_m_tiles(proj, M);
   float bv = -INFINITY;
   int bi = 0x7fffffff;
-  // the complete logits are written back in place (later readers of the buffer see final values)
-  for (int i = threadIdx.x * 4; i < V; i += blockDim.x * 4) {
-    const float4 q = gemm_value4(proj, m_tiles, m, i);
-    *reinterpret_cast<float4*>(r + i) = q;
-    const float e[4] = {q.x, q.y, q.z, q.w};
+  // the complete logits are written back in place (later readers of the buffer see final values); four float4 per
+  // thread and pass, every load of the four in flight before the first is used
+  constexpr int ARG_BATCH = 4, ARG_FOLD = 2;
+  for (int i0 = threadIdx.x * 4; i0 < V; i0 += blockDim.x * 4 * ARG_BATCH) {
+    GemmPending4<ARG_FOLD> pd[ARG_BATCH];
 #pragma unroll
-    for (int k = 0; k < 4; ++k)
-      if (e[k] > bv || (e[k] == bv && i + k < bi)) { bv = e[k]; bi = i + k; }
+    for (int u = 0; u < ARG_BATCH; ++u) {
+      const int i = i0 + u * blockDim.x * 4;
+      if (i < V) pd[u] = gemm_issue4<ARG_FOLD>(proj, m_tiles, m, i);
+    }
+#pragma unroll
+    for (int u = 0; u < ARG_BATCH; ++u) {
+      const int i = i0 + u * blockDim.x * 4;
+      if (i < V) {
+        const float4 q = gemm_finish4(proj, m_tiles, pd[u]);
+        *reinterpret_cast<float4*>(r + i) = q;
+        const float e[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (e[k] > bv || (e[k] == bv && i + k < bi)) { bv = e[k]; bi = i + k; }
+      }
+    }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
