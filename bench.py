@@ -278,6 +278,53 @@ def run_sweep(args, cfg):
               r["hbm_bound_ms"], r["tensor_bound_ms"], r["bound"], r["frac_of_roofline"]), file=sys.stderr)
 
 
+def run_prefill(args, cfg):
+    """Prompt processing (the pass that precedes the decode loop) at the workload's layer shapes: many rows per launch,
+    causal attention.  One line of JSON per (batch, prompt length) and a table on stderr.  Not part of the default run."""
+    from paper_2403_09919_b200 import binding
+    device = "cuda:0"
+    torch.cuda.set_device(device)
+    peak_bw, _ = measured_peaks()
+    peak_tf = 1411.0
+    try:
+        with open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "MEASURED_PEAKS.json")) as f:
+            peak_tf = float(json.load(f).get("bf16_tflops_sustained", peak_tf))
+    except Exception:
+        pass
+    w = synth.make_weights(cfg, device)
+    es = 2
+    rows = []
+    for B in [int(x) for x in args.prefill_batch.split(",")]:
+        for P in [int(x) for x in args.prefill_len.split(",")]:
+            c = dict(cfg, max_batch=B, prompt_len=P)
+            c["max_ctx"] = P + 2 * (c["beam_length"] + 1) + 2 + c["beam_width"] * c["beam_length"]
+            eng = binding.ReDrafter(c, w, device=device)
+            prompts = synth.make_prompts(c, B, seed=c.get("seed", 0))
+            reps = 3
+            eng.prefill(prompts)                      # warm-up
+            ms = timed_loop(eng, reps, lambda i: eng.prefill(prompts)) / reps
+            eng.poll()
+            sb = step_bytes(c, 0)
+            n_tok = B * P
+            cap = max(1024, B * (1 + c["beam_width"] * c["beam_length"]))      # rows one pass holds
+            passes = (n_tok + cap - 1) // cap
+            flops = 2.0 * n_tok * (sb["llm"] / es) + 4.0 * B * (P * (P + 1) / 2) * c["d_model"] * c["n_layers"]
+            t_bw, t_tc = passes * sb["llm"] / (peak_bw * 1e9) * 1e3, flops / (peak_tf * 1e12) * 1e3
+            row = {"prefill": True, "batch": B, "prompt_len": P, "tokens": n_tok, "passes": passes, "rows_per_pass": cap,
+                   "ms": ms, "tokens_per_s": n_tok / ms * 1e3, "dense_tflop": flops / 1e12, "tflops": flops / ms / 1e9,
+                   "weight_stream_ms": t_bw, "tensor_bound_ms": t_tc, "frac_of_roofline": max(t_bw, t_tc) / ms}
+            rows.append(row)
+            print(json.dumps(row), flush=True)
+            eng.close()
+            del eng
+    print("| batch | prompt | tokens | passes x rows | ms | tokens/s | TFLOP/s | weight-stream ms | tensor-bound ms | roofline frac |", file=sys.stderr)
+    print("|---|---|---|---|---|---|---|---|---|---|", file=sys.stderr)
+    for r in rows:
+        print("| %d | %d | %d | %d x %d | %.2f | %.0f | %.0f | %.2f | %.2f | %.2f |" % (r["batch"], r["prompt_len"], r["tokens"], r["passes"],
+              r["rows_per_pass"], r["ms"], r["tokens_per_s"], r["tflops"], r["weight_stream_ms"], r["tensor_bound_ms"],
+              r["frac_of_roofline"]), file=sys.stderr)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -295,6 +342,9 @@ def main():
     ap.add_argument("--sweep-bw", default="1,4,8,16,32")
     ap.add_argument("--sweep-batch", default="1,2,4,8,16")
     ap.add_argument("--sweep-prompt", type=int, default=256)
+    ap.add_argument("--prefill", action="store_true", help="prompt-processing timings instead of the benchmark line")
+    ap.add_argument("--prefill-batch", default="1,16")
+    ap.add_argument("--prefill-len", default="512,2048")
     args = ap.parse_args()
     cfg = dict(synth.CONFIGS[args.workload])
     if args.layers:
@@ -304,6 +354,9 @@ def main():
         return
     if args.sweep:
         run_sweep(args, cfg)
+        return
+    if args.prefill:
+        run_prefill(args, cfg)
         return
     if args.warmup < 3:
         args.warmup = 3

@@ -152,9 +152,12 @@ constexpr int TRACE_SLOTS = 512;
 constexpr int TC_MAX_GRID = 160;  // upper bound of the SM count the scratch is sized for
 constexpr int ATT_MAX_SPLIT_BLOCKS = 4 * TC_MAX_GRID;  // (blocks x splits) the split-KV scratch holds
 
+// Rows one forward pass can hold: a verification pass needs B x NMAX; prompt processing takes passes of this many
+// rows, and every pass streams all weights, so the floor is four row tiles (the workspace grows by about 0.2 MB per
+// row at the 7B shape).
 int m_cap_of(const Dims& dm) {
   const int v = dm.B * dm.NMAX;
-  return v > 256 ? v : 256;
+  return v > 1024 ? v : 1024;
 }
 
 void carve(Bump& bp, const Dims& dm, int m_cap, Workspace* w) {
@@ -175,7 +178,7 @@ void carve(Bump& bp, const Dims& dm, int m_cap, Workspace* w) {
   w->proj_d = bp.take<float>((size_t)m_cap * dm.d);
   w->gu = bp.take<float>((size_t)m_cap * 2 * dm.F);
   w->hidden_f = bp.take<float>((size_t)m_cap * dm.d);
-  w->logits = bp.take<float>((size_t)m_cap * dm.V);
+  w->logits = bp.take<float>((size_t)dm.B * dm.NMAX * dm.V);   // verification rows only (prompt passes need B rows)
   w->rope_tab = bp.take<float>((size_t)m_cap * dm.hd);
   w->a_t = bp.take<char>((size_t)m_cap * dm.d * es);
   w->attn_t = bp.take<char>((size_t)m_cap * dm.d * es);
