@@ -364,7 +364,7 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
     CKP(h, PROF_NORM, launch_rmsnorm(dm.dtype, w.x, &g_o, h->ffn_norm[l], w.a_t, nullptr, dm.d, dm.eps, w.m_total, m_max, ch, st));
     rc = gemm(h, w.a_t, dm.d, h->w_gate_up[l], 2 * dm.F, dm.d, w.m_total, m_max, w.gu, 2 * dm.F, &g_gu, ch, st, /*pair=*/1);
     if (rc) return rc;
-    CKP(h, PROF_SWIGLU, launch_swiglu(dm.dtype, g_gu, w.act_t, dm.F, w.m_total, m_max, ch, st));
+    CKP(h, PROF_SWIGLU, launch_swiglu(dm.dtype, g_gu, w.act_t, dm.F, w.m_total, m_max, w.status, ch, st));
     rc = gemm(h, w.act_t, dm.F, h->w_down[l], dm.d, dm.F, w.m_total, m_max, w.proj_d, dm.d, &g_dn, ch, st, /*pair=*/1);
     if (rc) return rc;
   }

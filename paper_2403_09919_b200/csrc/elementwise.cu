@@ -5,6 +5,7 @@
 #include "rd_internal.cuh"
 #include "gemm_out.cuh"
 #include "pdl.cuh"
+#include "stage.cuh"
 
 namespace rd {
 
@@ -574,62 +575,122 @@ __global__ void __maxnreg__(88) swiglu_kernel(GemmOut proj, T* __restrict__ out,
 }
 
 
-// Rows in a loop (see rmsnorm_wide_kernel): blockIdx.x picks the columns, blockIdx.y the first row.
+// Many rows: blockIdx.x picks SWS_COLS consecutive columns, blockIdx.y a contiguous run of rows.  The gate and the up
+// segment of a row (SWS_COLS x 4 bytes each, contiguous) come in through a ring of shared-memory stages filled by
+// thread 0 with bulk asynchronous copies, SWS_STAGES - 1 rows ahead of the row being worked on (stage.cuh), so what
+// the CTA has in flight does not depend on its registers.  Partial sums (with far more tiles than CTAs a tile is cut at
+// most once, and about one tile in five is) are added from global memory by the threads whose columns they concern.
+constexpr int SWS_THREADS = 256;
+constexpr int SWS_COLS = 2048;      // two float4 per thread
+constexpr int SWS_STAGES = 4;       // 4 x (8 + 8) KB per CTA
 template <typename T>
-__global__ void __launch_bounds__(SWIGLU_THREADS, 6)
-    swiglu_wide_kernel(GemmOut proj, T* __restrict__ out, int F, const int32_t* __restrict__ m_total, ChainSync cs) {
+__global__ void __launch_bounds__(SWS_THREADS, 3)
+    swiglu_wide_kernel(GemmOut proj, T* __restrict__ out, int F, const int32_t* __restrict__ m_total, int32_t* status,
+                       ChainSync cs) {
   chain_begin(cs);
+  extern __shared__ __align__(128) uint8_t sws_smem[];
+  __shared__ __align__(8) unsigned long long sws_bars[SWS_STAGES];
+  float* ring = reinterpret_cast<float*>(sws_smem);   // [SWS_STAGES][gate | up][SWS_COLS]
+  const uint32_t ring_u = stage_smem_u32(ring), bars_u = stage_smem_u32(sws_bars);
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < SWS_STAGES; ++s) stage_bar_init(bars_u + 8u * s, 1);
+    stage_bar_init_fence();
+  }
   // inside a chain the row count, written ahead of the chain, may be read before the wait
   const bool early = cs.signal_ptr != nullptr && cs.wait_ptr != nullptr;
   int M = early ? *m_total : 0;
-  chain_wait_cta(cs);
+  chain_wait_cta(cs);   // (its barrier also publishes the initialised mbarriers)
   if (!early) M = *m_total;
   const GemmRows m_tiles = gemm_m_tiles(proj, M);
-  const int f0 = (blockIdx.x * SWIGLU_ITEMS * SWIGLU_THREADS + threadIdx.x) * 4;
-  // each CTA takes a contiguous run of rows; the fold of a column changes only from one row tile to the next
-  const int m_end = gemm_rows_begin(M, gridDim.y, blockIdx.y + 1);
-  int cur_tile = -1;
-  GemmFold fg[SWIGLU_ITEMS], fu[SWIGLU_ITEMS];
-  for (int m = gemm_rows_begin(M, gridDim.y, blockIdx.y); m < m_end; ++m) {
-    GemmPending4f<WIDE_FOLD_SWIGLU> pg[SWIGLU_ITEMS], pu[SWIGLU_ITEMS];
-    const int m_tile = m / m_tiles.rows;
-    const size_t doff = (size_t)(m - m_tile * m_tiles.rows) * 128;
-    if (m_tile != cur_tile) {
-      cur_tile = m_tile;
+  const int c0 = blockIdx.x * SWS_COLS;
+  const int ncol = min(SWS_COLS, F - c0);
+  const uint32_t seg_bytes = (uint32_t)ncol * 4u;
+  const int m_begin = gemm_rows_begin(M, gridDim.y, blockIdx.y), m_end = gemm_rows_begin(M, gridDim.y, blockIdx.y + 1);
+  const int n_rows = m_end - m_begin;
+  auto issue = [&](int i) {   // thread 0: row m_begin + i into slot i % SWS_STAGES
+    const int s = i % SWS_STAGES;
+    const float* src = proj.raw + (size_t)(m_begin + i) * proj.ld + c0;
+    stage_expect_tx(bars_u + 8u * s, 2u * seg_bytes);
+    stage_copy(ring_u + (uint32_t)(s * 2) * SWS_COLS * 4u, src, seg_bytes, bars_u + 8u * s);
+    stage_copy(ring_u + (uint32_t)(s * 2 + 1) * SWS_COLS * 4u, src + F, seg_bytes, bars_u + 8u * s);
+  };
+  if (threadIdx.x == 0) {
+    chain_fence_async_reads();   // the projection wrote its output with ordinary stores
+    for (int i = 0; i < SWS_STAGES - 1 && i < n_rows; ++i) issue(i);
+  }
+  const int j0 = threadIdx.x * 4, j1 = j0 + SWS_THREADS * 4;   // this thread's two float4 inside the segment
+  const bool cut_any = proj.partial != nullptr;
+  int tile_end = 0, cur_tile = 0;
+  const size_t slot = gemm_slot_stride(proj);
+  GemmFold fg[2], fu[2];   // the fold of a column changes only from one row tile to the next
+  bool cut[2] = {false, false};
+  uint32_t s = 0, ph = 0;
+  for (int i = 0; i < n_rows; ++i) {
+    const int m = m_begin + i;
+    if (threadIdx.x == 0 && i + SWS_STAGES - 1 < n_rows) issue(i + SWS_STAGES - 1);   // slot released by the last barrier
+    if (cut_any && m >= tile_end) {
+      cur_tile = m / m_tiles.rows;
+      tile_end = (cur_tile + 1) * m_tiles.rows;
 #pragma unroll
-      for (int k = 0; k < SWIGLU_ITEMS; ++k) {
-        const int f = f0 + k * SWIGLU_THREADS * 4;
-        if (f < F) { fg[k] = gemm_fold_or_none(proj, m_tiles, m_tile * m_tiles.rows, f); fu[k] = gemm_fold_or_none(proj, m_tiles, m_tile * m_tiles.rows, F + f); }
+      for (int k = 0; k < 2; ++k) {
+        const int j = k ? j1 : j0;
+        if (j < ncol) {
+          fg[k] = gemm_fold(proj, m_tiles, cur_tile * m_tiles.rows, c0 + j);
+          fu[k] = gemm_fold(proj, m_tiles, cur_tile * m_tiles.rows, F + c0 + j);
+          cut[k] = fg[k].c_next <= fg[k].c_last || fu[k].c_next <= fu[k].c_last;
+        }
       }
     }
+    stage_wait(bars_u + 8u * s, ph, status, DEV_ERR_TIMEOUT);
+    const float* sg = ring + (size_t)(s * 2) * SWS_COLS;
+    const float* su = sg + SWS_COLS;
 #pragma unroll
-    for (int k = 0; k < SWIGLU_ITEMS; ++k) {
-      const int f = f0 + k * SWIGLU_THREADS * 4;
-      if (f < F) { pg[k] = gemm_issue4f<WIDE_FOLD_SWIGLU>(proj, m_tiles, fg[k], m, f, doff); pu[k] = gemm_issue4f<WIDE_FOLD_SWIGLU>(proj, m_tiles, fu[k], m, F + f, doff); }
-    }
-#pragma unroll
-    for (int k = 0; k < SWIGLU_ITEMS; ++k) {
-      const int f = f0 + k * SWIGLU_THREADS * 4;
-      if (f < F) {
-        const float4 g = gemm_finish4f(proj, m_tiles, fg[k], doff, pg[k]), u = gemm_finish4f(proj, m_tiles, fu[k], doff, pu[k]);
-        store4(out + (size_t)m * F + f, silu_f(g.x) * u.x, silu_f(g.y) * u.y, silu_f(g.z) * u.z, silu_f(g.w) * u.w);
+    for (int k = 0; k < 2; ++k) {
+      const int j = k ? j1 : j0;
+      if (j < ncol) {
+        float4 g = *reinterpret_cast<const float4*>(sg + j), u = *reinterpret_cast<const float4*>(su + j);
+        if (cut[k]) {   // add the other contributors' sums in CTA order
+          const size_t doff = (size_t)(m - cur_tile * m_tiles.rows) * 128;
+          for (int c = fg[k].c_next; c <= fg[k].c_last; ++c)
+            if (gemm_has_work(proj, m_tiles, c)) {
+              const float4 t = __ldcg(reinterpret_cast<const float4*>(proj.partial + (size_t)c * slot + fg[k].off + doff));
+              g.x += t.x; g.y += t.y; g.z += t.z; g.w += t.w;
+            }
+          for (int c = fu[k].c_next; c <= fu[k].c_last; ++c)
+            if (gemm_has_work(proj, m_tiles, c)) {
+              const float4 t = __ldcg(reinterpret_cast<const float4*>(proj.partial + (size_t)c * slot + fu[k].off + doff));
+              u.x += t.x; u.y += t.y; u.z += t.z; u.w += t.w;
+            }
+        }
+        store4(out + (size_t)m * F + c0 + j, silu_f(g.x) * u.x, silu_f(g.y) * u.y, silu_f(g.z) * u.z, silu_f(g.w) * u.w);
       }
     }
+    __syncthreads();   // every thread is done with the slot
+    if (++s == SWS_STAGES) { s = 0; ph ^= 1u; }
   }
   chain_exit(cs);
 }
 
 // proj: the gate|up projection [M][2F]; out: [M][F].  F must be a multiple of 4.
 cudaError_t launch_swiglu(int dtype, const GemmOut& proj, void* out_t, int F, const int32_t* m_total, int m_max,
-                          Chain* chain, cudaStream_t st) {
+                          int32_t* status, Chain* chain, cudaStream_t st) {
   const int per_cta = SWIGLU_THREADS * SWIGLU_ITEMS * 4;
   dim3 grid((F + per_cta - 1) / per_cta, m_max);
-  if (m_max > WIDE_ROWS_MIN) {   // several row tiles
-    // four CTAs per SM: they share the SM with a CTA of the projection before and of the one after (measured: 3 to 6 alike)
-    const int gy = (4 * wide_sm_count() + (int)grid.x - 1) / (int)grid.x;
-    if (gy < m_max) grid.y = gy;
+  if (m_max > WIDE_ROWS_MIN) {   // several row tiles: three CTAs per SM (64 KB of stages each) walk the rows
+    const size_t smem = (size_t)SWS_STAGES * 2 * SWS_COLS * sizeof(float);
+    static bool attr_set[2] = {false, false};
+    const int di = dtype == RD_DTYPE_FP32 ? 0 : 1;
+    if (!attr_set[di]) {
+      cudaError_t e = cudaErrorInvalidValue;
+      RD_DISPATCH(dtype, e = cudaFuncSetAttribute(swiglu_wide_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      if (e != cudaSuccess) return e;
+      attr_set[di] = true;
+    }
+    grid.x = (F + SWS_COLS - 1) / SWS_COLS;
+    const int gy = (3 * wide_sm_count() + (int)grid.x - 1) / (int)grid.x;
+    grid.y = gy < m_max ? gy : m_max;
     const ChainSync cs = chain ? chain->link(grid.x * grid.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
-    RD_DISPATCH(dtype, launch_pdl(swiglu_wide_kernel<T>, grid, SWIGLU_THREADS, 0, st, proj, (T*)out_t, F, m_total, cs));
+    RD_DISPATCH(dtype, launch_pdl(swiglu_wide_kernel<T>, grid, SWS_THREADS, smem, st, proj, (T*)out_t, F, m_total, status, cs));
     return cudaGetLastError();
   }
   const ChainSync cs = chain ? chain->link(grid.x * grid.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
