@@ -4,6 +4,9 @@
 
 A step is one pass of the whole hot path (draft -> pack -> verify -> accept) for one batch; the
 default workload is the Vicuna-7B-shaped bs1 configuration.  Prints ONE JSON line.
+
+Two side modes print one JSON line per point and a table on stderr instead: `--sweep` (beam width x
+batch at the workload's layer shapes) and `--prefill` (prompt processing).
 """
 from __future__ import annotations
 
