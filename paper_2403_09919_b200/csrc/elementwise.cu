@@ -437,58 +437,115 @@ __global__ void __maxnreg__(88) rope_kv_kernel(float* __restrict__ qkv, GemmOut 
 }
 
 
-// Rows in a loop (see rmsnorm_wide_kernel): blockIdx.y picks the items of a row, blockIdx.x the first row.
+// Many rows: blockIdx.x picks a group of heads (ROPW_COLS columns), blockIdx.y a contiguous run of rows.  The Q, K
+// and V segments of a row (contiguous, ROPW_COLS x 4 bytes each) come in through a ring of shared-memory stages filled
+// by thread 0 with bulk asynchronous copies, ROPW_STAGES - 1 rows ahead (stage.cuh; see swiglu_wide_kernel).  Partial
+// sums of tiles cut between CTAs are added from global memory by the threads whose columns they concern.
+constexpr int ROPW_THREADS = 256;
+constexpr int ROPW_COLS = 1024;     // one item (two adjacent dimensions and their partners half a head on) per thread
+constexpr int ROPW_STAGES = 3;      // 3 x 3 x 4 KB per CTA (static shared memory)
 template <typename T>
-__global__ void __launch_bounds__(ROPE_THREADS, 2)
+__global__ void __launch_bounds__(ROPW_THREADS, 4)
     rope_kv_wide_kernel(float* __restrict__ qkv, GemmOut proj, T* __restrict__ kc, T* __restrict__ vc,
                         const float2* __restrict__ table, RowTables rt, Dims dm, int* status, ChainSync cs) {
   chain_begin(cs);
+  __shared__ __align__(128) float ring[ROPW_STAGES][3][ROPW_COLS];   // 36 KB
+  __shared__ __align__(8) unsigned long long bars[ROPW_STAGES];
+  const uint32_t ring_u = stage_smem_u32(ring), bars_u = stage_smem_u32(bars);
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < ROPW_STAGES; ++s) stage_bar_init(bars_u + 8u * s, 1);
+    stage_bar_init_fence();
+  }
   const int d = dm.d, hd = dm.hd, half = hd >> 1;
-  const int n_items = dm.H * (half >> 1);
-  const int idx = blockIdx.y * ROPE_THREADS + threadIdx.x;
-  const int h = idx / (half >> 1), i = (idx - h * (half >> 1)) * 2;
-  const int o = h * hd + i;
+  const int heads_per_cta = ROPW_COLS / hd;
+  const int h0 = blockIdx.x * heads_per_cta;
+  const int n_heads = min(heads_per_cta, dm.H - h0);
+  const int c0 = h0 * hd, ncol = n_heads * hd;           // this CTA's columns inside each of Q, K, V
+  const uint32_t seg_bytes = (uint32_t)ncol * 4u;
+  const int hl = threadIdx.x / (half >> 1), i = (threadIdx.x - hl * (half >> 1)) * 2;   // head inside the group, dimension
+  const bool active = hl < n_heads;
+  const int j = hl * hd + i;                              // column inside the segment
+  const int h = h0 + hl, o = c0 + j;
   // inside a chain the row count, written ahead of the chain, may be read before the wait
   const bool early = cs.signal_ptr != nullptr && cs.wait_ptr != nullptr;
   int M = early ? *rt.m_total : 0;
-  chain_wait_cta(cs);
+  chain_wait_cta(cs);   // (its barrier also publishes the initialised mbarriers)
   if (!early) M = *rt.m_total;
   const GemmRows m_tiles = gemm_m_tiles(proj, M);
-  if (idx < n_items) {
-    // each CTA takes a contiguous run of rows; the fold of a column changes only from one row tile to the next
-    const int m_end = gemm_rows_begin(M, gridDim.x, blockIdx.x + 1);
-    int cur_tile = -1;
-    GemmFold fq, fk, fv;
-    for (int m = gemm_rows_begin(M, gridDim.x, blockIdx.x); m < m_end; ++m) {
-      float* row = qkv + (size_t)m * 3 * d;
-      const int b = rt.seq[m], slot = rt.slot[m];
-      const float4 cs2 = *reinterpret_cast<const float4*>(table + (size_t)m * half + i);   // (cos, sin) of i and i+1
-      const int m_tile = m / m_tiles.rows;
-      const int r0 = (m - m_tile * m_tiles.rows) * 128, r1 = r0 + half;
-      if (m_tile != cur_tile) {
-        cur_tile = m_tile;
-        fq = gemm_fold_or_none(proj, m_tiles, m_tile * m_tiles.rows, o);
-        fk = gemm_fold_or_none(proj, m_tiles, m_tile * m_tiles.rows, d + o);
-        fv = gemm_fold_or_none(proj, m_tiles, m_tile * m_tiles.rows, 2 * d + o);
-      }
-      const auto pq1 = gemm_issue2<WIDE_FOLD_ROPE>(proj, m_tiles, fq, m, o, r0), pq2 = gemm_issue2<WIDE_FOLD_ROPE>(proj, m_tiles, fq, m, o + half, r1);
-      const auto pk1 = gemm_issue2<WIDE_FOLD_ROPE>(proj, m_tiles, fk, m, d + o, r0), pk2 = gemm_issue2<WIDE_FOLD_ROPE>(proj, m_tiles, fk, m, d + o + half, r1);
-      const auto pv1 = gemm_issue2<WIDE_FOLD_ROPE>(proj, m_tiles, fv, m, 2 * d + o, r0), pv2 = gemm_issue2<WIDE_FOLD_ROPE>(proj, m_tiles, fv, m, 2 * d + o + half, r1);
-      const bool slot_ok = slot >= 0 && slot < dm.max_ctx;
-      if (!slot_ok && idx == 0) atomicOr(status, DEV_ERR_CAPACITY);
-      const float2 q1 = gemm_finish2(proj, m_tiles, fq, r0, pq1), q2 = gemm_finish2(proj, m_tiles, fq, r1, pq2);
-      const float2 k1 = gemm_finish2(proj, m_tiles, fk, r0, pk1), k2 = gemm_finish2(proj, m_tiles, fk, r1, pk2);
-      const float2 v1 = gemm_finish2(proj, m_tiles, fv, r0, pv1), v2 = gemm_finish2(proj, m_tiles, fv, r1, pv2);
-      store2(row + o, q1.x * cs2.x - q2.x * cs2.y, q1.y * cs2.z - q2.y * cs2.w);
-      store2(row + o + half, q2.x * cs2.x + q1.x * cs2.y, q2.y * cs2.z + q1.y * cs2.w);
-      if (slot_ok) {
-        const size_t base = (((size_t)b * dm.H + h) * dm.max_ctx + slot) * hd + i;
-        store2(kc + base, k1.x * cs2.x - k2.x * cs2.y, k1.y * cs2.z - k2.y * cs2.w);
-        store2(kc + base + half, k2.x * cs2.x + k1.x * cs2.y, k2.y * cs2.z + k1.y * cs2.w);
-        store2(vc + base, v1.x, v1.y);
-        store2(vc + base + half, v2.x, v2.y);
+  const int m_begin = gemm_rows_begin(M, gridDim.y, blockIdx.y), m_end = gemm_rows_begin(M, gridDim.y, blockIdx.y + 1);
+  const int n_rows = m_end - m_begin;
+  auto issue = [&](int r) {   // thread 0: row m_begin + r into slot r % ROPW_STAGES
+    const int s = r % ROPW_STAGES;
+    const float* src = qkv + (size_t)(m_begin + r) * 3 * d + c0;
+    stage_expect_tx(bars_u + 8u * s, 3u * seg_bytes);
+#pragma unroll
+    for (int part = 0; part < 3; ++part)
+      stage_copy(ring_u + (uint32_t)((s * 3 + part) * ROPW_COLS) * 4u, src + (size_t)part * d, seg_bytes, bars_u + 8u * s);
+  };
+  if (threadIdx.x == 0) {
+    chain_fence_async_reads();   // the projection wrote its output with ordinary stores
+    for (int r = 0; r < ROPW_STAGES - 1 && r < n_rows; ++r) issue(r);
+  }
+  const bool cut_any = proj.partial != nullptr;
+  const size_t slot_stride = gemm_slot_stride(proj);
+  int tile_end = 0, cur_tile = 0;
+  GemmFold f3[3];          // folds of this thread's Q, K and V columns: they change only from one row tile to the next
+  bool cut = false;
+  uint32_t s = 0, ph = 0;
+  for (int r = 0; r < n_rows; ++r) {
+    const int m = m_begin + r;
+    if (threadIdx.x == 0 && r + ROPW_STAGES - 1 < n_rows) issue(r + ROPW_STAGES - 1);   // slot released by the last barrier
+    int b = 0, slot = -1;
+    float4 cs2 = make_float4(0.f, 0.f, 0.f, 0.f);   // (cos, sin) of i and i+1
+    if (active) {
+      b = rt.seq[m]; slot = rt.slot[m];
+      cs2 = *reinterpret_cast<const float4*>(table + (size_t)m * half + i);
+      if (cut_any && m >= tile_end) {
+        cur_tile = m / m_tiles.rows;
+        tile_end = (cur_tile + 1) * m_tiles.rows;
+        cut = false;
+#pragma unroll
+        for (int part = 0; part < 3; ++part) {
+          f3[part] = gemm_fold(proj, m_tiles, cur_tile * m_tiles.rows, part * d + o);
+          cut = cut || f3[part].c_next <= f3[part].c_last;
+        }
       }
     }
+    stage_wait(bars_u + 8u * s, ph, status, DEV_ERR_TIMEOUT);
+    if (active) {
+      float2 v1[3], v2[3];   // (i, i+1) and (i + half, i + half + 1) of Q, K, V
+#pragma unroll
+      for (int part = 0; part < 3; ++part) {
+        v1[part] = *reinterpret_cast<const float2*>(&ring[s][part][j]);
+        v2[part] = *reinterpret_cast<const float2*>(&ring[s][part][j + half]);
+      }
+      if (cut) {   // add the other contributors' sums in CTA order
+        const size_t doff = (size_t)(m - cur_tile * m_tiles.rows) * 128;
+#pragma unroll
+        for (int part = 0; part < 3; ++part)
+          for (int c = f3[part].c_next; c <= f3[part].c_last; ++c)
+            if (gemm_has_work(proj, m_tiles, c)) {
+              const float* pp = proj.partial + (size_t)c * slot_stride + f3[part].off + doff;
+              const float2 t1 = __ldcg(reinterpret_cast<const float2*>(pp)), t2 = __ldcg(reinterpret_cast<const float2*>(pp + half));
+              v1[part].x += t1.x; v1[part].y += t1.y; v2[part].x += t2.x; v2[part].y += t2.y;
+            }
+      }
+      const bool slot_ok = slot >= 0 && slot < dm.max_ctx;
+      if (!slot_ok && i == 0 && h == 0) atomicOr(status, DEV_ERR_CAPACITY);
+      // the attention kernel reads the rotated Q from the projection's own buffer
+      float* row = qkv + (size_t)m * 3 * d;
+      store2(row + o, v1[0].x * cs2.x - v2[0].x * cs2.y, v1[0].y * cs2.z - v2[0].y * cs2.w);
+      store2(row + o + half, v2[0].x * cs2.x + v1[0].x * cs2.y, v2[0].y * cs2.z + v1[0].y * cs2.w);
+      if (slot_ok) {
+        const size_t base = (((size_t)b * dm.H + h) * dm.max_ctx + slot) * hd + i;
+        store2(kc + base, v1[1].x * cs2.x - v2[1].x * cs2.y, v1[1].y * cs2.z - v2[1].y * cs2.w);
+        store2(kc + base + half, v2[1].x * cs2.x + v1[1].x * cs2.y, v2[1].y * cs2.z + v1[1].y * cs2.w);
+        store2(vc + base, v1[2].x, v1[2].y);
+        store2(vc + base + half, v2[2].x, v2[2].y);
+      }
+    }
+    __syncthreads();   // every thread is done with the slot
+    if (++s == ROPW_STAGES) { s = 0; ph ^= 1u; }
   }
   chain_exit(cs);
 }
@@ -497,11 +554,14 @@ cudaError_t launch_rope_kv(int dtype, float* qkv, const GemmOut& proj, void* kca
                            const RowTables& rt, const Dims& dm, int m_max, int* status, Chain* chain, cudaStream_t st) {
   const int n_items = dm.H * (dm.hd / 4);
   dim3 grid(m_max, (n_items + ROPE_THREADS - 1) / ROPE_THREADS);
-  if (m_max > WIDE_ROWS_MIN) {   // several row tiles
-    const int gx = (2 * wide_sm_count() + (int)grid.y - 1) / (int)grid.y;   // two resident CTAs per SM: one wave walks all rows
-    if (gx < m_max) grid.x = gx;
-    const ChainSync cs = chain ? chain->link(grid.x * grid.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
-    RD_DISPATCH(dtype, launch_pdl(rope_kv_wide_kernel<T>, grid, ROPE_THREADS, 0, st, qkv, proj, (T*)kcache, (T*)vcache,
+  if (m_max > WIDE_ROWS_MIN && ROPW_COLS % dm.hd == 0 && (ROPW_COLS / dm.hd) * (dm.hd / 4) <= ROPW_THREADS) {
+    // several row tiles: four CTAs per SM (36 KB of stages each) walk the rows
+    const int heads_per_cta = ROPW_COLS / dm.hd;
+    dim3 gw((dm.H + heads_per_cta - 1) / heads_per_cta, 1);
+    const int gy = (4 * wide_sm_count() + (int)gw.x - 1) / (int)gw.x;
+    gw.y = gy < m_max ? gy : m_max;
+    const ChainSync cs = chain ? chain->link(gw.x * gw.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
+    RD_DISPATCH(dtype, launch_pdl(rope_kv_wide_kernel<T>, gw, ROPW_THREADS, 0, st, qkv, proj, (T*)kcache, (T*)vcache,
                                   reinterpret_cast<const float2*>(table), rt, dm, status, cs));
     return cudaGetLastError();
   }
