@@ -504,6 +504,11 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
   Bump bp{(char*)workspace, 0};
   carve(bp, dm, h->m_cap, &h->ws);
   h->use_tc = dm.dtype == RD_DTYPE_BF16 && !(cfg->flags & RD_FLAG_FORCE_SIMT);
+  {
+    cudaError_t ce = elementwise_prepare(dm.dtype);
+    if (ce == cudaSuccess) ce = drafter_prepare(dm.dtype);
+    if (ce != cudaSuccess) return init_fail(h, RD_ERR_CUDA, "kernel set-up: %s", cudaGetErrorString(ce));
+  }
   if (h->use_tc) {
     int dev = 0, sms = 0;
     cudaError_t ce = cudaGetDevice(&dev);

@@ -663,6 +663,13 @@ int draft_select_segments(const Dims& dm, int rows, int grid_hint) {
   return S;
 }
 
+// Once per handle (and so per device): opt-in of the one-kernel selection's shared-memory row (opted in by init).
+cudaError_t drafter_prepare(int dtype) {
+  return dtype == RD_DTYPE_FP32
+             ? cudaFuncSetAttribute(draft_select_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)
+             : cudaFuncSetAttribute(draft_select_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+}
+
 // rows = B (call 1) or B * BW.  counters: [B] zero between launches.
 cudaError_t launch_draft_select(int dtype, const GemmOut& proj, int call, float* lse, float* val, int32_t* idx,
                                 const float* score_in, float* score_out, const int32_t* hist_in, int32_t* hist_out,
@@ -700,14 +707,6 @@ cudaError_t launch_draft_select(int dtype, const GemmOut& proj, int call, float*
   const size_t prune = (size_t)dm.BW * dm.BW * sizeof(Cand);
   const size_t smem = select > prune ? select : prune;
   if (smem > 200 * 1024) return cudaErrorInvalidValue;   // vocabulary too large for the shared-memory row
-  static bool attr_set[2] = {false, false};
-  if (!attr_set[dtype == RD_DTYPE_FP32 ? 0 : 1]) {
-    cudaError_t e = dtype == RD_DTYPE_FP32
-                        ? cudaFuncSetAttribute(draft_select_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)
-                        : cudaFuncSetAttribute(draft_select_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e != cudaSuccess) return e;
-    attr_set[dtype == RD_DTYPE_FP32 ? 0 : 1] = true;
-  }
   const ChainSync cs = chain ? chain->link((unsigned)rows) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
   RD_DISPATCH(dtype, launch_pdl(draft_select_kernel<T>, rows, SEL_THREADS, smem, st, proj, call, lse, val, idx, score_in,
                                 score_out, hist_in, hist_out, (const T*)emb, s_new_f, ld_s, (T*)se_t, dm, beams_out,

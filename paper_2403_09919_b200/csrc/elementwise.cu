@@ -731,21 +731,21 @@ __global__ void __launch_bounds__(SWS_THREADS, 3)
   chain_exit(cs);
 }
 
+// Once per handle (and so per device): opt-in of the kernels that take more than 48 KB of dynamic shared memory.
+cudaError_t elementwise_prepare(int dtype) {
+  cudaError_t e = cudaErrorInvalidValue;
+  const int smem = SWS_STAGES * 2 * SWS_COLS * (int)sizeof(float);
+  RD_DISPATCH(dtype, e = cudaFuncSetAttribute(swiglu_wide_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  return e;
+}
+
 // proj: the gate|up projection [M][2F]; out: [M][F].  F must be a multiple of 4.
 cudaError_t launch_swiglu(int dtype, const GemmOut& proj, void* out_t, int F, const int32_t* m_total, int m_max,
                           int32_t* status, Chain* chain, cudaStream_t st) {
   const int per_cta = SWIGLU_THREADS * SWIGLU_ITEMS * 4;
   dim3 grid((F + per_cta - 1) / per_cta, m_max);
   if (m_max > WIDE_ROWS_MIN) {   // several row tiles: three CTAs per SM (64 KB of stages each) walk the rows
-    const size_t smem = (size_t)SWS_STAGES * 2 * SWS_COLS * sizeof(float);
-    static bool attr_set[2] = {false, false};
-    const int di = dtype == RD_DTYPE_FP32 ? 0 : 1;
-    if (!attr_set[di]) {
-      cudaError_t e = cudaErrorInvalidValue;
-      RD_DISPATCH(dtype, e = cudaFuncSetAttribute(swiglu_wide_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-      if (e != cudaSuccess) return e;
-      attr_set[di] = true;
-    }
+    const size_t smem = (size_t)SWS_STAGES * 2 * SWS_COLS * sizeof(float);   // opted in by elementwise_prepare
     grid.x = (F + SWS_COLS - 1) / SWS_COLS;
     const int gy = (3 * wide_sm_count() + (int)grid.x - 1) / (int)grid.x;
     grid.y = gy < m_max ? gy : m_max;

@@ -86,6 +86,8 @@ cudaError_t attn_tc_prepare(int hd, int MW);
 cudaError_t launch_attention_tc(const float* qkv, const void* kcache, const void* vcache, void* out, const RowTables& rt,
                                 const int32_t* seq_off, const Dims& dm, int n_seq, int row_blocks, int n_splits,
                                 float* scratch, int32_t* counters, unsigned long long* dbg, Chain* chain, int shallow, cudaStream_t st);
+cudaError_t elementwise_prepare(int dtype);
+cudaError_t drafter_prepare(int dtype);
 cudaError_t launch_swiglu(int dtype, const GemmOut& proj, void* out_t, int F, const int32_t* m_total, int m_max,
                           int32_t* status, Chain* chain, cudaStream_t st);
 cudaError_t launch_argmax_rows(float* logits, const GemmOut& proj, int V, int32_t* out, const int32_t* out_index,
