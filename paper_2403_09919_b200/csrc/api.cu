@@ -88,6 +88,7 @@ struct rd_handle {
   int trace_next;  // next trace slot, -1 = tracing off
   std::vector<double> trace_bytes;  // weight bytes of each traced launch (0: not a projection)
   int tc_grid, tc_smem;
+  std::vector<TensorMapBox> kv_maps;   // [layer][K | V]: cache planes as [sequences * heads * max_ctx][head dim] matrices
   Chain chain;  // counter hand-off between the launches of a forward pass
   std::unordered_map<const void*, TensorMapBox> maps;               // weights
   std::unordered_map<const void*, std::pair<int, int>> act_shape;   // activation buffers: rows, cols
@@ -311,7 +312,7 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
   // attention launch geometry (tensor-core path): tiles of 16 rows per sequence; keys split over CTAs only
   // for long contexts with few tiles
   int row_blocks = 1, n_splits = 1;
-  bool att_wide = false, att_shallow = false;
+  bool att_wide = false, att_shallow = false, att_t5 = false;
   if (h->use_tc) {
     const int rpb = attn_tc_rows_per_block();
     row_blocks = (rows_per_seq_max + rpb - 1) / rpb;
@@ -320,7 +321,10 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
     // K/V chunk staged once for four times the rows) takes over.
     static const int wide_waves = getenv("RD_ATT_WIDE") ? atoi(getenv("RD_ATT_WIDE")) : 4;   // tuning toggle
     att_wide = wide_waves < 0 || (wide_waves > 0 && blocks > wide_waves * h->tc_grid);   // negative: always
-    if (att_wide) row_blocks = (rows_per_seq_max + attn_wide_rows_per_block() - 1) / attn_wide_rows_per_block();
+    static const int t5_ok = getenv("RD_ATT_T5") ? atoi(getenv("RD_ATT_T5")) : 1;   // tuning toggle
+    att_t5 = att_wide && t5_ok && !h->kv_maps.empty();
+    if (att_t5) row_blocks = (rows_per_seq_max + attn_t5_rows_per_block() - 1) / attn_t5_rows_per_block();
+    else if (att_wide) row_blocks = (rows_per_seq_max + attn_wide_rows_per_block() - 1) / attn_wide_rows_per_block();
     // more 16-row CTAs than SMs (many sequences of a few rows): a two-chunk ring so that three CTAs share an SM
     static const int shallow_ok = getenv("RD_ATT_SHALLOW") ? atoi(getenv("RD_ATT_SHALLOW")) : 1;   // tuning toggle
     att_shallow = shallow_ok && !att_wide && blocks > h->tc_grid;
@@ -347,7 +351,10 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
                                      m_max, w.status, ch, st));
     {
       ProfScope ps(h, 1, 0.0, st);
-      if (h->use_tc && att_wide)
+      if (h->use_tc && att_t5)
+        CK(h, launch_attention_t5(h->kv_maps[(size_t)l * 2].bytes, h->kv_maps[(size_t)l * 2 + 1].bytes, w.qkv, w.attn_t, rt, w.seq_off, dm, n_seq,
+                                  row_blocks, w.status, ch, st));
+      else if (h->use_tc && att_wide)
         CK(h, launch_attention_wide(w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.attn_t, rt, w.seq_off, dm, n_seq,
                                     row_blocks, ch, st));
       else if (h->use_tc)
@@ -516,9 +523,20 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
     if (ce == cudaSuccess) ce = tc_prepare(&h->tc_smem);
     if (ce == cudaSuccess) ce = attn_tc_prepare(dm.hd, dm.MW);
     if (ce == cudaSuccess) ce = attn_wide_prepare(dm.hd, dm.MW);
+    if (ce == cudaSuccess) ce = attn_t5_prepare(dm.hd, dm.MW);
     if (ce != cudaSuccess || sms <= 0)
       return init_fail(h, RD_ERR_CUDA, "tensor-core path set-up: %s", cudaGetErrorString(ce));
     h->tc_grid = sms < TC_MAX_GRID ? sms : TC_MAX_GRID;
+    if (attn_t5_supported(dm.hd)) {
+      // The tensor-core attention multiplies masked-out V rows by exact zeros: the cache has to hold finite values.
+      ce = cudaMemset(h->kv, 0, (size_t)dm.n_layers * 2 * h->kv_plane * esize(dm.dtype));
+      if (ce != cudaSuccess) return init_fail(h, RD_ERR_CUDA, "clearing the KV cache: %s", cudaGetErrorString(ce));
+      h->kv_maps.resize((size_t)dm.n_layers * 2);
+      for (int l = 0; l < dm.n_layers; ++l)
+        for (int which = 0; which < 2; ++which)
+          if (tc_make_map(h->kv_maps[(size_t)l * 2 + which].bytes, kv_plane_ptr(h, l, which), (uint64_t)dm.B * dm.H * dm.max_ctx, dm.hd, 128) != 0)
+            return init_fail(h, RD_ERR_CUDA, "tensor map of the KV cache (layer %d)", l);
+    }
     if (dm.d % 8 || dm.F % 8 || dm.dh % 8) return init_fail(h, RD_ERR_SHAPE, "bf16 needs d_model, d_ffn multiples of 8");
     bool ok = true;
     int failed_rc = 0;

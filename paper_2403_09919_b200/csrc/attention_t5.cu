@@ -1,0 +1,522 @@
+// Tree-masked / causal attention on the 5th-generation tensor cores for launches with many rows per sequence
+// (Sections 3.3, 3.4): head dimension 128, bf16 operands, fp32 accumulation in tensor memory.
+//
+// One CTA = (head, sequence, tile of 128 of its rows).  Keys come in chunks of 128:
+//   S = Q K^T   tcgen05.mma, A = Q tile (128 rows x 128 dims, K-major in shared memory, converted once from the fp32
+//               rows the rotary kernel wrote), B = K chunk (128 keys x 128 dims, K-major, straight from the cache by
+//               TMA), D = S in tensor memory (two buffers, so the next chunk's scores are computed during this
+//               chunk's softmax);
+//   softmax     two threads per query row (= TMEM lane), half of the chunk's keys each: scale, mask, running maximum
+//               and sum in registers (base 2), P written to shared memory as bf16 in the K-major swizzled layout, O in
+//               tensor memory rescaled in place when a row's maximum moved;
+//   O += P V    tcgen05.mma, A = P, B = V chunk as it lies in the cache ([key][dim], i.e. MN-major for this product:
+//               leading byte offset = one 64-dim box of the chunk, stride byte offset = 8 keys, 2048 bytes per 16 keys).
+// Roles: warp 0 lane 0 = TMA producer (K and V rings of two chunks), warp 1 lane 0 = MMA issuer (warp 1 owns the tensor
+// memory), warps 2..9 = softmax and output.  Every wait is bounded (one second): on expiry the CTA raises
+// DEV_ERR_TIMEOUT, lets its copies land, frees its tensor memory and leaves.
+//
+// The chunk's keys past a row's extent are masked by selection, never by arithmetic, and their V rows are multiplied by
+// exact zeros: the cache must hold finite values everywhere (it is cleared once when the handle is created).
+#include <cuda.h>
+
+#include "pdl.cuh"
+#include "rd_internal.cuh"
+
+namespace rd {
+
+namespace {
+
+constexpr int T5_ROWS = 128;      // query rows per CTA (one TMEM lane each)
+constexpr int T5_KEYS = 128;      // keys per chunk
+constexpr int T5_HD = 128;
+constexpr int T5_STAGES = 2;      // K and V chunks in flight
+constexpr int T5_SOFT = 256;       // softmax threads: two per query row
+constexpr int T5_THREADS = 64 + T5_SOFT;
+constexpr uint32_t T5_BLOCK = 128 * 128;            // bytes of one 64-column block of 128 rows (128 B per row)
+constexpr uint32_t T5_TILE = 2 * T5_BLOCK;          // Q tile, K chunk, V chunk, P tile: 32 KB each
+constexpr unsigned long long T5_WAIT_NS = 1000000000ull;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long now_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the CTA is aborting (this or another role gave up).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = now_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try(bar, parity)) return true;
+    if ((it & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (now_ns() - t0 > T5_WAIT_NS) {
+        *abort_flag = 1;
+        atomicOr(status, DEV_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+      "l"(map), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+// K-major operand, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// MN-major operand, 128-byte swizzle: 64 MN-elements (128 bytes) per row of a block, 8 K-rows 1024 bytes apart, the next
+// 64 MN-elements one block (T5_BLOCK bytes) further.
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(T5_BLOCK >> 4) << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// 32 consecutive columns of this thread's lane; the caller waits once after issuing all its loads (a load followed
+// at once by its wait costs a few hundred nanoseconds each time).
+__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, float* r) {
+  uint32_t u[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, "
+      "%20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]), "=r"(u[8]), "=r"(u[9]),
+        "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]), "=r"(u[16]), "=r"(u[17]), "=r"(u[18]),
+        "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]), "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]),
+        "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
+      : "r"(taddr));
+#pragma unroll
+  for (int j = 0; j < 32; ++j) r[j] = __uint_as_float(u[j]);
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, "
+      "%19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+      "r"(__float_as_uint(r[0])), "r"(__float_as_uint(r[1])), "r"(__float_as_uint(r[2])), "r"(__float_as_uint(r[3])),
+      "r"(__float_as_uint(r[4])), "r"(__float_as_uint(r[5])), "r"(__float_as_uint(r[6])), "r"(__float_as_uint(r[7])),
+      "r"(__float_as_uint(r[8])), "r"(__float_as_uint(r[9])), "r"(__float_as_uint(r[10])), "r"(__float_as_uint(r[11])),
+      "r"(__float_as_uint(r[12])), "r"(__float_as_uint(r[13])), "r"(__float_as_uint(r[14])), "r"(__float_as_uint(r[15])),
+      "r"(__float_as_uint(r[16])), "r"(__float_as_uint(r[17])), "r"(__float_as_uint(r[18])), "r"(__float_as_uint(r[19])),
+      "r"(__float_as_uint(r[20])), "r"(__float_as_uint(r[21])), "r"(__float_as_uint(r[22])), "r"(__float_as_uint(r[23])),
+      "r"(__float_as_uint(r[24])), "r"(__float_as_uint(r[25])), "r"(__float_as_uint(r[26])), "r"(__float_as_uint(r[27])),
+      "r"(__float_as_uint(r[28])), "r"(__float_as_uint(r[29])), "r"(__float_as_uint(r[30])), "r"(__float_as_uint(r[31]))
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void soft_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+struct T5Params {
+  const float* qkv;            // [M][3d] fp32, Q rotated in place by the rotary kernel
+  __nv_bfloat16* out;          // [M][d]
+  RowTables rt;
+  const int32_t* seq_off;
+  Dims dm;
+  int row_tiles;               // 128-row tiles per sequence (bound)
+  int32_t* status;
+  ChainSync cs;
+};
+
+__global__ void __launch_bounds__(T5_THREADS, 1)
+    attention_t5_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const T5Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // ---- shared memory carve-up (operand tiles 1024-byte aligned for the 128-byte swizzle)
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - raw);                 // generic pointer to the same place
+  const uint32_t sQ = base, sK = sQ + T5_TILE, sV = sK + T5_STAGES * T5_TILE, sP = sV + T5_STAGES * T5_TILE;
+  const uint32_t bar0 = sP + T5_TILE;
+  enum { Q_FULL = 0, K_FULL = 1, V_FULL = 3, K_EMPTY = 5, V_EMPTY = 7, S_FULL = 9, S_EMPTY = 11, P_FULL = 13, P_EMPTY = 14, N_BARS = 15 };
+  auto bar = [&](int i) { return bar0 + 8u * i; };
+  uint8_t* misc = gen + (bar0 - base) + 8u * 16;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
+  volatile int* soft_ok = reinterpret_cast<volatile int*>(misc + 8);     // [2]: outcome of a bounded wait, told to all rows
+  int32_t* s_ncache = reinterpret_cast<int32_t*>(misc + 16);              // [T5_ROWS]
+  float* s_red = reinterpret_cast<float*>(misc + 16 + T5_ROWS * 4);       // [2][2][T5_ROWS] row maxima of the halves, [2][T5_ROWS] their sums
+  uint32_t* s_mask = reinterpret_cast<uint32_t*>(misc + 16 + T5_ROWS * 4 + 6 * T5_ROWS * 4);   // [T5_ROWS][MW]
+
+  // Tensor memory first (512 columns: two score buffers and the output), before the dependents may start.
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  chain_begin(p.cs);
+  // Launched inside a chain, the kernel may read before its wait whatever the launches ahead of the chain wrote: the
+  // row tables and the tree mask.  Q and this pass's K/V come from the kernel right before it.
+  const bool early = p.cs.signal_ptr != nullptr;
+  if (!early) chain_wait_cta(p.cs);
+  if (threadIdx.x == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
+    mbar_init(bar(Q_FULL), T5_SOFT);
+    for (int s = 0; s < T5_STAGES; ++s) {
+      mbar_init(bar(K_FULL + s), 1); mbar_init(bar(V_FULL + s), 1);
+      mbar_init(bar(K_EMPTY + s), 1); mbar_init(bar(V_EMPTY + s), 1);
+      mbar_init(bar(S_FULL + s), 1); mbar_init(bar(S_EMPTY + s), T5_SOFT);
+    }
+    mbar_init(bar(P_FULL), T5_SOFT); mbar_init(bar(P_EMPTY), 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  const Dims& dm = p.dm;
+  const int h = blockIdx.x;
+  // the tiles of a sequence are handed out last first: without a tree mask a later tile has more keys to walk, and
+  // the longest CTAs should not be the last to start
+  const int b = blockIdx.y / p.row_tiles, rb = p.row_tiles - 1 - (blockIdx.y - b * p.row_tiles);
+  const int seq_row0 = p.seq_off[b], seq_rows = p.seq_off[b + 1] - seq_row0;
+  const int row0 = seq_row0 + rb * T5_ROWS;
+  const int nrows = min(T5_ROWS, seq_rows - rb * T5_ROWS);   // <= 0: nothing to do for this tile (same for all roles)
+  const bool tree = p.rt.mask != nullptr;
+  const int MW = dm.MW;
+  int kext = 0, nc_min = 0, tree_base = 0;
+  if (nrows > 0) {
+    const int nc_first = p.rt.n_cache[row0], nc_last = p.rt.n_cache[row0 + nrows - 1];
+    tree_base = nc_first;
+    kext = min(tree ? tree_base + seq_rows : nc_last, dm.max_ctx);
+    nc_min = tree ? tree_base : nc_first;   // every valid row attends at least the keys below this
+  }
+  const int n_chunks = (kext + T5_KEYS - 1) / T5_KEYS;
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;   // columns [0,128) and [128,256): scores, [256,384): output
+
+  if (warp == 0) {
+    // ===================== TMA producer =====================
+    if (lane == 0 && n_chunks > 0) {
+      if (early) chain_wait_thread(p.cs);
+      chain_fence_async_reads();   // this pass's keys and values were written with ordinary stores by the rotary kernel
+      const int key_row0 = (b * dm.H + h) * dm.max_ctx;   // first row of this (sequence, head) in the cache plane
+      bool ok = true;
+      for (int c = 0; c < n_chunks && ok; ++c) {
+        const int s = c & 1;
+        const uint32_t ph = (c >> 1) & 1;
+        if (c >= T5_STAGES) {
+          if (!mbar_wait(bar(K_EMPTY + s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        }
+        mbar_expect_tx(bar(K_FULL + s), T5_TILE);
+        tma_load_2d(sK + s * T5_TILE, &map_k, bar(K_FULL + s), 0, key_row0 + c * T5_KEYS);
+        tma_load_2d(sK + s * T5_TILE + T5_BLOCK, &map_k, bar(K_FULL + s), 64, key_row0 + c * T5_KEYS);
+        if (c >= T5_STAGES) {
+          if (!mbar_wait(bar(V_EMPTY + s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        }
+        mbar_expect_tx(bar(V_FULL + s), T5_TILE);
+        tma_load_2d(sV + s * T5_TILE, &map_v, bar(V_FULL + s), 0, key_row0 + c * T5_KEYS);
+        tma_load_2d(sV + s * T5_TILE + T5_BLOCK, &map_v, bar(V_FULL + s), 64, key_row0 + c * T5_KEYS);
+      }
+      if (!ok || *abort_flag) {  // give the copies already issued time to land before the CTA's shared memory is released
+        const unsigned long long t0 = now_ns();
+        while (now_ns() - t0 < 2000000ull) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer =====================
+    if (lane == 0 && n_chunks > 0) {
+      const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(T5_KEYS >> 3) << 17) | ((uint32_t)(T5_ROWS >> 4) << 24);
+      const uint32_t idesc_pv = idesc_qk | (1u << 16);   // second operand MN-major; N = 128 head dimensions
+      bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag, p.status);
+      auto issue_qk = [&](int c) {
+        const int s = c & 1;
+        const uint32_t ph = (c >> 1) & 1;
+        if (!mbar_wait(bar(K_FULL + s), ph, abort_flag, p.status)) return false;
+        if (!mbar_wait(bar(S_EMPTY + s), ph ^ 1u, abort_flag, p.status)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < T5_HD / 16; ++kk) {
+          const uint32_t off = (uint32_t)(kk >> 2) * T5_BLOCK + (uint32_t)(kk & 3) * 32u;
+          umma_bf16(tmem + (uint32_t)s * T5_KEYS, desc_kmajor(sQ + off), desc_kmajor(sK + s * T5_TILE + off), idesc_qk, kk > 0 ? 1u : 0u);
+        }
+        umma_commit(bar(S_FULL + s));
+        umma_commit(bar(K_EMPTY + s));
+        return true;
+      };
+      if (ok) ok = issue_qk(0);
+      for (int c = 0; c < n_chunks && ok; ++c) {
+        const int s = c & 1;
+        const uint32_t ph = (c >> 1) & 1;
+        if (c + 1 < n_chunks) {
+          if (!issue_qk(c + 1)) { ok = false; break; }
+        }
+        if (!mbar_wait(bar(P_FULL), (uint32_t)(c & 1), abort_flag, p.status)) { ok = false; break; }
+        if (!mbar_wait(bar(V_FULL + s), ph, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < T5_KEYS / 16; ++kk) {
+          const uint32_t aoff = (uint32_t)(kk >> 2) * T5_BLOCK + (uint32_t)(kk & 3) * 32u;   // P: 16 keys further along K
+          umma_bf16(tmem + 2u * T5_KEYS, desc_kmajor(sP + aoff), desc_mnmajor(sV + s * T5_TILE + (uint32_t)kk * 2048u), idesc_pv,
+                    (c > 0 || kk > 0) ? 1u : 0u);
+        }
+        umma_commit(bar(V_EMPTY + s));
+        umma_commit(bar(P_EMPTY));   // P may be overwritten and O is up to date
+      }
+    }
+  } else {
+    // ===================== softmax and output (warps 2..9) =====================
+    // Two threads per query row (= TMEM lane): a warp may only touch the lane quarter (warp id mod 4), so warps w and
+    // w + 4 share a quarter; the first takes keys 0..63 of a chunk and output dimensions 0..63, the second the rest.
+    const int q4 = warp & 3;                      // TMEM lane quarter this warp may access
+    const int hf = (warp - 2) >> 2;               // which half of the chunk's keys / of the head dimensions
+    const int t = q4 * 32 + lane;                 // row inside the tile
+    const int st = threadIdx.x - 64;              // 0..255 (for cooperative loads)
+    const uint32_t lane_addr = (uint32_t)(q4 * 32) << 16;
+    const bool valid = t < nrows;
+    if (n_chunks > 0) {
+      // row tables and mask do not depend on the preceding kernel
+      if (st < T5_ROWS) s_ncache[st] = st < nrows ? p.rt.n_cache[row0 + st] : 0;
+      if (tree)
+        for (int idx = st; idx < T5_ROWS * MW; idx += T5_SOFT) {
+          const int r = idx / MW, wd = idx - r * MW;
+          s_mask[idx] = r < nrows ? p.rt.mask[((size_t)b * dm.NMAX + rb * T5_ROWS + r) * MW + wd] : 0u;
+        }
+      if (st == 0 && early) chain_wait_thread(p.cs);
+      soft_bar_sync();
+      // Q tile -> bf16, K-major swizzled (16-byte chunk c of row r lands at chunk c ^ (r & 7) of its 128-byte line).
+      // A warp converts two rows per pass: lane l takes the eight dimensions of chunk l & 15 of row 2i + (l >> 4), so a
+      // pass reads two contiguous 512-byte rows.
+      {
+        const int cq = lane & 15;
+        const int wrow0 = (warp - 2) * (T5_ROWS / 8);   // sixteen rows per warp
+#pragma unroll 4
+        for (int i = 0; i < T5_ROWS / 16; ++i) {
+          const int r = wrow0 + 2 * i + (lane >> 4);
+          uint4 v = make_uint4(0u, 0u, 0u, 0u);
+          if (r < nrows) {
+            const float* q = p.qkv + (size_t)(row0 + r) * 3 * dm.d + h * T5_HD + cq * 8;
+            const float4 a = __ldcg(reinterpret_cast<const float4*>(q)), bq = __ldcg(reinterpret_cast<const float4*>(q + 4));
+            v = make_uint4(pack_bf16(a.x, a.y), pack_bf16(a.z, a.w), pack_bf16(bq.x, bq.y), pack_bf16(bq.z, bq.w));
+          }
+          *reinterpret_cast<uint4*>(gen + (size_t)(cq >> 3) * T5_BLOCK + r * 128 + (((cq & 7) ^ (r & 7)) << 4)) = v;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(bar(Q_FULL));
+      }
+      const int nc_row = s_ncache[t];
+      const float scale2 = rsqrtf((float)T5_HD) * 1.4426950408889634f;   // 1/sqrt(hd) * log2(e)
+      float m_run = -INFINITY, l_run = 0.f;       // l_run: this thread's half of the row's sum
+      bool ok = true;
+      uint32_t vote = 0;
+      // one thread does each bounded wait and tells the others, so that all of them take the same branch
+      auto wait_all = [&](uint32_t b, uint32_t parity) {
+        volatile int* slot = soft_ok + (vote & 1u);
+        ++vote;
+        if (st == 0) *slot = mbar_wait(b, parity, abort_flag, p.status) ? 1 : 0;
+        soft_bar_sync();
+        return *slot != 0;
+      };
+      // may row t attend key `key`?  (selection, never arithmetic: masked scores may be anything)
+      auto visible = [&](int key) {
+        bool vis = key < nc_row;
+        if (tree && key >= tree_base) {
+          const int tb = key - tree_base;
+          if (tb < seq_rows) vis = (s_mask[t * MW + (tb >> 5)] >> (tb & 31)) & 1u;
+        }
+        return vis;
+      };
+      constexpr int HALF = T5_KEYS / 2;
+      for (int c = 0; c < n_chunks; ++c) {
+        const int s = c & 1;
+        const uint32_t ph = (c >> 1) & 1;
+        const int k0 = c * T5_KEYS + hf * HALF;   // first key of this thread's half
+        ok = wait_all(bar(S_FULL + s), ph);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t s_addr = tmem + lane_addr + (uint32_t)s * T5_KEYS + (uint32_t)hf * HALF;
+        const bool all_visible = c * T5_KEYS + T5_KEYS <= nc_min;
+        // ---- pass A over this thread's 64 scores, 32 at a time (rolled loops: the unrolled code of a whole row does
+        // not fit the instruction cache): maximum of the visible ones
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll 1
+        for (int g = 0; g < HALF / 32; ++g) {
+          float sc[32];
+          tmem_ld32_nowait(s_addr + g * 32, sc);
+          tmem_ld_wait();
+          if (all_visible) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (visible(k0 + g * 32 + j)) mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
+          }
+        }
+        // the softmax runs in base 2: 1/sqrt(hd) * log2(e) is folded into one multiply-add per score
+        float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale2;   // scale2 > 0
+        // the row's maximum over both halves; the same barrier tells that the previous chunk's P V has read P (which also
+        // means O is up to date), so P may be written after it
+        s_red[(c & 1) * 2 * T5_ROWS + hf * T5_ROWS + t] = mx;
+        if (c > 0) {
+          ok = wait_all(bar(P_EMPTY), (uint32_t)((c - 1) & 1));
+          if (!ok) break;
+          tc_fence_after();
+        } else {
+          soft_bar_sync();
+        }
+        mx = fmaxf(mx, s_red[(c & 1) * 2 * T5_ROWS + (hf ^ 1) * T5_ROWS + t]);
+        const float m_new = fmaxf(m_run, mx);
+        const float corr = (m_new == -INFINITY) ? 1.f : fast_exp2(m_run - m_new);
+        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+        // ---- pass B: probabilities -> shared memory (bf16, K-major swizzled: 16-byte chunk cc of row t lands at chunk
+        // cc ^ (t & 7) of its 128-byte line; this thread's 64 keys are block hf of the tile), row sum
+        float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+        for (int g = 0; g < HALF / 32; ++g) {
+          float sc[32];
+          tmem_ld32_nowait(s_addr + g * 32, sc);
+          tmem_ld_wait();
+          if (all_visible) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) { sc[j] = fast_exp2(fmaf(sc[j], scale2, -m_use)); sum4[j & 3] += sc[j]; }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              sc[j] = visible(k0 + g * 32 + j) ? fast_exp2(fmaf(sc[j], scale2, -m_use)) : 0.f;
+              sum4[j & 3] += sc[j];
+            }
+          }
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int cc = g * 4 + q;   // 16-byte chunk (8 keys) inside block hf
+            const uint4 v = make_uint4(pack_bf16(sc[q * 8], sc[q * 8 + 1]), pack_bf16(sc[q * 8 + 2], sc[q * 8 + 3]),
+                                       pack_bf16(sc[q * 8 + 4], sc[q * 8 + 5]), pack_bf16(sc[q * 8 + 6], sc[q * 8 + 7]));
+            *reinterpret_cast<uint4*>(gen + (sP - base) + (size_t)hf * T5_BLOCK + t * 128 + ((cc ^ (t & 7)) << 4)) = v;
+          }
+        }
+        // the score buffer is free for the chunk after next
+        tc_fence_before();
+        mbar_arrive(bar(S_EMPTY + s));
+        l_run = l_run * corr + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+        m_run = m_new;
+        // ---- O *= corr (this thread's 64 dimensions, in tensor memory), unless no row of this warp changed its maximum
+        if (c > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
+          const uint32_t o_addr = tmem + lane_addr + 2u * T5_KEYS + (uint32_t)hf * (T5_HD / 2);
+#pragma unroll 1
+          for (int g = 0; g < T5_HD / 64; ++g) {
+            float ov[32];
+            tmem_ld32_nowait(o_addr + g * 32, ov);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) ov[j] *= corr;
+            tmem_st32(o_addr + g * 32, ov);
+          }
+          tmem_st_wait();
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P was written with ordinary stores
+        tc_fence_before();
+        mbar_arrive(bar(P_FULL));
+      }
+      // ---- output: O / l, each thread its 64 dimensions
+      if (ok) {
+        s_red[4 * T5_ROWS + hf * T5_ROWS + t] = l_run;
+        ok = wait_all(bar(P_EMPTY), (uint32_t)((n_chunks - 1) & 1));
+      }
+      if (ok) {
+        tc_fence_after();
+        const float l_row = l_run + s_red[4 * T5_ROWS + (hf ^ 1) * T5_ROWS + t];
+        const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
+        const uint32_t o_addr = tmem + lane_addr + 2u * T5_KEYS + (uint32_t)hf * (T5_HD / 2);
+        __nv_bfloat16* o = p.out + (size_t)(row0 + (valid ? t : 0)) * dm.d + h * T5_HD + hf * (T5_HD / 2);
+#pragma unroll 1
+        for (int g = 0; g < T5_HD / 64; ++g) {
+          float ov[32];
+          tmem_ld32_nowait(o_addr + g * 32, ov);
+          tmem_ld_wait();
+          if (valid) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              *reinterpret_cast<uint4*>(o + g * 32 + q * 8) =
+                  make_uint4(pack_bf16(ov[q * 8] * inv, ov[q * 8 + 1] * inv), pack_bf16(ov[q * 8 + 2] * inv, ov[q * 8 + 3] * inv),
+                             pack_bf16(ov[q * 8 + 4] * inv, ov[q * 8 + 5] * inv), pack_bf16(ov[q * 8 + 6] * inv, ov[q * 8 + 7] * inv));
+          }
+        }
+      }
+    }
+  }
+
+  // a tile without rows still waits for its predecessor before it reports completion (the hand-off's ordering is
+  // transitive only through CTAs that have seen the launch before them complete)
+  if (n_chunks == 0 && threadIdx.x == 0) chain_wait_thread(p.cs);
+  // ---- teardown: everyone meets, then the allocating warp frees the tensor memory
+  tc_fence_before();
+  __syncthreads();
+  chain_exit(p.cs);
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+  }
+}
+
+size_t t5_smem_bytes(int MW) {
+  return 1024 + (size_t)(1 + 2 * T5_STAGES + 1) * T5_TILE + 8 * 16 + 16 + T5_ROWS * 4 + 6 * T5_ROWS * 4 + (size_t)T5_ROWS * MW * 4 + 64;
+}
+
+}  // namespace
+
+int attn_t5_rows_per_block() { return T5_ROWS; }
+bool attn_t5_supported(int hd) { return hd == T5_HD; }
+
+cudaError_t attn_t5_prepare(int hd, int MW) {
+  if (hd != T5_HD) return cudaSuccess;
+  return cudaFuncSetAttribute(attention_t5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t5_smem_bytes(MW));
+}
+
+// map_k / map_v: tensor maps of the layer's K and V planes ([sequences * heads * max_ctx rows][128 dims], box 64 x 128).
+// grid (H, sequences * row_tiles): row_tiles tiles of 128 rows cover the longest sequence of the launch.
+cudaError_t launch_attention_t5(const void* map_k, const void* map_v, const float* qkv, void* out, const RowTables& rt,
+                                const int32_t* seq_off, const Dims& dm, int n_seq, int row_tiles, int32_t* status, Chain* chain,
+                                cudaStream_t st) {
+  if (dm.hd != T5_HD) return cudaErrorInvalidValue;
+  dim3 grid(dm.H, n_seq * row_tiles);
+  T5Params p;
+  p.qkv = qkv; p.out = (__nv_bfloat16*)out; p.rt = rt; p.seq_off = seq_off; p.dm = dm; p.row_tiles = row_tiles; p.status = status;
+  p.cs = chain ? chain->link(grid.x * grid.y) : ChainSync{nullptr, 0u, nullptr, status, nullptr};
+  launch_pdl(attention_t5_kernel, grid, T5_THREADS, t5_smem_bytes(dm.MW), st, *(const CUtensorMap*)map_k, *(const CUtensorMap*)map_v, p);
+  return cudaGetLastError();
+}
+
+}  // namespace rd

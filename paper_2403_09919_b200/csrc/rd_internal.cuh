@@ -77,6 +77,13 @@ cudaError_t launch_attention(int dtype, const float* qkv, const void* kcache, co
 // Tensor-core attention (bf16): KV tiles staged through shared memory, split over the keys.
 size_t attn_tc_scratch_floats(int blocks, int n_splits, int hd);
 // many rows per sequence (prompts, wide beams, large batches): tiles of 64 rows, a warp per 16 of them
+// head dimension 128, many rows per sequence: tcgen05 attention, tiles of 128 rows
+int attn_t5_rows_per_block();
+bool attn_t5_supported(int hd);
+cudaError_t attn_t5_prepare(int hd, int MW);
+cudaError_t launch_attention_t5(const void* map_k, const void* map_v, const float* qkv, void* out, const RowTables& rt,
+                                const int32_t* seq_off, const Dims& dm, int n_seq, int row_tiles, int32_t* status, Chain* chain,
+                                cudaStream_t st);
 int attn_wide_rows_per_block();
 cudaError_t attn_wide_prepare(int hd, int MW);
 cudaError_t launch_attention_wide(const float* qkv, const void* kcache, const void* vcache, void* out, const RowTables& rt,
