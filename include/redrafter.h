@@ -119,7 +119,9 @@ RD_API size_t redrafter_kv_bytes(const rd_config* cfg);
 
 /* Create a handle.  `kv_cache` and `workspace` are device pointers (256-byte aligned) that the
  * handle uses until redrafter_destroy; their contents are owned by the library while it lives.
- * Host-only apart from building TMA descriptors; enqueues a clear of the state on `stream 0`.
+ * Host-only apart from building TMA descriptors; enqueues a clear of the state on `stream 0` and, in bf16 with head
+ * dimension 128, clears the KV cache (the tensor-core attention kernel multiplies the value rows of masked-out keys by
+ * exact zeros, so every slot has to hold finite values).
  * Errors: INVALID_ARG, SHAPE (head_dim not 64 or 128, d_model/d_ffn not multiples of 64 in bf16,
  * beam_width > vocab, NMAX > 1024), CAPACITY (buffers too small), CUDA. */
 RD_API int redrafter_init(const rd_config* cfg, const rd_weights* weights, void* kv_cache, size_t kv_bytes,

@@ -226,6 +226,44 @@ def test_wide_beam_whose_rows_fit_one_tile_after_all():
     check_verify(rig, beams_alphabet=3)
 
 
+def test_long_prompts_head_dim_128():
+    """Four prompts (700, 300, 120 and 40 tokens) at head dimension 128 in an engine sized for 16 sequences: passes of up
+    to 656 rows.  The long sequence's first pass takes the tensor-core (tcgen05) attention kernel -- 128-row causal
+    tiles, the last one partly filled, chunks of 128 keys of which the last lies partly beyond every row's extent, tiles
+    of the other sequences without rows; later passes run on top of the cache the first wrote.  State and a verification
+    on top of it must match the oracle for every sequence."""
+    cfg = dict(RAGGED, max_batch=16, max_ctx=800)   # d_model 512, 4 heads of 128
+    rig = Rig(cfg=cfg)
+    rng = np.random.default_rng(12)
+    prompts = [rng.integers(0, 1000, size=n) for n in (700, 300, 120, 40)]
+    rig.eng.prefill(prompts)
+    rig.eng.poll()
+    c_ctx, c_root, c_h = rig.eng.get_state()
+    refs = []
+    for b, pr in enumerate(prompts):
+        kv = rig.new_kv()
+        ctx, g, h = ora.prefill(rig.W, cfg, pr, kv)
+        assert int(c_ctx[b]) == ctx
+        assert rel_err(c_h[b].cpu().numpy()[None], np.asarray(h)[None]) < REL
+        refs.append((kv, ctx, g, h))
+    roots = np.array([r[2] for r in refs])
+    hs = np.stack([np.asarray(r[3]) for r in refs]).astype(np.float32)
+    rig.eng.set_state(None, dev(roots), dev(hs, torch.float32))
+    beams = rng.integers(0, 4, size=(4, 8, 5))
+    pk = rig.eng.pack(dev(beams))
+    argmax, hidden, logits = rig.eng.verify(pk, want_logits=True)
+    rig.eng.poll()
+    for b, (kv, ctx, g, h) in enumerate(refs):
+        aug = np.concatenate([np.full((8, 1), g), beams[b]], axis=1)
+        p = ora.pack_beam(aug, ctx)
+        n = p["n"]
+        assert int(pk.n[b]) == n
+        rh, rl = ora.llm_forward(rig.W, cfg, p["tokens"], p["pos"], p["mask"], kv, ctx)
+        assert rel_err(logits[b, :n].cpu().numpy(), rl) < REL
+        sure = decided(rl)
+        assert (argmax[b, :n].cpu().numpy()[sure] == rl.argmax(1)[sure]).all()
+
+
 def test_batched_ragged_many_rows():
     """Batch 16 x beam width 16: up to 1296 compact rows, six activation tiles, per-sequence contexts."""
     cfg = dict(RAGGED, max_batch=16, beam_width=16, beam_length=5, max_ctx=260)
