@@ -193,13 +193,13 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
   if (threadIdx.x == 0) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
-    mbar_init(bar(Q_FULL), T5_SOFT);
+    mbar_init(bar(Q_FULL), T5_SOFT / 32);   // one arrival per softmax warp (256 arrivals on one barrier would serialise)
     for (int s = 0; s < T5_STAGES; ++s) {
       mbar_init(bar(K_FULL + s), 1); mbar_init(bar(V_FULL + s), 1);
       mbar_init(bar(K_EMPTY + s), 1); mbar_init(bar(V_EMPTY + s), 1);
-      mbar_init(bar(S_FULL + s), 1); mbar_init(bar(S_EMPTY + s), T5_SOFT);
+      mbar_init(bar(S_FULL + s), 1); mbar_init(bar(S_EMPTY + s), T5_SOFT / 32);
     }
-    mbar_init(bar(P_FULL), T5_SOFT); mbar_init(bar(P_EMPTY), 1);
+    mbar_init(bar(P_FULL), T5_SOFT / 32); mbar_init(bar(P_EMPTY), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -334,7 +334,8 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
           *reinterpret_cast<uint4*>(gen + (size_t)(cq >> 3) * T5_BLOCK + r * 128 + (((cq & 7) ^ (r & 7)) << 4)) = v;
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(bar(Q_FULL));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(Q_FULL));
       }
       const int nc_row = s_ncache[t];
       const float scale2 = rsqrtf((float)T5_HD) * 1.4426950408889634f;   // 1/sqrt(hd) * log2(e)
@@ -368,21 +369,25 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         tc_fence_after();
         const uint32_t s_addr = tmem + lane_addr + (uint32_t)s * T5_KEYS + (uint32_t)hf * HALF;
         const bool all_visible = c * T5_KEYS + T5_KEYS <= nc_min;
-        // ---- pass A over this thread's 64 scores, 32 at a time (rolled loops: the unrolled code of a whole row does
-        // not fit the instruction cache): maximum of the visible ones
+        // ---- this thread's 64 scores into registers (one wait for both loads); the score buffer is then free for the
+        // chunk after next
+        float sc[HALF];
+        tmem_ld32_nowait(s_addr, sc);
+        tmem_ld32_nowait(s_addr + 32, sc + 32);
+        tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(S_EMPTY + s));
+        // ---- maximum of the visible ones (masked scores become -inf by selection)
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll 1
-        for (int g = 0; g < HALF / 32; ++g) {
-          float sc[32];
-          tmem_ld32_nowait(s_addr + g * 32, sc);
-          tmem_ld_wait();
-          if (all_visible) {
+        if (all_visible) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
-          } else {
+          for (int j = 0; j < HALF; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
+        } else {
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (visible(k0 + g * 32 + j)) mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
+          for (int j = 0; j < HALF; ++j) {
+            sc[j] = visible(k0 + j) ? sc[j] : -INFINITY;
+            mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
           }
         }
         // the softmax runs in base 2: 1/sqrt(hd) * log2(e) is folded into one multiply-add per score
@@ -401,35 +406,17 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         const float m_new = fmaxf(m_run, mx);
         const float corr = (m_new == -INFINITY) ? 1.f : fast_exp2(m_run - m_new);
         const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-        // ---- pass B: probabilities -> shared memory (bf16, K-major swizzled: 16-byte chunk cc of row t lands at chunk
+        // ---- probabilities -> shared memory (bf16, K-major swizzled: 16-byte chunk cc of row t lands at chunk
         // cc ^ (t & 7) of its 128-byte line; this thread's 64 keys are block hf of the tile), row sum
         float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 1
-        for (int g = 0; g < HALF / 32; ++g) {
-          float sc[32];
-          tmem_ld32_nowait(s_addr + g * 32, sc);
-          tmem_ld_wait();
-          if (all_visible) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) { sc[j] = fast_exp2(fmaf(sc[j], scale2, -m_use)); sum4[j & 3] += sc[j]; }
-          } else {
+        for (int j = 0; j < HALF; ++j) { sc[j] = fast_exp2(fmaf(sc[j], scale2, -m_use)); sum4[j & 3] += sc[j]; }   // 2^(-inf) = 0
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              sc[j] = visible(k0 + g * 32 + j) ? fast_exp2(fmaf(sc[j], scale2, -m_use)) : 0.f;
-              sum4[j & 3] += sc[j];
-            }
-          }
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const int cc = g * 4 + q;   // 16-byte chunk (8 keys) inside block hf
-            const uint4 v = make_uint4(pack_bf16(sc[q * 8], sc[q * 8 + 1]), pack_bf16(sc[q * 8 + 2], sc[q * 8 + 3]),
-                                       pack_bf16(sc[q * 8 + 4], sc[q * 8 + 5]), pack_bf16(sc[q * 8 + 6], sc[q * 8 + 7]));
-            *reinterpret_cast<uint4*>(gen + (sP - base) + (size_t)hf * T5_BLOCK + t * 128 + ((cc ^ (t & 7)) << 4)) = v;
-          }
+        for (int cc = 0; cc < HALF / 8; ++cc) {
+          const uint4 v = make_uint4(pack_bf16(sc[cc * 8], sc[cc * 8 + 1]), pack_bf16(sc[cc * 8 + 2], sc[cc * 8 + 3]),
+                                     pack_bf16(sc[cc * 8 + 4], sc[cc * 8 + 5]), pack_bf16(sc[cc * 8 + 6], sc[cc * 8 + 7]));
+          *reinterpret_cast<uint4*>(gen + (sP - base) + (size_t)hf * T5_BLOCK + t * 128 + ((cc ^ (t & 7)) << 4)) = v;
         }
-        // the score buffer is free for the chunk after next
-        tc_fence_before();
-        mbar_arrive(bar(S_EMPTY + s));
         l_run = l_run * corr + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
         m_run = m_new;
         // ---- O *= corr (this thread's 64 dimensions, in tensor memory), unless no row of this warp changed its maximum
@@ -448,7 +435,8 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P was written with ordinary stores
         tc_fence_before();
-        mbar_arrive(bar(P_FULL));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(P_FULL));
       }
       // ---- output: O / l, each thread its 64 dimensions
       if (ok) {
