@@ -169,12 +169,11 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
   uint8_t* gen = smem_raw + (base - raw);                 // generic pointer to the same place
   const uint32_t sQ = base, sK = sQ + T5_TILE, sV = sK + T5_STAGES * T5_TILE, sP = sV + T5_STAGES * T5_TILE;
   const uint32_t bar0 = sP + T5_TILE;
-  enum { Q_FULL = 0, K_FULL = 1, V_FULL = 3, K_EMPTY = 5, V_EMPTY = 7, S_FULL = 9, S_EMPTY = 11, P_FULL = 13, P_EMPTY = 14, N_BARS = 15 };
+  enum { Q_FULL = 0, K_FULL = 1, V_FULL = 3, K_EMPTY = 5, V_EMPTY = 7, S_FULL = 9, S_EMPTY = 11, P_FULL = 13, P_EMPTY = 14, X_FULL = 15, N_BARS = 16 };
   auto bar = [&](int i) { return bar0 + 8u * i; };
   uint8_t* misc = gen + (bar0 - base) + 8u * 16;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
-  volatile int* soft_ok = reinterpret_cast<volatile int*>(misc + 8);     // [2]: outcome of a bounded wait, told to all rows
   int32_t* s_ncache = reinterpret_cast<int32_t*>(misc + 16);              // [T5_ROWS]
   float* s_red = reinterpret_cast<float*>(misc + 16 + T5_ROWS * 4);       // [2][2][T5_ROWS] row maxima of the halves, [2][T5_ROWS] their sums
   uint32_t* s_mask = reinterpret_cast<uint32_t*>(misc + 16 + T5_ROWS * 4 + 6 * T5_ROWS * 4);   // [T5_ROWS][MW]
@@ -199,7 +198,7 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
       mbar_init(bar(K_EMPTY + s), 1); mbar_init(bar(V_EMPTY + s), 1);
       mbar_init(bar(S_FULL + s), 1); mbar_init(bar(S_EMPTY + s), T5_SOFT / 32);
     }
-    mbar_init(bar(P_FULL), T5_SOFT / 32); mbar_init(bar(P_EMPTY), 1);
+    mbar_init(bar(P_FULL), T5_SOFT / 32); mbar_init(bar(P_EMPTY), 1); mbar_init(bar(X_FULL), T5_SOFT / 32);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -341,14 +340,20 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
       const float scale2 = rsqrtf((float)T5_HD) * 1.4426950408889634f;   // 1/sqrt(hd) * log2(e)
       float m_run = -INFINITY, l_run = 0.f;       // l_run: this thread's half of the row's sum
       bool ok = true;
-      uint32_t vote = 0;
-      // one thread does each bounded wait and tells the others, so that all of them take the same branch
+      // Every thread waits on the barrier itself (bounded) and the warp takes one decision, so that the warp-wide
+      // tensor-memory instructions stay converged.  A warp that gives up stops arriving on the barriers the others wait
+      // for; they give up in turn (the abort flag is checked in every bounded wait).
       auto wait_all = [&](uint32_t b, uint32_t parity) {
-        volatile int* slot = soft_ok + (vote & 1u);
-        ++vote;
-        if (st == 0) *slot = mbar_wait(b, parity, abort_flag, p.status) ? 1 : 0;
-        soft_bar_sync();
-        return *slot != 0;
+        return __all_sync(0xffffffffu, mbar_wait(b, parity, abort_flag, p.status)) != 0;
+      };
+      // exchange between the two threads of a row: every warp arrives once it has written, then waits for all eight
+      uint32_t x_phase = 0;
+      auto exchange = [&]() {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(X_FULL));
+        const bool r = wait_all(bar(X_FULL), x_phase);
+        x_phase ^= 1u;
+        return r;
       };
       // may row t attend key `key`?  (selection, never arithmetic: masked scores may be anything)
       auto visible = [&](int key) {
@@ -392,15 +397,15 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         }
         // the softmax runs in base 2: 1/sqrt(hd) * log2(e) is folded into one multiply-add per score
         float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale2;   // scale2 > 0
-        // the row's maximum over both halves; the same barrier tells that the previous chunk's P V has read P (which also
-        // means O is up to date), so P may be written after it
+        // the row's maximum over both halves; P may be written once the previous chunk's P V has read it (which also
+        // means O is up to date)
         s_red[(c & 1) * 2 * T5_ROWS + hf * T5_ROWS + t] = mx;
+        ok = exchange();
+        if (!ok) break;
         if (c > 0) {
           ok = wait_all(bar(P_EMPTY), (uint32_t)((c - 1) & 1));
           if (!ok) break;
           tc_fence_after();
-        } else {
-          soft_bar_sync();
         }
         mx = fmaxf(mx, s_red[(c & 1) * 2 * T5_ROWS + (hf ^ 1) * T5_ROWS + t]);
         const float m_new = fmaxf(m_run, mx);
@@ -441,8 +446,9 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
       // ---- output: O / l, each thread its 64 dimensions
       if (ok) {
         s_red[4 * T5_ROWS + hf * T5_ROWS + t] = l_run;
-        ok = wait_all(bar(P_EMPTY), (uint32_t)((n_chunks - 1) & 1));
+        ok = exchange();
       }
+      if (ok) ok = wait_all(bar(P_EMPTY), (uint32_t)((n_chunks - 1) & 1));
       if (ok) {
         tc_fence_after();
         const float l_row = l_run + s_red[4 * T5_ROWS + (hf ^ 1) * T5_ROWS + t];
