@@ -30,7 +30,8 @@ constexpr int T5_ROWS = 128;      // query rows per CTA (one TMEM lane each)
 constexpr int T5_KEYS = 128;      // keys per chunk
 constexpr int T5_HD = 128;
 constexpr int T5_STAGES = 2;      // K and V chunks in flight
-constexpr int T5_SOFT = 256;       // softmax threads: two per query row
+constexpr int T5_PARTS = 4;        // softmax threads per query row (each a part of the chunk's keys and of the head dimensions)
+constexpr int T5_SOFT = 128 * T5_PARTS;
 constexpr int T5_THREADS = 64 + T5_SOFT;
 constexpr uint32_t T5_BLOCK = 128 * 128;            // bytes of one 64-column block of 128 rows (128 B per row)
 constexpr uint32_t T5_TILE = 2 * T5_BLOCK;          // Q tile, K chunk, V chunk, P tile: 32 KB each
@@ -137,7 +138,7 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* r) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void soft_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ void soft_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(T5_SOFT) : "memory"); }
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -176,7 +177,7 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
   int32_t* s_ncache = reinterpret_cast<int32_t*>(misc + 16);              // [T5_ROWS]
   float* s_red = reinterpret_cast<float*>(misc + 16 + T5_ROWS * 4);       // [2][2][T5_ROWS] row maxima of the halves, [2][T5_ROWS] their sums
-  uint32_t* s_mask = reinterpret_cast<uint32_t*>(misc + 16 + T5_ROWS * 4 + 6 * T5_ROWS * 4);   // [T5_ROWS][MW]
+  uint32_t* s_mask = reinterpret_cast<uint32_t*>(misc + 16 + T5_ROWS * 4 + 3 * T5_PARTS * T5_ROWS * 4);   // [T5_ROWS][MW]
 
   // Tensor memory first (512 columns: two score buffers and the output), before the dependents may start.
   if (warp == 1) {
@@ -300,7 +301,7 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
     // Two threads per query row (= TMEM lane): a warp may only touch the lane quarter (warp id mod 4), so warps w and
     // w + 4 share a quarter; the first takes keys 0..63 of a chunk and output dimensions 0..63, the second the rest.
     const int q4 = warp & 3;                      // TMEM lane quarter this warp may access
-    const int hf = (warp - 2) >> 2;               // which half of the chunk's keys / of the head dimensions
+    const int hf = (warp - 2) >> 2;               // which part of the chunk's keys / of the head dimensions
     const int t = q4 * 32 + lane;                 // row inside the tile
     const int st = threadIdx.x - 64;              // 0..255 (for cooperative loads)
     const uint32_t lane_addr = (uint32_t)(q4 * 32) << 16;
@@ -320,9 +321,10 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
       // pass reads two contiguous 512-byte rows.
       {
         const int cq = lane & 15;
-        const int wrow0 = (warp - 2) * (T5_ROWS / 8);   // sixteen rows per warp
+        constexpr int WROWS = T5_ROWS / (T5_SOFT / 32);   // rows per warp
+        const int wrow0 = (warp - 2) * WROWS;
 #pragma unroll 4
-        for (int i = 0; i < T5_ROWS / 16; ++i) {
+        for (int i = 0; i < WROWS / 2; ++i) {
           const int r = wrow0 + 2 * i + (lane >> 4);
           uint4 v = make_uint4(0u, 0u, 0u, 0u);
           if (r < nrows) {
@@ -364,7 +366,7 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         }
         return vis;
       };
-      constexpr int HALF = T5_KEYS / 2;
+      constexpr int HALF = T5_KEYS / T5_PARTS;   // keys (and output dimensions) of this thread
       for (int c = 0; c < n_chunks; ++c) {
         const int s = c & 1;
         const uint32_t ph = (c >> 1) & 1;
@@ -377,8 +379,8 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         // ---- this thread's 64 scores into registers (one wait for both loads); the score buffer is then free for the
         // chunk after next
         float sc[HALF];
-        tmem_ld32_nowait(s_addr, sc);
-        tmem_ld32_nowait(s_addr + 32, sc + 32);
+#pragma unroll
+        for (int g = 0; g < HALF / 32; ++g) tmem_ld32_nowait(s_addr + g * 32, sc + g * 32);
         tmem_ld_wait();
         tc_fence_before();
         __syncwarp();
@@ -399,7 +401,7 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale2;   // scale2 > 0
         // the row's maximum over both halves; P may be written once the previous chunk's P V has read it (which also
         // means O is up to date)
-        s_red[(c & 1) * 2 * T5_ROWS + hf * T5_ROWS + t] = mx;
+        s_red[((c & 1) * T5_PARTS + hf) * T5_ROWS + t] = mx;
         ok = exchange();
         if (!ok) break;
         if (c > 0) {
@@ -407,7 +409,8 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
           if (!ok) break;
           tc_fence_after();
         }
-        mx = fmaxf(mx, s_red[(c & 1) * 2 * T5_ROWS + (hf ^ 1) * T5_ROWS + t]);
+#pragma unroll
+        for (int q = 0; q < T5_PARTS; ++q) mx = fmaxf(mx, s_red[((c & 1) * T5_PARTS + q) * T5_ROWS + t]);
         const float m_new = fmaxf(m_run, mx);
         const float corr = (m_new == -INFINITY) ? 1.f : fast_exp2(m_run - m_new);
         const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
@@ -420,15 +423,16 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         for (int cc = 0; cc < HALF / 8; ++cc) {
           const uint4 v = make_uint4(pack_bf16(sc[cc * 8], sc[cc * 8 + 1]), pack_bf16(sc[cc * 8 + 2], sc[cc * 8 + 3]),
                                      pack_bf16(sc[cc * 8 + 4], sc[cc * 8 + 5]), pack_bf16(sc[cc * 8 + 6], sc[cc * 8 + 7]));
-          *reinterpret_cast<uint4*>(gen + (sP - base) + (size_t)hf * T5_BLOCK + t * 128 + ((cc ^ (t & 7)) << 4)) = v;
+          const int kc = hf * (HALF / 8) + cc;   // 16-byte chunk (8 keys) of the row: block kc >> 3, chunk kc & 7
+          *reinterpret_cast<uint4*>(gen + (sP - base) + (size_t)(kc >> 3) * T5_BLOCK + t * 128 + (((kc & 7) ^ (t & 7)) << 4)) = v;
         }
         l_run = l_run * corr + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
         m_run = m_new;
         // ---- O *= corr (this thread's 64 dimensions, in tensor memory), unless no row of this warp changed its maximum
         if (c > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
-          const uint32_t o_addr = tmem + lane_addr + 2u * T5_KEYS + (uint32_t)hf * (T5_HD / 2);
+          const uint32_t o_addr = tmem + lane_addr + 2u * T5_KEYS + (uint32_t)hf * (T5_HD / T5_PARTS);
 #pragma unroll 1
-          for (int g = 0; g < T5_HD / 64; ++g) {
+          for (int g = 0; g < T5_HD / T5_PARTS / 32; ++g) {
             float ov[32];
             tmem_ld32_nowait(o_addr + g * 32, ov);
             tmem_ld_wait();
@@ -445,18 +449,20 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
       }
       // ---- output: O / l, each thread its 64 dimensions
       if (ok) {
-        s_red[4 * T5_ROWS + hf * T5_ROWS + t] = l_run;
+        s_red[(2 * T5_PARTS + hf) * T5_ROWS + t] = l_run;
         ok = exchange();
       }
       if (ok) ok = wait_all(bar(P_EMPTY), (uint32_t)((n_chunks - 1) & 1));
       if (ok) {
         tc_fence_after();
-        const float l_row = l_run + s_red[4 * T5_ROWS + (hf ^ 1) * T5_ROWS + t];
+        float l_row = 0.f;
+#pragma unroll
+        for (int q = 0; q < T5_PARTS; ++q) l_row += s_red[(2 * T5_PARTS + q) * T5_ROWS + t];
         const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
-        const uint32_t o_addr = tmem + lane_addr + 2u * T5_KEYS + (uint32_t)hf * (T5_HD / 2);
-        __nv_bfloat16* o = p.out + (size_t)(row0 + (valid ? t : 0)) * dm.d + h * T5_HD + hf * (T5_HD / 2);
+        const uint32_t o_addr = tmem + lane_addr + 2u * T5_KEYS + (uint32_t)hf * (T5_HD / T5_PARTS);
+        __nv_bfloat16* o = p.out + (size_t)(row0 + (valid ? t : 0)) * dm.d + h * T5_HD + hf * (T5_HD / T5_PARTS);
 #pragma unroll 1
-        for (int g = 0; g < T5_HD / 64; ++g) {
+        for (int g = 0; g < T5_HD / T5_PARTS / 32; ++g) {
           float ov[32];
           tmem_ld32_nowait(o_addr + g * 32, ov);
           tmem_ld_wait();
@@ -486,7 +492,7 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
 }
 
 size_t t5_smem_bytes(int MW) {
-  return 1024 + (size_t)(1 + 2 * T5_STAGES + 1) * T5_TILE + 8 * 16 + 16 + T5_ROWS * 4 + 6 * T5_ROWS * 4 + (size_t)T5_ROWS * MW * 4 + 64;
+  return 1024 + (size_t)(1 + 2 * T5_STAGES + 1) * T5_TILE + 8 * 16 + 16 + T5_ROWS * 4 + 3 * T5_PARTS * T5_ROWS * 4 + (size_t)T5_ROWS * MW * 4 + 64;
 }
 
 }  // namespace
