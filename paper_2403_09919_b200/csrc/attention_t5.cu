@@ -6,11 +6,14 @@
 //               rows the rotary kernel wrote), B = K chunk (128 keys x 128 dims, K-major, straight from the cache by
 //               TMA), D = S in tensor memory (two buffers, so the next chunk's scores are computed during this
 //               chunk's softmax);
-//   softmax     two threads per query row (= TMEM lane), half of the chunk's keys each: scale, mask, running maximum
-//               and sum in registers (base 2), P written to shared memory as bf16 in the K-major swizzled layout, O in
-//               tensor memory rescaled in place when a row's maximum moved;
-//   O += P V    tcgen05.mma, A = P, B = V chunk as it lies in the cache ([key][dim], i.e. MN-major for this product:
-//               leading byte offset = one 64-dim box of the chunk, stride byte offset = 8 keys, 2048 bytes per 16 keys).
+//   softmax     four threads per query row (= TMEM lane), a quarter of the chunk's keys each: scale, mask, running
+//               maximum and sum in registers (base 2), P written back to tensor memory as packed bf16 (two buffers, so
+//               a chunk's probabilities are formed while the previous chunk's P V runs), O in tensor memory rescaled in
+//               place when a row's maximum moved;
+//   O += P V    tcgen05.mma with A = P read from tensor memory (8 packed columns per 16 keys), B = V chunk as it lies
+//               in the cache ([key][dim], i.e. MN-major for this product: leading byte offset = one 64-dim box of the
+//               chunk, stride byte offset = 8 keys, 2048 bytes per 16 keys).
+// Tensor memory: columns 0..255 the two score buffers, 256..383 O, 384..511 the two P buffers.
 // Roles: warp 0 lane 0 = TMA producer (K and V rings of two chunks), warp 1 lane 0 = MMA issuer (warp 1 owns the tensor
 // memory), warps 2..9 = softmax and output.  Every wait is bounded (one second): on expiry the CTA raises
 // DEV_ERR_TIMEOUT, lets its copies land, frees its tensor memory and leaves.
@@ -102,6 +105,15 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint6
       "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
       : "memory");
 }
+// A operand read from tensor memory (lane = row, packed bf16 pairs along the columns).
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -137,6 +149,13 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* r) {
       "r"(__float_as_uint(r[28])), "r"(__float_as_uint(r[29])), "r"(__float_as_uint(r[30])), "r"(__float_as_uint(r[31]))
       : "memory");
 }
+__device__ __forceinline__ void tmem_st16_u32(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+      "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void soft_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(T5_SOFT) : "memory"); }
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -168,11 +187,11 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - raw);                 // generic pointer to the same place
-  const uint32_t sQ = base, sK = sQ + T5_TILE, sV = sK + T5_STAGES * T5_TILE, sP = sV + T5_STAGES * T5_TILE;
-  const uint32_t bar0 = sP + T5_TILE;
-  enum { Q_FULL = 0, K_FULL = 1, V_FULL = 3, K_EMPTY = 5, V_EMPTY = 7, S_FULL = 9, S_EMPTY = 11, P_FULL = 13, P_EMPTY = 14, X_FULL = 15, N_BARS = 16 };
+  const uint32_t sQ = base, sK = sQ + T5_TILE, sV = sK + T5_STAGES * T5_TILE;
+  const uint32_t bar0 = sV + T5_STAGES * T5_TILE;
+  enum { Q_FULL = 0, K_FULL = 1, V_FULL = 3, K_EMPTY = 5, V_EMPTY = 7, S_FULL = 9, S_EMPTY = 11, P_FULL = 13, P_EMPTY = 15, X_FULL = 17, N_BARS = 18 };
   auto bar = [&](int i) { return bar0 + 8u * i; };
-  uint8_t* misc = gen + (bar0 - base) + 8u * 16;
+  uint8_t* misc = gen + (bar0 - base) + 8u * 32;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
   int32_t* s_ncache = reinterpret_cast<int32_t*>(misc + 16);              // [T5_ROWS]
@@ -199,7 +218,8 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
       mbar_init(bar(K_EMPTY + s), 1); mbar_init(bar(V_EMPTY + s), 1);
       mbar_init(bar(S_FULL + s), 1); mbar_init(bar(S_EMPTY + s), T5_SOFT / 32);
     }
-    mbar_init(bar(P_FULL), T5_SOFT / 32); mbar_init(bar(P_EMPTY), 1); mbar_init(bar(X_FULL), T5_SOFT / 32);
+    for (int s = 0; s < 2; ++s) { mbar_init(bar(P_FULL + s), T5_SOFT / 32); mbar_init(bar(P_EMPTY + s), 1); }
+    mbar_init(bar(X_FULL), T5_SOFT / 32);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -283,17 +303,17 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         if (c + 1 < n_chunks) {
           if (!issue_qk(c + 1)) { ok = false; break; }
         }
-        if (!mbar_wait(bar(P_FULL), (uint32_t)(c & 1), abort_flag, p.status)) { ok = false; break; }
+        if (!mbar_wait(bar(P_FULL + (c & 1)), ph, abort_flag, p.status)) { ok = false; break; }
         if (!mbar_wait(bar(V_FULL + s), ph, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < T5_KEYS / 16; ++kk) {
-          const uint32_t aoff = (uint32_t)(kk >> 2) * T5_BLOCK + (uint32_t)(kk & 3) * 32u;   // P: 16 keys further along K
-          umma_bf16(tmem + 2u * T5_KEYS, desc_kmajor(sP + aoff), desc_mnmajor(sV + s * T5_TILE + (uint32_t)kk * 2048u), idesc_pv,
-                    (c > 0 || kk > 0) ? 1u : 0u);
+          // P from tensor memory: buffer c & 1, 16 keys = 8 packed columns further per step
+          umma_bf16_ts(tmem + 2u * T5_KEYS, tmem + 3u * T5_KEYS + (uint32_t)(c & 1) * (T5_KEYS / 2) + (uint32_t)kk * 8u,
+                       desc_mnmajor(sV + s * T5_TILE + (uint32_t)kk * 2048u), idesc_pv, (c > 0 || kk > 0) ? 1u : 0u);
         }
         umma_commit(bar(V_EMPTY + s));
-        umma_commit(bar(P_EMPTY));   // P may be overwritten and O is up to date
+        umma_commit(bar(P_EMPTY + (c & 1)));   // this P buffer may be overwritten and O is up to date through chunk c
       }
     }
   } else {
@@ -399,13 +419,13 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         }
         // the softmax runs in base 2: 1/sqrt(hd) * log2(e) is folded into one multiply-add per score
         float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale2;   // scale2 > 0
-        // the row's maximum over both halves; P may be written once the previous chunk's P V has read it (which also
-        // means O is up to date)
+        // the row's maximum over all parts
         s_red[((c & 1) * T5_PARTS + hf) * T5_ROWS + t] = mx;
         ok = exchange();
         if (!ok) break;
-        if (c > 0) {
-          ok = wait_all(bar(P_EMPTY), (uint32_t)((c - 1) & 1));
+        // this chunk's P buffer is free once the P V of the chunk before last has read it
+        if (c >= 2) {
+          ok = wait_all(bar(P_EMPTY + (c & 1)), ph ^ 1u);
           if (!ok) break;
           tc_fence_after();
         }
@@ -414,22 +434,25 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         const float m_new = fmaxf(m_run, mx);
         const float corr = (m_new == -INFINITY) ? 1.f : fast_exp2(m_run - m_new);
         const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-        // ---- probabilities -> shared memory (bf16, K-major swizzled: 16-byte chunk cc of row t lands at chunk
-        // cc ^ (t & 7) of its 128-byte line; this thread's 64 keys are block hf of the tile), row sum
+        // ---- probabilities -> tensor memory (packed bf16: key pair (2j, 2j + 1) of this thread's keys in column j of its
+        // part of buffer c & 1), row sum
         float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int j = 0; j < HALF; ++j) { sc[j] = fast_exp2(fmaf(sc[j], scale2, -m_use)); sum4[j & 3] += sc[j]; }   // 2^(-inf) = 0
+        {
+          uint32_t pk[HALF / 2];
 #pragma unroll
-        for (int cc = 0; cc < HALF / 8; ++cc) {
-          const uint4 v = make_uint4(pack_bf16(sc[cc * 8], sc[cc * 8 + 1]), pack_bf16(sc[cc * 8 + 2], sc[cc * 8 + 3]),
-                                     pack_bf16(sc[cc * 8 + 4], sc[cc * 8 + 5]), pack_bf16(sc[cc * 8 + 6], sc[cc * 8 + 7]));
-          const int kc = hf * (HALF / 8) + cc;   // 16-byte chunk (8 keys) of the row: block kc >> 3, chunk kc & 7
-          *reinterpret_cast<uint4*>(gen + (sP - base) + (size_t)(kc >> 3) * T5_BLOCK + t * 128 + (((kc & 7) ^ (t & 7)) << 4)) = v;
+          for (int j = 0; j < HALF / 2; ++j) pk[j] = pack_bf16(sc[2 * j], sc[2 * j + 1]);
+          tmem_st16_u32(tmem + lane_addr + 3u * T5_KEYS + (uint32_t)(c & 1) * (T5_KEYS / 2) + (uint32_t)hf * (HALF / 2), pk);
         }
         l_run = l_run * corr + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
         m_run = m_new;
-        // ---- O *= corr (this thread's 64 dimensions, in tensor memory), unless no row of this warp changed its maximum
+        // ---- O *= corr (this thread's dimensions, in tensor memory), unless no row of this warp changed its maximum; O has
+        // to be complete through the previous chunk first
         if (c > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
+          ok = wait_all(bar(P_EMPTY + ((c - 1) & 1)), (uint32_t)(((c - 1) >> 1) & 1));
+          if (!ok) break;
+          tc_fence_after();
           const uint32_t o_addr = tmem + lane_addr + 2u * T5_KEYS + (uint32_t)hf * (T5_HD / T5_PARTS);
 #pragma unroll 1
           for (int g = 0; g < T5_HD / T5_PARTS / 32; ++g) {
@@ -440,19 +463,18 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
             for (int j = 0; j < 32; ++j) ov[j] *= corr;
             tmem_st32(o_addr + g * 32, ov);
           }
-          tmem_st_wait();
         }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P was written with ordinary stores
+        tmem_st_wait();   // P (and O) are in tensor memory
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(bar(P_FULL));
+        if (lane == 0) mbar_arrive(bar(P_FULL + (c & 1)));
       }
       // ---- output: O / l, each thread its 64 dimensions
       if (ok) {
         s_red[(2 * T5_PARTS + hf) * T5_ROWS + t] = l_run;
         ok = exchange();
       }
-      if (ok) ok = wait_all(bar(P_EMPTY), (uint32_t)((n_chunks - 1) & 1));
+      if (ok) ok = wait_all(bar(P_EMPTY + ((n_chunks - 1) & 1)), (uint32_t)(((n_chunks - 1) >> 1) & 1));
       if (ok) {
         tc_fence_after();
         float l_row = 0.f;
@@ -492,7 +514,7 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
 }
 
 size_t t5_smem_bytes(int MW) {
-  return 1024 + (size_t)(1 + 2 * T5_STAGES + 1) * T5_TILE + 8 * 16 + 16 + T5_ROWS * 4 + 3 * T5_PARTS * T5_ROWS * 4 + (size_t)T5_ROWS * MW * 4 + 64;
+  return 1024 + (size_t)(1 + 2 * T5_STAGES) * T5_TILE + 8 * 32 + 16 + T5_ROWS * 4 + 3 * T5_PARTS * T5_ROWS * 4 + (size_t)T5_ROWS * MW * 4 + 64;
 }
 
 }  // namespace
