@@ -32,10 +32,26 @@ architecture, KV cache handling, tie breaking).  The readings used here:
     length j+1 is shared when all of its j+1 positions match, and the FIRST such
     candidate is reported.
 
+  * Acceptance at temperature > 0 (Section 3.4 names rejection sampling and gives no
+    procedure).  Beam search proposes tokens deterministically, so the proposal at a
+    tree node is a point mass per child.  For such a proposal the accept/resample
+    rule of speculative sampling -- keep the proposed token x with probability
+    min(1, p(x)/q(x)) = p(x), otherwise draw from the residual, which is p with x
+    removed, child after child -- has the same law as: draw y ~ p at the node and
+    descend iff y is one of its children.  The draw is made with the Gumbel-max rule
+    y = argmax_v (logit_v / T + G_v), G_v = -ln(-ln u_v), with u_v from the
+    counter-based generator Philox-4x32-10 keyed by (seed; sequence, position of the
+    token being chosen, v), so the token chosen for a position does not depend on the
+    branch or the step that reaches it: speculative decoding reproduces plain sampled
+    decoding token for token.
+
 Parity pins (tests/test_oracle_*.py): the printed dedup example, brute-force
 prefix sets, packed-tree == per-beam causal verification, speculative == plain
 greedy decoding, beam width 1 == greedy drafting, exhaustive beam search on a tiny
-vocabulary, closed forms for the RNN cell and the head, library cross-checks.
+vocabulary, closed forms for the RNN cell and the head, library cross-checks; for
+sampling: the generator's published known answers, sample frequencies against the
+softmax, the accept/resample rule worked out exactly on small cases, speculative ==
+plain sampled decoding.
 Parity unpinned: nothing in the paper prints a weights-to-beams example, so the
 drafter's exact beams are pinned by properties only.
 """
@@ -102,6 +118,66 @@ def top_k_ordered(values, k):
 
 
 # ----------------------------------------------------------------------------
+# token choice at temperature > 0 (Section 3.4: "rejection sampling")
+# ----------------------------------------------------------------------------
+PHILOX_M0, PHILOX_M1 = 0xD2511F53, 0xCD9E8D57
+PHILOX_W0, PHILOX_W1 = 0x9E3779B9, 0xBB67AE85
+
+
+def philox4x32(counter, key, rounds=10):
+    """Philox-4x32 (Salmon et al., SC'11): four 32-bit counter words, two key words.
+
+    counter: four integers or equally shaped integer arrays; key: two integers.
+    Returns four uint64 arrays holding 32-bit values.
+    """
+    c = [np.asarray(x, dtype=np.uint64) & np.uint64(0xFFFFFFFF) for x in counter]
+    c = list(np.broadcast_arrays(*c))
+    k0, k1 = int(key[0]) & 0xFFFFFFFF, int(key[1]) & 0xFFFFFFFF
+    lo32, sh = np.uint64(0xFFFFFFFF), np.uint64(32)
+    for _ in range(rounds):
+        p0 = np.uint64(PHILOX_M0) * c[0]        # 32 x 32 -> 64 bits, exact in uint64
+        p1 = np.uint64(PHILOX_M1) * c[2]
+        c = [(p1 >> sh) ^ c[1] ^ np.uint64(k0), p1 & lo32, (p0 >> sh) ^ c[3] ^ np.uint64(k1), p0 & lo32]
+        k0 = (k0 + PHILOX_W0) & 0xFFFFFFFF
+        k1 = (k1 + PHILOX_W1) & 0xFFFFFFFF
+    return c
+
+
+def uniform_open(x32):
+    """32 random bits -> u in (0, 1): the top 23 bits plus one half, over 2^23 (exact in fp32 and fp64)."""
+    return ((np.asarray(x32, dtype=np.uint64) >> np.uint64(9)).astype(np.float64) + 0.5) / float(1 << 23)
+
+
+def gumbel_noise(seed, seq, pos, vocab):
+    """G_v = -ln(-ln u_v), v < vocab, for the token at position `pos` of sequence `seq`.
+
+    Vocabulary entries 4k .. 4k+3 are the four output words of the counter (k, pos, seq, 0)
+    under the key (seed mod 2^32, seed >> 32).
+    """
+    blocks = np.arange((vocab + 3) // 4, dtype=np.uint64)
+    words = philox4x32((blocks, pos, seq, 0), (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF))
+    u = uniform_open(np.stack(words, axis=1).reshape(-1)[:vocab])
+    return -np.log(-np.log(u))
+
+
+def choose_token(logits, sampling=None, seq=0, pos=0, want_scores=False):
+    """The LLM's token for position `pos` given its logits there.
+
+    sampling None (or temperature 0): the greedy token.  Otherwise sampling =
+    dict(temperature=T, seed=s): a draw from softmax(logits / T) by the Gumbel-max rule.
+    """
+    z = np.asarray(logits, dtype=F)
+    if sampling is not None and sampling["temperature"] > 0:
+        z = z / sampling["temperature"] + gumbel_noise(sampling["seed"], seq, pos, z.shape[0])
+    return (argmax_first(z), z) if want_scores else argmax_first(z)
+
+
+def choose_rows(logits, pos, sampling=None, seq=0):
+    """choose_token for every row; row r's logits choose the token at position pos[r] + 1."""
+    return np.array([choose_token(logits[r], sampling, seq, int(pos[r]) + 1) for r in range(logits.shape[0])], dtype=np.int64)
+
+
+# ----------------------------------------------------------------------------
 # target LLM (verification forward, Section 3.4)
 # ----------------------------------------------------------------------------
 class KVCache:
@@ -159,19 +235,19 @@ def llm_forward(W, cfg, tokens, pos, mask, kv, ctx, dtype=F, want_logits=True):
     return hidden, logits
 
 
-def prefill(W, cfg, prompt, kv, dtype=F):
+def prefill(W, cfg, prompt, kv, dtype=F, sampling=None, seq=0):
     """Causal forward over the prompt.  Returns (ctx, root token g, h)."""
     P = len(prompt)
     mask = np.tril(np.ones((P, P), dtype=bool))
     hidden, _ = llm_forward(W, cfg, prompt, np.arange(P), mask, kv, 0, dtype, want_logits=False)
     logits_last = hidden[P - 1] @ _c(W["lm_head"], dtype).T
-    return P, argmax_first(logits_last), hidden[P - 1].copy()
+    return P, choose_token(logits_last, sampling, seq, P), hidden[P - 1].copy()
 
 
-def ar_step(W, cfg, kv, ctx, g, dtype=F):
+def ar_step(W, cfg, kv, ctx, g, dtype=F, sampling=None, seq=0):
     """One plain autoregressive step: feed g at position ctx, return next token, h, logits."""
     hidden, logits = llm_forward(W, cfg, [g], [ctx], np.ones((1, 1), bool), kv, ctx, dtype)
-    return argmax_first(logits[0]), hidden[0].copy(), logits[0]
+    return choose_token(logits[0], sampling, seq, ctx + 1), hidden[0].copy(), logits[0]
 
 
 # ----------------------------------------------------------------------------
@@ -326,13 +402,13 @@ def flat_beam(beam_aug, ctx):
 
 
 # ----------------------------------------------------------------------------
-# greedy acceptance + KV compaction (Section 3.4)
+# acceptance + KV compaction (Section 3.4)
 # ----------------------------------------------------------------------------
 def accept_greedy(beams, unpack, llm_argmax):
-    """Longest prefix of a candidate whose tokens equal the LLM's greedy tokens.
+    """Longest prefix of a candidate whose tokens equal the LLM's own tokens.
 
     beams [BW, L]; unpack [BW, L+1] (column 0 = root); llm_argmax[N] = the LLM's
-    greedy next token after each packed node.  Returns (a, best, emitted) where
+    next token after each packed node (greedy, or drawn: see choose_token).  Returns (a, best, emitted) where
     emitted = accepted draft tokens followed by the bonus token.
     """
     beams = np.asarray(beams)
@@ -364,7 +440,7 @@ def compact_kv(kv, ctx, unpack, best, a):
 # the whole step (Section 3.4) for one sequence
 # ----------------------------------------------------------------------------
 def spec_step(W, D, cfg, kv, ctx, g, h, beam_width, beam_length, planted=None,
-              tree=True, dtype=F, run_drafter=True):
+              tree=True, dtype=F, run_drafter=True, sampling=None, seq=0):
     """One speculative decode step.  Returns a dict with every intermediate.
 
     planted: optional [BW, L] beams used in place of the drafter's (the drafter
@@ -379,7 +455,7 @@ def spec_step(W, D, cfg, kv, ctx, g, h, beam_width, beam_length, planted=None,
     beam_aug = np.concatenate([np.full((beams.shape[0], 1), g, dtype=np.int64), beams], axis=1)
     packed = pack_beam(beam_aug, ctx) if tree else flat_beam(beam_aug, ctx)
     hidden, logits = llm_forward(W, cfg, packed["tokens"], packed["pos"], packed["mask"], kv, ctx, dtype)
-    am = np.argmax(logits, axis=1)
+    am = choose_rows(logits, packed["pos"], sampling, seq)
     a, best, emitted = accept_greedy(beams, packed["unpack"], am)
     node = int(packed["unpack"][best, a])
     new_ctx = compact_kv(kv, ctx, packed["unpack"], best, a)
@@ -389,13 +465,13 @@ def spec_step(W, D, cfg, kv, ctx, g, h, beam_width, beam_length, planted=None,
     return out
 
 
-def generate_ar(W, cfg, prompt, n_tokens, max_ctx, dtype=F):
-    """Plain greedy decoding: the definition the speculative path must reproduce."""
+def generate_ar(W, cfg, prompt, n_tokens, max_ctx, dtype=F, sampling=None, seq=0):
+    """Plain decoding (greedy, or sampled): the definition the speculative path must reproduce."""
     kv = KVCache(cfg["n_layers"], max_ctx, cfg["n_heads"], cfg["d_model"] // cfg["n_heads"], dtype)
-    ctx, g, h = prefill(W, cfg, prompt, kv, dtype)
+    ctx, g, h = prefill(W, cfg, prompt, kv, dtype, sampling, seq)
     out = [g]
     while len(out) < n_tokens:
-        nxt, h, _ = ar_step(W, cfg, kv, ctx, g, dtype)
+        nxt, h, _ = ar_step(W, cfg, kv, ctx, g, dtype, sampling, seq)
         ctx += 1
         g = nxt
         out.append(g)
@@ -403,16 +479,16 @@ def generate_ar(W, cfg, prompt, n_tokens, max_ctx, dtype=F):
 
 
 def generate_spec(W, D, cfg, prompt, n_steps, beam_width, beam_length, max_ctx,
-                  planted_fn=None, tree=True, dtype=F):
+                  planted_fn=None, tree=True, dtype=F, sampling=None, seq=0):
     """Speculative decoding for n_steps.  planted_fn(step, ctx, g) -> beams or None."""
     kv = KVCache(cfg["n_layers"], max_ctx, cfg["n_heads"], cfg["d_model"] // cfg["n_heads"], dtype)
-    ctx, g, h = prefill(W, cfg, prompt, kv, dtype)
+    ctx, g, h = prefill(W, cfg, prompt, kv, dtype, sampling, seq)
     out = [g]
     accepted = []
     for step in range(n_steps):
         planted = planted_fn(step, len(out), g) if planted_fn is not None else None
         r = spec_step(W, D, cfg, kv, ctx, g, h, beam_width, beam_length, planted, tree, dtype,
-                      run_drafter=planted is None)
+                      run_drafter=planted is None, sampling=sampling, seq=seq)
         ctx, g, h = r["ctx"], r["g"], r["h"]
         out.extend(r["emitted"])
         accepted.append(r["n_accept"])
