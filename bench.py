@@ -110,8 +110,9 @@ class OracleSample:
     layers, fp32 numpy arithmetic.  One step is timed in parts and scaled to the full depth:
     t_step = t_draft + t_pack + (n_layers / sample_layers) * t_layers + t_lm_head + t_accept."""
 
-    def __init__(self, cfg, sample_layers=2):
+    def __init__(self, cfg, sample_layers=2, sampling=None):
         self.cfg = cfg
+        self.sampling = sampling
         self.sample_layers = min(sample_layers, cfg["n_layers"])
         self.c = synth.with_layers(cfg, self.sample_layers)
         w = synth.make_weights(self.c, "cpu")
@@ -139,7 +140,7 @@ class OracleSample:
         hidden, _ = ora.llm_forward(W, c, p["tokens"], p["pos"], p["mask"], kv, ctx, dt, want_logits=False)
         t3 = time.perf_counter()
         logits = hidden @ W["lm_head"].T
-        am = logits.argmax(1)
+        am = ora.choose_rows(logits, p["pos"], self.sampling)
         t4 = time.perf_counter()
         a, best, emitted = ora.accept_greedy(beams, p["unpack"], am)
         ora.compact_kv(kv, ctx, p["unpack"], best, a)
@@ -161,6 +162,10 @@ class OracleSample:
         return dict(value=tot_tok / tot_s, ms_per_step=1e3 * tot_s / steps, sample=sample)
 
 
+def oracle_sampling(args):
+    return dict(temperature=args.temperature, seed=args.sample_seed) if args.temperature > 0 else None
+
+
 def cpu_cores():
     try:
         return len(os.sched_getaffinity(0))
@@ -174,7 +179,7 @@ def run_reference(args, cfg):
     if rank != 0:
         return
     steps = max(1, min(args.steps, args.reference_max_steps))
-    r = OracleSample(cfg, args.oracle_layers).run(steps, warmup=min(args.warmup, 1))
+    r = OracleSample(cfg, args.oracle_layers, oracle_sampling(args)).run(steps, warmup=min(args.warmup, 1))
     value, sample = r["value"], r["sample"]
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
             "warmup": min(args.warmup, 1), "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "weak",
@@ -188,7 +193,9 @@ def run_reference(args, cfg):
 def workload_config(args, cfg):
     return {"workload": f"{args.workload}: {cfg['n_layers']} layers d={cfg['d_model']} heads={cfg['n_heads']} ffn={cfg['d_ffn']} "
                         f"vocab={cfg['vocab']} {cfg['dtype']}, batch {cfg['max_batch']}, prompt {cfg['prompt_len']} uniform-random "
-                        f"tokens, beam width {cfg['beam_width']}, beam length {cfg['beam_length']}, greedy acceptance, random-init weights",
+                        f"tokens, beam width {cfg['beam_width']}, beam length {cfg['beam_length']}, "
+                        + (f"acceptance against the LLM's own draws at temperature {args.temperature}" if args.temperature > 0
+                           else "greedy acceptance") + ", random-init weights",
             "beams": "drafter's own (random-init drafter and LLM are uncorrelated: about 1 token per step by construction)",
             "l2": "inputs larger than L2: every step streams all weights (>= 13 GB at 7B) so nothing is reused from the 126 MB L2",
             "parallelism": "replicas only (no collective)"}
@@ -345,6 +352,10 @@ def main():
     ap.add_argument("--sweep-bw", default="1,4,8,16,32")
     ap.add_argument("--sweep-batch", default="1,2,4,8,16")
     ap.add_argument("--sweep-prompt", type=int, default=256)
+    ap.add_argument("--temperature", type=float, default=0.0,
+                    help="> 0: the LLM's tokens are draws (Gumbel-max, counter-based noise) instead of greedy; the paper's "
+                         "headline numbers and this benchmark's default are temperature 0")
+    ap.add_argument("--sample-seed", type=int, default=1)
     ap.add_argument("--prefill", action="store_true", help="prompt-processing timings instead of the benchmark line")
     ap.add_argument("--prefill-batch", default="1,16")
     ap.add_argument("--prefill-len", default="512,2048")
@@ -381,6 +392,8 @@ def main():
                          + need * (L + 1) + 2 + BW * L)
     w = synth.make_weights(cfg, device)
     eng = binding.ReDrafter(cfg, w, device=device)
+    if args.temperature > 0:
+        eng.set_sampling(args.temperature, args.sample_seed)
     prompts = synth.make_prompts(cfg, B, seed=cfg.get("seed", 0) + shard_of_rank(rank)["prompt_seed_offset"])
     out = binding.AcceptOut(B, L, device)
 
@@ -571,7 +584,7 @@ def main():
                                        "teacher-forced root, accepted length read by the host every step (one sync per step)"}
             line["speedup_vs_autoregressive"] = value / world / (n_ar * B / (ms_ar * 1e-3))
         if not args.no_cpu_baseline and world == 1:
-            r = OracleSample(cfg, args.oracle_layers).run(args.cpu_steps, warmup=1)
+            r = OracleSample(cfg, args.oracle_layers, oracle_sampling(args)).run(args.cpu_steps, warmup=1)
             line["cpu_baseline"] = {"value": r["value"], "unit": UNIT, "cores": cpu_cores(), "kind": "oracle",
                                     "ms_per_step": r["ms_per_step"], "sample": r["sample"]}
         print(json.dumps(line))

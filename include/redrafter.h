@@ -154,7 +154,8 @@ RD_API int redrafter_pack(rd_handle* h, const int32_t* beams, void* stream, cons
 
 /* Target-LLM forward over the packed rows against the KV cache and the tree mask (Section 3.4).
  * K/V of row n are written provisionally to cache slot ctx[b] + n.
- * argmax: device [B][NMAX] int32 greedy next token per packed row (lowest id on ties; -1 on padding);
+ * argmax: device [B][NMAX] int32 the LLM's next token per packed row: greedy (lowest id on ties), or drawn
+ *   after redrafter_set_sampling; -1 on padding;
  * hidden: device [B][NMAX][d_model] fp32 output of the final norm, or NULL;
  * logits: device [B][NMAX][vocab] fp32, or NULL.  Padding rows are left untouched in hidden/logits. */
 RD_API int redrafter_verify(rd_handle* h, const rd_packed* packed, void* stream, int32_t* argmax, float* hidden,
@@ -200,6 +201,22 @@ RD_API int redrafter_step(rd_handle* h, const int32_t* planted_beams, void* stre
  * Section 4): feeds g at position ctx, advances ctx by 1, sets the new g and h.
  * token: device [B] int32 (the new g), may be NULL. */
 RD_API int redrafter_ar_step(rd_handle* h, void* stream, int32_t* token);
+
+/* Acceptance at temperature > 0 (Section 3.4 names rejection sampling as the other end of the selection
+ * methods and gives no procedure).  Beam search proposes tokens deterministically, so the proposal at a tree
+ * node is a point mass per child; the accept/resample rule of speculative sampling then has the law of
+ * "draw y from the LLM's distribution p at the node and descend iff y is a child".  After this call every
+ * token the LLM chooses -- the root after the prompt, the per-row tokens of redrafter_verify (its `argmax`
+ * output) and redrafter_step, the token of redrafter_ar_step -- is such a draw from softmax(logits / T),
+ * made by the Gumbel-max rule: argmax_v (logit_v / T - ln(-ln u_v)), lowest id on ties, with
+ * u_v = (top 23 bits of word (v mod 4) of Philox-4x32-10(counter = (v / 4, position, sequence, 0),
+ * key = (seed mod 2^32, seed >> 32)) + 1/2) / 2^23 and `position` the index of the token being chosen in
+ * its sequence (prompt tokens count from 0), `sequence` its batch index.  The draw for a position therefore
+ * does not depend on the branch, the row or the step that reaches it: speculative steps and
+ * redrafter_ar_step generate the same tokens.  Acceptance, compaction and hand-off are unchanged (they
+ * compare tokens).  temperature == 0 restores greedy choice (the default).  Takes effect for calls made
+ * after it; enqueues nothing.  Errors: INVALID_ARG (negative or non-finite temperature). */
+RD_API int redrafter_set_sampling(rd_handle* h, float temperature, uint64_t seed);
 
 /* Copy the decode state out of / into the handle.  Device pointers; any may be NULL.
  * ctx [B] int32 context lengths, root [B] int32 guaranteed tokens, hvec [B][d_model] fp32. */

@@ -26,7 +26,7 @@ EXPORTS = ["redrafter_workspace_bytes", "redrafter_kv_bytes", "redrafter_init", 
            "redrafter_accept", "redrafter_step", "redrafter_ar_step", "redrafter_get_state", "redrafter_set_state",
            "redrafter_set_ctx_bound", "redrafter_poll", "redrafter_launch_count", "redrafter_profile",
            "redrafter_profile_read", "redrafter_trace", "redrafter_trace_read", "redrafter_trace_bytes",
-           "redrafter_accept_static", "redrafter_selftest_wait"]
+           "redrafter_accept_static", "redrafter_selftest_wait", "redrafter_set_sampling"]
 
 
 class RdConfig(C.Structure):
@@ -81,6 +81,7 @@ def lib():
         L.redrafter_get_state.argtypes = [vp, vp, vp, vp, vp]
         L.redrafter_set_state.argtypes = [vp, vp, vp, vp, vp, i32]
         L.redrafter_set_ctx_bound.argtypes = [vp, i32]
+        L.redrafter_set_sampling.argtypes = [vp, C.c_float, C.c_uint64]
         L.redrafter_poll.argtypes = [vp, vp]
         L.redrafter_launch_count.restype = C.c_int64
         L.redrafter_launch_count.argtypes = [vp]
@@ -269,6 +270,10 @@ class ReDrafter:
     def ar_step(self, token=None):
         self._ck(self.L.redrafter_ar_step(self.h, _stream(), _ptr(token)))
         return token
+
+    def set_sampling(self, temperature, seed=0):
+        """temperature > 0: the LLM's tokens are draws keyed by (seed; sequence, position); 0: greedy."""
+        self._ck(self.L.redrafter_set_sampling(self.h, float(temperature), int(seed)))
 
     def get_state(self):
         ctx = torch.empty(self.B, dtype=torch.int32, device=self.device)

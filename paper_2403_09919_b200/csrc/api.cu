@@ -5,6 +5,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <cmath>
 #include <map>
 #include <new>
 #include <unordered_map>
@@ -82,6 +83,7 @@ struct rd_handle {
   bool prefilled;
   int batch;      // active sequences
   int ctx_bound;  // host-side upper bound of every sequence's context length
+  Sampling sampling;  // how the LLM's tokens are chosen (inv_t = 0: greedy)
   int64_t launches;
   // tensor-core path (bf16): TMA descriptors by base pointer, launch geometry
   bool use_tc;
@@ -452,7 +454,7 @@ int do_verify(rd_handle* h, const rd_packed& pk, cudaStream_t st, int32_t* argma
   rc = gemm(h, w.hidden_t, dm.d, h->w.lm_head, dm.V, dm.d, w.m_total, m_max, w.logits, dm.V, &g, nullptr, st, /*pair=*/1);
   if (rc) return rc;
   CKP(h, PROF_MISC, launch_fill_i32(argmax, -1, B * dm.NMAX, st));
-  CKP(h, PROF_MISC, launch_argmax_rows(w.logits, g, dm.V, argmax, w.row_out_index, w.m_total, m_max, st));
+  CKP(h, PROF_MISC, launch_argmax_rows(w.logits, g, dm.V, argmax, w.row_out_index, w.m_total, m_max, h->sampling, w.row_seq, w.row_pos, 1, st));
   if (hidden) CKP(h, PROF_MISC, launch_scatter_rows(w.hidden_f, dm.d, hidden, w.row_out_index, w.m_total, m_max, st));
   if (logits) CK(h, launch_scatter_rows(w.logits, dm.V, logits, w.row_out_index, w.m_total, m_max, st));
   return RD_OK;
@@ -570,6 +572,7 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
     if (!ok) return init_fail(h, RD_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d for operand %p", failed_rc, failed_ptr);
   }
   h->prefilled = false; h->batch = dm.B; h->ctx_bound = 0; h->launches = 0; h->err[0] = 0;
+  h->sampling = Sampling{0.0f, 0u, 0u};
   h->profiling = false;
   h->trace_next = -1;
   h->chain.ctr = h->ws.chain_ctr; h->chain.status = h->ws.status;
@@ -669,8 +672,9 @@ int redrafter_prefill(rd_handle* h, const int32_t* tokens, const int32_t* prompt
   GemmOut g;
   rc = gemm(h, w.h_t, dm.d, h->w.lm_head, dm.V, dm.d, w.one_b, batch, w.logits, dm.V, &g, nullptr, st);
   if (rc) return rc;
-  CK(h, launch_argmax_rows(w.logits, g, dm.V, w.root, nullptr, w.one_b, batch, st));
   CKRT(h, cudaMemcpyAsync(w.ctx, prompt_len, batch * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+  // row b is sequence b's last prompt row: the root is the token at position prompt_len[b]
+  CK(h, launch_argmax_rows(w.logits, g, dm.V, w.root, nullptr, w.one_b, batch, h->sampling, nullptr, w.ctx, 0, st));
   h->prefilled = true;
   h->ctx_bound = longest;
   return RD_OK;
@@ -774,9 +778,18 @@ int redrafter_ar_step(rd_handle* h, void* stream, int32_t* token) {
   GemmOut g;
   rc = gemm(h, w.hidden_t, dm.d, h->w.lm_head, dm.V, dm.d, w.m_total, B, w.logits, dm.V, &g, nullptr, st);
   if (rc) return rc;
-  CK(h, launch_argmax_rows(w.logits, g, dm.V, w.argmax_c, nullptr, w.m_total, B, st));
+  CK(h, launch_argmax_rows(w.logits, g, dm.V, w.argmax_c, nullptr, w.m_total, B, h->sampling, w.row_seq, w.row_pos, 1, st));
   CK(h, launch_ar_finish(w.argmax_c, w.hidden_f, w.ctx, w.root, w.h, token, dm, B, st));
   h->ctx_bound += 1;
+  return RD_OK;
+}
+
+int redrafter_set_sampling(rd_handle* h, float temperature, uint64_t seed) {
+  if (!h) return RD_ERR_INVALID_ARG;
+  if (!(temperature >= 0.0f) || !std::isfinite(temperature)) return fail(h, RD_ERR_INVALID_ARG, "temperature %g", (double)temperature);
+  h->sampling.inv_t = temperature > 0.0f ? 1.0f / temperature : 0.0f;
+  h->sampling.k0 = (uint32_t)(seed & 0xffffffffull);
+  h->sampling.k1 = (uint32_t)(seed >> 32);
   return RD_OK;
 }
 

@@ -758,9 +758,33 @@ cudaError_t launch_swiglu(int dtype, const GemmOut& proj, void* out_t, int F, co
   return cudaGetLastError();
 }
 
-// ---------------------------------------------------------------- row argmax (lowest index on ties)
+// ---------------------------------------------------------------- the LLM's token per row (lowest index on ties)
+// Philox-4x32-10 (Salmon et al., SC'11): counter (c0..c3), key (k0, k1) -> four words.
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t h0 = __umulhi(0xD2511F53u, c0), l0 = 0xD2511F53u * c0;
+    const uint32_t h1 = __umulhi(0xCD9E8D57u, c2), l1 = 0xCD9E8D57u * c2;
+    c0 = h1 ^ c1 ^ k0; c1 = l1;
+    c2 = h0 ^ c3 ^ k1; c3 = l0;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
+// 32 random bits -> standard Gumbel noise: u = (top 23 bits + 1/2) / 2^23 lies in (0, 1) and is exact in fp32.
+__device__ __forceinline__ float gumbel_of(uint32_t x) {
+  const float u = ((float)(x >> 9) + 0.5f) * (1.0f / 8388608.0f);
+  return -logf(-logf(u));
+}
+
+// SAMPLE = false: greedy token.  SAMPLE = true: a draw from softmax(logits / T) by the Gumbel-max rule (Section 3.4's
+// rejection sampling for deterministic proposals: the LLM's own draw at a node, which acceptance compares with the
+// node's children); the noise of vocabulary entry v depends on (seed; sequence, position of the token being chosen, v)
+// only, so every row that predicts the same position of a sequence uses the same noise.
+template <bool SAMPLE>
 __global__ void __launch_bounds__(512) argmax_rows_kernel(float* __restrict__ logits, GemmOut proj, int V, int32_t* __restrict__ out,
-                                   const int32_t* __restrict__ out_index, const int32_t* __restrict__ m_total) {
+                                   const int32_t* __restrict__ out_index, const int32_t* __restrict__ m_total, Sampling smp,
+                                   const int32_t* __restrict__ row_seq, const int32_t* __restrict__ row_pos, int pos_add) {
   pdl_enter();
   __shared__ float sv[32];
   __shared__ int si[32];
@@ -769,6 +793,11 @@ __global__ void __launch_bounds__(512) argmax_rows_kernel(float* __restrict__ lo
   if (m >= M) return;
   float* r = logits + (size_t)m * V;
   const GemmRows m_tiles = gemm_m_tiles(proj, M);
+  uint32_t seq = 0, pos = 0;
+  if (SAMPLE) {
+    seq = row_seq ? (uint32_t)row_seq[m] : (uint32_t)m;
+    pos = (uint32_t)(row_pos[m] + pos_add);
+  }
   float bv = -INFINITY;
   int bi = 0x7fffffff;
   // the complete logits are written back in place (later readers of the buffer see final values); four float4 per
@@ -787,7 +816,14 @@ __global__ void __launch_bounds__(512) argmax_rows_kernel(float* __restrict__ lo
       if (i < V) {
         const float4 q = gemm_finish4(proj, m_tiles, pd[u]);
         *reinterpret_cast<float4*>(r + i) = q;
-        const float e[4] = {q.x, q.y, q.z, q.w};
+        float e[4] = {q.x, q.y, q.z, q.w};
+        if (SAMPLE) {
+          const uint4 x = philox4x32_10((uint32_t)i >> 2, pos, seq, 0u, smp.k0, smp.k1);
+          e[0] = e[0] * smp.inv_t + gumbel_of(x.x);
+          e[1] = e[1] * smp.inv_t + gumbel_of(x.y);
+          e[2] = e[2] * smp.inv_t + gumbel_of(x.z);
+          e[3] = e[3] * smp.inv_t + gumbel_of(x.w);
+        }
 #pragma unroll
         for (int k = 0; k < 4; ++k)
           if (e[k] > bv || (e[k] == bv && i + k < bi)) { bv = e[k]; bi = i + k; }
@@ -817,10 +853,15 @@ __global__ void __launch_bounds__(512) argmax_rows_kernel(float* __restrict__ lo
   }
 }
 
-// logits: the projection's output buffer [M][V] (V a multiple of 4), completed in place.
+// logits: the projection's output buffer [M][V] (V a multiple of 4), completed in place.  With smp.inv_t > 0 row m
+// draws the token at position row_pos[m] + pos_add of sequence row_seq[m] (row m itself where row_seq is null).
 cudaError_t launch_argmax_rows(float* logits, const GemmOut& proj, int V, int32_t* out, const int32_t* out_index,
-                               const int32_t* m_total, int m_max, cudaStream_t st) {
-  launch_pdl(argmax_rows_kernel, m_max, 512, 0, st, logits, proj, V, out, out_index, m_total);
+                               const int32_t* m_total, int m_max, const Sampling& smp, const int32_t* row_seq,
+                               const int32_t* row_pos, int pos_add, cudaStream_t st) {
+  if (smp.inv_t > 0.0f)
+    launch_pdl(argmax_rows_kernel<true>, m_max, 512, 0, st, logits, proj, V, out, out_index, m_total, smp, row_seq, row_pos, pos_add);
+  else
+    launch_pdl(argmax_rows_kernel<false>, m_max, 512, 0, st, logits, proj, V, out, out_index, m_total, smp, row_seq, row_pos, pos_add);
   return cudaGetLastError();
 }
 

@@ -97,8 +97,14 @@ cudaError_t elementwise_prepare(int dtype);
 cudaError_t drafter_prepare(int dtype);
 cudaError_t launch_swiglu(int dtype, const GemmOut& proj, void* out_t, int F, const int32_t* m_total, int m_max,
                           int32_t* status, Chain* chain, cudaStream_t st);
+// Token choice at temperature > 0: inv_t = 1 / temperature (0: greedy), (k0, k1) the seed's two halves.
+struct Sampling {
+  float inv_t;
+  uint32_t k0, k1;
+};
 cudaError_t launch_argmax_rows(float* logits, const GemmOut& proj, int V, int32_t* out, const int32_t* out_index,
-                               const int32_t* m_total, int m_max, cudaStream_t st);
+                               const int32_t* m_total, int m_max, const Sampling& smp, const int32_t* row_seq,
+                               const int32_t* row_pos, int pos_add, cudaStream_t st);
 
 // drafter
 cudaError_t launch_draft_init(int dtype, const void* emb, const int32_t* root, const float* h, void* x_t, float* x_f,

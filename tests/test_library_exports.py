@@ -44,3 +44,4 @@ def test_null_arguments_rejected_without_gpu():
     assert L.redrafter_init(None, None, None, 0, None, 0, None) == 1
     assert L.redrafter_step(None, None, None, None) == 1
     assert L.redrafter_destroy(None) == 1
+    assert L.redrafter_set_sampling(None, 1.0, 0) == 1
