@@ -90,6 +90,7 @@ struct rd_handle {
   int trace_next;  // next trace slot, -1 = tracing off
   std::vector<double> trace_bytes;  // weight bytes of each traced launch (0: not a projection)
   int tc_grid, tc_smem;
+  int tc_pairs;   // CTA pairs of the pair projection kernel that fit the device at once (0: not used)
   std::vector<TensorMapBox> kv_maps;   // [layer][K | V]: cache planes as [sequences * heads * max_ctx][head dim] matrices
   Chain chain;  // counter hand-off between the launches of a forward pass
   std::unordered_map<const void*, TensorMapBox> maps;               // weights
@@ -269,9 +270,11 @@ int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, cons
     // actual row count); made on first use
     const void* amaps[16] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr,
                              nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+    // (on CTA pairs each CTA loads half a row tile: heights 8..mt/2 in steps of 8)
+    const int box_step = tc_use_pairs(m_max, N, h->tc_grid, h->tc_pairs) ? 8 : 16;
     const int n_maps = mt / 16;
     for (int i = 0; i < n_maps; ++i) {
-      const int box_rows = 16 * (i + 1);
+      const int box_rows = box_step * (i + 1);
       auto key = std::make_pair(A, box_rows);
       auto ia = h->act_maps.find(key);
       if (ia == h->act_maps.end()) {
@@ -290,7 +293,7 @@ int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, cons
       tr = h->ws.trace + (size_t)8 * h->trace_next++;
     }
     CK(h, launch_gemm_tc(&iw->second, amaps, N, K, m_total, m_max, raw, ld_raw, h->ws.tc_partial, h->ws.status,
-                         h->tc_grid, h->tc_smem, tr, out, chain, pair, st));
+                         h->tc_grid, h->tc_pairs, h->tc_smem, tr, out, chain, pair, st));
     return RD_OK;
   }
   if (chain) chain->cut();
@@ -523,11 +526,12 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
     if (ce == cudaSuccess) ce = drafter_prepare(dm.dtype);
     if (ce != cudaSuccess) return init_fail(h, RD_ERR_CUDA, "kernel set-up: %s", cudaGetErrorString(ce));
   }
+  h->tc_pairs = 0;
   if (h->use_tc) {
     int dev = 0, sms = 0;
     cudaError_t ce = cudaGetDevice(&dev);
     if (ce == cudaSuccess) ce = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (ce == cudaSuccess) ce = tc_prepare(&h->tc_smem);
+    if (ce == cudaSuccess) ce = tc_prepare(&h->tc_smem, &h->tc_pairs);
     if (ce == cudaSuccess) ce = attn_tc_prepare(dm.hd, dm.MW);
     if (ce == cudaSuccess) ce = attn_wide_prepare(dm.hd, dm.MW);
     if (ce == cudaSuccess) ce = attn_t5_prepare(dm.hd, dm.MW);

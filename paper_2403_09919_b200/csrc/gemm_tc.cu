@@ -29,6 +29,7 @@
 // status word, lets its copies land, frees its TMEM and exits; later launches see the flag and
 // return at once.
 #include <cuda.h>
+#include <stdio.h>
 #include <stdlib.h>
 
 #include "gemm_out.cuh"
@@ -420,6 +421,311 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
   }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// CTA pairs (tcgen05 cta_group::2) for launches of more than 128 rows
+// ---------------------------------------------------------------------------------------------
+// Beyond 128 rows a stage holds one weight tile (16 KB) and an activation box of up to 256 rows (32 KB): an SM
+// pulls in two to three times as many activation bytes (from L2) as weight bytes, and that intake, not the
+// weight stream or the tensor pipe, bounds the projection.  Here the two CTAs of a cluster work as one: each loads
+// ITS weight tile of a pair of adjacent tiles and HALF of the activation box, and one MMA of shape 256 x N x 16
+// issued by the leader multiplies both weight tiles by the whole box (the hardware reads each half from the CTA
+// that holds it).  Each CTA's tensor memory receives the accumulator of its own weight tile, so the epilogue and
+// the output layout are those of the pair mode above with "CTA" read as "cluster": units run over (row tile,
+// pair of weight tiles, k-block), cluster c owns [c*U/C, (c+1)*U/C), a partial slot holds the two tiles of a pair.
+//
+// Barriers.  full[s]: in the leader, completed by the bytes of both CTAs' copies (the peer's copies name the
+// leader's barrier).  empty[s] and tfull[a]: one in each CTA, the leader's MMA thread commits to both.
+// tempty[a]: in the leader, one arrival per epilogue warp of either CTA.  Before a CTA leaves, its producer waits
+// until the commits to its own empty barriers have landed and the cluster meets once more, so that no signal is
+// sent to shared memory that has been given back.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_id_x() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r));
+  return r;
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Copy into this CTA's shared memory; the bytes are counted on `bar`, which may lie in the peer CTA.
+__device__ __forceinline__ void tma_load_2d_pair_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;" ::"r"(dst),
+      "l"(map), "r"(bar), "r"(x), "r"(y), "l"(pol)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+      "l"(map), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// Arrives on one barrier (an address of the cluster's shared-memory window) once the MMAs issued so far are done.
+__device__ __forceinline__ void umma_commit_pair(uint32_t cluster_bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_bar) : "memory");
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_w,
+                                                                  const __grid_constant__ ActMaps maps_a,   // box heights 8, 16, ..., 128
+                                                                  const TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  pdl_launch_dependents();
+  if (p.trace && threadIdx.x == 0) { atomicMin(p.trace + 0, globaltimer()); }
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();        // 0: leader (issues the MMAs), 1: peer
+  const uint32_t cluster = cluster_id_x();
+  const bool chained = p.cs.signal_ptr != nullptr;
+  const bool early = (p.m_tiles_max == 1) || chained;
+  if (!early) {
+    if (threadIdx.x == 0) chain_wait_thread(p.cs);
+    __syncthreads();
+  }
+  GemmRows rows(1, p.mt);
+  if (p.m_tiles_max > 1) rows = gemm_row_tiles(p.mt, p.m_tiles_max, *p.m_total);
+  else if (chained) rows.rows = min(p.mt, max(16, (*p.m_total + 15) & ~15));
+  const int m_tiles = rows.n;
+  const long long C = gridDim.x >> 1;             // clusters
+  const int n_wt = (p.n_tiles + 1) / 2;           // pairs of weight tiles
+  const int n_groups = n_wt * m_tiles;
+  const long long U = (long long)n_groups * p.nkb;
+  const long long u0 = gemm_range_begin(cluster, U, C), u1 = gemm_range_begin(cluster + 1, U, C);
+  const int mt_eff = rows.rows, half = mt_eff >> 1;   // rows of a row tile; rows of it this CTA loads
+  const CUtensorMap* map_a = &maps_a.m[(half >> 3) - 1];
+
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  const uint32_t a_stage_bytes = (uint32_t)(p.mt >> 1) * TILE_K * 2;   // reserved
+  const uint32_t stage_bytes = (uint32_t)W_STAGE_BYTES + a_stage_bytes;
+  const uint32_t tx_bytes = 2u * ((uint32_t)W_STAGE_BYTES + (uint32_t)half * TILE_K * 2);   // both CTAs' copies of a stage
+  const uint32_t bar_base = base + p.stages * stage_bytes;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (p.stages + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * p.stages + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * p.stages + 2 + a); };
+  uint8_t* misc = smem_raw + (bar_base - raw) + 8u * (2 * p.stages + 4);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
+  volatile int* epi_ok = reinterpret_cast<volatile int*>(misc + 12);
+
+  const uint32_t n_it = (uint32_t)(u1 - u0);
+  const uint32_t pre = early ? min(n_it, (uint32_t)p.stages) : 0u;
+  const uint64_t pol_w = l2_policy_evict_first();
+  struct UnitPos {
+    int g, m_tile, kb;
+    uint32_t s, ph;
+  };
+  auto pos_at = [&](long long u) {
+    UnitPos q;
+    const int t = (int)(u / p.nkb);
+    q.kb = (int)(u - (long long)t * p.nkb);
+    q.m_tile = t / n_wt;
+    q.g = t - q.m_tile * n_wt;
+    q.s = 0; q.ph = 0;
+    return q;
+  };
+  auto advance = [&](UnitPos& q) {
+    if (++q.kb == p.nkb) {
+      q.kb = 0;
+      if (++q.g == n_wt) { q.g = 0; ++q.m_tile; }
+    }
+    if (++q.s == (uint32_t)p.stages) { q.s = 0; q.ph ^= 1u; }
+  };
+  // the bytes of both CTAs are counted on the leader's barrier; the leader announces them
+  auto issue_w = [&](const UnitPos& q) {
+    if (rank == 0) mbar_expect_tx(full_bar(q.s), tx_bytes);
+    // tile 2g + rank (the odd one may lie past the matrix: the copy then delivers zeros)
+    tma_load_2d_pair_hint(base + q.s * stage_bytes, &map_w, map_to_cta(full_bar(q.s), 0), q.kb * TILE_K,
+                          (2 * q.g + (int)rank) * TILE_N, pol_w);
+  };
+  auto issue_a = [&](const UnitPos& q) {
+    tma_load_2d_pair(base + q.s * stage_bytes + W_STAGE_BYTES, map_a, map_to_cta(full_bar(q.s), 0), q.kb * TILE_K,
+                     q.m_tile * mt_eff + (int)rank * half);
+  };
+
+  if (threadIdx.x == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map_a) : "memory");
+    for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }   // 4 epilogue warps x 2 CTAs
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
+                 "r"((uint32_t)p.tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  // both CTAs' barriers exist before either sends a signal to the other
+  tc_fence_before();
+  __syncwarp();
+  cluster_sync_all();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ===================== TMA producer (one per CTA) =====================
+    if (lane == 0 && u0 < u1) {
+      UnitPos q = pos_at(u0);
+      for (uint32_t i = 0; i < pre; ++i) { issue_w(q); advance(q); }
+      if (p.trace) atomicMax(p.trace + 7, globaltimer());
+      const int32_t status_before = *(volatile int32_t*)p.status;
+      if (early) chain_wait_thread(p.cs);
+      chain_fence_async_reads();
+      if (p.trace) { atomicMin(p.trace + 1, globaltimer()); atomicMax(p.trace + 2, globaltimer()); }
+      if (status_before & DEV_ERR_TIMEOUT) *abort_flag = 1;
+      q = pos_at(u0);
+      for (uint32_t i = 0; i < pre; ++i) { issue_a(q); advance(q); }
+      bool ok = true;
+      for (uint32_t i = pre; i < n_it; ++i) {
+        if (!mbar_wait(empty_bar(q.s), q.ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        issue_w(q);
+        issue_a(q);
+        advance(q);
+      }
+      // the leader's commits to this CTA's empty barriers must have landed before its shared memory is given back
+      if (ok) {
+        if (n_it < (uint32_t)p.stages) {
+          for (uint32_t s = 0; s < n_it && ok; ++s) ok = mbar_wait(empty_bar(s), 0u, abort_flag, p.status);
+        } else {
+          for (int j = 0; j < p.stages && ok; ++j) {
+            ok = mbar_wait(empty_bar(q.s), q.ph ^ 1u, abort_flag, p.status);
+            if (++q.s == (uint32_t)p.stages) { q.s = 0; q.ph ^= 1u; }
+          }
+        }
+      }
+      if (!ok || *abort_flag) {
+        const unsigned long long t0 = globaltimer();
+        while (globaltimer() - t0 < 2000000ull) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer (leader only) =====================
+    if (lane == 0 && u0 < u1 && rank == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(mt_eff >> 3) << 17) | ((uint32_t)((2 * TILE_N) >> 4) << 24);
+      uint32_t seg = 0, s = 0, ph = 0;
+      bool ok = true;
+      for (long long u = u0; u < u1 && ok; ++seg) {
+        const int t = (int)(u / p.nkb), kb0 = (int)(u - (long long)t * p.nkb);
+        const int kb1 = (int)min((long long)p.nkb, kb0 + (u1 - u));
+        const uint32_t a = seg & 1u, aph = (seg >> 1) & 1u;
+        if (!mbar_wait(tempty_bar(a), aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + a * (uint32_t)p.mt;
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(full_bar(s), ph, abort_flag, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t wdesc = umma_desc(base + s * stage_bytes);
+          const uint64_t adesc = umma_desc(base + s * stage_bytes + W_STAGE_BYTES);
+#pragma unroll
+          for (int k = 0; k < TILE_K / 16; ++k)
+            umma_bf16_pair(d_tmem, wdesc + 2 * k, adesc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+          umma_commit_pair(empty_bar(s));                  // this CTA's stage
+          umma_commit_pair(map_to_cta(empty_bar(s), 1));   // and the peer's
+          if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; }
+        }
+        if (ok) {
+          umma_commit_pair(tfull_bar(a));
+          umma_commit_pair(map_to_cta(tfull_bar(a), 1));
+        }
+        u += kb1 - kb0;
+      }
+      // the epilogue warps' arrivals for the last accumulators (the peer's come over the cluster) land before the end
+      for (uint32_t k = 0; k < 2u && k < seg && ok; ++k) {
+        const uint32_t sg = seg - 1 - k;
+        ok = mbar_wait(tempty_bar(sg & 1u), (sg >> 1) & 1u, abort_flag, p.status);
+      }
+      if (p.trace) { atomicMin(p.trace + 3, globaltimer()); atomicMax(p.trace + 4, globaltimer()); }
+    }
+  } else {
+    // ===================== epilogue (warps 2..5 of both CTAs) =====================
+    if (early) {
+      if (threadIdx.x == 64) chain_wait_thread(p.cs);
+      epi_bar_sync();
+    }
+    const int M = *p.m_total;
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    const int et = threadIdx.x - 64;
+    const uint32_t tempty_leader0 = map_to_cta(tempty_bar(0), 0), tempty_leader1 = map_to_cta(tempty_bar(1), 0);
+    uint32_t seg = 0;
+    bool ok = true;
+    for (long long u = u0; u < u1 && ok; ++seg) {
+      const int t = (int)(u / p.nkb), kb0 = (int)(u - (long long)t * p.nkb);
+      const int kb1 = (int)min((long long)p.nkb, kb0 + (u1 - u));
+      const int m_tile = t / n_wt, grp = t - m_tile * n_wt;
+      const int m_base = m_tile * mt_eff;
+      const int c_end = min(mt_eff, ((M - m_base) + 15) & ~15);
+      const uint32_t a = seg & 1u, aph = (seg >> 1) & 1u;
+      if (et == 0) *epi_ok = mbar_wait(tfull_bar(a), aph, abort_flag, p.status) ? 1 : 0;
+      epi_bar_sync();
+      if (!*epi_ok) { ok = false; break; }
+      tc_fence_after();
+      const int n = (2 * grp + (int)rank) * TILE_N + row;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * (uint32_t)p.mt;
+      // slot of the cluster: [tile 2g | tile 2g + 1], each [mt][128]
+      float* my_partial = p.partial + ((size_t)cluster * 2 + rank) * (size_t)p.mt * TILE_N;
+      for (int c0 = 0; c0 < c_end; c0 += 16) {
+        uint32_t r[16];
+        tmem_ld16(taddr + c0, r);
+        if (kb0 == 0) {
+          if (n < p.N) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int m = m_base + c0 + j;
+              if (m < M) p.raw[(size_t)m * p.ld_raw + n] = __uint_as_float(r[j]);
+            }
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) my_partial[(size_t)(c0 + j) * TILE_N + row] = __uint_as_float(r[j]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(a ? tempty_leader1 : tempty_leader0);
+      u += kb1 - kb0;
+    }
+  }
+
+  // ---- teardown: the pair meets (no signal is under way to either CTA's shared memory), then the tensor memory goes back
+  tc_fence_before();
+  __syncthreads();
+  if (p.trace && threadIdx.x == 0) { atomicMin(p.trace + 5, globaltimer()); atomicMax(p.trace + 6, globaltimer()); }
+  chain_exit(p.cs);
+  __syncwarp();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
+  }
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------------------------------------
@@ -468,7 +774,28 @@ int tc_pick_mt(int m_max) {
 
 size_t tc_partial_floats(int grid, int mt) { return (size_t)grid * mt * TILE_N * 2; }   // room for pair mode
 
-cudaError_t tc_prepare(int* smem_limit_out) {
+// Launch helpers for the CTA-pair kernel: clusters of two CTAs along x.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_pairs(bool ordered, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  prefer_max_shared(reinterpret_cast<const void*>(kernel));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = ordered ? 1 : 2;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(std::forward<Args>(args))...);
+}
+
+// smem_limit_out: dynamic shared memory a projection CTA may ask for.  pairs_out: CTA pairs (clusters of two) of
+// the pair kernel that can be resident at once with that much shared memory, 0 when it cannot be used.
+cudaError_t tc_prepare(int* smem_limit_out, int* pairs_out) {
   int dev = 0, lim = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
@@ -480,13 +807,85 @@ cudaError_t tc_prepare(int* smem_limit_out) {
   lim -= (int)fa.sharedSizeBytes;  // the opt-in limit covers static + dynamic shared memory
   e = cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
   if (smem_limit_out) *smem_limit_out = lim;
+  if (pairs_out) {
+    *pairs_out = 0;
+    if (e == cudaSuccess) {
+      int sms = 0;
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3((unsigned)(sms & ~1));
+      cfg.blockDim = dim3(NUM_THREADS);
+      cfg.dynamicSmemBytes = (size_t)lim;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      int n = 0;
+      const cudaError_t oe = cudaOccupancyMaxActiveClusters(&n, gemm_tc2_kernel, &cfg);
+      if (getenv("RD_DEBUG")) fprintf(stderr, "pair kernel: occupancy query %s, %d clusters of 2 on %d SMs, smem %d\n", cudaGetErrorString(oe), n, sms, lim);
+      if (oe == cudaSuccess) *pairs_out = n;
+      else cudaGetLastError();
+    }
+  }
   return e;
 }
 
+// Whether a launch bounded by m_max rows runs on CTA pairs (gemm_tc2_kernel): more than 128 rows (below, two
+// weight tiles per stage already share an activation box inside one CTA), at least one pair of weight tiles, and
+// pairs for (nearly) every SM resident at once.  The activation descriptors of such a launch have box heights
+// 8, 16, ..., mt / 2.
+bool tc_use_pairs(int m_max, int N, int grid, int pairs) {
+  static const int on = getenv("RD_TC_CTA2") ? atoi(getenv("RD_TC_CTA2")) : 1;                 // tuning toggles
+  static const int min_rows = getenv("RD_TC_CTA2_MIN") ? atoi(getenv("RD_TC_CTA2_MIN")) : 129;
+  return on && m_max >= min_rows && N > TILE_N && pairs > 0 && 2 * pairs >= grid - 4;
+}
+
+// The CTA-pair kernel: `pairs` clusters of two CTAs.  map_a: box heights 8, 16, ..., mt / 2.
+static cudaError_t launch_gemm_tc2(const void* map_w, const void* const map_a[16], int N, int K, const int32_t* m_total, int m_max,
+                                   float* raw, int ld_raw, float* partial, int32_t* status, int pairs, int smem_limit,
+                                   unsigned long long* trace, GemmOut* out_desc, Chain* chain, cudaStream_t st) {
+  TcParams p;
+  p.N = N; p.K = K; p.nkb = (K + TILE_K - 1) / TILE_K; p.n_tiles = (N + TILE_N - 1) / TILE_N;
+  p.mt = tc_pick_mt(m_max);
+  p.m_tiles_max = (m_max + p.mt - 1) / p.mt;
+  p.pair = 1;
+  const long long n_units = (long long)((p.n_tiles + 1) / 2) * p.nkb;
+  if (out_desc) {
+    // for the consumers a cluster is what a CTA is in pair mode: units over pairs of tiles, a slot holds both tiles
+    out_desc->raw = raw; out_desc->partial = partial; out_desc->ld = ld_raw; out_desc->nkb = p.nkb;
+    out_desc->n_tiles = p.n_tiles; out_desc->mt = p.mt; out_desc->grid = pairs; out_desc->m_tiles_max = p.m_tiles_max;
+    out_desc->all_work = (n_units >= pairs) ? 1 : 0;
+    out_desc->pair = 1;
+    out_desc->small32 = ((n_units * p.m_tiles_max + 1) * pairs < (1ll << 31)) ? 1 : 0;
+  }
+  const int stage_bytes = W_STAGE_BYTES + (p.mt / 2) * TILE_K * 2;
+  const int overhead = 1024 + 8 * (2 * 16 + 4) + 64;
+  int stages = (smem_limit - overhead) / stage_bytes;
+  if (stages > 16) stages = 16;
+  if (stages < 2) return cudaErrorInvalidConfiguration;
+  p.stages = stages;
+  int cols = 32;
+  while (cols < 2 * p.mt) cols <<= 1;
+  p.tmem_cols = cols;
+  p.m_total = m_total; p.raw = raw; p.ld_raw = ld_raw; p.partial = partial; p.status = status; p.trace = trace;
+  const bool first = chain && chain->enabled && chain->prev_ptr == nullptr;
+  p.cs = chain ? chain->link((unsigned)(2 * pairs)) : ChainSync{nullptr, 0u, nullptr, status, nullptr};
+  const size_t smem = (size_t)stages * stage_bytes + overhead;
+  ActMaps am;
+  for (int i = 0; i < ACT_MAPS; ++i) am.m[i] = *(const CUtensorMap*)(map_a[i] ? map_a[i] : map_a[0]);
+  launch_pairs(first, gemm_tc2_kernel, 2 * pairs, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[16], int N, int K, const int32_t* m_total, int m_max,
-                           float* raw, int ld_raw, float* partial, int32_t* status, int grid, int smem_limit,
+                           float* raw, int ld_raw, float* partial, int32_t* status, int grid, int pairs, int smem_limit,
                            unsigned long long* trace, GemmOut* out_desc, Chain* chain, int pair, cudaStream_t st) {
+  if (tc_use_pairs(m_max, N, grid, pairs))
+    return launch_gemm_tc2(map_w, map_a, N, K, m_total, m_max, raw, ld_raw, partial, status, pairs < grid / 2 ? pairs : grid / 2,
+                           smem_limit, trace, out_desc, chain, st);
   TcParams p;
   p.N = N; p.K = K; p.nkb = (K + TILE_K - 1) / TILE_K; p.n_tiles = (N + TILE_N - 1) / TILE_N;
   p.mt = tc_pick_mt(m_max > 0 ? m_max : 1);
