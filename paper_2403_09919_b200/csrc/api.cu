@@ -91,6 +91,8 @@ struct rd_handle {
   std::vector<double> trace_bytes;  // weight bytes of each traced launch (0: not a projection)
   int tc_grid, tc_smem;
   int tc_pairs;   // CTA pairs of the pair projection kernel that fit the device at once (0: not used)
+  int tc_pairs_avail, tc_pairs_min_rows;   // the pairs the device offers; row bound from which launches use them
+  bool tc_pairs_prefill;
   std::vector<TensorMapBox> kv_maps;   // [layer][K | V]: cache planes as [sequences * heads * max_ctx][head dim] matrices
   Chain chain;  // counter hand-off between the launches of a forward pass
   std::unordered_map<const void*, TensorMapBox> maps;               // weights
@@ -271,7 +273,8 @@ int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, cons
     const void* amaps[16] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr,
                              nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
     // (on CTA pairs each CTA loads half a row tile: heights 8..mt/2 in steps of 8)
-    const int box_step = tc_use_pairs(m_max, N, h->tc_grid, h->tc_pairs) ? 8 : 16;
+    const int pairs = tc_use_pairs(m_max, N, h->tc_grid, h->tc_pairs, h->tc_pairs_min_rows) ? h->tc_pairs : 0;
+    const int box_step = pairs ? 8 : 16;
     const int n_maps = mt / 16;
     for (int i = 0; i < n_maps; ++i) {
       const int box_rows = box_step * (i + 1);
@@ -293,7 +296,7 @@ int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, cons
       tr = h->ws.trace + (size_t)8 * h->trace_next++;
     }
     CK(h, launch_gemm_tc(&iw->second, amaps, N, K, m_total, m_max, raw, ld_raw, h->ws.tc_partial, h->ws.status,
-                         h->tc_grid, h->tc_pairs, h->tc_smem, tr, out, chain, pair, st));
+                         h->tc_grid, pairs, h->tc_smem, tr, out, chain, pair, st));
     return RD_OK;
   }
   if (chain) chain->cut();
@@ -526,18 +529,25 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
     if (ce == cudaSuccess) ce = drafter_prepare(dm.dtype);
     if (ce != cudaSuccess) return init_fail(h, RD_ERR_CUDA, "kernel set-up: %s", cudaGetErrorString(ce));
   }
-  h->tc_pairs = 0;
+  h->tc_pairs = 0; h->tc_pairs_avail = 0; h->tc_pairs_min_rows = 512; h->tc_pairs_prefill = false;
   if (h->use_tc) {
     int dev = 0, sms = 0;
     cudaError_t ce = cudaGetDevice(&dev);
     if (ce == cudaSuccess) ce = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (ce == cudaSuccess) ce = tc_prepare(&h->tc_smem, &h->tc_pairs);
+    if (ce == cudaSuccess) ce = tc_prepare(&h->tc_smem, &h->tc_pairs_avail);
     if (ce == cudaSuccess) ce = attn_tc_prepare(dm.hd, dm.MW);
     if (ce == cudaSuccess) ce = attn_wide_prepare(dm.hd, dm.MW);
     if (ce == cudaSuccess) ce = attn_t5_prepare(dm.hd, dm.MW);
     if (ce != cudaSuccess || sms <= 0)
       return init_fail(h, RD_ERR_CUDA, "tensor-core path set-up: %s", cudaGetErrorString(ce));
     h->tc_grid = sms < TC_MAX_GRID ? sms : TC_MAX_GRID;
+    // CTA-pair projections (tuning toggles, read when the handle is made): from a bound of 512 rows in decode steps
+    // (measured: 3-5 % of the step from about 700 packed rows, nothing between 130 and 450, where the one-CTA kernel
+    // starts earlier); RD_TC_CTA2=0 never, RD_TC_CTA2_MIN the row bound, RD_TC_CTA2_PREFILL=1 also in prompt passes.
+    if (getenv("RD_TC_CTA2") && atoi(getenv("RD_TC_CTA2")) == 0) h->tc_pairs_avail = 0;
+    h->tc_pairs_min_rows = getenv("RD_TC_CTA2_MIN") ? atoi(getenv("RD_TC_CTA2_MIN")) : 512;
+    h->tc_pairs_prefill = getenv("RD_TC_CTA2_PREFILL") && atoi(getenv("RD_TC_CTA2_PREFILL")) != 0;
+    h->tc_pairs = h->tc_pairs_avail;
     if (attn_t5_supported(dm.hd)) {
       // The tensor-core attention multiplies masked-out V rows by exact zeros: the cache has to hold finite values.
       ce = cudaMemset(h->kv, 0, (size_t)dm.n_layers * 2 * h->kv_plane * esize(dm.dtype));
@@ -667,7 +677,11 @@ int redrafter_prefill(rd_handle* h, const int32_t* tokens, const int32_t* prompt
     CKRT(h, cudaMemcpyAsync(w.m_total, &m, sizeof(int32_t), cudaMemcpyHostToDevice, st));
     CKRT(h, cudaStreamSynchronize(st));  // the host staging vectors are reused by the next pass
     h->ctx_bound = longest;  // bound of the key extent for this pass
+    // Prompt passes keep the one-CTA projection: their rows fill 256-row tiles exactly, projection plus consumer
+    // take the same time with either kernel (the fp32 intermediate bounds the pair), and the CTA pairs start later.
+    if (!h->tc_pairs_prefill) h->tc_pairs = 0;
     rc = forward_layers(h, nullptr, m, batch, longest_run, nullptr, st);
+    h->tc_pairs = h->tc_pairs_avail;
     if (rc) return rc;
     CK(h, launch_prefill_finish(w.hidden_f, w.last_row, w.h, dm.d, batch, st));
   }

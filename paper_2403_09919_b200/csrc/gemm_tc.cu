@@ -29,7 +29,6 @@
 // status word, lets its copies land, frees its TMEM and exits; later launches see the flag and
 // return at once.
 #include <cuda.h>
-#include <stdio.h>
 #include <stdlib.h>
 
 #include "gemm_out.cuh"
@@ -655,12 +654,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc2_kernel(const __grid_c
         }
         u += kb1 - kb0;
       }
+      if (p.trace) { atomicMin(p.trace + 3, globaltimer()); atomicMax(p.trace + 4, globaltimer()); }
       // the epilogue warps' arrivals for the last accumulators (the peer's come over the cluster) land before the end
       for (uint32_t k = 0; k < 2u && k < seg && ok; ++k) {
         const uint32_t sg = seg - 1 - k;
         ok = mbar_wait(tempty_bar(sg & 1u), (sg >> 1) & 1u, abort_flag, p.status);
       }
-      if (p.trace) { atomicMin(p.trace + 3, globaltimer()); atomicMax(p.trace + 4, globaltimer()); }
     }
   } else {
     // ===================== epilogue (warps 2..5 of both CTAs) =====================
@@ -825,7 +824,6 @@ cudaError_t tc_prepare(int* smem_limit_out, int* pairs_out) {
       cfg.numAttrs = 1;
       int n = 0;
       const cudaError_t oe = cudaOccupancyMaxActiveClusters(&n, gemm_tc2_kernel, &cfg);
-      if (getenv("RD_DEBUG")) fprintf(stderr, "pair kernel: occupancy query %s, %d clusters of 2 on %d SMs, smem %d\n", cudaGetErrorString(oe), n, sms, lim);
       if (oe == cudaSuccess) *pairs_out = n;
       else cudaGetLastError();
     }
@@ -833,14 +831,11 @@ cudaError_t tc_prepare(int* smem_limit_out, int* pairs_out) {
   return e;
 }
 
-// Whether a launch bounded by m_max rows runs on CTA pairs (gemm_tc2_kernel): more than 128 rows (below, two
-// weight tiles per stage already share an activation box inside one CTA), at least one pair of weight tiles, and
-// pairs for (nearly) every SM resident at once.  The activation descriptors of such a launch have box heights
-// 8, 16, ..., mt / 2.
-bool tc_use_pairs(int m_max, int N, int grid, int pairs) {
-  static const int on = getenv("RD_TC_CTA2") ? atoi(getenv("RD_TC_CTA2")) : 1;                 // tuning toggles
-  static const int min_rows = getenv("RD_TC_CTA2_MIN") ? atoi(getenv("RD_TC_CTA2_MIN")) : 129;
-  return on && m_max >= min_rows && N > TILE_N && pairs > 0 && 2 * pairs >= grid - 4;
+// Whether a launch bounded by m_max rows runs on CTA pairs (gemm_tc2_kernel): a bound of at least min_rows (the
+// caller's threshold), at least one pair of weight tiles, and pairs for (nearly) every SM resident at once.  The
+// activation descriptors of such a launch have box heights 8, 16, ..., mt / 2.
+bool tc_use_pairs(int m_max, int N, int grid, int pairs, int min_rows) {
+  return m_max >= min_rows && m_max > 16 && N > TILE_N && pairs > 0 && 2 * pairs >= grid - 4;
 }
 
 // The CTA-pair kernel: `pairs` clusters of two CTAs.  map_a: box heights 8, 16, ..., mt / 2.
@@ -883,7 +878,7 @@ static cudaError_t launch_gemm_tc2(const void* map_w, const void* const map_a[16
 cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[16], int N, int K, const int32_t* m_total, int m_max,
                            float* raw, int ld_raw, float* partial, int32_t* status, int grid, int pairs, int smem_limit,
                            unsigned long long* trace, GemmOut* out_desc, Chain* chain, int pair, cudaStream_t st) {
-  if (tc_use_pairs(m_max, N, grid, pairs))
+  if (tc_use_pairs(m_max, N, grid, pairs, 0))   // the caller passes pairs = 0 below its row threshold
     return launch_gemm_tc2(map_w, map_a, N, K, m_total, m_max, raw, ld_raw, partial, status, pairs < grid / 2 ? pairs : grid / 2,
                            smem_limit, trace, out_desc, chain, st);
   TcParams p;

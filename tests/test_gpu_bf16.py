@@ -346,3 +346,46 @@ def test_free_running_lossless_up_to_the_first_near_tie():
         steps += 1
     rig.eng.poll()
     assert steps >= 2 and spec == ref[:len(spec)]
+
+
+def _rig_with_env(env, **kw):
+    import os
+    old = {k: os.environ.get(k) for k in env}
+    os.environ.update(env)
+    try:
+        return Rig(**kw)
+    finally:
+        for k, v in old.items():
+            if v is None:
+                del os.environ[k]
+            else:
+                os.environ[k] = v
+
+
+@pytest.mark.parametrize("bw,batch,prompt", [(8, 1, 96), (16, 3, 300), (32, 2, 700)])
+def test_projection_on_cta_pairs_matches_the_one_cta_kernel(bw, batch, prompt):
+    """The CTA-pair projection (two CTAs share one MMA: each loads its weight tile and half of the activation box)
+    against the one-CTA kernel on the same weights and inputs: one row tile of 48 rows, one of 243 rows at most, and
+    several row tiles with a prompt processed in one pass of three; shapes that are not multiples of the tiles (an odd
+    number of weight tiles leaves the pair's second tile past the matrix).  Both sum each output element over the same
+    k-blocks in fp32, only the grouping into partial sums differs; a last-bit difference becomes a bf16 step (2^-9)
+    where an activation is rounded in front of the next projection, hence the same bound as between the tensor-core
+    and the CUDA-core path."""
+    cfg = dict(RAGGED, vocab=1100, d_ffn=1440, beam_width=bw, max_batch=batch, max_ctx=prompt + 200)
+    outs = []
+    for env in (dict(RD_TC_CTA2_MIN="17", RD_TC_CTA2_PREFILL="1"), dict(RD_TC_CTA2="0")):
+        r = _rig_with_env(env, cfg=cfg)
+        rng = np.random.default_rng(0)
+        prompts = [rng.integers(0, cfg["vocab"], size=prompt - 7 * b) for b in range(batch)]
+        r.eng.prefill(prompts)
+        beams = np.random.default_rng(1).integers(0, 3, size=(batch, bw, 5))
+        pk = r.eng.pack(dev(beams))
+        am, hid, lg = r.eng.verify(pk, want_logits=True)
+        r.eng.poll()
+        outs.append((pk.n.cpu().numpy(), lg.cpu().numpy(), r.eng.get_state()[2].cpu().numpy()))
+        r.eng.close()
+    assert (outs[0][0] == outs[1][0]).all()
+    for b in range(batch):
+        n = int(outs[0][0][b])
+        assert rel_err(outs[0][1][b, :n], outs[1][1][b, :n]) < 1e-2
+    assert rel_err(outs[0][2], outs[1][2]) < 1e-2
