@@ -25,6 +25,9 @@
 // the MMA issuer are single threads: their loops carry their positions along and contain no
 // division (a division by a run-time value per stage was what bounded the stream).
 //
+// Launches bounded by many rows run on CTA pairs instead (gemm_tc2_kernel below: tcgen05 cta_group::2, the
+// two CTAs of a cluster share one activation box).
+//
 // Every mbarrier wait is bounded (one second); on expiry the CTA raises DEV_ERR_TIMEOUT in the
 // status word, lets its copies land, frees its TMEM and exits; later launches see the flag and
 // return at once.
