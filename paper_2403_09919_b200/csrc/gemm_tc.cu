@@ -19,8 +19,8 @@
 // partial slot, and the consuming kernel folds them in CTA order (gemm_out.cuh).
 //
 // Roles: warp 0 = TMA producer (one or two 128x64 weight boxes and one activation box per stage),
-// warp 1 = MMA issuer and TMEM owner, warps 2..5 = epilogue (tcgen05.ld, one TMEM lane quarter
-// each).  Two TMEM accumulator buffers alternate so the epilogue of one segment overlaps the MMAs
+// warp 1 = MMA issuer and TMEM owner, warps 2.. = epilogue (tcgen05.ld; one warp per TMEM lane quarter,
+// or two that take every other group of 16 accumulator columns: see tc_threads).  Two TMEM accumulator buffers alternate so the epilogue of one segment overlaps the MMAs
 // of the next; the smem ring (full/empty mbarriers) never drains between tiles.  The producer and
 // the MMA issuer are single threads: their loops carry their positions along and contain no
 // division (a division by a run-time value per stage was what bounded the stream).
@@ -45,7 +45,10 @@ namespace {
 constexpr int TILE_N = 128;       // weight rows per tile (MMA M)
 constexpr int TILE_K = 64;        // bf16 per k-block = one 128-byte swizzle row
 constexpr int W_STAGE_BYTES = TILE_N * TILE_K * 2;
-constexpr int NUM_THREADS = 192;
+// Epilogue warps: one per tensor-memory lane quarter at decode size (fewer registers held beside the short kernels
+// that share the SM), two per quarter -- each takes every other group of 16 accumulator columns -- for launches of
+// more than 128 rows, whose accumulators are up to 256 columns wide.  EW (4 or 8) is a template parameter.
+__host__ __device__ constexpr int tc_threads(int ew) { return 64 + 32 * ew; }
 constexpr unsigned long long WAIT_LIMIT_NS = 1000000000ull;
 
 // Activation operand: one descriptor per box height, 16, 32, ..., 256 rows in m[0..15] (up to the launch's own
@@ -166,14 +169,15 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+template <int EW>
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(32 * EW) : "memory"); }
 
 // PAIR (one row tile of at most 128 rows): two adjacent weight tiles per stage share one activation box, and an
 // accumulator buffer holds both tiles.  Measured and dropped: the same pairing at up to 256 rows and with several
 // row tiles (a 256 x 256 output tile per unit).  Its two accumulators fill the tensor memory, so the epilogue no
 // longer overlaps the next tile's MMAs, and that costs what the shared activation box saves.
-template <bool PAIR>
-__global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
+template <bool PAIR, int EW>
+__global__ void __launch_bounds__(tc_threads(EW), EW == 4 ? 4 : 2) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
                                                                  const __grid_constant__ ActMaps maps_a,
                                                                  const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -276,7 +280,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(map_a) : "memory");
     for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 32 * EW); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -357,15 +361,18 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
       if (p.trace) { atomicMin(p.trace + 3, globaltimer()); atomicMax(p.trace + 4, globaltimer()); }   // all MMAs issued
     }
   } else {
-    // ===================== epilogue (warps 2..5) =====================
+    // ===================== epilogue (warps 2..) =====================
     if (early) {                            // the row count comes from preceding kernels, and their readers of
       if (threadIdx.x == 64) chain_wait_thread(p.cs);   // this launch's output buffers must be done
-      epi_bar_sync();
+      epi_bar_sync<EW>();
     }
     const int M = *p.m_total;
     const int q = warp & 3;                 // TMEM lane quarter this warp may read
     const int row = q * 32 + lane;          // weight row inside the tile
-    const int et = threadIdx.x - 64;        // 0..127
+    const int et = threadIdx.x - 64;        // 0 .. (epilogue threads - 1)
+    constexpr bool two_per_quarter = EW == 8;
+    const int chunk_par = ((warp - 2) >> 2) & 1;   // which of the quarter's two warps: it takes every other 16 columns
+    constexpr int chunk_step = two_per_quarter ? 32 : 16;
     uint32_t seg = 0;
     bool ok = true;
     for (long long u = u0; u < u1 && ok; ++seg) {
@@ -378,7 +385,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
       const uint32_t a = seg & 1u, aph = (seg >> 1) & 1u;
       // one thread does the bounded wait and tells the others, so that all 128 take the same branch
       if (et == 0) *epi_ok = mbar_wait(tfull_bar(a), aph, abort_flag, p.status) ? 1 : 0;
-      epi_bar_sync();
+      epi_bar_sync<EW>();
       if (!*epi_ok) { ok = false; break; }
       tc_fence_after();
       const uint32_t acc_cols = (uint32_t)p.mt * (PAIR ? 2u : 1u);
@@ -387,7 +394,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc_kernel(const __grid_co
         const int n = (n_tile0 + sub) * TILE_N + row;
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * acc_cols + (uint32_t)sub * (uint32_t)p.mt;
         float* my_partial = p.partial + (size_t)blockIdx.x * slot_floats + (size_t)sub * p.mt * TILE_N;
-        for (int c0 = 0; c0 < c_end; c0 += 16) {
+        for (int c0 = two_per_quarter ? 16 * (chunk_par ^ (sub & 1)) : 0; c0 < c_end; c0 += chunk_step) {
           uint32_t r[16];
           tmem_ld16(taddr + c0, r);
           if (kb0 == 0) {
@@ -490,7 +497,8 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t cluster_bar) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_bar) : "memory");
 }
 
-__global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_w,
+template <int EW>
+__global__ void __launch_bounds__(tc_threads(EW), EW == 4 ? 4 : 2) gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_w,
                                                                   const __grid_constant__ ActMaps maps_a,   // box heights 8, 16, ..., 128
                                                                   const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -572,7 +580,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc2_kernel(const __grid_c
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(map_a) : "memory");
     for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }   // 4 epilogue warps x 2 CTAs
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 2 * EW); }   // one arrival per epilogue warp of either CTA
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -665,15 +673,18 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc2_kernel(const __grid_c
       }
     }
   } else {
-    // ===================== epilogue (warps 2..5 of both CTAs) =====================
+    // ===================== epilogue (warps 2.. of both CTAs) =====================
     if (early) {
       if (threadIdx.x == 64) chain_wait_thread(p.cs);
-      epi_bar_sync();
+      epi_bar_sync<EW>();
     }
     const int M = *p.m_total;
     const int q = warp & 3;
     const int row = q * 32 + lane;
     const int et = threadIdx.x - 64;
+    constexpr bool two_per_quarter = EW == 8;
+    const int chunk_par = ((warp - 2) >> 2) & 1;
+    constexpr int chunk_step = two_per_quarter ? 32 : 16;
     const uint32_t tempty_leader0 = map_to_cta(tempty_bar(0), 0), tempty_leader1 = map_to_cta(tempty_bar(1), 0);
     uint32_t seg = 0;
     bool ok = true;
@@ -685,14 +696,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 4) gemm_tc2_kernel(const __grid_c
       const int c_end = min(mt_eff, ((M - m_base) + 15) & ~15);
       const uint32_t a = seg & 1u, aph = (seg >> 1) & 1u;
       if (et == 0) *epi_ok = mbar_wait(tfull_bar(a), aph, abort_flag, p.status) ? 1 : 0;
-      epi_bar_sync();
+      epi_bar_sync<EW>();
       if (!*epi_ok) { ok = false; break; }
       tc_fence_after();
       const int n = (2 * grp + (int)rank) * TILE_N + row;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * (uint32_t)p.mt;
       // slot of the cluster: [tile 2g | tile 2g + 1], each [mt][128]
       float* my_partial = p.partial + ((size_t)cluster * 2 + rank) * (size_t)p.mt * TILE_N;
-      for (int c0 = 0; c0 < c_end; c0 += 16) {
+      for (int c0 = two_per_quarter ? 16 * chunk_par : 0; c0 < c_end; c0 += chunk_step) {
         uint32_t r[16];
         tmem_ld16(taddr + c0, r);
         if (kb0 == 0) {
@@ -804,12 +815,13 @@ cudaError_t tc_prepare(int* smem_limit_out, int* pairs_out) {
   e = cudaDeviceGetAttribute(&lim, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   if (e != cudaSuccess) return e;
   cudaFuncAttributes fa;
-  e = cudaFuncGetAttributes(&fa, gemm_tc_kernel<false>);
+  e = cudaFuncGetAttributes(&fa, gemm_tc_kernel<false, 4>);
   if (e != cudaSuccess) return e;
   lim -= (int)fa.sharedSizeBytes;  // the opt-in limit covers static + dynamic shared memory
-  e = cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
+  e = cudaFuncSetAttribute(gemm_tc_kernel<false, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<false, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc2_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
   if (smem_limit_out) *smem_limit_out = lim;
   if (pairs_out) {
     *pairs_out = 0;
@@ -818,7 +830,7 @@ cudaError_t tc_prepare(int* smem_limit_out, int* pairs_out) {
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
       cudaLaunchConfig_t cfg = {};
       cfg.gridDim = dim3((unsigned)(sms & ~1));
-      cfg.blockDim = dim3(NUM_THREADS);
+      cfg.blockDim = dim3(tc_threads(8));
       cfg.dynamicSmemBytes = (size_t)lim;
       cudaLaunchAttribute attr[1];
       attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -826,7 +838,7 @@ cudaError_t tc_prepare(int* smem_limit_out, int* pairs_out) {
       cfg.attrs = attr;
       cfg.numAttrs = 1;
       int n = 0;
-      const cudaError_t oe = cudaOccupancyMaxActiveClusters(&n, gemm_tc2_kernel, &cfg);
+      const cudaError_t oe = cudaOccupancyMaxActiveClusters(&n, gemm_tc2_kernel<8>, &cfg);
       if (oe == cudaSuccess) *pairs_out = n;
       else cudaGetLastError();
     }
@@ -874,7 +886,7 @@ static cudaError_t launch_gemm_tc2(const void* map_w, const void* const map_a[16
   const size_t smem = (size_t)stages * stage_bytes + overhead;
   ActMaps am;
   for (int i = 0; i < ACT_MAPS; ++i) am.m[i] = *(const CUtensorMap*)(map_a[i] ? map_a[i] : map_a[0]);
-  launch_pairs(first, gemm_tc2_kernel, 2 * pairs, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+  launch_pairs(first, gemm_tc2_kernel<8>, 2 * pairs, tc_threads(8), smem, st, *(const CUtensorMap*)map_w, am, p);
   return cudaGetLastError();
 }
 
@@ -922,11 +934,16 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[16], int N
   ActMaps am;
   for (int i = 0; i < ACT_MAPS; ++i) am.m[i] = *(const CUtensorMap*)(map_a[i] ? map_a[i] : map_a[0]);
   if (p.pair) {
-    if (first) launch_ordered(gemm_tc_kernel<true>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
-    else launch_pdl(gemm_tc_kernel<true>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+    if (first) launch_ordered(gemm_tc_kernel<true, 4>, grid, tc_threads(4), smem, st, *(const CUtensorMap*)map_w, am, p);
+    else launch_pdl(gemm_tc_kernel<true, 4>, grid, tc_threads(4), smem, st, *(const CUtensorMap*)map_w, am, p);
   } else {
-    if (first) launch_ordered(gemm_tc_kernel<false>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
-    else launch_pdl(gemm_tc_kernel<false>, grid, NUM_THREADS, smem, st, *(const CUtensorMap*)map_w, am, p);
+    if (p.mt > 128) {
+      if (first) launch_ordered(gemm_tc_kernel<false, 8>, grid, tc_threads(8), smem, st, *(const CUtensorMap*)map_w, am, p);
+      else launch_pdl(gemm_tc_kernel<false, 8>, grid, tc_threads(8), smem, st, *(const CUtensorMap*)map_w, am, p);
+    } else {
+      if (first) launch_ordered(gemm_tc_kernel<false, 4>, grid, tc_threads(4), smem, st, *(const CUtensorMap*)map_w, am, p);
+      else launch_pdl(gemm_tc_kernel<false, 4>, grid, tc_threads(4), smem, st, *(const CUtensorMap*)map_w, am, p);
+    }
   }
   return cudaGetLastError();
 }
