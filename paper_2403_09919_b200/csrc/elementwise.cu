@@ -192,9 +192,10 @@ __global__ void __maxnreg__(88)
 // latency of a single short pass per CTA; with thousands of rows that becomes wave after wave of CTAs that each pay
 // the hand-off poll, the row-count load and one round trip for their data.  The *_wide variants fill the SMs once
 // and walk the rows in a loop, every load of a row in flight before the first is used.
-// The row-loop variants take over where the host-side bound on the rows exceeds one and a half row tiles: below that the
-// rows actually present mostly fit a single tile, which the kernels above handle on their fast path.
-constexpr int WIDE_ROWS_MIN = 384;
+// The row-loop variants take over where the host-side bound on the rows exceeds one row tile (measured at bounds of
+// 330 rows, 170-220 rows present: 2-5 % of the step against the kernels above; at a bound of 164 rows they lose).
+// RD_WIDE_MIN: tuning toggle.
+static const int WIDE_ROWS_MIN = getenv("RD_WIDE_MIN") ? atoi(getenv("RD_WIDE_MIN")) : 256;
 static int wide_sm_count() {
   static int n = 0;
   if (!n) {
