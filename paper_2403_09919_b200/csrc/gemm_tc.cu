@@ -45,6 +45,7 @@ namespace {
 constexpr int TILE_N = 128;       // weight rows per tile (MMA M)
 constexpr int TILE_K = 64;        // bf16 per k-block = one 128-byte swizzle row
 constexpr int W_STAGE_BYTES = TILE_N * TILE_K * 2;
+constexpr int MAX_STAGES = 16;    // ring slots the barrier block has room for
 // Epilogue warps: one per tensor-memory lane quarter at decode size (fewer registers held beside the short kernels
 // that share the SM), two per quarter -- each takes every other group of 16 accumulator columns -- for launches of
 // more than 128 rows, whose accumulators are up to 256 columns wide.  EW (4 or 8) is a template parameter.
@@ -60,6 +61,7 @@ struct ActMaps {
 
 struct TcParams {
   int N, K, nkb, n_tiles, mt, m_tiles_max, stages, tmem_cols;
+  int ring_bytes;     // shared memory of the stage ring (at least stages full-height stages)
   const int32_t* m_total;
   float* raw;         // [M][ld_raw] fp32 output
   int ld_raw;
@@ -216,23 +218,26 @@ __global__ void __launch_bounds__(tc_threads(EW), EW == 4 ? 4 : 2) gemm_tc_kerne
   // ---- shared memory carve-up (stage buffers 1024-byte aligned for the 128-byte swizzle)
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
-  const uint32_t a_stage_bytes = (uint32_t)p.mt * TILE_K * 2;          // reserved
   const uint32_t w_bytes = PAIR ? 2u * W_STAGE_BYTES : (uint32_t)W_STAGE_BYTES;
-  const uint32_t stage_bytes = w_bytes + a_stage_bytes;
+  const uint32_t ring_bytes = (uint32_t)p.ring_bytes;   // what the host reserved: p.stages stages of full height, or more
+  // Outside the pair mode the ring is cut by the rows actually present: a launch laid out for 256-row tiles that
+  // turns out to have 200 rows gets five stages instead of four, and the bytes in flight are what bounds the stream.
+  const uint32_t stage_bytes = w_bytes + (uint32_t)(PAIR ? p.mt : mt_eff) * TILE_K * 2;
+  const int n_stages = PAIR ? p.stages : min(MAX_STAGES, (int)(ring_bytes / stage_bytes));
   const uint32_t tx_bytes = w_bytes + (uint32_t)mt_eff * TILE_K * 2;   // arriving per stage
-  const uint32_t bar_base = base + p.stages * stage_bytes;  // 8-byte aligned
+  const uint32_t bar_base = base + ring_bytes;  // 8-byte aligned
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (p.stages + s); };
-  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * p.stages + a); };
-  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * p.stages + 2 + a); };
-  uint8_t* misc = smem_raw + (bar_base - raw) + 8u * (2 * p.stages + 4);
+  auto empty_bar = [&](int s) { return bar_base + 8u * (MAX_STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + 2 + a); };
+  uint8_t* misc = smem_raw + (bar_base - raw) + 8u * (2 * MAX_STAGES + 4);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
   volatile int* epi_ok = reinterpret_cast<volatile int*>(misc + 12);
 
   // iteration i of this CTA = unit u0 + i
   const uint32_t n_it = (uint32_t)(u1 - u0);
-  const uint32_t pre = early ? min(n_it, (uint32_t)p.stages) : 0u;
+  const uint32_t pre = early ? min(n_it, (uint32_t)n_stages) : 0u;
   const uint64_t pol_w = l2_policy_evict_first();
   // Position of the producer in its unit range, advanced without divisions: the producer is a single thread, and
   // a division by a run-time value is a chain of a hundred dependent instructions -- several of them per stage
@@ -255,7 +260,7 @@ __global__ void __launch_bounds__(tc_threads(EW), EW == 4 ? 4 : 2) gemm_tc_kerne
       q.kb = 0;
       if (++q.g == n_wt) { q.g = 0; ++q.m_tile; }
     }
-    if (++q.s == (uint32_t)p.stages) { q.s = 0; q.ph ^= 1u; }
+    if (++q.s == (uint32_t)n_stages) { q.s = 0; q.ph ^= 1u; }
   };
   auto issue_w = [&](const UnitPos& q) {
     const uint32_t dst = base + q.s * stage_bytes;
@@ -279,7 +284,7 @@ __global__ void __launch_bounds__(tc_threads(EW), EW == 4 ? 4 : 2) gemm_tc_kerne
     // (tensor-memory allocation, the other roles' start) needs to come first.
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(map_a) : "memory");
-    for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 32 * EW); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -353,7 +358,7 @@ __global__ void __launch_bounds__(tc_threads(EW), EW == 4 ? 4 : 2) gemm_tc_kerne
               umma_bf16(d_tmem + (uint32_t)p.mt, wdesc2 + 2 * k, adesc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
           }
           umma_commit(empty_bar(s));  // the stage is free once these MMAs have read it
-          if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; }
+          if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; }
         }
         if (ok) umma_commit(tfull_bar(a));
         u += kb1 - kb0;
@@ -923,6 +928,8 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[16], int N
   if (stages > 16) stages = 16;
   if (stages < 2) return cudaErrorInvalidConfiguration;
   p.stages = stages;
+  // outside the pair mode the kernel cuts the ring itself, by the rows present: it gets everything the budget allows
+  p.ring_bytes = p.pair ? stages * stage_bytes : ((budget - overhead) & ~1023);
   int cols = 32;
   while (cols < 2 * p.mt * (p.pair ? 2 : 1)) cols <<= 1;
   p.tmem_cols = cols;
@@ -930,7 +937,7 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[16], int N
   // the first launch of a chain starts after everything before it has completed (see launch_ordered)
   const bool first = chain && chain->enabled && chain->prev_ptr == nullptr;
   p.cs = chain ? chain->link((unsigned)grid) : ChainSync{nullptr, 0u, nullptr, status, nullptr};
-  const size_t smem = (size_t)stages * stage_bytes + overhead;
+  const size_t smem = (size_t)p.ring_bytes + overhead;
   ActMaps am;
   for (int i = 0; i < ACT_MAPS; ++i) am.m[i] = *(const CUtensorMap*)(map_a[i] ? map_a[i] : map_a[0]);
   if (p.pair) {
