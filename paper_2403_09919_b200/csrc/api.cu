@@ -529,7 +529,7 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
     if (ce == cudaSuccess) ce = drafter_prepare(dm.dtype);
     if (ce != cudaSuccess) return init_fail(h, RD_ERR_CUDA, "kernel set-up: %s", cudaGetErrorString(ce));
   }
-  h->tc_pairs = 0; h->tc_pairs_avail = 0; h->tc_pairs_min_rows = 512; h->tc_pairs_prefill = false;
+  h->tc_pairs = 0; h->tc_pairs_avail = 0; h->tc_pairs_min_rows = 1024; h->tc_pairs_prefill = false;
   if (h->use_tc) {
     int dev = 0, sms = 0;
     cudaError_t ce = cudaGetDevice(&dev);
@@ -541,11 +541,11 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
     if (ce != cudaSuccess || sms <= 0)
       return init_fail(h, RD_ERR_CUDA, "tensor-core path set-up: %s", cudaGetErrorString(ce));
     h->tc_grid = sms < TC_MAX_GRID ? sms : TC_MAX_GRID;
-    // CTA-pair projections (tuning toggles, read when the handle is made): from a bound of 512 rows in decode steps
-    // (measured: 3-5 % of the step from about 700 packed rows, nothing between 130 and 450, where the one-CTA kernel
-    // starts earlier); RD_TC_CTA2=0 never, RD_TC_CTA2_MIN the row bound, RD_TC_CTA2_PREFILL=1 also in prompt passes.
+    // CTA-pair projections (tuning toggles, read when the handle is made): from a bound of 1024 rows in decode steps
+    // (measured: 1-4 % of the step from about 650 packed rows; with bounds around 650 rows, 300-420 rows present, the
+    // one-CTA kernel, which starts earlier and has shorter tails, is 3-5 % ahead); RD_TC_CTA2=0 never, RD_TC_CTA2_MIN the row bound, RD_TC_CTA2_PREFILL=1 also in prompt passes.
     if (getenv("RD_TC_CTA2") && atoi(getenv("RD_TC_CTA2")) == 0) h->tc_pairs_avail = 0;
-    h->tc_pairs_min_rows = getenv("RD_TC_CTA2_MIN") ? atoi(getenv("RD_TC_CTA2_MIN")) : 512;
+    h->tc_pairs_min_rows = getenv("RD_TC_CTA2_MIN") ? atoi(getenv("RD_TC_CTA2_MIN")) : 1024;
     h->tc_pairs_prefill = getenv("RD_TC_CTA2_PREFILL") && atoi(getenv("RD_TC_CTA2_PREFILL")) != 0;
     h->tc_pairs = h->tc_pairs_avail;
     if (attn_t5_supported(dm.hd)) {
