@@ -240,3 +240,43 @@ def test_set_sampling_arguments_and_reset():
     r.eng.poll()
     assert int(root0[0]) == int(root1[0])
     r.eng.close()
+
+
+def test_draw_frequencies_on_the_gpu_follow_the_softmax():
+    """Distribution-level check through the CUDA path: the same verification pass under 600 seeds; for every packed
+    row the counts of its eight likeliest tokens and of the rest against softmax(logits / T) of the logits the GPU
+    returned (chi-square, 8 degrees of freedom, all rows pooled by their worst statistic)."""
+    r = Rig()
+    c = r.cfg
+    T = 0.6
+    prompt = synth.make_prompts(c, 1)[0]
+    r.eng.prefill([prompt])                                   # greedy root: the same rows under every seed
+    beams = np.random.default_rng(5).integers(0, 3, size=(1, c["beam_width"], c["beam_length"]))
+    pk = r.eng.pack(dev(beams))
+    n = int(pk.n[0])
+    n_seeds = 600
+    draws = np.zeros((n_seeds, n), dtype=np.int64)
+    logits = None
+    for seed in range(n_seeds):
+        r.eng.set_sampling(T, 1000 + seed)
+        toks, _, lg = r.eng.verify(pk, want_logits=logits is None)
+        draws[seed] = toks[0, :n].cpu().numpy()
+        if logits is None:
+            logits = lg[0, :n].cpu().numpy().astype(np.float64)
+    r.eng.poll()
+    worst = 0.0
+    for row in range(n):
+        z = logits[row] / T
+        p = np.exp(z - z.max())
+        p /= p.sum()
+        top = np.argsort(-p)[:8]
+        expect = np.append(p[top], 1.0 - p[top].sum()) * n_seeds
+        counts = np.array([(draws[:, row] == t).sum() for t in top] + [0])
+        counts[-1] = n_seeds - counts[:-1].sum()
+        worst = max(worst, float(((counts - expect) ** 2 / np.maximum(expect, 1e-9)).sum()))
+    # P[chi2_8 > 40] is about 3e-6 per row; 17 rows at most
+    assert worst < 40.0, worst
+    # rows that choose the token of the same position share their noise: with equal logits they would agree; across
+    # seeds the draws of one row do vary
+    assert len(set(draws[:, 0].tolist())) > 3
+    r.eng.close()
