@@ -1,7 +1,7 @@
 """Parity at the per-layer shapes of the larger workloads (13B, 7B batch 16, 33B), depth-reduced.
 
-The oracle cannot run these models at full depth in test time (tens of TFLOP per step on host cores),
-so each case keeps the workload's exact per-layer shapes, beam width, beam length and batch, cuts the
+With hundred-token prompts and every sequence followed, the oracle cannot run these models at full depth in
+test time (tens of TFLOP per step on host cores), so each case keeps the workload's exact per-layer shapes, beam width, beam length and batch, cuts the
 depth to two layers and the prompts to about a hundred tokens, and checks one planted-beam step:
 packing bit-exact, verification logits within the bf16 bound, greedy tokens where the oracle's gap
 decides them, acceptance + hand-off bit-exact against the oracle's rule on the GPU's own greedy tokens.
