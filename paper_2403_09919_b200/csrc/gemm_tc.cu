@@ -826,6 +826,7 @@ cudaError_t tc_prepare(int* smem_limit_out, int* pairs_out) {
   e = cudaFuncSetAttribute(gemm_tc_kernel<false, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<false, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<true, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc2_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
   if (smem_limit_out) *smem_limit_out = lim;
   if (pairs_out) {
@@ -941,8 +942,13 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[16], int N
   ActMaps am;
   for (int i = 0; i < ACT_MAPS; ++i) am.m[i] = *(const CUtensorMap*)(map_a[i] ? map_a[i] : map_a[0]);
   if (p.pair) {
-    if (first) launch_ordered(gemm_tc_kernel<true, 4>, grid, tc_threads(4), smem, st, *(const CUtensorMap*)map_w, am, p);
-    else launch_pdl(gemm_tc_kernel<true, 4>, grid, tc_threads(4), smem, st, *(const CUtensorMap*)map_w, am, p);
+    if (p.mt > 64) {   // two tiles of up to 128 columns per accumulator buffer: the epilogue on eight warps
+      if (first) launch_ordered(gemm_tc_kernel<true, 8>, grid, tc_threads(8), smem, st, *(const CUtensorMap*)map_w, am, p);
+      else launch_pdl(gemm_tc_kernel<true, 8>, grid, tc_threads(8), smem, st, *(const CUtensorMap*)map_w, am, p);
+    } else {
+      if (first) launch_ordered(gemm_tc_kernel<true, 4>, grid, tc_threads(4), smem, st, *(const CUtensorMap*)map_w, am, p);
+      else launch_pdl(gemm_tc_kernel<true, 4>, grid, tc_threads(4), smem, st, *(const CUtensorMap*)map_w, am, p);
+    }
   } else {
     if (p.mt > 128) {
       if (first) launch_ordered(gemm_tc_kernel<false, 8>, grid, tc_threads(8), smem, st, *(const CUtensorMap*)map_w, am, p);
