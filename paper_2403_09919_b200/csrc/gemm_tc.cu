@@ -47,8 +47,9 @@ constexpr int TILE_K = 64;        // bf16 per k-block = one 128-byte swizzle row
 constexpr int W_STAGE_BYTES = TILE_N * TILE_K * 2;
 constexpr int MAX_STAGES = 16;    // ring slots the barrier block has room for
 // Epilogue warps: one per tensor-memory lane quarter at decode size (fewer registers held beside the short kernels
-// that share the SM), two per quarter -- each takes every other group of 16 accumulator columns -- for launches of
-// more than 128 rows, whose accumulators are up to 256 columns wide.  EW (4 or 8) is a template parameter.
+// that share the SM), two per quarter -- each takes every other group of 16 accumulator columns -- where an
+// accumulator buffer is wide: launches of more than 128 rows (up to 256 columns) and pair-mode launches of more than
+// 64 rows (two tiles of up to 128 columns).  EW (4 or 8) is a template parameter.
 __host__ __device__ constexpr int tc_threads(int ew) { return 64 + 32 * ew; }
 constexpr unsigned long long WAIT_LIMIT_NS = 1000000000ull;
 
