@@ -410,7 +410,7 @@ __global__ void __launch_bounds__(SEL_THREADS) draft_select_kernel(
   chain_exit(cs);
 }
 
-// ---------------------------------------------------------------- selection in two short kernels (BW <= 32)
+// ---------------------------------------------------------------- selection in two short kernels (BW <= 64)
 // The one-CTA-per-row kernel above pulls a whole row of logits through one SM and ranks it there; with a
 // handful of rows that leaves most of the GPU idle for tens of microseconds.  Here every row is cut into S
 // segments (rows x S CTAs, about one per SM): a segment's CTA folds its logits, and reduces them to the
@@ -444,6 +444,7 @@ constexpr int SEG_ITEMS_MAX = 4;     // float4 per thread at most (the kernel is
 constexpr int SEG_FOLD = 2;
 constexpr int SEG_MAX_CAND = 512;    // S * BW candidates per row at most
 constexpr int MRG_THREADS = 256;
+constexpr int MRG_MAX_BW = 64;       // the merge kernel ranks BW x BW keys in shared memory
 
 template <int SEG_ITEMS>
 __global__ void __maxnreg__(88) draft_seg_kernel(GemmOut proj, int V, int BW, int seg_len4, float* __restrict__ seg_max,
@@ -552,7 +553,7 @@ __global__ void __launch_bounds__(MRG_THREADS) draft_merge_kernel(
   chain_enter(cs);
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[1]));
   __shared__ unsigned long long wbuf[MRG_THREADS / 32][SEG_MAX_CAND];
-  __shared__ unsigned long long top[32 * 32];
+  extern __shared__ unsigned long long top[];   // rows * BW keys (dynamic: 32 KB at beam width 64)
   __shared__ Cand s_win;
   const int BW = dm.BW, L = dm.L, V = dm.V;
   const int kout = blockIdx.x, b = blockIdx.y;
@@ -651,7 +652,7 @@ __global__ void __launch_bounds__(MRG_THREADS) draft_merge_kernel(
 
 // Segments per row for the two-kernel selection, or 0 when the shape does not fit it.
 int draft_select_segments(const Dims& dm, int rows, int grid_hint) {
-  if (dm.BW > 32 || (dm.V & 3)) return 0;
+  if (dm.BW > MRG_MAX_BW || (dm.V & 3)) return 0;
   int S = grid_hint / (rows > 0 ? rows : 1);
   const int s_cap = SEG_MAX_CAND / dm.BW < 32 ? SEG_MAX_CAND / dm.BW : 32;
   if (S > s_cap) S = s_cap;
@@ -665,6 +666,11 @@ int draft_select_segments(const Dims& dm, int rows, int grid_hint) {
 
 // Once per handle (and so per device): opt-in of the one-kernel selection's shared-memory row (opted in by init).
 cudaError_t drafter_prepare(int dtype) {
+  const int top_bytes = MRG_MAX_BW * MRG_MAX_BW * (int)sizeof(unsigned long long);   // beside 32 KB of static buffers
+  cudaError_t e = dtype == RD_DTYPE_FP32
+                      ? cudaFuncSetAttribute(draft_merge_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, top_bytes)
+                      : cudaFuncSetAttribute(draft_merge_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, top_bytes);
+  if (e != cudaSuccess) return e;
   return dtype == RD_DTYPE_FP32
              ? cudaFuncSetAttribute(draft_select_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)
              : cudaFuncSetAttribute(draft_select_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
@@ -697,7 +703,8 @@ cudaError_t launch_draft_select(int dtype, const GemmOut& proj, int call, float*
     if (e != cudaSuccess) return e;
     dim3 g2(dm.BW, B);
     const ChainSync c2 = chain ? chain->link(g2.x * g2.y) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
-    RD_DISPATCH(dtype, launch_pdl(draft_merge_kernel<T>, g2, MRG_THREADS, 0, st, S, call, (const float*)sc.seg_max,
+    const size_t top_bytes = (size_t)(call == 1 ? 1 : dm.BW) * dm.BW * sizeof(unsigned long long);
+    RD_DISPATCH(dtype, launch_pdl(draft_merge_kernel<T>, g2, MRG_THREADS, top_bytes, st, S, call, (const float*)sc.seg_max,
                                   (const float*)sc.seg_sum, (const float*)sc.seg_val, (const int32_t*)sc.seg_idx, score_in,
                                   score_out, hist_in, hist_out, (const T*)emb, s_new_f, ld_s, (T*)se_t, dm, beams_out,
                                   scores_out, dbg, c2));

@@ -389,3 +389,32 @@ def test_projection_on_cta_pairs_matches_the_one_cta_kernel(bw, batch, prompt):
         n = int(outs[0][0][b])
         assert rel_err(outs[0][1][b, :n], outs[1][1][b, :n]) < 1e-2
     assert rel_err(outs[0][2], outs[1][2]) < 1e-2
+
+
+@pytest.mark.parametrize("bw", [33, 64])
+def test_draft_scores_wide_beams(bw):
+    """Beam widths above 32 through the two-kernel selection (segments of the vocabulary, then one merging CTA per
+    surviving beam ranking BW x BW candidates): scores sorted, every score the log-probability of its sequence, best
+    score and total mass as the oracle's, identical beams where the oracle's candidate gaps are clear of the bound."""
+    cfg = dict(RAGGED, beam_width=bw, max_ctx=96 + 2 + bw * 5 + 8)
+    rig = Rig(cfg=cfg)
+    prompt, kv, ctx, g, h = prefilled(rig)
+    rig.eng.set_state(None, dev([g]), dev(np.asarray(h, dtype=np.float32)[None], torch.float32))
+    beams, scores = rig.eng.draft()
+    rig.eng.poll()
+    rb, rs, cand = ora.beam_search(rig.D, rig.W["tok_emb"], g, h, bw, 5, rig.odt, return_logp=True)
+    sc = scores[0].cpu().numpy()
+    bm = beams[0].cpu().numpy()
+    assert (np.diff(sc) <= 0).all()
+    assert len({tuple(b) for b in bm.tolist()}) == bw                      # distinct sequences
+    for i in (0, 1, bw // 2, bw - 1):
+        assert abs(ora.sequence_logprob(rig.D, rig.W["tok_emb"], g, h, bm[i], rig.odt) - sc[i]) < REL * abs(sc[i])
+    assert abs(sc[0] - rs[0]) < REL * abs(rs[0])
+    assert abs(sc.sum() - rs.sum()) < REL * abs(rs.sum())
+    clear = True
+    for c in cand:
+        s = np.sort(c)[::-1][:bw + 1]
+        clear = clear and (np.diff(s) < -2 * REL).all()
+    if clear:
+        assert bm.tolist() == rb.tolist()
+    rig.eng.close()
