@@ -445,6 +445,7 @@ constexpr int SEG_FOLD = 2;
 constexpr int SEG_MAX_CAND = 512;    // S * BW candidates per row at most
 constexpr int MRG_THREADS = 256;
 constexpr int MRG_MAX_BW = 64;       // the merge kernel ranks BW x BW keys in shared memory
+constexpr int MRG_NARROW_BW = 16;    // up to here the narrow variant (candidates re-read from shared memory) is the faster
 
 template <int SEG_ITEMS>
 __global__ void __maxnreg__(88) draft_seg_kernel(GemmOut proj, int V, int BW, int seg_len4, float* __restrict__ seg_max,
@@ -541,7 +542,7 @@ __global__ void __maxnreg__(88) draft_seg_kernel(GemmOut proj, int V, int BW, in
   chain_exit(cs);
 }
 
-template <typename T>
+template <typename T, bool WIDE>
 __global__ void __launch_bounds__(MRG_THREADS) draft_merge_kernel(
     int S, int call, const float* __restrict__ seg_max, const float* __restrict__ seg_sum, const float* __restrict__ seg_val,
     const int32_t* __restrict__ seg_idx, const float* __restrict__ score_in, float* __restrict__ score_out,
@@ -552,7 +553,6 @@ __global__ void __launch_bounds__(MRG_THREADS) draft_merge_kernel(
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[0]));
   chain_enter(cs);
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[1]));
-  __shared__ unsigned long long wbuf[MRG_THREADS / 32][SEG_MAX_CAND];
   extern __shared__ unsigned long long top[];   // rows * BW keys (dynamic: 32 KB at beam width 64)
   __shared__ Cand s_win;
   const int BW = dm.BW, L = dm.L, V = dm.V;
@@ -561,57 +561,131 @@ __global__ void __launch_bounds__(MRG_THREADS) draft_merge_kernel(
   const int rows = call == 1 ? 1 : BW;
   const int row0 = call == 1 ? b : b * BW;
   const int n = S * BW;
-  for (int rr = warp; rr < rows; rr += MRG_THREADS / 32) {
-    const int r = row0 + rr;
-    // every load of the row first: segment maxima and sums (S <= 32: one per lane), candidates, the row's score
-    const float sm = lane < S ? __ldcg(seg_max + (size_t)r * S + lane) : -INFINITY;
-    const float ss = lane < S ? __ldcg(seg_sum + (size_t)r * S + lane) : 0.f;
-    const float base = call == 1 ? 0.f : __ldcg(score_in + r);
-    for (int c = lane; c < n; c += 32) {
-      const float cv = __ldcg(seg_val + (size_t)r * n + c);
-      const int ci = __ldcg(seg_idx + (size_t)r * n + c);
-      wbuf[warp][c] = ci == 0x7fffffff ? 0ull : cand_key(cv, ci);
+  if constexpr (WIDE) {
+    // beam widths above 16: every thread keeps its share of the candidates in registers for all rounds
+    __shared__ unsigned long long shk[2][MRG_THREADS / 32];
+    constexpr int KPL = SEG_MAX_CAND / 32;   // keys per lane: the candidates of a row stay in registers for all rounds
+    for (int rr = warp; rr < rows; rr += MRG_THREADS / 32) {
+      const int r = row0 + rr;
+      // every load of the row first: segment maxima and sums (S <= 32: one per lane), candidates, the row's score
+      const float sm = lane < S ? __ldcg(seg_max + (size_t)r * S + lane) : -INFINITY;
+      const float ss = lane < S ? __ldcg(seg_sum + (size_t)r * S + lane) : 0.f;
+      const float base = call == 1 ? 0.f : __ldcg(score_in + r);
+      unsigned long long key[KPL];
+  #pragma unroll
+      for (int j = 0; j < KPL; ++j) {
+        const int c = lane + 32 * j;
+        key[j] = 0ull;
+        if (c < n) {
+          const float cv = __ldcg(seg_val + (size_t)r * n + c);
+          const int ci = __ldcg(seg_idx + (size_t)r * n + c);
+          key[j] = ci == 0x7fffffff ? 0ull : cand_key(cv, ci);
+        }
+      }
+      // log-sum-exp of the row from its segments
+      float m = sm;
+  #pragma unroll
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      float sum = sm > -INFINITY ? ss * __expf(sm - m) : 0.f;
+  #pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      const float row_lse = m + logf(sum);
+      unsigned long long pv = ~0ull;
+      for (int p = 0; p < BW; ++p) {
+        unsigned long long mine = 0ull;
+  #pragma unroll
+        for (int j = 0; j < KPL; ++j) mine = max(mine, key[j] < pv ? key[j] : 0ull);
+        mine = warp_max_key(mine);
+        if (lane == 0) {
+          const int bi = key_index(mine);
+          top[rr * BW + p] = cand_key(base + (key_value(mine) - row_lse), rr * V + (bi == 0x7fffffff ? 0 : bi));
+        }
+        pv = mine;
+      }
     }
-    // log-sum-exp of the row from its segments
-    float m = sm;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    float sum = sm > -INFINITY ? ss * __expf(sm - m) : 0.f;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    const float row_lse = m + logf(sum);
-    __syncwarp();
-    unsigned long long pv = ~0ull;
-    for (int p = 0; p < BW; ++p) {
-      unsigned long long mine = 0ull;
+    __syncthreads();
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[2]));
+    // the beam of rank kout among the rows * BW candidates, (score desc, flat index asc): all threads hold their share
+    // of the candidates in registers; one warp reduction and one barrier per round (two result buffers in turn)
+    {
+      const int n_cand = rows * BW;
+      constexpr int KPT = MRG_MAX_BW * MRG_MAX_BW / MRG_THREADS;
+      unsigned long long key[KPT];
+  #pragma unroll
+      for (int j = 0; j < KPT; ++j) {
+        const int c = threadIdx.x + MRG_THREADS * j;
+        key[j] = c < n_cand ? top[c] : 0ull;
+      }
+      unsigned long long pv = ~0ull;
+      for (int p = 0; p <= kout; ++p) {
+        unsigned long long mine = 0ull;
+  #pragma unroll
+        for (int j = 0; j < KPT; ++j) mine = max(mine, key[j] < pv ? key[j] : 0ull);
+        mine = warp_max_key(mine);
+        if (lane == 0) shk[p & 1][warp] = mine;
+        __syncthreads();
+        unsigned long long best = 0ull;
+  #pragma unroll
+        for (int w = 0; w < MRG_THREADS / 32; ++w) best = max(best, shk[p & 1][w]);
+        pv = best;
+      }
+      if (threadIdx.x == 0) s_win = Cand{key_value(pv), key_index(pv)};
+    }
+  } else {
+    // narrow beams: a row has a few candidates per lane and the final ranking a few per lane of one warp
+    __shared__ unsigned long long wbuf[MRG_THREADS / 32][SEG_MAX_CAND];
+    for (int rr = warp; rr < rows; rr += MRG_THREADS / 32) {
+      const int r = row0 + rr;
+      // every load of the row first: segment maxima and sums (S <= 32: one per lane), candidates, the row's score
+      const float sm = lane < S ? __ldcg(seg_max + (size_t)r * S + lane) : -INFINITY;
+      const float ss = lane < S ? __ldcg(seg_sum + (size_t)r * S + lane) : 0.f;
+      const float base = call == 1 ? 0.f : __ldcg(score_in + r);
       for (int c = lane; c < n; c += 32) {
-        const unsigned long long x = wbuf[warp][c];
-        mine = max(mine, x < pv ? x : 0ull);
+        const float cv = __ldcg(seg_val + (size_t)r * n + c);
+        const int ci = __ldcg(seg_idx + (size_t)r * n + c);
+        wbuf[warp][c] = ci == 0x7fffffff ? 0ull : cand_key(cv, ci);
       }
-      mine = warp_max_key(mine);
-      if (lane == 0) {
-        const int bi = key_index(mine);
-        top[rr * BW + p] = cand_key(base + (key_value(mine) - row_lse), rr * V + (bi == 0x7fffffff ? 0 : bi));
+      // log-sum-exp of the row from its segments
+      float m = sm;
+  #pragma unroll
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      float sum = sm > -INFINITY ? ss * __expf(sm - m) : 0.f;
+  #pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      const float row_lse = m + logf(sum);
+      __syncwarp();
+      unsigned long long pv = ~0ull;
+      for (int p = 0; p < BW; ++p) {
+        unsigned long long mine = 0ull;
+        for (int c = lane; c < n; c += 32) {
+          const unsigned long long x = wbuf[warp][c];
+          mine = max(mine, x < pv ? x : 0ull);
+        }
+        mine = warp_max_key(mine);
+        if (lane == 0) {
+          const int bi = key_index(mine);
+          top[rr * BW + p] = cand_key(base + (key_value(mine) - row_lse), rr * V + (bi == 0x7fffffff ? 0 : bi));
+        }
+        pv = mine;
       }
-      pv = mine;
+      __syncwarp();
     }
-    __syncwarp();
-  }
-  __syncthreads();
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[2]));
-  // the beam of rank kout among the rows * BW candidates, (score desc, flat index asc)
-  if (warp == 0) {
-    const int n_cand = rows * BW;
-    unsigned long long pv = ~0ull;
-    for (int p = 0; p <= kout; ++p) {
-      unsigned long long mine = 0ull;
-      for (int c = lane; c < n_cand; c += 32) {
-        const unsigned long long x = top[c];
-        mine = max(mine, x < pv ? x : 0ull);
+    __syncthreads();
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[2]));
+    // the beam of rank kout among the rows * BW candidates, (score desc, flat index asc)
+    if (warp == 0) {
+      const int n_cand = rows * BW;
+      unsigned long long pv = ~0ull;
+      for (int p = 0; p <= kout; ++p) {
+        unsigned long long mine = 0ull;
+        for (int c = lane; c < n_cand; c += 32) {
+          const unsigned long long x = top[c];
+          mine = max(mine, x < pv ? x : 0ull);
+        }
+        pv = warp_max_key(mine);
       }
-      pv = warp_max_key(mine);
+      if (lane == 0) s_win = Cand{key_value(pv), key_index(pv)};
     }
-    if (lane == 0) s_win = Cand{key_value(pv), key_index(pv)};
   }
   __syncthreads();
   const Cand win = s_win;
@@ -666,10 +740,10 @@ int draft_select_segments(const Dims& dm, int rows, int grid_hint) {
 
 // Once per handle (and so per device): opt-in of the one-kernel selection's shared-memory row (opted in by init).
 cudaError_t drafter_prepare(int dtype) {
-  const int top_bytes = MRG_MAX_BW * MRG_MAX_BW * (int)sizeof(unsigned long long);   // beside 32 KB of static buffers
+  const int top_bytes = MRG_MAX_BW * MRG_MAX_BW * (int)sizeof(unsigned long long);
   cudaError_t e = dtype == RD_DTYPE_FP32
-                      ? cudaFuncSetAttribute(draft_merge_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, top_bytes)
-                      : cudaFuncSetAttribute(draft_merge_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, top_bytes);
+                      ? cudaFuncSetAttribute(draft_merge_kernel<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, top_bytes)
+                      : cudaFuncSetAttribute(draft_merge_kernel<__nv_bfloat16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, top_bytes);
   if (e != cudaSuccess) return e;
   return dtype == RD_DTYPE_FP32
              ? cudaFuncSetAttribute(draft_select_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)
@@ -704,10 +778,19 @@ cudaError_t launch_draft_select(int dtype, const GemmOut& proj, int call, float*
     dim3 g2(dm.BW, B);
     const ChainSync c2 = chain ? chain->link(g2.x * g2.y) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
     const size_t top_bytes = (size_t)(call == 1 ? 1 : dm.BW) * dm.BW * sizeof(unsigned long long);
-    RD_DISPATCH(dtype, launch_pdl(draft_merge_kernel<T>, g2, MRG_THREADS, top_bytes, st, S, call, (const float*)sc.seg_max,
-                                  (const float*)sc.seg_sum, (const float*)sc.seg_val, (const int32_t*)sc.seg_idx, score_in,
-                                  score_out, hist_in, hist_out, (const T*)emb, s_new_f, ld_s, (T*)se_t, dm, beams_out,
-                                  scores_out, dbg, c2));
+    if (dm.BW > MRG_NARROW_BW) {
+      constexpr bool WIDE_ = true;
+      RD_DISPATCH(dtype, launch_pdl(draft_merge_kernel<T, WIDE_>, g2, MRG_THREADS, top_bytes, st, S, call, (const float*)sc.seg_max,
+                                    (const float*)sc.seg_sum, (const float*)sc.seg_val, (const int32_t*)sc.seg_idx, score_in,
+                                    score_out, hist_in, hist_out, (const T*)emb, s_new_f, ld_s, (T*)se_t, dm, beams_out,
+                                    scores_out, dbg, c2));
+    } else {
+      constexpr bool WIDE_ = false;
+      RD_DISPATCH(dtype, launch_pdl(draft_merge_kernel<T, WIDE_>, g2, MRG_THREADS, top_bytes, st, S, call, (const float*)sc.seg_max,
+                                    (const float*)sc.seg_sum, (const float*)sc.seg_val, (const int32_t*)sc.seg_idx, score_in,
+                                    score_out, hist_in, hist_out, (const T*)emb, s_new_f, ld_s, (T*)se_t, dm, beams_out,
+                                    scores_out, dbg, c2));
+    }
     return cudaGetLastError();
   }
   const size_t select = ((size_t)32 * dm.BW + SEL_LIST_CAP) * sizeof(Cand) + (size_t)dm.V * sizeof(float);
