@@ -447,7 +447,7 @@ constexpr int MRG_THREADS = 256;
 constexpr int MRG_MAX_BW = 64;       // the merge kernel ranks BW x BW keys in shared memory
 constexpr int MRG_NARROW_BW = 16;    // up to here the narrow variant (candidates re-read from shared memory) is the faster
 
-template <int SEG_ITEMS>
+template <int SEG_ITEMS, bool SORTED>
 __global__ void __maxnreg__(88) draft_seg_kernel(GemmOut proj, int V, int BW, int seg_len4, float* __restrict__ seg_max,
                                                  float* __restrict__ seg_sum, float* __restrict__ seg_val,
                                                  int32_t* __restrict__ seg_idx, const int32_t* __restrict__ m_total,
@@ -522,22 +522,61 @@ __global__ void __maxnreg__(88) draft_seg_kernel(GemmOut proj, int V, int BW, in
   for (int k = 0; k < SEG_ITEMS; ++k)
 #pragma unroll
     for (int e = 0; e < 4; ++e) key[k * 4 + e] = ok[k] ? cand_key(v[k][e], col[k] + e) : 0ull;
-  unsigned long long prev = ~0ull;
-  for (int p = 0; p < BW; ++p) {
-    unsigned long long mine = 0ull;
+  constexpr int NK = SEG_ITEMS * 4;
+  if constexpr (SORTED) {
+    // Wide beams: every thread first sorts its own keys (best first, a bitonic network in registers); a round then
+    // looks at one key per thread, the head of its list, and the thread that held the winner moves its list up.
+    // BW rounds of NK compares each become one sort and BW rounds of one.
 #pragma unroll
-    for (int q = 0; q < SEG_ITEMS * 4; ++q) mine = max(mine, key[q] < prev ? key[q] : 0ull);
-    mine = warp_max_key(mine);
-    if (lane == 0) shk[p & 1][warp] = mine;
-    __syncthreads();
-    unsigned long long best = 0ull;
+    for (int k = 2; k <= NK; k <<= 1)
 #pragma unroll
-    for (int w = 0; w < SEG_THREADS / 32; ++w) best = max(best, shk[p & 1][w]);
-    if (threadIdx.x == 0) {
-      seg_val[((size_t)r * S + sgm) * BW + p] = key_value(best);
-      seg_idx[((size_t)r * S + sgm) * BW + p] = key_index(best);
+      for (int j = k >> 1; j > 0; j >>= 1)
+#pragma unroll
+        for (int i = 0; i < NK; ++i) {
+          const int l = i ^ j;
+          if (l > i) {
+            const bool desc = (i & k) == 0;
+            const unsigned long long a = key[i], b = key[l];
+            const bool sw = desc ? a < b : a > b;
+            key[i] = sw ? b : a;
+            key[l] = sw ? a : b;
+          }
+        }
+    for (int p = 0; p < BW; ++p) {
+      const unsigned long long mine = warp_max_key(key[0]);
+      if (lane == 0) shk[p & 1][warp] = mine;
+      __syncthreads();
+      unsigned long long best = 0ull;
+#pragma unroll
+      for (int w = 0; w < SEG_THREADS / 32; ++w) best = max(best, shk[p & 1][w]);
+      if (threadIdx.x == 0) {
+        seg_val[((size_t)r * S + sgm) * BW + p] = key_value(best);
+        seg_idx[((size_t)r * S + sgm) * BW + p] = key_index(best);
+      }
+      if (key[0] == best && best != 0ull) {   // keys are unique: one thread of the CTA
+#pragma unroll
+        for (int i = 0; i + 1 < NK; ++i) key[i] = key[i + 1];
+        key[NK - 1] = 0ull;
+      }
     }
-    prev = best;
+  } else {
+    unsigned long long prev = ~0ull;
+    for (int p = 0; p < BW; ++p) {
+      unsigned long long mine = 0ull;
+#pragma unroll
+      for (int q = 0; q < NK; ++q) mine = max(mine, key[q] < prev ? key[q] : 0ull);
+      mine = warp_max_key(mine);
+      if (lane == 0) shk[p & 1][warp] = mine;
+      __syncthreads();
+      unsigned long long best = 0ull;
+#pragma unroll
+      for (int w = 0; w < SEG_THREADS / 32; ++w) best = max(best, shk[p & 1][w]);
+      if (threadIdx.x == 0) {
+        seg_val[((size_t)r * S + sgm) * BW + p] = key_value(best);
+        seg_idx[((size_t)r * S + sgm) * BW + p] = key_index(best);
+      }
+      prev = best;
+    }
   }
   chain_exit(cs);
 }
@@ -764,15 +803,14 @@ cudaError_t launch_draft_select(int dtype, const GemmOut& proj, int call, float*
     dim3 g1(S, rows);
     const ChainSync c1 = chain ? chain->link(g1.x * g1.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
     const int items = (seg_len4 + SEG_THREADS - 1) / SEG_THREADS;
-    if (items <= 1)
-      launch_pdl(draft_seg_kernel<1>, g1, SEG_THREADS, 0, st, proj, dm.V, dm.BW, seg_len4, sc.seg_max, sc.seg_sum, sc.seg_val,
-                 sc.seg_idx, m_total, c1);
-    else if (items == 2)
-      launch_pdl(draft_seg_kernel<2>, g1, SEG_THREADS, 0, st, proj, dm.V, dm.BW, seg_len4, sc.seg_max, sc.seg_sum, sc.seg_val,
-                 sc.seg_idx, m_total, c1);
-    else
-      launch_pdl(draft_seg_kernel<4>, g1, SEG_THREADS, 0, st, proj, dm.V, dm.BW, seg_len4, sc.seg_max, sc.seg_sum, sc.seg_val,
-                 sc.seg_idx, m_total, c1);
+    const bool sorted = dm.BW > MRG_NARROW_BW;   // wide beams: the threads sort their keys once
+#define RD_SEG_LAUNCH(ITEMS, SRT)                                                                                        \
+  launch_pdl(draft_seg_kernel<ITEMS, SRT>, g1, SEG_THREADS, 0, st, proj, dm.V, dm.BW, seg_len4, sc.seg_max, sc.seg_sum, \
+             sc.seg_val, sc.seg_idx, m_total, c1)
+    if (items <= 1) { if (sorted) RD_SEG_LAUNCH(1, true); else RD_SEG_LAUNCH(1, false); }
+    else if (items == 2) { if (sorted) RD_SEG_LAUNCH(2, true); else RD_SEG_LAUNCH(2, false); }
+    else { if (sorted) RD_SEG_LAUNCH(4, true); else RD_SEG_LAUNCH(4, false); }
+#undef RD_SEG_LAUNCH
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     dim3 g2(dm.BW, B);
