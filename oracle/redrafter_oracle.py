@@ -45,13 +45,29 @@ architecture, KV cache handling, tie breaking).  The readings used here:
     branch or the step that reaches it: speculative decoding reproduces plain sampled
     decoding token for token.
 
+  * Precision (the paper states none).  By default everything is computed in the
+    working precision.  The bf16 configurations of the CUDA library STORE some
+    intermediates in bfloat16: every vector that feeds a projection (the normalised
+    residual stream, the attention output, the SwiGLU output, the drafter's [s, e] and
+    [s, h] vectors and its head activations), the rotated queries and keys and the values
+    (the K/V cache), and the softmax weights that multiply V.  With store="bf16" the
+    functions below round exactly those arrays, element by element, to the nearest
+    bfloat16 (ties to even) and change nothing else: no blocking, no reordering, sums
+    and softmax statistics stay in the working precision, the residual stream and the
+    hidden state handed to the drafter stay unrounded.  Comparing the two modes on the
+    CPU measures what that storage costs in accuracy, independently of any kernel.
+
 Parity pins (tests/test_oracle_*.py): the printed dedup example, brute-force
 prefix sets, packed-tree == per-beam causal verification, speculative == plain
 greedy decoding, beam width 1 == greedy drafting, exhaustive beam search on a tiny
 vocabulary, closed forms for the RNN cell and the head, library cross-checks; for
 sampling: the generator's published known answers, sample frequencies against the
 softmax, the accept/resample rule worked out exactly on small cases, speculative ==
-plain sampled decoding.
+plain sampled decoding; for store="bf16": round_bf16 against the bit-level definition
+and a library cast, idempotence, the unrounded mode's own pins re-run in this mode
+(packed-tree == per-beam, speculative == plain decoding, beam width 1 == greedy
+drafting, scores == sequence log-probabilities), and the size of the storage error and
+its growth with depth (tests/test_oracle_storage.py).
 Parity unpinned: nothing in the paper prints a weights-to-beams example, so the
 drafter's exact beams are pinned by properties only.
 """
@@ -75,6 +91,24 @@ def convert_weights(W, D, dtype):
     def conv(v):
         return [_c(t, dtype) for t in v] if isinstance(v, list) else _c(v, dtype)
     return {k: conv(v) for k, v in W.items()}, {k: conv(v) for k, v in D.items()}
+
+
+def round_bf16(a):
+    """Every element rounded to the nearest bfloat16 (8 significand bits, float32's exponent range; ties to even),
+    returned in the input's dtype.  The value is first taken to float32, as the stored intermediates are."""
+    a = np.asarray(a)
+    u = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+    lsb = (u >> np.uint32(16)) & np.uint32(1)                 # last bit that survives: decides ties
+    u = (u + np.uint32(0x7FFF) + lsb) & np.uint32(0xFFFF0000)
+    return u.view(np.float32).astype(a.dtype if a.dtype.kind == "f" else np.float32)
+
+
+def _st(a, store):
+    """`a` as it is stored between two operations: unchanged, or rounded to bfloat16."""
+    if store is None:
+        return a
+    assert store == "bf16"
+    return round_bf16(a)
 
 
 def silu(x):
@@ -188,12 +222,13 @@ class KVCache:
         self.v = np.zeros((n_layers, max_ctx, n_heads, hd), dtype=dtype)
 
 
-def llm_forward(W, cfg, tokens, pos, mask, kv, ctx, dtype=F, want_logits=True):
+def llm_forward(W, cfg, tokens, pos, mask, kv, ctx, dtype=F, want_logits=True, store=None):
     """Forward over `tokens` (rows) with explicit positions and mask.
 
     Row n attends cache slots [0, ctx) and the rows m with mask[n, m] True (self
     included); its key/value are written provisionally to slot ctx + n.
     Returns (hidden [rows, d] after the final norm, logits [rows, V] or None).
+    store="bf16": projection inputs, Q, K, V and the softmax weights are rounded (module docstring).
     """
     H = cfg["n_heads"]
     d = cfg["d_model"]
@@ -207,11 +242,11 @@ def llm_forward(W, cfg, tokens, pos, mask, kv, ctx, dtype=F, want_logits=True):
     x = np.asarray(W["tok_emb"][tokens], dtype=dtype)
     scale = 1.0 / np.sqrt(hd)
     for l in range(cfg["n_layers"]):
-        a = rmsnorm(x, _c(W["attn_norm"][l], dtype), eps)
+        a = _st(rmsnorm(x, _c(W["attn_norm"][l], dtype), eps), store)
         qkv = a @ _c(W["wqkv"][l], dtype).T                          # [n, 3d]
-        q = rope(qkv[:, :d].reshape(n, H, hd), pos, theta)
-        k = rope(qkv[:, d:2 * d].reshape(n, H, hd), pos, theta)
-        v = qkv[:, 2 * d:].reshape(n, H, hd)
+        q = _st(rope(qkv[:, :d].reshape(n, H, hd), pos, theta), store)
+        k = _st(rope(qkv[:, d:2 * d].reshape(n, H, hd), pos, theta), store)
+        v = _st(qkv[:, 2 * d:].reshape(n, H, hd), store)
         kv.k[l, ctx:ctx + n] = k
         kv.v[l, ctx:ctx + n] = v
         attn = np.zeros((n, H, hd), dtype=dtype)
@@ -222,51 +257,52 @@ def llm_forward(W, cfg, tokens, pos, mask, kv, ctx, dtype=F, want_logits=True):
             sc = np.einsum("hd,khd->hk", q[r], kk) * scale              # [H, keys]
             sc = sc - sc.max(axis=1, keepdims=True)
             p = np.exp(sc)
-            p = p / p.sum(axis=1, keepdims=True)
-            attn[r] = np.einsum("hk,khd->hd", p, vv)
-        x = x + attn.reshape(n, d) @ _c(W["wo"][l], dtype).T
-        f = rmsnorm(x, _c(W["ffn_norm"][l], dtype), eps)
+            # softmax(sc) V as (p V) / sum(p): the stored copy of p multiplies V, the sum is exact
+            attn[r] = np.einsum("hk,khd->hd", _st(p, store), vv) / p.sum(axis=1, keepdims=True)
+        x = x + _st(attn.reshape(n, d), store) @ _c(W["wo"][l], dtype).T
+        f = _st(rmsnorm(x, _c(W["ffn_norm"][l], dtype), eps), store)
         gu = f @ _c(W["w_gate_up"][l], dtype).T                      # [n, 2F]: gate rows then up rows
         Fd = cfg["d_ffn"]
-        act = silu(gu[:, :Fd]) * gu[:, Fd:]
+        act = _st(silu(gu[:, :Fd]) * gu[:, Fd:], store)
         x = x + act @ _c(W["w_down"][l], dtype).T
     hidden = rmsnorm(x, _c(W["final_norm"], dtype), eps)
-    logits = hidden @ _c(W["lm_head"], dtype).T if want_logits else None
+    logits = _st(hidden, store) @ _c(W["lm_head"], dtype).T if want_logits else None
     return hidden, logits
 
 
-def prefill(W, cfg, prompt, kv, dtype=F, sampling=None, seq=0):
+def prefill(W, cfg, prompt, kv, dtype=F, sampling=None, seq=0, store=None):
     """Causal forward over the prompt.  Returns (ctx, root token g, h)."""
     P = len(prompt)
     mask = np.tril(np.ones((P, P), dtype=bool))
-    hidden, _ = llm_forward(W, cfg, prompt, np.arange(P), mask, kv, 0, dtype, want_logits=False)
-    logits_last = hidden[P - 1] @ _c(W["lm_head"], dtype).T
+    hidden, _ = llm_forward(W, cfg, prompt, np.arange(P), mask, kv, 0, dtype, want_logits=False, store=store)
+    logits_last = _st(hidden[P - 1], store) @ _c(W["lm_head"], dtype).T
     return P, choose_token(logits_last, sampling, seq, P), hidden[P - 1].copy()
 
 
-def ar_step(W, cfg, kv, ctx, g, dtype=F, sampling=None, seq=0):
+def ar_step(W, cfg, kv, ctx, g, dtype=F, sampling=None, seq=0, store=None):
     """One plain autoregressive step: feed g at position ctx, return next token, h, logits."""
-    hidden, logits = llm_forward(W, cfg, [g], [ctx], np.ones((1, 1), bool), kv, ctx, dtype)
+    hidden, logits = llm_forward(W, cfg, [g], [ctx], np.ones((1, 1), bool), kv, ctx, dtype, store=store)
     return choose_token(logits[0], sampling, seq, ctx + 1), hidden[0].copy(), logits[0]
 
 
 # ----------------------------------------------------------------------------
 # drafter (Sections 3.1 and 3.2)
 # ----------------------------------------------------------------------------
-def rnn_cell(D, s_prev, e, dtype=F):
+def rnn_cell(D, s_prev, e, dtype=F, store=None):
     """s_t = f(U s_{t-1} + W e_t + b) (Section 3.1)."""
-    return silu(_c(D["rnn_u"], dtype) @ s_prev + _c(D["rnn_w"], dtype) @ e + _c(D["rnn_b"], dtype))
+    return silu(_c(D["rnn_u"], dtype) @ _st(s_prev, store) + _c(D["rnn_w"], dtype) @ _st(e, store) + _c(D["rnn_b"], dtype))
 
 
-def draft_head(D, g_t, dtype=F):
-    """MLP layers with skip connections, then the vocabulary projection (Section 3.1).  Returns logits."""
+def draft_head(D, g_t, dtype=F, store=None):
+    """MLP layers with skip connections, then the vocabulary projection (Section 3.1).  Returns logits.
+    store="bf16": each projection reads a rounded copy of x; the skip path keeps x itself."""
     x = g_t
     for A, c in zip(D["head_w"], D["head_b"]):
-        x = x + silu(_c(A, dtype) @ x + _c(c, dtype))
-    return _c(D["draft_out"], dtype) @ x
+        x = x + silu(_c(A, dtype) @ _st(x, store) + _c(c, dtype))
+    return _c(D["draft_out"], dtype) @ _st(x, store)
 
 
-def beam_search(D, E, g, h, beam_width, beam_length, dtype=F, return_logp=False):
+def beam_search(D, E, g, h, beam_width, beam_length, dtype=F, return_logp=False, store=None):
     """Beam search over the drafter (Section 3.2).
 
     Returns beams [BW, L] (int64), scores [BW]: candidates sorted by cumulative
@@ -278,7 +314,7 @@ def beam_search(D, E, g, h, beam_width, beam_length, dtype=F, return_logp=False)
     E = _c(E, dtype)
     h = np.asarray(h, dtype=dtype)
     s1 = E[g]
-    logp = log_softmax(draft_head(D, np.concatenate([s1, h]), dtype))
+    logp = log_softmax(draft_head(D, np.concatenate([s1, h]), dtype, store))
     top = top_k_ordered(logp, beam_width)
     hist = [[int(v)] for v in top]
     scores = logp[top].copy()
@@ -288,9 +324,9 @@ def beam_search(D, E, g, h, beam_width, beam_length, dtype=F, return_logp=False)
         cand = np.empty(beam_width * V, dtype=dtype)
         new_states = []
         for b in range(beam_width):
-            s = rnn_cell(D, states[b], E[hist[b][-1]], dtype)
+            s = rnn_cell(D, states[b], E[hist[b][-1]], dtype, store)
             new_states.append(s)
-            lp = log_softmax(draft_head(D, np.concatenate([s, h]), dtype))
+            lp = log_softmax(draft_head(D, np.concatenate([s, h]), dtype, store))
             cand[b * V:(b + 1) * V] = scores[b] + lp
         top = top_k_ordered(cand, beam_width)
         cand_log.append(cand)
@@ -303,15 +339,15 @@ def beam_search(D, E, g, h, beam_width, beam_length, dtype=F, return_logp=False)
     return beams, scores
 
 
-def sequence_logprob(D, E, g, h, seq, dtype=F):
+def sequence_logprob(D, E, g, h, seq, dtype=F, store=None):
     """log p_draft(seq | g, h): the drafter run along one fixed sequence."""
     E = _c(E, dtype)
     s = E[g]
     total = 0.0
     for t, tok in enumerate(seq):
         if t > 0:
-            s = rnn_cell(D, s, E[seq[t - 1]], dtype)
-        lp = log_softmax(draft_head(D, np.concatenate([s, np.asarray(h, dtype=dtype)]), dtype))
+            s = rnn_cell(D, s, E[seq[t - 1]], dtype, store)
+        lp = log_softmax(draft_head(D, np.concatenate([s, np.asarray(h, dtype=dtype)]), dtype, store))
         total += lp[tok]
     return total
 
@@ -440,7 +476,7 @@ def compact_kv(kv, ctx, unpack, best, a):
 # the whole step (Section 3.4) for one sequence
 # ----------------------------------------------------------------------------
 def spec_step(W, D, cfg, kv, ctx, g, h, beam_width, beam_length, planted=None,
-              tree=True, dtype=F, run_drafter=True, sampling=None, seq=0):
+              tree=True, dtype=F, run_drafter=True, sampling=None, seq=0, store=None):
     """One speculative decode step.  Returns a dict with every intermediate.
 
     planted: optional [BW, L] beams used in place of the drafter's (the drafter
@@ -448,13 +484,13 @@ def spec_step(W, D, cfg, kv, ctx, g, h, beam_width, beam_length, planted=None,
     """
     out = {}
     if run_drafter or planted is None:
-        beams, scores = beam_search(D, W["tok_emb"], g, h, beam_width, beam_length, dtype)
+        beams, scores = beam_search(D, W["tok_emb"], g, h, beam_width, beam_length, dtype, store=store)
         out["drafted_beams"], out["scores"] = beams, scores
     if planted is not None:
         beams = np.asarray(planted, dtype=np.int64)
     beam_aug = np.concatenate([np.full((beams.shape[0], 1), g, dtype=np.int64), beams], axis=1)
     packed = pack_beam(beam_aug, ctx) if tree else flat_beam(beam_aug, ctx)
-    hidden, logits = llm_forward(W, cfg, packed["tokens"], packed["pos"], packed["mask"], kv, ctx, dtype)
+    hidden, logits = llm_forward(W, cfg, packed["tokens"], packed["pos"], packed["mask"], kv, ctx, dtype, store=store)
     am = choose_rows(logits, packed["pos"], sampling, seq)
     a, best, emitted = accept_greedy(beams, packed["unpack"], am)
     node = int(packed["unpack"][best, a])
@@ -465,13 +501,13 @@ def spec_step(W, D, cfg, kv, ctx, g, h, beam_width, beam_length, planted=None,
     return out
 
 
-def generate_ar(W, cfg, prompt, n_tokens, max_ctx, dtype=F, sampling=None, seq=0):
+def generate_ar(W, cfg, prompt, n_tokens, max_ctx, dtype=F, sampling=None, seq=0, store=None):
     """Plain decoding (greedy, or sampled): the definition the speculative path must reproduce."""
     kv = KVCache(cfg["n_layers"], max_ctx, cfg["n_heads"], cfg["d_model"] // cfg["n_heads"], dtype)
-    ctx, g, h = prefill(W, cfg, prompt, kv, dtype, sampling, seq)
+    ctx, g, h = prefill(W, cfg, prompt, kv, dtype, sampling, seq, store)
     out = [g]
     while len(out) < n_tokens:
-        nxt, h, _ = ar_step(W, cfg, kv, ctx, g, dtype, sampling, seq)
+        nxt, h, _ = ar_step(W, cfg, kv, ctx, g, dtype, sampling, seq, store)
         ctx += 1
         g = nxt
         out.append(g)
@@ -479,16 +515,16 @@ def generate_ar(W, cfg, prompt, n_tokens, max_ctx, dtype=F, sampling=None, seq=0
 
 
 def generate_spec(W, D, cfg, prompt, n_steps, beam_width, beam_length, max_ctx,
-                  planted_fn=None, tree=True, dtype=F, sampling=None, seq=0):
+                  planted_fn=None, tree=True, dtype=F, sampling=None, seq=0, store=None):
     """Speculative decoding for n_steps.  planted_fn(step, ctx, g) -> beams or None."""
     kv = KVCache(cfg["n_layers"], max_ctx, cfg["n_heads"], cfg["d_model"] // cfg["n_heads"], dtype)
-    ctx, g, h = prefill(W, cfg, prompt, kv, dtype, sampling, seq)
+    ctx, g, h = prefill(W, cfg, prompt, kv, dtype, sampling, seq, store)
     out = [g]
     accepted = []
     for step in range(n_steps):
         planted = planted_fn(step, len(out), g) if planted_fn is not None else None
         r = spec_step(W, D, cfg, kv, ctx, g, h, beam_width, beam_length, planted, tree, dtype,
-                      run_drafter=planted is None, sampling=sampling, seq=seq)
+                      run_drafter=planted is None, sampling=sampling, seq=seq, store=store)
         ctx, g, h = r["ctx"], r["g"], r["h"]
         out.extend(r["emitted"])
         accepted.append(r["n_accept"])

@@ -7,7 +7,11 @@ packing bit-exact, verification logits within the bf16 bound, greedy tokens wher
 decides them, acceptance + hand-off bit-exact against the oracle's rule on the GPU's own greedy tokens.
 
 The `*_full_depth` cases run the same step at the workloads' own depth (40, 32 and 60 layers) with prompts of a few
-dozen tokens, the oracle following one or two of the sequences, and a bound scaled to the depth (full_depth_bound).
+dozen tokens, the oracle following one or two of the sequences.  Every case is held to the stated 3e-2 against the
+oracle that applies the path's bf16 storage points (store="bf16": projection inputs, Q, K, V and the softmax weights
+rounded element by element).  The two-layer cases also meet it against the unrounded oracle; at full depth that
+distance is printed and only sanity-bounded, because the storage noise alone grows as the square root of the depth
+(tests/test_oracle_storage.py measures it between the two oracle modes, without any kernel).
 """
 import numpy as np
 import pytest
@@ -31,43 +35,22 @@ def decided(ref_logits, rel=REL):
     return top2_gap(ref_logits) > np.maximum(0.05, 2 * bound)
 
 
-def full_depth_bound(n_layers):
-    """Bound on a row's relative L2 error of logits and hidden states at a workload's own depth.
-
-    The bf16 path rounds every projection input and the KV cache to bf16, the fp32 oracle does not; the noise of the
-    layers is independent and adds up as the square root of the depth, slowly amplified on its way up by the
-    random-init layers.  Measured relative L2 error of the logits / sqrt(depth), mean over the rows:
-      7B shape   0.81e-2 (1 layer)  0.77e-2 (2)  0.72e-2 (8)   0.73e-2 (32)
-      13B shape               0.74e-2 (2)  0.75e-2 (8)   0.80e-2 (20)  0.83e-2 (40)
-      33B shape  0.86e-2 (1)  0.86e-2 (2)  0.95e-2 (8)   1.06e-2 (30)  1.2e-2 (60; worst row 1.3e-2)
-    Returned: 1.6e-2 x sqrt(depth); a single element (the worst of up to a million) is allowed twice as much.  An
-    error in a kernel (a dropped term, a wrong row or key) shows as an error of order one at any depth; the two-layer
-    cases above hold the same kernels to 3e-2."""
-    return 1.6e-2 * np.sqrt(n_layers)
-
-
 def rel_l2(got, ref):
     return float((np.linalg.norm(got - ref, axis=-1) / np.linalg.norm(ref, axis=-1)).max())
 
 
-def close(got, ref, rel, full_depth):
-    if not full_depth:
-        assert rel_err(got, ref) < rel
-    else:
-        l2, mx = rel_l2(got, ref), rel_err(got, ref)
-        assert l2 < rel and mx < 2 * rel, (l2, mx, rel)
-    return True
+SANITY_PLAIN = 0.05     # x sqrt(depth / 8): a loose bound on the distance to the unrounded oracle at full depth
 
 
 def one_step(name, prompt_lens, check_seqs, rho, layers=2):
-    """layers=None: the workload's own depth, with the bound scaled to it."""
+    """layers=None: the workload's own depth."""
     base = synth.CONFIGS[name]
     B = len(prompt_lens)
     cfg = dict(base, max_batch=B, max_ctx=max(prompt_lens) + 2 + base["beam_width"] * base["beam_length"] + 8)
     if layers is not None:
         cfg = synth.with_layers(cfg, layers)
     full = layers is None
-    REL = 3e-2 if not full else full_depth_bound(cfg["n_layers"])
+    tag = f"[{name}, {cfg['n_layers']} layers]"
     rig = Rig(cfg=cfg, oracle_dtype=np.float32)
     BW, L, V = cfg["beam_width"], cfg["beam_length"], cfg["vocab"]
     rng = np.random.default_rng(cfg["seed"])
@@ -82,12 +65,18 @@ def one_step(name, prompt_lens, check_seqs, rho, layers=2):
     refs = {}
     for b in check_seqs:
         kv = rig.new_kv()
-        ctx, g, h = ora.prefill(rig.W, cfg, prompts[b], kv, np.float32)
+        ctx, g, h = ora.prefill(rig.W, cfg, prompts[b], kv, np.float32, store="bf16")
+        kv_plain = rig.new_kv()
+        _, _, h_plain = ora.prefill(rig.W, cfg, prompts[b], kv_plain, np.float32)
         assert int(c_ctx[b]) == ctx
-        assert close(hs[b][None], np.asarray(h)[None], REL, full)
+        print(f"{tag} sequence {b}, h after the prompt: {rel_err(hs[b][None], np.asarray(h)[None]):.4f} of the max against "
+              f"the oracle with bf16 storage, {rel_err(hs[b][None], np.asarray(h_plain)[None]):.4f} against the unrounded oracle")
+        assert rel_err(hs[b][None], np.asarray(h)[None]) < REL
+        if not full:
+            assert rel_err(hs[b][None], np.asarray(h_plain)[None]) < REL
         roots[b] = g                                    # teacher-force the oracle's root and hidden state
         hs[b] = h
-        refs[b] = (kv, ctx, g, h)
+        refs[b] = (kv, ctx, g, h, kv_plain)
     rig.eng.set_state(None, dev(roots), dev(hs.astype(np.float32), torch.float32))
     beams_d = dev(beams)
     pk = rig.eng.pack(beams_d)
@@ -95,7 +84,7 @@ def one_step(name, prompt_lens, check_seqs, rho, layers=2):
     out = rig.eng.accept(beams_d, pk, argmax, hidden)
     rig.eng.poll()
     n_ctx, n_root, n_h = rig.eng.get_state()
-    for b, (kv, ctx, g, h) in refs.items():
+    for b, (kv, ctx, g, h, kv_plain) in refs.items():
         aug = np.concatenate([np.full((BW, 1), g), beams[b]], axis=1)
         p = ora.pack_beam(aug, ctx)
         n = p["n"]
@@ -104,11 +93,20 @@ def one_step(name, prompt_lens, check_seqs, rho, layers=2):
         assert pk.unpack[b].cpu().numpy().tolist() == p["unpack"].tolist()
         assert pk.pos[b, :n].tolist() == p["pos"].tolist()
         assert (pk.mask_bool(b) == p["mask"]).all()
-        rh, rl = ora.llm_forward(rig.W, cfg, p["tokens"], p["pos"], p["mask"], kv, ctx, np.float32)
-        assert close(logits[b, :n].cpu().numpy(), rl, REL, full)
-        assert close(hidden[b, :n].cpu().numpy(), rh, REL, full)
+        rh, rl = ora.llm_forward(rig.W, cfg, p["tokens"], p["pos"], p["mask"], kv, ctx, np.float32, store="bf16")
+        _, rl_plain = ora.llm_forward(rig.W, cfg, p["tokens"], p["pos"], p["mask"], kv_plain, ctx, np.float32)
+        got = logits[b, :n].cpu().numpy()
+        print(f"{tag} sequence {b}, verification logits: {rel_err(got, rl):.4f} of the row's max (worst row's relative L2 "
+              f"{rel_l2(got, rl):.4f}) against the oracle with bf16 storage, {rel_err(got, rl_plain):.4f} ({rel_l2(got, rl_plain):.4f}) "
+              f"against the unrounded oracle")
+        assert rel_err(got, rl) < REL
+        assert rel_err(hidden[b, :n].cpu().numpy(), rh) < REL
+        if full:
+            assert rel_err(got, rl_plain) < SANITY_PLAIN * np.sqrt(cfg["n_layers"] / 8)
+        else:
+            assert rel_err(got, rl_plain) < REL
         am = argmax[b, :n].cpu().numpy()
-        sure = decided(rl, 2 * REL if full else REL)
+        sure = decided(rl)
         assert (am[sure] == rl.argmax(1)[sure]).all()
         a, best, toks = ora.accept_greedy(beams[b], p["unpack"], am)
         assert int(out.n_accept[b]) == a and int(out.best[b]) == best

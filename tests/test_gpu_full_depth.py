@@ -8,12 +8,14 @@ the oracle's gap decides them, and acceptance + hand-off bit-exact against the o
 own greedy tokens.  The beams of the verified step are planted from the GPU's own autoregressive continuation (an
 input recipe, not an expected value), so that several tokens are accepted.
 
-Tolerance.  The bf16 path rounds every projection input and the KV cache to bf16 (relative step 2^-8); the oracle
-does not.  That rounding noise is independent from layer to layer and, with random-init weights, is neither damped
-nor amplified much on its way up, so it grows as the square root of the depth: measured relative L2 error of the
-logits at this shape 0.8e-2 (1 layer), 1.1e-2 (2), 1.5e-2 (4), 2.0e-2 (8), 2.9e-2 (16), 4.1e-2 (32), i.e.
-0.8e-2 x sqrt(depth); the worst row's max |error| / max |logit| is 1.5e-2 at two layers and 4.8e-2 at 32.  The
-3e-2 bound of the depth-reduced parity cases therefore becomes 0.8e-2 x sqrt(32) x 1.5 = 7e-2 here.
+Tolerance.  The bf16 path stores every projection input, Q, K, V and the softmax weights that multiply V in bf16
+(relative step 2^-8).  That storage is part of the path's definition, and the oracle can apply it (store="bf16":
+the same arrays rounded element by element, nothing else changed); against that oracle the stated bound of 3e-2 of
+the row's largest |logit| holds at the full 32 layers and is what this case asserts.  The distance to the UNROUNDED
+oracle is printed, not bounded by 3e-2: the storage noise of the layers is independent and grows as the square
+root of the depth, 0.7e-2 after one layer and 1.6e-2 after eight between the two oracle modes on the CPU
+(tests/test_oracle_storage.py), about 3e-2 for the average row at 32 layers and more for the worst element of the
+worst row.  It is only held to a loose sanity bound here.
 """
 import numpy as np
 import pytest
@@ -25,7 +27,8 @@ from paper_2403_09919_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
-REL = 7e-2   # 0.8e-2 x sqrt(32 layers) x 1.5: see the module docstring
+REL = 3e-2          # against the oracle with the path's bf16 storage points
+SANITY_PLAIN = 0.12  # against the unrounded oracle: reported; four times the two-mode distance the CPU test extrapolates
 
 
 def rel_err(got, ref):
@@ -56,11 +59,15 @@ def test_one_step_of_the_7b_workload_at_full_depth():
     # state after the prompt
     rig.eng.prefill([prompt])
     kv = rig.new_kv()
-    ctx, g, h = ora.prefill(rig.W, cfg, prompt, kv, rig.odt)
+    ctx, g, h = ora.prefill(rig.W, cfg, prompt, kv, rig.odt, store="bf16")
+    kv_plain = rig.new_kv()
+    _, _, h_plain = ora.prefill(rig.W, cfg, prompt, kv_plain, rig.odt)
     c_ctx, c_root, c_h = rig.eng.get_state()
     rig.eng.poll()
     assert int(c_ctx[0]) == ctx == 32
     assert rel_err(c_h[0].cpu().numpy()[None], np.asarray(h)[None]) < REL
+    figures = {"h after the prompt": (rel_err(c_h[0].cpu().numpy()[None], np.asarray(h)[None]),
+                                      rel_err(c_h[0].cpu().numpy()[None], np.asarray(h_plain)[None]))}
     logits_last = np.asarray(h, dtype=np.float64) @ np.asarray(rig.W["lm_head"], dtype=np.float64).T
     if decided(logits_last[None])[0]:
         assert int(c_root[0]) == g
@@ -74,13 +81,17 @@ def test_one_step_of_the_7b_workload_at_full_depth():
     sc = scores[0].cpu().numpy()
     assert (np.diff(sc) <= 0).all()
     for i in (0, BW - 1):
-        ref = ora.sequence_logprob(rig.D, rig.W["tok_emb"], g, h, beams[0, i].cpu().numpy(), rig.odt)
+        ref = ora.sequence_logprob(rig.D, rig.W["tok_emb"], g, h, beams[0, i].cpu().numpy(), rig.odt, store="bf16")
         assert abs(ref - sc[i]) < REL * abs(ref)
 
     # one verified step on planted beams
     rng = np.random.default_rng(41)
     planted = synth.plant_beams(cont, BW, L, cfg["vocab"], rng, p=0.3, rho=0.3)
-    ref = ora.spec_step(rig.W, rig.D, cfg, kv, ctx, g, h, BW, L, planted=planted, run_drafter=False, dtype=rig.odt)
+    ref = ora.spec_step(rig.W, rig.D, cfg, kv, ctx, g, h, BW, L, planted=planted, run_drafter=False, dtype=rig.odt,
+                        store="bf16")
+    # the unrounded oracle on the same rows, from its own cache but the same root and hidden state: a reported figure
+    ref_plain = ora.spec_step(rig.W, rig.D, cfg, kv_plain, ctx, g, h, BW, L, planted=planted, run_drafter=False,
+                              dtype=rig.odt)
     beams_d = dev(planted[None])
     pk = rig.eng.pack(beams_d)
     argmax, hidden, logits = rig.eng.verify(pk, want_logits=True)
@@ -91,8 +102,17 @@ def test_one_step_of_the_7b_workload_at_full_depth():
     assert pk.tokens[0, :n].tolist() == ref["packed"]["tokens"].tolist()
     assert pk.unpack[0].cpu().numpy().tolist() == ref["packed"]["unpack"].tolist()
     assert (pk.mask_bool(0) == ref["packed"]["mask"]).all()
-    assert rel_err(logits[0, :n].cpu().numpy(), ref["logits"]) < REL
+    got = logits[0, :n].cpu().numpy()
+    figures["verification logits"] = (rel_err(got, ref["logits"]), rel_err(got, ref_plain["logits"]))
+    figures["verification logits, relative L2 of the worst row"] = (
+        float((np.linalg.norm(got - ref["logits"], axis=1) / np.linalg.norm(ref["logits"], axis=1)).max()),
+        float((np.linalg.norm(got - ref_plain["logits"], axis=1) / np.linalg.norm(ref_plain["logits"], axis=1)).max()))
+    for what, (r_store, r_plain) in figures.items():
+        print(f"[7B, 32 layers] {what}: {r_store:.4f} of the row's max against the oracle with bf16 storage, "
+              f"{r_plain:.4f} against the unrounded oracle")
+    assert rel_err(got, ref["logits"]) < REL
     assert rel_err(hidden[0, :n].cpu().numpy(), ref["hidden"]) < REL
+    assert rel_err(got, ref_plain["logits"]) < SANITY_PLAIN
     am = argmax[0, :n].cpu().numpy()
     sure = decided(ref["logits"])
     assert (am[sure] == ref["argmax"][sure]).all()
