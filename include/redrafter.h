@@ -275,6 +275,31 @@ RD_API int redrafter_selftest_wait(rd_handle* h, void* stream);
 /* Number of kernels this handle has launched since it was created (for launch accounting). */
 RD_API int64_t redrafter_launch_count(const rd_handle* h);
 
+/* Diagnostic (the paper has no counterpart): copies rows [0, rows) of the logits computed by the handle's last
+ * forward pass into the DEVICE buffer out[rows][vocab] (fp32), enqueued on `stream`.  After redrafter_ar_step row b
+ * is sequence b's next-token logits; after redrafter_verify / redrafter_step the rows are the packed rows of all
+ * sequences back to back.  rows must not exceed max_batch * (1 + beam_width * beam_length): RD_ERR_INVALID_ARG. */
+RD_API int redrafter_last_logits(rd_handle* h, void* stream, float* out, int32_t rows);
+
+/* Which kernel variants the handle's attention and projection launches have taken since it was created (the paper
+ * has no counterpart: Section 3.4's verification pass is one attention over the cache plus the tree mask, and this
+ * library picks among several kernels for it by row count and context length).  Fills the HOST array out[0 .. n-1],
+ * n <= RD_ROUTE_COUNT, with launch counts; tests use it to check that a workload exercises the kernel it is meant
+ * to.  Never touches the device. */
+enum {
+  RD_ROUTE_ATT_ROWS16 = 0,        /* 16-row tiles, four-chunk ring (decode steps) */
+  RD_ROUTE_ATT_ROWS16_SHALLOW = 1,/* 16-row tiles, two-chunk ring (more tiles than SMs) */
+  RD_ROUTE_ATT_ROWS64 = 2,        /* 64-row tiles */
+  RD_ROUTE_ATT_ROWS128_TC5 = 3,   /* 128-row tiles on tcgen05 */
+  RD_ROUTE_ATT_KEY_SPLIT = 4,     /* of the 16-row launches: those whose keys were split over several CTAs */
+  RD_ROUTE_ATT_FP32 = 5,          /* the fp32 configuration's kernel */
+  RD_ROUTE_GEMM_PAIRS = 6,        /* projections on CTA pairs */
+  RD_ROUTE_GEMM_ONE_CTA = 7,      /* projections on single CTAs (tensor cores) */
+  RD_ROUTE_GEMM_SIMT = 8,         /* projections on CUDA cores */
+  RD_ROUTE_COUNT = 9
+};
+RD_API int redrafter_route_counts(const rd_handle* h, int64_t* out, int32_t n);
+
 #ifdef __cplusplus
 }
 #endif

@@ -26,7 +26,10 @@ EXPORTS = ["redrafter_workspace_bytes", "redrafter_kv_bytes", "redrafter_init", 
            "redrafter_accept", "redrafter_step", "redrafter_ar_step", "redrafter_get_state", "redrafter_set_state",
            "redrafter_set_ctx_bound", "redrafter_poll", "redrafter_launch_count", "redrafter_profile",
            "redrafter_profile_read", "redrafter_trace", "redrafter_trace_read", "redrafter_trace_bytes",
-           "redrafter_accept_static", "redrafter_selftest_wait", "redrafter_set_sampling"]
+           "redrafter_accept_static", "redrafter_selftest_wait", "redrafter_set_sampling", "redrafter_route_counts", "redrafter_last_logits"]
+
+ROUTES = ("att_rows16", "att_rows16_shallow", "att_rows64", "att_rows128_tc5", "att_key_split", "att_fp32", "gemm_pairs",
+          "gemm_one_cta", "gemm_simt")
 
 
 class RdConfig(C.Structure):
@@ -92,6 +95,8 @@ def lib():
         L.redrafter_trace_read.argtypes = [vp, vp, vp, i32]
         L.redrafter_trace_bytes.argtypes = [vp, vp, i32]
         L.redrafter_selftest_wait.argtypes = [vp, vp]
+        L.redrafter_last_logits.argtypes = [vp, vp, vp, i32]
+        L.redrafter_route_counts.argtypes = [vp, C.POINTER(C.c_int64), i32]
         _lib = L
     return _lib
 
@@ -324,6 +329,18 @@ class ReDrafter:
         if n < 0:
             self._ck(-n)
         return buf[:n]
+
+    def last_logits(self, rows):
+        """[rows, V] fp32 logits of the last forward pass (device tensor)."""
+        out = torch.empty(rows, self.V, dtype=torch.float32, device=self.device)
+        self._ck(self.L.redrafter_last_logits(self.h, _stream(), _ptr(out), rows))
+        return out
+
+    def route_counts(self):
+        """Launches per kernel variant since the handle was made: dict keyed by ROUTES."""
+        buf = (C.c_int64 * len(ROUTES))()
+        self._ck(self.L.redrafter_route_counts(self.h, buf, len(ROUTES)))
+        return dict(zip(ROUTES, list(buf)))
 
     def launch_count(self):
         return int(self.L.redrafter_launch_count(self.h))

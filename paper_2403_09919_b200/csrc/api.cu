@@ -85,6 +85,7 @@ struct rd_handle {
   int ctx_bound;  // host-side upper bound of every sequence's context length
   Sampling sampling;  // how the LLM's tokens are chosen (inv_t = 0: greedy)
   int64_t launches;
+  int64_t route[RD_ROUTE_COUNT];  // launches per kernel variant (redrafter_route_counts)
   // tensor-core path (bf16): TMA descriptors by base pointer, launch geometry
   bool use_tc;
   int trace_next;  // next trace slot, -1 = tracing off
@@ -297,9 +298,11 @@ int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, cons
     }
     CK(h, launch_gemm_tc(&iw->second, amaps, N, K, m_total, m_max, raw, ld_raw, h->ws.tc_partial, h->ws.status,
                          h->tc_grid, pairs, h->tc_smem, tr, out, chain, pair, st));
+    h->route[pairs ? RD_ROUTE_GEMM_PAIRS : RD_ROUTE_GEMM_ONE_CTA]++;
     return RD_OK;
   }
   if (chain) chain->cut();
+  h->route[RD_ROUTE_GEMM_SIMT]++;
   CK(h, launch_gemm_simt(h->dm.dtype, A, lda, W, N, K, m_total, m_max, raw, ld_raw, out, st));
   return RD_OK;
 }
@@ -364,6 +367,9 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
                                      m_max, w.status, ch, st));
     {
       ProfScope ps(h, 1, 0.0, st);
+      h->route[!h->use_tc ? RD_ROUTE_ATT_FP32 : att_t5 ? RD_ROUTE_ATT_ROWS128_TC5 : att_wide ? RD_ROUTE_ATT_ROWS64
+               : att_shallow ? RD_ROUTE_ATT_ROWS16_SHALLOW : RD_ROUTE_ATT_ROWS16]++;
+      if (h->use_tc && !att_t5 && !att_wide && n_splits > 1) h->route[RD_ROUTE_ATT_KEY_SPLIT]++;
       if (h->use_tc && att_t5)
         CK(h, launch_attention_t5(h->kv_maps[(size_t)l * 2].bytes, h->kv_maps[(size_t)l * 2 + 1].bytes, w.qkv, w.attn_t, rt, w.seq_off, dm, n_seq,
                                   row_blocks, w.status, ch, st));
@@ -586,6 +592,7 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
     if (!ok) return init_fail(h, RD_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d for operand %p", failed_rc, failed_ptr);
   }
   h->prefilled = false; h->batch = dm.B; h->ctx_bound = 0; h->launches = 0; h->err[0] = 0;
+  for (int i = 0; i < RD_ROUTE_COUNT; ++i) h->route[i] = 0;
   h->sampling = Sampling{0.0f, 0u, 0u};
   h->profiling = false;
   h->trace_next = -1;
@@ -620,6 +627,19 @@ int redrafter_destroy(rd_handle* h) {
 const char* redrafter_last_error(const rd_handle* h) { return h ? h->err : g_init_err; }
 
 int64_t redrafter_launch_count(const rd_handle* h) { return h ? h->launches : 0; }
+
+int redrafter_last_logits(rd_handle* h, void* stream, float* out, int32_t rows) {
+  if (!h || !out || rows <= 0 || rows > h->dm.B * h->dm.NMAX) return RD_ERR_INVALID_ARG;
+  CKRT(h, cudaMemcpyAsync(out, h->ws.logits, (size_t)rows * h->dm.V * sizeof(float), cudaMemcpyDeviceToDevice,
+                          (cudaStream_t)stream));
+  return RD_OK;
+}
+
+int redrafter_route_counts(const rd_handle* h, int64_t* out, int32_t n) {
+  if (!h || !out || n < 0 || n > RD_ROUTE_COUNT) return RD_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i) out[i] = h->route[i];
+  return RD_OK;
+}
 
 static int set_row_counts(rd_handle* h, cudaStream_t st) {
   CK(h, launch_fill_i32(h->ws.one_b, h->batch, 1, st));

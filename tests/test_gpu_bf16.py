@@ -9,13 +9,14 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import Rig, dev, top2_gap
+from helpers import Rig, check_beams_within, dev, tolerant_beam_search, top2_gap
 from oracle import redrafter_oracle as ora
 from paper_2403_09919_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
 REL = 3e-2
+EPS_SCORE = 2e-3     # drafter scores against the oracle with bf16 storage: measured 5.7e-4 (tests/test_gpu_drafter_beams.py)
 
 # shapes that are NOT multiples of the 128 x 64 tiles: vocabulary 1000, d_ffn 1376
 RAGGED = dict(synth.CONFIGS["tiny"], dtype="bf16", d_model=512, n_heads=4, d_ffn=1376, vocab=1000, d_rnn=512,
@@ -153,22 +154,16 @@ def test_draft_scores_ragged():
     rig.eng.set_state(None, dev([g]), dev(np.asarray(h, dtype=np.float32)[None], torch.float32))
     beams, scores = rig.eng.draft()
     rig.eng.poll()
-    rb, rs, cand = ora.beam_search(rig.D, rig.W["tok_emb"], g, h, 8, 5, rig.odt, return_logp=True)
     sc = scores[0].cpu().numpy()
     assert (np.diff(sc) <= 0).all()
     # each returned score is the drafter's log-probability of that sequence (within the bf16 bound)
     for b, s in zip(beams[0].cpu().numpy(), sc):
         assert abs(ora.sequence_logprob(rig.D, rig.W["tok_emb"], g, h, b, rig.odt) - s) < REL * abs(s)
-    # and the beam is as good as the oracle's: best score and total mass agree within the bound
-    assert abs(sc[0] - rs[0]) < REL * abs(rs[0])
-    assert abs(sc.sum() - rs.sum()) < REL * abs(rs.sum())
-    # identical beams when every candidate decision of the oracle is clear of the bound
-    clear = True
-    for c in cand:
-        s = np.sort(c)[::-1][:9]
-        clear = clear and (np.diff(s) < -2 * REL).all()
-    if clear:
-        assert beams[0].cpu().numpy().tolist() == rb.tolist()
+    # the beams themselves, against the oracle with the path's bf16 storage and every decision widened by the score
+    # error bound (tests/test_gpu_drafter_beams.py derives it): no certain beam missing, none that is ruled out
+    sets = tolerant_beam_search(ora, rig.D, rig.W["tok_emb"], g, np.asarray(h, np.float32).astype(np.float64), 8, 5, EPS_SCORE, store="bf16")
+    check_beams_within(sets, beams[0].cpu().numpy(), sc, EPS_SCORE)
+    assert len(sets[0]) >= 4
 
 
 def test_wide_beam_two_row_tiles():
@@ -402,19 +397,13 @@ def test_draft_scores_wide_beams(bw):
     rig.eng.set_state(None, dev([g]), dev(np.asarray(h, dtype=np.float32)[None], torch.float32))
     beams, scores = rig.eng.draft()
     rig.eng.poll()
-    rb, rs, cand = ora.beam_search(rig.D, rig.W["tok_emb"], g, h, bw, 5, rig.odt, return_logp=True)
     sc = scores[0].cpu().numpy()
     bm = beams[0].cpu().numpy()
     assert (np.diff(sc) <= 0).all()
     assert len({tuple(b) for b in bm.tolist()}) == bw                      # distinct sequences
     for i in (0, 1, bw // 2, bw - 1):
         assert abs(ora.sequence_logprob(rig.D, rig.W["tok_emb"], g, h, bm[i], rig.odt) - sc[i]) < REL * abs(sc[i])
-    assert abs(sc[0] - rs[0]) < REL * abs(rs[0])
-    assert abs(sc.sum() - rs.sum()) < REL * abs(rs.sum())
-    clear = True
-    for c in cand:
-        s = np.sort(c)[::-1][:bw + 1]
-        clear = clear and (np.diff(s) < -2 * REL).all()
-    if clear:
-        assert bm.tolist() == rb.tolist()
+    sets = tolerant_beam_search(ora, rig.D, rig.W["tok_emb"], g, np.asarray(h, np.float32).astype(np.float64), bw, 5, EPS_SCORE, store="bf16")
+    check_beams_within(sets, bm, sc, EPS_SCORE)
+    assert len(sets[0]) >= bw // 2
     rig.eng.close()

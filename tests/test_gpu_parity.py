@@ -14,9 +14,10 @@ pytestmark = pytest.mark.gpu
 
 GAP = 0.05
 TOL_FP32 = 2e-3
+EPS_SCORE = 2e-5     # fp32 drafter scores against the fp64 oracle: measured 3e-6 at scores of about -25
 
 
-from helpers import Rig, dev, top2_gap  # noqa: E402
+from helpers import Rig, check_beams_within, dev, tolerant_beam_search, top2_gap  # noqa: E402
 
 
 @pytest.fixture(scope="module")
@@ -133,15 +134,14 @@ def test_draft_beams_and_scores(rig):
     prompt, kv, ctx, g, h = prefilled(rig)
     beams, scores = rig.eng.draft()
     rig.eng.poll()
-    rb, rs, cand = ora.beam_search(rig.D, rig.W["tok_emb"], g, h, 4, 4, return_logp=True)
-    # the beams are decided by float comparisons: require the oracle's candidate gaps at every call
-    ok = True
-    for c in cand:
-        s = np.sort(c)[::-1][:5]
-        ok = ok and (np.diff(s) < -2 * TOL_FP32).all()
-    if ok:
-        assert beams[0].cpu().numpy().tolist() == rb.tolist()
-        assert np.abs(scores[0].cpu().numpy() - rs).max() < TOL_FP32
+    # the oracle's beam search with every decision widened by the fp32 error bound: for this state no decision comes
+    # within it (an oracle-side fact, asserted), so the beams must be the oracle's element by element
+    sets = tolerant_beam_search(ora, rig.D, rig.W["tok_emb"], g, h, 4, 4, EPS_SCORE)
+    assert len(sets[0]) == 4 and not sets[1] and sets[2] == 0
+    assert check_beams_within(sets, beams[0].cpu().numpy(), scores[0].cpu().numpy(), EPS_SCORE) == 4
+    rb, rs = ora.beam_search(rig.D, rig.W["tok_emb"], g, h, 4, 4)
+    assert beams[0].cpu().numpy().tolist() == rb.tolist()
+    assert np.abs(scores[0].cpu().numpy() - rs).max() < EPS_SCORE
     assert (np.diff(scores[0].cpu().numpy()) <= 0).all()
     # whatever the ties, each returned score is the drafter's log-probability of that sequence
     for b, s in zip(beams[0].cpu().numpy(), scores[0].cpu().numpy()):
@@ -167,16 +167,23 @@ def run_steps(rig, n_steps, p, rho, seed, drafted=False):
     out = rig.binding.AcceptOut(1, L, "cuda:0")
     emitted = [g]
     accepted = []
+    drafted_equal = []
     for step in range(n_steps):
         planted = None if drafted else synth.plant_beams(ar[len(emitted):len(emitted) + L], BW, L, cfg["vocab"], rng, p=p, rho=rho)
         ref = ora.spec_step(rig.W, rig.D, cfg, kv, ctx, g, h, BW, L, planted=planted, run_drafter=drafted)
         # teacher forcing: both sides start the step from the oracle's state
         rig.eng.set_state(dev([ctx]), dev([g]), dev(h[None], torch.float32), batch=1, ctx_bound=ctx)
         if drafted:
-            gb, _ = rig.eng.draft()
-            if gb[0].cpu().numpy().tolist() != ref["beams"].tolist():
-                break                                # a near-tie in the drafter: stop comparing here
-            rig.eng.step(gb, out)
+            gb, gs = rig.eng.draft()
+            sets = tolerant_beam_search(ora, rig.D, rig.W["tok_emb"], g, h, BW, L, EPS_SCORE)
+            check_beams_within(sets, gb[0].cpu().numpy(), gs[0].cpu().numpy(), EPS_SCORE)
+            if not sets[1]:
+                # no decision within the error bound: the drafter's beams are the oracle's, and the step runs on them
+                assert gb[0].cpu().numpy().tolist() == ref["beams"].tolist()
+                drafted_equal.append(step)
+                rig.eng.step(None, out)
+            else:
+                rig.eng.step(dev(ref["beams"][None]), out)   # a near-tie: both sides verify the oracle's beams
         else:
             rig.eng.step(dev(planted[None]), out)
         rig.eng.poll()
@@ -199,6 +206,8 @@ def run_steps(rig, n_steps, p, rho, seed, drafted=False):
         assert np.abs(kvg[:, 0].transpose(0, 2, 1, 3) - kv.k[:, :ctx]).max() < TOL_FP32
         assert np.abs(kvg[:, 1].transpose(0, 2, 1, 3) - kv.v[:, :ctx]).max() < TOL_FP32
     assert emitted == ar[:len(emitted)]
+    if drafted:
+        return accepted, drafted_equal
     return accepted
 
 
@@ -218,7 +227,10 @@ def test_step_all_accepted_and_none_accepted(rig):
 
 
 def test_step_with_drafted_beams(rig):
-    run_steps(rig, 4, 0.0, 0.0, seed=11, drafted=True)
+    """Whole steps on the drafter's own beams (no planted input): in at least three of the four steps the GPU's beams
+    equal the oracle's element by element and the step's outcome is compared on them."""
+    accepted, drafted_equal = run_steps(rig, 4, 0.0, 0.0, seed=11, drafted=True)
+    assert len(accepted) == 4 and len(drafted_equal) >= 3
 
 
 def test_full_tiny_config_32_steps_lossless_free_running(rig):

@@ -152,3 +152,30 @@ def test_storage_error_grows_as_sqrt_depth_at_the_7b_layer_shape():
         assert 0.75 < err[depth] / (err[1] * np.sqrt(depth)) < 1.25, err
     # extrapolated to the workloads' depths the storage alone exceeds the 3e-2 that holds for shallow copies
     assert err[8] * np.sqrt(32 / 8) > 2.5e-2
+
+    # Two correct implementations of the SAME rounded arithmetic drift apart: perturb every array by a relative 1e-6
+    # before it is rounded (what a different summation order does to an fp32 sum) and the logits after eight layers
+    # differ from the unperturbed rounded run by more than half the storage noise itself, while both stay equally far
+    # from the unrounded oracle.  A tight bound against the rounded oracle is therefore not a property any kernel can
+    # have; the GPU parity cases bound the distance to BOTH oracle modes by the distance between them.
+    def mean_l2(a, b):
+        return float(np.mean(np.linalg.norm(a - b, axis=1) / np.linalg.norm(b, axis=1)))
+    rng = np.random.default_rng(1)
+    plain_st = ora._st
+
+    def jittered_st(a, store):
+        if store is None:
+            return a
+        return ora.round_bf16(a * (1 + 1e-6 * rng.standard_normal(a.shape).astype(a.dtype)))
+    c = dict(cfg, n_layers=8)
+    runs = {}
+    for name, st, store in (("U", plain_st, None), ("R", plain_st, "bf16"), ("R2", jittered_st, "bf16")):
+        ora._st = st
+        try:
+            kv = ora.KVCache(8, 32, cfg["n_heads"], 128, np.float32)
+            runs[name] = ora.llm_forward(W, c, prompt, np.arange(P), mask, kv, 0, np.float32, store=store)[1]
+        finally:
+            ora._st = plain_st
+    noise = mean_l2(runs["R"], runs["U"])
+    assert 0.5 * noise < mean_l2(runs["R2"], runs["R"]) < 1.1 * noise
+    assert abs(mean_l2(runs["R2"], runs["U"]) - noise) < 0.05 * noise
