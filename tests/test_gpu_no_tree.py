@@ -65,7 +65,8 @@ def flat_against_oracle_and_packed(cfg, tol_abs, tol_rel, n_steps, seed):
         assert out.tokens[0, :a + 1].tolist() == toks and (out.tokens[0, a + 1:] == -1).all()
         # packed tree on the GPU: a node and each of its flat copies see the same logits
         pk_t = tree.eng.pack(beams_d)
-        _, _, logits_t = tree.eng.verify(pk_t, want_logits=True)
+        argmax_t, hidden_t, logits_t = tree.eng.verify(pk_t, want_logits=True)
+        tree.eng.accept(beams_d, pk_t, argmax_t, hidden_t)         # keeps this engine's cache in step with the other's
         tree.eng.poll()
         up_t, up_f = pk_t.unpack[0].cpu().numpy(), pk.unpack[0].cpu().numpy()
         lt = logits_t[0].cpu().numpy()
