@@ -224,8 +224,13 @@ RD_API int redrafter_get_state(rd_handle* h, void* stream, int32_t* ctx, int32_t
 RD_API int redrafter_set_state(rd_handle* h, void* stream, const int32_t* ctx, const int32_t* root, const float* hvec,
                         int32_t batch);
 
-/* Tell the handle the largest context length any sequence can have now (host-side bound used by
- * the capacity check; set_state callers use it after rewinding or advancing the state). */
+/* Tell the handle the largest context length any sequence can have now.  The handle keeps this bound on the host
+ * (it never reads device memory synchronously): the capacity check (RD_ERR_CAPACITY when bound + 1 + beam_width *
+ * beam_length > max_ctx) and the attention launch geometry follow it.  Every step adds 1 + beam_length to it, the most
+ * a step can accept; every eighth call also enqueues a copy of the true context lengths to pinned host memory, and a
+ * later call that finds the copy complete lowers the bound to what it implies, so the bound runs ahead of the real
+ * contexts by at most eight steps' worth.  A caller that passes `ctx` to redrafter_set_state MUST call this function
+ * too (set_state does not read the array it is given): the bound is not raised by the feedback. */
 RD_API int redrafter_set_ctx_bound(rd_handle* h, int32_t max_ctx_now);
 
 /* Synchronise `stream`, read the device status word and clear it.  Returns RD_OK or the first

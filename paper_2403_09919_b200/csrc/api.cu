@@ -96,6 +96,17 @@ struct rd_handle {
   bool tc_pairs_prefill;
   std::vector<TensorMapBox> kv_maps;   // [layer][K | V]: cache planes as [sequences * heads * max_ctx][head dim] matrices
   Chain chain;  // counter hand-off between the launches of a forward pass
+  bool chain_dirty;  // a launch failed after the chain had counted it: reset the counters before the next pass
+  int device;        // ordinal of the device the handle was made on
+  // Context-bound feedback: after a step the device-side context lengths are copied to pinned host memory without
+  // waiting; a later call that finds the copy complete tightens the host-side bound with it.
+  int32_t* fb_host;          // [2][max_batch] pinned
+  cudaEvent_t fb_event[2];
+  bool fb_pending[2];
+  int64_t fb_growth_at[2];   // value of fb_growth when the copy was enqueued
+  int64_t fb_growth;         // tokens by which a sequence's context can have grown since the handle was made
+  int fb_next;
+  unsigned fb_calls;         // a copy is enqueued on every eighth call: the bound lags by at most 8 (1 + L) tokens
   std::unordered_map<const void*, TensorMapBox> maps;               // weights
   std::unordered_map<const void*, std::pair<int, int>> act_shape;   // activation buffers: rows, cols
   std::map<std::pair<const void*, int>, TensorMapBox> act_maps;     // by (buffer, rows per box), made on first use
@@ -122,6 +133,7 @@ int init_fail(rd_handle* h, int code, const char* fmt, ...) {
 }
 
 int fail(rd_handle* h, int code, const char* fmt, ...) {
+  if (h && code == RD_ERR_CUDA) h->chain_dirty = true;
   if (h) {
     va_list ap;
     va_start(ap, fmt);
@@ -307,6 +319,52 @@ int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, cons
   return RD_OK;
 }
 
+// Start of a chained region: counters back in step with the host if an earlier launch was counted but never ran.
+int chain_start(rd_handle* h, cudaStream_t st) {
+  if (h->chain_dirty) {
+    cudaError_t e = h->chain.reset(st);
+    if (e != cudaSuccess) return fail(h, RD_ERR_CUDA, "resetting the hand-off counters: %s", cudaGetErrorString(e));
+    h->chain_dirty = false;
+  }
+  h->chain.cut();
+  return RD_OK;
+}
+
+// ---- context-bound feedback (host side only; never waits)
+void fb_invalidate(rd_handle* h) { h->fb_pending[0] = h->fb_pending[1] = false; }
+
+// A copy of the context lengths that has completed bounds every sequence's context by its largest value plus
+// whatever the calls enqueued since can have added.
+void fb_poll(rd_handle* h) {
+  if (!h->fb_host) return;
+  for (int s = 0; s < 2; ++s) {
+    if (!h->fb_pending[s] || cudaEventQuery(h->fb_event[s]) != cudaSuccess) continue;
+    h->fb_pending[s] = false;
+    int mx = 0;
+    for (int b = 0; b < h->batch; ++b) mx = h->fb_host[(size_t)s * h->dm.B + b] > mx ? h->fb_host[(size_t)s * h->dm.B + b] : mx;
+    const long long bound = (long long)mx + (h->fb_growth - h->fb_growth_at[s]);
+    if (bound < h->ctx_bound) h->ctx_bound = (int)bound;
+  }
+  (void)cudaGetLastError();   // cudaEventQuery's cudaErrorNotReady is not an error of this handle
+}
+
+// After a call that advanced the contexts by at most `grow` tokens each.
+void fb_advance(rd_handle* h, int grow, cudaStream_t st) {
+  h->ctx_bound += grow;
+  h->fb_growth += grow;
+  if (!h->fb_host || (h->fb_calls++ & 7u) != 0u) return;
+  const int s = h->fb_next;
+  if (h->fb_pending[s]) return;   // that slot's copy is still on its way: try again after the next call
+  if (cudaMemcpyAsync(h->fb_host + (size_t)s * h->dm.B, h->ws.ctx, (size_t)h->batch * sizeof(int32_t), cudaMemcpyDeviceToHost, st) !=
+          cudaSuccess || cudaEventRecord(h->fb_event[s], st) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return;
+  }
+  h->fb_pending[s] = true;
+  h->fb_growth_at[s] = h->fb_growth;
+  h->fb_next = s ^ 1;
+}
+
 char* kv_plane_ptr(rd_handle* h, int layer, int which) {
   return h->kv + ((size_t)(layer * 2 + which)) * h->kv_plane * esize(h->dm.dtype);
 }
@@ -356,7 +414,7 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
   // inside the layer loop every launch hands over to the next through a counter; the launches before
   // and after it use the grid dependency
   Chain* ch = h->use_tc ? &h->chain : nullptr;
-  h->chain.cut();
+  if (int rc0 = chain_start(h, st)) return rc0;
   for (int l = 0; l < dm.n_layers; ++l) {
     // attention block: (x += down of the previous layer) -> norm -> QKV -> rotary + KV write -> attention -> O
     CKP(h, PROF_NORM, launch_rmsnorm(dm.dtype, w.x, l ? &g_dn : nullptr, h->attn_norm[l], w.a_t, nullptr, dm.d, dm.eps,
@@ -403,6 +461,7 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
 int check_stepable(rd_handle* h) {
   if (!h) return RD_ERR_INVALID_ARG;
   if (!h->prefilled) return fail(h, RD_ERR_STATE, "no state: call redrafter_prefill or redrafter_set_state first");
+  fb_poll(h);
   if (h->ctx_bound + h->dm.NMAX > h->dm.max_ctx)
     return fail(h, RD_ERR_CAPACITY, "context bound %d + %d packed rows exceeds max_ctx %d", h->ctx_bound, h->dm.NMAX,
                 h->dm.max_ctx);
@@ -420,7 +479,7 @@ int do_draft(rd_handle* h, cudaStream_t st, int32_t* beams, float* scores) {
   GemmOut g;
   // the calls' launches hand over to each other through counters (tensor-core path)
   Chain* ch = h->use_tc ? &h->chain : nullptr;
-  h->chain.cut();
+  if (int rc0 = chain_start(h, st)) return rc0;
   for (int call = 1; call <= dm.L; ++call) {
     const int rows = call == 1 ? B : R;
     const int32_t* mt = call == 1 ? w.one_b : w.one_r;
@@ -599,6 +658,19 @@ int redrafter_init(const rd_config* cfg, const rd_weights* wt, void* kv_cache, s
   h->chain.ctr = h->ws.chain_ctr; h->chain.status = h->ws.status;
   h->chain.trace_base = h->ws.trace; h->chain.trace_next = &h->trace_next; h->chain.trace_cap = TRACE_SLOTS;
   h->chain.enabled = !(getenv("RD_CHAIN") && atoi(getenv("RD_CHAIN")) == 0);
+  h->chain_dirty = false;
+  h->device = 0;
+  (void)cudaGetDevice(&h->device);
+  // pinned host memory and two events for the context-bound feedback (host resources; no device memory)
+  h->fb_host = nullptr; h->fb_pending[0] = h->fb_pending[1] = false; h->fb_growth = 0; h->fb_next = 0; h->fb_calls = 0;
+  h->fb_event[0] = h->fb_event[1] = nullptr;
+  if (cudaHostAlloc((void**)&h->fb_host, (size_t)2 * dm.B * sizeof(int32_t), cudaHostAllocDefault) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->fb_event[0], cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->fb_event[1], cudaEventDisableTiming) != cudaSuccess) {
+    (void)cudaGetLastError();
+    if (h->fb_host) cudaFreeHost(h->fb_host);
+    h->fb_host = nullptr;   // the bound then simply grows by 1 + L per step until the caller refreshes it
+  }
   for (int c = 0; c < PROF_CLASSES; ++c) { h->ev_used[c] = 0; h->prof_ms[c] = 0; h->prof_bytes[c] = 0; h->prof_n[c] = 0; }
   // clear the state and the constants the kernels read from device memory
   cudaError_t e = cudaMemsetAsync(workspace, 0, (size_t)((char*)h->ws.x - (char*)workspace), 0);
@@ -620,6 +692,13 @@ int redrafter_destroy(rd_handle* h) {
   if (!h) return RD_ERR_INVALID_ARG;
   for (int c = 0; c < PROF_CLASSES; ++c)
     for (cudaEvent_t e : h->ev[c]) cudaEventDestroy(e);
+  if (h->fb_host) {
+    for (int s = 0; s < 2; ++s)
+      if (h->fb_pending[s]) cudaEventSynchronize(h->fb_event[s]);   // a copy into the pinned buffer may still be in flight
+    cudaFreeHost(h->fb_host);
+  }
+  for (int s = 0; s < 2; ++s)
+    if (h->fb_event[s]) cudaEventDestroy(h->fb_event[s]);
   delete h;
   return RD_OK;
 }
@@ -715,6 +794,7 @@ int redrafter_prefill(rd_handle* h, const int32_t* tokens, const int32_t* prompt
   CK(h, launch_argmax_rows(w.logits, g, dm.V, w.root, nullptr, w.one_b, batch, h->sampling, nullptr, w.ctx, 0, st));
   h->prefilled = true;
   h->ctx_bound = longest;
+  fb_invalidate(h);
   return RD_OK;
 }
 
@@ -756,7 +836,7 @@ int redrafter_accept(rd_handle* h, const int32_t* beams, const rd_packed* packed
   CK(h, launch_accept(h->dm.dtype, beams, *packed, argmax, hidden, h->kv, w.ctx, w.root, w.h, o, w.n_accept, w.best,
                       w.ctx_prev, h->dm, h->batch, w.status, (cudaStream_t)stream));
   h->launches++;  // accept + compaction
-  h->ctx_bound += 1 + h->dm.L;
+  fb_advance(h, 1 + h->dm.L, (cudaStream_t)stream);
   return RD_OK;
 }
 
@@ -765,6 +845,9 @@ int redrafter_accept_static(rd_handle* h, const int32_t* beams, const rd_packed*
   int rc = check_stepable(h);
   if (rc) return rc;
   if (!beams || !packed_ok(packed) || !argmax || !hidden) return fail(h, RD_ERR_INVALID_ARG, "null argument");
+  int dev_now = -1;
+  if (cudaGetDevice(&dev_now) != cudaSuccess || dev_now != h->device)
+    return fail(h, RD_ERR_STATE, "current device %d is not the device %d this handle was made on", dev_now, h->device);
   if (h->batch > accept_static_max_batch())
     return fail(h, RD_ERR_CAPACITY, "batch %d exceeds the %d sequences the built-in scratch holds", h->batch,
                 accept_static_max_batch());
@@ -777,7 +860,7 @@ int redrafter_accept_static(rd_handle* h, const int32_t* beams, const rd_packed*
   CK(h, launch_accept(h->dm.dtype, beams, *packed, argmax, hidden, h->kv, w.ctx, w.root, w.h, o, n_accept, best, ctx_prev,
                       h->dm, h->batch, w.status, (cudaStream_t)stream));
   h->launches++;  // accept + compaction
-  h->ctx_bound += 1 + h->dm.L;
+  fb_advance(h, 1 + h->dm.L, (cudaStream_t)stream);
   return RD_OK;
 }
 
@@ -797,13 +880,14 @@ int redrafter_step(rd_handle* h, const int32_t* planted_beams, void* stream, con
   CKP(h, PROF_PACK_ACCEPT, launch_accept(h->dm.dtype, beams, w.pk, w.argmax_p, w.hidden_p, h->kv, w.ctx, w.root, w.h, o, w.n_accept,
                       w.best, w.ctx_prev, h->dm, h->batch, w.status, st));
   h->launches++;
-  h->ctx_bound += 1 + h->dm.L;
+  fb_advance(h, 1 + h->dm.L, st);
   return RD_OK;
 }
 
 int redrafter_ar_step(rd_handle* h, void* stream, int32_t* token) {
   if (!h) return RD_ERR_INVALID_ARG;
   if (!h->prefilled) return fail(h, RD_ERR_STATE, "no state: call redrafter_prefill or redrafter_set_state first");
+  fb_poll(h);
   if (h->ctx_bound + 1 > h->dm.max_ctx) return fail(h, RD_ERR_CAPACITY, "KV cache full");
   cudaStream_t st = (cudaStream_t)stream;
   Workspace& w = h->ws;
@@ -818,7 +902,7 @@ int redrafter_ar_step(rd_handle* h, void* stream, int32_t* token) {
   if (rc) return rc;
   CK(h, launch_argmax_rows(w.logits, g, dm.V, w.argmax_c, nullptr, w.m_total, B, h->sampling, w.row_seq, w.row_pos, 1, st));
   CK(h, launch_ar_finish(w.argmax_c, w.hidden_f, w.ctx, w.root, w.h, token, dm, B, st));
-  h->ctx_bound += 1;
+  fb_advance(h, 1, st);
   return RD_OK;
 }
 
@@ -850,7 +934,10 @@ int redrafter_set_state(rd_handle* h, void* stream, const int32_t* ctx, const in
   int rc = set_row_counts(h, st);
   if (rc) return rc;
   const size_t B = batch;
-  if (ctx) CKRT(h, cudaMemcpyAsync(h->ws.ctx, ctx, B * sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
+  if (ctx) {
+    CKRT(h, cudaMemcpyAsync(h->ws.ctx, ctx, B * sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
+    fb_invalidate(h);   // copies of the old context lengths say nothing about the new ones
+  }
   if (root) CKRT(h, cudaMemcpyAsync(h->ws.root, root, B * sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
   if (hvec) CKRT(h, cudaMemcpyAsync(h->ws.h, hvec, B * h->dm.d * sizeof(float), cudaMemcpyDeviceToDevice, st));
   h->prefilled = true;
@@ -860,6 +947,7 @@ int redrafter_set_state(rd_handle* h, void* stream, const int32_t* ctx, const in
 int redrafter_set_ctx_bound(rd_handle* h, int32_t max_ctx_now) {
   if (!h || max_ctx_now < 0) return RD_ERR_INVALID_ARG;
   h->ctx_bound = max_ctx_now;
+  fb_invalidate(h);
   return RD_OK;
 }
 
@@ -941,6 +1029,7 @@ int redrafter_poll(rd_handle* h, void* stream) {
   CKRT(h, cudaStreamSynchronize(st));
   if (v == 0) return RD_OK;
   CKRT(h, cudaMemsetAsync(h->ws.status, 0, sizeof(int32_t), st));
+  if (v & DEV_ERR_TIMEOUT) h->chain_dirty = true;   // launches behind the wait that gave up may not have signalled
   if (v & DEV_ERR_TIMEOUT) return fail(h, RD_ERR_TIMEOUT, "device status 0x%x: a bounded wait gave up", v);
   if (v & DEV_ERR_CAPACITY) return fail(h, RD_ERR_CAPACITY, "device status 0x%x: a KV slot beyond max_ctx was skipped", v);
   return fail(h, RD_ERR_INVALID_ARG, "device status 0x%x: token id or index out of range", v);

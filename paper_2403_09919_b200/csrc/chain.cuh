@@ -61,6 +61,15 @@ struct Chain {
   }
   // An un-chained launch follows: whatever comes after it must wait on the grid dependency again.
   void cut() { prev_ptr = nullptr; }
+  // Counters and targets back to zero (enqueued on `st`; nothing of the chain may be in flight on another stream).
+  // Needed when a launch that link() had already counted never ran, or a wait gave up: the device counters would
+  // stay behind their host-side targets for good.
+  cudaError_t reset(cudaStream_t st) {
+    for (int i = 0; i < CHAIN_SLOTS; ++i) cum[i] = 0;
+    next = 0;
+    cut();
+    return ctr ? cudaMemsetAsync(ctr, 0, CHAIN_SLOTS * sizeof(unsigned int), st) : cudaSuccess;
+  }
 };
 
 #ifdef __CUDACC__

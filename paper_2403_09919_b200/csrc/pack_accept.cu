@@ -1,6 +1,8 @@
 // Dynamic tree attention packing (Section 3.3, Appendix A.1) and greedy acceptance with KV-cache
 // compaction (Section 3.4).  Integer work on at most a few thousand entries per sequence: one CTA
 // per sequence, everything staged in shared memory, no host involvement.
+#include <mutex>
+
 #include "rd_internal.cuh"
 #include "pdl.cuh"
 
@@ -221,10 +223,12 @@ int accept_static_max_batch() { return ACCEPT_STATIC_MAX_BATCH; }
 cudaError_t accept_static_scratch(int32_t** n_accept, int32_t** best, int32_t** ctx_prev) {
   constexpr int MAX_DEVICES = 64;
   static int32_t* base[MAX_DEVICES] = {};
+  static std::mutex mu;   // host threads may make their first call on a device at the same time
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(mu);
   if (base[dev] == nullptr) {
     void* p = nullptr;
     e = cudaGetSymbolAddress(&p, g_accept_scratch);

@@ -303,6 +303,24 @@ def test_batched_ragged_step():
             assert np.abs(kvg - kv.k[:, :ref["ctx"]]).max() < TOL_FP32
 
 
+def test_context_bound_follows_the_real_context():
+    """The handle's host-side context bound grows by 1 + L per step, the most a step can accept; copies of the real
+    context lengths that arrive later pull it back.  Here 48 steps accept about one token each: without the feedback
+    the bound would pass 16 + 48 * 5 = 256 and the capacity check would refuse a step long before the cache is full."""
+    cfg = dict(synth.CONFIGS["tiny"], max_ctx=16 + 48 * 2 + 17 + 10 * 5)
+    r = Rig(cfg=cfg)
+    r.eng.prefill([np.random.default_rng(14).integers(0, 1024, size=16)])
+    out = r.binding.AcceptOut(1, 4, "cuda:0")
+    rng = np.random.default_rng(15)
+    for step in range(48):
+        r.eng.step(dev(rng.integers(0, 1024, size=(1, 4, 4))), out)     # random candidates: at most a lucky token accepted
+        if step % 8 == 7:
+            r.eng.poll()                                                  # a serving loop reads its results now and then
+    ctx = int(r.eng.get_state()[0][0])
+    assert 16 + 48 <= ctx <= 16 + 48 * 2
+    r.eng.close()
+
+
 def test_errors(rig):
     from paper_2403_09919_b200.binding import RdError, ReDrafter
     eng = ReDrafter(rig.cfg, rig.w)

@@ -60,3 +60,30 @@ def test_accept_static_rejects_null_arguments():
     with pytest.raises(RdError) as e:
         r.eng.accept_static(beams, pk, am, None)
     assert e.value.code == 1
+
+
+def test_accept_static_refuses_more_sequences_than_its_scratch_holds():
+    """The built-in scratch holds 4096 sequences; a batch of 4097 is refused before anything is enqueued (a caller
+    that cannot allocate must learn this from the status code, not from a fault)."""
+    from paper_2403_09919_b200.binding import AcceptOut, RdError
+    cfg = dict(synth.CONFIGS["tiny"], n_layers=1, d_model=64, n_heads=1, d_ffn=64, vocab=128, d_rnn=64, max_batch=4097,
+               max_ctx=8, beam_width=1, beam_length=1)
+    r = Rig(cfg=cfg)
+    B = 4097
+    r.eng.set_state(dev(np.ones(B)), dev(np.zeros(B)), None, batch=B, ctx_bound=1)
+    beams = torch.zeros(B, 1, 1, dtype=torch.int32, device="cuda:0")
+    pk = r.eng.pack(beams)
+    am, hid, _ = r.eng.verify(pk)
+    launches = r.eng.launch_count()
+    with pytest.raises(RdError) as e:
+        r.eng.accept_static(beams, pk, am, hid, AcceptOut(B, 1, "cuda:0"))
+    assert e.value.code == 3 and r.eng.launch_count() == launches      # RD_ERR_CAPACITY, nothing enqueued
+    r.eng.accept(beams, pk, am, hid)                                      # the workspace-backed entry point takes it
+    r.eng.poll()
+    # 4096 sequences fit
+    r.eng.set_state(dev(np.ones(4096)), dev(np.zeros(4096)), None, batch=4096, ctx_bound=1)
+    beams = beams[:4096].contiguous()
+    pk = r.eng.pack(beams)
+    am, hid, _ = r.eng.verify(pk)
+    r.eng.accept_static(beams, pk, am, hid, AcceptOut(4096, 1, "cuda:0"))
+    r.eng.poll()
