@@ -105,10 +105,57 @@ def step_bytes(cfg, ctx, n_rows=None):
 
 
 # --------------------------------------------------------------------------- CPU oracle legs
+def host_weights(cfg):
+    """The workload's seeded weights as host fp32 arrays for the oracle.  Drawn on the GPU when there is one (the same
+    generator and seeds the CUDA arm uses, seconds instead of minutes for 7 G values) and copied to the host, else on
+    the CPU.  Input generation only: none of the library's kernels is involved."""
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    w = synth.make_weights(cfg, dev)
+    W, D = synth.weights_to_numpy(w, cfg)
+    del w
+    if dev != "cpu":
+        torch.cuda.empty_cache()
+    return W, D
+
+
+class OracleFull:
+    """The oracle, as it stands, on the workload itself: all layers, its own prefill of the workload's prompt (untimed,
+    like the CUDA arm's), then whole speculative steps timed one by one.  fp32 numpy, batch 1."""
+
+    def __init__(self, cfg, sampling=None, weights=None):
+        from oracle import redrafter_oracle as ora
+        self.ora, self.cfg, self.sampling = ora, cfg, sampling
+        self.W, self.D = weights if weights is not None else host_weights(cfg)
+        self.prompt = synth.make_prompts(cfg, 1, seed=cfg.get("seed", 0))[0]
+        self.extrapolated = False
+
+    def run(self, steps, warmup=0):
+        ora, cfg = self.ora, self.cfg
+        BW, L = cfg["beam_width"], cfg["beam_length"]
+        hd = cfg["d_model"] // cfg["n_heads"]
+        cap = len(self.prompt) + (steps + warmup) * (L + 1) + 2 + BW * L
+        kv = ora.KVCache(cfg["n_layers"], cap, cfg["n_heads"], hd, np.float32)
+        t0 = time.perf_counter()
+        ctx, g, h = ora.prefill(self.W, cfg, self.prompt, kv, np.float32, self.sampling)
+        prefill_s = time.perf_counter() - t0
+        tot_s, tot_tok, rows = 0.0, 0, 0
+        for s in range(warmup + steps):
+            t0 = time.perf_counter()
+            r = ora.spec_step(self.W, self.D, cfg, kv, ctx, g, h, BW, L, dtype=np.float32, sampling=self.sampling)
+            dt = time.perf_counter() - t0
+            ctx, g, h = r["ctx"], r["g"], r["h"]
+            if s >= warmup:
+                tot_s += dt; tot_tok += len(r["emitted"]); rows += int(r["packed"]["n"])
+        sample = (f"{steps} whole oracle steps of the workload itself ({cfg['n_layers']} layers, fp32 numpy) after {warmup} warm-up, "
+                  f"on the cache its own prefill of the {len(self.prompt)}-token prompt wrote ({prefill_s:.0f} s, untimed); drafter's own "
+                  f"beams, mean {rows / steps:.0f} packed rows; {tot_s:.1f} s of timed CPU work")
+        return dict(value=tot_tok / tot_s, ms_per_step=1e3 * tot_s / steps, sample=sample, timed_s=tot_s)
+
+
 class OracleSample:
-    """The oracle on a depth-reduced copy of the workload: full per-layer shapes, `sample_layers`
-    layers, fp32 numpy arithmetic.  One step is timed in parts and scaled to the full depth:
-    t_step = t_draft + t_pack + (n_layers / sample_layers) * t_layers + t_lm_head + t_accept."""
+    """For the workloads whose full-depth oracle step takes minutes (13B, batched 7B, 33B): the oracle on a
+    depth-reduced copy, full per-layer shapes, `sample_layers` layers, fp32 numpy.  One step is timed in parts and
+    EXTRAPOLATED to the full depth: t_step = t_draft + t_pack + (n_layers / sample_layers) * t_layers + t_lm_head + t_accept."""
 
     def __init__(self, cfg, sample_layers=2, sampling=None):
         self.cfg = cfg
@@ -117,6 +164,7 @@ class OracleSample:
         self.c = synth.with_layers(cfg, self.sample_layers)
         w = synth.make_weights(self.c, "cpu")
         self.W, self.D = synth.weights_to_numpy(w, self.c)
+        self.extrapolated = True
 
     def step(self, seed=0):
         from oracle import redrafter_oracle as ora
@@ -156,10 +204,16 @@ class OracleSample:
         for s in range(steps):
             r = self.step(s)
             tot_s += r["step_s"]; tot_tok += r["tokens"]; cpu_s += r["cpu_s"]; rows += r["rows"]
-        sample = (f"{steps} oracle steps on a {self.sample_layers}-layer copy of the workload at full per-layer shapes "
-                  f"(fp32 numpy, filled cache of {self.cfg['prompt_len']} tokens, drafter's own beams, mean {rows / steps:.0f} "
-                  f"packed rows); the layer time is scaled by n_layers/{self.sample_layers}; {cpu_s:.1f} s of CPU work")
-        return dict(value=tot_tok / tot_s, ms_per_step=1e3 * tot_s / steps, sample=sample)
+        sample = (f"EXTRAPOLATED: {steps} oracle steps on a {self.sample_layers}-layer copy of the workload at full per-layer "
+                  f"shapes (fp32 numpy, filled cache of {self.cfg['prompt_len']} tokens, drafter's own beams, one sequence, mean "
+                  f"{rows / steps:.0f} packed rows); the layer time is scaled by n_layers/{self.sample_layers}; {cpu_s:.1f} s of CPU work")
+        return dict(value=tot_tok / tot_s, ms_per_step=1e3 * tot_s / steps, sample=sample, timed_s=cpu_s)
+
+
+def oracle_leg(args, cfg):
+    """The full-depth oracle where a step takes seconds (tiny, 7B bs1); the depth-reduced, extrapolated sample elsewhere."""
+    full = cfg["max_batch"] == 1 and cfg["n_layers"] * cfg["d_model"] <= 32 * 4096 and not args.oracle_sample
+    return OracleFull(cfg, oracle_sampling(args)) if full else OracleSample(cfg, args.oracle_layers, oracle_sampling(args))
 
 
 def oracle_sampling(args):
@@ -179,14 +233,19 @@ def run_reference(args, cfg):
     if rank != 0:
         return
     steps = max(1, min(args.steps, args.reference_max_steps))
-    r = OracleSample(cfg, args.oracle_layers, oracle_sampling(args)).run(steps, warmup=min(args.warmup, 1))
+    warm = min(args.warmup, 1)
+    leg = oracle_leg(args, cfg)
+    r = leg.run(steps, warmup=warm)
     value, sample = r["value"], r["sample"]
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
-            "warmup": min(args.warmup, 1), "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+            "warmup": warm, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": workload_config(args, cfg),
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_cores(), "kind": "oracle", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_cores(), "kind": "oracle", "sample": sample,
+                             "extrapolated": leg.extrapolated},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    if not leg.extrapolated:
+        line["ms_per_step"] = r["ms_per_step"]      # a measured step time; an extrapolated one is not reported as such
     print(json.dumps(line))
 
 
@@ -221,6 +280,18 @@ def shard_of_rank(rank):
 
 
 # --------------------------------------------------------------------------- GPU legs
+def packed_rows_summary(n, BW, L):
+    """Packed rows per sequence and step (root + deduplicated draft tokens) against the 1 + BW * L rows the flat layout
+    would verify: the synthetic analogue of Figure 5 (left)."""
+    n = np.asarray(n).reshape(-1)
+    flat = 1 + BW * L
+    edges = np.linspace(0, flat, 9).round().astype(int)
+    hist, _ = np.histogram(n, bins=edges)
+    return {"flat_rows": flat, "mean": float(n.mean()), "min": int(n.min()), "max": int(n.max()),
+            "reduction": float(1.0 - n.mean() / flat), "histogram": {f"{edges[i] + (i > 0)}-{edges[i + 1]}": int(hist[i]) for i in range(8)},
+            "first_steps": [int(x) for x in n[:16]]}
+
+
 def timed_loop(eng, n, fn):
     """n calls of fn between two events on the current stream; returns ms."""
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -344,8 +415,9 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="depth-reduced run (0 = the workload's depth)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--oracle-layers", type=int, default=2)
-    ap.add_argument("--reference-max-steps", type=int, default=8)
-    ap.add_argument("--cpu-steps", type=int, default=20)
+    ap.add_argument("--reference-max-steps", type=int, default=3)
+    ap.add_argument("--cpu-steps", type=int, default=3)
+    ap.add_argument("--oracle-sample", action="store_true", help="time the depth-reduced oracle sample even where the full oracle is affordable")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the planted-beam and autoregressive comparison legs")
     ap.add_argument("--sweep", action="store_true", help="beam width x batch sweep instead of the benchmark line")
@@ -408,6 +480,7 @@ def main():
         eng.step(None, out)
     eng.poll()
     n_acc = torch.zeros(args.steps, B, dtype=torch.int32, device=device)
+    n_rows = torch.zeros(args.steps, B, dtype=torch.int32, device=device)
     launches0 = eng.launch_count()
     sampler = ClockSampler(local_rank)
     barrier()
@@ -416,6 +489,7 @@ def main():
     def one(i):
         eng.step(None, out)
         n_acc[i].copy_(out.n_accept)
+        eng.last_packed_rows(n_rows[i])
     ms = timed_loop(eng, args.steps, one)
     clocks = sampler.stop()
     launches = eng.launch_count() - launches0
@@ -427,11 +501,14 @@ def main():
     ms, tokens = reduce_over_ranks(ms, tokens, device)
     value = tokens / (ms * 1e-3)
     ms_per_step = ms / args.steps
+    packed = packed_rows_summary(n_rows.cpu().numpy(), BW, L)
 
     # ---- e2e leg: the same steps driven the way a serving loop does, results read to the host each step
     pin_a = torch.zeros(B, dtype=torch.int32).pin_memory()
     pin_t = torch.zeros(B, L + 1, dtype=torch.int32).pin_memory()
     e2e_tokens = [0]
+
+    ctx_host = [0]
 
     def one_e2e(i):
         eng.step(None, out)
@@ -439,9 +516,14 @@ def main():
         pin_t.copy_(out.tokens, non_blocking=True)
         torch.cuda.current_stream().synchronize()
         e2e_tokens[0] += int(pin_a.sum()) + B
+        # the loop knows what was accepted: it keeps the handle's context bound exact
+        ctx_host[0] += int(pin_a.max()) + 1
+        eng.set_ctx_bound(ctx_host[0])
     eng.prefill(prompts)
     for _ in range(args.warmup):
         eng.step(None, out)
+    ctx_host[0] = int(eng.get_state()[0].max().item())
+    eng.set_ctx_bound(ctx_host[0])
     barrier()
     ms_e2e = timed_loop(eng, args.steps, one_e2e)
     ms_e2e, e2e_tokens[0] = reduce_over_ranks(ms_e2e, e2e_tokens[0], device)
@@ -455,7 +537,7 @@ def main():
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if cfg["dtype"] == "bf16" else "f32", "data": "synthetic", "config": workload_config(args, cfg),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-            "tokens_per_step": tokens / (args.steps * B * world)}
+            "tokens_per_step": tokens / (args.steps * B * world), "packed_rows": packed}
 
     if rank == 0:
         # ---- roofline of the dominant kernel (the weight-streaming projection), timed per launch with CUDA events
@@ -485,13 +567,22 @@ def main():
             torch.cuda.synchronize()
             tr = eng.trace_read().astype(np.int64)
             tb = eng.trace_bytes()
+            tp = eng.trace_prefetched()
             eng.trace(False)
             sel = [i for i in range(len(tb)) if tb[i] > 0 and tr[i][6] > tr[i][2] > 0]
             body_ns = float(sum(int(tr[i][6] - tr[i][2]) for i in sel))
             if body_ns > 0:
-                in_step = {"gbs": float(sum(tb[i] for i in sel)) / body_ns, "launches": len(sel), "ms_per_step": body_ns * 1e-6,
-                           "note": "in-kernel %globaltimer records of one traced step (not CUDA events): weight bytes / time from "
-                                   "the last CTA's dependency wait to the last CTA's end, summed over the projections"}
+                all_b, pre_b = float(sum(tb[i] for i in sel)), float(sum(tp[i] for i in sel))
+                in_step = {"gbs": (all_b - pre_b) / body_ns, "launches": len(sel), "ms_per_step": body_ns * 1e-6,
+                           "prefetched_fraction": pre_b / all_b,
+                           "gbs_counting_prefetched_bytes": all_b / body_ns,
+                           "dram_busy_fraction_of_step": body_ns * 1e-6 / ms_per_step,
+                           "note": "in-kernel %globaltimer records of one traced step (not CUDA events).  Window of a projection: "
+                                   "from the LAST CTA's dependency wait to the LAST CTA's end; gbs counts the weight bytes "
+                                   "requested inside the window (every CTA's first ring-full of stages is requested before "
+                                   "its wait and streams in under the preceding kernel: prefetched_fraction); "
+                                   "gbs_counting_prefetched_bytes divides ALL weight bytes by the same windows and is an upper "
+                                   "bound, not a rate; dram_busy_fraction_of_step = sum of the windows / step time"}
                 in_step["frac_of_measured_peak"] = in_step["gbs"] / peak
         except Exception as e:  # measurement aid only
             in_step = {"error": str(e)}
@@ -511,6 +602,16 @@ def main():
                                                   zip(("rmsnorm", "rope", "swiglu", "draft_select", "pack_accept", "misc"), others)},
                             "other_launches_per_step": {n: o[2] / prof_steps for n, o in
                                                         zip(("rmsnorm", "rope", "swiglu", "draft_select", "pack_accept", "misc"), others)}}
+        line["headline"] = {"ms_per_step": ms_per_step, "frac_of_nominal_8tbs": sb["total"] / (ms_per_step * 1e-3) / 8e12,
+                            "frac_of_measured_peak": sb["total"] / (ms_per_step * 1e-3) / 1e9 / peak,
+                            "target": "north_star: >= 0.70 of the step's bytes / 8 TB/s",
+                            "note": "whole step (weights + KV bytes once) against the HBM roofline; roofline.frac is the "
+                                    "projection kernel timed launch by launch (serialised), roofline.in_step the same kernel in place"}
+        line["bf16_logits_tolerance"] = {
+            "stated": 3e-2, "met": "two-layer copies of every workload, against the unrounded and the bf16-storage oracle",
+            "full_depth": "not met against the unrounded oracle and not meetable: the oracle's own bf16-storage mode is 0.040 "
+                          "(7B, 32 layers), 0.057 (13B, 40) and 0.088 (33B, 60) relative L2 from its unrounded mode; the GPU "
+                          "measures 0.0395 / 0.0569 / 0.0872 and is held to 1.15 x the oracle pair's distance (tests/helpers.py)"}
         line["step_roofline"] = {"algorithmic_bytes_per_step": sb["total"], "achieved_gbs": sb["total"] / (ms_per_step * 1e-3) / 1e9,
                                  "frac_of_measured_peak": sb["total"] / (ms_per_step * 1e-3) / 1e9 / peak,
                                  "frac_of_nominal_8tbs": sb["total"] / (ms_per_step * 1e-3) / 8e12,
@@ -540,6 +641,8 @@ def main():
             # the position and hands the step the stream's own token as root.  Accepted tokens are stream tokens by
             # construction; only a bonus token can differ (a near-tie between the two kernels' summation orders),
             # which the root hand-off overrides -- counted as "bonus_flips".
+            sys.path.insert(0, os.path.join(ROOT, "tests"))
+            from helpers import first_mismatch            # closed form of greedy acceptance on planted beams (test arithmetic)
             rng = np.random.default_rng(2000 + cfg.get("seed", 0))
             n_pos = n_ar - L
             table = np.zeros((n_pos, B, BW, L), dtype=np.int32)
@@ -554,6 +657,9 @@ def main():
             pin_a2 = torch.zeros(B, dtype=torch.int32).pin_memory()
             pin_t2 = torch.zeros(B, L + 1, dtype=torch.int32).pin_memory()
             stats = dict(tokens=0, flips=0, closed=0, steps=0)
+            rows_p = torch.zeros(args.warmup + args.steps + 1, B, dtype=torch.int32, device=device)
+            step_no = [0]
+            ctx_p = eng.get_state()[0].cpu().numpy().astype(np.int64)
 
             def one_p(i, count=True):
                 for b in range(B):
@@ -561,16 +667,21 @@ def main():
                 eng.step(beams_d, out)
                 pin_a2.copy_(out.n_accept, non_blocking=True)
                 pin_t2.copy_(out.tokens, non_blocking=True)
+                if count:
+                    eng.last_packed_rows(rows_p[step_no[0]])
+                    step_no[0] += 1
                 torch.cuda.current_stream().synchronize()
                 for b in range(B):
                     a_ = int(pin_a2[b])
+                    ctx_p[b] += a_ + 1
                     if count:
                         stats["tokens"] += a_ + 1
                         stats["steps"] += 1
-                        stats["closed"] += int(a_ == synth.first_mismatch(table[posn[b], b], cont_h[posn[b]:posn[b] + L, b]).max())
+                        stats["closed"] += int(a_ == first_mismatch(table[posn[b], b], cont_h[posn[b]:posn[b] + L, b]).max())
                         stats["flips"] += int(int(pin_t2[b, a_]) != int(cont_h[posn[b] + a_, b]))
                     posn[b] += a_ + 1
                 eng.set_state(None, cont[posn[0] - 1] if B == 1 else torch.stack([cont[posn[b] - 1, b] for b in range(B)]), None)
+                eng.set_ctx_bound(int(ctx_p.max()))
             for s_ in range(args.warmup):
                 one_p(s_, count=False)
             ms_p = timed_loop(eng, args.steps, one_p)
@@ -579,14 +690,18 @@ def main():
             line["planted"] = {"tokens_per_s": tok_p / (ms_p * 1e-3), "ms_per_step": ms_p / args.steps,
                                "tokens_per_step": tok_p / max(1, stats["steps"]),
                                "steps_matching_closed_form": stats["closed"], "bonus_flips": stats["flips"],
+                               "packed_rows": packed_rows_summary(rows_p[:step_no[0]].cpu().numpy(), BW, L),
                                "speedup_vs_autoregressive": (tok_p / ms_p) / (n_ar * B / ms_ar),
                                "note": "beams = the autoregressive stream's continuation with each token replaced at p=0.3; "
                                        "teacher-forced root, accepted length read by the host every step (one sync per step)"}
             line["speedup_vs_autoregressive"] = value / world / (n_ar * B / (ms_ar * 1e-3))
         if not args.no_cpu_baseline and world == 1:
-            r = OracleSample(cfg, args.oracle_layers, oracle_sampling(args)).run(args.cpu_steps, warmup=1)
+            leg = oracle_leg(args, cfg)
+            r = leg.run(args.cpu_steps, warmup=1)
             line["cpu_baseline"] = {"value": r["value"], "unit": UNIT, "cores": cpu_cores(), "kind": "oracle",
-                                    "ms_per_step": r["ms_per_step"], "sample": r["sample"]}
+                                    "extrapolated": leg.extrapolated, "sample": r["sample"]}
+            if not leg.extrapolated:
+                line["cpu_baseline"]["ms_per_step"] = r["ms_per_step"]
         print(json.dumps(line))
     if dist is not None:
         dist.barrier()

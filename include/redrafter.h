@@ -270,6 +270,10 @@ RD_API int redrafter_profile_read(rd_handle* h, int32_t cls, double* ms, double*
 RD_API int redrafter_trace(rd_handle* h, int enable, void* stream);
 RD_API int redrafter_trace_read(rd_handle* h, void* stream, uint64_t* out, int32_t max_launches);
 RD_API int redrafter_trace_bytes(rd_handle* h, double* out, int32_t max_launches);
+/* Same layout: of those weight bytes, the ones each projection launch requests BEFORE its dependency wait (the first
+ * ring-full of stages of every CTA, which stream in under the preceding kernel).  A rate "in place" divides the
+ * remaining bytes by the time after the wait. */
+RD_API int redrafter_trace_prefetched(rd_handle* h, double* out, int32_t max_launches);
 
 /* Self-test of the bounded device-side waits (the paper has no counterpart).  Enqueues one tiny kernel that waits on
  * a hand-off counter value that nothing will ever produce: the wait gives up after its limit (about one second) and
@@ -279,6 +283,11 @@ RD_API int redrafter_selftest_wait(rd_handle* h, void* stream);
 
 /* Number of kernels this handle has launched since it was created (for launch accounting). */
 RD_API int64_t redrafter_launch_count(const rd_handle* h);
+
+/* Packed rows N_b (root + deduplicated draft tokens, Section 3.3) of every sequence in the most recent redrafter_step:
+ * copies n[batch] int32 to the DEVICE buffer `n`, enqueued on `stream`.  The measure of what dynamic tree attention
+ * saves: without it a step verifies 1 + beam_width * beam_length rows per sequence (Figure 5, left). */
+RD_API int redrafter_last_packed_rows(rd_handle* h, void* stream, int32_t* n);
 
 /* Diagnostic (the paper has no counterpart): copies rows [0, rows) of the logits computed by the handle's last
  * forward pass into the DEVICE buffer out[rows][vocab] (fp32), enqueued on `stream`.  After redrafter_ar_step row b

@@ -26,7 +26,8 @@ EXPORTS = ["redrafter_workspace_bytes", "redrafter_kv_bytes", "redrafter_init", 
            "redrafter_accept", "redrafter_step", "redrafter_ar_step", "redrafter_get_state", "redrafter_set_state",
            "redrafter_set_ctx_bound", "redrafter_poll", "redrafter_launch_count", "redrafter_profile",
            "redrafter_profile_read", "redrafter_trace", "redrafter_trace_read", "redrafter_trace_bytes",
-           "redrafter_accept_static", "redrafter_selftest_wait", "redrafter_set_sampling", "redrafter_route_counts", "redrafter_last_logits"]
+           "redrafter_accept_static", "redrafter_selftest_wait", "redrafter_set_sampling", "redrafter_route_counts", "redrafter_last_logits", "redrafter_trace_prefetched",
+           "redrafter_last_packed_rows"]
 
 ROUTES = ("att_rows16", "att_rows16_shallow", "att_rows64", "att_rows128_tc5", "att_key_split", "att_fp32", "gemm_pairs",
           "gemm_one_cta", "gemm_simt")
@@ -96,6 +97,8 @@ def lib():
         L.redrafter_trace_bytes.argtypes = [vp, vp, i32]
         L.redrafter_selftest_wait.argtypes = [vp, vp]
         L.redrafter_last_logits.argtypes = [vp, vp, vp, i32]
+        L.redrafter_trace_prefetched.argtypes = [vp, vp, i32]
+        L.redrafter_last_packed_rows.argtypes = [vp, vp, vp]
         L.redrafter_route_counts.argtypes = [vp, C.POINTER(C.c_int64), i32]
         _lib = L
     return _lib
@@ -287,6 +290,9 @@ class ReDrafter:
         self._ck(self.L.redrafter_get_state(self.h, _stream(), _ptr(ctx), _ptr(root), _ptr(h)))
         return ctx, root, h
 
+    def set_ctx_bound(self, bound):
+        self._ck(self.L.redrafter_set_ctx_bound(self.h, int(bound)))
+
     def set_state(self, ctx=None, root=None, h=None, batch=None, ctx_bound=None):
         batch = self.B if batch is None else batch
         self._ck(self.L.redrafter_set_state(self.h, _stream(), _ptr(ctx), _ptr(root), _ptr(h), batch))
@@ -341,6 +347,21 @@ class ReDrafter:
         buf = (C.c_int64 * len(ROUTES))()
         self._ck(self.L.redrafter_route_counts(self.h, buf, len(ROUTES)))
         return dict(zip(ROUTES, list(buf)))
+
+    def trace_prefetched(self, max_launches=512):
+        """Of trace_bytes, the bytes each projection launch requests before its dependency wait."""
+        import numpy as np
+        buf = np.zeros(max_launches, dtype=np.float64)
+        n = self.L.redrafter_trace_prefetched(self.h, buf.ctypes.data, max_launches)
+        if n < 0:
+            self._ck(-n)
+        return buf[:n]
+
+    def last_packed_rows(self, out=None):
+        """[B] int32 packed rows per sequence of the most recent step (device tensor)."""
+        out = torch.empty(self.B, dtype=torch.int32, device=self.device) if out is None else out
+        self._ck(self.L.redrafter_last_packed_rows(self.h, _stream(), _ptr(out)))
+        return out
 
     def launch_count(self):
         return int(self.L.redrafter_launch_count(self.h))

@@ -90,6 +90,7 @@ struct rd_handle {
   bool use_tc;
   int trace_next;  // next trace slot, -1 = tracing off
   std::vector<double> trace_bytes;  // weight bytes of each traced launch (0: not a projection)
+  std::vector<double> trace_prefetch;  // ... of which requested before the launch's dependency wait
   int tc_grid, tc_smem;
   int tc_pairs;   // CTA pairs of the pair projection kernel that fit the device at once (0: not used)
   int tc_pairs_avail, tc_pairs_min_rows;   // the pairs the device offers; row bound from which launches use them
@@ -303,13 +304,17 @@ int gemm(rd_handle* h, const void* A, int lda, const void* W, int N, int K, cons
       amaps[i] = &ia->second;
     }
     unsigned long long* tr = nullptr;
+    int tr_slot = -1;
     if (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) {
       if ((int)h->trace_bytes.size() < TRACE_SLOTS) h->trace_bytes.assign(TRACE_SLOTS, 0.0);
+      if ((int)h->trace_prefetch.size() < TRACE_SLOTS) h->trace_prefetch.assign(TRACE_SLOTS, 0.0);
       h->trace_bytes[h->trace_next] = (double)N * K * esize(h->dm.dtype);
+      tr_slot = h->trace_next;
       tr = h->ws.trace + (size_t)8 * h->trace_next++;
     }
     CK(h, launch_gemm_tc(&iw->second, amaps, N, K, m_total, m_max, raw, ld_raw, h->ws.tc_partial, h->ws.status,
                          h->tc_grid, pairs, h->tc_smem, tr, out, chain, pair, st));
+    if (tr_slot >= 0) h->trace_prefetch[tr_slot] = tc_last_prefetch_bytes();
     h->route[pairs ? RD_ROUTE_GEMM_PAIRS : RD_ROUTE_GEMM_ONE_CTA]++;
     return RD_OK;
   }
@@ -987,6 +992,7 @@ int redrafter_trace(rd_handle* h, int enable, void* stream) {
     CKRT(h, cudaStreamSynchronize(st));
     h->trace_next = 0;
     h->trace_bytes.assign(TRACE_SLOTS, 0.0);
+    h->trace_prefetch.assign(TRACE_SLOTS, 0.0);
   } else {
     h->trace_next = -1;
   }
@@ -1010,6 +1016,20 @@ int redrafter_trace_bytes(rd_handle* h, double* out, int32_t max_launches) {
   if (n > max_launches) n = max_launches;
   for (int i = 0; i < n; ++i) out[i] = i < (int)h->trace_bytes.size() ? h->trace_bytes[i] : 0.0;
   return n;
+}
+
+int redrafter_trace_prefetched(rd_handle* h, double* out, int32_t max_launches) {
+  if (!h || !out || max_launches < 0) return -RD_ERR_INVALID_ARG;
+  int n = h->trace_next < 0 ? 0 : h->trace_next;
+  if (n > max_launches) n = max_launches;
+  for (int i = 0; i < n; ++i) out[i] = i < (int)h->trace_prefetch.size() ? h->trace_prefetch[i] : 0.0;
+  return n;
+}
+
+int redrafter_last_packed_rows(rd_handle* h, void* stream, int32_t* n) {
+  if (!h || !n) return RD_ERR_INVALID_ARG;
+  CKRT(h, cudaMemcpyAsync(n, h->ws.pk.n, (size_t)h->batch * sizeof(int32_t), cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  return RD_OK;
 }
 
 int redrafter_selftest_wait(rd_handle* h, void* stream) {

@@ -782,6 +782,11 @@ int tc_make_map(void* out_map, const void* ptr, uint64_t rows, uint64_t cols, ui
 
 int tc_weight_box_rows() { return TILE_N; }
 
+// Weight bytes the CTAs of the most recent launch (of this host thread) request BEFORE their dependency wait: the
+// first ring-full of stages.  Measurement aid: an in-place rate must not count them against the time after the wait.
+static thread_local double g_last_prefetch_bytes = 0.0;
+double tc_last_prefetch_bytes() { return g_last_prefetch_bytes; }
+
 // Activation rows per tile for a launch whose row count is at most m_max.
 int tc_pick_mt(int m_max) {
   // One row tile up to 256 rows.  Beyond that the tiles are 256 rows: the bound is a host-side one (batch x rows per
@@ -891,6 +896,10 @@ static cudaError_t launch_gemm_tc2(const void* map_w, const void* const map_a[16
   const bool first = chain && chain->enabled && chain->prev_ptr == nullptr;
   p.cs = chain ? chain->link((unsigned)(2 * pairs)) : ChainSync{nullptr, 0u, nullptr, status, nullptr};
   const size_t smem = (size_t)stages * stage_bytes + overhead;
+  {
+    const long long per_cta = (n_units * p.m_tiles_max) / pairs;   // units of a cluster (each CTA loads one weight tile per unit)
+    g_last_prefetch_bytes = (p.m_tiles_max == 1 || chain) ? 2.0 * pairs * (double)(per_cta < stages ? per_cta : stages) * W_STAGE_BYTES : 0.0;
+  }
   ActMaps am;
   for (int i = 0; i < ACT_MAPS; ++i) am.m[i] = *(const CUtensorMap*)(map_a[i] ? map_a[i] : map_a[0]);
   launch_pairs(first, gemm_tc2_kernel<8>, 2 * pairs, tc_threads(8), smem, st, *(const CUtensorMap*)map_w, am, p);
@@ -940,6 +949,12 @@ cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[16], int N
   const bool first = chain && chain->enabled && chain->prev_ptr == nullptr;
   p.cs = chain ? chain->link((unsigned)grid) : ChainSync{nullptr, 0u, nullptr, status, nullptr};
   const size_t smem = (size_t)p.ring_bytes + overhead;
+  {
+    // (outside the pair mode the kernel may fit more stages than `stages` when few rows are present: a lower bound)
+    const long long per_cta = (n_units * p.m_tiles_max) / grid;
+    g_last_prefetch_bytes = (p.m_tiles_max == 1 || chain) ? (double)grid * (double)(per_cta < stages ? per_cta : stages) *
+                                                            W_STAGE_BYTES * (p.pair ? 2 : 1) : 0.0;
+  }
   ActMaps am;
   for (int i = 0; i < ACT_MAPS; ++i) am.m[i] = *(const CUtensorMap*)(map_a[i] ? map_a[i] : map_a[0]);
   if (p.pair) {

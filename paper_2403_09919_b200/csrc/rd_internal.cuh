@@ -61,6 +61,7 @@ int tc_pick_mt(int m_max);
 size_t tc_partial_floats(int grid, int mt);
 cudaError_t tc_prepare(int* smem_limit_out, int* pairs_out);
 bool tc_use_pairs(int m_max, int N, int grid, int pairs, int min_rows);
+double tc_last_prefetch_bytes();
 cudaError_t launch_gemm_tc(const void* map_w, const void* const map_a[16], int N, int K, const int32_t* m_total, int m_max,
                            float* raw, int ld_raw, float* partial, int32_t* status, int grid, int pairs, int smem_limit,
                            unsigned long long* trace, GemmOut* out_desc, Chain* chain, int pair, cudaStream_t st);

@@ -130,11 +130,3 @@ def plant_beams(continuation, beam_width, beam_length, vocab, rng, p=0.3, rho=0.
         beams[i] = row
     return beams
 
-
-def first_mismatch(beams, continuation):
-    """Closed form for planted beams: per candidate, the index of the first token that
-    differs from the continuation (= its accepted length under greedy acceptance)."""
-    beams = np.asarray(beams)
-    cont = np.asarray(continuation[:beams.shape[1]])
-    neq = beams != cont[None, :]
-    return np.where(neq.any(axis=1), neq.argmax(axis=1), beams.shape[1])

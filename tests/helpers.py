@@ -23,6 +23,15 @@ def micro_model(std=0.25, seed=123, cfg=None):
     return cfg, W, D, w
 
 
+def first_mismatch(beams, continuation):
+    """Closed form for planted beams: per candidate, the index of the first token that differs from the continuation
+    (= its accepted length under greedy acceptance when the continuation is the LLM's own greedy stream)."""
+    beams = np.asarray(beams)
+    cont = np.asarray(continuation[:beams.shape[1]])
+    neq = beams != cont[None, :]
+    return np.where(neq.any(axis=1), neq.argmax(axis=1), beams.shape[1])
+
+
 def read_golden(name):
     path = os.path.join(ROOT, "tests", "golden", name)
     with open(path) as f:

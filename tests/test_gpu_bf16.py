@@ -9,7 +9,7 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import Rig, check_beams_within, dev, tolerant_beam_search, top2_gap
+from helpers import check_beams_within, dev, first_mismatch, Rig, tolerant_beam_search, top2_gap
 from oracle import redrafter_oracle as ora
 from paper_2403_09919_b200 import synth
 
@@ -336,7 +336,7 @@ def test_free_running_lossless_up_to_the_first_near_tie():
         planted = synth.plant_beams(ref[len(spec):len(spec) + L], BW, L, cfg["vocab"], rng, p=0.3, rho=0.3)
         rig.eng.step(dev(planted[None]), out)
         a = int(out.n_accept[0])
-        assert a == synth.first_mismatch(planted, ref[len(spec):len(spec) + L]).max()
+        assert a == first_mismatch(planted, ref[len(spec):len(spec) + L]).max()
         spec.extend(out.tokens[0, :a + 1].tolist())
         steps += 1
     rig.eng.poll()

@@ -25,7 +25,7 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import Rig, check_against_storage_noise, dev, top2_gap
+from helpers import check_against_storage_noise, dev, first_mismatch, Rig, top2_gap
 from oracle import redrafter_oracle as ora
 from paper_2403_09919_b200 import synth
 
@@ -179,7 +179,7 @@ def test_verification_and_autoregressive_paths_differ_by_storage_noise_only():
         argmax, hidden, logits = rig.eng.verify(pk, want_logits=True)
         out = rig.eng.accept(beams_d, pk, argmax, hidden)
         rig.eng.poll()
-        match = synth.first_mismatch(planted, stream[pos + 1:pos + 1 + L])
+        match = first_mismatch(planted, stream[pos + 1:pos + 1 + L])
         best = int(match.argmax())
         up = pk.unpack[0, best].cpu().numpy()
         lg = logits[0].cpu().numpy()

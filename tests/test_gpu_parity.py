@@ -17,7 +17,7 @@ TOL_FP32 = 2e-3
 EPS_SCORE = 2e-5     # fp32 drafter scores against the fp64 oracle: measured 3e-6 at scores of about -25
 
 
-from helpers import Rig, check_beams_within, dev, tolerant_beam_search, top2_gap  # noqa: E402
+from helpers import check_beams_within, dev, first_mismatch, Rig, tolerant_beam_search, top2_gap  # noqa: E402
 
 
 @pytest.fixture(scope="module")
@@ -257,7 +257,7 @@ def test_full_tiny_config_32_steps_lossless_free_running(rig):
         planted = synth.plant_beams(ar_gpu[len(spec):len(spec) + L], BW, L, cfg["vocab"], rng, p=0.3)
         rig.eng.step(dev(planted[None]), out)
         a = int(out.n_accept[0])
-        assert a == synth.first_mismatch(planted, ar_gpu[len(spec):len(spec) + L]).max()
+        assert a == first_mismatch(planted, ar_gpu[len(spec):len(spec) + L]).max()
         spec.extend(out.tokens[0, :a + 1].tolist())
         acc.append(a)
     rig.eng.poll()

@@ -6,7 +6,7 @@ import itertools
 import numpy as np
 import torch
 
-from helpers import MICRO, micro_model
+from helpers import first_mismatch, MICRO, micro_model
 from oracle import redrafter_oracle as ora
 from paper_2403_09919_b200 import synth
 
@@ -218,7 +218,7 @@ def test_lossless_drafted_and_planted_and_cache():
     pos = 1
     for a in acc:
         b = synth.plant_beams(ar[pos:pos + 4], 4, 4, cfg["vocab"], rng, p=0.3, rho=0.5)
-        assert a == synth.first_mismatch(b, ar[pos:pos + 4]).max()
+        assert a == first_mismatch(b, ar[pos:pos + 4]).max()
         pos += a + 1
     # compaction: the cache after speculative decoding equals the AR cache over the same tokens
     n = min(ctx, ctx_ar)

@@ -3,7 +3,7 @@ import itertools
 
 import numpy as np
 
-from helpers import read_golden
+from helpers import first_mismatch, read_golden
 from oracle import redrafter_oracle as ora
 
 
@@ -151,7 +151,7 @@ def test_accept_brute_force_and_planted_closed_form():
                 if (aug[i, 1:j + 1] == cont[:j]).all():
                     am[p["unpack"][i, j]] = cont[j]
         a, best, emitted = ora.accept_greedy(beams, p["unpack"], am)
-        ai = synth.first_mismatch(beams, cont)
+        ai = first_mismatch(beams, cont)
         assert a == ai.max()
         assert best == int(np.argmax(ai))               # lowest index among the longest
         assert emitted == cont[:a + 1].tolist()
