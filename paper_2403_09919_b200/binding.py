@@ -12,7 +12,8 @@ import os
 
 import torch
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libredrafter.so")
+# REDRAFTER_LIB: another build of the same library (a measurement build with extra defines, see build.py)
+_LIB_PATH = os.environ.get("REDRAFTER_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libredrafter.so")
 _lib = None
 
 RD_DTYPE = {"fp32": 0, "bf16": 1}

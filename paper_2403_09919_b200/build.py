@@ -12,6 +12,13 @@ CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "build")
 LIB = os.path.join(PKG, "libredrafter.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+# Measurement builds: RD_BUILD_DEFINES="-DRD_PROBE_EMPTY_BODIES" with RD_BUILD_TAG=probe writes libredrafter_probe.so
+# (objects under build_probe/); the binding loads it when REDRAFTER_LIB names it.  The default build defines nothing.
+DEFINES = os.environ.get("RD_BUILD_DEFINES", "").split()
+TAG = os.environ.get("RD_BUILD_TAG", "")
+if TAG:
+    OBJ = os.path.join(PKG, "build_" + TAG)
+    LIB = os.path.join(PKG, f"libredrafter_{TAG}.so")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 
@@ -35,7 +42,7 @@ def build(force=False, verbose=False):
     for src in sources():
         obj = os.path.join(OBJ, src[:-3] + ".o")
         if force or _stale(obj, [os.path.join(CSRC, src)] + headers):
-            cmd = [NVCC, *FLAGS, "-c", os.path.join(CSRC, src), "-o", obj]
+            cmd = [NVCC, *FLAGS, *DEFINES, "-c", os.path.join(CSRC, src), "-o", obj]
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
             jobs.append(cmd)

@@ -59,6 +59,11 @@ __global__ void __launch_bounds__(128) attention_tc_kernel(const float* __restri
   unsigned long long t_dbg[6] = {0, 0, 0, 0, 0, 0};
   RD_STAMP(0);
   chain_begin(cs);
+#ifdef RD_PROBE_EMPTY_BODIES   // ceiling probe (a build flag, never in the shipped library): keep the hand-off, drop the work
+  chain_wait_cta(cs);
+  chain_exit(cs);
+  return;
+#endif
   // Launched inside a chain, the kernel may read before its wait whatever the launches ahead of the chain
   // wrote: the row tables, the tree mask and the cache entries of earlier steps.  Only Q and the K/V of
   // this pass's own rows come from the kernel right before it.
