@@ -49,6 +49,7 @@ struct Workspace {
   int32_t *cand_idx, *hist_a, *hist_b, *one_b, *one_r;
   float *seg_max, *seg_sum, *seg_val;   // two-kernel selection: per (row, segment) maximum, sum, candidates
   int32_t* seg_idx;
+  unsigned long long* sel_top;          // [rows][BW] keys of every row's BW best continuations
   // tensor-core projection scratch
   float* tc_partial;
   // tensor-core attention scratch
@@ -222,6 +223,7 @@ void carve(Bump& bp, const Dims& dm, int m_cap, Workspace* w) {
   w->dlogits = bp.take<float>((size_t)R * dm.V);
   w->seg_max = bp.take<float>((size_t)R * 32); w->seg_sum = bp.take<float>((size_t)R * 32);
   w->seg_val = bp.take<float>((size_t)R * 512); w->seg_idx = bp.take<int32_t>((size_t)R * 512);
+  w->sel_top = bp.take<unsigned long long>((size_t)R * dm.BW);
   w->lse = bp.take<float>(R); w->cand_val = bp.take<float>((size_t)R * dm.BW);
   w->score_a = bp.take<float>(R); w->score_b = bp.take<float>(R);
   w->cand_idx = bp.take<int32_t>((size_t)R * dm.BW); w->hist_a = bp.take<int32_t>((size_t)R * dm.L);
@@ -509,8 +511,8 @@ int do_draft(rd_handle* h, cudaStream_t st, int32_t* beams, float* scores) {
     CKP(h, PROF_DRAFT_SMALL, launch_draft_select(dm.dtype, g, call, w.lse, w.cand_val, w.cand_idx, sc_in, sc_out, hi_in, hi_out,
                                                  h->w.tok_emb, w.x0_f, dm.dh, w.se_t, dm, B, beams, scores, w.sel_counters, mt,
                                                  (h->trace_next >= 0 && h->trace_next < TRACE_SLOTS) ? w.trace + (size_t)8 * h->trace_next++ : nullptr,
-                                                 SelectScratch{h->use_tc ? w.seg_max : nullptr, w.seg_sum, w.seg_val, w.seg_idx, h->tc_grid}, ch, st));
-    if (h->use_tc && draft_select_segments(dm, rows, h->tc_grid) > 0) h->launches++;   // that selection is two launches
+                                                 SelectScratch{h->use_tc ? w.seg_max : nullptr, w.seg_sum, w.seg_val, w.seg_idx, h->tc_grid, w.sel_top}, ch, st));
+    if (h->use_tc && draft_select_segments(dm, rows, h->tc_grid) > 0) h->launches += 2;   // that selection is three launches
     float* tf = sc_in; sc_in = sc_out; sc_out = tf;
     int32_t* ti = hi_in; hi_in = hi_out; hi_out = ti;
   }

@@ -581,10 +581,71 @@ __global__ void __maxnreg__(88) draft_seg_kernel(GemmOut proj, int V, int BW, in
   chain_exit(cs);
 }
 
+// Second of the three selection kernels: one CTA per drafter row.  The row's S segments each bring their maximum,
+// their sum of exponentials and their BW best candidates; the CTA forms the row's log-sum-exp and ranks the S * BW
+// candidates by counting (every key is unique: the index is part of it), so the BW best leave in order with one pass
+// over shared memory per candidate instead of BW rounds of a maximum search.  Output: top[r][p], p < BW, the keys
+// (cumulative score, flat index row-in-sequence * V + token) of the row's BW best continuations, best first; 0 where a
+// row has fewer candidates.  Without this kernel every one of a sequence's BW merging CTAs repeated this work for all
+// BW rows (178 us per call at beam width 64).
+constexpr int ROWTOP_THREADS = 256;
+static_assert(SEG_MAX_CAND <= 2 * ROWTOP_THREADS, "two candidates per thread");
+__global__ void __launch_bounds__(ROWTOP_THREADS) draft_rowtop_kernel(int S, int call, int BW, int V, const float* __restrict__ seg_max,
+                                                                      const float* __restrict__ seg_sum, const float* __restrict__ seg_val,
+                                                                      const int32_t* __restrict__ seg_idx, const float* __restrict__ score_in,
+                                                                      unsigned long long* __restrict__ top, ChainSync cs) {
+  chain_enter(cs);
+  __shared__ unsigned long long keys[SEG_MAX_CAND];
+  __shared__ unsigned long long out[MRG_MAX_BW];
+  __shared__ float s_lse;
+  const int r = blockIdx.x;
+  const int rr = call == 1 ? 0 : r % BW;     // the row's index inside its sequence (call 1: one row per sequence)
+  const int n = S * BW;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int c = threadIdx.x; c < n; c += ROWTOP_THREADS) {
+    const float cv = __ldcg(seg_val + (size_t)r * n + c);
+    const int ci = __ldcg(seg_idx + (size_t)r * n + c);
+    keys[c] = ci == 0x7fffffff ? 0ull : cand_key(cv, ci);
+  }
+  if (threadIdx.x < BW) out[threadIdx.x] = 0ull;
+  if (warp == 0) {
+    // log-sum-exp of the row from its segments (S <= 32: one per lane)
+    const float sm = lane < S ? __ldcg(seg_max + (size_t)r * S + lane) : -INFINITY;
+    const float ss = lane < S ? __ldcg(seg_sum + (size_t)r * S + lane) : 0.f;
+    float m = sm;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    float sum = sm > -INFINITY ? ss * __expf(sm - m) : 0.f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if (lane == 0) s_lse = m + logf(sum);
+  }
+  __syncthreads();
+  const float base = call == 1 ? 0.f : __ldcg(score_in + r);
+  const float row_lse = s_lse;
+  // a thread ranks its two candidates (c and c + 256; SEG_MAX_CAND = 2 * ROWTOP_THREADS) in one pass: every key read
+  // from shared memory (a broadcast) serves both comparisons, eight reads in flight at a time
+  {
+    const int c0 = threadIdx.x, c1 = threadIdx.x + ROWTOP_THREADS;
+    const unsigned long long k0 = c0 < n ? keys[c0] : 0ull, k1 = c1 < n ? keys[c1] : 0ull;
+    int r0 = 0, r1 = 0;
+#pragma unroll 8
+    for (int j = 0; j < n; ++j) {
+      const unsigned long long x = keys[j];
+      r0 += x > k0 ? 1 : 0;
+      r1 += x > k1 ? 1 : 0;
+    }
+    if (k0 != 0ull && r0 < BW) out[r0] = cand_key(base + (key_value(k0) - row_lse), rr * V + key_index(k0));
+    if (k1 != 0ull && r1 < BW) out[r1] = cand_key(base + (key_value(k1) - row_lse), rr * V + key_index(k1));
+  }
+  __syncthreads();
+  if (threadIdx.x < BW) top[(size_t)r * BW + threadIdx.x] = out[threadIdx.x];
+  chain_exit(cs);
+}
+
 template <typename T, bool WIDE>
 __global__ void __launch_bounds__(MRG_THREADS) draft_merge_kernel(
-    int S, int call, const float* __restrict__ seg_max, const float* __restrict__ seg_sum, const float* __restrict__ seg_val,
-    const int32_t* __restrict__ seg_idx, const float* __restrict__ score_in, float* __restrict__ score_out,
+    int call, const unsigned long long* __restrict__ top_g, float* __restrict__ score_out,
     const int32_t* __restrict__ hist_in, int32_t* __restrict__ hist_out, const T* __restrict__ emb,
     const float* __restrict__ s_new_f, int ld_s, T* __restrict__ se_t, Dims dm, int32_t* __restrict__ beams_out,
     float* __restrict__ scores_out, unsigned long long* dbg, ChainSync cs) {
@@ -599,49 +660,10 @@ __global__ void __launch_bounds__(MRG_THREADS) draft_merge_kernel(
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int rows = call == 1 ? 1 : BW;
   const int row0 = call == 1 ? b : b * BW;
-  const int n = S * BW;
+  // the rows' BW best continuations each (draft_rowtop_kernel), in row order
+  for (int c = threadIdx.x; c < rows * BW; c += MRG_THREADS) top[c] = __ldcg(top_g + (size_t)row0 * BW + c);
   if constexpr (WIDE) {
-    // beam widths above 16: every thread keeps its share of the candidates in registers for all rounds
     __shared__ unsigned long long shk[2][MRG_THREADS / 32];
-    constexpr int KPL = SEG_MAX_CAND / 32;   // keys per lane: the candidates of a row stay in registers for all rounds
-    for (int rr = warp; rr < rows; rr += MRG_THREADS / 32) {
-      const int r = row0 + rr;
-      // every load of the row first: segment maxima and sums (S <= 32: one per lane), candidates, the row's score
-      const float sm = lane < S ? __ldcg(seg_max + (size_t)r * S + lane) : -INFINITY;
-      const float ss = lane < S ? __ldcg(seg_sum + (size_t)r * S + lane) : 0.f;
-      const float base = call == 1 ? 0.f : __ldcg(score_in + r);
-      unsigned long long key[KPL];
-  #pragma unroll
-      for (int j = 0; j < KPL; ++j) {
-        const int c = lane + 32 * j;
-        key[j] = 0ull;
-        if (c < n) {
-          const float cv = __ldcg(seg_val + (size_t)r * n + c);
-          const int ci = __ldcg(seg_idx + (size_t)r * n + c);
-          key[j] = ci == 0x7fffffff ? 0ull : cand_key(cv, ci);
-        }
-      }
-      // log-sum-exp of the row from its segments
-      float m = sm;
-  #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-      float sum = sm > -INFINITY ? ss * __expf(sm - m) : 0.f;
-  #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-      const float row_lse = m + logf(sum);
-      unsigned long long pv = ~0ull;
-      for (int p = 0; p < BW; ++p) {
-        unsigned long long mine = 0ull;
-  #pragma unroll
-        for (int j = 0; j < KPL; ++j) mine = max(mine, key[j] < pv ? key[j] : 0ull);
-        mine = warp_max_key(mine);
-        if (lane == 0) {
-          const int bi = key_index(mine);
-          top[rr * BW + p] = cand_key(base + (key_value(mine) - row_lse), rr * V + (bi == 0x7fffffff ? 0 : bi));
-        }
-        pv = mine;
-      }
-    }
     __syncthreads();
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[2]));
     // the beam of rank kout among the rows * BW candidates, (score desc, flat index asc): all threads hold their share
@@ -668,47 +690,10 @@ __global__ void __launch_bounds__(MRG_THREADS) draft_merge_kernel(
         for (int w = 0; w < MRG_THREADS / 32; ++w) best = max(best, shk[p & 1][w]);
         pv = best;
       }
-      if (threadIdx.x == 0) s_win = Cand{key_value(pv), key_index(pv)};
+      if (threadIdx.x == 0) s_win = Cand{key_value(pv), pv == 0ull ? 0 : key_index(pv)};   // (fewer candidates than beams cannot happen: BW <= V)
     }
   } else {
-    // narrow beams: a row has a few candidates per lane and the final ranking a few per lane of one warp
-    __shared__ unsigned long long wbuf[MRG_THREADS / 32][SEG_MAX_CAND];
-    for (int rr = warp; rr < rows; rr += MRG_THREADS / 32) {
-      const int r = row0 + rr;
-      // every load of the row first: segment maxima and sums (S <= 32: one per lane), candidates, the row's score
-      const float sm = lane < S ? __ldcg(seg_max + (size_t)r * S + lane) : -INFINITY;
-      const float ss = lane < S ? __ldcg(seg_sum + (size_t)r * S + lane) : 0.f;
-      const float base = call == 1 ? 0.f : __ldcg(score_in + r);
-      for (int c = lane; c < n; c += 32) {
-        const float cv = __ldcg(seg_val + (size_t)r * n + c);
-        const int ci = __ldcg(seg_idx + (size_t)r * n + c);
-        wbuf[warp][c] = ci == 0x7fffffff ? 0ull : cand_key(cv, ci);
-      }
-      // log-sum-exp of the row from its segments
-      float m = sm;
-  #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-      float sum = sm > -INFINITY ? ss * __expf(sm - m) : 0.f;
-  #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-      const float row_lse = m + logf(sum);
-      __syncwarp();
-      unsigned long long pv = ~0ull;
-      for (int p = 0; p < BW; ++p) {
-        unsigned long long mine = 0ull;
-        for (int c = lane; c < n; c += 32) {
-          const unsigned long long x = wbuf[warp][c];
-          mine = max(mine, x < pv ? x : 0ull);
-        }
-        mine = warp_max_key(mine);
-        if (lane == 0) {
-          const int bi = key_index(mine);
-          top[rr * BW + p] = cand_key(base + (key_value(mine) - row_lse), rr * V + (bi == 0x7fffffff ? 0 : bi));
-        }
-        pv = mine;
-      }
-      __syncwarp();
-    }
+    // narrow beams: the final ranking has a few candidates per lane of one warp
     __syncthreads();
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[2]));
     // the beam of rank kout among the rows * BW candidates, (score desc, flat index asc)
@@ -723,7 +708,7 @@ __global__ void __launch_bounds__(MRG_THREADS) draft_merge_kernel(
         }
         pv = warp_max_key(mine);
       }
-      if (lane == 0) s_win = Cand{key_value(pv), key_index(pv)};
+      if (lane == 0) s_win = Cand{key_value(pv), pv == 0ull ? 0 : key_index(pv)};   // (fewer candidates than beams cannot happen: BW <= V)
     }
   }
   __syncthreads();
@@ -813,19 +798,23 @@ cudaError_t launch_draft_select(int dtype, const GemmOut& proj, int call, float*
 #undef RD_SEG_LAUNCH
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    // the rows' BW best continuations, one CTA per row
+    const ChainSync c15 = chain ? chain->link((unsigned)rows, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
+    launch_pdl(draft_rowtop_kernel, rows, ROWTOP_THREADS, 0, st, S, call, dm.BW, dm.V, (const float*)sc.seg_max, (const float*)sc.seg_sum,
+               (const float*)sc.seg_val, (const int32_t*)sc.seg_idx, score_in, sc.top, c15);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
     dim3 g2(dm.BW, B);
     const ChainSync c2 = chain ? chain->link(g2.x * g2.y) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
     const size_t top_bytes = (size_t)(call == 1 ? 1 : dm.BW) * dm.BW * sizeof(unsigned long long);
     if (dm.BW > MRG_NARROW_BW) {
       constexpr bool WIDE_ = true;
-      RD_DISPATCH(dtype, launch_pdl(draft_merge_kernel<T, WIDE_>, g2, MRG_THREADS, top_bytes, st, S, call, (const float*)sc.seg_max,
-                                    (const float*)sc.seg_sum, (const float*)sc.seg_val, (const int32_t*)sc.seg_idx, score_in,
+      RD_DISPATCH(dtype, launch_pdl(draft_merge_kernel<T, WIDE_>, g2, MRG_THREADS, top_bytes, st, call, (const unsigned long long*)sc.top,
                                     score_out, hist_in, hist_out, (const T*)emb, s_new_f, ld_s, (T*)se_t, dm, beams_out,
                                     scores_out, dbg, c2));
     } else {
       constexpr bool WIDE_ = false;
-      RD_DISPATCH(dtype, launch_pdl(draft_merge_kernel<T, WIDE_>, g2, MRG_THREADS, top_bytes, st, S, call, (const float*)sc.seg_max,
-                                    (const float*)sc.seg_sum, (const float*)sc.seg_val, (const int32_t*)sc.seg_idx, score_in,
+      RD_DISPATCH(dtype, launch_pdl(draft_merge_kernel<T, WIDE_>, g2, MRG_THREADS, top_bytes, st, call, (const unsigned long long*)sc.top,
                                     score_out, hist_in, hist_out, (const T*)emb, s_new_f, ld_s, (T*)se_t, dm, beams_out,
                                     scores_out, dbg, c2));
     }

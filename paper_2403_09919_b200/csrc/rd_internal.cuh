@@ -118,6 +118,7 @@ struct SelectScratch {
   float *seg_max, *seg_sum, *seg_val;   // [rows][32], [rows][32], [rows][512]
   int32_t* seg_idx;                     // [rows][512]
   int grid_hint;                        // CTAs to aim for (the SM count)
+  unsigned long long* top;              // [rows][BW] keys of every row's BW best continuations
 };
 int draft_select_segments(const Dims& dm, int rows, int grid_hint);
 cudaError_t launch_draft_select(int dtype, const GemmOut& proj, int call, float* lse, float* val, int32_t* idx,
