@@ -326,12 +326,12 @@ def run_sweep(args, cfg):
             c = dict(cfg, beam_width=BW, max_batch=B, prompt_len=args.sweep_prompt)
             need = args.warmup + args.steps
             c["max_ctx"] = args.sweep_prompt + (need + 2) * (L + 1) + 2 + BW * L
-            eng = binding.ReDrafter(c, w, device=device)
+            eng = binding.ReDrafter(c, w, device=device, flags=binding.RD_FLAG_NO_TREE if args.flat else 0)
             prompts = synth.make_prompts(c, B, seed=c.get("seed", 0))
             out = binding.AcceptOut(B, L, device)
             eng.prefill(prompts)
             beams, _ = eng.draft()
-            n_rows = int(eng.pack(beams).n.sum().item())       # packed rows of a typical step (the drafter's own beams)
+            n_rows = int(eng.pack(beams).n.sum().item())       # rows of a typical step (the drafter's own beams)
             for _ in range(args.warmup):
                 eng.step(None, out)
 
@@ -344,7 +344,7 @@ def run_sweep(args, cfg):
             es = 2
             flops = 2.0 * n_rows * (sb["llm"] / es) + 2.0 * (B * BW) * (sb["drafter"] / es) + 4.0 * n_rows * ctx * c["d_model"] * c["n_layers"]
             t_bw, t_tc = sb["total"] / (peak_bw * 1e9) * 1e3, flops / (peak_tf * 1e12) * 1e3
-            row = {"sweep": True, "beam_width": BW, "batch": B, "packed_rows": n_rows, "ms_per_step": ms,
+            row = {"sweep": True, "tree_attention": not args.flat, "beam_width": BW, "batch": B, "packed_rows": n_rows, "ms_per_step": ms,
                    "algorithmic_gb": sb["total"] / 1e9, "dense_tflop": flops / 1e12, "hbm_bound_ms": t_bw, "tensor_bound_ms": t_tc,
                    "roofline_ms": max(t_bw, t_tc), "frac_of_roofline": max(t_bw, t_tc) / ms,
                    "bound": "hbm" if t_bw >= t_tc else "tensor"}
@@ -424,6 +424,7 @@ def main():
     ap.add_argument("--sweep-bw", default="1,4,8,16,32")
     ap.add_argument("--sweep-batch", default="1,2,4,8,16")
     ap.add_argument("--sweep-prompt", type=int, default=256)
+    ap.add_argument("--flat", action="store_true", help="sweep without dynamic tree attention: every candidate sends all its tokens")
     ap.add_argument("--temperature", type=float, default=0.0,
                     help="> 0: the LLM's tokens are draws (Gumbel-max, counter-based noise) instead of greedy; the paper's "
                          "headline numbers and this benchmark's default are temperature 0")
