@@ -8,14 +8,18 @@
 //               chunk's softmax);
 //   softmax     four threads per query row (= TMEM lane), a quarter of the chunk's keys each: scale, mask, running
 //               maximum and sum in registers (base 2), P written back to tensor memory as packed bf16 (two buffers, so
-//               a chunk's probabilities are formed while the previous chunk's P V runs), O in tensor memory rescaled in
-//               place when a row's maximum moved;
+//               a chunk's probabilities are formed while the previous chunk's P V runs);
+//   correction  two more threads per query row scale O in tensor memory when the row's maximum moved, between the previous
+//               chunk's P V and this one's -- off the softmax threads' path, which publish the factor before they
+//               exponentiate (measured: with the rescale inside the softmax loop a chunk took 1.7 us, 0.5 us of it
+//               waiting for the previous P V);
 //   O += P V    tcgen05.mma with A = P read from tensor memory (8 packed columns per 16 keys), B = V chunk as it lies
 //               in the cache ([key][dim], i.e. MN-major for this product: leading byte offset = one 64-dim box of the
 //               chunk, stride byte offset = 8 keys, 2048 bytes per 16 keys).
 // Tensor memory: columns 0..255 the two score buffers, 256..383 O, 384..511 the two P buffers.
 // Roles: warp 0 lane 0 = TMA producer (K and V rings of two chunks), warp 1 lane 0 = MMA issuer (warp 1 owns the tensor
-// memory), warps 2..9 = softmax and output.  Every wait is bounded (one second): on expiry the CTA raises
+// memory; the whole warp runs the issue loop and an elected lane issues, see there),
+// warps 2..17 = softmax and output, warps 18..25 = correction.  Every wait is bounded (one second): on expiry the CTA raises
 // DEV_ERR_TIMEOUT, lets its copies land, frees its tensor memory and leaves.
 //
 // The chunk's keys past a row's extent are masked by selection, never by arithmetic, and their V rows are multiplied by
@@ -35,7 +39,9 @@ constexpr int T5_HD = 128;
 constexpr int T5_STAGES = 2;      // K and V chunks in flight
 constexpr int T5_PARTS = 4;        // softmax threads per query row (each a part of the chunk's keys and of the head dimensions)
 constexpr int T5_SOFT = 128 * T5_PARTS;
-constexpr int T5_THREADS = 64 + T5_SOFT;
+constexpr int T5_CORR_PARTS = 2;  // correction threads per query row (each half of the head dimensions)
+constexpr int T5_CORR = 128 * T5_CORR_PARTS;
+constexpr int T5_THREADS = 64 + T5_SOFT + T5_CORR;
 constexpr uint32_t T5_BLOCK = 128 * 128;            // bytes of one 64-column block of 128 rows (128 B per row)
 constexpr uint32_t T5_TILE = 2 * T5_BLOCK;          // Q tile, K chunk, V chunk, P tile: 32 KB each
 constexpr unsigned long long T5_WAIT_NS = 1000000000ull;
@@ -189,14 +195,15 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
   uint8_t* gen = smem_raw + (base - raw);                 // generic pointer to the same place
   const uint32_t sQ = base, sK = sQ + T5_TILE, sV = sK + T5_STAGES * T5_TILE;
   const uint32_t bar0 = sV + T5_STAGES * T5_TILE;
-  enum { Q_FULL = 0, K_FULL = 1, V_FULL = 3, K_EMPTY = 5, V_EMPTY = 7, S_FULL = 9, S_EMPTY = 11, P_FULL = 13, P_EMPTY = 15, X_FULL = 17, N_BARS = 18 };
+  enum { Q_FULL = 0, K_FULL = 1, V_FULL = 3, K_EMPTY = 5, V_EMPTY = 7, S_FULL = 9, S_EMPTY = 11, P_FULL = 13, P_EMPTY = 15, X_FULL = 17, C_FULL = 18, O_READY = 20, N_BARS = 22 };
   auto bar = [&](int i) { return bar0 + 8u * i; };
   uint8_t* misc = gen + (bar0 - base) + 8u * 32;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
   int32_t* s_ncache = reinterpret_cast<int32_t*>(misc + 16);              // [T5_ROWS]
-  float* s_red = reinterpret_cast<float*>(misc + 16 + T5_ROWS * 4);       // [2][2][T5_ROWS] row maxima of the halves, [2][T5_ROWS] their sums
-  uint32_t* s_mask = reinterpret_cast<uint32_t*>(misc + 16 + T5_ROWS * 4 + 3 * T5_PARTS * T5_ROWS * 4);   // [T5_ROWS][MW]
+  float* s_red = reinterpret_cast<float*>(misc + 16 + T5_ROWS * 4);       // [2][PARTS][T5_ROWS] row maxima of the parts, [PARTS][T5_ROWS] their sums
+  float* s_corr = s_red + 3 * T5_PARTS * T5_ROWS;                         // [2][T5_ROWS] factor by which chunk c scales the row's running output
+  uint32_t* s_mask = reinterpret_cast<uint32_t*>(s_corr + 2 * T5_ROWS);   // [T5_ROWS][MW]
 
   // Tensor memory first (512 columns: two score buffers and the output), before the dependents may start.
   if (warp == 1) {
@@ -220,6 +227,9 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
     }
     for (int s = 0; s < 2; ++s) { mbar_init(bar(P_FULL + s), T5_SOFT / 32); mbar_init(bar(P_EMPTY + s), 1); }
     mbar_init(bar(X_FULL), T5_SOFT / 32);
+    // (two of each, by chunk parity: the softmax and correction warps can be a chunk ahead of the warp that waits --
+    // a single barrier could then complete two phases between two looks of its waiter, which reads as "not yet")
+    for (int s = 0; s < 2; ++s) { mbar_init(bar(C_FULL + s), 4); mbar_init(bar(O_READY + s), T5_CORR / 32); }   // C_FULL: the four warps that hold part 0 of their rows
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -250,25 +260,47 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
   if (warp == 0) {
     // ===================== TMA producer =====================
     if (lane == 0 && n_chunks > 0) {
-      if (early) chain_wait_thread(p.cs);
-      chain_fence_async_reads();   // this pass's keys and values were written with ordinary stores by the rotary kernel
       const int key_row0 = (b * dm.H + h) * dm.max_ctx;   // first row of this (sequence, head) in the cache plane
       bool ok = true;
-      for (int c = 0; c < n_chunks && ok; ++c) {
+      auto load_k = [&](int c) {
         const int s = c & 1;
-        const uint32_t ph = (c >> 1) & 1;
-        if (c >= T5_STAGES) {
-          if (!mbar_wait(bar(K_EMPTY + s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-        }
         mbar_expect_tx(bar(K_FULL + s), T5_TILE);
         tma_load_2d(sK + s * T5_TILE, &map_k, bar(K_FULL + s), 0, key_row0 + c * T5_KEYS);
         tma_load_2d(sK + s * T5_TILE + T5_BLOCK, &map_k, bar(K_FULL + s), 64, key_row0 + c * T5_KEYS);
-        if (c >= T5_STAGES) {
-          if (!mbar_wait(bar(V_EMPTY + s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-        }
+      };
+      auto load_v = [&](int c) {
+        const int s = c & 1;
         mbar_expect_tx(bar(V_FULL + s), T5_TILE);
         tma_load_2d(sV + s * T5_TILE, &map_v, bar(V_FULL + s), 0, key_row0 + c * T5_KEYS);
         tma_load_2d(sV + s * T5_TILE + T5_BLOCK, &map_v, bar(V_FULL + s), 64, key_row0 + c * T5_KEYS);
+      };
+      // Chunks that hold only keys of earlier passes (tree: the context; causal: everything before the slot of the
+      // sequence's first row of this pass) do not depend on the launch before this one: requested before the wait.
+      int pre_k = 0, pre_v = 0;
+      if (early) {
+        const int const_keys = tree ? tree_base : p.rt.n_cache[seq_row0] - 1;
+        while (pre_k < 2 && pre_k < n_chunks && (pre_k + 1) * T5_KEYS <= const_keys) load_k(pre_k++);
+        if (pre_k > 0) { load_v(0); pre_v = 1; }
+        chain_wait_thread(p.cs);
+      }
+      chain_fence_async_reads();   // this pass's keys and values were written with ordinary stores by the rotary kernel
+      // K runs two chunks ahead (its slot is free once the scores of the chunk before last exist), V one (its slot is
+      // free once the chunk before last has been added to the output, which is later): the order of the requests follows
+      // the order in which the slots come free, so that no request waits behind one whose slot is still in use.
+      for (int c = pre_k; c < 2 && c < n_chunks; ++c) load_k(c);
+      for (int c = 0; c < n_chunks && ok; ++c) {
+        const int s = c & 1;
+        const uint32_t ph = (c >> 1) & 1;
+        if (c >= pre_v) {
+          if (c >= T5_STAGES) {
+            if (!mbar_wait(bar(V_EMPTY + s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+          }
+          load_v(c);
+        }
+        if (c + 2 < n_chunks) {
+          if (!mbar_wait(bar(K_EMPTY + s), ph, abort_flag, p.status)) { ok = false; break; }   // Q K^T of chunk c is done
+          load_k(c + 2);
+        }
       }
       if (!ok || *abort_flag) {  // give the copies already issued time to land before the CTA's shared memory is released
         const unsigned long long t0 = now_ns();
@@ -277,23 +309,40 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
     }
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
-    if (lane == 0 && n_chunks > 0) {
+    // The WHOLE warp runs this loop (waits, descriptor arithmetic), and one elected lane issues: values that are the
+    // same in every lane stay in the uniform datapath, from which the MMA instruction takes its descriptors.  With a
+    // single active lane the compiler cannot know that and moves every descriptor across per MMA -- a dozen extra
+    // instructions in a warp that gets only every seventh issue slot beside the softmax warps (measured: 80 ns per
+    // MMA issued against 39 ns this way; the MMA itself takes 35 ns).
+    if (n_chunks > 0) {
+      uint32_t leader;
+      asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(leader));
       const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(T5_KEYS >> 3) << 17) | ((uint32_t)(T5_ROWS >> 4) << 24);
       const uint32_t idesc_pv = idesc_qk | (1u << 16);   // second operand MN-major; N = 128 head dimensions
-      bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag, p.status);
+      auto wait_warp = [&](uint32_t b, uint32_t parity) {
+        return __all_sync(0xffffffffu, mbar_wait(b, parity, abort_flag, p.status)) != 0;
+      };
+      bool ok = wait_warp(bar(Q_FULL), 0);
+      // descriptors once; a k-step adds a constant to the start-address field (16-byte units)
+      const uint64_t q_desc = desc_kmajor(sQ);
       auto issue_qk = [&](int c) {
         const int s = c & 1;
         const uint32_t ph = (c >> 1) & 1;
-        if (!mbar_wait(bar(K_FULL + s), ph, abort_flag, p.status)) return false;
-        if (!mbar_wait(bar(S_EMPTY + s), ph ^ 1u, abort_flag, p.status)) return false;
+        if (!wait_warp(bar(K_FULL + s), ph)) return false;
+        if (!wait_warp(bar(S_EMPTY + s), ph ^ 1u)) return false;
         tc_fence_after();
+        const uint64_t kd = desc_kmajor(sK + (uint32_t)s * T5_TILE);
+        const uint32_t d = tmem + (uint32_t)s * T5_KEYS;
+        if (leader) {
 #pragma unroll
-        for (int kk = 0; kk < T5_HD / 16; ++kk) {
-          const uint32_t off = (uint32_t)(kk >> 2) * T5_BLOCK + (uint32_t)(kk & 3) * 32u;
-          umma_bf16(tmem + (uint32_t)s * T5_KEYS, desc_kmajor(sQ + off), desc_kmajor(sK + s * T5_TILE + off), idesc_qk, kk > 0 ? 1u : 0u);
+          for (int kk = 0; kk < T5_HD / 16; ++kk) {
+            const uint64_t off = (uint64_t)(((uint32_t)(kk >> 2) * T5_BLOCK + (uint32_t)(kk & 3) * 32u) >> 4);
+            umma_bf16(d, q_desc + off, kd + off, idesc_qk, kk > 0 ? 1u : 0u);
+          }
+          umma_commit(bar(S_FULL + s));
+          umma_commit(bar(K_EMPTY + s));
         }
-        umma_commit(bar(S_FULL + s));
-        umma_commit(bar(K_EMPTY + s));
+        __syncwarp();
         return true;
       };
       if (ok) ok = issue_qk(0);
@@ -303,23 +352,29 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         if (c + 1 < n_chunks) {
           if (!issue_qk(c + 1)) { ok = false; break; }
         }
-        if (!mbar_wait(bar(P_FULL + (c & 1)), ph, abort_flag, p.status)) { ok = false; break; }
-        if (!mbar_wait(bar(V_FULL + s), ph, abort_flag, p.status)) { ok = false; break; }
+        if (!wait_warp(bar(P_FULL + (c & 1)), ph)) { ok = false; break; }
+        if (!wait_warp(bar(V_FULL + s), ph)) { ok = false; break; }
+        // the running output has been scaled to this chunk's reference maximum (correction warps)
+        if (!wait_warp(bar(O_READY + (c & 1)), ph)) { ok = false; break; }
         tc_fence_after();
+        const uint64_t vd = desc_mnmajor(sV + (uint32_t)s * T5_TILE);
+        const uint32_t pa = tmem + 3u * T5_KEYS + (uint32_t)(c & 1) * (T5_KEYS / 2);
+        if (leader) {
 #pragma unroll
-        for (int kk = 0; kk < T5_KEYS / 16; ++kk) {
-          // P from tensor memory: buffer c & 1, 16 keys = 8 packed columns further per step
-          umma_bf16_ts(tmem + 2u * T5_KEYS, tmem + 3u * T5_KEYS + (uint32_t)(c & 1) * (T5_KEYS / 2) + (uint32_t)kk * 8u,
-                       desc_mnmajor(sV + s * T5_TILE + (uint32_t)kk * 2048u), idesc_pv, (c > 0 || kk > 0) ? 1u : 0u);
+          for (int kk = 0; kk < T5_KEYS / 16; ++kk) {
+            // P from tensor memory: buffer c & 1, 16 keys = 8 packed columns further per step; V: 16 keys = 2048 bytes further
+            umma_bf16_ts(tmem + 2u * T5_KEYS, pa + (uint32_t)kk * 8u, vd + (uint64_t)(kk * 128), idesc_pv, (c > 0 || kk > 0) ? 1u : 0u);
+          }
+          umma_commit(bar(V_EMPTY + s));
+          umma_commit(bar(P_EMPTY + (c & 1)));   // this P buffer may be overwritten and O is up to date through chunk c
         }
-        umma_commit(bar(V_EMPTY + s));
-        umma_commit(bar(P_EMPTY + (c & 1)));   // this P buffer may be overwritten and O is up to date through chunk c
+        __syncwarp();
       }
     }
-  } else {
-    // ===================== softmax and output (warps 2..9) =====================
-    // Two threads per query row (= TMEM lane): a warp may only touch the lane quarter (warp id mod 4), so warps w and
-    // w + 4 share a quarter; the first takes keys 0..63 of a chunk and output dimensions 0..63, the second the rest.
+  } else if (warp < 2 + T5_SOFT / 32) {
+    // ===================== softmax and output (warps 2..17) =====================
+    // Four threads per query row (= TMEM lane): a warp may only touch the lane quarter (warp id mod 4), so warps w,
+    // w + 4, w + 8 and w + 12 share a quarter; each takes a quarter of a chunk's keys and of the output dimensions.
     const int q4 = warp & 3;                      // TMEM lane quarter this warp may access
     const int hf = (warp - 2) >> 2;               // which part of the chunk's keys / of the head dimensions
     const int t = q4 * 32 + lane;                 // row inside the tile
@@ -434,6 +489,14 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         const float m_new = fmaxf(m_run, mx);
         const float corr = (m_new == -INFINITY) ? 1.f : fast_exp2(m_run - m_new);
         const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+        // the factor for the running output goes to the correction warps at once: they scale O (once the previous
+        // chunk's P V has completed) while this thread forms the probabilities.  All parts of a row compute the same
+        // factor; part 0 publishes it.
+        if (hf == 0) {
+          s_corr[(c & 1) * T5_ROWS + t] = corr;
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(C_FULL + (c & 1)));
+        }
         // ---- probabilities -> tensor memory (packed bf16: key pair (2j, 2j + 1) of this thread's keys in column j of its
         // part of buffer c & 1), row sum
         float sum4[4] = {0.f, 0.f, 0.f, 0.f};
@@ -447,24 +510,7 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         }
         l_run = l_run * corr + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
         m_run = m_new;
-        // ---- O *= corr (this thread's dimensions, in tensor memory), unless no row of this warp changed its maximum; O has
-        // to be complete through the previous chunk first
-        if (c > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
-          ok = wait_all(bar(P_EMPTY + ((c - 1) & 1)), (uint32_t)(((c - 1) >> 1) & 1));
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t o_addr = tmem + lane_addr + 2u * T5_KEYS + (uint32_t)hf * (T5_HD / T5_PARTS);
-#pragma unroll 1
-          for (int g = 0; g < T5_HD / T5_PARTS / 32; ++g) {
-            float ov[32];
-            tmem_ld32_nowait(o_addr + g * 32, ov);
-            tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 32; ++j) ov[j] *= corr;
-            tmem_st32(o_addr + g * 32, ov);
-          }
-        }
-        tmem_st_wait();   // P (and O) are in tensor memory
+        tmem_st_wait();   // P is in tensor memory
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(P_FULL + (c & 1)));
@@ -498,6 +544,39 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         }
       }
     }
+  } else {
+    // ===================== correction (warps 18..25) =====================
+    // Two threads per query row, half of the head dimensions each: O *= 2^(m_old - m_new) in tensor memory whenever a
+    // row's reference maximum moved, between the previous chunk's P V and this one's.  Off the softmax threads' path:
+    // they publish the factor before they exponentiate, and the MMA issuer waits for O_READY before the chunk's P V.
+    const int q4 = warp & 3;
+    const int hf = (warp - 2 - T5_SOFT / 32) >> 2;
+    const int t = q4 * 32 + lane;
+    const uint32_t o_addr = tmem + ((uint32_t)(q4 * 32) << 16) + 2u * T5_KEYS + (uint32_t)hf * (T5_HD / T5_CORR_PARTS);
+    auto wait_all = [&](uint32_t b, uint32_t parity) {
+      return __all_sync(0xffffffffu, mbar_wait(b, parity, abort_flag, p.status)) != 0;
+    };
+    for (int c = 0; c < n_chunks; ++c) {
+      if (!wait_all(bar(C_FULL + (c & 1)), (uint32_t)((c >> 1) & 1))) break;
+      const float corr = s_corr[(c & 1) * T5_ROWS + t];
+      if (c > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
+        // O has to be complete through the previous chunk first
+        if (!wait_all(bar(P_EMPTY + ((c - 1) & 1)), (uint32_t)(((c - 1) >> 1) & 1))) break;
+        tc_fence_after();
+        float ov[T5_HD / T5_CORR_PARTS];
+#pragma unroll
+        for (int g = 0; g < T5_HD / T5_CORR_PARTS / 32; ++g) tmem_ld32_nowait(o_addr + g * 32, ov + g * 32);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < T5_HD / T5_CORR_PARTS; ++j) ov[j] *= corr;
+#pragma unroll
+        for (int g = 0; g < T5_HD / T5_CORR_PARTS / 32; ++g) tmem_st32(o_addr + g * 32, ov + g * 32);
+        tmem_st_wait();
+        tc_fence_before();
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(O_READY + (c & 1)));
+    }
   }
 
   // a tile without rows still waits for its predecessor before it reports completion (the hand-off's ordering is
@@ -514,7 +593,7 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
 }
 
 size_t t5_smem_bytes(int MW) {
-  return 1024 + (size_t)(1 + 2 * T5_STAGES) * T5_TILE + 8 * 32 + 16 + T5_ROWS * 4 + 3 * T5_PARTS * T5_ROWS * 4 + (size_t)T5_ROWS * MW * 4 + 64;
+  return 1024 + (size_t)(1 + 2 * T5_STAGES) * T5_TILE + 8 * 32 + 16 + T5_ROWS * 4 + 3 * T5_PARTS * T5_ROWS * 4 + 2 * T5_ROWS * 4 + (size_t)T5_ROWS * MW * 4 + 64;
 }
 
 }  // namespace
