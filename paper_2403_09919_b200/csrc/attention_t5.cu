@@ -25,6 +25,7 @@
 // The chunk's keys past a row's extent are masked by selection, never by arithmetic, and their V rows are multiplied by
 // exact zeros: the cache must hold finite values everywhere (it is cleared once when the handle is created).
 #include <cuda.h>
+#include <stdio.h>
 
 #include "pdl.cuh"
 #include "rd_internal.cuh"
@@ -174,6 +175,17 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// Measurement build (-DRD_T5_STAMPS, never the shipped library): the CTA of head 0 / sequence 0 / first row tile of the
+// 41st launch records %globaltimer at the steps of chunks 2..9 in one softmax thread, the MMA warp and one correction
+// thread, and prints the timeline when it is done.
+#ifdef RD_T5_STAMPS
+__device__ unsigned long long g_t5_st[3][8][8];
+__device__ int g_t5_launch = 0;
+#define T5_STAMP(on, role, c, i) do { if ((on) && (c) >= 2 && (c) < 10) g_t5_st[role][(c) - 2][i] = now_ns(); } while (0)
+#else
+#define T5_STAMP(on, role, c, i) do { } while (0)
+#endif
+
 struct T5Params {
   const float* qkv;            // [M][3d] fp32, Q rotated in place by the rotary kernel
   __nv_bfloat16* out;          // [M][d]
@@ -252,9 +264,16 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
     nc_min = tree ? tree_base : nc_first;   // every valid row attends at least the keys below this
   }
   const int n_chunks = (kext + T5_KEYS - 1) / T5_KEYS;
+#ifdef RD_T5_STAMPS
+  if (threadIdx.x == 0)
+    *reinterpret_cast<volatile int*>(misc + 8) = (blockIdx.x == 0 && blockIdx.y == (unsigned)(p.row_tiles - 1)) ? atomicAdd(&g_t5_launch, 1) : -1;
+#endif
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+#ifdef RD_T5_STAMPS
+  const bool dbg_on = *reinterpret_cast<volatile int*>(misc + 8) == 40 && n_chunks >= 10;
+#endif
   const uint32_t tmem = *tmem_slot;   // columns [0,128) and [128,256): scores, [256,384): output
 
   if (warp == 0) {
@@ -329,7 +348,9 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         const int s = c & 1;
         const uint32_t ph = (c >> 1) & 1;
         if (!wait_warp(bar(K_FULL + s), ph)) return false;
+        T5_STAMP(dbg_on && leader, 1, c - 1, 0);
         if (!wait_warp(bar(S_EMPTY + s), ph ^ 1u)) return false;
+        T5_STAMP(dbg_on && leader, 1, c - 1, 1);
         tc_fence_after();
         const uint64_t kd = desc_kmajor(sK + (uint32_t)s * T5_TILE);
         const uint32_t d = tmem + (uint32_t)s * T5_KEYS;
@@ -352,10 +373,15 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         if (c + 1 < n_chunks) {
           if (!issue_qk(c + 1)) { ok = false; break; }
         }
-        if (!wait_warp(bar(P_FULL + (c & 1)), ph)) { ok = false; break; }
+        T5_STAMP(dbg_on && leader, 1, c, 2);
+        // (the probabilities come last of the three: the other two waits are out of the way when they arrive)
         if (!wait_warp(bar(V_FULL + s), ph)) { ok = false; break; }
+        T5_STAMP(dbg_on && leader, 1, c, 3);
         // the running output has been scaled to this chunk's reference maximum (correction warps)
         if (!wait_warp(bar(O_READY + (c & 1)), ph)) { ok = false; break; }
+        T5_STAMP(dbg_on && leader, 1, c, 4);
+        if (!wait_warp(bar(P_FULL + (c & 1)), ph)) { ok = false; break; }
+        T5_STAMP(dbg_on && leader, 1, c, 5);
         tc_fence_after();
         const uint64_t vd = desc_mnmajor(sV + (uint32_t)s * T5_TILE);
         const uint32_t pa = tmem + 3u * T5_KEYS + (uint32_t)(c & 1) * (T5_KEYS / 2);
@@ -369,6 +395,7 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
           umma_commit(bar(P_EMPTY + (c & 1)));   // this P buffer may be overwritten and O is up to date through chunk c
         }
         __syncwarp();
+        T5_STAMP(dbg_on && leader, 1, c, 6);
       }
     }
   } else if (warp < 2 + T5_SOFT / 32) {
@@ -432,22 +459,44 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         x_phase ^= 1u;
         return r;
       };
-      // may row t attend key `key`?  (selection, never arithmetic: masked scores may be anything)
-      auto visible = [&](int key) {
-        bool vis = key < nc_row;
-        if (tree && key >= tree_base) {
-          const int tb = key - tree_base;
-          if (tb < seq_rows) vis = (s_mask[t * MW + (tb >> 5)] >> (tb & 31)) & 1u;
+      // Which of this thread's 32 keys [k0, k0 + 32) may row t attend?  One bit per key, formed from whole words: the
+      // keys below the row's extent, with the bits of the tree part (keys tree_base .. tree_base + seq_rows) replaced
+      // by the row's mask bits.  (Evaluated per key, with a shared-memory load each, the two masked chunks of a tile
+      // took 2.3 us apiece.)  Masking is by selection, never arithmetic: masked scores may be anything.
+      auto visible_word = [&](int k0) {
+        const int n = nc_row - k0;
+        uint32_t w = n >= 32 ? 0xffffffffu : (n <= 0 ? 0u : ((1u << n) - 1u));
+        if (tree) {
+          const int tb0 = k0 - tree_base;   // mask bit of key k0; negative when the chunk starts inside the context
+          if (tb0 > -32 && tb0 < seq_rows) {
+            const int j_lo = max(0, -tb0), j_hi = min(32, seq_rows - tb0);   // bit positions that lie in the tree part
+            const uint32_t range = (j_hi >= 32 ? 0xffffffffu : ((1u << j_hi) - 1u)) & ~((1u << j_lo) - 1u);
+            uint32_t bits;
+            if (tb0 >= 0) {
+              const int wd = tb0 >> 5;
+              const uint32_t lo = s_mask[t * MW + wd], hi = (wd + 1 < MW) ? s_mask[t * MW + wd + 1] : 0u;
+              bits = __funnelshift_r(lo, hi, (uint32_t)(tb0 & 31));
+            } else {
+              bits = s_mask[t * MW] << (-tb0);
+            }
+            w = (w & ~range) | (bits & range);
+          }
         }
-        return vis;
+        return w;
       };
       constexpr int HALF = T5_KEYS / T5_PARTS;   // keys (and output dimensions) of this thread
+      static_assert(HALF == 32, "visible_word forms one 32-bit word per thread and chunk");
       for (int c = 0; c < n_chunks; ++c) {
         const int s = c & 1;
         const uint32_t ph = (c >> 1) & 1;
         const int k0 = c * T5_KEYS + hf * HALF;   // first key of this thread's half
+#ifdef RD_T5_STAMPS
+        const bool dbg_me = dbg_on && threadIdx.x == 64;
+#endif
+        T5_STAMP(dbg_me, 0, c, 0);
         ok = wait_all(bar(S_FULL + s), ph);
         if (!ok) break;
+        T5_STAMP(dbg_me, 0, c, 1);
         tc_fence_after();
         const uint32_t s_addr = tmem + lane_addr + (uint32_t)s * T5_KEYS + (uint32_t)hf * HALF;
         const bool all_visible = c * T5_KEYS + T5_KEYS <= nc_min;
@@ -457,6 +506,7 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
 #pragma unroll
         for (int g = 0; g < HALF / 32; ++g) tmem_ld32_nowait(s_addr + g * 32, sc + g * 32);
         tmem_ld_wait();
+        T5_STAMP(dbg_me, 0, c, 2);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(S_EMPTY + s));
@@ -466,9 +516,10 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
 #pragma unroll
           for (int j = 0; j < HALF; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
         } else {
+          const uint32_t vw = visible_word(k0);
 #pragma unroll
           for (int j = 0; j < HALF; ++j) {
-            sc[j] = visible(k0 + j) ? sc[j] : -INFINITY;
+            sc[j] = ((vw >> j) & 1u) ? sc[j] : -INFINITY;
             mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
           }
         }
@@ -476,8 +527,10 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale2;   // scale2 > 0
         // the row's maximum over all parts
         s_red[((c & 1) * T5_PARTS + hf) * T5_ROWS + t] = mx;
+        T5_STAMP(dbg_me, 0, c, 3);
         ok = exchange();
         if (!ok) break;
+        T5_STAMP(dbg_me, 0, c, 4);
         // this chunk's P buffer is free once the P V of the chunk before last has read it
         if (c >= 2) {
           ok = wait_all(bar(P_EMPTY + (c & 1)), ph ^ 1u);
@@ -486,6 +539,7 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         }
 #pragma unroll
         for (int q = 0; q < T5_PARTS; ++q) mx = fmaxf(mx, s_red[((c & 1) * T5_PARTS + q) * T5_ROWS + t]);
+        T5_STAMP(dbg_me, 0, c, 5);
         const float m_new = fmaxf(m_run, mx);
         const float corr = (m_new == -INFINITY) ? 1.f : fast_exp2(m_run - m_new);
         const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
@@ -510,7 +564,9 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         }
         l_run = l_run * corr + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
         m_run = m_new;
+        T5_STAMP(dbg_me, 0, c, 6);
         tmem_st_wait();   // P is in tensor memory
+        T5_STAMP(dbg_me, 0, c, 7);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(P_FULL + (c & 1)));
@@ -558,10 +614,15 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
     };
     for (int c = 0; c < n_chunks; ++c) {
       if (!wait_all(bar(C_FULL + (c & 1)), (uint32_t)((c >> 1) & 1))) break;
+#ifdef RD_T5_STAMPS
+      const bool dbg_c = dbg_on && warp == 2 + T5_SOFT / 32 && lane == 0;
+#endif
+      T5_STAMP(dbg_c, 2, c, 0);
       const float corr = s_corr[(c & 1) * T5_ROWS + t];
       if (c > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
         // O has to be complete through the previous chunk first
         if (!wait_all(bar(P_EMPTY + ((c - 1) & 1)), (uint32_t)(((c - 1) >> 1) & 1))) break;
+        T5_STAMP(dbg_c, 2, c, 1);
         tc_fence_after();
         float ov[T5_HD / T5_CORR_PARTS];
 #pragma unroll
@@ -574,6 +635,7 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
         tmem_st_wait();
         tc_fence_before();
       }
+      T5_STAMP(dbg_c, 2, c, 2);
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(O_READY + (c & 1)));
     }
@@ -586,6 +648,19 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
   tc_fence_before();
   __syncthreads();
   chain_exit(p.cs);
+#ifdef RD_T5_STAMPS
+  if (dbg_on && threadIdx.x == 0) {
+    const unsigned long long t0 = g_t5_st[0][0][0];
+    auto rel = [&](int role, int c, int i) { return (long long)(g_t5_st[role][c][i] - t0); };
+    printf("t5 stamps (ns from the softmax thread's start of chunk 2), %d chunks, %d rows\n", n_chunks, nrows);
+    for (int c = 0; c < 8; ++c)
+      printf("c%d soft: start %lld Sfull %lld ld %lld max %lld xchg %lld Pempty %lld exp %lld st %lld | mma: Kfull(c+1) %lld Sempty %lld "
+             "qk_issued %lld Vfull %lld Oready %lld Pfull %lld pv_issued %lld | corr: Cfull %lld PVdone %lld done %lld\n",
+             c + 2, rel(0, c, 0), rel(0, c, 1), rel(0, c, 2), rel(0, c, 3), rel(0, c, 4), rel(0, c, 5), rel(0, c, 6), rel(0, c, 7),
+             rel(1, c, 0), rel(1, c, 1), rel(1, c, 2), rel(1, c, 3), rel(1, c, 4), rel(1, c, 5), rel(1, c, 6), rel(2, c, 0),
+             rel(2, c, 1), rel(2, c, 2));
+  }
+#endif
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
