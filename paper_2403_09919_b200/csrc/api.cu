@@ -399,10 +399,12 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
     att_wide = wide_waves < 0 || (wide_waves > 0 && blocks > wide_waves * h->tc_grid);   // negative: always
     static const int t5_ok = getenv("RD_ATT_T5") ? atoi(getenv("RD_ATT_T5")) : 1;   // tuning toggle
     // (its 128-row tiles and 128-key chunks pay off when a sequence brings several hundred rows to the launch -- prompt
-    // processing -- or, in a verification pass of a wide beam, when the context is long enough that a CTA's set-up is
-    // spread over eight chunks or more; with tens of rows per sequence most of a tile would be padding.  RD_ATT_T5=2
-    // takes it whenever the 64-row kernel would run.)
-    const bool t5_pays = rows_per_seq_max >= 512 || (rows_per_seq_max >= 128 && h->ctx_bound + rows_per_seq_max >= 1024);
+    // processing -- or, in a verification pass, when a sequence fills at least half a tile and the context is long
+    // enough that a CTA's set-up is spread over eight chunks or more: the batched 7B step takes 17.5 ms this way
+    // against 17.9 ms through the 64-row kernel, with 46 of 128 rows used on average.  RD_ATT_T5=2 takes it whenever
+    // the 64-row kernel would run.)
+    static const int t5_rows = getenv("RD_ATT_T5_ROWS") ? atoi(getenv("RD_ATT_T5_ROWS")) : 64;   // tuning toggle
+    const bool t5_pays = rows_per_seq_max >= 512 || (rows_per_seq_max >= t5_rows && h->ctx_bound + rows_per_seq_max >= 1024);
     att_t5 = att_wide && !h->kv_maps.empty() && ((t5_ok == 1 && t5_pays) || t5_ok >= 2);
     if (att_t5) row_blocks = (rows_per_seq_max + attn_t5_rows_per_block() - 1) / attn_t5_rows_per_block();
     else if (att_wide) row_blocks = (rows_per_seq_max + attn_wide_rows_per_block() - 1) / attn_wide_rows_per_block();

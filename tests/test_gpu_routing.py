@@ -88,16 +88,28 @@ def test_wide_beam_long_context_takes_the_tcgen05_kernel():
     assert route["att_rows128_tc5"] == cfg["n_layers"] and route["att_rows64"] == 0 and route["att_rows16"] == 0
 
 
-def test_ragged_batch_long_contexts_take_the_64_row_kernel():
+def test_ragged_batch_takes_the_64_row_kernel_below_a_thousand_keys():
+    """Batch 16, beam width 16 (up to 81 rows per sequence), contexts from 256 to 900 tokens (4 to 15 chunks of keys):
+    tree-masked 64-row tiles, every sequence with its own context length and row count."""
+    cfg = dict(BASE, d_model=512, n_heads=8, d_rnn=512, max_batch=16, beam_width=16, max_ctx=900 + 81 + 16)
+    lens = [int(x) for x in np.random.default_rng(22).integers(256, 901, size=16)]
+    lens[0], lens[5], lens[15] = 900, 256, 640
+    route, n_max, n_sum = verify_on_long_contexts(cfg, lens, follow=[0, 5, 15], rho=0.3, seed=22)
+    assert n_sum > 512
+    assert route["att_rows64"] == cfg["n_layers"] and route["att_rows128_tc5"] == 0 and route["att_rows16"] == 0
+
+
+def test_ragged_batch_long_contexts_take_the_tcgen05_kernel():
     """The batched 7B workload's regime: batch 16, beam width 16 (up to 81 rows per sequence), contexts from 256 to 2048
-    tokens (4 to 32 chunks of keys): tree-masked 64-row tiles, every sequence with its own context length and row
-    count."""
-    cfg = dict(BASE, d_model=512, n_heads=8, d_rnn=512, max_batch=16, beam_width=16, max_ctx=2048 + 81 + 16)
+    tokens (2 to 17 chunks of 128 keys): from a thousand keys up, sequences that can fill half a 128-row tile go
+    through the tcgen05 kernel (head dimension 128), every sequence with its own context length and row count, most of
+    every tile unused."""
+    cfg = dict(BASE, d_model=1024, n_heads=8, d_rnn=1024, max_batch=16, beam_width=16, max_ctx=2048 + 81 + 16)
     lens = [int(x) for x in np.random.default_rng(22).integers(256, 2049, size=16)]
     lens[0], lens[5], lens[15] = 2048, 256, 1400
     route, n_max, n_sum = verify_on_long_contexts(cfg, lens, follow=[0, 5, 15], rho=0.3, seed=22)
     assert n_sum > 512
-    assert route["att_rows64"] == cfg["n_layers"] and route["att_rows128_tc5"] == 0 and route["att_rows16"] == 0
+    assert route["att_rows128_tc5"] == cfg["n_layers"] and route["att_rows64"] == 0 and route["att_rows16"] == 0
 
 
 def test_long_context_few_heads_splits_the_keys():
