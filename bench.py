@@ -587,14 +587,15 @@ def main():
                 in_step["frac_of_measured_peak"] = in_step["gbs"] / peak
         except Exception as e:  # measurement aid only
             in_step = {"error": str(e)}
-        # DRAM traffic per launch: an ncu capture of six consecutive projection launches of this workload (summary
-        # under profiles/) read and wrote 1.026 x their algorithmic bytes in total (the surplus is the activation
-        # operand and the partial sums); traffic grows with the weight bytes, so that ratio scales the mean launch.
-        NCU_TRAFFIC_RATIO = 1.026
+        # DRAM traffic per launch: an ncu capture of six consecutive projection launches of this workload (the four of a
+        # layer, the LM head and a drafter layer; summary under profiles/) read and wrote 1.040 x their algorithmic
+        # bytes in total (the surplus is the activation operand and the partial sums; 1.026 in an earlier capture of
+        # six other launches); traffic grows with the weight bytes, so that ratio scales the mean launch.
+        NCU_TRAFFIC_RATIO = 1.040
         traffic = NCU_TRAFFIC_RATIO * g_bytes / g_n if g_n else None
         line["roofline"] = {"bound": "hbm", "kernel": "projection (weight-streaming GEMM)", "achieved": achieved, "peak": peak,
                             "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
-                            "traffic_note": "bytes per launch: mean algorithmic bytes x 1.026, the DRAM read+write / algorithmic ratio of an ncu capture of six launches",
+                            "traffic_note": "bytes per launch: mean algorithmic bytes x 1.040, the DRAM read+write / algorithmic ratio of an ncu capture of six launches",
                             "algorithmic_bytes_per_launch": g_bytes / g_n if g_n else None, "peak_source": peak_src,
                             "in_step": in_step,
                             "launches_per_step": g_n / prof_steps, "ms_per_step_in_kernel": g_ms / prof_steps,
