@@ -443,18 +443,18 @@ constexpr int SEG_THREADS = 256;
 constexpr int SEG_ITEMS_MAX = 4;     // float4 per thread at most (the kernel is instantiated for 1, 2 and 4)
 constexpr int SEG_FOLD = 2;
 constexpr int SEG_MAX_CAND = 512;    // S * BW candidates per row at most
+constexpr int SEG_LIST_CAP = 1024;   // candidates at or above a segment's threshold that the counting path takes
 constexpr int MRG_THREADS = 256;
 constexpr int MRG_MAX_BW = 64;       // the merge kernel ranks BW x BW keys in shared memory
 constexpr int MRG_NARROW_BW = 16;    // up to here the narrow variant (candidates re-read from shared memory) is the faster
 
-template <int SEG_ITEMS, bool SORTED>
+template <int SEG_ITEMS>
 __global__ void __maxnreg__(88) draft_seg_kernel(GemmOut proj, int V, int BW, int seg_len4, float* __restrict__ seg_max,
                                                  float* __restrict__ seg_sum, float* __restrict__ seg_val,
                                                  int32_t* __restrict__ seg_idx, const int32_t* __restrict__ m_total,
                                                  ChainSync cs) {
   chain_begin(cs);
   __shared__ float shf[32];
-  __shared__ unsigned long long shk[2][SEG_THREADS / 32];
   const int r = blockIdx.y, sgm = blockIdx.x, S = gridDim.x;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const bool fast = proj.m_tiles_max == 1 && (proj.partial == nullptr || proj.all_work);
@@ -514,70 +514,54 @@ __global__ void __maxnreg__(88) draft_seg_kernel(GemmOut proj, int V, int BW, in
   sum = block_reduce_sum(sum, shf);
   if (threadIdx.x == 0) { seg_max[(size_t)r * S + sgm] = smax; seg_sum[(size_t)r * S + sgm] = sum; }
   // ---- the segment's BW best in (value desc, index asc) order.  Every candidate becomes one 64-bit key whose
-  // unsigned order is that order (ordered value bits, then the complemented index): keys are unique, so round
-  // p's winner is simply the largest key below round p-1's, and nothing is marked or removed.  One redux pair
-  // per warp, one barrier per round (the per-warp results alternate between two shared buffers).
+  // unsigned order is that order (ordered value bits, then the complemented index): keys are unique.
   unsigned long long key[SEG_ITEMS * 4];
 #pragma unroll
   for (int k = 0; k < SEG_ITEMS; ++k)
 #pragma unroll
     for (int e = 0; e < 4; ++e) key[k * 4 + e] = ok[k] ? cand_key(v[k][e], col[k] + e) : 0ull;
   constexpr int NK = SEG_ITEMS * 4;
-  if constexpr (SORTED) {
-    // Wide beams: every thread first sorts its own keys (best first, a bitonic network in registers); a round then
-    // looks at one key per thread, the head of its list, and the thread that held the winner moves its list up.
-    // BW rounds of NK compares each become one sort and BW rounds of one.
+  // A threshold that at least BW candidates reach -- the BW-th largest of the threads' own maxima, ranked by counting --,
+  // then the candidates at or above it go to a shared list that is ranked by counting as well.  Every key is touched
+  // a constant number of times, whatever BW is (BW rounds of a block-wide maximum took 54 us per call at beam
+  // width 64).  Exactly BW threads hold a maximum at or above the threshold, each with at most NK keys: the list
+  // holds BW * NK keys at most.
+  static_assert(MRG_MAX_BW * SEG_ITEMS_MAX * 4 <= SEG_LIST_CAP, "the list takes every key of BW threads");
+  __shared__ unsigned long long s_tmax[SEG_THREADS];
+  __shared__ unsigned long long s_list[SEG_LIST_CAP];
+  __shared__ unsigned long long s_tau;
+  __shared__ int s_n;
+  unsigned long long tk = 0ull;
 #pragma unroll
-    for (int k = 2; k <= NK; k <<= 1)
-#pragma unroll
-      for (int j = k >> 1; j > 0; j >>= 1)
-#pragma unroll
-        for (int i = 0; i < NK; ++i) {
-          const int l = i ^ j;
-          if (l > i) {
-            const bool desc = (i & k) == 0;
-            const unsigned long long a = key[i], b = key[l];
-            const bool sw = desc ? a < b : a > b;
-            key[i] = sw ? b : a;
-            key[l] = sw ? a : b;
-          }
-        }
-    for (int p = 0; p < BW; ++p) {
-      const unsigned long long mine = warp_max_key(key[0]);
-      if (lane == 0) shk[p & 1][warp] = mine;
-      __syncthreads();
-      unsigned long long best = 0ull;
-#pragma unroll
-      for (int w = 0; w < SEG_THREADS / 32; ++w) best = max(best, shk[p & 1][w]);
-      if (threadIdx.x == 0) {
-        seg_val[((size_t)r * S + sgm) * BW + p] = key_value(best);
-        seg_idx[((size_t)r * S + sgm) * BW + p] = key_index(best);
-      }
-      if (key[0] == best && best != 0ull) {   // keys are unique: one thread of the CTA
-#pragma unroll
-        for (int i = 0; i + 1 < NK; ++i) key[i] = key[i + 1];
-        key[NK - 1] = 0ull;
-      }
-    }
-  } else {
-    unsigned long long prev = ~0ull;
-    for (int p = 0; p < BW; ++p) {
-      unsigned long long mine = 0ull;
-#pragma unroll
-      for (int q = 0; q < NK; ++q) mine = max(mine, key[q] < prev ? key[q] : 0ull);
-      mine = warp_max_key(mine);
-      if (lane == 0) shk[p & 1][warp] = mine;
-      __syncthreads();
-      unsigned long long best = 0ull;
-#pragma unroll
-      for (int w = 0; w < SEG_THREADS / 32; ++w) best = max(best, shk[p & 1][w]);
-      if (threadIdx.x == 0) {
-        seg_val[((size_t)r * S + sgm) * BW + p] = key_value(best);
-        seg_idx[((size_t)r * S + sgm) * BW + p] = key_index(best);
-      }
-      prev = best;
-    }
+  for (int q = 0; q < NK; ++q) tk = max(tk, key[q]);
+  s_tmax[threadIdx.x] = tk;
+  if (threadIdx.x == 0) { s_n = 0; s_tau = 0ull; }
+  __syncthreads();
+  if (tk != 0ull) {
+    int rank = 0;
+#pragma unroll 8
+    for (int j = 0; j < SEG_THREADS; ++j) rank += s_tmax[j] > tk ? 1 : 0;
+    if (rank == BW - 1) s_tau = tk;   // keys are unique: one thread at most
   }
+  __syncthreads();
+  const unsigned long long tau = s_tau;   // 0: fewer than BW threads hold a candidate, every candidate qualifies
+#pragma unroll
+  for (int q = 0; q < NK; ++q)
+    if (key[q] != 0ull && key[q] >= tau) {
+      const int pos = atomicAdd(&s_n, 1);
+      if (pos < SEG_LIST_CAP) s_list[pos] = key[q];
+    }
+  __syncthreads();
+  const int n = min(s_n, SEG_LIST_CAP);
+  float* out_v = seg_val + ((size_t)r * S + sgm) * BW;
+  int32_t* out_i = seg_idx + ((size_t)r * S + sgm) * BW;
+  for (int i = threadIdx.x; i < n; i += SEG_THREADS) {
+    const unsigned long long k = s_list[i];
+    int rank = 0;
+    for (int j = 0; j < n; ++j) rank += s_list[j] > k ? 1 : 0;
+    if (rank < BW) { out_v[rank] = key_value(k); out_i[rank] = key_index(k); }
+  }
+  for (int p = n + threadIdx.x; p < BW; p += SEG_THREADS) { out_v[p] = key_value(0ull); out_i[p] = key_index(0ull); }
   chain_exit(cs);
 }
 
@@ -663,34 +647,54 @@ __global__ void __launch_bounds__(MRG_THREADS) draft_merge_kernel(
   // the rows' BW best continuations each (draft_rowtop_kernel), in row order
   for (int c = threadIdx.x; c < rows * BW; c += MRG_THREADS) top[c] = __ldcg(top_g + (size_t)row0 * BW + c);
   if constexpr (WIDE) {
-    __shared__ unsigned long long shk[2][MRG_THREADS / 32];
+    __shared__ unsigned long long s_tmax[MRG_THREADS];
+    __shared__ unsigned long long s_list[SEG_LIST_CAP];
+    __shared__ unsigned long long s_tau;
+    __shared__ int s_n;
     __syncthreads();
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_dbg[2]));
-    // the beam of rank kout among the rows * BW candidates, (score desc, flat index asc): all threads hold their share
-    // of the candidates in registers; one warp reduction and one barrier per round (two result buffers in turn)
+    // The beam of rank kout among the rows * BW candidates, (score desc, flat index asc), in a constant number of
+    // steps: every thread holds its share of the candidates in registers; the (kout + 1)-th largest of the threads'
+    // own maxima (ranked by counting) is a threshold that at least kout + 1 candidates reach; the candidates at or
+    // above it -- those of exactly kout + 1 threads, KPT each at most -- go to a list that is ranked by counting.
+    // (kout + 1 rounds of a block-wide maximum took 28 us per call at beam width 64.)
     {
       const int n_cand = rows * BW;
       constexpr int KPT = MRG_MAX_BW * MRG_MAX_BW / MRG_THREADS;
+      static_assert(MRG_MAX_BW * KPT <= SEG_LIST_CAP, "the list takes every key of kout + 1 threads");
       unsigned long long key[KPT];
+      unsigned long long tk = 0ull;
   #pragma unroll
       for (int j = 0; j < KPT; ++j) {
         const int c = threadIdx.x + MRG_THREADS * j;
         key[j] = c < n_cand ? top[c] : 0ull;
+        tk = max(tk, key[j]);
       }
-      unsigned long long pv = ~0ull;
-      for (int p = 0; p <= kout; ++p) {
-        unsigned long long mine = 0ull;
-  #pragma unroll
-        for (int j = 0; j < KPT; ++j) mine = max(mine, key[j] < pv ? key[j] : 0ull);
-        mine = warp_max_key(mine);
-        if (lane == 0) shk[p & 1][warp] = mine;
-        __syncthreads();
-        unsigned long long best = 0ull;
-  #pragma unroll
-        for (int w = 0; w < MRG_THREADS / 32; ++w) best = max(best, shk[p & 1][w]);
-        pv = best;
+      s_tmax[threadIdx.x] = tk;
+      if (threadIdx.x == 0) { s_n = 0; s_tau = 0ull; s_win = Cand{-INFINITY, 0}; }
+      __syncthreads();
+      if (tk != 0ull) {
+        int rank = 0;
+  #pragma unroll 8
+        for (int j = 0; j < MRG_THREADS; ++j) rank += s_tmax[j] > tk ? 1 : 0;
+        if (rank == kout) s_tau = tk;   // keys are unique: one thread at most
       }
-      if (threadIdx.x == 0) s_win = Cand{key_value(pv), pv == 0ull ? 0 : key_index(pv)};   // (fewer candidates than beams cannot happen: BW <= V)
+      __syncthreads();
+      const unsigned long long tau = s_tau;   // 0: at most kout threads hold a candidate, every candidate qualifies
+  #pragma unroll
+      for (int j = 0; j < KPT; ++j)
+        if (key[j] != 0ull && key[j] >= tau) {
+          const int pos = atomicAdd(&s_n, 1);
+          if (pos < SEG_LIST_CAP) s_list[pos] = key[j];
+        }
+      __syncthreads();
+      const int n = min(s_n, SEG_LIST_CAP);
+      for (int i = threadIdx.x; i < n; i += MRG_THREADS) {
+        const unsigned long long k = s_list[i];
+        int rank = 0;
+        for (int j = 0; j < n; ++j) rank += s_list[j] > k ? 1 : 0;
+        if (rank == kout) s_win = Cand{key_value(k), key_index(k)};   // (fewer candidates than beams cannot happen: BW <= V)
+      }
     }
   } else {
     // narrow beams: the final ranking has a few candidates per lane of one warp
@@ -788,13 +792,12 @@ cudaError_t launch_draft_select(int dtype, const GemmOut& proj, int call, float*
     dim3 g1(S, rows);
     const ChainSync c1 = chain ? chain->link(g1.x * g1.y, true) : ChainSync{nullptr, 0u, nullptr, nullptr, nullptr};
     const int items = (seg_len4 + SEG_THREADS - 1) / SEG_THREADS;
-    const bool sorted = dm.BW > MRG_NARROW_BW;   // wide beams: the threads sort their keys once
-#define RD_SEG_LAUNCH(ITEMS, SRT)                                                                                        \
-  launch_pdl(draft_seg_kernel<ITEMS, SRT>, g1, SEG_THREADS, 0, st, proj, dm.V, dm.BW, seg_len4, sc.seg_max, sc.seg_sum, \
+#define RD_SEG_LAUNCH(ITEMS)                                                                                             \
+  launch_pdl(draft_seg_kernel<ITEMS>, g1, SEG_THREADS, 0, st, proj, dm.V, dm.BW, seg_len4, sc.seg_max, sc.seg_sum,         \
              sc.seg_val, sc.seg_idx, m_total, c1)
-    if (items <= 1) { if (sorted) RD_SEG_LAUNCH(1, true); else RD_SEG_LAUNCH(1, false); }
-    else if (items == 2) { if (sorted) RD_SEG_LAUNCH(2, true); else RD_SEG_LAUNCH(2, false); }
-    else { if (sorted) RD_SEG_LAUNCH(4, true); else RD_SEG_LAUNCH(4, false); }
+    if (items <= 1) RD_SEG_LAUNCH(1);
+    else if (items == 2) RD_SEG_LAUNCH(2);
+    else RD_SEG_LAUNCH(4);
 #undef RD_SEG_LAUNCH
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
