@@ -34,7 +34,7 @@ struct Workspace {
   int32_t *ctx, *root, *status;
   float* h;
   // row tables of the current forward
-  int32_t *row_tok, *row_seq, *row_pos, *row_slot, *row_ncache, *row_local, *row_out_index, *m_total, *last_row, *seq_off;
+  int32_t *row_tok, *row_seq, *row_pos, *row_slot, *row_ncache, *row_local, *row_out_index, *m_total, *last_row, *seq_off, *seq_order;
   // activations of the forward (compact rows)
   float *x, *qkv, *proj_d, *gu, *hidden_f, *logits, *rope_tab;
   void *a_t, *attn_t, *act_t, *hidden_t, *h_t;
@@ -93,6 +93,7 @@ struct rd_handle {
   std::vector<double> trace_bytes;  // weight bytes of each traced launch (0: not a projection)
   std::vector<double> trace_prefetch;  // ... of which requested before the launch's dependency wait
   int tc_grid, tc_smem;
+  const int32_t* att_seq_order = nullptr;   // sequences longest first for the pass being enqueued, or nullptr
   int tc_pairs;   // CTA pairs of the pair projection kernel that fit the device at once (0: not used)
   int tc_pairs_avail, tc_pairs_min_rows;   // the pairs the device offers; row bound from which launches use them
   bool tc_pairs_prefill;
@@ -191,6 +192,7 @@ void carve(Bump& bp, const Dims& dm, int m_cap, Workspace* w) {
   w->row_out_index = bp.take<int32_t>(m_cap); w->m_total = bp.take<int32_t>(4); w->last_row = bp.take<int32_t>(B);
   w->one_b = bp.take<int32_t>(4); w->one_r = bp.take<int32_t>(4);
   w->seq_off = bp.take<int32_t>(B + 1);
+  w->seq_order = bp.take<int32_t>(B);
   w->att_counters = bp.take<int32_t>(ATT_MAX_SPLIT_BLOCKS);
   w->sel_counters = bp.take<int32_t>(B);
   w->chain_ctr = bp.take<unsigned int>(CHAIN_SLOTS);
@@ -438,7 +440,7 @@ int forward_layers(rd_handle* h, const uint32_t* mask, int m_max, int n_seq, int
                : att_shallow ? RD_ROUTE_ATT_ROWS16_SHALLOW : RD_ROUTE_ATT_ROWS16]++;
       if (h->use_tc && !att_t5 && !att_wide && n_splits > 1) h->route[RD_ROUTE_ATT_KEY_SPLIT]++;
       if (h->use_tc && att_t5)
-        CK(h, launch_attention_t5(h->kv_maps[(size_t)l * 2].bytes, h->kv_maps[(size_t)l * 2 + 1].bytes, w.qkv, w.attn_t, rt, w.seq_off, dm, n_seq,
+        CK(h, launch_attention_t5(h->kv_maps[(size_t)l * 2].bytes, h->kv_maps[(size_t)l * 2 + 1].bytes, w.qkv, w.attn_t, rt, w.seq_off, h->att_seq_order, dm, n_seq,
                                   row_blocks, w.status, ch, st));
       else if (h->use_tc && att_wide)
         CK(h, launch_attention_wide(w.qkv, kv_plane_ptr(h, l, 0), kv_plane_ptr(h, l, 1), w.attn_t, rt, w.seq_off, dm, n_seq,
@@ -527,8 +529,10 @@ int do_verify(rd_handle* h, const rd_packed& pk, cudaStream_t st, int32_t* argma
   const Dims& dm = h->dm;
   const int B = h->batch, m_max = B * dm.NMAX;
   CKP(h, PROF_MISC, launch_build_rows_tree(pk, w.ctx, w.row_tok, w.row_seq, w.row_pos, w.row_slot, w.row_ncache, w.row_local,
-                               w.row_out_index, w.seq_off, w.m_total, dm, B, w.status, st));
+                               w.row_out_index, w.seq_off, w.seq_order, w.m_total, dm, B, w.status, st));
+  h->att_seq_order = B <= 1024 ? w.seq_order : nullptr;   // the row tables of this pass carry the sequences' order
   int rc = forward_layers(h, pk.mask, m_max, B, dm.NMAX, h->w.lm_head, st);
+  h->att_seq_order = nullptr;
   if (rc) return rc;
   GemmOut g;
   rc = gemm(h, w.hidden_t, dm.d, h->w.lm_head, dm.V, dm.d, w.m_total, m_max, w.logits, dm.V, &g, nullptr, st, /*pair=*/1);

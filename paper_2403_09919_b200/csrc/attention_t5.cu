@@ -191,6 +191,7 @@ struct T5Params {
   __nv_bfloat16* out;          // [M][d]
   RowTables rt;
   const int32_t* seq_off;
+  const int32_t* seq_order;    // the launch's sequences, longest key extent first, or nullptr (index order)
   Dims dm;
   int row_tiles;               // 128-row tiles per sequence (bound)
   int32_t* status;
@@ -250,7 +251,9 @@ __global__ void __launch_bounds__(T5_THREADS, 1)
   const int h = blockIdx.x;
   // the tiles of a sequence are handed out last first: without a tree mask a later tile has more keys to walk, and
   // the longest CTAs should not be the last to start
-  const int b = blockIdx.y / p.row_tiles, rb = p.row_tiles - 1 - (blockIdx.y - b * p.row_tiles);
+  // ... and the sequences longest first (the row tables' order, when the launch has one)
+  const int bi = blockIdx.y / p.row_tiles, rb = p.row_tiles - 1 - (blockIdx.y - bi * p.row_tiles);
+  const int b = p.seq_order ? p.seq_order[bi] : bi;
   const int seq_row0 = p.seq_off[b], seq_rows = p.seq_off[b + 1] - seq_row0;
   const int row0 = seq_row0 + rb * T5_ROWS;
   const int nrows = min(T5_ROWS, seq_rows - rb * T5_ROWS);   // <= 0: nothing to do for this tile (same for all roles)
@@ -684,12 +687,13 @@ cudaError_t attn_t5_prepare(int hd, int MW) {
 // map_k / map_v: tensor maps of the layer's K and V planes ([sequences * heads * max_ctx rows][128 dims], box 64 x 128).
 // grid (H, sequences * row_tiles): row_tiles tiles of 128 rows cover the longest sequence of the launch.
 cudaError_t launch_attention_t5(const void* map_k, const void* map_v, const float* qkv, void* out, const RowTables& rt,
-                                const int32_t* seq_off, const Dims& dm, int n_seq, int row_tiles, int32_t* status, Chain* chain,
+                                const int32_t* seq_off, const int32_t* seq_order, const Dims& dm, int n_seq, int row_tiles,
+                                int32_t* status, Chain* chain,
                                 cudaStream_t st) {
   if (dm.hd != T5_HD) return cudaErrorInvalidValue;
   dim3 grid(dm.H, n_seq * row_tiles);
   T5Params p;
-  p.qkv = qkv; p.out = (__nv_bfloat16*)out; p.rt = rt; p.seq_off = seq_off; p.dm = dm; p.row_tiles = row_tiles; p.status = status;
+  p.qkv = qkv; p.out = (__nv_bfloat16*)out; p.rt = rt; p.seq_off = seq_off; p.seq_order = seq_order; p.dm = dm; p.row_tiles = row_tiles; p.status = status;
   p.cs = chain ? chain->link(grid.x * grid.y) : ChainSync{nullptr, 0u, nullptr, status, nullptr};
   launch_pdl(attention_t5_kernel, grid, T5_THREADS, t5_smem_bytes(dm.MW), st, *(const CUtensorMap*)map_k, *(const CUtensorMap*)map_v, p);
   return cudaGetLastError();

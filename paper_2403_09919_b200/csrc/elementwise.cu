@@ -928,8 +928,8 @@ cudaError_t launch_fill_i32(int32_t* p, int32_t v, int n, cudaStream_t st) {
 // provisional cache slot ctx_b + n, attends cache [0, ctx_b) plus its mask row.
 __global__ void build_rows_tree_kernel(rd_packed pk, const int32_t* __restrict__ ctx, int32_t* row_tok, int32_t* row_seq,
                                        int32_t* row_pos, int32_t* row_slot, int32_t* row_ncache, int32_t* row_local,
-                                       int32_t* row_out_index, int32_t* seq_off, int32_t* m_total, Dims dm, int B,
-                                       int* status) {
+                                       int32_t* row_out_index, int32_t* seq_off, int32_t* seq_order, int32_t* m_total, Dims dm,
+                                       int B, int* status) {
   pdl_enter();
   extern __shared__ int32_t off[];  // [B+1]
   if (threadIdx.x == 0) {
@@ -945,6 +945,18 @@ __global__ void build_rows_tree_kernel(rd_packed pk, const int32_t* __restrict__
   }
   __syncthreads();
   for (int b = threadIdx.x; b <= B; b += blockDim.x) seq_off[b] = off[b];
+  // The sequences by key extent, longest first (ties by index): attention kernels whose CTAs walk a whole sequence's keys
+  // hand the long sequences out first, so that the last CTAs to start are short ones.  Ranked by counting.
+  if (seq_order)
+    for (int b = threadIdx.x; b < B; b += blockDim.x) {
+      const int kb = ctx[b] + (off[b + 1] - off[b]);
+      int rank = 0;
+      for (int o = 0; o < B; ++o) {
+        const int ko = ctx[o] + (off[o + 1] - off[o]);
+        rank += (ko > kb || (ko == kb && o < b)) ? 1 : 0;
+      }
+      seq_order[rank] = b;
+    }
   for (int idx = threadIdx.x; idx < B * dm.NMAX; idx += blockDim.x) {
     const int b = idx / dm.NMAX, n = idx - b * dm.NMAX;
     if (n >= off[b + 1] - off[b]) continue;
@@ -963,11 +975,11 @@ __global__ void build_rows_tree_kernel(rd_packed pk, const int32_t* __restrict__
 
 cudaError_t launch_build_rows_tree(const rd_packed& pk, const int32_t* ctx, int32_t* row_tok, int32_t* row_seq,
                                    int32_t* row_pos, int32_t* row_slot, int32_t* row_ncache, int32_t* row_local,
-                                   int32_t* row_out_index, int32_t* seq_off, int32_t* m_total, const Dims& dm, int B,
-                                   int* status, cudaStream_t st) {
+                                   int32_t* row_out_index, int32_t* seq_off, int32_t* seq_order, int32_t* m_total,
+                                   const Dims& dm, int B, int* status, cudaStream_t st) {
   launch_pdl(build_rows_tree_kernel, 1, 1024, (B + 1) * sizeof(int32_t), st, pk, ctx, row_tok, row_seq, row_pos, row_slot,
                                                                     row_ncache, row_local, row_out_index, seq_off,
-                                                                    m_total, dm, B, status);
+                                                                    B <= 1024 ? seq_order : nullptr, m_total, dm, B, status);
   return cudaGetLastError();
 }
 

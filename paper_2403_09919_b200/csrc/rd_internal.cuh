@@ -84,7 +84,7 @@ int attn_t5_rows_per_block();
 bool attn_t5_supported(int hd);
 cudaError_t attn_t5_prepare(int hd, int MW);
 cudaError_t launch_attention_t5(const void* map_k, const void* map_v, const float* qkv, void* out, const RowTables& rt,
-                                const int32_t* seq_off, const Dims& dm, int n_seq, int row_tiles, int32_t* status, Chain* chain,
+                                const int32_t* seq_off, const int32_t* seq_order, const Dims& dm, int n_seq, int row_tiles, int32_t* status, Chain* chain,
                                 cudaStream_t st);
 int attn_wide_rows_per_block();
 cudaError_t attn_wide_prepare(int hd, int MW);
@@ -133,7 +133,7 @@ cudaError_t launch_pack(const int32_t* beams, const int32_t* root, const int32_t
                         const Dims& dm, int B, int no_tree, cudaStream_t st);
 cudaError_t launch_build_rows_tree(const rd_packed& pk, const int32_t* ctx, int32_t* row_tok, int32_t* row_seq,
                                    int32_t* row_pos, int32_t* row_slot, int32_t* row_ncache, int32_t* row_local,
-                                   int32_t* row_out_index, int32_t* seq_off, int32_t* m_total, const Dims& dm, int B,
+                                   int32_t* row_out_index, int32_t* seq_off, int32_t* seq_order, int32_t* m_total, const Dims& dm, int B,
                                    int* status, cudaStream_t st);
 cudaError_t launch_build_rows_ar(const int32_t* root, const int32_t* ctx, int32_t* row_tok, int32_t* row_seq,
                                  int32_t* row_pos, int32_t* row_slot, int32_t* row_ncache, int32_t* row_local,
